@@ -1,0 +1,165 @@
+/*
+ * fa.h -- C ABI of the B200 (sm_100a) hybrid-KV decode path of FourierAttention.
+ *
+ * The cache of one attention layer keeps, per KV head,
+ *   - the first l_init and the most recent l_local tokens in all head dims
+ *     (Sec. 3.3, Eq.1),
+ *   - for the tokens in between ("middle"), the context-sensitive dims
+ *     D^ku / D^vu per token (K^mu, V^mu, Eq.2) and
+ *   - the remaining dims D^kc / D^vc only as n_coef = 2k real coefficients of
+ *     the translated Fourier basis along the token axis (K^mc, V^mc, Eq.3-4).
+ *
+ * fa_compress builds that cache from a prefilled K, V (Eq.1-3), fa_append
+ * pushes one token and folds the token that leaves the local window into the
+ * coefficients (Eq.5), fa_decode_attention computes softmax attention of one
+ * query per head over the cache, rebuilding the compressed dims on the fly
+ * without ever writing a dense K or V (Eq.6).
+ *
+ * Conventions for every call
+ *   - All buffers are caller-owned DEVICE memory on the current device unless
+ *     a parameter says "host".  The library allocates nothing, keeps no
+ *     mutable global state and runs every kernel on the stream passed in
+ *     (a cudaStream_t handed over as void*; NULL is the default stream).
+ *   - Calls are asynchronous.  Argument errors are found on the host before
+ *     anything is launched and returned as fa_status.  Conditions only the
+ *     device can see (middle segment full) are written to cache->status and
+ *     read back with fa_poll_status; a call that hits one changes nothing.
+ *   - Device pointers must be 16-byte aligned.  Index arrays are int32,
+ *     strictly ascending per head.
+ *   - No call throws, aborts or traps.
+ */
+#ifndef FA_H_
+#define FA_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    FA_OK = 0,
+    FA_ERR_INVALID_ARG = 1,   /* NULL pointer, bad size, inconsistent layout       */
+    FA_ERR_UNSUPPORTED = 2,   /* valid but outside what the kernels implement      */
+    FA_ERR_CAPACITY = 3,      /* the middle segment would exceed max_mid / period  */
+    FA_ERR_WORKSPACE = 4,     /* workspace pointer NULL / misaligned / too small   */
+    FA_ERR_CUDA = 5,          /* a CUDA runtime call failed                        */
+    FA_ERR_TIMEOUT = 6,       /* a bounded device-side wait gave up                */
+    FA_ERR_INDEX = 7          /* index sets are not a sorted disjoint cover        */
+} fa_status;
+
+typedef enum { FA_F32 = 0, FA_BF16 = 1 } fa_dtype;
+
+/* Reconstruction weights of Eq.6.  ORTHO: 1/T for the constant row, 2/T for
+ * the others, which inverts Eq.3 exactly on the span of the basis over a full
+ * period.  PAPER: the literal 1/k of Eq.6. */
+typedef enum { FA_NORM_ORTHO = 0, FA_NORM_PAPER = 1 } fa_norm;
+
+/* How fa_decode_attention evaluates the compressed dims.  DIRECT sums the
+ * n_coef basis terms per token; FFT evaluates each residue class of tokens
+ * (token index mod mid_classes) with one length period/mid_classes transform.
+ * AUTO picks FFT when the layout allows it. */
+typedef enum { FA_DECODE_AUTO = 0, FA_DECODE_DIRECT = 1, FA_DECODE_FFT = 2 } fa_decode_algo;
+
+/* Immutable description of one layer's cache. */
+typedef struct fa_layout {
+    int32_t batch;          /* B                                                        */
+    int32_t n_q_heads;      /* H_q; query head g reads KV head g / (H_q / H_kv)         */
+    int32_t n_kv_heads;     /* H_kv, divides H_q                                        */
+    int32_t head_dim;       /* d, multiple of 8, <= 256                                 */
+    int32_t n_full_k;       /* |D^ku|, 0..d, multiple of 8                              */
+    int32_t n_full_v;       /* |D^vu|, 0..d, multiple of 8                              */
+    int32_t n_coef;         /* M = 2k real coefficients (Eq.4), even, 2 <= M <= period  */
+    int32_t period;         /* T of Eq.4; middle token j uses basis column j, j < T     */
+    int32_t l_init;         /* Eq.1                                                     */
+    int32_t l_local;        /* Eq.1                                                     */
+    int32_t max_mid;        /* capacity of the middle segment in tokens, <= period      */
+    int32_t mid_classes;    /* P >= 1: K^mu / V^mu are stored [P][ceil(max_mid/P)][n_full],
+                               middle token j in class j % P at slot j / P; 1 = token-major */
+    int32_t kv_dtype;       /* fa_dtype of K, V, q, out and of the cached K/V rows      */
+    int32_t norm;           /* fa_norm                                                  */
+    int32_t decode_algo;    /* fa_decode_algo                                           */
+    float   softmax_scale;  /* logits = softmax_scale * q . k                           */
+} fa_layout;
+
+/* Device buffers of one layer's cache (sizes from fa_cache_sizes). */
+typedef struct fa_cache {
+    const int32_t* idx_full_k;  /* [H_kv][n_full_k]        D^ku                         */
+    const int32_t* idx_comp_k;  /* [H_kv][d - n_full_k]    D^kc                         */
+    const int32_t* idx_full_v;  /* [H_kv][n_full_v]        D^vu                         */
+    const int32_t* idx_comp_v;  /* [H_kv][d - n_full_v]    D^vc                         */
+    void*  k_init;              /* [B][H_kv][l_init][d]                                 */
+    void*  v_init;
+    void*  k_local;             /* [B][H_kv][l_local][d], a ring: oldest row at state.local_head */
+    void*  v_local;
+    void*  k_mid;               /* [B][H_kv][P][ceil(max_mid/P)][n_full_k]   K^mu       */
+    void*  v_mid;               /* [B][H_kv][P][ceil(max_mid/P)][n_full_v]   V^mu       */
+    float* coef_k;              /* [B][H_kv][M][d - n_full_k]  K^mc, raw sums of Eq.3   */
+    float* coef_v;              /* [B][H_kv][M][d - n_full_v]  V^mc                     */
+    int32_t* state;             /* [B][8]: n_init, n_local, n_mid, local_head, ticket, 3 spare */
+    int32_t* status;            /* [4]: sticky fa_status word, then scratch counters    */
+} fa_cache;
+
+/* Bytes of every buffer of fa_cache, in the order of its fields. */
+typedef struct fa_cache_sizes {
+    size_t idx_full_k, idx_comp_k, idx_full_v, idx_comp_v;
+    size_t k_init, v_init, k_local, v_local, k_mid, v_mid;
+    size_t coef_k, coef_v, state, status;
+} fa_cache_sizes;
+
+/* Host only.  Checks the layout and fills *out.  INVALID_ARG / UNSUPPORTED on a bad layout. */
+fa_status fa_cache_sizes_of(const fa_layout* layout, fa_cache_sizes* out);
+
+/* Host only.  Bytes of workspace fa_decode_attention and fa_compress need for this layout
+ * (the larger of the two).  The workspace is scratch: its contents need not survive
+ * between calls and need no initialisation. */
+fa_status fa_workspace_bytes(const fa_layout* layout, size_t* out);
+
+/* Clears state and status (an empty cache: no tokens, zero coefficients). */
+fa_status fa_cache_reset(const fa_layout* layout, fa_cache* cache, void* stream);
+
+/* Checks on the device that, per KV head, idx_full_* and idx_comp_* are strictly ascending,
+ * in range and together cover 0..d-1 exactly once (Eq.2's D^u, D^c).  Synchronises the
+ * stream.  Returns FA_ERR_INDEX if they do not. */
+fa_status fa_validate(const fa_layout* layout, const fa_cache* cache, void* stream);
+
+/* Eq.1-3.  K, V: prefilled keys / values of L tokens, element (b, t, h, e) at
+ * b*stride_b + t*stride_t + h*stride_h + e (strides in elements, multiples of 8), dtype
+ * layout->kv_dtype.  Overwrites the whole cache: windows, K^mu / V^mu, coefficients
+ * (basis column j = t - n_init for middle token t) and state.  n_init = min(L, l_init),
+ * n_local = min(L - n_init, l_local), the rest is the middle.  FA_ERR_CAPACITY (host side)
+ * if the middle exceeds max_mid.  ws / ws_bytes: workspace as sized by fa_workspace_bytes. */
+fa_status fa_compress(const fa_layout* layout, fa_cache* cache, const void* K, const void* V,
+                      int64_t stride_b, int64_t stride_t, int64_t stride_h, int32_t L,
+                      void* ws, size_t ws_bytes, void* stream);
+
+/* Eq.5.  k_new, v_new: [B][H_kv][d].  The token goes to the init window while that has
+ * room, else to the local window; when the local window is full its oldest token leaves:
+ * its D^u dims are appended to K^mu / V^mu and its D^c dims are added to the coefficients
+ * with basis column j = n_mid.  If the middle is full nothing changes and FA_ERR_CAPACITY
+ * is written to cache->status. */
+fa_status fa_append(const fa_layout* layout, fa_cache* cache, const void* k_new, const void* v_new,
+                    void* stream);
+
+/* Eq.6.  q, out: [B][H_q][d].  Softmax attention (no mask) of every query head over
+ * cat(init, middle, local) of its KV head, where the D^c dims of a middle token j are
+ * sum_m w_m F[m][j] C[m][.]; evaluated as Phi (W C^K q) for the scores and
+ * (p^T Phi) W C^V for the outputs.  Does not modify the cache.  An empty cache gives zeros. */
+fa_status fa_decode_attention(const fa_layout* layout, const fa_cache* cache, const void* q, void* out,
+                              void* ws, size_t ws_bytes, void* stream);
+
+/* Synchronises the stream and returns (then clears) the sticky device status word. */
+fa_status fa_poll_status(const fa_cache* cache, void* stream);
+
+/* Number of kernels one call launches for this layout (what = 0 compress, 1 append,
+ * 2 decode); for launch accounting by callers. */
+int fa_launch_count(const fa_layout* layout, int what);
+
+const char* fa_status_string(fa_status s);
+int fa_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* FA_H_ */

@@ -1,0 +1,263 @@
+// Host side of the C ABI declared in include/fa.h: argument checks, buffer
+// sizes, launch plans.  Every entry point validates on the host, then launches
+// on the caller's stream; nothing here allocates device memory.
+#include <cstring>
+
+#include "fa_common.cuh"
+
+namespace fa {
+
+static inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+static inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+static inline size_t elt_bytes(int dtype) { return dtype == FA_BF16 ? 2 : 4; }
+
+fa_status check_layout(const fa_layout* l) {
+    if (!l) return FA_ERR_INVALID_ARG;
+    if (l->batch < 1 || l->n_q_heads < 1 || l->n_kv_heads < 1 || l->head_dim < 8) return FA_ERR_INVALID_ARG;
+    if (l->n_q_heads % l->n_kv_heads != 0) return FA_ERR_INVALID_ARG;
+    if (l->n_full_k < 0 || l->n_full_k > l->head_dim || l->n_full_v < 0 || l->n_full_v > l->head_dim)
+        return FA_ERR_INVALID_ARG;
+    if (l->n_coef < 2 || (l->n_coef & 1) || l->period < 2 || l->n_coef > l->period) return FA_ERR_INVALID_ARG;
+    if (l->l_init < 0 || l->l_local < 0 || l->max_mid < 0 || l->max_mid > l->period) return FA_ERR_INVALID_ARG;
+    if (l->mid_classes < 1) return FA_ERR_INVALID_ARG;
+    if (l->kv_dtype != FA_F32 && l->kv_dtype != FA_BF16) return FA_ERR_INVALID_ARG;
+    if (l->norm != FA_NORM_ORTHO && l->norm != FA_NORM_PAPER) return FA_ERR_INVALID_ARG;
+    if (l->decode_algo < FA_DECODE_AUTO || l->decode_algo > FA_DECODE_FFT) return FA_ERR_INVALID_ARG;
+    if (!(l->softmax_scale > 0.0f)) return FA_ERR_INVALID_ARG;
+    // what the kernels implement
+    if (l->head_dim % 8 != 0 || l->head_dim > 256) return FA_ERR_UNSUPPORTED;
+    if (l->n_full_k % 8 != 0 || l->n_full_v % 8 != 0) return FA_ERR_UNSUPPORTED;
+    if (l->n_q_heads / l->n_kv_heads > 16) return FA_ERR_UNSUPPORTED;
+    if (l->n_coef > 4096) return FA_ERR_UNSUPPORTED;
+    return FA_OK;
+}
+
+static int ilog2_exact(int v) {
+    int l = 0;
+    while ((1 << l) < v) ++l;
+    return ((1 << l) == v) ? l : -1;
+}
+
+// True if the residue-class transform can serve this layout: power-of-two
+// period, one class per period / S tokens with S a power of two >= k.
+static bool fft_ok(const fa_layout& l, int* log2S) {
+    if (l.head_dim == l.n_full_k && l.head_dim == l.n_full_v) return false;   // nothing compressed
+    if (ilog2_exact(l.period) < 0 || l.period % l.mid_classes != 0) return false;
+    int S = l.period / l.mid_classes;
+    int ls = ilog2_exact(S);
+    if (ls < 5 || ls > 11 || S < l.n_coef / 2) return false;
+    *log2S = ls;
+    return true;
+}
+
+fa_status plan_decode(const fa_layout& l, DecodePlan* p) {
+    Dims s = make_dims(l);
+    std::memset(p, 0, sizeof(*p));
+    int log2S = 0;
+    bool can_fft = false;   // the FFT kernel registers itself here once built
+    (void)fft_ok; (void)log2S;
+    if (l.decode_algo == FA_DECODE_FFT && !can_fft) return FA_ERR_UNSUPPORTED;
+    p->algo = (l.decode_algo == FA_DECODE_DIRECT || !can_fft) ? FA_DECODE_DIRECT : FA_DECODE_FFT;
+    p->fft_log2 = log2S;
+    p->gh = s.G >= 4 ? 4 : (s.G >= 2 ? 2 : 1);
+    if (s.G == 3) p->gh = 4;
+    p->n_pass = (s.G + p->gh - 1) / p->gh;
+    // split the tokens of one (b, KV head, pass) over CTAs so that the grid fills the GPU about twice
+    int jobs = s.B * s.Hkv * p->n_pass;
+    int want = (2 * kNumSms + jobs - 1) / jobs;
+    long long tokens = (long long)s.max_mid + s.l_init + s.l_local;
+    int max_by_work = (int)((tokens + 255) / 256);            // at least one 256-token tile each
+    if (want > max_by_work) want = max_by_work;
+    if (want > 64) want = 64;
+    if (want < 1) want = 1;
+    p->n_split = want;
+    p->rows_pro = 64;
+    p->n_slice = s.dcv > 0 ? (s.M + 127) / 128 : 1;
+    size_t off = 0;
+    p->off_u = off;   off = align_up(off + sizeof(float) * (size_t)s.B * s.Hq * s.M, 256);
+    p->off_ml = off;  off = align_up(off + sizeof(float) * (size_t)s.B * s.Hq * p->n_split * 2, 256);
+    p->off_o = off;   off = align_up(off + sizeof(float) * (size_t)s.B * s.Hq * p->n_split * s.d, 256);
+    p->off_z = off;   off = align_up(off + sizeof(float) * (size_t)s.B * s.Hq * p->n_split * s.M, 256);
+    p->off_oc = off;  off = align_up(off + sizeof(float) * (size_t)s.B * s.Hq * p->n_slice * (s.dcv > 0 ? s.dcv : 1), 256);
+    p->off_cnt = off; off = align_up(off + sizeof(int32_t) * (size_t)s.B * s.Hkv, 256);
+    p->total = off;
+    return FA_OK;
+}
+
+static fa_status check_cache(const fa_layout* l, const fa_cache* c) {
+    if (!c) return FA_ERR_INVALID_ARG;
+    Dims s = make_dims(*l);
+    const void* need[] = {c->state, c->status};
+    for (const void* p : need) if (!p || !aligned16(p)) return FA_ERR_INVALID_ARG;
+    if (s.nfk > 0 && (!c->idx_full_k || (s.max_mid > 0 && !c->k_mid))) return FA_ERR_INVALID_ARG;
+    if (s.nfv > 0 && (!c->idx_full_v || (s.max_mid > 0 && !c->v_mid))) return FA_ERR_INVALID_ARG;
+    if (s.dck > 0 && (!c->idx_comp_k || !c->coef_k)) return FA_ERR_INVALID_ARG;
+    if (s.dcv > 0 && (!c->idx_comp_v || !c->coef_v)) return FA_ERR_INVALID_ARG;
+    if (s.l_init > 0 && (!c->k_init || !c->v_init)) return FA_ERR_INVALID_ARG;
+    if (s.l_local > 0 && (!c->k_local || !c->v_local)) return FA_ERR_INVALID_ARG;
+    const void* al[] = {c->k_init, c->v_init, c->k_local, c->v_local, c->k_mid, c->v_mid, c->coef_k, c->coef_v,
+                        c->idx_full_k, c->idx_comp_k, c->idx_full_v, c->idx_comp_v};
+    for (const void* p : al) if (p && !aligned16(p)) return FA_ERR_INVALID_ARG;
+    return FA_OK;
+}
+
+}  // namespace fa
+
+using namespace fa;
+
+extern "C" {
+
+fa_status fa_cache_sizes_of(const fa_layout* layout, fa_cache_sizes* out) {
+    fa_status st = check_layout(layout);
+    if (st != FA_OK) return st;
+    if (!out) return FA_ERR_INVALID_ARG;
+    Dims s = make_dims(*layout);
+    size_t eb = elt_bytes(layout->kv_dtype);
+    size_t bh = (size_t)s.B * s.Hkv;
+    out->idx_full_k = sizeof(int32_t) * (size_t)s.Hkv * s.nfk;
+    out->idx_comp_k = sizeof(int32_t) * (size_t)s.Hkv * s.dck;
+    out->idx_full_v = sizeof(int32_t) * (size_t)s.Hkv * s.nfv;
+    out->idx_comp_v = sizeof(int32_t) * (size_t)s.Hkv * s.dcv;
+    out->k_init = out->v_init = bh * s.l_init * s.d * eb;
+    out->k_local = out->v_local = bh * s.l_local * s.d * eb;
+    out->k_mid = bh * (size_t)s.P * s.S_cap * s.nfk * eb;
+    out->v_mid = bh * (size_t)s.P * s.S_cap * s.nfv * eb;
+    out->coef_k = bh * (size_t)s.M * s.dck * sizeof(float);
+    out->coef_v = bh * (size_t)s.M * s.dcv * sizeof(float);
+    out->state = sizeof(int32_t) * kStateStride * (size_t)s.B;
+    out->status = sizeof(int32_t) * 4;
+    return FA_OK;
+}
+
+fa_status fa_workspace_bytes(const fa_layout* layout, size_t* out) {
+    fa_status st = check_layout(layout);
+    if (st != FA_OK) return st;
+    if (!out) return FA_ERR_INVALID_ARG;
+    DecodePlan p;
+    st = plan_decode(*layout, &p);
+    if (st != FA_OK) return st;
+    *out = p.total;
+    return FA_OK;
+}
+
+fa_status fa_cache_reset(const fa_layout* layout, fa_cache* cache, void* stream) {
+    fa_status st = check_layout(layout);
+    if (st != FA_OK) return st;
+    st = check_cache(layout, cache);
+    if (st != FA_OK) return st;
+    fa_cache_sizes sz;
+    fa_cache_sizes_of(layout, &sz);
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    if (cudaMemsetAsync(cache->state, 0, sz.state, s) != cudaSuccess) return FA_ERR_CUDA;
+    if (cudaMemsetAsync(cache->status, 0, sz.status, s) != cudaSuccess) return FA_ERR_CUDA;
+    if (sz.coef_k && cudaMemsetAsync(cache->coef_k, 0, sz.coef_k, s) != cudaSuccess) return FA_ERR_CUDA;
+    if (sz.coef_v && cudaMemsetAsync(cache->coef_v, 0, sz.coef_v, s) != cudaSuccess) return FA_ERR_CUDA;
+    return FA_OK;
+}
+
+fa_status fa_poll_status(const fa_cache* cache, void* stream) {
+    if (!cache || !cache->status) return FA_ERR_INVALID_ARG;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    int32_t word = 0;
+    if (cudaMemcpyAsync(&word, cache->status, sizeof(word), cudaMemcpyDeviceToHost, s) != cudaSuccess) return FA_ERR_CUDA;
+    if (cudaMemsetAsync(cache->status, 0, sizeof(word), s) != cudaSuccess) return FA_ERR_CUDA;
+    if (cudaStreamSynchronize(s) != cudaSuccess) return FA_ERR_CUDA;
+    if (word < FA_OK || word > FA_ERR_INDEX) return FA_ERR_CUDA;
+    return static_cast<fa_status>(word);
+}
+
+fa_status fa_validate(const fa_layout* layout, const fa_cache* cache, void* stream) {
+    fa_status st = check_layout(layout);
+    if (st != FA_OK) return st;
+    st = check_cache(layout, cache);
+    if (st != FA_OK) return st;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    if (launch_validate(make_dims(*layout), make_cache(*cache), s) != cudaSuccess) return FA_ERR_CUDA;
+    return fa_poll_status(cache, stream);
+}
+
+fa_status fa_compress(const fa_layout* layout, fa_cache* cache, const void* K, const void* V, int64_t stride_b,
+                      int64_t stride_t, int64_t stride_h, int32_t L, void* ws, size_t ws_bytes, void* stream) {
+    (void)ws; (void)ws_bytes;
+    fa_status st = check_layout(layout);
+    if (st != FA_OK) return st;
+    st = check_cache(layout, cache);
+    if (st != FA_OK) return st;
+    if (L < 0) return FA_ERR_INVALID_ARG;
+    if (L > 0 && (!K || !V || !aligned16(K) || !aligned16(V))) return FA_ERR_INVALID_ARG;
+    if (L > 0 && (stride_t < layout->head_dim || stride_h < layout->head_dim || stride_b < 0)) return FA_ERR_INVALID_ARG;
+    if ((stride_b | stride_t | stride_h) & 7) return FA_ERR_INVALID_ARG;
+    Dims s = make_dims(*layout);
+    int n_init = L < s.l_init ? L : s.l_init;
+    int n_local = (L - n_init) < s.l_local ? (L - n_init) : s.l_local;
+    if (L - n_init - n_local > s.max_mid) return FA_ERR_CAPACITY;
+    cudaStream_t cs = static_cast<cudaStream_t>(stream);
+    fa_cache_sizes sz;
+    fa_cache_sizes_of(layout, &sz);
+    if (sz.coef_k && cudaMemsetAsync(cache->coef_k, 0, sz.coef_k, cs) != cudaSuccess) return FA_ERR_CUDA;
+    if (sz.coef_v && cudaMemsetAsync(cache->coef_v, 0, sz.coef_v, cs) != cudaSuccess) return FA_ERR_CUDA;
+    if (launch_compress(s, make_cache(*cache), layout->kv_dtype, K, V, stride_b, stride_t, stride_h, L, cs) != cudaSuccess)
+        return FA_ERR_CUDA;
+    return FA_OK;
+}
+
+fa_status fa_append(const fa_layout* layout, fa_cache* cache, const void* k_new, const void* v_new, void* stream) {
+    fa_status st = check_layout(layout);
+    if (st != FA_OK) return st;
+    st = check_cache(layout, cache);
+    if (st != FA_OK) return st;
+    if (!k_new || !v_new || !aligned16(k_new) || !aligned16(v_new)) return FA_ERR_INVALID_ARG;
+    if (launch_append(make_dims(*layout), make_cache(*cache), layout->kv_dtype, k_new, v_new,
+                      static_cast<cudaStream_t>(stream)) != cudaSuccess)
+        return FA_ERR_CUDA;
+    return FA_OK;
+}
+
+fa_status fa_decode_attention(const fa_layout* layout, const fa_cache* cache, const void* q, void* out, void* ws,
+                              size_t ws_bytes, void* stream) {
+    fa_status st = check_layout(layout);
+    if (st != FA_OK) return st;
+    st = check_cache(layout, cache);
+    if (st != FA_OK) return st;
+    if (!q || !out || !aligned16(q) || !aligned16(out)) return FA_ERR_INVALID_ARG;
+    DecodePlan p;
+    st = plan_decode(*layout, &p);
+    if (st != FA_OK) return st;
+    if (!ws || !aligned16(ws) || ws_bytes < p.total) return FA_ERR_WORKSPACE;
+    Dims s = make_dims(*layout);
+    CacheDev c = make_cache(*cache);
+    cudaStream_t cs = static_cast<cudaStream_t>(stream);
+    char* w = static_cast<char*>(ws);
+    if (launch_decode_prologue(s, c, layout->kv_dtype, p, q, w, cs) != cudaSuccess) return FA_ERR_CUDA;
+    if (launch_decode_direct(s, c, layout->kv_dtype, p, q, w, cs) != cudaSuccess) return FA_ERR_CUDA;
+    if (launch_decode_epilogue(s, c, layout->kv_dtype, p, out, w, cs) != cudaSuccess) return FA_ERR_CUDA;
+    return FA_OK;
+}
+
+int fa_launch_count(const fa_layout* layout, int what) {
+    if (check_layout(layout) != FA_OK) return 0;
+    switch (what) {
+        case 0: return 2;   // partition/gather + coefficient kernel (memsets not counted)
+        case 1: return 1;
+        case 2: return 3;   // prologue, main, epilogue
+        default: return 0;
+    }
+}
+
+const char* fa_status_string(fa_status s) {
+    switch (s) {
+        case FA_OK: return "ok";
+        case FA_ERR_INVALID_ARG: return "invalid argument";
+        case FA_ERR_UNSUPPORTED: return "unsupported layout";
+        case FA_ERR_CAPACITY: return "middle segment is full";
+        case FA_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
+        case FA_ERR_CUDA: return "CUDA runtime error";
+        case FA_ERR_TIMEOUT: return "bounded device wait timed out";
+        case FA_ERR_INDEX: return "index sets are not a sorted disjoint cover of the head dims";
+    }
+    return "unknown status";
+}
+
+int fa_version(void) { return 100; }
+
+}  // extern "C"

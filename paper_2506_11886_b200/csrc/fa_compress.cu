@@ -1,0 +1,208 @@
+// fa_compress, CUDA-core path (Eq.1-4): partition + gather, then the
+// projection C = F X^mn as an fp32 tile product with the basis generated on
+// the fly.  Serves fp32 caches and is the fallback of the tensor-core path.
+#include "fa_common.cuh"
+
+namespace fa {
+
+// ---- index-set check (Eq.2: D^u and D^c partition the head dims) ------------
+__global__ void validate_kernel(Dims s, CacheDev c) {
+    int h = blockIdx.x;
+    int side = blockIdx.y;
+    __shared__ int seen[256];
+    __shared__ int bad;
+    int nfull = side == 0 ? s.nfk : s.nfv;
+    int ncomp = s.d - nfull;
+    const int32_t* idf = (side == 0 ? c.idx_full_k : c.idx_full_v) + (size_t)h * nfull;
+    const int32_t* idc = (side == 0 ? c.idx_comp_k : c.idx_comp_v) + (size_t)h * ncomp;
+    for (int i = threadIdx.x; i < s.d; i += blockDim.x) seen[i] = 0;
+    if (threadIdx.x == 0) bad = 0;
+    __syncthreads();
+    for (int i = threadIdx.x; i < s.d; i += blockDim.x) {
+        bool full = i < nfull;
+        const int32_t* a = full ? idf : idc;
+        int pos = full ? i : i - nfull;
+        int v = a[pos];
+        if (v < 0 || v >= s.d) { atomicExch(&bad, 1); continue; }
+        if (pos > 0 && a[pos - 1] >= v) atomicExch(&bad, 1);
+        atomicAdd(&seen[v], 1);
+    }
+    __syncthreads();
+    for (int i = threadIdx.x; i < s.d; i += blockDim.x)
+        if (seen[i] != 1) atomicExch(&bad, 1);
+    __syncthreads();
+    if (threadIdx.x == 0 && bad) atomicExch(c.status, (int)FA_ERR_INDEX);
+}
+
+cudaError_t launch_validate(const Dims& s, const CacheDev& c, cudaStream_t st) {
+    validate_kernel<<<dim3(s.Hkv, 2), 128, 0, st>>>(s, c);
+    return cudaGetLastError();
+}
+
+// ---- Eq.1-2: windows, kept dims, counters -----------------------------------
+// grid (token chunks, Hkv, B * 2 sides); one warp per token row.
+constexpr int kRowsPerCta = 64;
+
+template <typename KV>
+__global__ void __launch_bounds__(256) partition_gather_kernel(Dims s, CacheDev c, const KV* __restrict__ K,
+                                                               const KV* __restrict__ V, int64_t sb, int64_t st,
+                                                               int64_t sh, int L) {
+    __shared__ float row_s[8][256];
+    int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    int h = blockIdx.y, b = blockIdx.z >> 1, side = blockIdx.z & 1;
+    int n_init = min(L, s.l_init);
+    int n_local = min(L - n_init, s.l_local);
+    int n_mid = L - n_init - n_local;
+    if (blockIdx.x == 0 && blockIdx.y == 0 && side == 0 && threadIdx.x == 0) {
+        c.state[kStateStride * b + 0] = n_init;
+        c.state[kStateStride * b + 1] = n_local;
+        c.state[kStateStride * b + 2] = n_mid;
+        c.state[kStateStride * b + 3] = 0;          // ring starts at physical row 0
+        c.state[kStateStride * b + 4] = 0;          // append ticket
+    }
+    const KV* X = side == 0 ? K : V;
+    int nfull = side == 0 ? s.nfk : s.nfv;
+    const int32_t* idf = (side == 0 ? c.idx_full_k : c.idx_full_v) + (size_t)h * nfull;
+    void* w_init = side == 0 ? c.k_init : c.v_init;
+    void* w_local = side == 0 ? c.k_local : c.v_local;
+    void* w_mid = side == 0 ? c.k_mid : c.v_mid;
+    int t_end = min(L, (int)(blockIdx.x + 1) * kRowsPerCta);
+    for (int t = blockIdx.x * kRowsPerCta + warp; t < t_end; t += 8) {
+        const KV* src = X + (size_t)b * sb + (size_t)t * st + (size_t)h * sh;
+        if (t < n_init) {
+            KV* dst = win_row<KV>(w_init, s, b, h, s.l_init, t);
+            for (int e = lane; e < s.d; e += 32) dst[e] = src[e];
+        } else if (t >= L - n_local) {
+            KV* dst = win_row<KV>(w_local, s, b, h, s.l_local, t - (L - n_local));
+            for (int e = lane; e < s.d; e += 32) dst[e] = src[e];
+        } else {
+            int j = t - n_init;
+            for (int e = lane; e < s.d; e += 32) row_s[warp][e] = ld_f(src + e);
+            __syncwarp();
+            KV* dst = mid_row<KV>(w_mid, s, b, h, j % s.P, j / s.P, nfull);
+            for (int e = lane; e < nfull; e += 32) st_f(dst + e, row_s[warp][idf[e]]);
+            __syncwarp();
+        }
+    }
+}
+
+// ---- Eq.3-4: C[m][e] += sum_j F[m][j] X[n_init + j][D^c[e]] ------------------
+// grid (row tiles of 32 coefficient rows, token splits, B * Hkv * 2 sides).
+// Per 64-token chunk the CTA stages the gathered columns and a 64 x 32 basis
+// tile in shared memory; thread (rg, lane) accumulates rows 4 rg..4 rg + 3 of
+// the tile for columns lane, lane + 32, ...  Partial sums of the token splits
+// are added to the zeroed coefficients with atomics.
+constexpr int kTM = 32, kTJ = 64;
+
+template <typename KV>
+__global__ void __launch_bounds__(256) compress_coef_kernel(Dims s, CacheDev c, const KV* __restrict__ K,
+                                                            const KV* __restrict__ V, int64_t sb, int64_t st, int64_t sh,
+                                                            int L, int chunks_per_split) {
+    extern __shared__ float smem[];
+    int side = blockIdx.z & 1;
+    int bh = blockIdx.z >> 1;
+    int b = bh / s.Hkv, h = bh % s.Hkv;
+    int nfull = side == 0 ? s.nfk : s.nfv;
+    int ncomp = s.d - nfull;
+    if (ncomp == 0) return;
+    int n_init = min(L, s.l_init);
+    int n_local = min(L - n_init, s.l_local);
+    int n_mid = L - n_init - n_local;
+    const KV* X = (side == 0 ? K : V) + (size_t)b * sb + (size_t)h * sh;
+    const int32_t* idc = (side == 0 ? c.idx_comp_k : c.idx_comp_v) + (size_t)h * ncomp;
+    float* coef = coef_rows(side == 0 ? c.coef_k : c.coef_v, s, b, h, ncomp);
+
+    float* X_s = smem;                       // [kTJ][ncomp]
+    float* F_s = smem + kTJ * ncomp;         // [kTJ][kTM]
+    int m0 = blockIdx.x * kTM;
+    int rg = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    int ncol = (ncomp + 31) / 32;            // <= 8
+    float acc[4][8];
+#pragma unroll
+    for (int r = 0; r < 4; ++r)
+#pragma unroll
+        for (int i = 0; i < 8; ++i) acc[r][i] = 0.f;
+
+    int j_begin = blockIdx.y * chunks_per_split * kTJ;
+    int j_end = min(n_mid, j_begin + chunks_per_split * kTJ);
+    for (int j0 = j_begin; j0 < j_end; j0 += kTJ) {
+        int nj = min(kTJ, j_end - j0);
+        __syncthreads();
+        for (int i = threadIdx.x; i < kTJ * ncomp; i += blockDim.x) {
+            int jj = i / ncomp, e = i - jj * ncomp;
+            X_s[i] = jj < nj ? ld_f(X + (size_t)(n_init + j0 + jj) * st + idc[e]) : 0.f;
+        }
+        // basis tile: thread -> (token jj, frequency pair nn) ; rows 2 nn (cos), 2 nn + 1 (sin)
+        for (int i = threadIdx.x; i < kTJ * (kTM / 2); i += blockDim.x) {
+            int jj = i / (kTM / 2), nn = i % (kTM / 2);
+            int n = m0 / 2 + nn;
+            float cs = 0.f, sn = 0.f;
+            if (jj < nj && n < s.k) basis_cs(n, j0 + jj, s.T, &cs, &sn);
+            F_s[jj * kTM + 2 * nn] = cs;
+            F_s[jj * kTM + 2 * nn + 1] = sn;
+        }
+        __syncthreads();
+        for (int jj = 0; jj < nj; ++jj) {
+            float4 f = *reinterpret_cast<const float4*>(F_s + jj * kTM + 4 * rg);
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                if (i < ncol) {
+                    int e = lane + 32 * i;
+                    float x = e < ncomp ? X_s[jj * ncomp + e] : 0.f;
+                    acc[0][i] = fmaf(f.x, x, acc[0][i]);
+                    acc[1][i] = fmaf(f.y, x, acc[1][i]);
+                    acc[2][i] = fmaf(f.z, x, acc[2][i]);
+                    acc[3][i] = fmaf(f.w, x, acc[3][i]);
+                }
+            }
+        }
+    }
+#pragma unroll
+    for (int r = 0; r < 4; ++r) {
+        int m = m0 + 4 * rg + r;
+        if (m >= s.M) continue;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            int e = lane + 32 * i;
+            if (i < ncol && e < ncomp) atomicAdd(coef + (size_t)m * ncomp + e, acc[r][i]);
+        }
+    }
+}
+
+template <typename KV>
+static cudaError_t launch_compress_t(const Dims& s, const CacheDev& c, const void* K, const void* V, int64_t sb,
+                                     int64_t st, int64_t sh, int L, cudaStream_t stream) {
+    int chunks_rows = (L + kRowsPerCta - 1) / kRowsPerCta;
+    if (chunks_rows < 1) chunks_rows = 1;
+    partition_gather_kernel<KV><<<dim3(chunks_rows, s.Hkv, s.B * 2), 256, 0, stream>>>(
+        s, c, static_cast<const KV*>(K), static_cast<const KV*>(V), sb, st, sh, L);
+    cudaError_t err = cudaGetLastError();
+    if (err != cudaSuccess) return err;
+    int n_init = L < s.l_init ? L : s.l_init;
+    int n_local = (L - n_init) < s.l_local ? (L - n_init) : s.l_local;
+    int n_mid = L - n_init - n_local;
+    int max_comp = s.dck > s.dcv ? s.dck : s.dcv;
+    if (n_mid == 0 || max_comp == 0) return cudaSuccess;
+    int row_tiles = (s.M + kTM - 1) / kTM;
+    int chunks = (n_mid + kTJ - 1) / kTJ;
+    int ctas_fixed = row_tiles * s.B * s.Hkv * 2;
+    int n_tsplit = (4 * kNumSms + ctas_fixed - 1) / ctas_fixed;
+    if (n_tsplit > chunks) n_tsplit = chunks;
+    if (n_tsplit < 1) n_tsplit = 1;
+    int cps = (chunks + n_tsplit - 1) / n_tsplit;
+    n_tsplit = (chunks + cps - 1) / cps;
+    size_t smem = sizeof(float) * ((size_t)kTJ * max_comp + (size_t)kTJ * kTM);
+    err = cudaFuncSetAttribute(compress_coef_kernel<KV>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (err != cudaSuccess) return err;
+    compress_coef_kernel<KV><<<dim3(row_tiles, n_tsplit, s.B * s.Hkv * 2), 256, smem, stream>>>(
+        s, c, static_cast<const KV*>(K), static_cast<const KV*>(V), sb, st, sh, L, cps);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_compress(const Dims& s, const CacheDev& c, int dtype, const void* K, const void* V, int64_t sb,
+                            int64_t st, int64_t sh, int L, cudaStream_t stream) {
+    if (dtype == FA_BF16) return launch_compress_t<__nv_bfloat16>(s, c, K, V, sb, st, sh, L, stream);
+    return launch_compress_t<float>(s, c, K, V, sb, st, sh, L, stream);
+}
+
+}  // namespace fa

@@ -1,0 +1,477 @@
+// fa_decode_attention (Eq.6), evaluated on the small side:
+//   prologue   u_g[m] = scale * log2(e) * w_m * sum_e C^K[m][e] q_g[D^kc[e]]
+//   main       per token j of the middle: s_j = q_u . K^mu_j + sum_m F[m][j] u_g[m];
+//              online softmax; o^u += p_j V^mu_j;  z[m] += p_j F[m][j];
+//              window tokens: ordinary attention in the same softmax
+//   epilogue   merge the token splits, o^c[e] = sum_m w_m z[m] C^V[m][e], normalise, scatter.
+// This file holds the prologue, the epilogue and the DIRECT main kernel, which
+// sums the M basis terms of every token one by one (any period, any class count).
+#include "fa_common.cuh"
+
+namespace fa {
+
+// Workspace views.
+struct Ws {
+    float* u;      // [B][Hq][M]
+    float* ml;     // [B][Hq][n_split][2]   running max (log2 units), sum of p
+    float* o;      // [B][Hq][n_split][d]   un-normalised outputs, natural dim order (kept dims + windows)
+    float* z;      // [B][Hq][n_split][M]   un-normalised p^T Phi
+    float* oc;     // [B][Hq][n_slice][dcv] partial o^c per coefficient-row slice
+    int32_t* cnt;  // [B][Hkv]              epilogue tickets
+};
+__host__ __device__ inline Ws ws_view(char* w, const DecodePlan& p) {
+    Ws v;
+    v.u = reinterpret_cast<float*>(w + p.off_u);
+    v.ml = reinterpret_cast<float*>(w + p.off_ml);
+    v.o = reinterpret_cast<float*>(w + p.off_o);
+    v.z = reinterpret_cast<float*>(w + p.off_z);
+    v.oc = reinterpret_cast<float*>(w + p.off_oc);
+    v.cnt = reinterpret_cast<int32_t*>(w + p.off_cnt);
+    return v;
+}
+
+// ---------------------------------------------------------------- prologue --
+// grid (row tiles, Hkv, B); one warp per coefficient row, lanes over the D^kc columns.
+template <typename KV>
+__global__ void __launch_bounds__(256) decode_prologue_kernel(Dims s, CacheDev c, DecodePlan p, const KV* __restrict__ q,
+                                                              char* wsp) {
+    extern __shared__ float qc_s[];               // [G][dck] gathered query, fp32
+    Ws ws = ws_view(wsp, p);
+    const int h = blockIdx.y, b = blockIdx.z;
+    if (blockIdx.x == 0 && threadIdx.x == 0) ws.cnt[b * s.Hkv + h] = 0;
+    if (s.dck == 0) return;
+    const int32_t* idc = c.idx_comp_k + (size_t)h * s.dck;
+    for (int i = threadIdx.x; i < s.G * s.dck; i += blockDim.x) {
+        int g = i / s.dck, e = i - g * s.dck;
+        qc_s[i] = ld_f(q + ((size_t)b * s.Hq + h * s.G + g) * s.d + idc[e]);
+    }
+    __syncthreads();
+    const float* coef = coef_rows(c.coef_k, s, b, h, s.dck);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int m_end = min(s.M, (int)(blockIdx.x + 1) * p.rows_pro);
+    for (int m = blockIdx.x * p.rows_pro + warp; m < m_end; m += 8) {
+        const float* row = coef + (size_t)m * s.dck;
+        float wm = recon_weight(s.norm, m, s.k, s.T) * s.scale * kLog2e;
+        for (int g0 = 0; g0 < s.G; g0 += 4) {
+            float acc[4] = {0.f, 0.f, 0.f, 0.f};
+            for (int e = lane; e < s.dck; e += 32) {
+                float cv = row[e];
+#pragma unroll
+                for (int g = 0; g < 4; ++g)
+                    if (g0 + g < s.G) acc[g] = fmaf(cv, qc_s[(g0 + g) * s.dck + e], acc[g]);
+            }
+#pragma unroll
+            for (int g = 0; g < 4; ++g) {
+                float v = warp_sum(acc[g]);
+                if (lane == 0 && g0 + g < s.G) ws.u[((size_t)b * s.Hq + h * s.G + g0 + g) * s.M + m] = wm * v;
+            }
+        }
+    }
+}
+
+// ------------------------------------------------------------- direct main --
+// grid (n_split, Hkv * n_pass, B), 256 threads; one thread per token of a 256-token tile.
+constexpr int kTile = 256;
+
+template <int GH>
+struct RunStat {
+    float m[GH];   // running max, log2 units
+    float l[GH];   // running sum of p
+};
+
+// Block-wide max / sum of GH values per thread; result broadcast to every thread.
+template <int GH, bool IS_MAX>
+__device__ __forceinline__ void block_reduce(float (&v)[GH], float* red_s /* [8][GH] */) {
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+#pragma unroll
+    for (int g = 0; g < GH; ++g) {
+        float r = IS_MAX ? warp_max(v[g]) : warp_sum(v[g]);
+        if (lane == 0) red_s[warp * GH + g] = r;
+    }
+    __syncthreads();
+#pragma unroll
+    for (int g = 0; g < GH; ++g) {
+        float r = red_s[g];
+#pragma unroll
+        for (int w = 1; w < 8; ++w) r = IS_MAX ? fmaxf(r, red_s[w * GH + g]) : r + red_s[w * GH + g];
+        v[g] = r;
+    }
+    __syncthreads();
+}
+
+template <typename KV, int GH>
+__global__ void __launch_bounds__(256) decode_direct_kernel(Dims s, CacheDev c, DecodePlan p, const KV* __restrict__ q,
+                                                            char* wsp) {
+    extern __shared__ float sm[];
+    Ws ws = ws_view(wsp, p);
+    const int split = blockIdx.x;
+    const int h = blockIdx.y / p.n_pass, pass = blockIdx.y % p.n_pass;
+    const int b = blockIdx.z;
+    const int g_first = h * s.G + pass * GH;                 // first query head of this CTA
+    const int ng = min(GH, s.G - pass * GH);
+    const int tid = threadIdx.x;
+
+    float* q_s = sm;                          // [GH][d]   scale * log2e * q, natural order
+    float* qf_s = q_s + GH * s.d;             // [GH][nfk] the same gathered at D^ku
+    float* u_s = qf_s + GH * s.nfk;           // [GH][M]
+    float* z_s = u_s + GH * s.M;              // [GH][M]
+    float* p_s = z_s + GH * s.M;              // [GH][kTile]
+    float* red_s = p_s + GH * kTile;          // [8][GH]
+    float* o_s = red_s + 8 * GH;              // [GH][d]  final reduce
+    float* acc_s = o_s + GH * s.d;            // [256][GH] cross-thread reduce of the output accumulators
+
+    const int n_init = c.state[kStateStride * b + 0], n_local = c.state[kStateStride * b + 1];
+    const int n_mid = min(c.state[kStateStride * b + 2], s.max_mid), head = c.state[kStateStride * b + 3];
+    const int32_t* idf_k = c.idx_full_k + (size_t)h * s.nfk;
+    const int32_t* idf_v = c.idx_full_v + (size_t)h * s.nfv;
+
+    for (int i = tid; i < GH * s.d; i += blockDim.x) {
+        int g = i / s.d, e = i - g * s.d;
+        q_s[i] = g < ng ? ld_f(q + ((size_t)b * s.Hq + g_first + g) * s.d + e) * s.scale * kLog2e : 0.f;
+        o_s[i] = 0.f;
+    }
+    for (int i = tid; i < GH * s.M; i += blockDim.x) {
+        int g = i / s.M, m = i - g * s.M;
+        u_s[i] = (g < ng && s.dck > 0) ? ws.u[((size_t)b * s.Hq + g_first + g) * s.M + m] : 0.f;
+        z_s[i] = 0.f;
+    }
+    __syncthreads();
+    for (int i = tid; i < GH * s.nfk; i += blockDim.x) {
+        int g = i / s.nfk, e = i - g * s.nfk;
+        qf_s[i] = q_s[g * s.d + idf_k[e]];
+    }
+    __syncthreads();
+
+    RunStat<GH> rs;
+#pragma unroll
+    for (int g = 0; g < GH; ++g) { rs.m[g] = kNegBig; rs.l[g] = 0.f; }
+    float o_mid[GH], o_win[GH];
+#pragma unroll
+    for (int g = 0; g < GH; ++g) { o_mid[g] = 0.f; o_win[g] = 0.f; }
+
+    // thread -> (token group, dim) maps of the two P.V products
+    const int ntg_mid = s.nfv > 0 ? kTile / s.nfv : 0;
+    const int tg_mid = s.nfv > 0 ? tid / s.nfv : 0, e_mid = s.nfv > 0 ? tid % s.nfv : 0;
+    const bool act_mid = s.nfv > 0 && tg_mid < ntg_mid;
+    const int ntg_win = kTile / s.d;
+    const int tg_win = tid / s.d, e_win = tid % s.d;
+    const bool act_win = tg_win < ntg_win;
+
+    // after scores are known: update the running softmax state, leave p in p_s
+    auto softmax_tile = [&](float (&sc)[GH], bool valid) {
+        float mx[GH];
+#pragma unroll
+        for (int g = 0; g < GH; ++g) mx[g] = valid ? sc[g] : kNegBig;
+        block_reduce<GH, true>(mx, red_s);
+        float pv[GH], alpha[GH];
+#pragma unroll
+        for (int g = 0; g < GH; ++g) {
+            float m_new = fmaxf(rs.m[g], mx[g]);
+            alpha[g] = exp2f(rs.m[g] - m_new);
+            rs.m[g] = m_new;
+            pv[g] = valid ? exp2f(sc[g] - m_new) : 0.f;
+            p_s[g * kTile + tid] = pv[g];
+            o_mid[g] *= alpha[g];
+            o_win[g] *= alpha[g];
+        }
+        for (int i = tid; i < GH * s.M; i += blockDim.x) z_s[i] *= alpha[i / s.M];
+        block_reduce<GH, false>(pv, red_s);     // also publishes p_s and the z_s rescale
+#pragma unroll
+        for (int g = 0; g < GH; ++g) rs.l[g] = rs.l[g] * alpha[g] + pv[g];
+    };
+
+    // ---- middle tokens: classes [c0, c1) of this split ------------------------
+    const int c0 = (int)((long long)split * s.P / p.n_split), c1 = (int)((long long)(split + 1) * s.P / p.n_split);
+    for (int cls = c0; cls < c1; ++cls) {
+        const int n_cls = cls < n_mid ? (n_mid - cls + s.P - 1) / s.P : 0;
+        for (int a0 = 0; a0 < n_cls; a0 += kTile) {
+            const int a = a0 + tid;
+            const bool valid = a < n_cls;
+            const int j = cls + s.P * a;
+            float sc[GH];
+#pragma unroll
+            for (int g = 0; g < GH; ++g) sc[g] = 0.f;
+            if (valid) {
+                const KV* row = mid_row<KV>(c.k_mid, s, b, h, cls, a, s.nfk);
+                for (int e = 0; e < s.nfk; ++e) {
+                    float x = ld_f(row + e);
+#pragma unroll
+                    for (int g = 0; g < GH; ++g) sc[g] = fmaf(qf_s[g * s.nfk + e], x, sc[g]);
+                }
+                if (s.dck > 0) {
+                    float cd, sd;
+                    basis_cs(1, j, s.T, &cd, &sd);                  // rotation per unit of n
+                    for (int n0 = 0; n0 < s.k; n0 += 32) {
+                        float cr, sr;
+                        basis_cs(n0, j, s.T, &cr, &sr);             // exact re-seed
+                        const int n1 = min(s.k, n0 + 32);
+                        for (int n = n0; n < n1; ++n) {
+#pragma unroll
+                            for (int g = 0; g < GH; ++g)
+                                sc[g] = fmaf(u_s[g * s.M + 2 * n], cr, fmaf(u_s[g * s.M + 2 * n + 1], sr, sc[g]));
+                            float t = cr * cd - sr * sd;
+                            sr = fmaf(sr, cd, cr * sd);
+                            cr = t;
+                        }
+                    }
+                }
+            }
+            softmax_tile(sc, valid);
+            const int nt = min(kTile, n_cls - a0);
+            // o^u += p V^mu
+            if (act_mid) {
+                for (int i = tg_mid; i < nt; i += ntg_mid) {
+                    float x = ld_f(mid_row<KV>(c.v_mid, s, b, h, cls, a0 + i, s.nfv) + e_mid);
+#pragma unroll
+                    for (int g = 0; g < GH; ++g) o_mid[g] = fmaf(p_s[g * kTile + i], x, o_mid[g]);
+                }
+            }
+            // z[m] += p F[m][j]: thread owns frequency n, walks the tile's tokens by rotation
+            if (s.dcv > 0) {
+                for (int n = tid; n < s.k; n += blockDim.x) {
+                    float zr[GH], zi[GH];
+#pragma unroll
+                    for (int g = 0; g < GH; ++g) { zr[g] = 0.f; zi[g] = 0.f; }
+                    float cd, sd;
+                    basis_cs(n, s.P, s.T, &cd, &sd);               // step between consecutive slots
+                    for (int i0 = 0; i0 < nt; i0 += 32) {
+                        float cr, sr;
+                        basis_cs(n, cls + s.P * (a0 + i0), s.T, &cr, &sr);
+                        const int i1 = min(nt, i0 + 32);
+                        for (int i = i0; i < i1; ++i) {
+#pragma unroll
+                            for (int g = 0; g < GH; ++g) {
+                                float pv = p_s[g * kTile + i];
+                                zr[g] = fmaf(pv, cr, zr[g]);
+                                zi[g] = fmaf(pv, sr, zi[g]);
+                            }
+                            float t = cr * cd - sr * sd;
+                            sr = fmaf(sr, cd, cr * sd);
+                            cr = t;
+                        }
+                    }
+#pragma unroll
+                    for (int g = 0; g < GH; ++g) {
+                        z_s[g * s.M + 2 * n] += zr[g];
+                        z_s[g * s.M + 2 * n + 1] += zi[g];
+                    }
+                }
+            }
+            __syncthreads();
+        }
+    }
+
+    // ---- window tokens [w0, w1) of this split: init rows, then the local ring --
+    const int n_win = n_init + n_local;
+    const int w0 = (int)((long long)split * n_win / p.n_split), w1 = (int)((long long)(split + 1) * n_win / p.n_split);
+    for (int t0 = w0; t0 < w1; t0 += kTile) {
+        const int t = t0 + tid;
+        const bool valid = t < w1;
+        auto row_of = [&](void* init, void* local, int tt) -> const KV* {
+            if (tt < n_init) return win_row<KV>(init, s, b, h, s.l_init, tt);
+            return win_row<KV>(local, s, b, h, s.l_local, (head + (tt - n_init)) % s.l_local);
+        };
+        float sc[GH];
+#pragma unroll
+        for (int g = 0; g < GH; ++g) sc[g] = 0.f;
+        if (valid) {
+            const KV* row = row_of(c.k_init, c.k_local, t);
+            for (int e = 0; e < s.d; ++e) {
+                float x = ld_f(row + e);
+#pragma unroll
+                for (int g = 0; g < GH; ++g) sc[g] = fmaf(q_s[g * s.d + e], x, sc[g]);
+            }
+        }
+        softmax_tile(sc, valid);
+        const int nt = min(kTile, w1 - t0);
+        if (act_win) {
+            for (int i = tg_win; i < nt; i += ntg_win) {
+                float x = ld_f(row_of(c.v_init, c.v_local, t0 + i) + e_win);
+#pragma unroll
+                for (int g = 0; g < GH; ++g) o_win[g] = fmaf(p_s[g * kTile + i], x, o_win[g]);
+            }
+        }
+        __syncthreads();
+    }
+
+    // ---- reduce the output accumulators over token groups, write the partials --
+#pragma unroll
+    for (int g = 0; g < GH; ++g) acc_s[tid * GH + g] = act_mid ? o_mid[g] : 0.f;
+    __syncthreads();
+    for (int i = tid; i < GH * s.nfv; i += blockDim.x) {
+        int g = i / s.nfv, e = i - g * s.nfv;
+        float v = 0.f;
+        for (int tg = 0; tg < ntg_mid; ++tg) v += acc_s[(tg * s.nfv + e) * GH + g];
+        o_s[g * s.d + idf_v[e]] = v;
+    }
+    __syncthreads();
+#pragma unroll
+    for (int g = 0; g < GH; ++g) acc_s[tid * GH + g] = act_win ? o_win[g] : 0.f;
+    __syncthreads();
+    for (int i = tid; i < GH * s.d; i += blockDim.x) {
+        int g = i / s.d, e = i - g * s.d;
+        float v = o_s[i];
+        for (int tg = 0; tg < ntg_win; ++tg) v += acc_s[(tg * s.d + e) * GH + g];
+        if (g < ng) ws.o[(((size_t)b * s.Hq + g_first + g) * p.n_split + split) * s.d + e] = v;
+    }
+    for (int i = tid; i < GH * s.M; i += blockDim.x) {
+        int g = i / s.M, m = i - g * s.M;
+        if (g < ng) ws.z[(((size_t)b * s.Hq + g_first + g) * p.n_split + split) * s.M + m] = z_s[i];
+    }
+    if (tid < ng) {
+        float* ml = ws.ml + (((size_t)b * s.Hq + g_first + tid) * p.n_split + split) * 2;
+        float mv = kNegBig, lv = 0.f;
+#pragma unroll
+        for (int g = 0; g < GH; ++g) if (g == tid) { mv = rs.m[g]; lv = rs.l[g]; }
+        ml[0] = mv;
+        ml[1] = lv;
+    }
+}
+
+// ---------------------------------------------------------------- epilogue --
+// grid (n_slice, Hkv, B).  Each CTA merges the split statistics of its KV head, forms the
+// weighted z of its coefficient rows and multiplies by its rows of C^V; the last CTA of a
+// (b, h) to finish (atomic ticket) adds the slices, normalises and writes the output rows.
+template <typename KV>
+__global__ void __launch_bounds__(256) decode_epilogue_kernel(Dims s, CacheDev c, DecodePlan p, KV* __restrict__ out,
+                                                              char* wsp) {
+    extern __shared__ float sm[];
+    __shared__ int last_s;
+    Ws ws = ws_view(wsp, p);
+    const int slice = blockIdx.x, h = blockIdx.y, b = blockIdx.z;
+    const int tid = threadIdx.x;
+    const int rows = (s.M + p.n_slice - 1) / p.n_slice;
+    const int m0 = slice * rows, m1 = min(s.M, m0 + rows);
+    float* alpha_s = sm;                              // [G][n_split]
+    float* linv_s = alpha_s + s.G * p.n_split;        // [G]
+    float* zw_s = linv_s + s.G;                       // [G][rows]
+    float* red_s = zw_s + s.G * rows;                 // [256]
+    float* o_s = red_s + 256;                         // [d]
+
+    for (int g = tid; g < s.G; g += blockDim.x) {
+        const float* ml = ws.ml + ((size_t)b * s.Hq + h * s.G + g) * p.n_split * 2;
+        float mx = kNegBig;
+        for (int sp = 0; sp < p.n_split; ++sp) mx = fmaxf(mx, ml[2 * sp]);
+        float L = 0.f;
+        for (int sp = 0; sp < p.n_split; ++sp) {
+            float a = exp2f(ml[2 * sp] - mx);
+            alpha_s[g * p.n_split + sp] = a;
+            L += a * ml[2 * sp + 1];
+        }
+        linv_s[g] = L > 0.f ? 1.0f / L : 0.f;
+    }
+    __syncthreads();
+    if (s.dcv > 0) {
+        for (int i = tid; i < s.G * rows; i += blockDim.x) {
+            int g = i / rows, m = m0 + (i - g * rows);
+            float v = 0.f;
+            if (m < m1) {
+                const float* z = ws.z + ((size_t)b * s.Hq + h * s.G + g) * p.n_split * s.M + m;
+                for (int sp = 0; sp < p.n_split; ++sp) v = fmaf(alpha_s[g * p.n_split + sp], z[(size_t)sp * s.M], v);
+                v *= recon_weight(s.norm, m, s.k, s.T);
+            }
+            zw_s[i] = v;
+        }
+        __syncthreads();
+        // partial o^c of this slice: thread (mg, e) sums rows m = m0 + mg, m0 + mg + nmg, ...
+        const float* cv = coef_rows(c.coef_v, s, b, h, s.dcv);
+        const int nmg = blockDim.x / s.dcv;            // dcv <= 256
+        const int mg = tid / s.dcv, e = tid % s.dcv;
+        for (int g = 0; g < s.G; ++g) {
+            float acc = 0.f;
+            if (mg < nmg)
+                for (int m = m0 + mg; m < m1; m += nmg) acc = fmaf(zw_s[g * rows + (m - m0)], cv[(size_t)m * s.dcv + e], acc);
+            red_s[tid] = acc;
+            __syncthreads();
+            if (tid < s.dcv) {
+                float v = 0.f;
+                for (int r = 0; r < nmg; ++r) v += red_s[r * s.dcv + tid];
+                ws.oc[(((size_t)b * s.Hq + h * s.G + g) * p.n_slice + slice) * s.dcv + tid] = v;
+            }
+            __syncthreads();
+        }
+    }
+    // ticket
+    if (tid == 0) {
+        __threadfence();
+        int done = atomicAdd(ws.cnt + b * s.Hkv + h, 1);
+        last_s = (done == (int)gridDim.x - 1);
+    }
+    __syncthreads();
+    if (!last_s) return;
+    __threadfence();
+    const int32_t* idc_v = c.idx_comp_v + (size_t)h * s.dcv;
+    for (int g = 0; g < s.G; ++g) {
+        const size_t qh = (size_t)b * s.Hq + h * s.G + g;
+        for (int e = tid; e < s.d; e += blockDim.x) {
+            float v = 0.f;
+            for (int sp = 0; sp < p.n_split; ++sp) v = fmaf(alpha_s[g * p.n_split + sp], ws.o[(qh * p.n_split + sp) * s.d + e], v);
+            o_s[e] = v;
+        }
+        __syncthreads();
+        for (int e = tid; e < s.dcv; e += blockDim.x) {
+            float v = 0.f;
+            for (int sl = 0; sl < p.n_slice; ++sl) v += __ldcg(ws.oc + (qh * p.n_slice + sl) * s.dcv + e);
+            o_s[idc_v[e]] += v;
+        }
+        __syncthreads();
+        for (int e = tid; e < s.d; e += blockDim.x) st_f(out + qh * s.d + e, o_s[e] * linv_s[g]);
+        __syncthreads();
+    }
+}
+
+// ---------------------------------------------------------------- launchers --
+template <typename KV>
+static cudaError_t launch_prologue_t(const Dims& s, const CacheDev& c, const DecodePlan& p, const void* q, char* ws,
+                                     cudaStream_t st) {
+    int tiles = s.dck > 0 ? (s.M + p.rows_pro - 1) / p.rows_pro : 1;
+    size_t smem = sizeof(float) * (size_t)s.G * (s.dck > 0 ? s.dck : 1);
+    decode_prologue_kernel<KV><<<dim3(tiles, s.Hkv, s.B), 256, smem, st>>>(s, c, p, static_cast<const KV*>(q), ws);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_decode_prologue(const Dims& s, const CacheDev& c, int dtype, const DecodePlan& p, const void* q,
+                                   char* ws, cudaStream_t st) {
+    if (dtype == FA_BF16) return launch_prologue_t<__nv_bfloat16>(s, c, p, q, ws, st);
+    return launch_prologue_t<float>(s, c, p, q, ws, st);
+}
+
+template <typename KV, int GH>
+static cudaError_t launch_direct_t(const Dims& s, const CacheDev& c, const DecodePlan& p, const void* q, char* ws,
+                                   cudaStream_t st) {
+    size_t smem = sizeof(float) * ((size_t)GH * s.d * 2 + (size_t)GH * s.nfk + 2 * (size_t)GH * s.M + (size_t)GH * kTile +
+                                   8 * GH + (size_t)256 * GH);
+    cudaError_t err = cudaFuncSetAttribute(decode_direct_kernel<KV, GH>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (err != cudaSuccess) return err;
+    decode_direct_kernel<KV, GH><<<dim3(p.n_split, s.Hkv * p.n_pass, s.B), 256, smem, st>>>(s, c, p, static_cast<const KV*>(q), ws);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_decode_direct(const Dims& s, const CacheDev& c, int dtype, const DecodePlan& p, const void* q, char* ws,
+                                 cudaStream_t st) {
+    if (dtype == FA_BF16) {
+        if (p.gh == 4) return launch_direct_t<__nv_bfloat16, 4>(s, c, p, q, ws, st);
+        if (p.gh == 2) return launch_direct_t<__nv_bfloat16, 2>(s, c, p, q, ws, st);
+        return launch_direct_t<__nv_bfloat16, 1>(s, c, p, q, ws, st);
+    }
+    if (p.gh == 4) return launch_direct_t<float, 4>(s, c, p, q, ws, st);
+    if (p.gh == 2) return launch_direct_t<float, 2>(s, c, p, q, ws, st);
+    return launch_direct_t<float, 1>(s, c, p, q, ws, st);
+}
+
+template <typename KV>
+static cudaError_t launch_epilogue_t(const Dims& s, const CacheDev& c, const DecodePlan& p, void* out, char* ws,
+                                     cudaStream_t st) {
+    int rows = (s.M + p.n_slice - 1) / p.n_slice;
+    size_t smem = sizeof(float) * ((size_t)s.G * p.n_split + s.G + (size_t)s.G * rows + 256 + s.d);
+    decode_epilogue_kernel<KV><<<dim3(p.n_slice, s.Hkv, s.B), 256, smem, st>>>(s, c, p, static_cast<KV*>(out), ws);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_decode_epilogue(const Dims& s, const CacheDev& c, int dtype, const DecodePlan& p, void* out, char* ws,
+                                   cudaStream_t st) {
+    if (dtype == FA_BF16) return launch_epilogue_t<__nv_bfloat16>(s, c, p, out, ws, st);
+    return launch_epilogue_t<float>(s, c, p, out, ws, st);
+}
+
+}  // namespace fa

@@ -1,0 +1,241 @@
+"""Thin ctypes binding of the C ABI in ``include/fa.h`` (same names, argument
+marshalling only: every step of the path runs in the CUDA kernels of
+``csrc/libfa.so``).  PyTorch is used for device memory and streams.
+
+There is no CPU fallback: if the library has not been built, or a call returns
+a non-zero status, this module raises.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from dataclasses import dataclass
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "csrc", "libfa.so")
+
+FA_OK, FA_ERR_INVALID_ARG, FA_ERR_UNSUPPORTED, FA_ERR_CAPACITY = 0, 1, 2, 3
+FA_ERR_WORKSPACE, FA_ERR_CUDA, FA_ERR_TIMEOUT, FA_ERR_INDEX = 4, 5, 6, 7
+FA_F32, FA_BF16 = 0, 1
+FA_NORM_ORTHO, FA_NORM_PAPER = 0, 1
+FA_DECODE_AUTO, FA_DECODE_DIRECT, FA_DECODE_FFT = 0, 1, 2
+
+
+class fa_layout(C.Structure):
+    _fields_ = [(n, C.c_int32) for n in (
+        "batch", "n_q_heads", "n_kv_heads", "head_dim", "n_full_k", "n_full_v", "n_coef", "period",
+        "l_init", "l_local", "max_mid", "mid_classes", "kv_dtype", "norm", "decode_algo")] + [("softmax_scale", C.c_float)]
+
+
+_CACHE_FIELDS = ("idx_full_k", "idx_comp_k", "idx_full_v", "idx_comp_v", "k_init", "v_init", "k_local", "v_local",
+                 "k_mid", "v_mid", "coef_k", "coef_v", "state", "status")
+
+
+class fa_cache(C.Structure):
+    _fields_ = [(n, C.c_void_p) for n in _CACHE_FIELDS]
+
+
+class fa_cache_sizes(C.Structure):
+    _fields_ = [(n, C.c_size_t) for n in _CACHE_FIELDS]
+
+
+class FaError(RuntimeError):
+    def __init__(self, status: int, what: str):
+        self.status = status
+        super().__init__(f"{what}: fa_status {status} ({status_string(status)})")
+
+
+_lib = None
+
+
+def lib() -> C.CDLL:
+    """Loads csrc/libfa.so; raises if it has not been built (no fallback)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise ImportError(
+                f"{LIB_PATH} is missing: build it with `python -m paper_2506_11886_b200.build` "
+                "(there is no CPU or PyTorch fallback for this path)")
+        L = C.CDLL(LIB_PATH)
+        vp, i32, i64, sz = C.c_void_p, C.c_int32, C.c_int64, C.c_size_t
+        lp, cp = C.POINTER(fa_layout), C.POINTER(fa_cache)
+        L.fa_cache_sizes_of.argtypes = [lp, C.POINTER(fa_cache_sizes)]
+        L.fa_workspace_bytes.argtypes = [lp, C.POINTER(sz)]
+        L.fa_cache_reset.argtypes = [lp, cp, vp]
+        L.fa_validate.argtypes = [lp, cp, vp]
+        L.fa_compress.argtypes = [lp, cp, vp, vp, i64, i64, i64, i32, vp, sz, vp]
+        L.fa_append.argtypes = [lp, cp, vp, vp, vp]
+        L.fa_decode_attention.argtypes = [lp, cp, vp, vp, vp, sz, vp]
+        L.fa_poll_status.argtypes = [cp, vp]
+        L.fa_launch_count.argtypes = [lp, C.c_int]
+        L.fa_status_string.argtypes = [C.c_int]
+        L.fa_status_string.restype = C.c_char_p
+        for name in ("fa_cache_sizes_of", "fa_workspace_bytes", "fa_cache_reset", "fa_validate", "fa_compress",
+                     "fa_append", "fa_decode_attention", "fa_poll_status", "fa_launch_count", "fa_version"):
+            getattr(L, name).restype = C.c_int
+        _lib = L
+    return _lib
+
+
+def status_string(status: int) -> str:
+    return lib().fa_status_string(int(status)).decode()
+
+
+def _check(status: int, what: str) -> None:
+    if status != FA_OK:
+        raise FaError(status, what)
+
+
+def _stream(stream) -> C.c_void_p:
+    s = torch.cuda.current_stream() if stream is None else stream
+    return C.c_void_p(s.cuda_stream)
+
+
+def _ptr(t) -> C.c_void_p:
+    return C.c_void_p(0 if t is None or t.numel() == 0 else t.data_ptr())
+
+
+@dataclass
+class Layout:
+    """Python mirror of ``fa_layout`` (field meanings: include/fa.h)."""
+    batch: int
+    n_q_heads: int
+    n_kv_heads: int
+    head_dim: int
+    n_full_k: int
+    n_full_v: int
+    n_coef: int
+    period: int
+    l_init: int
+    l_local: int
+    max_mid: int
+    mid_classes: int = 1
+    kv_dtype: int = FA_BF16
+    norm: int = FA_NORM_ORTHO
+    decode_algo: int = FA_DECODE_AUTO
+    softmax_scale: float = 1.0
+
+    def c(self) -> fa_layout:
+        return fa_layout(self.batch, self.n_q_heads, self.n_kv_heads, self.head_dim, self.n_full_k, self.n_full_v,
+                         self.n_coef, self.period, self.l_init, self.l_local, self.max_mid, self.mid_classes,
+                         self.kv_dtype, self.norm, self.decode_algo, float(self.softmax_scale))
+
+    @property
+    def torch_dtype(self) -> torch.dtype:
+        return torch.bfloat16 if self.kv_dtype == FA_BF16 else torch.float32
+
+    @property
+    def slots(self) -> int:
+        return (self.max_mid + self.mid_classes - 1) // self.mid_classes
+
+
+def fa_cache_sizes_of(layout: Layout) -> dict:
+    out = fa_cache_sizes()
+    _check(lib().fa_cache_sizes_of(C.byref(layout.c()), C.byref(out)), "fa_cache_sizes_of")
+    return {n: int(getattr(out, n)) for n in _CACHE_FIELDS}
+
+
+def fa_workspace_bytes(layout: Layout) -> int:
+    out = C.c_size_t(0)
+    _check(lib().fa_workspace_bytes(C.byref(layout.c()), C.byref(out)), "fa_workspace_bytes")
+    return int(out.value)
+
+
+class Cache:
+    """Caller-owned device buffers of one layer's cache, allocated with torch and
+    sized by ``fa_cache_sizes_of``.  Typed views: ``k_mid`` is
+    [B][H_kv][P][slots][n_full_k], ``coef_k`` is [B][H_kv][M][d - n_full_k], ..."""
+
+    def __init__(self, layout: Layout, idx_full_k: torch.Tensor, idx_full_v: torch.Tensor, device="cuda"):
+        self.layout = layout
+        self.device = torch.device(device)
+        sizes = fa_cache_sizes_of(layout)
+        L, dt = layout, layout.torch_dtype
+        B, H, d = L.batch, L.n_kv_heads, L.head_dim
+
+        def comp(idx_full):
+            rows = []
+            for h in range(H):
+                keep = torch.zeros(d, dtype=torch.bool)
+                keep[idx_full[h].long()] = True
+                rows.append(torch.nonzero(~keep).flatten().to(torch.int32))
+            return torch.stack(rows) if rows else torch.zeros((0, 0), dtype=torch.int32)
+
+        idx_full_k = idx_full_k.to(torch.int32).cpu().reshape(H, L.n_full_k)
+        idx_full_v = idx_full_v.to(torch.int32).cpu().reshape(H, L.n_full_v)
+        dev = self.device
+        self.idx_full_k = idx_full_k.contiguous().to(dev)
+        self.idx_full_v = idx_full_v.contiguous().to(dev)
+        self.idx_comp_k = comp(idx_full_k).contiguous().to(dev)
+        self.idx_comp_v = comp(idx_full_v).contiguous().to(dev)
+        z = lambda shape, dtype: torch.zeros(shape, dtype=dtype, device=dev)
+        self.k_init, self.v_init = z((B, H, L.l_init, d), dt), z((B, H, L.l_init, d), dt)
+        self.k_local, self.v_local = z((B, H, L.l_local, d), dt), z((B, H, L.l_local, d), dt)
+        self.k_mid = z((B, H, L.mid_classes, L.slots, L.n_full_k), dt)
+        self.v_mid = z((B, H, L.mid_classes, L.slots, L.n_full_v), dt)
+        self.coef_k = z((B, H, L.n_coef, d - L.n_full_k), torch.float32)
+        self.coef_v = z((B, H, L.n_coef, d - L.n_full_v), torch.float32)
+        self.state = z((B, 8), torch.int32)
+        self.status = z((4,), torch.int32)
+        for n in _CACHE_FIELDS:
+            t = getattr(self, n)
+            assert t.numel() * t.element_size() == sizes[n], (n, t.shape, sizes[n])
+        self._c = fa_cache(*[_ptr(getattr(self, n)).value for n in _CACHE_FIELDS])
+
+    def c(self) -> fa_cache:
+        return self._c
+
+    def bytes(self) -> int:
+        return sum(getattr(self, n).numel() * getattr(self, n).element_size() for n in _CACHE_FIELDS)
+
+
+def new_workspace(layout: Layout, device="cuda") -> torch.Tensor:
+    return torch.empty(max(256, fa_workspace_bytes(layout)), dtype=torch.uint8, device=device)
+
+
+def fa_cache_reset(layout: Layout, cache: Cache, stream=None) -> None:
+    _check(lib().fa_cache_reset(C.byref(layout.c()), C.byref(cache.c()), _stream(stream)), "fa_cache_reset")
+
+
+def fa_validate(layout: Layout, cache: Cache, stream=None) -> None:
+    _check(lib().fa_validate(C.byref(layout.c()), C.byref(cache.c()), _stream(stream)), "fa_validate")
+
+
+def fa_compress(layout: Layout, cache: Cache, K: torch.Tensor, V: torch.Tensor, ws: torch.Tensor, stream=None) -> None:
+    """K, V: [B][L][H_kv][d] (any strides with unit stride on d) in the layout's dtype."""
+    assert K.dtype == layout.torch_dtype and V.dtype == K.dtype and K.shape == V.shape and K.stride() == V.stride()
+    assert K.is_cuda and V.is_cuda and (K.shape[1] == 0 or K.stride(3) == 1)
+    L = K.shape[1]
+    sb, st, sh = (K.stride(0), K.stride(1), K.stride(2)) if L > 0 else (0, layout.head_dim * layout.n_kv_heads, layout.head_dim)
+    if K.shape[0] == 1:
+        sb = 0
+    _check(lib().fa_compress(C.byref(layout.c()), C.byref(cache.c()), _ptr(K), _ptr(V), sb, st, sh, L,
+                             _ptr(ws), ws.numel(), _stream(stream)), "fa_compress")
+
+
+def fa_append(layout: Layout, cache: Cache, k_new: torch.Tensor, v_new: torch.Tensor, stream=None) -> None:
+    """k_new, v_new: contiguous [B][H_kv][d]."""
+    assert k_new.is_contiguous() and v_new.is_contiguous() and k_new.dtype == layout.torch_dtype and k_new.is_cuda
+    _check(lib().fa_append(C.byref(layout.c()), C.byref(cache.c()), _ptr(k_new), _ptr(v_new), _stream(stream)), "fa_append")
+
+
+def fa_decode_attention(layout: Layout, cache: Cache, q: torch.Tensor, out: torch.Tensor, ws: torch.Tensor, stream=None) -> None:
+    """q, out: contiguous [B][H_q][d]."""
+    assert q.is_contiguous() and out.is_contiguous() and q.dtype == layout.torch_dtype and out.dtype == q.dtype
+    assert q.is_cuda and out.is_cuda
+    _check(lib().fa_decode_attention(C.byref(layout.c()), C.byref(cache.c()), _ptr(q), _ptr(out), _ptr(ws), ws.numel(),
+                                     _stream(stream)), "fa_decode_attention")
+
+
+def fa_poll_status(cache: Cache, stream=None) -> int:
+    return int(lib().fa_poll_status(C.byref(cache.c()), _stream(stream)))
+
+
+def fa_launch_count(layout: Layout, what: int) -> int:
+    return int(lib().fa_launch_count(C.byref(layout.c()), int(what)))
+
+
+def fa_version() -> int:
+    return int(lib().fa_version())

@@ -1,0 +1,80 @@
+"""The C-ABI library loads on a machine without a GPU and exports every symbol
+that include/fa.h declares; host-only entry points behave (no compute calls)."""
+import ctypes as C
+import os
+import re
+
+import pytest
+
+from paper_2506_11886_b200 import build, fa
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _built():
+    build.build_library()
+
+
+def _declared():
+    text = open(os.path.join(ROOT, "include", "fa.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(fa_[a-z_0-9]+)\s*\(", text)))
+
+
+def test_every_declared_symbol_is_exported():
+    names = _declared()
+    assert {"fa_compress", "fa_append", "fa_decode_attention"} <= set(names)
+    lib = fa.lib()
+    for n in names:
+        assert hasattr(lib, n), n
+
+
+def test_binding_mirrors_the_struct_layouts():
+    assert C.sizeof(fa.fa_layout) == 16 * 4
+    assert C.sizeof(fa.fa_cache) == 14 * C.sizeof(C.c_void_p)
+    assert fa.fa_version() >= 100
+
+
+def _layout(**kw):
+    base = dict(batch=1, n_q_heads=32, n_kv_heads=8, head_dim=128, n_full_k=32, n_full_v=32, n_coef=1024,
+                period=32768, l_init=4, l_local=1024, max_mid=32768, mid_classes=64)
+    base.update(kw)
+    return fa.Layout(**base)
+
+
+def test_cache_sizes_of_the_32k_configuration():
+    sz = fa.fa_cache_sizes_of(_layout())
+    assert sz["k_mid"] == 8 * 32768 * 32 * 2 and sz["v_mid"] == sz["k_mid"]
+    assert sz["coef_k"] == 8 * 1024 * 96 * 4
+    assert sz["k_local"] == 8 * 1024 * 128 * 2 and sz["k_init"] == 8 * 4 * 128 * 2
+    assert sz["idx_full_k"] == 8 * 32 * 4 and sz["idx_comp_v"] == 8 * 96 * 4
+    assert fa.fa_workspace_bytes(_layout()) > 0
+
+
+@pytest.mark.parametrize("kw,status", [
+    (dict(n_kv_heads=5), fa.FA_ERR_INVALID_ARG),
+    (dict(n_coef=1023), fa.FA_ERR_INVALID_ARG),
+    (dict(n_coef=65538, period=65536), fa.FA_ERR_INVALID_ARG),
+    (dict(max_mid=40000), fa.FA_ERR_INVALID_ARG),
+    (dict(mid_classes=0), fa.FA_ERR_INVALID_ARG),
+    (dict(softmax_scale=0.0), fa.FA_ERR_INVALID_ARG),
+    (dict(kv_dtype=7), fa.FA_ERR_INVALID_ARG),
+    (dict(n_full_k=33), fa.FA_ERR_UNSUPPORTED),
+    (dict(head_dim=512, n_full_k=32), fa.FA_ERR_UNSUPPORTED),
+    (dict(n_q_heads=8 * 32), fa.FA_ERR_UNSUPPORTED),
+])
+def test_bad_layouts_are_refused_on_the_host(kw, status):
+    with pytest.raises(fa.FaError) as e:
+        fa.fa_cache_sizes_of(_layout(**kw))
+    assert e.value.status == status
+    assert fa.status_string(status)
+
+
+def test_null_arguments():
+    lib = fa.lib()
+    assert lib.fa_cache_sizes_of(None, None) == fa.FA_ERR_INVALID_ARG
+    assert lib.fa_poll_status(None, None) == fa.FA_ERR_INVALID_ARG
+    lay = _layout().c()
+    assert lib.fa_decode_attention(C.byref(lay), None, None, None, None, 0, None) == fa.FA_ERR_INVALID_ARG
+    assert lib.fa_append(C.byref(lay), None, None, None, None) == fa.FA_ERR_INVALID_ARG

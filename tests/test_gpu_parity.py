@@ -1,0 +1,194 @@
+"""Parity of the CUDA path (through the C ABI) against the fp64 oracle on the
+same seeded inputs: cache metadata and stored rows bit-exact, coefficients and
+attention outputs within the stated tolerances.  Small and medium sizes that
+still span several tiles, classes and a ragged tail, plus the edge cases."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2506_11886_b200 import fa, synth
+from tests.parity_util import Pair, layout_of, make_pair, to64
+
+pytestmark = pytest.mark.gpu
+
+CFG0 = synth.CONFIGS[0]
+SMALL_BF16 = synth.Shape("small_bf16_gqa", B=2, layers=1, Hq=8, Hkv=2, d=128, L=1500, dtype="bf16", n_full_k=32,
+                         n_full_v=48, M=128, T=2048, L_init=4, L_local=64, decode_steps=40)
+ALGOS = [fa.FA_DECODE_DIRECT]
+
+
+@pytest.mark.parametrize("P", [1, 32])
+@pytest.mark.parametrize("algo", ALGOS)
+def test_cfg0_toy_compress_then_decode(P, algo):
+    """Configuration 0: fp32, GQA 4, L = 1024, 32 kept / 96 compressed dims, M = 64."""
+    pair, _ = make_pair(CFG0, seed=0, P=P, algo=algo)
+    pair.check_state()
+    for step in range(3):
+        pair.check_decode(synth.queries(CFG0, seed=0, step=step))
+    pair.check_decode(synth.queries(CFG0, seed=0, step=9, peak=8.0))      # peaked softmax
+
+
+@pytest.mark.parametrize("algo", ALGOS)
+def test_cfg0_with_windows_and_offgrid_frequencies(algo):
+    shape = CFG0.with_(L_init=4, L_local=64)
+    pair, _ = make_pair(shape, seed=1, algo=algo, freq="offgrid")
+    pair.check_state()
+    pair.check_decode(synth.queries(shape, seed=1))
+
+
+@pytest.mark.parametrize("algo", ALGOS)
+@pytest.mark.parametrize("P", [1, 32])
+def test_bf16_gqa_append_and_decode(algo, P):
+    """bf16, 2 batch rows, GQA 4, asymmetric K/V index sets, ragged classes; appends wrap the ring."""
+    shape = SMALL_BF16
+    pair, stream = make_pair(shape, seed=2, algo=algo, P=P, max_mid=2048)
+    pair.check_state()
+    pair.check_decode(synth.queries(shape, seed=2))
+    t = shape.L
+    for step in range(70):                       # more than l_local appends: the ring wraps
+        k_new, v_new = stream.tokens(t, t + 1)
+        pair.append(k_new[:, 0], v_new[:, 0])
+        t += 1
+        if step in (0, 1, 63, 64, 69):
+            pair.check_state()
+            pair.check_decode(synth.queries(shape, seed=2, step=step + 1))
+
+
+@pytest.mark.parametrize("algo", ALGOS)
+def test_append_from_empty_equals_compress(algo):
+    """Tokens fill init, then local, then spill into the middle; compare with one compress call."""
+    shape = SMALL_BF16.with_(B=1, Hq=2, Hkv=1, L=0, L_init=3, L_local=8, T=256, M=32, n_full_k=16, n_full_v=8)
+    layout = layout_of(shape, max_mid=256, P=8, algo=algo)
+    stream = synth.KVStream(shape, seed=3)
+    pair = Pair(layout, stream.idx_full_k, stream.idx_full_v)
+    fa.fa_cache_reset(layout, pair.gpu)
+    K0, V0 = stream.tokens(0, 0)
+    pair.ref.compress(to64(K0), to64(V0))
+    K, V = stream.tokens(0, 40)
+    for t in range(40):
+        pair.append(K[:, t], V[:, t])
+        if t in (0, 2, 3, 10, 11, 39):
+            pair.check_state()
+            pair.check_decode(synth.queries(shape, seed=3, step=t))
+    again = Pair(layout, stream.idx_full_k, stream.idx_full_v)
+    again.compress(K, V)
+    for name in ("k_init", "v_init", "k_mid", "v_mid"):
+        assert torch.equal(getattr(again.gpu, name), getattr(pair.gpu, name)), name
+    den = again.gpu.coef_k.abs().max()
+    assert (again.gpu.coef_k - pair.gpu.coef_k).abs().max() / den < 1e-4
+    assert torch.equal(again.gpu.state[:, :3], pair.gpu.state[:, :3])
+
+
+@pytest.mark.parametrize("algo", ALGOS)
+@pytest.mark.parametrize("nfk,nfv", [(0, 0), (128, 128), (128, 32), (8, 120)])
+def test_degenerate_index_sets(algo, nfk, nfv):
+    """Everything compressed, nothing compressed (plain attention), and mixed extremes."""
+    shape = SMALL_BF16.with_(B=1, Hq=4, Hkv=2, L=700, n_full_k=nfk, n_full_v=nfv, T=1024, M=64)
+    pair, stream = make_pair(shape, seed=4, algo=algo, P=32, max_mid=1024)
+    pair.check_state()
+    pair.check_decode(synth.queries(shape, seed=4))
+    k_new, v_new = stream.tokens(shape.L, shape.L + 1)
+    pair.append(k_new[:, 0], v_new[:, 0])
+    pair.check_state()
+    pair.check_decode(synth.queries(shape, seed=4, step=1))
+
+
+@pytest.mark.parametrize("algo", ALGOS)
+@pytest.mark.parametrize("L", [0, 1, 3, 4, 5, 67, 68, 69, 100])
+def test_short_prompts(algo, L):
+    """Prompts shorter than the windows, and the first few middle tokens."""
+    shape = SMALL_BF16.with_(B=2, L=L, T=512, M=32)
+    pair, _ = make_pair(shape, seed=5, L=L, algo=algo, P=16, max_mid=512)
+    pair.check_state()
+    got, want = pair.decode(synth.queries(shape, seed=5))
+    if L == 0:
+        assert not got.any() and not want.any()
+    else:
+        assert np.abs(got - want).max() < 2e-2
+
+
+@pytest.mark.parametrize("algo", ALGOS)
+def test_no_local_window_and_odd_period(algo):
+    """l_local = 0 (appended tokens go straight to the middle), period not a power of two, G = 1, fp32."""
+    shape = synth.Shape("odd", B=1, layers=1, Hq=2, Hkv=2, d=64, L=300, dtype="f32", n_full_k=16, n_full_v=24, M=50,
+                        T=777, L_init=2, L_local=0)
+    pair, stream = make_pair(shape, seed=6, algo=fa.FA_DECODE_DIRECT, P=7, max_mid=777)
+    pair.check_state()
+    pair.check_decode(synth.queries(shape, seed=6))
+    K, V = stream.tokens(300, 310)
+    for t in range(10):
+        pair.append(K[:, t], V[:, t])
+    pair.check_state()
+    pair.check_decode(synth.queries(shape, seed=6, step=1))
+
+
+def test_paper_literal_scale():
+    shape = CFG0.with_(L_init=4, L_local=64)
+    pair, _ = make_pair(shape, seed=7, norm=fa.FA_NORM_PAPER)
+    pair.check_decode(synth.queries(shape, seed=7))
+
+
+def test_strided_prefill_input():
+    """K, V given as slices of a larger [B][L][H][2d] buffer."""
+    shape = SMALL_BF16.with_(B=2, L=300, T=512, M=32)
+    layout = layout_of(shape, max_mid=512, P=16)
+    stream = synth.KVStream(shape, seed=8)
+    K, V = stream.tokens(0, 300)
+    big = torch.zeros((2, 300, shape.Hkv, 2, 2 * shape.d), dtype=K.dtype, device="cuda")
+    big[:, :, :, 0, :shape.d] = K.cuda()
+    big[:, :, :, 1, :shape.d] = V.cuda()
+    pair = Pair(layout, stream.idx_full_k, stream.idx_full_v)
+    fa.fa_compress(layout, pair.gpu, big[:, :, :, 0, :shape.d], big[:, :, :, 1, :shape.d], pair.ws)
+    pair.ref.compress(to64(K), to64(V))
+    pair.check_state()
+
+
+def test_errors_are_reported_not_raised_on_device():
+    shape = SMALL_BF16.with_(B=1, Hq=2, Hkv=1, L=80, T=128, M=16)
+    layout = layout_of(shape, max_mid=10, P=4)
+    stream = synth.KVStream(shape, seed=9)
+    pair = Pair(layout, stream.idx_full_k, stream.idx_full_v)
+    K, V = stream.tokens(0, 80)
+    with pytest.raises(fa.FaError) as e:                      # 80 - 4 - 64 = 12 middle tokens > 10
+        fa.fa_compress(layout, pair.gpu, K.cuda(), V.cuda(), pair.ws)
+    assert e.value.status == fa.FA_ERR_CAPACITY
+    pair.compress(K[:, :78], V[:, :78])                       # exactly full
+    pair.check_state()
+    before = {n: getattr(pair.gpu, n).clone() for n in ("coef_k", "coef_v", "k_mid", "k_local", "state")}
+    fa.fa_append(layout, pair.gpu, K[:, 79].cuda().contiguous(), V[:, 79].cuda().contiguous())
+    assert fa.fa_poll_status(pair.gpu) == fa.FA_ERR_CAPACITY   # reported through the status word
+    assert fa.fa_poll_status(pair.gpu) == fa.FA_OK             # and cleared by the poll
+    for n, t in before.items():
+        assert torch.equal(getattr(pair.gpu, n), t), n         # the refused append changed nothing
+    # workspace too small / missing
+    q = synth.queries(shape, seed=9).cuda()
+    out = torch.empty_like(q)
+    with pytest.raises(fa.FaError) as e:
+        fa.fa_decode_attention(layout, pair.gpu, q, out, pair.ws[:64])
+    assert e.value.status == fa.FA_ERR_WORKSPACE
+    # broken index sets are caught by fa_validate
+    bad = stream.idx_full_k.clone()
+    bad[0, 0], bad[0, 1] = bad[0, 1].item(), bad[0, 0].item()
+    c2 = fa.Cache(layout, stream.idx_full_k, stream.idx_full_v)
+    c2.idx_full_k.copy_(bad.cuda())
+    with pytest.raises(fa.FaError) as e:
+        fa.fa_validate(layout, c2)
+    assert e.value.status == fa.FA_ERR_INDEX
+
+
+def test_snapshot_restore():
+    """The cache is plain caller-owned memory: copying it back restores the outputs."""
+    shape = SMALL_BF16.with_(B=1, L=400, T=512, M=32)
+    pair, stream = make_pair(shape, seed=10, P=16, max_mid=512)
+    q = synth.queries(shape, seed=10).cuda()
+    out0, out1 = torch.empty_like(q), torch.empty_like(q)
+    fa.fa_decode_attention(pair.layout, pair.gpu, q, out0, pair.ws)
+    names = ("k_init", "v_init", "k_local", "v_local", "k_mid", "v_mid", "coef_k", "coef_v", "state")
+    snap = {n: getattr(pair.gpu, n).clone() for n in names}
+    K, V = stream.tokens(400, 416)
+    for t in range(16):
+        fa.fa_append(pair.layout, pair.gpu, K[:, t].cuda().contiguous(), V[:, t].cuda().contiguous())
+    for n in names:
+        getattr(pair.gpu, n).copy_(snap[n])
+    fa.fa_decode_attention(pair.layout, pair.gpu, q, out1, pair.ws)
+    assert torch.equal(out0, out1)
