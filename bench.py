@@ -1,0 +1,347 @@
+#!/usr/bin/env python
+"""Benchmark of the hybrid-KV decode path on B200.
+
+Workload (N = 1): the LLaMA-3.1-8B-shaped single-layer decode at 32K context
+(batch 1, 32 query / 8 KV heads, head_dim 128, bf16; per KV head 32 dims kept
+per token, 96 dims held as M = 1024 Fourier coefficients; 4 sink + 1024 recent
+tokens kept whole).  One STEP = one decode step of the whole hot path on a
+resident cache: fa_append (ring push + Eq.5 coefficient update of the token
+that leaves the local window) followed by fa_decode_attention (Eq.6).  The
+cache of one layer (43 MB) would fit the 126 MB L2, so the steps rotate over
+`--instances` independent caches (>= 8, > L2 in total).
+
+Printed JSON (one line, rank 0): metric / value = microseconds per step,
+device-timed with CUDA events around a CUDA-graph replay of exactly K steps;
+`e2e` = the same through fa_decode_step_host with pinned HOST q / k_new /
+v_new / out; `roofline` = fa_decode_attention alone (its three kernels) against
+the measured HBM peak on the bytes the hybrid cache holds; `cpu_baseline` = the
+fp64 oracle on the host cores on a stated sample.  `--impl reference` times the
+oracle instead.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "decode_attn_us_per_step_32k"
+UNIT = "us/step"
+SEED = 1000          # 1000 * config index
+# dram__bytes_read.sum + dram__bytes_write.sum per fa_decode_attention call from the committed
+# ncu capture (profiles/); None until a capture of the current kernels has been summarised.
+NCU_TRAFFIC_BYTES_PER_CALL = None
+
+
+def _peaks():
+    try:
+        with open(os.path.join(ROOT, "MEASURED_PEAKS.json")) as f:
+            p = json.load(f)
+        return float(p["hbm_gbs"]), "measured"
+    except Exception:
+        return 6650.0, "fallback"
+
+
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons while a region runs."""
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.rows, self.proc = index, [], None
+
+    def __enter__(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                                          "-lms", "50", "-i", str(self.index)], stdout=subprocess.PIPE, text=True)
+            self.thr = threading.Thread(target=self._read, daemon=True)
+            self.thr.start()
+        except Exception:
+            self.proc = None
+        return self
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([x.strip() for x in line.split(",")])
+
+    def __exit__(self, *a):
+        if self.proc:
+            self.proc.terminate()
+            try:
+                self.proc.wait(timeout=5)
+            except Exception:
+                pass
+
+    def summary(self):
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in self.rows:
+            try:
+                sm.append(float(r[0])); mx.append(float(r[1]))
+                for n, v in zip(names, r[3:7]):
+                    if v.lower().startswith("active"):
+                        reasons.add(n)
+            except Exception:
+                continue
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+def algorithmic_bytes(shape, n_mid: int, n_win: int) -> dict:
+    """Bytes the hybrid cache holds and one decode / append call must move (per layer)."""
+    eb = 2 if shape.dtype == "bf16" else 4
+    d, M = shape.d, shape.M
+    dck, dcv = d - shape.n_full_k, d - shape.n_full_v
+    per_head = n_mid * (shape.n_full_k + shape.n_full_v) * eb + n_win * 2 * d * eb + M * (dck + dcv) * 4 + 2 * shape.G * d * eb
+    append_head = 2 * M * (dck + dcv) * 4 + 4 * d * eb
+    return {"decode": shape.B * shape.Hkv * per_head, "append": shape.B * shape.Hkv * append_head}
+
+
+# ----------------------------------------------------------------- oracle arm
+def oracle_sample_time(shape, seed: int, n_heads: int, L: int, repeats: int = 1):
+    """Builds an oracle cache for the first n_heads KV heads and the first L tokens of the
+    workload and times one step (append + decode) on it.  Returns (seconds per step, threads)."""
+    import numpy as np
+    from oracle import fa_oracle as fo
+    from paper_2506_11886_b200 import synth
+    sub = shape.with_(Hkv=n_heads, Hq=n_heads * shape.G, L=L)
+    stream = synth.KVStream(sub, seed=seed)
+    K, V = stream.tokens(0, L + repeats + 1)
+    cfg = fo.OracleConfig(B=sub.B, Hq=sub.Hq, Hkv=sub.Hkv, d=sub.d, n_full_k=sub.n_full_k, n_full_v=sub.n_full_v,
+                          k=sub.k, T=sub.T, L_init=sub.L_init, L_local=sub.L_local, cap_mid=sub.T, scale=sub.softmax_scale)
+    cache = fo.OracleCache(cfg, stream.idx_full_k.numpy(), stream.idx_full_v.numpy())
+    Kd, Vd = K.to(dtype=__import__("torch").float64).numpy(), V.to(dtype=__import__("torch").float64).numpy()
+    cache.compress(Kd[:, :L], Vd[:, :L])
+    times = []
+    for r in range(repeats):
+        q = synth.queries(sub, seed=seed, step=r).to(dtype=__import__("torch").float64).numpy()
+        t0 = time.perf_counter()
+        cache.append(Kd[:, L + r], Vd[:, L + r])
+        out = cache.decode(q)
+        times.append(time.perf_counter() - t0)
+        assert np.isfinite(out).all()
+    return times, fo.num_threads()
+
+
+def run_reference(args):
+    """The reference arm: the fp64 oracle, as it stands, on the host cores."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from oracle import fa_oracle as fo
+    from paper_2506_11886_b200 import synth
+    fo.build()
+    shape = synth.CONFIGS[1]
+    total = args.steps + args.warmup
+    # bounded sample: one KV head, context truncated so that the whole run stays within ~2.5 minutes
+    calib, threads = oracle_sample_time(shape, SEED, 1, 2048 + shape.L_init + shape.L_local, repeats=1)
+    per_token = calib[0] / 2048.0
+    budget = 150.0 / max(1, total)
+    L_mid_full = shape.L - shape.L_init - shape.L_local
+    n_mid = int(max(256, min(L_mid_full, budget / max(per_token, 1e-9))))
+    L = n_mid + shape.L_init + shape.L_local
+    times, threads = oracle_sample_time(shape, SEED, 1, L, repeats=total)
+    timed = times[args.warmup:]
+    scale = shape.Hkv * (L_mid_full / n_mid)
+    sec = sum(timed) / len(timed)
+    us = sec * scale * 1e6
+    sample = f"1 of {shape.Hkv} KV heads, first {L} of {shape.L} tokens per step, time scaled x{scale:.1f}"
+    line = {"metric": METRIC, "value": us, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup,
+            "ms_per_step": us / 1e3, "higher_is_better": False, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
+            "data": "synthetic", "impl": "reference",
+            "config": {"workload": shape.name, "global_batch": shape.B, "seq_len": shape.L, "sample": sample},
+            "cpu_baseline": {"value": us, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": sample},
+            "e2e": {"value": us, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line), flush=True)
+
+
+# -------------------------------------------------------------------- our arm
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+    from paper_2506_11886_b200 import build, fa, synth
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    if not os.path.exists(fa.LIB_PATH):
+        if rank == 0:
+            build.build_library()
+        if world > 1:
+            dist.barrier()
+    dev = torch.device("cuda", local)
+    shape = synth.CONFIGS[1]
+    K_steps, W = args.steps, max(args.warmup, 3)
+    n_inst = max(args.instances, 2)
+    layout = fa.Layout(batch=shape.B, n_q_heads=shape.Hq, n_kv_heads=shape.Hkv, head_dim=shape.d, n_full_k=shape.n_full_k,
+                       n_full_v=shape.n_full_v, n_coef=shape.M, period=shape.T, l_init=shape.L_init, l_local=shape.L_local,
+                       max_mid=shape.T, mid_classes=shape.T // shape.k, kv_dtype=fa.FA_BF16, softmax_scale=shape.softmax_scale)
+    stream = synth.KVStream(shape, seed=SEED, device=str(dev))
+    Kp, Vp = stream.tokens(0, shape.L, work_dtype=torch.float32)
+    ws = fa.new_workspace(layout, device=dev)
+    caches = []
+    t0 = time.perf_counter()
+    for i in range(n_inst):
+        c = fa.Cache(layout, stream.idx_full_k, stream.idx_full_v, device=dev)
+        if i == 0:
+            fa.fa_validate(layout, c)
+        fa.fa_compress(layout, c, Kp, Vp, ws)
+        caches.append(c)
+    torch.cuda.synchronize()
+    # compress timing (one layer of the 32-layer prefill-compression configuration has this exact shape)
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    comp_ms = []
+    for _ in range(3):
+        ev0.record(); fa.fa_compress(layout, caches[-1], Kp, Vp, ws); ev1.record(); torch.cuda.synchronize()
+        comp_ms.append(ev0.elapsed_time(ev1))
+    n_mid0 = shape.L - shape.L_init - shape.L_local
+    comp_flop = 2.0 * shape.M * n_mid0 * ((shape.d - shape.n_full_k) + (shape.d - shape.n_full_v)) * shape.Hkv * shape.B
+    del Kp, Vp
+    # per-step inputs: visit r of an instance appends token L + r
+    regions = 4
+    visits = (W + K_steps + n_inst - 1) // n_inst * regions + 4
+    assert n_mid0 + visits <= layout.max_mid, "too many steps for the period of this configuration"
+    Kn, Vn = stream.tokens(shape.L, shape.L + visits, work_dtype=torch.float32)      # [B][visits][Hkv][d]
+    Kn, Vn = Kn.transpose(0, 1).contiguous(), Vn.transpose(0, 1).contiguous()          # [visits][B][Hkv][d]
+    n_q = W + K_steps
+    qs = torch.stack([synth.queries(shape, seed=SEED, step=s, device=str(dev)) for s in range(min(n_q, 64))])
+    outs = torch.empty((n_q,) + tuple(qs.shape[1:]), dtype=qs.dtype, device=dev)
+    visit = [0] * n_inst
+
+    def step(s, do_append=True, do_decode=True):
+        i = s % n_inst
+        if do_append:
+            fa.fa_append(layout, caches[i], Kn[visit[i]], Vn[visit[i]])
+            visit[i] += 1
+        if do_decode:
+            fa.fa_decode_attention(layout, caches[i], qs[s % qs.shape[0]], outs[s], ws)
+
+    def barrier():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+            torch.cuda.synchronize()
+
+    def timed_graph(body, n_warm, n_steps):
+        """Captures n_warm and n_steps steps as two CUDA graphs, replays the first untimed and the
+        second between CUDA events on the launching stream.  Returns milliseconds for n_steps steps."""
+        for s in range(2):
+            body(s)                                   # eager: sets kernel attributes before any capture
+        torch.cuda.synchronize()
+        g_warm, g_time = torch.cuda.CUDAGraph(), torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g_warm):
+            for s in range(n_warm):
+                body(s)
+        with torch.cuda.graph(g_time):
+            for s in range(n_warm, n_warm + n_steps):
+                body(s)
+        g_warm.replay()
+        barrier()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        g_time.replay()
+        e1.record()
+        barrier()
+        ms = e0.elapsed_time(e1)
+        if world > 1:
+            t = torch.tensor([ms], device=dev)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            ms = float(t.item())
+        return ms
+
+    with ClockSampler(local) as clk:
+        ms_step = timed_graph(lambda s: step(s), W, K_steps)
+        ms_decode = timed_graph(lambda s: step(s, do_append=False), W, K_steps)
+        ms_append = timed_graph(lambda s: step(s, do_decode=False), W, K_steps)
+        # end to end: host q / k_new / v_new in, host out, through the host-buffer C-ABI call
+        staging = torch.empty(fa.fa_step_staging_bytes(layout), dtype=torch.uint8, device=dev)
+        q_h = qs.cpu().pin_memory()
+        out_h = torch.empty((n_q,) + tuple(qs.shape[1:]), dtype=qs.dtype).pin_memory()
+        Kn_h, Vn_h = Kn.cpu().pin_memory(), Vn.cpu().pin_memory()
+
+        def e2e_step(s):
+            i = s % n_inst
+            fa.fa_decode_step_host(layout, caches[i], q_h[s % q_h.shape[0]], Kn_h[visit[i]], Vn_h[visit[i]], out_h[s], staging, ws)
+            visit[i] += 1
+        ms_e2e = timed_graph(e2e_step, W, K_steps)
+        time.sleep(0.2)
+    clocks = clk.summary()
+    for c in caches:
+        st = fa.fa_poll_status(c)
+        assert st == fa.FA_OK, fa.status_string(st)
+    assert torch.isfinite(outs[W:].float()).all() and torch.isfinite(out_h[W:].float()).all()
+
+    us_step = ms_step * 1e3 / K_steps
+    us_decode = ms_decode * 1e3 / K_steps
+    us_append = ms_append * 1e3 / K_steps
+    us_e2e = ms_e2e * 1e3 / K_steps
+    n_mid_now = int(caches[0].state[0, 2].item())
+    by = algorithmic_bytes(shape, n_mid0, shape.L_init + shape.L_local)
+    peak, peak_kind = _peaks()
+    dec_gbs = by["decode"] / (us_decode * 1e-6) / 1e9
+    eb = 2
+    q_bytes = shape.B * shape.Hq * shape.d * eb
+    kv_bytes = shape.B * shape.Hkv * shape.d * eb
+    launches = K_steps * (fa.fa_launch_count(layout, 1) + fa.fa_launch_count(layout, 2))
+    line = {
+        "metric": METRIC, "value": us_step / world, "unit": UNIT, "n_gpus": world, "steps": K_steps, "warmup": W,
+        "ms_per_step": us_step / 1e3, "higher_is_better": False, "scaling": "weak", "vs_baseline": None,
+        "dtype": "bf16 storage, f32 arithmetic", "data": "synthetic",
+        "config": {"workload": shape.name, "global_batch": shape.B * world, "seq_len": shape.L,
+                   "step": "fa_append + fa_decode_attention, one layer", "parallelism": f"replicas x{world}",
+                   "l2": f"inputs larger than L2: {n_inst} cache instances x {by['decode'] / 1e6:.1f} MB rotated",
+                   "timing": "CUDA events around one CUDA-graph replay of K steps", "n_mid_end": n_mid_now},
+        "breakdown": {"decode_us": us_decode, "append_us": us_append, "tokens_per_s": 1e6 / us_step * shape.B * world,
+                      "append_gbs": by["append"] / (us_append * 1e-6) / 1e9,
+                      "compress_ms_per_layer": min(comp_ms), "compress_tflops": comp_flop / (min(comp_ms) * 1e-3) / 1e12,
+                      "compress_path": "cuda-core fp32"},
+        "roofline": {"kernel": "fa_decode_attention (prologue + main + epilogue kernels)", "bound": "hbm",
+                     "achieved": dec_gbs, "peak": peak, "unit": "GB/s", "frac": dec_gbs / peak, "peak_kind": peak_kind,
+                     "algorithmic_bytes": by["decode"], "traffic": NCU_TRAFFIC_BYTES_PER_CALL,
+                     "frac_of_8tbs_nominal": dec_gbs / 8000.0},
+        "e2e": {"value": us_e2e / world, "unit": UNIT, "h2d_bytes_per_step": q_bytes + 2 * kv_bytes, "d2h_bytes_per_step": q_bytes},
+        "gpu_launches": launches, "clocks": clocks,
+    }
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        from oracle import fa_oracle as fo
+        fo.build()
+        L_s = 8192
+        times, threads = oracle_sample_time(shape, SEED, 1, L_s, repeats=1)
+        scale = shape.Hkv * (n_mid0 / (L_s - shape.L_init - shape.L_local))
+        line["cpu_baseline"] = {"value": times[0] * scale * 1e6, "unit": UNIT, "cores": threads, "kind": "oracle",
+                                "sample": f"1 of {shape.Hkv} KV heads, first {L_s} of {shape.L} tokens, one step, time scaled x{scale:.1f}"}
+    if rank == 0:
+        print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=400)
+    ap.add_argument("--warmup", type=int, default=8)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--instances", type=int, default=8)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -18,7 +18,7 @@
  * Conventions for every call
  *   - All buffers are caller-owned DEVICE memory on the current device unless
  *     a parameter says "host".  The library allocates nothing, keeps no
- *     mutable global state and runs every kernel on the stream passed in
+ *     state on the device besides the caller's buffers and runs every kernel on the stream passed in
  *     (a cudaStream_t handed over as void*; NULL is the default stream).
  *   - Calls are asynchronous.  Argument errors are found on the host before
  *     anything is launched and returned as fa_status.  Conditions only the
@@ -148,6 +148,17 @@ fa_status fa_append(const fa_layout* layout, fa_cache* cache, const void* k_new,
  * (p^T Phi) W C^V for the outputs.  Does not modify the cache.  An empty cache gives zeros. */
 fa_status fa_decode_attention(const fa_layout* layout, const fa_cache* cache, const void* q, void* out,
                               void* ws, size_t ws_bytes, void* stream);
+
+/* One decode step with HOST inputs and outputs (Eq.5 then Eq.6): copies q [B][H_q][d] and
+ * k_new, v_new [B][H_kv][d] from host memory (pinned for the copies to be asynchronous) into
+ * `staging`, runs fa_append and fa_decode_attention, and copies the result to out_host
+ * [B][H_q][d].  `staging` is caller-owned device memory of at least
+ * fa_step_staging_bytes(layout) bytes; k_new_host == NULL skips the append.  Asynchronous on
+ * `stream`: out_host is valid after the stream is synchronised. */
+fa_status fa_decode_step_host(const fa_layout* layout, fa_cache* cache, const void* q_host,
+                              const void* k_new_host, const void* v_new_host, void* out_host,
+                              void* staging, void* ws, size_t ws_bytes, void* stream);
+size_t fa_step_staging_bytes(const fa_layout* layout);
 
 /* Synchronises the stream and returns (then clears) the sticky device status word. */
 fa_status fa_poll_status(const fa_cache* cache, void* stream);

@@ -32,6 +32,26 @@ fa_status check_layout(const fa_layout* l) {
     return FA_OK;
 }
 
+// (kernel, device) -> largest dynamic shared memory size granted so far.
+cudaError_t ensure_dynamic_smem_impl(const void* kernel, size_t bytes) {
+    struct Entry { const void* fn; int dev; size_t bytes; };
+    static Entry table[256];
+    static int used = 0;
+    if (bytes <= 48 * 1024) return cudaSuccess;
+    int dev = 0;
+    cudaError_t err = cudaGetDevice(&dev);
+    if (err != cudaSuccess) return err;
+    Entry* hit = nullptr;
+    for (int i = 0; i < used; ++i)
+        if (table[i].fn == kernel && table[i].dev == dev) { hit = &table[i]; break; }
+    if (hit && bytes <= hit->bytes) return cudaSuccess;
+    err = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes);
+    if (err != cudaSuccess) return err;
+    if (hit) hit->bytes = bytes;
+    else if (used < 256) table[used++] = Entry{kernel, dev, bytes};
+    return cudaSuccess;
+}
+
 static int ilog2_exact(int v) {
     int l = 0;
     while ((1 << l) < v) ++l;
@@ -231,6 +251,41 @@ fa_status fa_decode_attention(const fa_layout* layout, const fa_cache* cache, co
     if (launch_decode_prologue(s, c, layout->kv_dtype, p, q, w, cs) != cudaSuccess) return FA_ERR_CUDA;
     if (launch_decode_direct(s, c, layout->kv_dtype, p, q, w, cs) != cudaSuccess) return FA_ERR_CUDA;
     if (launch_decode_epilogue(s, c, layout->kv_dtype, p, out, w, cs) != cudaSuccess) return FA_ERR_CUDA;
+    return FA_OK;
+}
+
+size_t fa_step_staging_bytes(const fa_layout* layout) {
+    if (check_layout(layout) != FA_OK) return 0;
+    size_t eb = elt_bytes(layout->kv_dtype);
+    size_t qb = align_up((size_t)layout->batch * layout->n_q_heads * layout->head_dim * eb, 256);
+    size_t kb = align_up((size_t)layout->batch * layout->n_kv_heads * layout->head_dim * eb, 256);
+    return 2 * qb + 2 * kb;
+}
+
+fa_status fa_decode_step_host(const fa_layout* layout, fa_cache* cache, const void* q_host, const void* k_new_host,
+                              const void* v_new_host, void* out_host, void* staging, void* ws, size_t ws_bytes,
+                              void* stream) {
+    fa_status st = check_layout(layout);
+    if (st != FA_OK) return st;
+    if (!q_host || !out_host || !staging || !aligned16(staging)) return FA_ERR_INVALID_ARG;
+    if ((k_new_host == nullptr) != (v_new_host == nullptr)) return FA_ERR_INVALID_ARG;
+    size_t eb = elt_bytes(layout->kv_dtype);
+    size_t q_bytes = (size_t)layout->batch * layout->n_q_heads * layout->head_dim * eb;
+    size_t k_bytes = (size_t)layout->batch * layout->n_kv_heads * layout->head_dim * eb;
+    size_t qb = align_up(q_bytes, 256), kb = align_up(k_bytes, 256);
+    char* base = static_cast<char*>(staging);
+    char *q_d = base, *o_d = base + qb, *k_d = base + 2 * qb, *v_d = base + 2 * qb + kb;
+    cudaStream_t cs = static_cast<cudaStream_t>(stream);
+    if (cudaMemcpyAsync(q_d, q_host, q_bytes, cudaMemcpyHostToDevice, cs) != cudaSuccess) return FA_ERR_CUDA;
+    if (k_new_host) {
+        if (cudaMemcpyAsync(k_d, k_new_host, k_bytes, cudaMemcpyHostToDevice, cs) != cudaSuccess) return FA_ERR_CUDA;
+        if (cudaMemcpyAsync(v_d, v_new_host, k_bytes, cudaMemcpyHostToDevice, cs) != cudaSuccess) return FA_ERR_CUDA;
+        st = fa_append(layout, cache, k_d, v_d, stream);
+        if (st != FA_OK) return st;
+    }
+    st = fa_decode_attention(layout, cache, q_d, o_d, ws, ws_bytes, stream);
+    if (st != FA_OK) return st;
+    if (cudaMemcpyAsync(out_host, o_d, q_bytes, cudaMemcpyDeviceToHost, cs) != cudaSuccess) return FA_ERR_CUDA;
     return FA_OK;
 }
 

@@ -84,6 +84,15 @@ cudaError_t launch_decode_direct(const Dims&, const CacheDev&, int dtype, const 
 cudaError_t launch_decode_epilogue(const Dims&, const CacheDev&, int dtype, const DecodePlan&, void* out, char* ws,
                                    cudaStream_t);
 
+// Raises a kernel's dynamic shared memory limit when a launch needs more than it has been
+// given so far on the current device (no CUDA call at all in the steady state, so launches
+// stay capturable in CUDA graphs after a warm-up call).
+cudaError_t ensure_dynamic_smem_impl(const void* kernel, size_t bytes);
+template <typename Kernel>
+inline cudaError_t ensure_dynamic_smem(Kernel kernel, size_t bytes) {
+    return ensure_dynamic_smem_impl(reinterpret_cast<const void*>(kernel), bytes);
+}
+
 #ifdef __CUDACC__
 // ---- element access ---------------------------------------------------------
 __device__ __forceinline__ float ld_f(const float* p) { return *p; }

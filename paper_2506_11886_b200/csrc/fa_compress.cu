@@ -192,7 +192,7 @@ static cudaError_t launch_compress_t(const Dims& s, const CacheDev& c, const voi
     int cps = (chunks + n_tsplit - 1) / n_tsplit;
     n_tsplit = (chunks + cps - 1) / cps;
     size_t smem = sizeof(float) * ((size_t)kTJ * max_comp + (size_t)kTJ * kTM);
-    err = cudaFuncSetAttribute(compress_coef_kernel<KV>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    err = ensure_dynamic_smem(compress_coef_kernel<KV>, smem);
     if (err != cudaSuccess) return err;
     compress_coef_kernel<KV><<<dim3(row_tiles, n_tsplit, s.B * s.Hkv * 2), 256, smem, stream>>>(
         s, c, static_cast<const KV*>(K), static_cast<const KV*>(V), sb, st, sh, L, cps);

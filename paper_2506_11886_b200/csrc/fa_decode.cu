@@ -441,7 +441,7 @@ static cudaError_t launch_direct_t(const Dims& s, const CacheDev& c, const Decod
                                    cudaStream_t st) {
     size_t smem = sizeof(float) * ((size_t)GH * s.d * 2 + (size_t)GH * s.nfk + 2 * (size_t)GH * s.M + (size_t)GH * kTile +
                                    8 * GH + (size_t)256 * GH);
-    cudaError_t err = cudaFuncSetAttribute(decode_direct_kernel<KV, GH>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    cudaError_t err = ensure_dynamic_smem(decode_direct_kernel<KV, GH>, smem);
     if (err != cudaSuccess) return err;
     decode_direct_kernel<KV, GH><<<dim3(p.n_split, s.Hkv * p.n_pass, s.B), 256, smem, st>>>(s, c, p, static_cast<const KV*>(q), ws);
     return cudaGetLastError();

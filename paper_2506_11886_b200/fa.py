@@ -69,11 +69,15 @@ def lib() -> C.CDLL:
         L.fa_append.argtypes = [lp, cp, vp, vp, vp]
         L.fa_decode_attention.argtypes = [lp, cp, vp, vp, vp, sz, vp]
         L.fa_poll_status.argtypes = [cp, vp]
+        L.fa_decode_step_host.argtypes = [lp, cp, vp, vp, vp, vp, vp, vp, sz, vp]
+        L.fa_step_staging_bytes.argtypes = [lp]
+        L.fa_step_staging_bytes.restype = sz
         L.fa_launch_count.argtypes = [lp, C.c_int]
         L.fa_status_string.argtypes = [C.c_int]
         L.fa_status_string.restype = C.c_char_p
         for name in ("fa_cache_sizes_of", "fa_workspace_bytes", "fa_cache_reset", "fa_validate", "fa_compress",
-                     "fa_append", "fa_decode_attention", "fa_poll_status", "fa_launch_count", "fa_version"):
+                     "fa_append", "fa_decode_attention", "fa_poll_status", "fa_launch_count", "fa_version",
+                     "fa_decode_step_host"):
             getattr(L, name).restype = C.c_int
         _lib = L
     return _lib
@@ -227,6 +231,22 @@ def fa_decode_attention(layout: Layout, cache: Cache, q: torch.Tensor, out: torc
     assert q.is_cuda and out.is_cuda
     _check(lib().fa_decode_attention(C.byref(layout.c()), C.byref(cache.c()), _ptr(q), _ptr(out), _ptr(ws), ws.numel(),
                                      _stream(stream)), "fa_decode_attention")
+
+
+def fa_step_staging_bytes(layout: Layout) -> int:
+    return int(lib().fa_step_staging_bytes(C.byref(layout.c())))
+
+
+def fa_decode_step_host(layout: Layout, cache: Cache, q_host: torch.Tensor, k_new_host, v_new_host,
+                        out_host: torch.Tensor, staging: torch.Tensor, ws: torch.Tensor, stream=None) -> None:
+    """Host-buffer decode step: q_host / out_host [B][H_q][d], k_new_host / v_new_host [B][H_kv][d]
+    (or None to skip the append) are CPU tensors, pinned for asynchronous copies."""
+    for t in (q_host, out_host, k_new_host, v_new_host):
+        assert t is None or (not t.is_cuda and t.is_contiguous() and t.dtype == layout.torch_dtype)
+    assert staging.is_cuda and staging.numel() * staging.element_size() >= fa_step_staging_bytes(layout)
+    _check(lib().fa_decode_step_host(C.byref(layout.c()), C.byref(cache.c()), _ptr(q_host), _ptr(k_new_host),
+                                     _ptr(v_new_host), _ptr(out_host), _ptr(staging), _ptr(ws), ws.numel(),
+                                     _stream(stream)), "fa_decode_step_host")
 
 
 def fa_poll_status(cache: Cache, stream=None) -> int:
