@@ -160,6 +160,25 @@ fa_status fa_decode_step_host(const fa_layout* layout, fa_cache* cache, const vo
                               void* staging, void* ws, size_t ws_bytes, void* stream);
 size_t fa_step_staging_bytes(const fa_layout* layout);
 
+/* fa_decode_attention without a caller workspace.  (The paper has no counterpart: this is a
+ * packaging variant of the same computation.)  It is meant for callers that cannot allocate
+ * device memory when they reach this call: an engine that gave all of its HBM to its own pools
+ * at start-up and hands plug-ins no scratch, or a decode loop in which cudaMalloc, which
+ * synchronises the device, is not allowed.  The scratch is a fixed array of
+ * fa_static_workspace_limit() bytes (8 MiB) built into the library; each GPU that loads the
+ * library holds it until the process exits.  No call made here allocates or frees.
+ *   - q, out, cache: exactly as for fa_decode_attention; the result is the same.
+ *   - Layouts whose fa_workspace_bytes exceeds the limit are refused with FA_ERR_WORKSPACE
+ *     before anything runs; use fa_decode_attention with your own workspace for those.
+ *   - The first call on each device looks the array's device address up (with that device
+ *     current); make that first call before any stream capture.
+ *   - All calls on one GPU share the one array.  It keeps whatever the previous call left; the
+ *     call clears the few counters it needs itself.  Two calls that overlap on the GPU (two
+ *     streams, two threads) race on it: serialise them. */
+fa_status fa_decode_attention_static(const fa_layout* layout, const fa_cache* cache, const void* q,
+                                     void* out, void* stream);
+size_t fa_static_workspace_limit(void);
+
 /* Synchronises the stream and returns (then clears) the sticky device status word. */
 fa_status fa_poll_status(const fa_cache* cache, void* stream);
 

@@ -259,3 +259,23 @@ def fa_launch_count(layout: Layout, what: int) -> int:
 
 def fa_version() -> int:
     return int(lib().fa_version())
+
+
+def fa_static_workspace_limit() -> int:
+    f = lib().fa_static_workspace_limit
+    f.restype, f.argtypes = C.c_size_t, []
+    return int(f())
+
+
+def fa_decode_attention_static(layout: Layout, cache: Cache, q: torch.Tensor, out: torch.Tensor, stream=None) -> None:
+    """``fa_decode_attention`` for callers that cannot allocate device memory (an engine
+    whose memory is all spoken for, a loop in which cudaMalloc is not allowed): the scratch
+    is the library's own fixed 8 MiB array, so no workspace is passed.  Layouts that need
+    more scratch raise FA_ERR_WORKSPACE.  Calls on one GPU share that array: do not overlap
+    them, and make the first call on a device outside any stream capture."""
+    assert q.is_contiguous() and out.is_contiguous() and q.dtype == layout.torch_dtype and out.dtype == q.dtype
+    assert q.is_cuda and out.is_cuda
+    f = lib().fa_decode_attention_static
+    f.restype = C.c_int
+    f.argtypes = [C.POINTER(fa_layout), C.POINTER(fa_cache), C.c_void_p, C.c_void_p, C.c_void_p]
+    _check(f(C.byref(layout.c()), C.byref(cache.c()), _ptr(q), _ptr(out), _stream(stream)), "fa_decode_attention_static")
