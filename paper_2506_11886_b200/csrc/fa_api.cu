@@ -58,14 +58,18 @@ static int ilog2_exact(int v) {
     return ((1 << l) == v) ? l : -1;
 }
 
-// True if the residue-class transform can serve this layout: power-of-two
-// period, one class per period / S tokens with S a power of two >= k.
-static bool fft_ok(const fa_layout& l, int* log2S) {
+// True if the residue-class transform kernel can serve this layout: power-of-two period split
+// into P classes of S = T / P slots, S a power of two in [32, 2048]; at most 64 kept dims per
+// side, head_dim <= 128, and the kernel's shared memory must fit.
+static bool fft_ok(const fa_layout& l, int gh, int* log2S) {
     if (l.head_dim == l.n_full_k && l.head_dim == l.n_full_v) return false;   // nothing compressed
     if (ilog2_exact(l.period) < 0 || l.period % l.mid_classes != 0) return false;
     int S = l.period / l.mid_classes;
     int ls = ilog2_exact(S);
-    if (ls < 5 || ls > 11 || S < l.n_coef / 2) return false;
+    if (ls < 5 || ls > 11) return false;
+    if ((l.n_coef / 2 + S - 1) / S > 8) return false;                          // at most 8-fold aliasing of the bins
+    if (l.n_full_k > 64 || l.n_full_v > 64 || l.head_dim > 128) return false;
+    if (decode_fft_smem_bytes(make_dims(l), gh) > 227 * 1024) return false;
     *log2S = ls;
     return true;
 }
@@ -74,23 +78,39 @@ fa_status plan_decode(const fa_layout& l, DecodePlan* p) {
     Dims s = make_dims(l);
     std::memset(p, 0, sizeof(*p));
     int log2S = 0;
-    bool can_fft = false;   // the FFT kernel registers itself here once built
-    (void)fft_ok; (void)log2S;
+    const int gh_fft = s.G >= 3 ? 4 : 2;
+    const bool can_fft = fft_ok(l, gh_fft, &log2S);
     if (l.decode_algo == FA_DECODE_FFT && !can_fft) return FA_ERR_UNSUPPORTED;
     p->algo = (l.decode_algo == FA_DECODE_DIRECT || !can_fft) ? FA_DECODE_DIRECT : FA_DECODE_FFT;
     p->fft_log2 = log2S;
-    p->gh = s.G >= 4 ? 4 : (s.G >= 2 ? 2 : 1);
-    if (s.G == 3) p->gh = 4;
-    p->n_pass = (s.G + p->gh - 1) / p->gh;
-    // split the tokens of one (b, KV head, pass) over CTAs so that the grid fills the GPU about twice
-    int jobs = s.B * s.Hkv * p->n_pass;
-    int want = (2 * kNumSms + jobs - 1) / jobs;
-    long long tokens = (long long)s.max_mid + s.l_init + s.l_local;
-    int max_by_work = (int)((tokens + 255) / 256);            // at least one 256-token tile each
-    if (want > max_by_work) want = max_by_work;
-    if (want > 64) want = 64;
-    if (want < 1) want = 1;
-    p->n_split = want;
+    if (p->algo == FA_DECODE_FFT) {
+        p->gh = gh_fft;
+        p->n_pass = (s.G + p->gh - 1) / p->gh;
+        // classes are indivisible: pick the split count that minimises waves * classes per CTA
+        // (one CTA per SM), smallest count on ties to keep the partial results small
+        const int jobs = s.B * s.Hkv * p->n_pass;
+        int best = 1;
+        long long best_cost = -1;
+        for (int n = 1; n <= s.P && n <= 64; ++n) {
+            long long waves = ((long long)jobs * n + kNumSms - 1) / kNumSms;
+            long long cost = waves * ((s.P + n - 1) / n);
+            if (best_cost < 0 || cost < best_cost) { best_cost = cost; best = n; }
+        }
+        p->n_split = best;
+    } else {
+        p->gh = s.G >= 4 ? 4 : (s.G >= 2 ? 2 : 1);
+        if (s.G == 3) p->gh = 4;
+        p->n_pass = (s.G + p->gh - 1) / p->gh;
+        // split the tokens of one (b, KV head, pass) over CTAs so that the grid fills the GPU about twice
+        int jobs = s.B * s.Hkv * p->n_pass;
+        int want = (2 * kNumSms + jobs - 1) / jobs;
+        long long tokens = (long long)s.max_mid + s.l_init + s.l_local;
+        int max_by_work = (int)((tokens + 255) / 256);            // at least one 256-token tile each
+        if (want > max_by_work) want = max_by_work;
+        if (want > 64) want = 64;
+        if (want < 1) want = 1;
+        p->n_split = want;
+    }
     p->rows_pro = 64;
     p->n_slice = s.dcv > 0 ? (s.M + 127) / 128 : 1;
     size_t off = 0;
@@ -249,7 +269,11 @@ fa_status fa_decode_attention(const fa_layout* layout, const fa_cache* cache, co
     cudaStream_t cs = static_cast<cudaStream_t>(stream);
     char* w = static_cast<char*>(ws);
     if (launch_decode_prologue(s, c, layout->kv_dtype, p, q, w, cs) != cudaSuccess) return FA_ERR_CUDA;
-    if (launch_decode_direct(s, c, layout->kv_dtype, p, q, w, cs) != cudaSuccess) return FA_ERR_CUDA;
+    if (p.algo == FA_DECODE_FFT) {
+        if (launch_decode_fft(s, c, layout->kv_dtype, p, q, w, cs) != cudaSuccess) return FA_ERR_CUDA;
+    } else {
+        if (launch_decode_direct(s, c, layout->kv_dtype, p, q, w, cs) != cudaSuccess) return FA_ERR_CUDA;
+    }
     if (launch_decode_epilogue(s, c, layout->kv_dtype, p, out, w, cs) != cudaSuccess) return FA_ERR_CUDA;
     return FA_OK;
 }

@@ -81,6 +81,9 @@ cudaError_t launch_decode_prologue(const Dims&, const CacheDev&, int dtype, cons
                                    cudaStream_t);
 cudaError_t launch_decode_direct(const Dims&, const CacheDev&, int dtype, const DecodePlan&, const void* q, char* ws,
                                  cudaStream_t);
+cudaError_t launch_decode_fft(const Dims&, const CacheDev&, int dtype, const DecodePlan&, const void* q, char* ws,
+                              cudaStream_t);
+size_t decode_fft_smem_bytes(const Dims&, int gh);
 cudaError_t launch_decode_epilogue(const Dims&, const CacheDev&, int dtype, const DecodePlan&, void* out, char* ws,
                                    cudaStream_t);
 
