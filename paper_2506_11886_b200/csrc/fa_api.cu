@@ -111,8 +111,8 @@ fa_status plan_decode(const fa_layout& l, DecodePlan* p) {
         if (want < 1) want = 1;
         p->n_split = want;
     }
-    p->rows_pro = 64;
-    p->n_slice = s.dcv > 0 ? (s.M + 127) / 128 : 1;
+    p->rows_pro = 32;
+    p->n_slice = s.dcv > 0 ? (s.M + 63) / 64 : 1;
     size_t off = 0;
     p->off_u = off;   off = align_up(off + sizeof(float) * (size_t)s.B * s.Hq * s.M, 256);
     p->off_ml = off;  off = align_up(off + sizeof(float) * (size_t)s.B * s.Hq * p->n_split * 2, 256);

@@ -1,55 +1,13 @@
-// fa_decode_attention (Eq.6), evaluated on the small side:
-//   prologue   u_g[m] = scale * log2(e) * w_m * sum_e C^K[m][e] q_g[D^kc[e]]
-//   main       per token j of the middle: s_j = q_u . K^mu_j + sum_m F[m][j] u_g[m];
-//              online softmax; o^u += p_j V^mu_j;  z[m] += p_j F[m][j];
-//              window tokens: ordinary attention in the same softmax
-//   epilogue   merge the token splits, o^c[e] = sum_m w_m z[m] C^V[m][e], normalise, scatter.
-// This file holds the prologue, the epilogue and the DIRECT main kernel, which
-// sums the M basis terms of every token one by one (any period, any class count).
+// fa_decode_attention (Eq.6), DIRECT main kernel: per token of the middle
+//   s_j = q_u . K^mu_j + sum_m F[m][j] u_g[m];  online softmax;  o^u += p_j V^mu_j;
+//   z[m] += p_j F[m][j];  window tokens: ordinary attention in the same softmax.
+// The M basis terms of every token are summed one by one (any period, any class count):
+// the reference of the GPU side and the fallback of the transform kernel.
 #include "fa_common.cuh"
 #include "fa_decode_ws.cuh"
 
 namespace fa {
 
-
-// ---------------------------------------------------------------- prologue --
-// grid (row tiles, Hkv, B); one warp per coefficient row, lanes over the D^kc columns.
-template <typename KV>
-__global__ void __launch_bounds__(256) decode_prologue_kernel(Dims s, CacheDev c, DecodePlan p, const KV* __restrict__ q,
-                                                              char* wsp) {
-    extern __shared__ float qc_s[];               // [G][dck] gathered query, fp32
-    Ws ws = ws_view(wsp, p);
-    const int h = blockIdx.y, b = blockIdx.z;
-    if (blockIdx.x == 0 && threadIdx.x == 0) ws.cnt[b * s.Hkv + h] = 0;
-    if (s.dck == 0) return;
-    const int32_t* idc = c.idx_comp_k + (size_t)h * s.dck;
-    for (int i = threadIdx.x; i < s.G * s.dck; i += blockDim.x) {
-        int g = i / s.dck, e = i - g * s.dck;
-        qc_s[i] = ld_f(q + ((size_t)b * s.Hq + h * s.G + g) * s.d + idc[e]);
-    }
-    __syncthreads();
-    const float* coef = coef_rows(c.coef_k, s, b, h, s.dck);
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int m_end = min(s.M, (int)(blockIdx.x + 1) * p.rows_pro);
-    for (int m = blockIdx.x * p.rows_pro + warp; m < m_end; m += 8) {
-        const float* row = coef + (size_t)m * s.dck;
-        float wm = recon_weight(s.norm, m, s.k, s.T) * s.scale * kLog2e;
-        for (int g0 = 0; g0 < s.G; g0 += 4) {
-            float acc[4] = {0.f, 0.f, 0.f, 0.f};
-            for (int e = lane; e < s.dck; e += 32) {
-                float cv = row[e];
-#pragma unroll
-                for (int g = 0; g < 4; ++g)
-                    if (g0 + g < s.G) acc[g] = fmaf(cv, qc_s[(g0 + g) * s.dck + e], acc[g]);
-            }
-#pragma unroll
-            for (int g = 0; g < 4; ++g) {
-                float v = warp_sum(acc[g]);
-                if (lane == 0 && g0 + g < s.G) ws.u[((size_t)b * s.Hq + h * s.G + g0 + g) * s.M + m] = wm * v;
-            }
-        }
-    }
-}
 
 // ------------------------------------------------------------- direct main --
 // grid (n_split, Hkv * n_pass, B), 256 threads; one thread per token of a 256-token tile.
@@ -310,113 +268,6 @@ __global__ void __launch_bounds__(256) decode_direct_kernel(Dims s, CacheDev c, 
     }
 }
 
-// ---------------------------------------------------------------- epilogue --
-// grid (n_slice, Hkv, B).  Each CTA merges the split statistics of its KV head, forms the
-// weighted z of its coefficient rows and multiplies by its rows of C^V; the last CTA of a
-// (b, h) to finish (atomic ticket) adds the slices, normalises and writes the output rows.
-template <typename KV>
-__global__ void __launch_bounds__(256) decode_epilogue_kernel(Dims s, CacheDev c, DecodePlan p, KV* __restrict__ out,
-                                                              char* wsp) {
-    extern __shared__ float sm[];
-    __shared__ int last_s;
-    Ws ws = ws_view(wsp, p);
-    const int slice = blockIdx.x, h = blockIdx.y, b = blockIdx.z;
-    const int tid = threadIdx.x;
-    const int rows = (s.M + p.n_slice - 1) / p.n_slice;
-    const int m0 = slice * rows, m1 = min(s.M, m0 + rows);
-    float* alpha_s = sm;                              // [G][n_split]
-    float* linv_s = alpha_s + s.G * p.n_split;        // [G]
-    float* zw_s = linv_s + s.G;                       // [G][rows]
-    float* red_s = zw_s + s.G * rows;                 // [256]
-    float* o_s = red_s + 256;                         // [d]
-
-    for (int g = tid; g < s.G; g += blockDim.x) {
-        const float* ml = ws.ml + ((size_t)b * s.Hq + h * s.G + g) * p.n_split * 2;
-        float mx = kNegBig;
-        for (int sp = 0; sp < p.n_split; ++sp) mx = fmaxf(mx, ml[2 * sp]);
-        float L = 0.f;
-        for (int sp = 0; sp < p.n_split; ++sp) {
-            float a = exp2f(ml[2 * sp] - mx);
-            alpha_s[g * p.n_split + sp] = a;
-            L += a * ml[2 * sp + 1];
-        }
-        linv_s[g] = L > 0.f ? 1.0f / L : 0.f;
-    }
-    __syncthreads();
-    if (s.dcv > 0) {
-        for (int i = tid; i < s.G * rows; i += blockDim.x) {
-            int g = i / rows, m = m0 + (i - g * rows);
-            float v = 0.f;
-            if (m < m1) {
-                const float* z = ws.z + ((size_t)b * s.Hq + h * s.G + g) * p.n_split * s.M + m;
-                for (int sp = 0; sp < p.n_split; ++sp) v = fmaf(alpha_s[g * p.n_split + sp], z[(size_t)sp * s.M], v);
-                v *= recon_weight(s.norm, m, s.k, s.T);
-            }
-            zw_s[i] = v;
-        }
-        __syncthreads();
-        // partial o^c of this slice: thread (mg, e) sums rows m = m0 + mg, m0 + mg + nmg, ...
-        const float* cv = coef_rows(c.coef_v, s, b, h, s.dcv);
-        const int nmg = blockDim.x / s.dcv;            // dcv <= 256
-        const int mg = tid / s.dcv, e = tid % s.dcv;
-        for (int g = 0; g < s.G; ++g) {
-            float acc = 0.f;
-            if (mg < nmg)
-                for (int m = m0 + mg; m < m1; m += nmg) acc = fmaf(zw_s[g * rows + (m - m0)], cv[(size_t)m * s.dcv + e], acc);
-            red_s[tid] = acc;
-            __syncthreads();
-            if (tid < s.dcv) {
-                float v = 0.f;
-                for (int r = 0; r < nmg; ++r) v += red_s[r * s.dcv + tid];
-                ws.oc[(((size_t)b * s.Hq + h * s.G + g) * p.n_slice + slice) * s.dcv + tid] = v;
-            }
-            __syncthreads();
-        }
-    }
-    // ticket
-    if (tid == 0) {
-        __threadfence();
-        int done = atomicAdd(ws.cnt + b * s.Hkv + h, 1);
-        last_s = (done == (int)gridDim.x - 1);
-    }
-    __syncthreads();
-    if (!last_s) return;
-    __threadfence();
-    const int32_t* idc_v = c.idx_comp_v + (size_t)h * s.dcv;
-    for (int g = 0; g < s.G; ++g) {
-        const size_t qh = (size_t)b * s.Hq + h * s.G + g;
-        for (int e = tid; e < s.d; e += blockDim.x) {
-            float v = 0.f;
-            for (int sp = 0; sp < p.n_split; ++sp) v = fmaf(alpha_s[g * p.n_split + sp], ws.o[(qh * p.n_split + sp) * s.d + e], v);
-            o_s[e] = v;
-        }
-        __syncthreads();
-        for (int e = tid; e < s.dcv; e += blockDim.x) {
-            float v = 0.f;
-            for (int sl = 0; sl < p.n_slice; ++sl) v += __ldcg(ws.oc + (qh * p.n_slice + sl) * s.dcv + e);
-            o_s[idc_v[e]] += v;
-        }
-        __syncthreads();
-        for (int e = tid; e < s.d; e += blockDim.x) st_f(out + qh * s.d + e, o_s[e] * linv_s[g]);
-        __syncthreads();
-    }
-}
-
-// ---------------------------------------------------------------- launchers --
-template <typename KV>
-static cudaError_t launch_prologue_t(const Dims& s, const CacheDev& c, const DecodePlan& p, const void* q, char* ws,
-                                     cudaStream_t st) {
-    int tiles = s.dck > 0 ? (s.M + p.rows_pro - 1) / p.rows_pro : 1;
-    size_t smem = sizeof(float) * (size_t)s.G * (s.dck > 0 ? s.dck : 1);
-    decode_prologue_kernel<KV><<<dim3(tiles, s.Hkv, s.B), 256, smem, st>>>(s, c, p, static_cast<const KV*>(q), ws);
-    return cudaGetLastError();
-}
-
-cudaError_t launch_decode_prologue(const Dims& s, const CacheDev& c, int dtype, const DecodePlan& p, const void* q,
-                                   char* ws, cudaStream_t st) {
-    if (dtype == FA_BF16) return launch_prologue_t<__nv_bfloat16>(s, c, p, q, ws, st);
-    return launch_prologue_t<float>(s, c, p, q, ws, st);
-}
 
 template <typename KV, int GH>
 static cudaError_t launch_direct_t(const Dims& s, const CacheDev& c, const DecodePlan& p, const void* q, char* ws,
@@ -439,21 +290,6 @@ cudaError_t launch_decode_direct(const Dims& s, const CacheDev& c, int dtype, co
     if (p.gh == 4) return launch_direct_t<float, 4>(s, c, p, q, ws, st);
     if (p.gh == 2) return launch_direct_t<float, 2>(s, c, p, q, ws, st);
     return launch_direct_t<float, 1>(s, c, p, q, ws, st);
-}
-
-template <typename KV>
-static cudaError_t launch_epilogue_t(const Dims& s, const CacheDev& c, const DecodePlan& p, void* out, char* ws,
-                                     cudaStream_t st) {
-    int rows = (s.M + p.n_slice - 1) / p.n_slice;
-    size_t smem = sizeof(float) * ((size_t)s.G * p.n_split + s.G + (size_t)s.G * rows + 256 + s.d);
-    decode_epilogue_kernel<KV><<<dim3(p.n_slice, s.Hkv, s.B), 256, smem, st>>>(s, c, p, static_cast<KV*>(out), ws);
-    return cudaGetLastError();
-}
-
-cudaError_t launch_decode_epilogue(const Dims& s, const CacheDev& c, int dtype, const DecodePlan& p, void* out, char* ws,
-                                   cudaStream_t st) {
-    if (dtype == FA_BF16) return launch_epilogue_t<__nv_bfloat16>(s, c, p, out, ws, st);
-    return launch_epilogue_t<float>(s, c, p, out, ws, st);
 }
 
 }  // namespace fa
