@@ -94,7 +94,11 @@ typedef struct fa_cache {
     void*  k_local;             /* [B][H_kv][l_local][d], a ring: oldest row at state.local_head */
     void*  v_local;
     void*  k_mid;               /* [B][H_kv][P][ceil(max_mid/P)][n_full_k]   K^mu       */
-    void*  v_mid;               /* [B][H_kv][P][ceil(max_mid/P)][n_full_v]   V^mu       */
+    void*  v_mid;               /* [B][H_kv][P][ceil(max_mid/P)][n_full_v]   V^mu.  In bf16
+                                   caches the 8-dim (16-byte) chunks of a row are permuted: chunk c
+                                   of slot a is stored at chunk c ^ x, x = (a>>2)&1 for 2 or 6 chunks
+                                   per row, (a>>1)&3 for 4, a&7 for 8, 0 otherwise (bank-conflict-free
+                                   shared-memory image for the tensor-core loads of the decode kernel) */
     float* coef_k;              /* [B][H_kv][M][d - n_full_k]  K^mc, raw sums of Eq.3   */
     float* coef_v;              /* [B][H_kv][M][d - n_full_v]  V^mc                     */
     int32_t* state;             /* [B][8]: n_init, n_local, n_mid, local_head, ticket, 3 spare */

@@ -62,14 +62,15 @@ static int ilog2_exact(int v) {
 // into P classes of S = T / P slots, S a power of two in [32, 2048]; at most 64 kept dims per
 // side, head_dim <= 128, and the kernel's shared memory must fit.
 static bool fft_ok(const fa_layout& l, int gh, int* log2S) {
+    if (l.kv_dtype != FA_BF16) return false;                                   // tensor-core dot products: bf16 caches
     if (l.head_dim == l.n_full_k && l.head_dim == l.n_full_v) return false;   // nothing compressed
     if (ilog2_exact(l.period) < 0 || l.period % l.mid_classes != 0) return false;
     int S = l.period / l.mid_classes;
     int ls = ilog2_exact(S);
     if (ls < 5 || ls > 11) return false;
-    if ((l.n_coef / 2 + S - 1) / S > 8) return false;                          // at most 8-fold aliasing of the bins
+    if (l.n_coef / 2 > S) return false;                                        // every frequency needs its own bin
     if (l.n_full_k > 64 || l.n_full_v > 64 || l.head_dim > 128) return false;
-    if (decode_fft_smem_bytes(make_dims(l), gh) > 227 * 1024) return false;
+    if (decode_fft_smem_bytes(make_dims(l), ls, gh, 1) > 227 * 1024) return false;
     *log2S = ls;
     return true;
 }
@@ -97,6 +98,15 @@ fa_status plan_decode(const fa_layout& l, DecodePlan* p) {
             if (best_cost < 0 || cost < best_cost) { best_cost = cost; best = n; }
         }
         p->n_split = best;
+        // classes transformed together: enough butterflies for all consumer threads, within shared memory
+        const int S = s.T / s.P;
+        int nb = 2048 / S;
+        if (nb < 1) nb = 1;
+        if (nb > 8) nb = 8;
+        const int per_cta = (s.P + best - 1) / best;
+        if (nb > per_cta) nb = per_cta;
+        while (nb > 1 && decode_fft_smem_bytes(s, log2S, p->gh, nb) > 227 * 1024) --nb;
+        p->nb = nb;
     } else {
         p->gh = s.G >= 4 ? 4 : (s.G >= 2 ? 2 : 1);
         if (s.G == 3) p->gh = 4;

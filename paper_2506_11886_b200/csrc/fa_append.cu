@@ -78,7 +78,8 @@ __global__ void __launch_bounds__(256) append_kernel(Dims s, CacheDev c, const K
                 const int nfull = side == 0 ? s.nfk : s.nfv;
                 const int32_t* idf = (side == 0 ? c.idx_full_k : c.idx_full_v) + (size_t)h * nfull;
                 KV* dst = mid_row<KV>(side == 0 ? c.k_mid : c.v_mid, s, b, h, j % s.P, j / s.P, nfull);
-                st_f(dst + e, x_s[side][idf[e]]);
+                const int col = side == 1 ? v_mid_col(j / s.P, e, nfull, sizeof(KV) == 2 ? FA_BF16 : FA_F32) : e;
+                st_f(dst + col, x_s[side][idf[e]]);
             }
         }
         __syncthreads();

@@ -65,9 +65,29 @@ struct DecodePlan {
     int n_slice;       // CTAs that share the coefficient rows of one (b, KV head) in the epilogue
     int rows_pro;      // coefficient rows per prologue CTA
     int fft_log2;      // log2 of the transform length (FFT path)
+    int nb;            // classes transformed together by one CTA (FFT path)
     // workspace offsets in bytes
     size_t off_u, off_ml, off_o, off_z, off_oc, off_cnt, total;
 };
+
+// V^mu of bf16 caches is stored with its 16-byte chunks (8 dims) permuted inside each row:
+// chunk c of slot a sits at chunk c ^ v_swz(a, chunks per row).  A bulk copy of a class then
+// lands in shared memory in an image whose 8x8 matrix loads (ldmatrix) of eight consecutive
+// slots hit eight different bank groups.  fp32 caches are stored plainly.
+__host__ __device__ inline int v_swz(int a, int nchunks) {
+    switch (nchunks) {
+        case 2: return (a >> 2) & 1;
+        case 4: return (a >> 1) & 3;
+        case 6: return (a >> 2) & 1;
+        case 8: return a & 7;
+        default: return 0;
+    }
+}
+// Element offset of dim slot e of V^mu row (slot) a inside its row of nfv elements.
+__host__ __device__ inline int v_mid_col(int a, int e, int nfv, int dtype) {
+    if (dtype != FA_BF16) return e;
+    return ((((e >> 3) ^ v_swz(a, nfv >> 3)) << 3) | (e & 7));
+}
 
 fa_status plan_decode(const fa_layout& l, DecodePlan* plan);
 fa_status check_layout(const fa_layout* l);
@@ -83,7 +103,7 @@ cudaError_t launch_decode_direct(const Dims&, const CacheDev&, int dtype, const 
                                  cudaStream_t);
 cudaError_t launch_decode_fft(const Dims&, const CacheDev&, int dtype, const DecodePlan&, const void* q, char* ws,
                               cudaStream_t);
-size_t decode_fft_smem_bytes(const Dims&, int gh);
+size_t decode_fft_smem_bytes(const Dims&, int log2S, int gh, int nb);
 cudaError_t launch_decode_epilogue(const Dims&, const CacheDev&, int dtype, const DecodePlan&, void* out, char* ws,
                                    cudaStream_t);
 

@@ -80,7 +80,10 @@ __global__ void __launch_bounds__(256) partition_gather_kernel(Dims s, CacheDev 
             for (int e = lane; e < s.d; e += 32) row_s[warp][e] = ld_f(src + e);
             __syncwarp();
             KV* dst = mid_row<KV>(w_mid, s, b, h, j % s.P, j / s.P, nfull);
-            for (int e = lane; e < nfull; e += 32) st_f(dst + e, row_s[warp][idf[e]]);
+            for (int e = lane; e < nfull; e += 32) {
+                const int col = side == 1 ? v_mid_col(j / s.P, e, nfull, sizeof(KV) == 2 ? FA_BF16 : FA_F32) : e;
+                st_f(dst + col, row_s[warp][idf[e]]);
+            }
             __syncwarp();
         }
     }

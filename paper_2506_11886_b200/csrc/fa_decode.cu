@@ -161,7 +161,8 @@ __global__ void __launch_bounds__(256) decode_direct_kernel(Dims s, CacheDev c, 
             // o^u += p V^mu
             if (act_mid) {
                 for (int i = tg_mid; i < nt; i += ntg_mid) {
-                    float x = ld_f(mid_row<KV>(c.v_mid, s, b, h, cls, a0 + i, s.nfv) + e_mid);
+                    float x = ld_f(mid_row<KV>(c.v_mid, s, b, h, cls, a0 + i, s.nfv) +
+                                   v_mid_col(a0 + i, e_mid, s.nfv, sizeof(KV) == 2 ? FA_BF16 : FA_F32));
 #pragma unroll
                     for (int g = 0; g < GH; ++g) o_mid[g] = fmaf(p_s[g * kTile + i], x, o_mid[g]);
                 }

@@ -33,6 +33,24 @@ def oracle_cfg(layout: fa.Layout, heads=None) -> fo.OracleConfig:
                            scale=layout.softmax_scale, norm=layout.norm)
 
 
+def unswizzle_v_rows(rows: np.ndarray, slots: np.ndarray, layout: fa.Layout) -> np.ndarray:
+    """V^mu rows of bf16 caches are stored with their 16-byte chunks (8 dims) XOR-permuted by a
+    function of the slot index (include/fa.h); returns the rows in logical dim order.
+    rows: [H][n][n_full_v] in stored order, slots: [n] slot index of each row."""
+    nfv = layout.n_full_v
+    nch = nfv // 8
+    if layout.kv_dtype != fa.FA_BF16 or nch not in (2, 4, 6, 8):
+        return rows
+    x = {2: (slots >> 2) & 1, 4: (slots >> 1) & 3, 6: (slots >> 2) & 1, 8: slots & 7}[nch]
+    out = np.empty_like(rows)
+    for c in range(nch):
+        pc = c ^ x                                              # physical chunk of logical chunk c, per row
+        for val in np.unique(pc):
+            sel = pc == val
+            out[:, sel, 8 * c:8 * c + 8] = rows[:, sel, 8 * val:8 * val + 8]
+    return out
+
+
 def to64(t: torch.Tensor) -> np.ndarray:
     return t.detach().to("cpu", torch.float64).numpy()
 
@@ -81,7 +99,10 @@ class Pair:
                     order = (head + np.arange(nl)) % L.l_local
                     np.testing.assert_array_equal(gl[:, order], rl[:, :nl], err_msg=f"{name}_local")
                 j = np.arange(nm)
-                np.testing.assert_array_equal(gm[:, j % L.mid_classes, j // L.mid_classes], rm[:, :nm], err_msg=f"{name}_mid")
+                got_mid = gm[:, j % L.mid_classes, j // L.mid_classes]          # [H][nm][n_full], stored order
+                if name == "v":
+                    got_mid = unswizzle_v_rows(got_mid, j // L.mid_classes, L)
+                np.testing.assert_array_equal(got_mid, rm[:, :nm], err_msg=f"{name}_mid")
         worst = 0.0
         for name in ("coef_k", "coef_v"):
             gc, rc = to64(getattr(g, name)), getattr(r, name)
