@@ -339,20 +339,23 @@ __global__ void __launch_bounds__(kThreads, 1) decode_fft_kernel(Dims s, CacheDe
                 mbar_expect_tx(full + st, bytes);
                 return stages + (size_t)st * kStageBytes;
             };
-            for (int cls = c0; cls < c1; ++cls) {
-                const int n_c = cls < n_mid ? (n_mid - cls + s.P - 1) / s.P : 0;
-                if (ts_k)
-                    for (int a0 = 0; a0 < n_c; a0 += ts_k) {
-                        const uint32_t bytes = (uint32_t)(min(ts_k, n_c - a0) * rowb_k);
-                        if (unsigned char* dst = acquire(bytes)) bulk_g2s(dst, mid_row<bf16>(c.k_mid, s, b, h, cls, a0, s.nfk), bytes, full + it % kStages);
-                        ++it;
+            // same order as the consumers: per batch of NB classes all K tiles, then all V tiles
+            for (int cb = c0; cb < c1; cb += NB) {
+                const int nb = min(NB, c1 - cb);
+                for (int side = 0; side < 2; ++side) {
+                    const int ts = side == 0 ? ts_k : ts_v, rowb = side == 0 ? rowb_k : rowb_v;
+                    if (!ts) continue;
+                    for (int cls = cb; cls < cb + nb; ++cls) {
+                        const int n_c = cls < n_mid ? (n_mid - cls + s.P - 1) / s.P : 0;
+                        for (int a0 = 0; a0 < n_c; a0 += ts) {
+                            const uint32_t bytes = (uint32_t)(min(ts, n_c - a0) * rowb);
+                            const bf16* src = side == 0 ? mid_row<bf16>(c.k_mid, s, b, h, cls, a0, s.nfk)
+                                                        : mid_row<bf16>(c.v_mid, s, b, h, cls, a0, s.nfv);
+                            if (unsigned char* dst = acquire(bytes)) bulk_g2s(dst, src, bytes, full + it % kStages);
+                            ++it;
+                        }
                     }
-                if (ts_v)
-                    for (int a0 = 0; a0 < n_c; a0 += ts_v) {
-                        const uint32_t bytes = (uint32_t)(min(ts_v, n_c - a0) * rowb_v);
-                        if (unsigned char* dst = acquire(bytes)) bulk_g2s(dst, mid_row<bf16>(c.v_mid, s, b, h, cls, a0, s.nfv), bytes, full + it % kStages);
-                        ++it;
-                    }
+                }
             }
             for (int t0 = w0; t0 < w1; t0 += wchunk) {
                 const WinSegs sg = win_segments(t0, min(w1, t0 + wchunk), n_init, n_local, head, s.l_local);

@@ -1,0 +1,69 @@
+"""Parity at the full size of the benchmark configuration, in the launch configuration bench.py
+times (32K context, 8 KV heads, GQA 4, bf16, M = 1024, 64 classes of 512 slots, FFT decode):
+the whole GPU cache is built and decoded; the oracle recomputes sampled KV heads one by one."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import fa_oracle as fo
+from paper_2506_11886_b200 import fa, synth
+from tests.parity_util import COEF_REL, OUT_ABS_BF16, layout_of, to64, unswizzle_v_rows
+
+pytestmark = pytest.mark.gpu
+
+
+def _sampled_head_check(shape, layout, heads, steps, seed):
+    stream = synth.KVStream(shape, seed=seed, device="cuda")
+    K, V = stream.tokens(0, shape.L, work_dtype=torch.float32)
+    cache = fa.Cache(layout, stream.idx_full_k, stream.idx_full_v)
+    ws = fa.new_workspace(layout)
+    fa.fa_validate(layout, cache)
+    fa.fa_compress(layout, cache, K, V, ws)
+    Kn, Vn = stream.tokens(shape.L, shape.L + steps, work_dtype=torch.float32)
+    for t in range(steps):
+        fa.fa_append(layout, cache, Kn[:, t].contiguous(), Vn[:, t].contiguous())
+    q = synth.queries(shape, seed=seed, device="cuda")
+    out = torch.empty_like(q)
+    fa.fa_decode_attention(layout, cache, q, out, ws)
+    torch.cuda.synchronize()
+    assert fa.fa_poll_status(cache) == fa.FA_OK
+    G = shape.Hq // shape.Hkv
+    worst_out = worst_coef = 0.0
+    for h in heads:
+        sub = fo.OracleConfig(B=shape.B, Hq=G, Hkv=1, d=shape.d, n_full_k=shape.n_full_k, n_full_v=shape.n_full_v,
+                              k=shape.k, T=shape.T, L_init=shape.L_init, L_local=shape.L_local, cap_mid=layout.max_mid,
+                              scale=shape.softmax_scale)
+        ref = fo.OracleCache(sub, stream.idx_full_k[h:h + 1].numpy(), stream.idx_full_v[h:h + 1].numpy())
+        ref.compress(to64(K[:, :, h:h + 1]), to64(V[:, :, h:h + 1]))
+        for t in range(steps):
+            ref.append(to64(Kn[:, t, h:h + 1]), to64(Vn[:, t, h:h + 1]))
+        want = ref.decode(to64(q[:, h * G:(h + 1) * G]))
+        got = to64(out[:, h * G:(h + 1) * G])
+        worst_out = max(worst_out, np.abs(got - want).max())
+        # metadata and stored rows of the sampled head: bit-exact; coefficients: norm-wise
+        st = cache.state.cpu().numpy()
+        assert (st[:, 2] == ref.n_mid).all() and (st[:, 1] == ref.n_local).all() and (st[:, 0] == ref.n_init).all()
+        for b in range(shape.B):
+            nm, head = int(st[b, 2]), int(st[b, 3])
+            j = np.arange(nm)
+            gk = to64(cache.k_mid[b, h])[j % layout.mid_classes, j // layout.mid_classes]
+            gv = to64(cache.v_mid[b, h])[j % layout.mid_classes, j // layout.mid_classes]
+            gv = unswizzle_v_rows(gv[None], j // layout.mid_classes, layout)[0]
+            np.testing.assert_array_equal(gk, ref.k_mid[b, 0, :nm])
+            np.testing.assert_array_equal(gv, ref.v_mid[b, 0, :nm])
+            order = (head + np.arange(shape.L_local)) % shape.L_local
+            np.testing.assert_array_equal(to64(cache.k_local[b, h])[order], ref.k_local[b, 0])
+            for name in ("coef_k", "coef_v"):
+                r = getattr(ref, name)[b, 0]
+                g = to64(getattr(cache, name)[b, h])
+                worst_coef = max(worst_coef, np.abs(g - r).max() / np.abs(r).max())
+    assert worst_coef <= COEF_REL, worst_coef
+    assert worst_out <= OUT_ABS_BF16, worst_out
+    return worst_out, worst_coef
+
+
+def test_llama31_8b_32k_sampled_heads():
+    shape = synth.CONFIGS[1]
+    layout = layout_of(shape, max_mid=shape.T, P=shape.T // shape.k)
+    assert layout.mid_classes == 64
+    _sampled_head_check(shape, layout, heads=(0, 7), steps=3, seed=1000)

@@ -203,3 +203,33 @@ def test_snapshot_restore():
         getattr(pair.gpu, n).copy_(snap[n])
     fa.fa_decode_attention(pair.layout, pair.gpu, q, out1, pair.ws)
     assert torch.equal(out0, out1)
+
+
+@pytest.mark.parametrize("algo", ALGOS)
+def test_many_classes_per_cta(algo):
+    """Several residue classes per CTA and per transform batch (B * H_kv large, 64 classes of 64 slots):
+    the producer and the consumers must walk the tiles of a batch in the same order."""
+    shape = synth.Shape("many_classes", B=2, layers=1, Hq=32, Hkv=8, d=128, L=3600, dtype="bf16", n_full_k=32,
+                        n_full_v=32, M=128, T=4096, L_init=4, L_local=128)
+    pair, stream = make_pair(shape, seed=11, algo=algo, P=64, max_mid=4096)
+    pair.check_state()
+    pair.check_decode(synth.queries(shape, seed=11))
+    K, V = stream.tokens(shape.L, shape.L + 3)
+    for t in range(3):
+        pair.append(K[:, t], V[:, t])
+    pair.check_decode(synth.queries(shape, seed=11, step=1, peak=4.0))
+
+
+@pytest.mark.parametrize("algo", ALGOS)
+def test_mha_48_kept_dims(algo):
+    """The MHA serving shape in small: G = 1, 48 kept / 80 compressed dims, M = 256, batch 3."""
+    shape = synth.Shape("mha48", B=3, layers=1, Hq=4, Hkv=4, d=128, L=2500, dtype="bf16", n_full_k=48, n_full_v=48,
+                        M=256, T=4096, L_init=4, L_local=256)
+    pair, stream = make_pair(shape, seed=12, algo=algo, P=32, max_mid=4096)
+    pair.check_state()
+    pair.check_decode(synth.queries(shape, seed=12))
+    K, V = stream.tokens(shape.L, shape.L + 2)
+    for t in range(2):
+        pair.append(K[:, t], V[:, t])
+    pair.check_state()
+    pair.check_decode(synth.queries(shape, seed=12, step=1))
