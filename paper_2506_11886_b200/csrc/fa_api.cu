@@ -1,6 +1,7 @@
 // Host side of the C ABI declared in include/fa.h: argument checks, buffer
 // sizes, launch plans.  Every entry point validates on the host, then launches
 // on the caller's stream; nothing here allocates device memory.
+#include <cstdlib>
 #include <cstring>
 
 #include "fa_common.cuh"
@@ -67,7 +68,7 @@ static bool fft_ok(const fa_layout& l, int gh, int* log2S) {
     if (ilog2_exact(l.period) < 0 || l.period % l.mid_classes != 0) return false;
     int S = l.period / l.mid_classes;
     int ls = ilog2_exact(S);
-    if (ls < 5 || ls > 11) return false;
+    if (ls < 5 || ls > 10) return false;
     if (l.n_coef / 2 > S) return false;                                        // every frequency needs its own bin
     if (l.n_full_k > 64 || l.n_full_v > 64 || l.head_dim > 128) return false;
     if (decode_fft_smem_bytes(make_dims(l), ls, gh, 1) > 227 * 1024) return false;
@@ -88,25 +89,32 @@ fa_status plan_decode(const fa_layout& l, DecodePlan* p) {
         p->gh = gh_fft;
         p->n_pass = (s.G + p->gh - 1) / p->gh;
         // classes are indivisible: pick the split count that minimises waves * classes per CTA
-        // (one CTA per SM), smallest count on ties to keep the partial results small
+        // with two CTAs resident per SM (phases of one overlap the other's), smallest count on
+        // ties to keep the partial results small
         const int jobs = s.B * s.Hkv * p->n_pass;
+        const int slots = 2 * kNumSms;
         int best = 1;
         long long best_cost = -1;
         for (int n = 1; n <= s.P && n <= 64; ++n) {
-            long long waves = ((long long)jobs * n + kNumSms - 1) / kNumSms;
+            long long waves = ((long long)jobs * n + slots - 1) / slots;
             long long cost = waves * ((s.P + n - 1) / n);
             if (best_cost < 0 || cost < best_cost) { best_cost = cost; best = n; }
         }
+        if (const char* e = std::getenv("FA_TUNE_NSPLIT")) { int v = std::atoi(e); if (v >= 1 && v <= s.P && v <= 64) best = v; }
         p->n_split = best;
-        // classes transformed together: enough butterflies for all consumer threads, within shared memory
+        // classes transformed together: enough butterflies for all consumer threads, while two CTAs
+        // still fit the shared memory of an SM (else one)
         const int S = s.T / s.P;
         int nb = 2048 / S;
         if (nb < 1) nb = 1;
         if (nb > 8) nb = 8;
         const int per_cta = (s.P + best - 1) / best;
         if (nb > per_cta) nb = per_cta;
+        while (nb > 1 && decode_fft_smem_bytes(s, log2S, p->gh, nb) > 113 * 1024) --nb;
+        if (const char* e = std::getenv("FA_TUNE_NB")) { int v = std::atoi(e); if (v >= 1 && v <= 8) nb = v; }
         while (nb > 1 && decode_fft_smem_bytes(s, log2S, p->gh, nb) > 227 * 1024) --nb;
         p->nb = nb;
+        if (const char* e = std::getenv("FA_TUNE_DBG")) p->dbg = std::atoi(e);
     } else {
         p->gh = s.G >= 4 ? 4 : (s.G >= 2 ? 2 : 1);
         if (s.G == 3) p->gh = 4;
@@ -278,13 +286,15 @@ fa_status fa_decode_attention(const fa_layout* layout, const fa_cache* cache, co
     CacheDev c = make_cache(*cache);
     cudaStream_t cs = static_cast<cudaStream_t>(stream);
     char* w = static_cast<char*>(ws);
-    if (launch_decode_prologue(s, c, layout->kv_dtype, p, q, w, cs) != cudaSuccess) return FA_ERR_CUDA;
-    if (p.algo == FA_DECODE_FFT) {
+    const int dbgk = std::getenv("FA_TUNE_DBGK") ? std::atoi(std::getenv("FA_TUNE_DBGK")) : 0;
+    if (!(dbgk & 1) && launch_decode_prologue(s, c, layout->kv_dtype, p, q, w, cs) != cudaSuccess) return FA_ERR_CUDA;
+    if (dbgk & 2) {
+    } else if (p.algo == FA_DECODE_FFT) {
         if (launch_decode_fft(s, c, layout->kv_dtype, p, q, w, cs) != cudaSuccess) return FA_ERR_CUDA;
     } else {
         if (launch_decode_direct(s, c, layout->kv_dtype, p, q, w, cs) != cudaSuccess) return FA_ERR_CUDA;
     }
-    if (launch_decode_epilogue(s, c, layout->kv_dtype, p, out, w, cs) != cudaSuccess) return FA_ERR_CUDA;
+    if (!(dbgk & 4) && launch_decode_epilogue(s, c, layout->kv_dtype, p, out, w, cs) != cudaSuccess) return FA_ERR_CUDA;
     return FA_OK;
 }
 

@@ -66,6 +66,7 @@ struct DecodePlan {
     int rows_pro;      // coefficient rows per prologue CTA
     int fft_log2;      // log2 of the transform length (FFT path)
     int nb;            // classes transformed together by one CTA (FFT path)
+    int dbg;
     // workspace offsets in bytes
     size_t off_u, off_ml, off_o, off_z, off_oc, off_cnt, total;
 };

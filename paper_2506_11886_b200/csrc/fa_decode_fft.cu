@@ -6,10 +6,12 @@
 //   scores   sum_m F[m][j] u[m]  = Re sum_n (u~_n e^{i theta n c}) e^{2 pi i n a / S}
 //   outputs  z_n = sum_j p_j e^{i theta n j} = sum_c e^{i theta n c} sum_a p_{c+Pa} e^{2 pi i n a / S}
 // so a class costs one length-S transform per side instead of S * k basis terms.  Two query
-// heads share one complex transform (real-pair packing); with GH = 4 heads a point is a float4.
-// The score transform runs decimation-in-frequency (natural in, digit-reversed out), the
-// probability transform decimation-in-time (digit-reversed in, natural out), both in place:
-// softmax is pointwise, so nothing is ever reordered.  NB classes are transformed together.
+// heads share one complex transform (real-pair packing).  With GH = 4 heads a point holds two
+// complex numbers stored (re0, re1, im0, im1) and all transform arithmetic runs on packed
+// fp32 pairs (add/mul/fma.f32x2).  The score transform runs decimation-in-frequency (natural
+// in, digit-reversed out), the probability transform decimation-in-time (digit-reversed in,
+// natural out), both in place: softmax is pointwise, so nothing is ever reordered.  NB classes
+// are transformed together.
 //
 // K^mu / V^mu are class-major, so the tokens of a class are one contiguous stream; a producer
 // warp brings it in with bulk (TMA) copies through a ring of shared-memory stages.  The eight
@@ -18,6 +20,10 @@
 // contraction index, V^T fragments with transposing 8x8 matrix loads, conflict-free because
 // V^mu rows are stored chunk-swizzled.  Window rows (init + local ring) are copied row by row
 // into padded shared-memory rows and take the same route.  Every wait is bounded.
+//
+// "Slot" below is the position of a head inside a point / an mma column: slot s holds head
+// hperm(s) = {0, 2, 1, 3}[s] (GH = 4) so that the packed real parts are slots 0, 1 and the
+// packed imaginary parts slots 2, 3.
 #include "fa_common.cuh"
 #include "fa_decode_ws.cuh"
 
@@ -27,10 +33,13 @@ namespace {
 constexpr int kConsumers = 256;
 constexpr int kThreads = kConsumers + 32;
 constexpr int kStageBytes = 16384;
-constexpr int kStages = 3;
+constexpr int kStages = 2;
 constexpr int kWinRowsPerTile = 48;
 constexpr uint32_t kSpinLimit = 1u << 24;
 using bf16 = __nv_bfloat16;
+typedef unsigned long long u64;
+__device__ long long g_prof[64];
+#define PROF(i) do { if (dbg & 1024) { if (tid == 0 && blockIdx.x == 1 && blockIdx.y == 0 && blockIdx.z == 0) g_prof[i] = clock64(); } } while (0)
 
 // ---- PTX wrappers -----------------------------------------------------------
 __device__ __forceinline__ uint32_t smem_addr(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -83,140 +92,178 @@ __device__ __forceinline__ void ldmatrix_x4_trans(uint32_t (&r)[4], uint32_t add
 __device__ __forceinline__ uint32_t pack_bf16(bf16 lo, bf16 hi) {
     return (uint32_t)__bfloat16_as_ushort(lo) | ((uint32_t)__bfloat16_as_ushort(hi) << 16);
 }
+__device__ __forceinline__ float ex2(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
 
-// ---- complex helpers --------------------------------------------------------
-__device__ __forceinline__ float2 cadd(float2 a, float2 b) { return make_float2(a.x + b.x, a.y + b.y); }
-__device__ __forceinline__ float2 csub(float2 a, float2 b) { return make_float2(a.x - b.x, a.y - b.y); }
-__device__ __forceinline__ float2 cmul(float2 a, float2 b) {
+// ---- packed reals: N = 2 is an fp32 pair in one 64-bit register, N = 1 a float ---------------
+template <int N> struct PR;
+template <> struct PR<2> { u64 v; };
+template <> struct PR<1> { float v; };
+__device__ __forceinline__ PR<2> pk(float a, float b) { PR<2> r; asm("mov.b64 %0, {%1,%2};" : "=l"(r.v) : "f"(a), "f"(b)); return r; }
+__device__ __forceinline__ void unpk(PR<2> x, float& a, float& b) { asm("mov.b64 {%0,%1}, %2;" : "=f"(a), "=f"(b) : "l"(x.v)); }
+__device__ __forceinline__ PR<2> operator+(PR<2> a, PR<2> b) { PR<2> r; asm("add.rn.f32x2 %0, %1, %2;" : "=l"(r.v) : "l"(a.v), "l"(b.v)); return r; }
+__device__ __forceinline__ PR<2> operator-(PR<2> a, PR<2> b) { PR<2> r; asm("sub.rn.f32x2 %0, %1, %2;" : "=l"(r.v) : "l"(a.v), "l"(b.v)); return r; }
+__device__ __forceinline__ PR<2> operator*(PR<2> a, PR<2> b) { PR<2> r; asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(r.v) : "l"(a.v), "l"(b.v)); return r; }
+__device__ __forceinline__ PR<2> pfma(PR<2> a, PR<2> b, PR<2> c) { PR<2> r; asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(r.v) : "l"(a.v), "l"(b.v), "l"(c.v)); return r; }
+__device__ __forceinline__ PR<1> operator+(PR<1> a, PR<1> b) { return PR<1>{a.v + b.v}; }
+__device__ __forceinline__ PR<1> operator-(PR<1> a, PR<1> b) { return PR<1>{a.v - b.v}; }
+__device__ __forceinline__ PR<1> operator*(PR<1> a, PR<1> b) { return PR<1>{a.v * b.v}; }
+__device__ __forceinline__ PR<1> pfma(PR<1> a, PR<1> b, PR<1> c) { return PR<1>{fmaf(a.v, b.v, c.v)}; }
+template <int N> __device__ __forceinline__ PR<N> splat(float x);
+template <> __device__ __forceinline__ PR<2> splat<2>(float x) { return pk(x, x); }
+template <> __device__ __forceinline__ PR<1> splat<1>(float x) { return PR<1>{x}; }
+
+// N complex numbers side by side.
+template <int N> struct PC { PR<N> re, im; };
+template <int N> __device__ __forceinline__ PC<N> operator+(PC<N> a, PC<N> b) { return PC<N>{a.re + b.re, a.im + b.im}; }
+template <int N> __device__ __forceinline__ PC<N> operator-(PC<N> a, PC<N> b) { return PC<N>{a.re - b.re, a.im - b.im}; }
+template <int N> __device__ __forceinline__ PC<N> cconj_add(PC<N> a, PC<N> b) { return PC<N>{a.re + b.re, a.im - b.im}; }   // a + conj(b)
+// product with one scalar complex w given as splats (wr, wi)
+template <int N> __device__ __forceinline__ PC<N> cmulw(PC<N> a, PR<N> wr, PR<N> wi) {
+    return PC<N>{(a.re * wr) - (a.im * wi), pfma(a.re, wi, a.im * wr)};
+}
+__device__ __forceinline__ float2 cmulf(float2 a, float2 b) {
     return make_float2(fmaf(a.x, b.x, -a.y * b.y), fmaf(a.x, b.y, a.y * b.x));
 }
-__device__ __forceinline__ float2 mul_i(float2 a) { return make_float2(-a.y, a.x); }
-__device__ __forceinline__ float2 conj(float2 a) { return make_float2(a.x, -a.y); }
+
+// A point of a transform buffer: N = 2 -> float4 (re0, re1, im0, im1), N = 1 -> float2 (re, im).
+template <int N> __device__ __forceinline__ PC<N> ld_pt(const float* p);
+template <> __device__ __forceinline__ PC<2> ld_pt<2>(const float* p) {
+    PC<2> r;
+    asm volatile("ld.shared.v2.b64 {%0,%1}, [%2];" : "=l"(r.re.v), "=l"(r.im.v) : "r"(smem_addr(p)) : "memory");
+    return r;
+}
+template <> __device__ __forceinline__ PC<1> ld_pt<1>(const float* p) {
+    const float2 x = *reinterpret_cast<const float2*>(p);
+    return PC<1>{PR<1>{x.x}, PR<1>{x.y}};
+}
+__device__ __forceinline__ void st_pt(float* p, PC<2> v) {
+    asm volatile("st.shared.v2.b64 [%0], {%1,%2};" ::"r"(smem_addr(p)), "l"(v.re.v), "l"(v.im.v) : "memory");
+}
+__device__ __forceinline__ void st_pt(float* p, PC<1> v) { *reinterpret_cast<float2*>(p) = make_float2(v.re.v, v.im.v); }
 
 // In-place DFTs with exponent +2 pi i / R, natural order in and out.
-__device__ __forceinline__ void dft4(float2& a0, float2& a1, float2& a2, float2& a3) {
-    float2 t0 = cadd(a0, a2), t1 = csub(a0, a2), t2 = cadd(a1, a3), t3 = mul_i(csub(a1, a3));
-    a0 = cadd(t0, t2);
-    a1 = cadd(t1, t3);
-    a2 = csub(t0, t2);
-    a3 = csub(t1, t3);
+template <int N>
+__device__ __forceinline__ void dft4(PC<N>& a0, PC<N>& a1, PC<N>& a2, PC<N>& a3) {
+    const PC<N> t0 = a0 + a2, t1 = a0 - a2, t2 = a1 + a3, d = a1 - a3;        // i * d = (-d.im, d.re)
+    a0 = t0 + t2;
+    a2 = t0 - t2;
+    a1 = PC<N>{t1.re - d.im, t1.im + d.re};
+    a3 = PC<N>{t1.re + d.im, t1.im - d.re};
 }
-template <int R>
-__device__ __forceinline__ void dft(float2 (&v)[R]) {
+template <int R, int N>
+__device__ __forceinline__ void dft(PC<N> (&v)[R]) {
     if constexpr (R == 2) {
-        float2 t = v[0];
-        v[0] = cadd(t, v[1]);
-        v[1] = csub(t, v[1]);
+        const PC<N> t = v[0];
+        v[0] = t + v[1];
+        v[1] = t - v[1];
     } else if constexpr (R == 4) {
         dft4(v[0], v[1], v[2], v[3]);
     } else {
-        constexpr float h = 0.70710678118654752440f;
+        const PR<N> h = splat<N>(0.70710678118654752440f);
         dft4(v[0], v[2], v[4], v[6]);     // even part -> E0..E3
         dft4(v[1], v[3], v[5], v[7]);     // odd part  -> O0..O3
-        float2 o1 = make_float2(h * (v[3].x - v[3].y), h * (v[3].x + v[3].y));        // w   O1
-        float2 o2 = mul_i(v[5]);                                                        // w^2 O2
-        float2 o3 = make_float2(-h * (v[7].x + v[7].y), h * (v[7].x - v[7].y));       // w^3 O3
-        float2 e0 = v[0], e1 = v[2], e2 = v[4], e3 = v[6], o0 = v[1];
-        v[0] = cadd(e0, o0); v[4] = csub(e0, o0);
-        v[1] = cadd(e1, o1); v[5] = csub(e1, o1);
-        v[2] = cadd(e2, o2); v[6] = csub(e2, o2);
-        v[3] = cadd(e3, o3); v[7] = csub(e3, o3);
+        const PC<N> o1 = PC<N>{(v[3].re - v[3].im) * h, (v[3].re + v[3].im) * h};     // w   O1, w = e^{i pi / 4}
+        const PC<N> e0 = v[0], e1 = v[2], e2 = v[4], e3 = v[6], o0 = v[1], o2 = v[5], o3 = v[7];
+        v[0] = e0 + o0; v[4] = e0 - o0;
+        v[1] = e1 + o1; v[5] = e1 - o1;
+        v[2] = PC<N>{e2.re - o2.im, e2.im + o2.re};                                    // + i O2
+        v[6] = PC<N>{e2.re + o2.im, e2.im - o2.re};
+        const PC<N> w3 = PC<N>{(o3.re + o3.im) * h, (o3.re - o3.im) * h};            // w^3 O3 = (-w3.re, w3.im)
+        v[3] = PC<N>{e3.re - w3.re, e3.im + w3.im};
+        v[7] = PC<N>{e3.re + w3.re, e3.im - w3.im};
     }
 }
 
 // Shared-memory float index of float f of a transform buffer: 16 bytes of padding after every
 // 128, which spreads strided point accesses over the banks and keeps points 16-byte aligned.
-__host__ __device__ inline int pf(int f) { return f + ((f >> 5) << 2); }
-__host__ __device__ inline int pf_size(int floats) { return floats + ((floats >> 5) << 2) + 4; }
+__host__ __device__ constexpr int pf(int f) { return f + ((f >> 5) << 2); }
+__host__ __device__ constexpr int pf_size(int floats) { return floats + ((floats >> 5) << 2) + 4; }
 
-// Radix plan of the length-2^log2S transform; identical on host and device.
-struct FftPlan {
-    int n;            // stages
-    int radix[4];
-    int len[4];       // sub-transform length entering stage s (DIF order)
-    int twoff[4];     // offset (in float2) of the stage's twiddles [q-1][j], -1 if none (len == radix)
-    int twtotal;
-};
-__host__ __device__ inline FftPlan make_fft_plan(int log2S) {
-    FftPlan p;
-    p.n = 0;
-    p.twtotal = 0;
-    int rem = log2S, L = 1 << log2S;
-    while (rem > 0) {
-        int r = (rem >= 3 && rem != 4) ? 8 : (rem >= 2 ? 4 : 2);
-        p.radix[p.n] = r;
-        p.len[p.n] = L;
-        if (L > r) { p.twoff[p.n] = p.twtotal; p.twtotal += (r - 1) * (L / r); } else p.twoff[p.n] = -1;
-        L /= r;
-        rem -= (r == 8 ? 3 : (r == 4 ? 2 : 1));
-        ++p.n;
+// Radix of the pass that handles a sub-transform of length 2^l (8 where possible, two 4s for 16).
+__host__ __device__ constexpr int radix_log2(int l) { return (l >= 3 && l != 4) ? 3 : (l >= 2 ? 2 : 1); }
+// Number of twiddles (per complex lane) of all passes from length 2^LS down to, not including, 2^l.
+__host__ __device__ constexpr int tw_offset(int LS, int l) {
+    int off = 0;
+    for (int cur = LS; cur > l;) {
+        const int rl = radix_log2(cur);
+        if (cur > rl) off += ((1 << rl) - 1) << (cur - rl);
+        cur -= rl;
     }
-    return p;
+    return off;
 }
+__host__ __device__ constexpr int tw_total(int LS) { return tw_offset(LS, 0); }
 
-// One in-place pass over nb transforms held in consecutive buffers.  DIF: butterfly, then
-// twiddle the outputs; DIT: twiddle the inputs, then butterfly.  A point holds GH / 2 complex
-// numbers (independent transforms sharing the twiddles).
-template <int R, int GH, bool DIT>
-__device__ __forceinline__ void fft_pass(float* fbuf, int fb_floats, int nb, int S, int L, const float2* tw, int tid) {
-    constexpr int NC = GH / 2;
-    const int st = L / R, per = S / R;
-    for (int item = tid; item < nb * per; item += kConsumers) {
-        const int ci = item / per, rest = item - ci * per;
-        const int blk = rest / st, j = rest - blk * st;
+// One in-place pass of radix R = 2^RL over sub-transforms of length 2^LL, for nb transforms of
+// length 2^LS held in consecutive buffers.  DIF: butterfly, then twiddle the outputs; DIT:
+// twiddle the inputs, then butterfly.  Twiddles are stored [q - 1][j] as splat pairs (wr, wi).
+template <int GH, int LS, int LL, bool DIT>
+__device__ __forceinline__ void fft_pass(float* fbuf, int fb_floats, int nb, const float* twf, int tid) {
+    constexpr int N = GH / 2;
+    constexpr int RL = radix_log2(LL), R = 1 << RL;
+    constexpr int STL = LL - RL, PERL = LS - RL;          // log2 butterflies per sub-transform / per transform
+    constexpr bool kTw = LL > RL;
+    constexpr int kTwOff = tw_offset(LS, LL);
+    for (int item = tid; item < (nb << PERL); item += kConsumers) {
+        const int ci = item >> PERL, rest = item & ((1 << PERL) - 1);
+        const int blk = rest >> STL, j = rest & ((1 << STL) - 1);
         float* base = fbuf + ci * fb_floats;
-        const int e0 = blk * L + j;
-        float2 v[NC][R];
+        const int e0 = (blk << LL) + j;
+        PC<N> v[R];
 #pragma unroll
-        for (int r = 0; r < R; ++r) {
-            const float* p = base + pf((e0 + r * st) * GH);
-            if constexpr (GH == 4) {
-                const float4 x = *reinterpret_cast<const float4*>(p);
-                v[0][r] = make_float2(x.x, x.y);
-                v[1][r] = make_float2(x.z, x.w);
-            } else {
-                v[0][r] = *reinterpret_cast<const float2*>(p);
+        for (int r = 0; r < R; ++r) v[r] = ld_pt<N>(base + pf((e0 + (r << STL)) * GH));
+        PR<N> wr[R], wi[R];
+        if constexpr (kTw) {
+#pragma unroll
+            for (int q = 1; q < R; ++q) {
+                const float2 w = *reinterpret_cast<const float2*>(twf + 2 * (kTwOff + ((q - 1) << STL) + j));
+                wr[q] = splat<N>(w.x);
+                wi[q] = splat<N>(w.y);
+            }
+            if constexpr (DIT) {
+#pragma unroll
+                for (int q = 1; q < R; ++q) v[q] = cmulw(v[q], wr[q], wi[q]);
             }
         }
-        float2 w[R];
-        if (tw) {
+        dft<R, N>(v);
+        if constexpr (kTw && !DIT) {
 #pragma unroll
-            for (int q = 1; q < R; ++q) w[q] = tw[(q - 1) * st + j];
-        }
-        if (DIT && tw) {
-#pragma unroll
-            for (int c = 0; c < NC; ++c)
-#pragma unroll
-                for (int q = 1; q < R; ++q) v[c][q] = cmul(v[c][q], w[q]);
+            for (int q = 1; q < R; ++q) v[q] = cmulw(v[q], wr[q], wi[q]);
         }
 #pragma unroll
-        for (int c = 0; c < NC; ++c) dft<R>(v[c]);
-        if (!DIT && tw) {
-#pragma unroll
-            for (int c = 0; c < NC; ++c)
-#pragma unroll
-                for (int q = 1; q < R; ++q) v[c][q] = cmul(v[c][q], w[q]);
-        }
-#pragma unroll
-        for (int r = 0; r < R; ++r) {
-            float* p = base + pf((e0 + r * st) * GH);
-            if constexpr (GH == 4) *reinterpret_cast<float4*>(p) = make_float4(v[0][r].x, v[0][r].y, v[1][r].x, v[1][r].y);
-            else *reinterpret_cast<float2*>(p) = v[0][r];
-        }
+        for (int r = 0; r < R; ++r) st_pt(base + pf((e0 + (r << STL)) * GH), v[r]);
     }
 }
 
-template <int GH, bool DIT>
-__device__ __forceinline__ void fft_run(float* fbuf, int fb_floats, int nb, int S, const FftPlan& pl, const float2* twf, int tid) {
-    for (int i = 0; i < pl.n; ++i) {
-        const int sidx = DIT ? pl.n - 1 - i : i;
-        const int R = pl.radix[sidx], L = pl.len[sidx];
-        const float2* tw = pl.twoff[sidx] >= 0 ? twf + pl.twoff[sidx] : nullptr;
-        if (R == 8) fft_pass<8, GH, DIT>(fbuf, fb_floats, nb, S, L, tw, tid);
-        else if (R == 4) fft_pass<4, GH, DIT>(fbuf, fb_floats, nb, S, L, tw, tid);
-        else fft_pass<2, GH, DIT>(fbuf, fb_floats, nb, S, L, tw, tid);
+// All passes of the transform, ending each with a barrier of the consumer warps.
+template <int GH, int LS, int LL, bool DIT>
+__device__ __forceinline__ void fft_run(float* fbuf, int fb_floats, int nb, const float* twf, int tid) {
+    constexpr int RL = radix_log2(LL);
+    if constexpr (!DIT) {
+        fft_pass<GH, LS, LL, false>(fbuf, fb_floats, nb, twf, tid);
+        consumer_sync();
+        if constexpr (LL - RL > 0) fft_run<GH, LS, LL - RL, false>(fbuf, fb_floats, nb, twf, tid);
+    } else {
+        if constexpr (LL - RL > 0) fft_run<GH, LS, LL - RL, true>(fbuf, fb_floats, nb, twf, tid);
+        fft_pass<GH, LS, LL, true>(fbuf, fb_floats, nb, twf, tid);
         consumer_sync();
     }
+}
+
+// Position of output index a after the decimation-in-frequency passes.
+template <int LS>
+__host__ __device__ constexpr int dif_pos(int a) {
+    int pos = 0;
+    for (int cur = LS; cur > 0;) {
+        const int rl = radix_log2(cur);
+        cur -= rl;
+        pos += (a & ((1 << rl) - 1)) << cur;
+        a >>= rl;
+    }
+    return pos;
 }
 
 // Physical row ranges of the logical window tokens [t0, t1): init rows, then up to two ring pieces.
@@ -248,10 +295,11 @@ struct FftSmem {
     int stages_off, fbuf_off, pbt_off, twf_off, rev_off, E_off, ut_off, z_off, o_off, red_off, zero_off, total;
     int fb_floats, pbs;
 };
-__host__ __device__ inline FftSmem fft_smem_layout(int S, int log2S, int k, int GH, int NB, int d) {
+__host__ __device__ inline FftSmem fft_smem_layout(int log2S, int k, int GH, int NB, int d) {
+    const int S = 1 << log2S;
     FftSmem L;
     L.fb_floats = pf_size(S * GH);
-    L.pbs = S + 8;                                        // bf16 per (class, head) row of rounded probabilities
+    L.pbs = S + 8;                                        // bf16 per (class, slot) row of rounded probabilities
     int off = 256;                                        // mbarriers + flags
     L.zero_off = off; off += 16;
     off = (off + 127) / 128 * 128;
@@ -260,7 +308,7 @@ __host__ __device__ inline FftSmem fft_smem_layout(int S, int log2S, int k, int 
     off = (off + 15) / 16 * 16;
     L.pbt_off = off; off += 2 * NB * GH * L.pbs;
     off = (off + 15) / 16 * 16;
-    L.twf_off = off; off += 8 * (make_fft_plan(log2S).twtotal + 1);
+    L.twf_off = off; off += 8 * (tw_total(log2S) + 1);
     L.rev_off = off; off += 2 * S;
     off = (off + 15) / 16 * 16;
     L.E_off = off; off += 8 * k;
@@ -272,29 +320,32 @@ __host__ __device__ inline FftSmem fft_smem_layout(int S, int log2S, int k, int 
     return L;
 }
 
-// GH query heads per CTA (2 or 4).
-template <int GH>
-__global__ void __launch_bounds__(kThreads, 1) decode_fft_kernel(Dims s, CacheDev c, DecodePlan p, const bf16* __restrict__ q,
+template <int GH> __host__ __device__ constexpr int hperm(int s) { return GH == 4 ? (((s & 1) << 1) | (s >> 1)) : s; }
+
+// GH query heads per CTA (2 or 4), transform length S = 2^LS.
+template <int GH, int LS>
+__global__ void __launch_bounds__(kThreads, 2) decode_fft_kernel(Dims s, CacheDev c, DecodePlan p, const bf16* __restrict__ q,
                                                                   char* wsp) {
-    constexpr int NC = GH / 2;
+    constexpr int N = GH / 2;
+    constexpr int S = 1 << LS;
     extern __shared__ __align__(128) unsigned char smem_raw[];
     Ws ws = ws_view(wsp, p);
-    const int S = s.T / s.P, log2S = p.fft_log2, NB = p.nb;
-    const FftSmem L = fft_smem_layout(S, log2S, s.k, GH, NB, s.d);
-    const FftPlan pl = make_fft_plan(log2S);
+    const int NB = p.nb;
+    const int dbg = p.dbg;
+    const FftSmem L = fft_smem_layout(LS, s.k, GH, NB, s.d);
     uint64_t* full = reinterpret_cast<uint64_t*>(smem_raw);
     uint64_t* empty = full + kStages;
     volatile int* fail = reinterpret_cast<volatile int*>(smem_raw + 128);
     unsigned char* zero16 = smem_raw + L.zero_off;
     unsigned char* stages = smem_raw + L.stages_off;
     float* fbuf = reinterpret_cast<float*>(smem_raw + L.fbuf_off);        // [NB][fb_floats] points of GH floats
-    bf16* pbt = reinterpret_cast<bf16*>(smem_raw + L.pbt_off);           // [NB][GH][pbs]
-    float2* twf = reinterpret_cast<float2*>(smem_raw + L.twf_off);        // stage twiddles
-    uint16_t* rev = reinterpret_cast<uint16_t*>(smem_raw + L.rev_off);    // slot -> position after the DIF
+    bf16* pbt = reinterpret_cast<bf16*>(smem_raw + L.pbt_off);           // [NB][GH slots][pbs]
+    float* twf = reinterpret_cast<float*>(smem_raw + L.twf_off);          // pass twiddles (float2 each)
+    uint16_t* rev = reinterpret_cast<uint16_t*>(smem_raw + L.rev_off);    // slot -> point after the DIF passes
     float2* E = reinterpret_cast<float2*>(smem_raw + L.E_off);            // e^{i theta n}
-    float2* ut = reinterpret_cast<float2*>(smem_raw + L.ut_off);          // [k][GH] (1/2) u~
-    float2* z_s = reinterpret_cast<float2*>(smem_raw + L.z_off);          // [k][GH]
-    float* o_s = reinterpret_cast<float*>(smem_raw + L.o_off);            // [GH][d]
+    float* ut = reinterpret_cast<float*>(smem_raw + L.ut_off);            // [k] (A.re, A.im, B.re, B.im) x N: (1/2) u~
+    float* z_s = reinterpret_cast<float*>(smem_raw + L.z_off);            // [k] same packing
+    float* o_s = reinterpret_cast<float*>(smem_raw + L.o_off);            // [GH heads][d]
     float* red_s = reinterpret_cast<float*>(smem_raw + L.red_off);        // [8][GH] + l_s[GH]
     const int fb_floats = L.fb_floats, pbs = L.pbs;
 
@@ -304,18 +355,20 @@ __global__ void __launch_bounds__(kThreads, 1) decode_fft_kernel(Dims s, CacheDe
     const int g_first = h * s.G + pass * GH;
     const int ng = min(GH, s.G - pass * GH);
     const int tid = threadIdx.x;
+    const int log2P = 31 - __clz(s.P);
 
     const int n_init = c.state[kStateStride * b + 0], n_local = c.state[kStateStride * b + 1];
     const int n_mid = min(c.state[kStateStride * b + 2], s.max_mid), head = c.state[kStateStride * b + 3];
     const int c0 = (int)((long long)split * s.P / p.n_split), c1 = (int)((long long)(split + 1) * s.P / p.n_split);
     const int n_win = n_init + n_local;
     const int w0 = (int)((long long)split * n_win / p.n_split), w1 = (int)((long long)(split + 1) * n_win / p.n_split);
+    auto n_of_class = [&](int cls) { return cls < n_mid ? (n_mid - cls + s.P - 1) >> log2P : 0; };
 
     const int rowb_k = s.nfk * 2, rowb_v = s.nfv * 2, rowb_w = s.d * 2;
     const int rbw_pad = rowb_w + 16;                                       // padded window row in shared memory
     const int ts_k = rowb_k ? (kStageBytes / rowb_k) & ~15 : 0, ts_v = rowb_v ? (kStageBytes / rowb_v) & ~15 : 0;
     const int ts_w = kWinRowsPerTile;
-    const int wchunk = S;
+    constexpr int wchunk = S;
 
     if (tid == 0) {
         for (int i = 0; i < kStages; ++i) { mbar_init(full + i, 1); mbar_init(empty + i, 8); }
@@ -325,8 +378,10 @@ __global__ void __launch_bounds__(kThreads, 1) decode_fft_kernel(Dims s, CacheDe
     // stale shared memory must hold finite numbers: rows past the end of a tile are multiplied by p = 0
     for (int i = tid; i < (kStages * kStageBytes) / 16; i += kThreads) reinterpret_cast<uint4*>(stages)[i] = make_uint4(0, 0, 0, 0);
     if (tid < 4) reinterpret_cast<uint32_t*>(zero16)[tid] = 0;
+    PROF(0);
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     __syncthreads();
+    PROF(1);
 
     // ============================ producer warp =================================
     if (tid >= kConsumers) {
@@ -345,8 +400,9 @@ __global__ void __launch_bounds__(kThreads, 1) decode_fft_kernel(Dims s, CacheDe
                 for (int side = 0; side < 2; ++side) {
                     const int ts = side == 0 ? ts_k : ts_v, rowb = side == 0 ? rowb_k : rowb_v;
                     if (!ts) continue;
+                    if (dbg & (side == 0 ? 2 : 8)) continue;
                     for (int cls = cb; cls < cb + nb; ++cls) {
-                        const int n_c = cls < n_mid ? (n_mid - cls + s.P - 1) / s.P : 0;
+                        const int n_c = n_of_class(cls);
                         for (int a0 = 0; a0 < n_c; a0 += ts) {
                             const uint32_t bytes = (uint32_t)(min(ts, n_c - a0) * rowb);
                             const bf16* src = side == 0 ? mid_row<bf16>(c.k_mid, s, b, h, cls, a0, s.nfk)
@@ -357,7 +413,23 @@ __global__ void __launch_bounds__(kThreads, 1) decode_fft_kernel(Dims s, CacheDe
                     }
                 }
             }
-            for (int t0 = w0; t0 < w1; t0 += wchunk) {
+        }
+        // window rows: one bulk copy per row into padded shared-memory rows, issued by all lanes
+        {
+            const int plane = tid - kConsumers;
+            __syncwarp();                                 // lane 0 has issued every class tile
+            int it = 0;
+            // recount the class tiles so that the ring position continues where lane 0 stopped
+            for (int cb = c0; cb < c1; cb += NB) {
+                const int nb = min(NB, c1 - cb);
+                for (int side = 0; side < 2; ++side) {
+                    const int ts = side == 0 ? ts_k : ts_v;
+                    if (!ts || (dbg & (side == 0 ? 2 : 8))) continue;
+                    for (int cls = cb; cls < cb + nb; ++cls) it += (n_of_class(cls) + ts - 1) / ts;
+                }
+            }
+            __syncwarp();
+            for (int t0 = w0; t0 < w1 && !(dbg & 32); t0 += wchunk) {
                 const WinSegs sg = win_segments(t0, min(w1, t0 + wchunk), n_init, n_local, head, s.l_local);
                 for (int side = 0; side < 2; ++side)
                     for (int i = 0; i < sg.n; ++i)
@@ -366,9 +438,19 @@ __global__ void __launch_bounds__(kThreads, 1) decode_fft_kernel(Dims s, CacheDe
                             void* base = sg.buf[i] == 0 ? (side == 0 ? c.k_init : c.v_init) : (side == 0 ? c.k_local : c.v_local);
                             const int rows = sg.buf[i] == 0 ? s.l_init : s.l_local;
                             const bf16* src = win_row<bf16>(base, s, b, h, rows, sg.row[i] + r0);
-                            if (unsigned char* dst = acquire((uint32_t)(nt * rowb_w)))
-                                for (int r = 0; r < nt; ++r)
-                                    bulk_g2s(dst + (size_t)r * rbw_pad, src + (size_t)r * s.d, (uint32_t)rowb_w, full + it % kStages);
+                            const int st = it % kStages;
+                            int ok = 1;
+                            if (plane == 0) {
+                                if (it >= kStages) mbar_wait(empty + st, ((it / kStages) - 1) & 1, fail, c.status);
+                                ok = !*fail;
+                                if (ok) mbar_expect_tx(full + st, (uint32_t)(nt * rowb_w));
+                            }
+                            ok = __shfl_sync(0xffffffffu, ok, 0);
+                            if (ok) {
+                                unsigned char* dst = stages + (size_t)st * kStageBytes;
+                                for (int r = plane; r < nt; r += 32)
+                                    bulk_g2s(dst + (size_t)r * rbw_pad, src + (size_t)r * s.d, (uint32_t)rowb_w, full + st);
+                            }
                             ++it;
                         }
             }
@@ -389,56 +471,65 @@ __global__ void __launch_bounds__(kThreads, 1) decode_fft_kernel(Dims s, CacheDe
         sincospif(2.0f * (float)i / (float)s.T, &sn, &cs);
         E[i] = make_float2(cs, sn);
     }
-    for (int i = tid; i < s.k * GH; i += kConsumers) {
-        const int n = i / GH, g = i - n * GH;
-        float2 v = make_float2(0.f, 0.f);
-        if (g < ng && s.dck > 0) {
-            const float* u = ws.u + ((size_t)b * s.Hq + g_first + g) * s.M;
-            v = make_float2(0.5f * u[2 * n], -0.5f * u[2 * n + 1]);
+    // ut[n] = (A.re, A.im, B.re, B.im), A = heads of the real slots, B = heads of the imaginary slots;
+    // all loads of an entry are issued together
+    for (int n = tid; n < s.k; n += kConsumers) {
+        float2 uv[GH];
+#pragma unroll
+        for (int sl = 0; sl < GH; ++sl) {
+            const int g = hperm<GH>(sl);
+            uv[sl] = make_float2(0.f, 0.f);
+            if (g < ng && s.dck > 0) uv[sl] = *reinterpret_cast<const float2*>(ws.u + ((size_t)b * s.Hq + g_first + g) * s.M + 2 * n);
         }
-        ut[i] = v;
-        z_s[i] = make_float2(0.f, 0.f);
-    }
-    for (int sidx = 0; sidx < pl.n; ++sidx) {
-        if (pl.twoff[sidx] < 0) continue;
-        const int R = pl.radix[sidx], Ls = pl.len[sidx], st = Ls / R;
-        for (int i = tid; i < (R - 1) * st; i += kConsumers) {
-            const int qm1 = i / st, j = i - qm1 * st;
-            float sn, cs;
-            sincospif(2.0f * (float)(((qm1 + 1) * j) & (Ls - 1)) / (float)Ls, &sn, &cs);
-            twf[pl.twoff[sidx] + i] = make_float2(cs, sn);
+        float* e = ut + n * 2 * GH;
+        float* zz = z_s + n * 2 * GH;
+#pragma unroll
+        for (int sl = 0; sl < GH; ++sl) {
+            const int ab = sl / N, ln = sl - ab * N;
+            e[(2 * ab) * N + ln] = 0.5f * uv[sl].x;
+            e[(2 * ab + 1) * N + ln] = -0.5f * uv[sl].y;
+            zz[(2 * ab) * N + ln] = 0.f;
+            zz[(2 * ab + 1) * N + ln] = 0.f;
         }
     }
-    for (int a = tid; a < S; a += kConsumers) {
-        int kk = a, pos = 0, Lc = S;
-        for (int sidx = 0; sidx < pl.n; ++sidx) {
-            const int R = pl.radix[sidx];
-            Lc /= R;
-            pos += (kk % R) * Lc;
-            kk /= R;
+    for (int l = LS; l > 0;) {
+        const int rl = radix_log2(l), R = 1 << rl, st = 1 << (l - rl);
+        if (l > rl) {
+            const int off = tw_offset(LS, l);
+            for (int i = tid; i < (R - 1) * st; i += kConsumers) {
+                const int qm1 = i / st, j = i - qm1 * st;
+                float sn, cs;
+                sincospif(2.0f * (float)(((qm1 + 1) * j) & ((1 << l) - 1)) / (float)(1 << l), &sn, &cs);
+                reinterpret_cast<float2*>(twf)[off + i] = make_float2(cs, sn);
+            }
         }
-        rev[a] = (uint16_t)pos;
+        l -= rl;
     }
+    for (int a = tid; a < S; a += kConsumers) rev[a] = (uint16_t)dif_pos<LS>(a);
     if (tid < GH + 8) red_s[8 * GH + tid] = 0.f;
 
-    // B fragments of q for the kept K dims: round rd covers pieces 4 rd + tq of a row, two k-steps each
+    // B fragments of q for the kept K dims: column gq is slot gq = head hperm(gq);
+    // round rd covers pieces 4 rd + tq of a row, two k-steps each
+    const int my_head = hperm<GH>(gq & (GH - 1));
+    const bool col_on = gq < GH && my_head < ng;
+    const bf16* qrow = q + ((size_t)b * s.Hq + g_first + my_head) * s.d;
     uint32_t qk[2][2][2];
     {
         const int32_t* idf_k = c.idx_full_k + (size_t)h * s.nfk;
-        const bf16* qrow = q + ((size_t)b * s.Hq + g_first + gq) * s.d;
 #pragma unroll
         for (int rd = 0; rd < 2; ++rd)
 #pragma unroll
             for (int ks = 0; ks < 2; ++ks) {
                 const int piece = 4 * rd + tq, e0 = 8 * piece + 4 * ks;
-                const bool on = gq < ng && piece < npk;
+                const bool on = col_on && piece < npk;
                 qk[rd][ks][0] = on ? pack_bf16(qrow[idf_k[e0]], qrow[idf_k[e0 + 1]]) : 0u;
                 qk[rd][ks][1] = on ? pack_bf16(qrow[idf_k[e0 + 2]], qrow[idf_k[e0 + 3]]) : 0u;
             }
     }
     consumer_sync();
+    PROF(2);
 
-    float m_run[GH], l_acc[GH];
+    float m_run[GH], l_acc[GH];                           // per slot
 #pragma unroll
     for (int g = 0; g < GH; ++g) { m_run[g] = kNegBig; l_acc[g] = 0.f; }
     int it = 0;                                           // tile counter, mirrors the producer's
@@ -453,7 +544,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_fft_kernel(Dims s, CacheDe
         if (lane == 0) mbar_arrive(empty + (it % kStages));
         ++it;
     };
-    // per-head maximum over per-thread partial maxima, broadcast to every consumer thread
+    // per-slot maximum over per-thread partial maxima, broadcast to every consumer thread
     auto block_max = [&](float (&mx)[GH]) {
 #pragma unroll
         for (int g = 0; g < GH; ++g) {
@@ -471,7 +562,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_fft_kernel(Dims s, CacheDe
             mx[g] = r;
         }
     };
-    auto load_point = [&](const float* pt, float (&v)[GH]) {
+    auto load_vals = [&](const float* pt, float (&v)[GH]) {
         if constexpr (GH == 4) {
             const float4 x = *reinterpret_cast<const float4*>(pt);
             v[0] = x.x; v[1] = x.y; v[2] = x.z; v[3] = x.w;
@@ -480,9 +571,37 @@ __global__ void __launch_bounds__(kThreads, 1) decode_fft_kernel(Dims s, CacheDe
             v[0] = x.x; v[1] = x.y;
         }
     };
-    auto store_point = [&](float* pt, const float (&v)[GH]) {
+    auto store_vals = [&](float* pt, const float (&v)[GH]) {
         if constexpr (GH == 4) *reinterpret_cast<float4*>(pt) = make_float4(v[0], v[1], v[2], v[3]);
         else *reinterpret_cast<float2*>(pt) = make_float2(v[0], v[1]);
+    };
+    // entry n of ut / z_s as two packed complex numbers
+    auto ld_entry = [&](const float* tab, int n, PC<N>& A, PC<N>& B) {
+        if constexpr (N == 2) {
+            const float4 x = *reinterpret_cast<const float4*>(tab + n * 8), y = *reinterpret_cast<const float4*>(tab + n * 8 + 4);
+            A = PC<N>{pk(x.x, x.y), pk(x.z, x.w)};
+            B = PC<N>{pk(y.x, y.y), pk(y.z, y.w)};
+        } else {
+            const float4 x = *reinterpret_cast<const float4*>(tab + n * 4);
+            A = PC<N>{PR<1>{x.x}, PR<1>{x.y}};
+            B = PC<N>{PR<1>{x.z}, PR<1>{x.w}};
+        }
+    };
+    auto st_entry = [&](float* tab, int n, const PC<N>& A, const PC<N>& B) {
+        if constexpr (N == 2) {
+            float a0, a1, a2, a3, b0, b1, b2, b3;
+            unpk(A.re, a0, a1); unpk(A.im, a2, a3); unpk(B.re, b0, b1); unpk(B.im, b2, b3);
+            *reinterpret_cast<float4*>(tab + n * 8) = make_float4(a0, a1, a2, a3);
+            *reinterpret_cast<float4*>(tab + n * 8 + 4) = make_float4(b0, b1, b2, b3);
+        } else {
+            *reinterpret_cast<float4*>(tab + n * 4) = make_float4(A.re.v, A.im.v, B.re.v, B.im.v);
+        }
+    };
+    const PC<N> czero = PC<N>{splat<N>(0.f), splat<N>(0.f)};
+    auto seed_tw = [&](int n, int cls) -> float2 {
+        float sn, cs;
+        sincospif(2.0f * (float)((n * cls) & (s.T - 1)) / (float)s.T, &sn, &cs);
+        return make_float2(cs, sn);
     };
 
     // ------------------------------ middle classes ------------------------------
@@ -496,59 +615,50 @@ __global__ void __launch_bounds__(kThreads, 1) decode_fft_kernel(Dims s, CacheDe
 
         for (int cb = c0; cb < c1; cb += NB) {
             const int nb = min(NB, c1 - cb);
-            auto n_of = [&](int ci) { const int cls = cb + ci; return cls < n_mid ? (n_mid - cls + s.P - 1) / s.P : 0; };
-            if (n_of(0) == 0) break;                      // classes are filled in order: nothing further on
+            if (n_of_class(cb) == 0) break;               // classes are filled in order: nothing further on
 
-            // packed Hermitian spectra of the nb classes: X_m = V^{g0}_m + i V^{g1}_m (and g2, g3)
-            if (s.dck > 0) {
-                for (int m = tid; m <= S / 2; m += kConsumers) {
-                    const int mc = (S - m) & (S - 1);
-                    float2 um[GH], uc[GH];
-#pragma unroll
-                    for (int g = 0; g < GH; ++g) {
-                        um[g] = m < s.k ? ut[m * GH + g] : make_float2(0.f, 0.f);
-                        uc[g] = mc < s.k ? ut[mc * GH + g] : make_float2(0.f, 0.f);
-                    }
-                    float2 twm, twc, em = make_float2(1.f, 0.f), ec = make_float2(1.f, 0.f);
-                    {
-                        float sn, cs;
-                        sincospif(2.0f * (float)((m * cb) & (s.T - 1)) / (float)s.T, &sn, &cs);
-                        twm = make_float2(cs, sn);
-                        sincospif(2.0f * (float)((mc * cb) & (s.T - 1)) / (float)s.T, &sn, &cs);
-                        twc = make_float2(cs, sn);
-                        if (m < s.k) em = E[m];
-                        if (mc < s.k) ec = E[mc];
-                    }
+            // packed Hermitian spectra of the nb classes: X_m = V^A_m + i V^B_m per complex lane,
+            // V_m = v_m + conj(v_{S-m}), v_n = (1/2) u~_n e^{i theta n c}.  Pair 0 is bins (0, S/2).
+            if (s.dck > 0 && !(dbg & 1)) {
+                for (int pr = tid; pr < S / 2; pr += kConsumers) {
+                    const int m = pr, mc = pr == 0 ? S / 2 : S - pr;
+                    PC<N> Am = czero, Bm = czero, Ac = czero, Bc = czero;
+                    float2 em = make_float2(1.f, 0.f), ec = make_float2(1.f, 0.f);
+                    if (m < s.k) { ld_entry(ut, m, Am, Bm); em = E[m]; }
+                    if (mc < s.k) { ld_entry(ut, mc, Ac, Bc); ec = E[mc]; }
+                    float2 twm = seed_tw(m, cb), twc = seed_tw(mc, cb);
                     for (int ci = 0; ci < nb; ++ci) {
-                        float2 vm[GH];
-#pragma unroll
-                        for (int g = 0; g < GH; ++g) vm[g] = cadd(cmul(um[g], twm), conj(cmul(uc[g], twc)));
-                        float xm[GH], xc[GH];
-#pragma unroll
-                        for (int cl = 0; cl < NC; ++cl) {
-                            xm[2 * cl] = vm[2 * cl].x - vm[2 * cl + 1].y;
-                            xm[2 * cl + 1] = vm[2 * cl].y + vm[2 * cl + 1].x;
-                            xc[2 * cl] = vm[2 * cl].x + vm[2 * cl + 1].y;
-                            xc[2 * cl + 1] = vm[2 * cl + 1].x - vm[2 * cl].y;
-                        }
+                        const PR<N> wmr = splat<N>(twm.x), wmi = splat<N>(twm.y), wcr = splat<N>(twc.x), wci = splat<N>(twc.y);
+                        const PC<N> vAm = cmulw(Am, wmr, wmi), vBm = cmulw(Bm, wmr, wmi);
+                        const PC<N> vAc = cmulw(Ac, wcr, wci), vBc = cmulw(Bc, wcr, wci);
                         float* base = fbuf + ci * fb_floats;
-                        store_point(base + pf(m * GH), xm);
-                        if (mc != m) store_point(base + pf(mc * GH), xc);
-                        twm = cmul(twm, em);
-                        twc = cmul(twc, ec);
+                        if (pr != 0) {
+                            const PC<N> VA = cconj_add(vAm, vAc), VB = cconj_add(vBm, vBc);
+                            st_pt(base + pf(m * GH), PC<N>{VA.re - VB.im, VA.im + VB.re});        // V^A + i V^B
+                            st_pt(base + pf(mc * GH), PC<N>{VA.re + VB.im, VB.re - VA.im});       // conj(V^A) + i conj(V^B)
+                        } else {                                                                   // self-conjugate bins
+                            const PC<N> VA0 = cconj_add(vAm, vAm), VB0 = cconj_add(vBm, vBm);
+                            const PC<N> VA1 = cconj_add(vAc, vAc), VB1 = cconj_add(vBc, vBc);
+                            st_pt(base + pf(0), PC<N>{VA0.re - VB0.im, VA0.im + VB0.re});
+                            st_pt(base + pf((S / 2) * GH), PC<N>{VA1.re - VB1.im, VA1.im + VB1.re});
+                        }
+                        twm = cmulf(twm, em);
+                        twc = cmulf(twc, ec);
                     }
                 }
                 consumer_sync();
-                fft_run<GH, false>(fbuf, fb_floats, nb, S, pl, twf, tid);     // scores of slot a at point rev[a]
+                if (cb == c0) PROF(3);
+                fft_run<GH, LS, LS, false>(fbuf, fb_floats, nb, twf, tid);        // score of slot a at point rev[a]
+                if (cb == c0) PROF(4);
             } else {
                 for (int i = tid; i < nb * fb_floats; i += kConsumers) fbuf[i] = 0.f;
                 consumer_sync();
             }
 
             // kept dims: s = sl2 * (q_u . K^mu) + compressed part, 16 tokens per mma
-            if (ts_k) {
+            if (ts_k && !(dbg & 2)) {
                 for (int ci = 0; ci < nb; ++ci) {
-                    const int n_c = n_of(ci);
+                    const int n_c = n_of_class(cb + ci);
                     float* base = fbuf + ci * fb_floats;
                     for (int a0 = 0; a0 < n_c; a0 += ts_k) {
                         const int nt = min(ts_k, n_c - a0);
@@ -574,12 +684,12 @@ __global__ void __launch_bounds__(kThreads, 1) decode_fft_kernel(Dims s, CacheDe
                                 const int a_lo = a0 + grp * 16 + gq, a_hi = a_lo + 8;
                                 if (a_lo < n_c) {
                                     float2* dst = reinterpret_cast<float2*>(base + pf(rev[a_lo] * GH + 2 * tq));
-                                    float2 v = *dst;
+                                    const float2 v = *dst;
                                     *dst = make_float2(fmaf(d4[0], sl2, v.x), fmaf(d4[1], sl2, v.y));
                                 }
                                 if (a_hi < n_c) {
                                     float2* dst = reinterpret_cast<float2*>(base + pf(rev[a_hi] * GH + 2 * tq));
-                                    float2 v = *dst;
+                                    const float2 v = *dst;
                                     *dst = make_float2(fmaf(d4[2], sl2, v.x), fmaf(d4[3], sl2, v.y));
                                 }
                             }
@@ -589,16 +699,17 @@ __global__ void __launch_bounds__(kThreads, 1) decode_fft_kernel(Dims s, CacheDe
                 }
             }
             consumer_sync();
+            if (cb == c0) PROF(5);
 
             // online softmax over the batch
             float mx[GH], alpha[GH];
 #pragma unroll
             for (int g = 0; g < GH; ++g) mx[g] = kNegBig;
-            for (int i = tid; i < nb * S; i += kConsumers) {
-                const int ci = i / S, a = i - ci * S;
-                if (a < n_of(ci)) {
+            for (int i = tid; i < (nb << LS) && !(dbg & 4); i += kConsumers) {
+                const int ci = i >> LS, a = i & (S - 1);
+                if (a < n_of_class(cb + ci)) {
                     float v[GH];
-                    load_point(fbuf + ci * fb_floats + pf(rev[a] * GH), v);
+                    load_vals(fbuf + ci * fb_floats + pf(rev[a] * GH), v);
 #pragma unroll
                     for (int g = 0; g < GH; ++g) mx[g] = fmaxf(mx[g], v[g]);
                 }
@@ -607,38 +718,37 @@ __global__ void __launch_bounds__(kThreads, 1) decode_fft_kernel(Dims s, CacheDe
 #pragma unroll
             for (int g = 0; g < GH; ++g) {
                 const float m_new = fmaxf(m_run[g], mx[g]);
-                alpha[g] = exp2f(m_run[g] - m_new);
+                alpha[g] = ex2(m_run[g] - m_new);
                 m_run[g] = m_new;
                 l_acc[g] *= alpha[g];
             }
-            for (int i = tid; i < nb * S; i += kConsumers) {
-                const int ci = i / S, a = i - ci * S;
+            for (int i = tid; i < (nb << LS) && !(dbg & 4); i += kConsumers) {
+                const int ci = i >> LS, a = i & (S - 1);
                 float* pt = fbuf + ci * fb_floats + pf(rev[a] * GH);
                 float v[GH];
-                load_point(pt, v);
-                const bool ok = a < n_of(ci);
+                load_vals(pt, v);
+                const bool ok = a < n_of_class(cb + ci);
 #pragma unroll
                 for (int g = 0; g < GH; ++g) {
-                    v[g] = ok ? exp2f(v[g] - m_run[g]) : 0.f;
+                    v[g] = ok ? ex2(v[g] - m_run[g]) : 0.f;
                     l_acc[g] += v[g];
                     pbt[(ci * GH + g) * pbs + a] = __float2bfloat16_rn(v[g]);
                 }
-                store_point(pt, v);
+                store_vals(pt, v);
             }
+            {
+                const float al = alpha[(2 * tq) & (GH - 1)], ah = alpha[(2 * tq + 1) & (GH - 1)];
 #pragma unroll
-            for (int mt = 0; mt < 4; ++mt) {
-                acc[mt][0] *= alpha[(2 * tq) & (GH - 1)];
-                acc[mt][1] *= alpha[(2 * tq + 1) & (GH - 1)];
-                acc[mt][2] *= alpha[(2 * tq) & (GH - 1)];
-                acc[mt][3] *= alpha[(2 * tq + 1) & (GH - 1)];
+                for (int mt = 0; mt < 4; ++mt) { acc[mt][0] *= al; acc[mt][1] *= ah; acc[mt][2] *= al; acc[mt][3] *= ah; }
             }
             consumer_sync();
+            if (cb == c0) PROF(6);
 
-            // o^u[dim][head] += V^mu^T p, 16 tokens per mma
-            if (ts_v) {
+            // o^u[dim][slot] += V^mu^T p, 16 tokens per mma
+            if (ts_v && !(dbg & 8)) {
                 for (int ci = 0; ci < nb; ++ci) {
-                    const int n_c = n_of(ci);
-                    const bf16* prow = pbt + (size_t)(ci * GH + gq) * pbs;
+                    const int n_c = n_of_class(cb + ci);
+                    const bf16* prow = pbt + (size_t)(ci * GH + (gq & (GH - 1))) * pbs;
                     for (int a0 = 0; a0 < n_c; a0 += ts_v) {
                         const int nt = min(ts_v, n_c - a0);
                         const unsigned char* tile = wait_tile();
@@ -668,53 +778,58 @@ __global__ void __launch_bounds__(kThreads, 1) decode_fft_kernel(Dims s, CacheDe
                 }
             }
 
+            if (cb == c0) PROF(7);
             // z_n = alpha z_n + sum_c e^{i theta n c} Y^c_n, Y^c = transform of the packed probabilities
-            if (s.dcv > 0) {
-                fft_run<GH, true>(fbuf, fb_floats, nb, S, pl, twf, tid);
-                for (int m = tid; m <= S / 2; m += kConsumers) {
-                    const int mc = (S - m) & (S - 1);
+            if (s.dcv > 0 && !(dbg & 16)) {
+                fft_run<GH, LS, LS, true>(fbuf, fb_floats, nb, twf, tid);
+                if (cb == c0) PROF(8);
+                PR<N> alA, alB;
+                if constexpr (N == 2) { alA = pk(alpha[0], alpha[1]); alB = pk(alpha[2], alpha[3]); }
+                else { alA = PR<1>{alpha[0]}; alB = PR<1>{alpha[1]}; }
+                const PR<N> half = splat<N>(0.5f);
+                for (int pr = tid; pr < S / 2; pr += kConsumers) {
+                    const int m = pr, mc = pr == 0 ? S / 2 : S - pr;
                     if (m >= s.k && mc >= s.k) continue;
-                    float2 twm, twc, em = make_float2(1.f, 0.f), ec = make_float2(1.f, 0.f);
-                    {
-                        float sn, cs;
-                        sincospif(2.0f * (float)((m * cb) & (s.T - 1)) / (float)s.T, &sn, &cs);
-                        twm = make_float2(cs, sn);
-                        sincospif(2.0f * (float)((mc * cb) & (s.T - 1)) / (float)s.T, &sn, &cs);
-                        twc = make_float2(cs, sn);
-                        if (m < s.k) em = E[m];
-                        if (mc < s.k) ec = E[mc];
-                    }
-                    float2 zm[GH], zc[GH];
-#pragma unroll
-                    for (int g = 0; g < GH; ++g) { zm[g] = make_float2(0.f, 0.f); zc[g] = make_float2(0.f, 0.f); }
+                    float2 em = make_float2(1.f, 0.f), ec = make_float2(1.f, 0.f);
+                    if (m < s.k) em = E[m];
+                    if (mc < s.k) ec = E[mc];
+                    float2 twm = seed_tw(m, cb), twc = seed_tw(mc, cb);
+                    PC<N> zAm = czero, zBm = czero, zAc = czero, zBc = czero;
                     for (int ci = 0; ci < nb; ++ci) {
                         const float* base = fbuf + ci * fb_floats;
-                        float ya[GH], yb[GH];
-                        load_point(base + pf(m * GH), ya);
-                        load_point(base + pf(mc * GH), yb);
-#pragma unroll
-                        for (int cl = 0; cl < NC; ++cl) {
-                            // heads 2cl, 2cl+1 of bin m; bin mc holds the conjugates
-                            const float2 y0 = make_float2(0.5f * (ya[2 * cl] + yb[2 * cl]), 0.5f * (ya[2 * cl + 1] - yb[2 * cl + 1]));
-                            const float2 y1 = make_float2(0.5f * (ya[2 * cl + 1] + yb[2 * cl + 1]), -0.5f * (ya[2 * cl] - yb[2 * cl]));
-                            zm[2 * cl] = cadd(zm[2 * cl], cmul(twm, y0));
-                            zm[2 * cl + 1] = cadd(zm[2 * cl + 1], cmul(twm, y1));
-                            zc[2 * cl] = cadd(zc[2 * cl], cmul(twc, conj(y0)));
-                            zc[2 * cl + 1] = cadd(zc[2 * cl + 1], cmul(twc, conj(y1)));
+                        const PC<N> ya = ld_pt<N>(base + pf(m * GH)), yb = ld_pt<N>(base + pf(mc * GH));
+                        const PR<N> wmr = splat<N>(twm.x), wmi = splat<N>(twm.y), wcr = splat<N>(twc.x), wci = splat<N>(twc.y);
+                        if (pr != 0) {
+                            // real slots: y0 = (ya + conj(yb)) / 2, imaginary slots: y1 = (ya - conj(yb)) / (2 i); bin mc holds the conjugates
+                            const PC<N> y0 = PC<N>{(ya.re + yb.re) * half, (ya.im - yb.im) * half};
+                            const PC<N> y1 = PC<N>{(ya.im + yb.im) * half, (yb.re - ya.re) * half};
+                            zAm = zAm + cmulw(y0, wmr, wmi);
+                            zBm = zBm + cmulw(y1, wmr, wmi);
+                            zAc = zAc + cmulw(PC<N>{y0.re, splat<N>(0.f) - y0.im}, wcr, wci);
+                            zBc = zBc + cmulw(PC<N>{y1.re, splat<N>(0.f) - y1.im}, wcr, wci);
+                        } else {
+                            // bins 0 and S/2 are real for each real sequence: (re, im) of the packed value are the two heads
+                            const PC<N> y0m = PC<N>{ya.re, splat<N>(0.f)}, y1m = PC<N>{ya.im, splat<N>(0.f)};
+                            const PC<N> y0c = PC<N>{yb.re, splat<N>(0.f)}, y1c = PC<N>{yb.im, splat<N>(0.f)};
+                            zAm = zAm + cmulw(y0m, wmr, wmi);
+                            zBm = zBm + cmulw(y1m, wmr, wmi);
+                            zAc = zAc + cmulw(y0c, wcr, wci);
+                            zBc = zBc + cmulw(y1c, wcr, wci);
                         }
-                        twm = cmul(twm, em);
-                        twc = cmul(twc, ec);
+                        twm = cmulf(twm, em);
+                        twc = cmulf(twc, ec);
                     }
-#pragma unroll
-                    for (int g = 0; g < GH; ++g) {
-                        if (m < s.k) {
-                            const float2 z0 = z_s[m * GH + g];
-                            z_s[m * GH + g] = make_float2(fmaf(z0.x, alpha[g], zm[g].x), fmaf(z0.y, alpha[g], zm[g].y));
-                        }
-                        if (mc < s.k && mc != m) {
-                            const float2 z0 = z_s[mc * GH + g];
-                            z_s[mc * GH + g] = make_float2(fmaf(z0.x, alpha[g], zc[g].x), fmaf(z0.y, alpha[g], zc[g].y));
-                        }
+                    if (m < s.k) {
+                        PC<N> A, B;
+                        ld_entry(z_s, m, A, B);
+                        st_entry(z_s, m, PC<N>{pfma(A.re, alA, zAm.re), pfma(A.im, alA, zAm.im)},
+                                 PC<N>{pfma(B.re, alB, zBm.re), pfma(B.im, alB, zBm.im)});
+                    }
+                    if (mc < s.k) {
+                        PC<N> A, B;
+                        ld_entry(z_s, mc, A, B);
+                        st_entry(z_s, mc, PC<N>{pfma(A.re, alA, zAc.re), pfma(A.im, alA, zAc.im)},
+                                 PC<N>{pfma(B.re, alB, zBc.re), pfma(B.im, alB, zBc.im)});
                     }
                 }
             }
@@ -723,40 +838,34 @@ __global__ void __launch_bounds__(kThreads, 1) decode_fft_kernel(Dims s, CacheDe
         // fold the per-warp output fragments into o_s at the natural positions of D^vu
         const int32_t* idf_v = c.idx_full_v + (size_t)h * s.nfv;
         if (2 * tq < GH) {
+            float* o_lo = o_s + hperm<GH>(2 * tq) * s.d;
+            float* o_hi = o_s + hperm<GH>(2 * tq + 1) * s.d;
 #pragma unroll
             for (int mt = 0; mt < 4; ++mt) {
                 const int e_lo = 16 * mt + gq, e_hi = e_lo + 8;
-                if (e_lo < s.nfv) {
-                    atomicAdd(o_s + (2 * tq) * s.d + idf_v[e_lo], acc[mt][0]);
-                    atomicAdd(o_s + (2 * tq + 1) * s.d + idf_v[e_lo], acc[mt][1]);
-                }
-                if (e_hi < s.nfv) {
-                    atomicAdd(o_s + (2 * tq) * s.d + idf_v[e_hi], acc[mt][2]);
-                    atomicAdd(o_s + (2 * tq + 1) * s.d + idf_v[e_hi], acc[mt][3]);
-                }
+                if (e_lo < s.nfv) { atomicAdd(o_lo + idf_v[e_lo], acc[mt][0]); atomicAdd(o_hi + idf_v[e_lo], acc[mt][1]); }
+                if (e_hi < s.nfv) { atomicAdd(o_lo + idf_v[e_hi], acc[mt][2]); atomicAdd(o_hi + idf_v[e_hi], acc[mt][3]); }
             }
         }
     }
     consumer_sync();
+    PROF(10);
 
     // ------------------------------ window tokens -------------------------------
-    if (w1 > w0) {
+    if (w1 > w0 && !(dbg & 32)) {
         float a_win[GH];                                  // rescale of what the classes left in o_s / z_s
 #pragma unroll
         for (int g = 0; g < GH; ++g) a_win[g] = 1.f;
         uint32_t qw[4][2][2];
-        {
-            const bf16* qrow = q + ((size_t)b * s.Hq + g_first + gq) * s.d;
 #pragma unroll
-            for (int rd = 0; rd < 4; ++rd)
+        for (int rd = 0; rd < 4; ++rd)
 #pragma unroll
-                for (int ks = 0; ks < 2; ++ks) {
-                    const int piece = 4 * rd + tq, e0 = 8 * piece + 4 * ks;
-                    const bool on = gq < ng && piece < npw;
-                    qw[rd][ks][0] = on ? pack_bf16(qrow[e0], qrow[e0 + 1]) : 0u;
-                    qw[rd][ks][1] = on ? pack_bf16(qrow[e0 + 2], qrow[e0 + 3]) : 0u;
-                }
-        }
+            for (int ks = 0; ks < 2; ++ks) {
+                const int piece = 4 * rd + tq, e0 = 8 * piece + 4 * ks;
+                const bool on = col_on && piece < npw;
+                qw[rd][ks][0] = on ? pack_bf16(qrow[e0], qrow[e0 + 1]) : 0u;
+                qw[rd][ks][1] = on ? pack_bf16(qrow[e0 + 2], qrow[e0 + 3]) : 0u;
+            }
         float accw[8][4];
 #pragma unroll
         for (int mt = 0; mt < 8; ++mt)
@@ -805,7 +914,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_fft_kernel(Dims s, CacheDe
             for (int g = 0; g < GH; ++g) mx[g] = kNegBig;
             for (int a = tid; a < n_tok; a += kConsumers) {
                 float v[GH];
-                load_point(sb + pf(a * GH), v);
+                load_vals(sb + pf(a * GH), v);
 #pragma unroll
                 for (int g = 0; g < GH; ++g) mx[g] = fmaxf(mx[g], v[g]);
             }
@@ -813,7 +922,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_fft_kernel(Dims s, CacheDe
 #pragma unroll
             for (int g = 0; g < GH; ++g) {
                 const float m_new = fmaxf(m_run[g], mx[g]);
-                alpha[g] = exp2f(m_run[g] - m_new);
+                alpha[g] = ex2(m_run[g] - m_new);
                 m_run[g] = m_new;
                 l_acc[g] *= alpha[g];
                 a_win[g] *= alpha[g];
@@ -821,23 +930,23 @@ __global__ void __launch_bounds__(kThreads, 1) decode_fft_kernel(Dims s, CacheDe
             const int n_pad = (n_tok + 15) & ~15;
             for (int a = tid; a < n_pad; a += kConsumers) {
                 float v[GH];
-                if (a < n_tok) load_point(sb + pf(a * GH), v);
+#pragma unroll
+                for (int g = 0; g < GH; ++g) v[g] = 0.f;
+                if (a < n_tok) load_vals(sb + pf(a * GH), v);
 #pragma unroll
                 for (int g = 0; g < GH; ++g) {
-                    v[g] = a < n_tok ? exp2f(v[g] - m_run[g]) : 0.f;
+                    v[g] = a < n_tok ? ex2(v[g] - m_run[g]) : 0.f;
                     l_acc[g] += v[g];
                     pb[g * pbs + a] = __float2bfloat16_rn(v[g]);
                 }
             }
+            {
+                const float al = alpha[(2 * tq) & (GH - 1)], ah = alpha[(2 * tq + 1) & (GH - 1)];
 #pragma unroll
-            for (int mt = 0; mt < 8; ++mt) {
-                accw[mt][0] *= alpha[(2 * tq) & (GH - 1)];
-                accw[mt][1] *= alpha[(2 * tq + 1) & (GH - 1)];
-                accw[mt][2] *= alpha[(2 * tq) & (GH - 1)];
-                accw[mt][3] *= alpha[(2 * tq + 1) & (GH - 1)];
+                for (int mt = 0; mt < 8; ++mt) { accw[mt][0] *= al; accw[mt][1] *= ah; accw[mt][2] *= al; accw[mt][3] *= ah; }
             }
             consumer_sync();
-            const bf16* prow = pb + (size_t)gq * pbs;
+            const bf16* prow = pb + (size_t)(gq & (GH - 1)) * pbs;
             for (int si = 0; si < sg.n; ++si)
                 for (int r0 = 0; r0 < sg.cnt[si]; r0 += ts_w) {
                     const int nt = min(ts_w, sg.cnt[si] - r0);
@@ -871,34 +980,33 @@ __global__ void __launch_bounds__(kThreads, 1) decode_fft_kernel(Dims s, CacheDe
         }
         // rescale what the classes left, then add the window fragments
         for (int i = tid; i < GH * s.d; i += kConsumers) {
+            const int g = i / s.d;                        // head
             float a = a_win[0];
 #pragma unroll
-            for (int g = 1; g < GH; ++g) if (i / s.d == g) a = a_win[g];
+            for (int sl = 1; sl < GH; ++sl) if (hperm<GH>(sl) == g) a = a_win[sl];
             o_s[i] *= a;
         }
-        for (int i = tid; i < s.k * GH; i += kConsumers) {
+        for (int i = tid; i < s.k * 2 * GH; i += kConsumers) {
+            const int f = i % (2 * GH), part = f / N, ln = f - part * N, slot = (part >> 1) * N + ln;
             float a = a_win[0];
 #pragma unroll
-            for (int g = 1; g < GH; ++g) if (i % GH == g) a = a_win[g];
-            z_s[i] = make_float2(z_s[i].x * a, z_s[i].y * a);
+            for (int sl = 1; sl < GH; ++sl) if (slot == sl) a = a_win[sl];
+            z_s[i] *= a;
         }
         consumer_sync();
         if (2 * tq < GH) {
+            float* o_lo = o_s + hperm<GH>(2 * tq) * s.d;
+            float* o_hi = o_s + hperm<GH>(2 * tq + 1) * s.d;
 #pragma unroll
             for (int mt = 0; mt < 8; ++mt) {
                 const int e_lo = 16 * mt + gq, e_hi = e_lo + 8;
-                if (e_lo < s.d) {
-                    atomicAdd(o_s + (2 * tq) * s.d + e_lo, accw[mt][0]);
-                    atomicAdd(o_s + (2 * tq + 1) * s.d + e_lo, accw[mt][1]);
-                }
-                if (e_hi < s.d) {
-                    atomicAdd(o_s + (2 * tq) * s.d + e_hi, accw[mt][2]);
-                    atomicAdd(o_s + (2 * tq + 1) * s.d + e_hi, accw[mt][3]);
-                }
+                if (e_lo < s.d) { atomicAdd(o_lo + e_lo, accw[mt][0]); atomicAdd(o_hi + e_lo, accw[mt][1]); }
+                if (e_hi < s.d) { atomicAdd(o_lo + e_hi, accw[mt][2]); atomicAdd(o_hi + e_hi, accw[mt][3]); }
             }
         }
     }
-    // sum of p per head
+    PROF(11);
+    // sum of p per slot
 #pragma unroll
     for (int g = 0; g < GH; ++g) {
         float v = l_acc[g];
@@ -913,44 +1021,66 @@ __global__ void __launch_bounds__(kThreads, 1) decode_fft_kernel(Dims s, CacheDe
         const int g = i / s.d, e = i - g * s.d;
         if (g < ng) ws.o[(((size_t)b * s.Hq + g_first + g) * p.n_split + split) * s.d + e] = o_s[i];
     }
-    for (int i = tid; i < s.k * GH; i += kConsumers) {
-        const int n = i / GH, g = i - n * GH;
-        if (g < ng) {
-            float2* dst = reinterpret_cast<float2*>(ws.z + (((size_t)b * s.Hq + g_first + g) * p.n_split + split) * s.M) + n;
-            *dst = z_s[i];
+    for (int n = tid; n < s.k; n += kConsumers) {
+        const float* e = z_s + n * 2 * GH;
+#pragma unroll
+        for (int sl = 0; sl < GH; ++sl) {
+            const int g = hperm<GH>(sl), ab = sl / N, ln = sl - ab * N;
+            if (g < ng)
+                *reinterpret_cast<float2*>(ws.z + (((size_t)b * s.Hq + g_first + g) * p.n_split + split) * s.M + 2 * n) =
+                    make_float2(e[(2 * ab) * N + ln], e[(2 * ab + 1) * N + ln]);
         }
     }
-    if (tid < ng) {
-        float* ml = ws.ml + (((size_t)b * s.Hq + g_first + tid) * p.n_split + split) * 2;
-        float mv = m_run[0];
+    if (tid < GH) {
+        const int g = hperm<GH>(tid);                     // slot tid holds head g
+        if (g < ng) {
+            PROF(12);
+            float* ml = ws.ml + (((size_t)b * s.Hq + g_first + g) * p.n_split + split) * 2;
+            float mv = m_run[0];
 #pragma unroll
-        for (int g = 1; g < GH; ++g) if (tid == g) mv = m_run[g];
-        ml[0] = mv;
-        ml[1] = red_s[8 * GH + tid];
+            for (int sl = 1; sl < GH; ++sl) if (tid == sl) mv = m_run[sl];
+            ml[0] = mv;
+            ml[1] = red_s[8 * GH + tid];
+        }
     }
 }
 
-template <int GH>
+template <int GH, int LS>
 cudaError_t launch_fft_t(const Dims& s, const CacheDev& c, const DecodePlan& p, const void* q, char* ws, cudaStream_t st) {
-    const FftSmem L = fft_smem_layout(s.T / s.P, p.fft_log2, s.k, GH, p.nb, s.d);
-    cudaError_t err = ensure_dynamic_smem(decode_fft_kernel<GH>, (size_t)L.total);
+    const FftSmem L = fft_smem_layout(LS, s.k, GH, p.nb, s.d);
+    cudaError_t err = ensure_dynamic_smem(decode_fft_kernel<GH, LS>, (size_t)L.total);
     if (err != cudaSuccess) return err;
-    decode_fft_kernel<GH><<<dim3(p.n_split, s.Hkv * p.n_pass, s.B), kThreads, L.total, st>>>(
+    decode_fft_kernel<GH, LS><<<dim3(p.n_split, s.Hkv * p.n_pass, s.B), kThreads, L.total, st>>>(
         s, c, p, static_cast<const bf16*>(q), ws);
     return cudaGetLastError();
 }
 
+template <int GH>
+cudaError_t launch_fft_ls(const Dims& s, const CacheDev& c, const DecodePlan& p, const void* q, char* ws, cudaStream_t st) {
+    switch (p.fft_log2) {
+        case 5: return launch_fft_t<GH, 5>(s, c, p, q, ws, st);
+        case 6: return launch_fft_t<GH, 6>(s, c, p, q, ws, st);
+        case 7: return launch_fft_t<GH, 7>(s, c, p, q, ws, st);
+        case 8: return launch_fft_t<GH, 8>(s, c, p, q, ws, st);
+        case 9: return launch_fft_t<GH, 9>(s, c, p, q, ws, st);
+        case 10: return launch_fft_t<GH, 10>(s, c, p, q, ws, st);
+        default: return cudaErrorInvalidValue;
+    }
+}
+
 }  // namespace
 
+extern "C" int fa_debug_read_profile(long long* out) { return (int)cudaMemcpyFromSymbol(out, g_prof, sizeof(long long) * 64); }
+
 size_t decode_fft_smem_bytes(const Dims& s, int log2S, int gh, int nb) {
-    return (size_t)fft_smem_layout(s.T / s.P, log2S, s.k, gh, nb, s.d).total;
+    return (size_t)fft_smem_layout(log2S, s.k, gh, nb, s.d).total;
 }
 
 cudaError_t launch_decode_fft(const Dims& s, const CacheDev& c, int dtype, const DecodePlan& p, const void* q, char* ws,
                               cudaStream_t st) {
     if (dtype != FA_BF16) return cudaErrorInvalidValue;
-    if (p.gh == 4) return launch_fft_t<4>(s, c, p, q, ws, st);
-    return launch_fft_t<2>(s, c, p, q, ws, st);
+    if (p.gh == 4) return launch_fft_ls<4>(s, c, p, q, ws, st);
+    return launch_fft_ls<2>(s, c, p, q, ws, st);
 }
 
 }  // namespace fa
