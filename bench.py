@@ -306,7 +306,7 @@ def run_ours(args):
         "breakdown": {"decode_us": us_decode, "append_us": us_append, "tokens_per_s": 1e6 / us_step * shape.B * world,
                       "append_gbs": by["append"] / (us_append * 1e-6) / 1e9,
                       "compress_ms_per_layer": min(comp_ms), "compress_tflops": comp_flop / (min(comp_ms) * 1e-3) / 1e12,
-                      "compress_path": "cuda-core fp32"},
+                      "compress_path": "tcgen05 bf16 x bf16 -> f32 (TMEM), basis tile generated in registers"},
         "roofline": {"kernel": "fa_decode_attention (prologue + main + epilogue kernels)", "bound": "hbm",
                      "achieved": dec_gbs, "peak": peak, "unit": "GB/s", "frac": dec_gbs / peak, "peak_kind": peak_kind,
                      "algorithmic_bytes": by["decode"], "traffic": NCU_TRAFFIC_BYTES_PER_CALL,

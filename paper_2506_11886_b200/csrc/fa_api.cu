@@ -1,7 +1,6 @@
 // Host side of the C ABI declared in include/fa.h: argument checks, buffer
 // sizes, launch plans.  Every entry point validates on the host, then launches
 // on the caller's stream; nothing here allocates device memory.
-#include <cstdlib>
 #include <cstring>
 
 #include "fa_common.cuh"
@@ -100,7 +99,6 @@ fa_status plan_decode(const fa_layout& l, DecodePlan* p) {
             long long cost = waves * ((s.P + n - 1) / n);
             if (best_cost < 0 || cost < best_cost) { best_cost = cost; best = n; }
         }
-        if (const char* e = std::getenv("FA_TUNE_NSPLIT")) { int v = std::atoi(e); if (v >= 1 && v <= s.P && v <= 64) best = v; }
         p->n_split = best;
         // classes transformed together: enough butterflies for all consumer threads, while two CTAs
         // still fit the shared memory of an SM (else one)
@@ -111,10 +109,8 @@ fa_status plan_decode(const fa_layout& l, DecodePlan* p) {
         const int per_cta = (s.P + best - 1) / best;
         if (nb > per_cta) nb = per_cta;
         while (nb > 1 && decode_fft_smem_bytes(s, log2S, p->gh, nb) > 113 * 1024) --nb;
-        if (const char* e = std::getenv("FA_TUNE_NB")) { int v = std::atoi(e); if (v >= 1 && v <= 8) nb = v; }
         while (nb > 1 && decode_fft_smem_bytes(s, log2S, p->gh, nb) > 227 * 1024) --nb;
         p->nb = nb;
-        if (const char* e = std::getenv("FA_TUNE_DBG")) p->dbg = std::atoi(e);
     } else {
         p->gh = s.G >= 4 ? 4 : (s.G >= 2 ? 2 : 1);
         if (s.G == 3) p->gh = 4;
@@ -254,8 +250,11 @@ fa_status fa_compress(const fa_layout* layout, fa_cache* cache, const void* K, c
     fa_cache_sizes_of(layout, &sz);
     if (sz.coef_k && cudaMemsetAsync(cache->coef_k, 0, sz.coef_k, cs) != cudaSuccess) return FA_ERR_CUDA;
     if (sz.coef_v && cudaMemsetAsync(cache->coef_v, 0, sz.coef_v, cs) != cudaSuccess) return FA_ERR_CUDA;
-    if (launch_compress(s, make_cache(*cache), layout->kv_dtype, K, V, stride_b, stride_t, stride_h, L, cs) != cudaSuccess)
+    const int64_t sbb = s.B > 1 ? stride_b : 0;
+    const bool tc = L > 0 && compress_tc_supported(s, layout->kv_dtype, sbb, stride_t, stride_h);
+    if (launch_compress(s, make_cache(*cache), layout->kv_dtype, K, V, stride_b, stride_t, stride_h, L, !tc, cs) != cudaSuccess)
         return FA_ERR_CUDA;
+    if (tc && launch_compress_tc(s, make_cache(*cache), K, V, sbb, stride_t, stride_h, L, cs) != cudaSuccess) return FA_ERR_CUDA;
     return FA_OK;
 }
 
@@ -286,15 +285,13 @@ fa_status fa_decode_attention(const fa_layout* layout, const fa_cache* cache, co
     CacheDev c = make_cache(*cache);
     cudaStream_t cs = static_cast<cudaStream_t>(stream);
     char* w = static_cast<char*>(ws);
-    const int dbgk = std::getenv("FA_TUNE_DBGK") ? std::atoi(std::getenv("FA_TUNE_DBGK")) : 0;
-    if (!(dbgk & 1) && launch_decode_prologue(s, c, layout->kv_dtype, p, q, w, cs) != cudaSuccess) return FA_ERR_CUDA;
-    if (dbgk & 2) {
-    } else if (p.algo == FA_DECODE_FFT) {
+    if (launch_decode_prologue(s, c, layout->kv_dtype, p, q, w, cs) != cudaSuccess) return FA_ERR_CUDA;
+    if (p.algo == FA_DECODE_FFT) {
         if (launch_decode_fft(s, c, layout->kv_dtype, p, q, w, cs) != cudaSuccess) return FA_ERR_CUDA;
     } else {
         if (launch_decode_direct(s, c, layout->kv_dtype, p, q, w, cs) != cudaSuccess) return FA_ERR_CUDA;
     }
-    if (!(dbgk & 4) && launch_decode_epilogue(s, c, layout->kv_dtype, p, out, w, cs) != cudaSuccess) return FA_ERR_CUDA;
+    if (launch_decode_epilogue(s, c, layout->kv_dtype, p, out, w, cs) != cudaSuccess) return FA_ERR_CUDA;
     return FA_OK;
 }
 

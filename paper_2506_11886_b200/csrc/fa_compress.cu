@@ -174,7 +174,7 @@ __global__ void __launch_bounds__(256) compress_coef_kernel(Dims s, CacheDev c, 
 
 template <typename KV>
 static cudaError_t launch_compress_t(const Dims& s, const CacheDev& c, const void* K, const void* V, int64_t sb,
-                                     int64_t st, int64_t sh, int L, cudaStream_t stream) {
+                                     int64_t st, int64_t sh, int L, bool with_coef, cudaStream_t stream) {
     int chunks_rows = (L + kRowsPerCta - 1) / kRowsPerCta;
     if (chunks_rows < 1) chunks_rows = 1;
     partition_gather_kernel<KV><<<dim3(chunks_rows, s.Hkv, s.B * 2), 256, 0, stream>>>(
@@ -185,7 +185,7 @@ static cudaError_t launch_compress_t(const Dims& s, const CacheDev& c, const voi
     int n_local = (L - n_init) < s.l_local ? (L - n_init) : s.l_local;
     int n_mid = L - n_init - n_local;
     int max_comp = s.dck > s.dcv ? s.dck : s.dcv;
-    if (n_mid == 0 || max_comp == 0) return cudaSuccess;
+    if (n_mid == 0 || max_comp == 0 || !with_coef) return cudaSuccess;
     int row_tiles = (s.M + kTM - 1) / kTM;
     int chunks = (n_mid + kTJ - 1) / kTJ;
     int ctas_fixed = row_tiles * s.B * s.Hkv * 2;
@@ -202,10 +202,11 @@ static cudaError_t launch_compress_t(const Dims& s, const CacheDev& c, const voi
     return cudaGetLastError();
 }
 
+// with_coef = false runs only the partition / gather kernel (the tensor-core path computes the coefficients).
 cudaError_t launch_compress(const Dims& s, const CacheDev& c, int dtype, const void* K, const void* V, int64_t sb,
-                            int64_t st, int64_t sh, int L, cudaStream_t stream) {
-    if (dtype == FA_BF16) return launch_compress_t<__nv_bfloat16>(s, c, K, V, sb, st, sh, L, stream);
-    return launch_compress_t<float>(s, c, K, V, sb, st, sh, L, stream);
+                            int64_t st, int64_t sh, int L, bool with_coef, cudaStream_t stream) {
+    if (dtype == FA_BF16) return launch_compress_t<__nv_bfloat16>(s, c, K, V, sb, st, sh, L, with_coef, stream);
+    return launch_compress_t<float>(s, c, K, V, sb, st, sh, L, with_coef, stream);
 }
 
 }  // namespace fa

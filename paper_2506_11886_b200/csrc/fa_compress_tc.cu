@@ -1,0 +1,341 @@
+// fa_compress, tensor-core path (Eq.3-4) for bf16 caches on sm_100a: C = F X^mn as a dense
+// [M x L_mid] x [L_mid x N] contraction on the 5th-generation tensor cores (tcgen05.mma,
+// bf16 x bf16 -> fp32 accumulators in tensor memory).
+//
+// One CTA owns 128 coefficient rows of one KV head, for K and V together: the N = 2 d columns
+// are all d dims of the K rows followed by all d dims of the V rows (the compressed dims are
+// picked out when the accumulators are read back; multiplying the kept dims too costs
+// d / d_c extra tensor work but lets the operand come straight from the prefilled K / V with
+// plain tiled TMA boxes).  The token axis is the contraction axis, cut into blocks of 64
+// tokens and split over several CTAs (partial sums are added with fp32 reductions to the
+// zeroed coefficients).  Per 64-token block and pipeline stage:
+//   * warp 0 (one lane) loads the K and V boxes [64 tokens x 64 dims] with TMA, 128-byte
+//     swizzle: the MN-major B operand, as laid out in the prefill tensor;
+//   * warps 2-5 generate the 128 x 64 basis tile in registers (integer phase for the first
+//     token of the block, then a rotation per token), round it to bf16 and store it in the
+//     K-major 128-byte-swizzled layout the tensor core reads: the A operand never exists in HBM;
+//   * warp 1 (one lane) issues four tcgen05.mma (K = 16 each) and commits the stage back.
+// At the end warps 2-5 read the accumulators from tensor memory and scatter the compressed
+// columns.  Every wait is bounded; tensor memory is freed on every path.
+#include <cuda.h>
+
+#include "fa_common.cuh"
+
+namespace fa {
+namespace {
+
+using bf16 = __nv_bfloat16;
+constexpr int kBM = 128;          // coefficient rows per CTA
+constexpr int kBK = 64;           // tokens per pipeline stage
+constexpr int kStagesTc = 4;
+constexpr int kThreadsTc = 192;
+constexpr uint32_t kSpinLimitTc = 1u << 24;
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ void mbar_init(uint64_t* b, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(b)), "r"(count));
+}
+__device__ __forceinline__ void mbar_arrive(uint64_t* b) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(b)) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint64_t* b, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(b)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint64_t* b, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}\n"
+        : "=r"(ok)
+        : "r"(smem_u32(b)), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+// Bounded wait; on time-out records the failure (nobody waits for ever, tensor memory is still freed).
+__device__ __forceinline__ bool mbar_wait(uint64_t* b, uint32_t parity, volatile int* fail, int32_t* status) {
+    if (*fail) return false;
+    for (uint32_t i = 0; i < kSpinLimitTc; ++i)
+        if (mbar_try_wait(b, parity)) return true;
+    *fail = 1;
+    atomicExch(status, (int)FA_ERR_TIMEOUT);
+    return false;
+}
+__device__ __forceinline__ void tma_load_4d(void* dst, const CUtensorMap* tm, int c0, int c1, int c2, int c3, uint64_t* bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.4d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5}], [%6];" ::"r"(
+            smem_u32(dst)),
+        "l"(reinterpret_cast<uint64_t>(tm)), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(smem_u32(bar))
+        : "memory");
+}
+
+// Shared-memory matrix descriptor of the tensor core (128-byte swizzle): start address, leading and
+// stride byte offsets in 16-byte units, descriptor version 1, layout type 2.
+__device__ __forceinline__ uint64_t umma_desc(uint32_t saddr, uint32_t lbo16, uint32_t sbo16) {
+    return (uint64_t)((saddr >> 4) & 0x3FFF) | ((uint64_t)(lbo16 & 0x3FFF) << 16) | ((uint64_t)(sbo16 & 0x3FFF) << 32) |
+           (1ull << 46) | (2ull << 61);
+}
+__device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n .reg .pred p;\n setp.ne.b32 p, %4, 0;\n tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}\n" ::"r"(tmem_d),
+        "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+__device__ __forceinline__ void umma_commit(uint64_t* bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&v)[32]) {
+    uint32_t r[32];
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]), "=r"(r[9]),
+          "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]), "=r"(r[17]), "=r"(r[18]),
+          "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]),
+          "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr));
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+    for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
+}
+
+// D = head dim (64 or 128): N = 2 D accumulator columns.
+template <int D>
+__global__ void __launch_bounds__(kThreadsTc, 1) compress_tc_kernel(const __grid_constant__ CUtensorMap tmK,
+                                                                    const __grid_constant__ CUtensorMap tmV, Dims s,
+                                                                    CacheDev c, int L, int n_tsplit) {
+    constexpr int N = 2 * D;
+    constexpr int kABytes = kBM * kBK * 2;                 // 16 KB basis tile
+    constexpr int kBoxBytes = kBK * 64 * 2;                // 8 KB per [64 tokens x 64 dims] box
+    constexpr int kBBytes = (N / 64) * kBoxBytes;
+    constexpr int kStageBytesTc = kABytes + kBBytes;
+    constexpr uint32_t kIdesc = (1u << 4) | (1u << 7) | (1u << 10) | (1u << 16) | ((uint32_t)(N >> 3) << 17) | ((uint32_t)(kBM >> 4) << 24);
+    extern __shared__ unsigned char smem_unaligned[];
+    unsigned char* smem = smem_unaligned + ((1024u - (smem_u32(smem_unaligned) & 1023u)) & 1023u);
+    unsigned char* stage0 = smem;                          // kStagesTc x (A | B boxes), 1024-byte aligned
+    uint64_t* fullA = reinterpret_cast<uint64_t*>(smem + kStagesTc * kStageBytesTc);
+    uint64_t* fullB = fullA + kStagesTc;
+    uint64_t* empty = fullB + kStagesTc;
+    uint64_t* acc_ready = empty + kStagesTc;
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_ready + 1);
+    volatile int* fail = reinterpret_cast<volatile int*>(tmem_slot + 1);
+    int* inv = reinterpret_cast<int*>(tmem_slot + 4);      // [2][D]: dim -> slot in D^kc / D^vc, or -1
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int mt = blockIdx.x, h = blockIdx.y;
+    const int b = blockIdx.z / n_tsplit, split = blockIdx.z % n_tsplit;
+    const int n_init = min(L, s.l_init);
+    const int n_local = min(L - n_init, s.l_local);
+    const int n_mid = L - n_init - n_local;
+    const int nkb = (n_mid + kBK - 1) / kBK;
+    const int per = (nkb + n_tsplit - 1) / n_tsplit;
+    const int kb0 = split * per, kb1 = min(nkb, kb0 + per);
+
+    if (tid == 0) {
+        for (int i = 0; i < kStagesTc; ++i) { mbar_init(fullA + i, 4); mbar_init(fullB + i, 1); mbar_init(empty + i, 1); }
+        mbar_init(acc_ready, 1);
+        *fail = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    for (int i = tid; i < 2 * D; i += kThreadsTc) inv[i] = -1;
+    __syncthreads();
+    for (int i = tid; i < s.dck + s.dcv; i += kThreadsTc) {
+        if (i < s.dck) inv[c.idx_comp_k[(size_t)h * s.dck + i]] = i;
+        else inv[D + c.idx_comp_v[(size_t)h * s.dcv + (i - s.dck)]] = i - s.dck;
+    }
+    if (warp == 1) {                                       // tensor memory: N fp32 columns x 128 lanes
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"((uint32_t)N) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    const uint32_t tmem_base = *tmem_slot;
+
+    if (kb1 > kb0) {
+        if (warp == 0) {
+            // ---------------- TMA producer: B operand = K and V rows of 64 tokens ----------------
+            if (lane == 0) {
+                for (int kb = kb0; kb < kb1; ++kb) {
+                    const int it = kb - kb0, st = it % kStagesTc;
+                    if (it >= kStagesTc && !mbar_wait(empty + st, ((it / kStagesTc) - 1) & 1, fail, c.status)) break;
+                    unsigned char* bdst = stage0 + (size_t)st * kStageBytesTc + kABytes;
+                    mbar_expect_tx(fullB + st, (uint32_t)kBBytes);
+                    const int tok = n_init + kb * kBK;
+#pragma unroll
+                    for (int bx = 0; bx < N / 64; ++bx) {
+                        const CUtensorMap* tm = bx < D / 64 ? &tmK : &tmV;
+                        const int dim0 = (bx % (D / 64)) * 64;
+                        tma_load_4d(bdst + bx * kBoxBytes, tm, dim0, h, tok, b, fullB + st);
+                    }
+                }
+            }
+        } else if (warp == 1) {
+            // ---------------- MMA issuer ----------------
+            if (lane == 0) {
+                for (int kb = kb0; kb < kb1; ++kb) {
+                    const int it = kb - kb0, st = it % kStagesTc;
+                    const uint32_t par = (it / kStagesTc) & 1;
+                    if (!mbar_wait(fullA + st, par, fail, c.status) || !mbar_wait(fullB + st, par, fail, c.status)) break;
+                    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                    const uint32_t a_addr = smem_u32(stage0 + (size_t)st * kStageBytesTc);
+                    const uint32_t b_addr = a_addr + kABytes;
+#pragma unroll
+                    for (int ks = 0; ks < kBK / 16; ++ks) {
+                        // A: K-major, rows of 128 bytes, 8-row groups 1024 bytes apart; 16 tokens = 32 bytes along the row
+                        const uint64_t adesc = umma_desc(a_addr + ks * 32, 1, 1024 >> 4);
+                        // B: MN-major, 64 dims per 128-byte row, 8-token groups 1024 bytes apart, next 64 dims one box further
+                        const uint64_t bdesc = umma_desc(b_addr + ks * 2048, kBoxBytes >> 4, 1024 >> 4);
+                        umma_bf16(tmem_base, adesc, bdesc, kIdesc, (it > 0 || ks > 0) ? 1u : 0u);
+                    }
+                    umma_commit(empty + st);               // frees the stage when these MMAs have read it
+                }
+                umma_commit(acc_ready);
+            }
+        } else {
+            // ---------------- basis generators: A operand ----------------
+            const int t = tid - 64;                        // 0..127
+            const int fi = t >> 1, th = t & 1;
+            const unsigned n = (unsigned)(mt * (kBM / 2) + fi);         // frequency of rows 2 fi (cos), 2 fi + 1 (sin)
+            const bool row_on = (int)(2 * n) < s.M;
+            float cs1, sn1;
+            sincospif(2.0f * (float)n / (float)s.T, &sn1, &cs1);          // rotation per token
+            const int r0 = 2 * fi, r1 = 2 * fi + 1;
+            const uint32_t row_off0 = (uint32_t)((r0 >> 3) * 1024 + (r0 & 7) * 128);
+            const uint32_t row_off1 = (uint32_t)((r1 >> 3) * 1024 + (r1 & 7) * 128);
+            for (int kb = kb0; kb < kb1; ++kb) {
+                const int it = kb - kb0, st = it % kStagesTc;
+                if (it >= kStagesTc && !mbar_wait(empty + st, ((it / kStagesTc) - 1) & 1, fail, c.status)) break;
+                unsigned char* a_dst = stage0 + (size_t)st * kStageBytesTc;
+                const int j0 = kb * kBK + 32 * th;
+                float cr, sr;
+                {
+                    const unsigned ph = (unsigned)(((unsigned long long)n * (unsigned)j0) % (unsigned)s.T);
+                    sincospif(2.0f * (float)ph / (float)s.T, &sr, &cr);
+                }
+#pragma unroll
+                for (int ch = 0; ch < 4; ++ch) {           // 8 tokens = one 16-byte chunk of each row
+                    uint32_t wc[4], wsn[4];
+#pragma unroll
+                    for (int i2 = 0; i2 < 4; ++i2) {
+                        float c0 = cr, s0 = sr;
+                        float c1 = fmaf(cr, cs1, -sr * sn1), s1 = fmaf(sr, cs1, cr * sn1);
+                        cr = fmaf(c1, cs1, -s1 * sn1);
+                        sr = fmaf(s1, cs1, c1 * sn1);
+                        const int j = j0 + ch * 8 + i2 * 2;
+                        const bool v0 = row_on && j < n_mid, v1 = row_on && j + 1 < n_mid;
+                        const __nv_bfloat162 pc = __floats2bfloat162_rn(v0 ? c0 : 0.f, v1 ? c1 : 0.f);
+                        const __nv_bfloat162 ps = __floats2bfloat162_rn(v0 ? s0 : 0.f, v1 ? s1 : 0.f);
+                        wc[i2] = *reinterpret_cast<const uint32_t*>(&pc);
+                        wsn[i2] = *reinterpret_cast<const uint32_t*>(&ps);
+                    }
+                    const int chunk = 4 * th + ch;
+                    *reinterpret_cast<uint4*>(a_dst + row_off0 + ((chunk ^ (r0 & 7)) << 4)) = make_uint4(wc[0], wc[1], wc[2], wc[3]);
+                    *reinterpret_cast<uint4*>(a_dst + row_off1 + ((chunk ^ (r1 & 7)) << 4)) = make_uint4(wsn[0], wsn[1], wsn[2], wsn[3]);
+                }
+                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic stores -> visible to the tensor core
+                __syncwarp();
+                if (lane == 0) mbar_arrive(fullA + st);
+            }
+            // ---------------- epilogue: accumulators -> compressed columns ----------------
+            const bool ok = mbar_wait(acc_ready, 0, fail, c.status);
+            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+            if (ok) {
+                const int lane_grp = warp & 3;             // a warp reads tensor-memory lanes 32 (warp % 4) ...
+                const int m = mt * kBM + lane_grp * 32 + lane;
+                float* ck = coef_rows(c.coef_k, s, b, h, s.dck) + (size_t)m * s.dck;
+                float* cv = coef_rows(c.coef_v, s, b, h, s.dcv) + (size_t)m * s.dcv;
+#pragma unroll 1
+                for (int col0 = 0; col0 < N; col0 += 32) {
+                    float v[32];
+                    tmem_ld32(tmem_base + ((uint32_t)(lane_grp * 32) << 16) + (uint32_t)col0, v);
+                    if (m < s.M) {
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) {
+                            const int col = col0 + i;
+                            const int slot = inv[col];
+                            if (slot >= 0) atomicAdd((col < D ? ck : cv) + slot, v[i]);
+                        }
+                    }
+                }
+            }
+        }
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    if (warp == 1) {
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)N) : "memory");
+    }
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                  const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_tiled_fn() {
+    static EncodeTiledFn fn = nullptr;
+    if (!fn) {
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess && q == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(p);
+    }
+    return fn;
+}
+
+// 4-D view (dim, head, token, batch) of a prefilled K or V with element strides (1, sh, st, sb); box = 64 dims x 64 tokens.
+bool make_map(CUtensorMap* tm, const void* base, const Dims& s, int64_t sb, int64_t st, int64_t sh, int L) {
+    EncodeTiledFn fn = encode_tiled_fn();
+    if (!fn) return false;
+    cuuint64_t dims[4] = {(cuuint64_t)s.d, (cuuint64_t)s.Hkv, (cuuint64_t)L, (cuuint64_t)s.B};
+    cuuint64_t strides[3] = {(cuuint64_t)sh * 2, (cuuint64_t)st * 2, (cuuint64_t)(s.B > 1 ? sb : st * (int64_t)L) * 2};
+    cuuint32_t box[4] = {64, 1, (cuuint32_t)kBK, 1};
+    cuuint32_t estr[4] = {1, 1, 1, 1};
+    return fn(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+              CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+template <int D>
+cudaError_t launch_tc_t(const CUtensorMap& tmK, const CUtensorMap& tmV, const Dims& s, const CacheDev& c, int L, int n_mid,
+                        cudaStream_t stream) {
+    constexpr int N = 2 * D;
+    constexpr size_t stage = (size_t)kBM * kBK * 2 + (size_t)(N / 64) * kBK * 64 * 2;
+    const size_t smem = kStagesTc * stage + 8 * (3 * kStagesTc + 1) + 16 + sizeof(int) * 2 * D + 64 + 1024;
+    cudaError_t err = ensure_dynamic_smem(compress_tc_kernel<D>, smem);
+    if (err != cudaSuccess) return err;
+    const int row_tiles = (s.M + kBM - 1) / kBM;
+    const int nkb = (n_mid + kBK - 1) / kBK;
+    const int fixed = row_tiles * s.Hkv * s.B;
+    int n_tsplit = (kNumSms + fixed - 1) / fixed;            // about one CTA per SM
+    if (n_tsplit > nkb) n_tsplit = nkb;
+    if (n_tsplit < 1) n_tsplit = 1;
+    compress_tc_kernel<D><<<dim3(row_tiles, s.Hkv, s.B * n_tsplit), kThreadsTc, smem, stream>>>(tmK, tmV, s, c, L, n_tsplit);
+    return cudaGetLastError();
+}
+
+}  // namespace
+
+// True if the tensor-core path serves this layout and these strides.
+bool compress_tc_supported(const Dims& s, int dtype, int64_t sb, int64_t st, int64_t sh) {
+    if (dtype != FA_BF16) return false;
+    if (s.d != 64 && s.d != 128) return false;
+    if (s.M % kBM != 0) return false;
+    if (s.dck == 0 && s.dcv == 0) return false;
+    if ((sh % 8) || (st % 8) || (sb % 8)) return false;
+    if ((unsigned long long)(s.M / 2) * (unsigned long long)s.T >= (1ull << 32)) return false;   // phase products stay in 32 x 32 -> 64 bits
+    return encode_tiled_fn() != nullptr;
+}
+
+// Coefficients only (the caller has zeroed them and runs the partition / gather kernel itself).
+cudaError_t launch_compress_tc(const Dims& s, const CacheDev& c, const void* K, const void* V, int64_t sb, int64_t st,
+                               int64_t sh, int L, cudaStream_t stream) {
+    const int n_init = L < s.l_init ? L : s.l_init;
+    const int n_local = (L - n_init) < s.l_local ? (L - n_init) : s.l_local;
+    const int n_mid = L - n_init - n_local;
+    if (n_mid <= 0) return cudaSuccess;
+    CUtensorMap tmK, tmV;
+    if (!make_map(&tmK, K, s, sb, st, sh, L) || !make_map(&tmV, V, s, sb, st, sh, L)) return cudaErrorInvalidValue;
+    if (s.d == 128) return launch_tc_t<128>(tmK, tmV, s, c, L, n_mid, stream);
+    return launch_tc_t<64>(tmK, tmV, s, c, L, n_mid, stream);
+}
+
+}  // namespace fa

@@ -38,8 +38,6 @@ constexpr int kWinRowsPerTile = 48;
 constexpr uint32_t kSpinLimit = 1u << 24;
 using bf16 = __nv_bfloat16;
 typedef unsigned long long u64;
-__device__ long long g_prof[64];
-#define PROF(i) do { if (dbg & 1024) { if (tid == 0 && blockIdx.x == 1 && blockIdx.y == 0 && blockIdx.z == 0) g_prof[i] = clock64(); } } while (0)
 
 // ---- PTX wrappers -----------------------------------------------------------
 __device__ __forceinline__ uint32_t smem_addr(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -331,7 +329,6 @@ __global__ void __launch_bounds__(kThreads, 2) decode_fft_kernel(Dims s, CacheDe
     extern __shared__ __align__(128) unsigned char smem_raw[];
     Ws ws = ws_view(wsp, p);
     const int NB = p.nb;
-    const int dbg = p.dbg;
     const FftSmem L = fft_smem_layout(LS, s.k, GH, NB, s.d);
     uint64_t* full = reinterpret_cast<uint64_t*>(smem_raw);
     uint64_t* empty = full + kStages;
@@ -378,10 +375,8 @@ __global__ void __launch_bounds__(kThreads, 2) decode_fft_kernel(Dims s, CacheDe
     // stale shared memory must hold finite numbers: rows past the end of a tile are multiplied by p = 0
     for (int i = tid; i < (kStages * kStageBytes) / 16; i += kThreads) reinterpret_cast<uint4*>(stages)[i] = make_uint4(0, 0, 0, 0);
     if (tid < 4) reinterpret_cast<uint32_t*>(zero16)[tid] = 0;
-    PROF(0);
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     __syncthreads();
-    PROF(1);
 
     // ============================ producer warp =================================
     if (tid >= kConsumers) {
@@ -400,7 +395,6 @@ __global__ void __launch_bounds__(kThreads, 2) decode_fft_kernel(Dims s, CacheDe
                 for (int side = 0; side < 2; ++side) {
                     const int ts = side == 0 ? ts_k : ts_v, rowb = side == 0 ? rowb_k : rowb_v;
                     if (!ts) continue;
-                    if (dbg & (side == 0 ? 2 : 8)) continue;
                     for (int cls = cb; cls < cb + nb; ++cls) {
                         const int n_c = n_of_class(cls);
                         for (int a0 = 0; a0 < n_c; a0 += ts) {
@@ -424,12 +418,12 @@ __global__ void __launch_bounds__(kThreads, 2) decode_fft_kernel(Dims s, CacheDe
                 const int nb = min(NB, c1 - cb);
                 for (int side = 0; side < 2; ++side) {
                     const int ts = side == 0 ? ts_k : ts_v;
-                    if (!ts || (dbg & (side == 0 ? 2 : 8))) continue;
+                    if (!ts) continue;
                     for (int cls = cb; cls < cb + nb; ++cls) it += (n_of_class(cls) + ts - 1) / ts;
                 }
             }
             __syncwarp();
-            for (int t0 = w0; t0 < w1 && !(dbg & 32); t0 += wchunk) {
+            for (int t0 = w0; t0 < w1; t0 += wchunk) {
                 const WinSegs sg = win_segments(t0, min(w1, t0 + wchunk), n_init, n_local, head, s.l_local);
                 for (int side = 0; side < 2; ++side)
                     for (int i = 0; i < sg.n; ++i)
@@ -527,7 +521,6 @@ __global__ void __launch_bounds__(kThreads, 2) decode_fft_kernel(Dims s, CacheDe
             }
     }
     consumer_sync();
-    PROF(2);
 
     float m_run[GH], l_acc[GH];                           // per slot
 #pragma unroll
@@ -619,7 +612,7 @@ __global__ void __launch_bounds__(kThreads, 2) decode_fft_kernel(Dims s, CacheDe
 
             // packed Hermitian spectra of the nb classes: X_m = V^A_m + i V^B_m per complex lane,
             // V_m = v_m + conj(v_{S-m}), v_n = (1/2) u~_n e^{i theta n c}.  Pair 0 is bins (0, S/2).
-            if (s.dck > 0 && !(dbg & 1)) {
+            if (s.dck > 0) {
                 for (int pr = tid; pr < S / 2; pr += kConsumers) {
                     const int m = pr, mc = pr == 0 ? S / 2 : S - pr;
                     PC<N> Am = czero, Bm = czero, Ac = czero, Bc = czero;
@@ -647,16 +640,14 @@ __global__ void __launch_bounds__(kThreads, 2) decode_fft_kernel(Dims s, CacheDe
                     }
                 }
                 consumer_sync();
-                if (cb == c0) PROF(3);
                 fft_run<GH, LS, LS, false>(fbuf, fb_floats, nb, twf, tid);        // score of slot a at point rev[a]
-                if (cb == c0) PROF(4);
             } else {
                 for (int i = tid; i < nb * fb_floats; i += kConsumers) fbuf[i] = 0.f;
                 consumer_sync();
             }
 
             // kept dims: s = sl2 * (q_u . K^mu) + compressed part, 16 tokens per mma
-            if (ts_k && !(dbg & 2)) {
+            if (ts_k) {
                 for (int ci = 0; ci < nb; ++ci) {
                     const int n_c = n_of_class(cb + ci);
                     float* base = fbuf + ci * fb_floats;
@@ -699,13 +690,12 @@ __global__ void __launch_bounds__(kThreads, 2) decode_fft_kernel(Dims s, CacheDe
                 }
             }
             consumer_sync();
-            if (cb == c0) PROF(5);
 
             // online softmax over the batch
             float mx[GH], alpha[GH];
 #pragma unroll
             for (int g = 0; g < GH; ++g) mx[g] = kNegBig;
-            for (int i = tid; i < (nb << LS) && !(dbg & 4); i += kConsumers) {
+            for (int i = tid; i < (nb << LS); i += kConsumers) {
                 const int ci = i >> LS, a = i & (S - 1);
                 if (a < n_of_class(cb + ci)) {
                     float v[GH];
@@ -722,7 +712,7 @@ __global__ void __launch_bounds__(kThreads, 2) decode_fft_kernel(Dims s, CacheDe
                 m_run[g] = m_new;
                 l_acc[g] *= alpha[g];
             }
-            for (int i = tid; i < (nb << LS) && !(dbg & 4); i += kConsumers) {
+            for (int i = tid; i < (nb << LS); i += kConsumers) {
                 const int ci = i >> LS, a = i & (S - 1);
                 float* pt = fbuf + ci * fb_floats + pf(rev[a] * GH);
                 float v[GH];
@@ -742,10 +732,9 @@ __global__ void __launch_bounds__(kThreads, 2) decode_fft_kernel(Dims s, CacheDe
                 for (int mt = 0; mt < 4; ++mt) { acc[mt][0] *= al; acc[mt][1] *= ah; acc[mt][2] *= al; acc[mt][3] *= ah; }
             }
             consumer_sync();
-            if (cb == c0) PROF(6);
 
             // o^u[dim][slot] += V^mu^T p, 16 tokens per mma
-            if (ts_v && !(dbg & 8)) {
+            if (ts_v) {
                 for (int ci = 0; ci < nb; ++ci) {
                     const int n_c = n_of_class(cb + ci);
                     const bf16* prow = pbt + (size_t)(ci * GH + (gq & (GH - 1))) * pbs;
@@ -778,11 +767,9 @@ __global__ void __launch_bounds__(kThreads, 2) decode_fft_kernel(Dims s, CacheDe
                 }
             }
 
-            if (cb == c0) PROF(7);
             // z_n = alpha z_n + sum_c e^{i theta n c} Y^c_n, Y^c = transform of the packed probabilities
-            if (s.dcv > 0 && !(dbg & 16)) {
+            if (s.dcv > 0) {
                 fft_run<GH, LS, LS, true>(fbuf, fb_floats, nb, twf, tid);
-                if (cb == c0) PROF(8);
                 PR<N> alA, alB;
                 if constexpr (N == 2) { alA = pk(alpha[0], alpha[1]); alB = pk(alpha[2], alpha[3]); }
                 else { alA = PR<1>{alpha[0]}; alB = PR<1>{alpha[1]}; }
@@ -849,10 +836,9 @@ __global__ void __launch_bounds__(kThreads, 2) decode_fft_kernel(Dims s, CacheDe
         }
     }
     consumer_sync();
-    PROF(10);
 
     // ------------------------------ window tokens -------------------------------
-    if (w1 > w0 && !(dbg & 32)) {
+    if (w1 > w0) {
         float a_win[GH];                                  // rescale of what the classes left in o_s / z_s
 #pragma unroll
         for (int g = 0; g < GH; ++g) a_win[g] = 1.f;
@@ -1005,7 +991,6 @@ __global__ void __launch_bounds__(kThreads, 2) decode_fft_kernel(Dims s, CacheDe
             }
         }
     }
-    PROF(11);
     // sum of p per slot
 #pragma unroll
     for (int g = 0; g < GH; ++g) {
@@ -1034,7 +1019,6 @@ __global__ void __launch_bounds__(kThreads, 2) decode_fft_kernel(Dims s, CacheDe
     if (tid < GH) {
         const int g = hperm<GH>(tid);                     // slot tid holds head g
         if (g < ng) {
-            PROF(12);
             float* ml = ws.ml + (((size_t)b * s.Hq + g_first + g) * p.n_split + split) * 2;
             float mv = m_run[0];
 #pragma unroll
@@ -1069,8 +1053,6 @@ cudaError_t launch_fft_ls(const Dims& s, const CacheDev& c, const DecodePlan& p,
 }
 
 }  // namespace
-
-extern "C" int fa_debug_read_profile(long long* out) { return (int)cudaMemcpyFromSymbol(out, g_prof, sizeof(long long) * 64); }
 
 size_t decode_fft_smem_bytes(const Dims& s, int log2S, int gh, int nb) {
     return (size_t)fft_smem_layout(log2S, s.k, gh, nb, s.d).total;
