@@ -90,6 +90,12 @@ __device__ __forceinline__ void ldmatrix_x4_trans(uint32_t (&r)[4], uint32_t add
 __device__ __forceinline__ uint32_t pack_bf16(bf16 lo, bf16 hi) {
     return (uint32_t)__bfloat16_as_ushort(lo) | ((uint32_t)__bfloat16_as_ushort(hi) << 16);
 }
+// cos and sin of 2 pi * frac, frac in [0, 1): hardware approximations on an angle folded into
+// [-pi, pi) (absolute error ~5e-7, far below what bf16 operands carry)
+__device__ __forceinline__ float2 cis_frac(float frac) {
+    const float a = 6.283185307179586f * (frac - (frac >= 0.5f ? 1.0f : 0.0f));
+    return make_float2(__cosf(a), __sinf(a));
+}
 __device__ __forceinline__ float ex2(float x) {
     float y;
     asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
@@ -177,9 +183,11 @@ __device__ __forceinline__ void dft(PC<N> (&v)[R]) {
 }
 
 // Shared-memory float index of float f of a transform buffer: 16 bytes of padding after every
-// 128, which spreads strided point accesses over the banks and keeps points 16-byte aligned.
-__host__ __device__ constexpr int pf(int f) { return f + ((f >> 5) << 2); }
-__host__ __device__ constexpr int pf_size(int floats) { return floats + ((floats >> 5) << 2) + 4; }
+// 128 bytes, every 1 KB and every 8 KB.  Points stay 16-byte aligned; the strided point accesses
+// of the passes and the digit-reversed accesses of token-ordered code (consecutive slots sit 64, 8
+// or 1 points apart after a radix-8 decimation) all spread over the banks.
+__host__ __device__ constexpr int pf(int f) { return f + ((f >> 5) << 2) + ((f >> 8) << 2) + ((f >> 11) << 2); }
+__host__ __device__ constexpr int pf_size(int floats) { return pf(floats) + 8; }
 
 // Radix of the pass that handles a sub-transform of length 2^l (8 where possible, two 4s for 16).
 __host__ __device__ constexpr int radix_log2(int l) { return (l >= 3 && l != 4) ? 3 : (l >= 2 ? 2 : 1); }
@@ -327,6 +335,7 @@ __global__ void __launch_bounds__(kThreads, 2) decode_fft_kernel(Dims s, CacheDe
     constexpr int N = GH / 2;
     constexpr int S = 1 << LS;
     extern __shared__ __align__(128) unsigned char smem_raw[];
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");      // the epilogue may be scheduled behind us at once
     Ws ws = ws_view(wsp, p);
     const int NB = p.nb;
     const FftSmem L = fft_smem_layout(LS, s.k, GH, NB, s.d);
@@ -380,8 +389,36 @@ __global__ void __launch_bounds__(kThreads, 2) decode_fft_kernel(Dims s, CacheDe
 
     // ============================ producer warp =================================
     if (tid >= kConsumers) {
-        if (tid == kConsumers) {
-            int it = 0;
+        // window rows first (same order as the consumers): one bulk copy per row into padded
+        // shared-memory rows, issued by all lanes of the warp
+        const int plane = tid - kConsumers;
+        int it = 0;
+        for (int t0 = w0; t0 < w1; t0 += wchunk) {
+            const WinSegs sg = win_segments(t0, min(w1, t0 + wchunk), n_init, n_local, head, s.l_local);
+            for (int side = 0; side < 2; ++side)
+                for (int i = 0; i < sg.n; ++i)
+                    for (int r0 = 0; r0 < sg.cnt[i]; r0 += ts_w) {
+                        const int nt = min(ts_w, sg.cnt[i] - r0);
+                        void* base = sg.buf[i] == 0 ? (side == 0 ? c.k_init : c.v_init) : (side == 0 ? c.k_local : c.v_local);
+                        const int rows = sg.buf[i] == 0 ? s.l_init : s.l_local;
+                        const bf16* src = win_row<bf16>(base, s, b, h, rows, sg.row[i] + r0);
+                        const int st = it % kStages;
+                        int ok = 1;
+                        if (plane == 0) {
+                            if (it >= kStages) mbar_wait(empty + st, ((it / kStages) - 1) & 1, fail, c.status);
+                            ok = !*fail;
+                            if (ok) mbar_expect_tx(full + st, (uint32_t)(nt * rowb_w));
+                        }
+                        ok = __shfl_sync(0xffffffffu, ok, 0);
+                        if (ok) {
+                            unsigned char* dst = stages + (size_t)st * kStageBytes;
+                            for (int r = plane; r < nt; r += 32)
+                                bulk_g2s(dst + (size_t)r * rbw_pad, src + (size_t)r * s.d, (uint32_t)rowb_w, full + st);
+                        }
+                        ++it;
+                    }
+        }
+        if (plane == 0) {
             auto acquire = [&](uint32_t bytes) -> unsigned char* {
                 const int st = it % kStages;
                 if (it >= kStages) mbar_wait(empty + st, ((it / kStages) - 1) & 1, fail, c.status);
@@ -389,7 +426,7 @@ __global__ void __launch_bounds__(kThreads, 2) decode_fft_kernel(Dims s, CacheDe
                 mbar_expect_tx(full + st, bytes);
                 return stages + (size_t)st * kStageBytes;
             };
-            // same order as the consumers: per batch of NB classes all K tiles, then all V tiles
+            // per batch of NB classes all K tiles, then all V tiles
             for (int cb = c0; cb < c1; cb += NB) {
                 const int nb = min(NB, c1 - cb);
                 for (int side = 0; side < 2; ++side) {
@@ -408,47 +445,6 @@ __global__ void __launch_bounds__(kThreads, 2) decode_fft_kernel(Dims s, CacheDe
                 }
             }
         }
-        // window rows: one bulk copy per row into padded shared-memory rows, issued by all lanes
-        {
-            const int plane = tid - kConsumers;
-            __syncwarp();                                 // lane 0 has issued every class tile
-            int it = 0;
-            // recount the class tiles so that the ring position continues where lane 0 stopped
-            for (int cb = c0; cb < c1; cb += NB) {
-                const int nb = min(NB, c1 - cb);
-                for (int side = 0; side < 2; ++side) {
-                    const int ts = side == 0 ? ts_k : ts_v;
-                    if (!ts) continue;
-                    for (int cls = cb; cls < cb + nb; ++cls) it += (n_of_class(cls) + ts - 1) / ts;
-                }
-            }
-            __syncwarp();
-            for (int t0 = w0; t0 < w1; t0 += wchunk) {
-                const WinSegs sg = win_segments(t0, min(w1, t0 + wchunk), n_init, n_local, head, s.l_local);
-                for (int side = 0; side < 2; ++side)
-                    for (int i = 0; i < sg.n; ++i)
-                        for (int r0 = 0; r0 < sg.cnt[i]; r0 += ts_w) {
-                            const int nt = min(ts_w, sg.cnt[i] - r0);
-                            void* base = sg.buf[i] == 0 ? (side == 0 ? c.k_init : c.v_init) : (side == 0 ? c.k_local : c.v_local);
-                            const int rows = sg.buf[i] == 0 ? s.l_init : s.l_local;
-                            const bf16* src = win_row<bf16>(base, s, b, h, rows, sg.row[i] + r0);
-                            const int st = it % kStages;
-                            int ok = 1;
-                            if (plane == 0) {
-                                if (it >= kStages) mbar_wait(empty + st, ((it / kStages) - 1) & 1, fail, c.status);
-                                ok = !*fail;
-                                if (ok) mbar_expect_tx(full + st, (uint32_t)(nt * rowb_w));
-                            }
-                            ok = __shfl_sync(0xffffffffu, ok, 0);
-                            if (ok) {
-                                unsigned char* dst = stages + (size_t)st * kStageBytes;
-                                for (int r = plane; r < nt; r += 32)
-                                    bulk_g2s(dst + (size_t)r * rbw_pad, src + (size_t)r * s.d, (uint32_t)rowb_w, full + st);
-                            }
-                            ++it;
-                        }
-            }
-        }
         return;
     }
 
@@ -461,30 +457,7 @@ __global__ void __launch_bounds__(kThreads, 2) decode_fft_kernel(Dims s, CacheDe
     // ---- one-time set-up ----
     for (int i = tid; i < GH * s.d; i += kConsumers) o_s[i] = 0.f;
     for (int i = tid; i < s.k; i += kConsumers) {
-        float sn, cs;
-        sincospif(2.0f * (float)i / (float)s.T, &sn, &cs);
-        E[i] = make_float2(cs, sn);
-    }
-    // ut[n] = (A.re, A.im, B.re, B.im), A = heads of the real slots, B = heads of the imaginary slots;
-    // all loads of an entry are issued together
-    for (int n = tid; n < s.k; n += kConsumers) {
-        float2 uv[GH];
-#pragma unroll
-        for (int sl = 0; sl < GH; ++sl) {
-            const int g = hperm<GH>(sl);
-            uv[sl] = make_float2(0.f, 0.f);
-            if (g < ng && s.dck > 0) uv[sl] = *reinterpret_cast<const float2*>(ws.u + ((size_t)b * s.Hq + g_first + g) * s.M + 2 * n);
-        }
-        float* e = ut + n * 2 * GH;
-        float* zz = z_s + n * 2 * GH;
-#pragma unroll
-        for (int sl = 0; sl < GH; ++sl) {
-            const int ab = sl / N, ln = sl - ab * N;
-            e[(2 * ab) * N + ln] = 0.5f * uv[sl].x;
-            e[(2 * ab + 1) * N + ln] = -0.5f * uv[sl].y;
-            zz[(2 * ab) * N + ln] = 0.f;
-            zz[(2 * ab + 1) * N + ln] = 0.f;
-        }
+        E[i] = cis_frac((float)i / (float)s.T);
     }
     for (int l = LS; l > 0;) {
         const int rl = radix_log2(l), R = 1 << rl, st = 1 << (l - rl);
@@ -492,9 +465,7 @@ __global__ void __launch_bounds__(kThreads, 2) decode_fft_kernel(Dims s, CacheDe
             const int off = tw_offset(LS, l);
             for (int i = tid; i < (R - 1) * st; i += kConsumers) {
                 const int qm1 = i / st, j = i - qm1 * st;
-                float sn, cs;
-                sincospif(2.0f * (float)(((qm1 + 1) * j) & ((1 << l) - 1)) / (float)(1 << l), &sn, &cs);
-                reinterpret_cast<float2*>(twf)[off + i] = make_float2(cs, sn);
+                reinterpret_cast<float2*>(twf)[off + i] = cis_frac((float)(((qm1 + 1) * j) & ((1 << l) - 1)) / (float)(1 << l));
             }
         }
         l -= rl;
@@ -519,6 +490,29 @@ __global__ void __launch_bounds__(kThreads, 2) decode_fft_kernel(Dims s, CacheDe
                 qk[rd][ks][0] = on ? pack_bf16(qrow[idf_k[e0]], qrow[idf_k[e0 + 1]]) : 0u;
                 qk[rd][ks][1] = on ? pack_bf16(qrow[idf_k[e0 + 2]], qrow[idf_k[e0 + 3]]) : 0u;
             }
+    }
+    // everything above is independent of the prologue kernel; its output u is first needed here
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    // ut[n] = (A.re, A.im, B.re, B.im), A = heads of the real slots, B = heads of the imaginary slots;
+    // all loads of an entry are issued together
+    for (int n = tid; n < s.k; n += kConsumers) {
+        float2 uv[GH];
+#pragma unroll
+        for (int sl = 0; sl < GH; ++sl) {
+            const int g = hperm<GH>(sl);
+            uv[sl] = make_float2(0.f, 0.f);
+            if (g < ng && s.dck > 0) uv[sl] = *reinterpret_cast<const float2*>(ws.u + ((size_t)b * s.Hq + g_first + g) * s.M + 2 * n);
+        }
+        float* e = ut + n * 2 * GH;
+        float* zz = z_s + n * 2 * GH;
+#pragma unroll
+        for (int sl = 0; sl < GH; ++sl) {
+            const int ab = sl / N, ln = sl - ab * N;
+            e[(2 * ab) * N + ln] = 0.5f * uv[sl].x;
+            e[(2 * ab + 1) * N + ln] = -0.5f * uv[sl].y;
+            zz[(2 * ab) * N + ln] = 0.f;
+            zz[(2 * ab + 1) * N + ln] = 0.f;
+        }
     }
     consumer_sync();
 
@@ -592,10 +586,145 @@ __global__ void __launch_bounds__(kThreads, 2) decode_fft_kernel(Dims s, CacheDe
     };
     const PC<N> czero = PC<N>{splat<N>(0.f), splat<N>(0.f)};
     auto seed_tw = [&](int n, int cls) -> float2 {
-        float sn, cs;
-        sincospif(2.0f * (float)((n * cls) & (s.T - 1)) / (float)s.T, &sn, &cs);
-        return make_float2(cs, sn);
+        return cis_frac((float)((n * cls) & (s.T - 1)) / (float)s.T);
     };
+
+    // ------------------------------ window tokens -------------------------------
+    if (w1 > w0) {
+        uint32_t qw[4][2][2];
+#pragma unroll
+        for (int rd = 0; rd < 4; ++rd)
+#pragma unroll
+            for (int ks = 0; ks < 2; ++ks) {
+                const int piece = 4 * rd + tq, e0 = 8 * piece + 4 * ks;
+                const bool on = col_on && piece < npw;
+                qw[rd][ks][0] = on ? pack_bf16(qrow[e0], qrow[e0 + 1]) : 0u;
+                qw[rd][ks][1] = on ? pack_bf16(qrow[e0 + 2], qrow[e0 + 3]) : 0u;
+            }
+        float accw[8][4];
+#pragma unroll
+        for (int mt = 0; mt < 8; ++mt)
+#pragma unroll
+            for (int i = 0; i < 4; ++i) accw[mt][i] = 0.f;
+        const int nmtw = (s.d + 15) >> 4;
+        float* sb = fbuf;                                 // natural order, no transform
+        bf16* pb = pbt;
+        for (int t0 = w0; t0 < w1; t0 += wchunk) {
+            const int n_tok = min(w1, t0 + wchunk) - t0;
+            const WinSegs sg = win_segments(t0, t0 + n_tok, n_init, n_local, head, s.l_local);
+            for (int si = 0; si < sg.n; ++si)
+                for (int r0 = 0; r0 < sg.cnt[si]; r0 += ts_w) {
+                    const int nt = min(ts_w, sg.cnt[si] - r0);
+                    const unsigned char* tile = wait_tile();
+                    for (int grp = warp; grp * 16 < nt; grp += 8) {
+                        const unsigned char* r_lo = tile + (size_t)(grp * 16 + gq) * rbw_pad;
+                        const unsigned char* r_hi = r_lo + 8 * rbw_pad;
+                        float d4[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+                        for (int rd = 0; rd < 4; ++rd) {
+                            const int piece = 4 * rd + tq;
+                            if (4 * rd < npw) {
+                                uint4 lo = make_uint4(0, 0, 0, 0), hi = make_uint4(0, 0, 0, 0);
+                                if (piece < npw) {
+                                    lo = *reinterpret_cast<const uint4*>(r_lo + 16 * piece);
+                                    hi = *reinterpret_cast<const uint4*>(r_hi + 16 * piece);
+                                }
+                                mma_bf16(d4, lo.x, hi.x, lo.y, hi.y, qw[rd][0][0], qw[rd][0][1]);
+                                mma_bf16(d4, lo.z, hi.z, lo.w, hi.w, qw[rd][1][0], qw[rd][1][1]);
+                            }
+                        }
+                        if (2 * tq < GH) {
+                            const int i_lo = grp * 16 + gq, i_hi = i_lo + 8;
+                            if (i_lo < nt)
+                                *reinterpret_cast<float2*>(sb + pf((sg.tok[si] + r0 + i_lo) * GH + 2 * tq)) = make_float2(d4[0] * sl2, d4[1] * sl2);
+                            if (i_hi < nt)
+                                *reinterpret_cast<float2*>(sb + pf((sg.tok[si] + r0 + i_hi) * GH + 2 * tq)) = make_float2(d4[2] * sl2, d4[3] * sl2);
+                        }
+                    }
+                    release_tile();
+                }
+            consumer_sync();
+            float mx[GH], alpha[GH];
+#pragma unroll
+            for (int g = 0; g < GH; ++g) mx[g] = kNegBig;
+            for (int a = tid; a < n_tok; a += kConsumers) {
+                float v[GH];
+                load_vals(sb + pf(a * GH), v);
+#pragma unroll
+                for (int g = 0; g < GH; ++g) mx[g] = fmaxf(mx[g], v[g]);
+            }
+            block_max(mx);
+#pragma unroll
+            for (int g = 0; g < GH; ++g) {
+                const float m_new = fmaxf(m_run[g], mx[g]);
+                alpha[g] = ex2(m_run[g] - m_new);
+                m_run[g] = m_new;
+                l_acc[g] *= alpha[g];
+            }
+            const int n_pad = (n_tok + 15) & ~15;
+            for (int a = tid; a < n_pad; a += kConsumers) {
+                float v[GH];
+#pragma unroll
+                for (int g = 0; g < GH; ++g) v[g] = 0.f;
+                if (a < n_tok) load_vals(sb + pf(a * GH), v);
+#pragma unroll
+                for (int g = 0; g < GH; ++g) {
+                    v[g] = a < n_tok ? ex2(v[g] - m_run[g]) : 0.f;
+                    l_acc[g] += v[g];
+                    pb[g * pbs + a] = __float2bfloat16_rn(v[g]);
+                }
+            }
+            {
+                const float al = alpha[(2 * tq) & (GH - 1)], ah = alpha[(2 * tq + 1) & (GH - 1)];
+#pragma unroll
+                for (int mt = 0; mt < 8; ++mt) { accw[mt][0] *= al; accw[mt][1] *= ah; accw[mt][2] *= al; accw[mt][3] *= ah; }
+            }
+            consumer_sync();
+            const bf16* prow = pb + (size_t)(gq & (GH - 1)) * pbs;
+            for (int si = 0; si < sg.n; ++si)
+                for (int r0 = 0; r0 < sg.cnt[si]; r0 += ts_w) {
+                    const int nt = min(ts_w, sg.cnt[si] - r0);
+                    const unsigned char* tile = wait_tile();
+                    for (int grp = warp; grp * 16 < nt; grp += 8) {
+                        const int a = sg.tok[si] + r0 + grp * 16;
+                        // the tile's rows may start at any token of the chunk: gather the four p values one by one
+                        uint32_t b0 = 0, b1 = 0;
+                        if (gq < GH) {
+                            const int rem = nt - grp * 16;
+                            const bf16 zero = __float2bfloat16_rn(0.f);
+                            b0 = pack_bf16(2 * tq < rem ? prow[a + 2 * tq] : zero, 2 * tq + 1 < rem ? prow[a + 2 * tq + 1] : zero);
+                            b1 = pack_bf16(2 * tq + 8 < rem ? prow[a + 2 * tq + 8] : zero, 2 * tq + 9 < rem ? prow[a + 2 * tq + 9] : zero);
+                        }
+                        const int mi = lane >> 3, tok = ((mi >> 1) << 3) + (lane & 7);
+                        const unsigned char* vrow = tile + (size_t)(grp * 16 + tok) * rbw_pad;
+#pragma unroll
+                        for (int mt = 0; mt < 8; ++mt) {
+                            if (mt < nmtw) {
+                                const int chunk = 2 * mt + (mi & 1);
+                                const unsigned char* src = chunk < npw ? vrow + 16 * chunk : zero16;
+                                uint32_t af[4];
+                                ldmatrix_x4_trans(af, smem_addr(src));
+                                mma_bf16(accw[mt], af[0], af[1], af[2], af[3], b0, b1);
+                            }
+                        }
+                    }
+                    release_tile();
+                }
+            consumer_sync();
+        }
+        // the window fragments open o_s; the class batches rescale it as the running maximum moves
+        if (2 * tq < GH) {
+            float* o_lo = o_s + hperm<GH>(2 * tq) * s.d;
+            float* o_hi = o_s + hperm<GH>(2 * tq + 1) * s.d;
+#pragma unroll
+            for (int mt = 0; mt < 8; ++mt) {
+                const int e_lo = 16 * mt + gq, e_hi = e_lo + 8;
+                if (e_lo < s.d) { atomicAdd(o_lo + e_lo, accw[mt][0]); atomicAdd(o_hi + e_lo, accw[mt][1]); }
+                if (e_hi < s.d) { atomicAdd(o_lo + e_hi, accw[mt][2]); atomicAdd(o_hi + e_hi, accw[mt][3]); }
+            }
+        }
+    }
+    consumer_sync();
 
     // ------------------------------ middle classes ------------------------------
     {
@@ -731,6 +860,13 @@ __global__ void __launch_bounds__(kThreads, 2) decode_fft_kernel(Dims s, CacheDe
 #pragma unroll
                 for (int mt = 0; mt < 4; ++mt) { acc[mt][0] *= al; acc[mt][1] *= ah; acc[mt][2] *= al; acc[mt][3] *= ah; }
             }
+            for (int i = tid; i < GH * s.d; i += kConsumers) {          // what the windows left in o_s (rows are heads)
+                const int g = i / s.d;
+                float a = alpha[0];
+#pragma unroll
+                for (int sl = 1; sl < GH; ++sl) if (hperm<GH>(sl) == g) a = alpha[sl];
+                o_s[i] *= a;
+            }
             consumer_sync();
 
             // o^u[dim][slot] += V^mu^T p, 16 tokens per mma
@@ -837,160 +973,6 @@ __global__ void __launch_bounds__(kThreads, 2) decode_fft_kernel(Dims s, CacheDe
     }
     consumer_sync();
 
-    // ------------------------------ window tokens -------------------------------
-    if (w1 > w0) {
-        float a_win[GH];                                  // rescale of what the classes left in o_s / z_s
-#pragma unroll
-        for (int g = 0; g < GH; ++g) a_win[g] = 1.f;
-        uint32_t qw[4][2][2];
-#pragma unroll
-        for (int rd = 0; rd < 4; ++rd)
-#pragma unroll
-            for (int ks = 0; ks < 2; ++ks) {
-                const int piece = 4 * rd + tq, e0 = 8 * piece + 4 * ks;
-                const bool on = col_on && piece < npw;
-                qw[rd][ks][0] = on ? pack_bf16(qrow[e0], qrow[e0 + 1]) : 0u;
-                qw[rd][ks][1] = on ? pack_bf16(qrow[e0 + 2], qrow[e0 + 3]) : 0u;
-            }
-        float accw[8][4];
-#pragma unroll
-        for (int mt = 0; mt < 8; ++mt)
-#pragma unroll
-            for (int i = 0; i < 4; ++i) accw[mt][i] = 0.f;
-        const int nmtw = (s.d + 15) >> 4;
-        float* sb = fbuf;                                 // natural order, no transform
-        bf16* pb = pbt;
-        for (int t0 = w0; t0 < w1; t0 += wchunk) {
-            const int n_tok = min(w1, t0 + wchunk) - t0;
-            const WinSegs sg = win_segments(t0, t0 + n_tok, n_init, n_local, head, s.l_local);
-            for (int si = 0; si < sg.n; ++si)
-                for (int r0 = 0; r0 < sg.cnt[si]; r0 += ts_w) {
-                    const int nt = min(ts_w, sg.cnt[si] - r0);
-                    const unsigned char* tile = wait_tile();
-                    for (int grp = warp; grp * 16 < nt; grp += 8) {
-                        const unsigned char* r_lo = tile + (size_t)(grp * 16 + gq) * rbw_pad;
-                        const unsigned char* r_hi = r_lo + 8 * rbw_pad;
-                        float d4[4] = {0.f, 0.f, 0.f, 0.f};
-#pragma unroll
-                        for (int rd = 0; rd < 4; ++rd) {
-                            const int piece = 4 * rd + tq;
-                            if (4 * rd < npw) {
-                                uint4 lo = make_uint4(0, 0, 0, 0), hi = make_uint4(0, 0, 0, 0);
-                                if (piece < npw) {
-                                    lo = *reinterpret_cast<const uint4*>(r_lo + 16 * piece);
-                                    hi = *reinterpret_cast<const uint4*>(r_hi + 16 * piece);
-                                }
-                                mma_bf16(d4, lo.x, hi.x, lo.y, hi.y, qw[rd][0][0], qw[rd][0][1]);
-                                mma_bf16(d4, lo.z, hi.z, lo.w, hi.w, qw[rd][1][0], qw[rd][1][1]);
-                            }
-                        }
-                        if (2 * tq < GH) {
-                            const int i_lo = grp * 16 + gq, i_hi = i_lo + 8;
-                            if (i_lo < nt)
-                                *reinterpret_cast<float2*>(sb + pf((sg.tok[si] + r0 + i_lo) * GH + 2 * tq)) = make_float2(d4[0] * sl2, d4[1] * sl2);
-                            if (i_hi < nt)
-                                *reinterpret_cast<float2*>(sb + pf((sg.tok[si] + r0 + i_hi) * GH + 2 * tq)) = make_float2(d4[2] * sl2, d4[3] * sl2);
-                        }
-                    }
-                    release_tile();
-                }
-            consumer_sync();
-            float mx[GH], alpha[GH];
-#pragma unroll
-            for (int g = 0; g < GH; ++g) mx[g] = kNegBig;
-            for (int a = tid; a < n_tok; a += kConsumers) {
-                float v[GH];
-                load_vals(sb + pf(a * GH), v);
-#pragma unroll
-                for (int g = 0; g < GH; ++g) mx[g] = fmaxf(mx[g], v[g]);
-            }
-            block_max(mx);
-#pragma unroll
-            for (int g = 0; g < GH; ++g) {
-                const float m_new = fmaxf(m_run[g], mx[g]);
-                alpha[g] = ex2(m_run[g] - m_new);
-                m_run[g] = m_new;
-                l_acc[g] *= alpha[g];
-                a_win[g] *= alpha[g];
-            }
-            const int n_pad = (n_tok + 15) & ~15;
-            for (int a = tid; a < n_pad; a += kConsumers) {
-                float v[GH];
-#pragma unroll
-                for (int g = 0; g < GH; ++g) v[g] = 0.f;
-                if (a < n_tok) load_vals(sb + pf(a * GH), v);
-#pragma unroll
-                for (int g = 0; g < GH; ++g) {
-                    v[g] = a < n_tok ? ex2(v[g] - m_run[g]) : 0.f;
-                    l_acc[g] += v[g];
-                    pb[g * pbs + a] = __float2bfloat16_rn(v[g]);
-                }
-            }
-            {
-                const float al = alpha[(2 * tq) & (GH - 1)], ah = alpha[(2 * tq + 1) & (GH - 1)];
-#pragma unroll
-                for (int mt = 0; mt < 8; ++mt) { accw[mt][0] *= al; accw[mt][1] *= ah; accw[mt][2] *= al; accw[mt][3] *= ah; }
-            }
-            consumer_sync();
-            const bf16* prow = pb + (size_t)(gq & (GH - 1)) * pbs;
-            for (int si = 0; si < sg.n; ++si)
-                for (int r0 = 0; r0 < sg.cnt[si]; r0 += ts_w) {
-                    const int nt = min(ts_w, sg.cnt[si] - r0);
-                    const unsigned char* tile = wait_tile();
-                    for (int grp = warp; grp * 16 < nt; grp += 8) {
-                        const int a = sg.tok[si] + r0 + grp * 16;
-                        // the tile's rows may start at any token of the chunk: gather the four p values one by one
-                        uint32_t b0 = 0, b1 = 0;
-                        if (gq < GH) {
-                            const int rem = nt - grp * 16;
-                            const bf16 zero = __float2bfloat16_rn(0.f);
-                            b0 = pack_bf16(2 * tq < rem ? prow[a + 2 * tq] : zero, 2 * tq + 1 < rem ? prow[a + 2 * tq + 1] : zero);
-                            b1 = pack_bf16(2 * tq + 8 < rem ? prow[a + 2 * tq + 8] : zero, 2 * tq + 9 < rem ? prow[a + 2 * tq + 9] : zero);
-                        }
-                        const int mi = lane >> 3, tok = ((mi >> 1) << 3) + (lane & 7);
-                        const unsigned char* vrow = tile + (size_t)(grp * 16 + tok) * rbw_pad;
-#pragma unroll
-                        for (int mt = 0; mt < 8; ++mt) {
-                            if (mt < nmtw) {
-                                const int chunk = 2 * mt + (mi & 1);
-                                const unsigned char* src = chunk < npw ? vrow + 16 * chunk : zero16;
-                                uint32_t af[4];
-                                ldmatrix_x4_trans(af, smem_addr(src));
-                                mma_bf16(accw[mt], af[0], af[1], af[2], af[3], b0, b1);
-                            }
-                        }
-                    }
-                    release_tile();
-                }
-            consumer_sync();
-        }
-        // rescale what the classes left, then add the window fragments
-        for (int i = tid; i < GH * s.d; i += kConsumers) {
-            const int g = i / s.d;                        // head
-            float a = a_win[0];
-#pragma unroll
-            for (int sl = 1; sl < GH; ++sl) if (hperm<GH>(sl) == g) a = a_win[sl];
-            o_s[i] *= a;
-        }
-        for (int i = tid; i < s.k * 2 * GH; i += kConsumers) {
-            const int f = i % (2 * GH), part = f / N, ln = f - part * N, slot = (part >> 1) * N + ln;
-            float a = a_win[0];
-#pragma unroll
-            for (int sl = 1; sl < GH; ++sl) if (slot == sl) a = a_win[sl];
-            z_s[i] *= a;
-        }
-        consumer_sync();
-        if (2 * tq < GH) {
-            float* o_lo = o_s + hperm<GH>(2 * tq) * s.d;
-            float* o_hi = o_s + hperm<GH>(2 * tq + 1) * s.d;
-#pragma unroll
-            for (int mt = 0; mt < 8; ++mt) {
-                const int e_lo = 16 * mt + gq, e_hi = e_lo + 8;
-                if (e_lo < s.d) { atomicAdd(o_lo + e_lo, accw[mt][0]); atomicAdd(o_hi + e_lo, accw[mt][1]); }
-                if (e_hi < s.d) { atomicAdd(o_lo + e_hi, accw[mt][2]); atomicAdd(o_hi + e_hi, accw[mt][3]); }
-            }
-        }
-    }
     // sum of p per slot
 #pragma unroll
     for (int g = 0; g < GH; ++g) {
@@ -1034,9 +1016,17 @@ cudaError_t launch_fft_t(const Dims& s, const CacheDev& c, const DecodePlan& p, 
     const FftSmem L = fft_smem_layout(LS, s.k, GH, p.nb, s.d);
     cudaError_t err = ensure_dynamic_smem(decode_fft_kernel<GH, LS>, (size_t)L.total);
     if (err != cudaSuccess) return err;
-    decode_fft_kernel<GH, LS><<<dim3(p.n_split, s.Hkv * p.n_pass, s.B), kThreads, L.total, st>>>(
-        s, c, p, static_cast<const bf16*>(q), ws);
-    return cudaGetLastError();
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(p.n_split, s.Hkv * p.n_pass, s.B);
+    cfg.blockDim = dim3(kThreads);
+    cfg.dynamicSmemBytes = (size_t)L.total;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;   // may start while the prologue kernel runs
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, decode_fft_kernel<GH, LS>, s, c, p, static_cast<const bf16*>(q), ws);
 }
 
 template <int GH>

@@ -2,7 +2,11 @@
 //   prologue   u_g[m] = scale * log2(e) * w_m * sum_e C^K[m][e] q_g[D^kc[e]]
 //   epilogue   merge the token splits, o^c[e] = sum_m w_m z[m] C^V[m][e], normalise, scatter.
 // Both read their coefficient matrix exactly once; each CTA brings a tile of rows into shared
-// memory with 16-byte asynchronous copies (all in flight together) and works from there.
+// memory with 16-byte asynchronous copies (all in flight together) and works from there.  All
+// loads of partial results are issued in independent batches so that a call costs a few memory
+// round trips, not one per split.  The three kernels of a decode call are chained with
+// programmatic dependent launch: each lets its successor start at once, and the successor waits
+// (griddepcontrol.wait) only where it first touches what its predecessor wrote.
 #include "fa_common.cuh"
 #include "fa_decode_ws.cuh"
 
@@ -15,6 +19,8 @@ __device__ __forceinline__ void cp_async16(void* smem_dst, const void* gmem_src)
 __device__ __forceinline__ void cp_async_wait_all() {
     asm volatile("cp.async.commit_group;\ncp.async.wait_group 0;" ::: "memory");
 }
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 
 // ---------------------------------------------------------------- prologue --
 // grid (ceil(M / rows_pro), Hkv, B), 256 threads.
@@ -22,6 +28,7 @@ template <typename KV>
 __global__ void __launch_bounds__(256) decode_prologue_kernel(Dims s, CacheDev c, DecodePlan p, const KV* __restrict__ q,
                                                               char* wsp) {
     extern __shared__ __align__(16) float sm_pro[];
+    pdl_launch_dependents();
     Ws ws = ws_view(wsp, p);
     const int h = blockIdx.y, b = blockIdx.z, tid = threadIdx.x;
     if (blockIdx.x == 0 && tid == 0) ws.cnt[b * s.Hkv + h] = 0;
@@ -78,13 +85,16 @@ __global__ void __launch_bounds__(256) decode_epilogue_kernel(Dims s, CacheDev c
     const int m0 = slice * rows_max;
     const int rows = max(0, min(rows_max, s.M - m0));
     const int stride = s.dcv + 4;
-    float* alpha_s = sm_epi;                               // [G][n_split]
-    float* linv_s = alpha_s + s.G * p.n_split;             // [G]
+    const int ns = p.n_split;
+    float* alpha_s = sm_epi;                               // [G][n_split]: first the maxima, then exp2(m - max)
+    float* l_s = alpha_s + s.G * ns;                       // [G][n_split]
+    float* linv_s = l_s + s.G * ns;                        // [G]
     float* zw_s = linv_s + s.G;                            // [G][rows_max]
     int* inv_s = reinterpret_cast<int*>(zw_s + s.G * rows_max);   // [d] dim -> slot in D^vc, or -1
     float* tile = reinterpret_cast<float*>(inv_s + s.d);   // [rows_max][stride]
     tile = reinterpret_cast<float*>((reinterpret_cast<uintptr_t>(tile) + 15) & ~uintptr_t(15));
 
+    // the coefficient tile does not depend on the main kernel: start it before waiting for it
     if (s.dcv > 0) {
         const float* cv = coef_rows(c.coef_v, s, b, h, s.dcv) + (size_t)m0 * s.dcv;
         const int vpr = s.dcv >> 2;
@@ -93,34 +103,45 @@ __global__ void __launch_bounds__(256) decode_epilogue_kernel(Dims s, CacheDev c
             cp_async16(tile + r * stride + 4 * v4, cv + (size_t)r * s.dcv + 4 * v4);
         }
     }
-    for (int g = tid; g < s.G; g += 256) {
-        const float* ml = ws.ml + ((size_t)b * s.Hq + h * s.G + g) * p.n_split * 2;
+    for (int e = tid; e < s.d; e += 256) inv_s[e] = -1;
+    pdl_wait();                                            // partial results of the main kernel are complete
+
+    // split statistics: one (head, split) pair per thread, then a tiny reduction per head
+    for (int i = tid; i < s.G * ns; i += 256) {
+        const int g = i / ns, sp = i - g * ns;
+        const float2 ml = *reinterpret_cast<const float2*>(ws.ml + (((size_t)b * s.Hq + h * s.G + g) * ns + sp) * 2);
+        alpha_s[i] = ml.x;
+        l_s[i] = ml.y;
+    }
+    __syncthreads();
+    if (tid < s.G) {
         float mx = kNegBig;
-        for (int sp = 0; sp < p.n_split; ++sp) mx = fmaxf(mx, ml[2 * sp]);
+        for (int sp = 0; sp < ns; ++sp) mx = fmaxf(mx, alpha_s[tid * ns + sp]);
         float L = 0.f;
-        for (int sp = 0; sp < p.n_split; ++sp) {
-            float a = exp2f(ml[2 * sp] - mx);
-            alpha_s[g * p.n_split + sp] = a;
-            L += a * ml[2 * sp + 1];
+        for (int sp = 0; sp < ns; ++sp) {
+            const float a = exp2f(alpha_s[tid * ns + sp] - mx);
+            alpha_s[tid * ns + sp] = a;
+            L = fmaf(a, l_s[tid * ns + sp], L);
         }
-        linv_s[g] = L > 0.f ? 1.0f / L : 0.f;
+        linv_s[tid] = L > 0.f ? 1.0f / L : 0.f;
     }
     __syncthreads();
     if (s.dcv > 0) {
         for (int t = tid; t < s.G * rows; t += 256) {
             const int g = t / rows, r = t - g * rows;
-            const float* z = ws.z + ((size_t)b * s.Hq + h * s.G + g) * p.n_split * s.M + m0 + r;
-            const float* al = alpha_s + g * p.n_split;
-            float v0 = 0.f, v1 = 0.f, v2 = 0.f, v3 = 0.f;
+            const float* z = ws.z + ((size_t)b * s.Hq + h * s.G + g) * ns * s.M + m0 + r;
+            const float* al = alpha_s + g * ns;
+            float v0 = 0.f, v1 = 0.f;
             int sp = 0;
-            for (; sp + 4 <= p.n_split; sp += 4) {
-                v0 = fmaf(al[sp], z[(size_t)sp * s.M], v0);
-                v1 = fmaf(al[sp + 1], z[(size_t)(sp + 1) * s.M], v1);
-                v2 = fmaf(al[sp + 2], z[(size_t)(sp + 2) * s.M], v2);
-                v3 = fmaf(al[sp + 3], z[(size_t)(sp + 3) * s.M], v3);
+            for (; sp + 8 <= ns; sp += 8) {                // eight independent loads in flight
+                float zz[8];
+#pragma unroll
+                for (int i = 0; i < 8; ++i) zz[i] = z[(size_t)(sp + i) * s.M];
+#pragma unroll
+                for (int i = 0; i < 8; i += 2) { v0 = fmaf(al[sp + i], zz[i], v0); v1 = fmaf(al[sp + i + 1], zz[i + 1], v1); }
             }
-            for (; sp < p.n_split; ++sp) v0 = fmaf(al[sp], z[(size_t)sp * s.M], v0);
-            zw_s[g * rows_max + r] = ((v0 + v1) + (v2 + v3)) * recon_weight(s.norm, m0 + r, s.k, s.T);
+            for (; sp < ns; ++sp) v0 = fmaf(al[sp], z[(size_t)sp * s.M], v0);
+            zw_s[g * rows_max + r] = (v0 + v1) * recon_weight(s.norm, m0 + r, s.k, s.T);
         }
         cp_async_wait_all();
         __syncthreads();
@@ -147,33 +168,37 @@ __global__ void __launch_bounds__(256) decode_epilogue_kernel(Dims s, CacheDev c
     __syncthreads();
     if (!last_s) return;
     __threadfence();
-    for (int e = tid; e < s.d; e += 256) inv_s[e] = -1;
-    __syncthreads();
     const int32_t* idc_v = c.idx_comp_v + (size_t)h * s.dcv;
     for (int e = tid; e < s.dcv; e += 256) inv_s[idc_v[e]] = e;
     __syncthreads();
     for (int t = tid; t < s.G * s.d; t += 256) {
         const int g = t / s.d, e = t - g * s.d;
         const size_t qh = (size_t)b * s.Hq + h * s.G + g;
-        const float* al = alpha_s + g * p.n_split;
-        const float* o = ws.o + qh * p.n_split * s.d + e;
+        const float* al = alpha_s + g * ns;
+        const float* o = ws.o + qh * ns * s.d + e;
         float v0 = 0.f, v1 = 0.f;
         int sp = 0;
-        for (; sp + 2 <= p.n_split; sp += 2) {
-            v0 = fmaf(al[sp], o[(size_t)sp * s.d], v0);
-            v1 = fmaf(al[sp + 1], o[(size_t)(sp + 1) * s.d], v1);
+        for (; sp + 8 <= ns; sp += 8) {
+            float oo[8];
+#pragma unroll
+            for (int i = 0; i < 8; ++i) oo[i] = o[(size_t)(sp + i) * s.d];
+#pragma unroll
+            for (int i = 0; i < 8; i += 2) { v0 = fmaf(al[sp + i], oo[i], v0); v1 = fmaf(al[sp + i + 1], oo[i + 1], v1); }
         }
-        if (sp < p.n_split) v0 = fmaf(al[sp], o[(size_t)sp * s.d], v0);
+        for (; sp < ns; ++sp) v0 = fmaf(al[sp], o[(size_t)sp * s.d], v0);
         const int slot = inv_s[e];
         if (slot >= 0) {
             const float* oc = ws.oc + qh * p.n_slice * s.dcv + slot;
             float w0 = 0.f, w1 = 0.f;
             int sl = 0;
-            for (; sl + 2 <= p.n_slice; sl += 2) {
-                w0 += __ldcg(oc + (size_t)sl * s.dcv);
-                w1 += __ldcg(oc + (size_t)(sl + 1) * s.dcv);
+            for (; sl + 8 <= p.n_slice; sl += 8) {
+                float cc[8];
+#pragma unroll
+                for (int i = 0; i < 8; ++i) cc[i] = __ldcg(oc + (size_t)(sl + i) * s.dcv);
+#pragma unroll
+                for (int i = 0; i < 8; i += 2) { w0 += cc[i]; w1 += cc[i + 1]; }
             }
-            if (sl < p.n_slice) w0 += __ldcg(oc + (size_t)sl * s.dcv);
+            for (; sl < p.n_slice; ++sl) w0 += __ldcg(oc + (size_t)sl * s.dcv);
             v0 += w0;
             v1 += w1;
         }
@@ -182,6 +207,24 @@ __global__ void __launch_bounds__(256) decode_epilogue_kernel(Dims s, CacheDev c
 }
 
 // ---------------------------------------------------------------- launchers --
+// Launch with the programmatic-stream-serialization attribute: the kernel may start while its
+// predecessor in the stream still runs; it synchronises with griddepcontrol.wait.
+template <typename... Params, typename... Args>
+static cudaError_t launch_pdl(void (*kernel)(Params...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, bool pdl,
+                              Args... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = pdl ? 1 : 0;
+    return cudaLaunchKernelEx(&cfg, kernel, static_cast<Params>(args)...);
+}
+
 template <typename KV>
 static cudaError_t launch_prologue_t(const Dims& s, const CacheDev& c, const DecodePlan& p, const void* q, char* ws,
                                      cudaStream_t st) {
@@ -203,11 +246,11 @@ template <typename KV>
 static cudaError_t launch_epilogue_t(const Dims& s, const CacheDev& c, const DecodePlan& p, void* out, char* ws,
                                      cudaStream_t st) {
     const int rows = (s.M + p.n_slice - 1) / p.n_slice;
-    const size_t smem = sizeof(float) * ((size_t)s.G * p.n_split + s.G + (size_t)s.G * rows + s.d + 4 + (size_t)rows * (s.dcv + 4));
+    const size_t smem = sizeof(float) * (2 * (size_t)s.G * p.n_split + s.G + (size_t)s.G * rows + s.d + 4 + (size_t)rows * (s.dcv + 4));
     cudaError_t err = ensure_dynamic_smem(decode_epilogue_kernel<KV>, smem);
     if (err != cudaSuccess) return err;
-    decode_epilogue_kernel<KV><<<dim3(p.n_slice, s.Hkv, s.B), 256, smem, st>>>(s, c, p, static_cast<KV*>(out), ws);
-    return cudaGetLastError();
+    return launch_pdl(decode_epilogue_kernel<KV>, dim3(p.n_slice, s.Hkv, s.B), dim3(256), smem, st, true, s, c, p,
+                      static_cast<KV*>(out), ws);
 }
 
 cudaError_t launch_decode_epilogue(const Dims& s, const CacheDev& c, int dtype, const DecodePlan& p, void* out, char* ws,
