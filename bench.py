@@ -168,7 +168,7 @@ def run_reference(args):
 def run_ours(args):
     import torch
     import torch.distributed as dist
-    from paper_2506_11886_b200 import build, fa, synth
+    from paper_2506_11886_b200 import build, fa, replicas, synth
 
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
@@ -230,9 +230,8 @@ def run_ours(args):
 
     def barrier():
         torch.cuda.synchronize()
-        if world > 1:
-            dist.barrier()
-            torch.cuda.synchronize()
+        replicas.barrier()
+        torch.cuda.synchronize()
 
     def timed_graph(body, n_warm, n_steps):
         """Captures n_warm and n_steps steps as two CUDA graphs, replays the first untimed and the
@@ -255,11 +254,7 @@ def run_ours(args):
         e1.record()
         barrier()
         ms = e0.elapsed_time(e1)
-        if world > 1:
-            t = torch.tensor([ms], device=dev)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            ms = float(t.item())
-        return ms
+        return replicas.max_over_ranks(ms, device=dev)
 
     with ClockSampler(local) as clk:
         ms_step = timed_graph(lambda s: step(s), W, K_steps)

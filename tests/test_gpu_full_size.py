@@ -12,7 +12,8 @@ from tests.parity_util import COEF_REL, OUT_ABS_BF16, layout_of, to64, unswizzle
 pytestmark = pytest.mark.gpu
 
 
-def _sampled_head_check(shape, layout, heads, steps, seed):
+def _sampled_head_check(shape, layout, heads, steps, seed, rows=None):
+    rows = list(range(shape.B)) if rows is None else list(rows)      # batch rows the oracle recomputes
     stream = synth.KVStream(shape, seed=seed, device="cuda")
     K, V = stream.tokens(0, shape.L, work_dtype=torch.float32)
     cache = fa.Cache(layout, stream.idx_full_k, stream.idx_full_v)
@@ -30,31 +31,31 @@ def _sampled_head_check(shape, layout, heads, steps, seed):
     G = shape.Hq // shape.Hkv
     worst_out = worst_coef = 0.0
     for h in heads:
-        sub = fo.OracleConfig(B=shape.B, Hq=G, Hkv=1, d=shape.d, n_full_k=shape.n_full_k, n_full_v=shape.n_full_v,
+        sub = fo.OracleConfig(B=len(rows), Hq=G, Hkv=1, d=shape.d, n_full_k=shape.n_full_k, n_full_v=shape.n_full_v,
                               k=shape.k, T=shape.T, L_init=shape.L_init, L_local=shape.L_local, cap_mid=layout.max_mid,
                               scale=shape.softmax_scale)
         ref = fo.OracleCache(sub, stream.idx_full_k[h:h + 1].numpy(), stream.idx_full_v[h:h + 1].numpy())
-        ref.compress(to64(K[:, :, h:h + 1]), to64(V[:, :, h:h + 1]))
+        ref.compress(to64(K[rows][:, :, h:h + 1]), to64(V[rows][:, :, h:h + 1]))
         for t in range(steps):
-            ref.append(to64(Kn[:, t, h:h + 1]), to64(Vn[:, t, h:h + 1]))
-        want = ref.decode(to64(q[:, h * G:(h + 1) * G]))
-        got = to64(out[:, h * G:(h + 1) * G])
+            ref.append(to64(Kn[rows][:, t, h:h + 1]), to64(Vn[rows][:, t, h:h + 1]))
+        want = ref.decode(to64(q[rows][:, h * G:(h + 1) * G]))
+        got = to64(out[rows][:, h * G:(h + 1) * G])
         worst_out = max(worst_out, np.abs(got - want).max())
         # metadata and stored rows of the sampled head: bit-exact; coefficients: norm-wise
-        st = cache.state.cpu().numpy()
+        st = cache.state.cpu().numpy()[rows]
         assert (st[:, 2] == ref.n_mid).all() and (st[:, 1] == ref.n_local).all() and (st[:, 0] == ref.n_init).all()
-        for b in range(shape.B):
-            nm, head = int(st[b, 2]), int(st[b, 3])
+        for bi, b in enumerate(rows):
+            nm, head = int(st[bi, 2]), int(st[bi, 3])
             j = np.arange(nm)
             gk = to64(cache.k_mid[b, h])[j % layout.mid_classes, j // layout.mid_classes]
             gv = to64(cache.v_mid[b, h])[j % layout.mid_classes, j // layout.mid_classes]
             gv = unswizzle_v_rows(gv[None], j // layout.mid_classes, layout)[0]
-            np.testing.assert_array_equal(gk, ref.k_mid[b, 0, :nm])
-            np.testing.assert_array_equal(gv, ref.v_mid[b, 0, :nm])
+            np.testing.assert_array_equal(gk, ref.k_mid[bi, 0, :nm])
+            np.testing.assert_array_equal(gv, ref.v_mid[bi, 0, :nm])
             order = (head + np.arange(shape.L_local)) % shape.L_local
-            np.testing.assert_array_equal(to64(cache.k_local[b, h])[order], ref.k_local[b, 0])
+            np.testing.assert_array_equal(to64(cache.k_local[b, h])[order], ref.k_local[bi, 0])
             for name in ("coef_k", "coef_v"):
-                r = getattr(ref, name)[b, 0]
+                r = getattr(ref, name)[bi, 0]
                 g = to64(getattr(cache, name)[b, h])
                 worst_coef = max(worst_coef, np.abs(g - r).max() / np.abs(r).max())
     assert worst_coef <= COEF_REL, worst_coef
@@ -67,3 +68,19 @@ def test_llama31_8b_32k_sampled_heads():
     layout = layout_of(shape, max_mid=shape.T, P=shape.T // shape.k)
     assert layout.mid_classes == 64
     _sampled_head_check(shape, layout, heads=(0, 7), steps=3, seed=1000)
+
+
+def test_llama2_7b_mha_batch8_sampled_heads():
+    """Serving configuration: MHA (G = 1), batch 8, 4K prompt, 48 kept / 80 compressed dims, M = 256;
+    a few append + decode steps, first and last head recomputed by the oracle for all batch rows."""
+    shape = synth.CONFIGS[3]
+    layout = layout_of(shape, max_mid=shape.T, P=shape.T // shape.k)
+    _sampled_head_check(shape, layout, heads=(0, 31), steps=5, seed=3000)
+
+
+def test_128k_batch4_one_sampled_head():
+    """Long-context stress shape: 128K tokens, batch 4, M = 2048, 2048-token recent window; the
+    oracle recomputes one (batch row, KV head)."""
+    shape = synth.CONFIGS[4]
+    layout = layout_of(shape, max_mid=shape.T, P=shape.T // shape.k)
+    _sampled_head_check(shape, layout, heads=(5,), steps=2, seed=4000, rows=(3,))
