@@ -11,11 +11,11 @@
 // zeroed coefficients).  Per 64-token block and pipeline stage:
 //   * warp 0 (one lane) loads the K and V boxes [64 tokens x 64 dims] with TMA, 128-byte
 //     swizzle: the MN-major B operand, as laid out in the prefill tensor;
-//   * warps 2-5 generate the 128 x 64 basis tile in registers (integer phase for the first
-//     token of the block, then a rotation per token), round it to bf16 and store it in the
+//   * warps 2-9 generate the 128 x 64 basis tile in registers (integer phase for the first
+//     two tokens of a thread's run, then packed fp32-pair rotations by two tokens), round it to bf16 and store it in the
 //     K-major 128-byte-swizzled layout the tensor core reads: the A operand never exists in HBM;
 //   * warp 1 (one lane) issues four tcgen05.mma (K = 16 each) and commits the stage back.
-// At the end warps 2-5 read the accumulators from tensor memory and scatter the compressed
+// At the end warps 2-9 read the accumulators from tensor memory and scatter the compressed
 // columns.  Every wait is bounded; tensor memory is freed on every path.
 #include <cuda.h>
 
@@ -28,7 +28,8 @@ using bf16 = __nv_bfloat16;
 constexpr int kBM = 128;          // coefficient rows per CTA
 constexpr int kBK = 64;           // tokens per pipeline stage
 constexpr int kStagesTc = 4;
-constexpr int kThreadsTc = 192;
+constexpr int kGenWarps = 8;       // basis generators (and epilogue): 16 tokens of two rows per thread and stage
+constexpr int kThreadsTc = 64 + 32 * kGenWarps;
 constexpr uint32_t kSpinLimitTc = 1u << 24;
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -130,7 +131,7 @@ __global__ void __launch_bounds__(kThreadsTc, 1) compress_tc_kernel(const __grid
     const int kb0 = split * per, kb1 = min(nkb, kb0 + per);
 
     if (tid == 0) {
-        for (int i = 0; i < kStagesTc; ++i) { mbar_init(fullA + i, 4); mbar_init(fullB + i, 1); mbar_init(empty + i, 1); }
+        for (int i = 0; i < kStagesTc; ++i) { mbar_init(fullA + i, kGenWarps); mbar_init(fullB + i, 1); mbar_init(empty + i, 1); }
         mbar_init(acc_ready, 1);
         *fail = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -192,12 +193,21 @@ __global__ void __launch_bounds__(kThreadsTc, 1) compress_tc_kernel(const __grid
             }
         } else {
             // ---------------- basis generators: A operand ----------------
-            const int t = tid - 64;                        // 0..127
-            const int fi = t >> 1, th = t & 1;
+            const int t = tid - 64;                        // 0 .. 32 kGenWarps - 1
+            const int fi = t >> 2, tqr = t & 3;            // frequency pair of the tile, quarter of the 64 tokens
             const unsigned n = (unsigned)(mt * (kBM / 2) + fi);         // frequency of rows 2 fi (cos), 2 fi + 1 (sin)
             const bool row_on = (int)(2 * n) < s.M;
-            float cs1, sn1;
-            sincospif(2.0f * (float)n / (float)s.T, &sn1, &cs1);          // rotation per token
+            const float inv_T = 1.0f / (float)s.T;
+            // rotation by two tokens, as splat pairs
+            unsigned long long CS2, SN2, NSN2;
+            {
+                const unsigned ph2 = (unsigned)((2ull * n) % (unsigned)s.T);
+                const float a = 6.283185307179586f * ((float)ph2 * inv_T - ((float)ph2 * inv_T >= 0.5f ? 1.0f : 0.0f));
+                const float c2 = __cosf(a), s2 = __sinf(a);
+                asm("mov.b64 %0, {%1,%1};" : "=l"(CS2) : "f"(c2));
+                asm("mov.b64 %0, {%1,%1};" : "=l"(SN2) : "f"(s2));
+                asm("mov.b64 %0, {%1,%1};" : "=l"(NSN2) : "f"(-s2));
+            }
             const int r0 = 2 * fi, r1 = 2 * fi + 1;
             const uint32_t row_off0 = (uint32_t)((r0 >> 3) * 1024 + (r0 & 7) * 128);
             const uint32_t row_off1 = (uint32_t)((r1 >> 3) * 1024 + (r1 & 7) * 128);
@@ -205,29 +215,45 @@ __global__ void __launch_bounds__(kThreadsTc, 1) compress_tc_kernel(const __grid
                 const int it = kb - kb0, st = it % kStagesTc;
                 if (it >= kStagesTc && !mbar_wait(empty + st, ((it / kStagesTc) - 1) & 1, fail, c.status)) break;
                 unsigned char* a_dst = stage0 + (size_t)st * kStageBytesTc;
-                const int j0 = kb * kBK + 32 * th;
-                float cr, sr;
+                const int j0 = kb * kBK + 16 * tqr;
+                // packed phasors of tokens (j0, j0 + 1): C = (cos, cos), S = (sin, sin), exact integer phases
+                unsigned long long C, S;
                 {
-                    const unsigned ph = (unsigned)(((unsigned long long)n * (unsigned)j0) % (unsigned)s.T);
-                    sincospif(2.0f * (float)ph / (float)s.T, &sr, &cr);
+                    const unsigned pa = (n * (unsigned)j0) % (unsigned)s.T, pb = (n * (unsigned)(j0 + 1)) % (unsigned)s.T;
+                    const float fa = (float)pa * inv_T, fb = (float)pb * inv_T;
+                    const float aa = 6.283185307179586f * (fa - (fa >= 0.5f ? 1.0f : 0.0f));
+                    const float ab = 6.283185307179586f * (fb - (fb >= 0.5f ? 1.0f : 0.0f));
+                    asm("mov.b64 %0, {%1,%2};" : "=l"(C) : "f"(__cosf(aa)), "f"(__cosf(ab)));
+                    asm("mov.b64 %0, {%1,%2};" : "=l"(S) : "f"(__sinf(aa)), "f"(__sinf(ab)));
                 }
+                const bool whole = row_on && j0 + 16 <= n_mid;          // no masking needed in the common case
 #pragma unroll
-                for (int ch = 0; ch < 4; ++ch) {           // 8 tokens = one 16-byte chunk of each row
+                for (int ch = 0; ch < 2; ++ch) {           // 8 tokens = one 16-byte chunk of each row
                     uint32_t wc[4], wsn[4];
 #pragma unroll
                     for (int i2 = 0; i2 < 4; ++i2) {
-                        float c0 = cr, s0 = sr;
-                        float c1 = fmaf(cr, cs1, -sr * sn1), s1 = fmaf(sr, cs1, cr * sn1);
-                        cr = fmaf(c1, cs1, -s1 * sn1);
-                        sr = fmaf(s1, cs1, c1 * sn1);
-                        const int j = j0 + ch * 8 + i2 * 2;
-                        const bool v0 = row_on && j < n_mid, v1 = row_on && j + 1 < n_mid;
-                        const __nv_bfloat162 pc = __floats2bfloat162_rn(v0 ? c0 : 0.f, v1 ? c1 : 0.f);
-                        const __nv_bfloat162 ps = __floats2bfloat162_rn(v0 ? s0 : 0.f, v1 ? s1 : 0.f);
+                        float c0, c1, s0, s1;
+                        asm("mov.b64 {%0,%1}, %2;" : "=f"(c0), "=f"(c1) : "l"(C));
+                        asm("mov.b64 {%0,%1}, %2;" : "=f"(s0), "=f"(s1) : "l"(S));
+                        if (!whole) {
+                            const int j = j0 + ch * 8 + i2 * 2;
+                            const bool v0 = row_on && j < n_mid, v1 = row_on && j + 1 < n_mid;
+                            c0 = v0 ? c0 : 0.f; s0 = v0 ? s0 : 0.f; c1 = v1 ? c1 : 0.f; s1 = v1 ? s1 : 0.f;
+                        }
+                        const __nv_bfloat162 pc = __floats2bfloat162_rn(c0, c1);
+                        const __nv_bfloat162 ps = __floats2bfloat162_rn(s0, s1);
                         wc[i2] = *reinterpret_cast<const uint32_t*>(&pc);
                         wsn[i2] = *reinterpret_cast<const uint32_t*>(&ps);
+                        // advance both phasors by two tokens: C' = C cs2 - S sn2, S' = S cs2 + C sn2
+                        unsigned long long tC, tS, nC, nS;
+                        asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(tC) : "l"(C), "l"(CS2));
+                        asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(tS) : "l"(S), "l"(CS2));
+                        asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(nC) : "l"(S), "l"(NSN2), "l"(tC));
+                        asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(nS) : "l"(C), "l"(SN2), "l"(tS));
+                        C = nC;
+                        S = nS;
                     }
-                    const int chunk = 4 * th + ch;
+                    const int chunk = 2 * tqr + ch;
                     *reinterpret_cast<uint4*>(a_dst + row_off0 + ((chunk ^ (r0 & 7)) << 4)) = make_uint4(wc[0], wc[1], wc[2], wc[3]);
                     *reinterpret_cast<uint4*>(a_dst + row_off1 + ((chunk ^ (r1 & 7)) << 4)) = make_uint4(wsn[0], wsn[1], wsn[2], wsn[3]);
                 }
@@ -240,11 +266,12 @@ __global__ void __launch_bounds__(kThreadsTc, 1) compress_tc_kernel(const __grid
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
             if (ok) {
                 const int lane_grp = warp & 3;             // a warp reads tensor-memory lanes 32 (warp % 4) ...
+                const int col_half = (warp - 2) >> 2;      // two warps share a lane group: one column half each
                 const int m = mt * kBM + lane_grp * 32 + lane;
                 float* ck = coef_rows(c.coef_k, s, b, h, s.dck) + (size_t)m * s.dck;
                 float* cv = coef_rows(c.coef_v, s, b, h, s.dcv) + (size_t)m * s.dcv;
 #pragma unroll 1
-                for (int col0 = 0; col0 < N; col0 += 32) {
+                for (int col0 = col_half * (N / 2); col0 < (col_half + 1) * (N / 2); col0 += 32) {
                     float v[32];
                     tmem_ld32(tmem_base + ((uint32_t)(lane_grp * 32) << 16) + (uint32_t)col0, v);
                     if (m < s.M) {
@@ -305,7 +332,7 @@ cudaError_t launch_tc_t(const CUtensorMap& tmK, const CUtensorMap& tmV, const Di
     const int row_tiles = (s.M + kBM - 1) / kBM;
     const int nkb = (n_mid + kBK - 1) / kBK;
     const int fixed = row_tiles * s.Hkv * s.B;
-    int n_tsplit = (kNumSms + fixed - 1) / fixed;            // about one CTA per SM
+    int n_tsplit = kNumSms / fixed;                          // one wave: one CTA per SM at most
     if (n_tsplit > nkb) n_tsplit = nkb;
     if (n_tsplit < 1) n_tsplit = 1;
     compress_tc_kernel<D><<<dim3(row_tiles, s.Hkv, s.B * n_tsplit), kThreadsTc, smem, stream>>>(tmK, tmV, s, c, L, n_tsplit);
