@@ -47,8 +47,7 @@ template <typename KV>
 __global__ void __launch_bounds__(256) partition_gather_kernel(Dims s, CacheDev c, const KV* __restrict__ K,
                                                                const KV* __restrict__ V, int64_t sb, int64_t st,
                                                                int64_t sh, int L) {
-    constexpr int EPV = 16 / (int)sizeof(KV);            // elements per 16-byte vector
-    __shared__ __align__(16) KV row_s[8][256];
+    __shared__ float row_s[8][256];
     int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     int h = blockIdx.y, b = blockIdx.z >> 1, side = blockIdx.z & 1;
     int n_init = min(L, s.l_init);
@@ -67,28 +66,23 @@ __global__ void __launch_bounds__(256) partition_gather_kernel(Dims s, CacheDev 
     void* w_init = side == 0 ? c.k_init : c.v_init;
     void* w_local = side == 0 ? c.k_local : c.v_local;
     void* w_mid = side == 0 ? c.k_mid : c.v_mid;
-    const int nvec = s.d / EPV;                          // 16-byte vectors per row (d is a multiple of 8)
-    const int nvec_full = nfull / EPV;
-    // gather indices of the kept dims this lane assembles: vector lane, lane + 32, ... of the output row
     int t_end = min(L, (int)(blockIdx.x + 1) * kRowsPerCta);
     for (int t = blockIdx.x * kRowsPerCta + warp; t < t_end; t += 8) {
-        const uint4* src = reinterpret_cast<const uint4*>(X + (size_t)b * sb + (size_t)t * st + (size_t)h * sh);
-        if (t < n_init || t >= L - n_local) {            // Eq.1: window rows, copied whole
-            KV* dst = t < n_init ? win_row<KV>(w_init, s, b, h, s.l_init, t)
-                                 : win_row<KV>(w_local, s, b, h, s.l_local, t - (L - n_local));
-            for (int v = lane; v < nvec; v += 32) reinterpret_cast<uint4*>(dst)[v] = src[v];
-        } else {                                         // Eq.2: kept dims of a middle row
-            const int j = t - n_init, a = j / s.P;
-            for (int v = lane; v < nvec; v += 32) reinterpret_cast<uint4*>(row_s[warp])[v] = src[v];
+        const KV* src = X + (size_t)b * sb + (size_t)t * st + (size_t)h * sh;
+        if (t < n_init) {
+            KV* dst = win_row<KV>(w_init, s, b, h, s.l_init, t);
+            for (int e = lane; e < s.d; e += 32) dst[e] = src[e];
+        } else if (t >= L - n_local) {
+            KV* dst = win_row<KV>(w_local, s, b, h, s.l_local, t - (L - n_local));
+            for (int e = lane; e < s.d; e += 32) dst[e] = src[e];
+        } else {
+            int j = t - n_init;
+            for (int e = lane; e < s.d; e += 32) row_s[warp][e] = ld_f(src + e);
             __syncwarp();
-            KV* dst = mid_row<KV>(w_mid, s, b, h, j % s.P, a, nfull);
-            for (int v = lane; v < nvec_full; v += 32) {
-                __align__(16) KV out[EPV];
-#pragma unroll
-                for (int i = 0; i < EPV; ++i) out[i] = row_s[warp][idf[v * EPV + i]];
-                // bf16 V^mu rows keep their 8-dim chunks permuted (one chunk = one vector)
-                const int pv = (side == 1 && sizeof(KV) == 2) ? (v ^ v_swz(a, nfull >> 3)) : v;
-                reinterpret_cast<uint4*>(dst)[pv] = *reinterpret_cast<const uint4*>(out);
+            KV* dst = mid_row<KV>(w_mid, s, b, h, j % s.P, j / s.P, nfull);
+            for (int e = lane; e < nfull; e += 32) {
+                const int col = side == 1 ? v_mid_col(j / s.P, e, nfull, sizeof(KV) == 2 ? FA_BF16 : FA_F32) : e;
+                st_f(dst + col, row_s[warp][idf[e]]);
             }
             __syncwarp();
         }
