@@ -38,7 +38,7 @@ UNIT = "us/step"
 SEED = 1000          # 1000 * config index
 # dram__bytes_read.sum + dram__bytes_write.sum per fa_decode_attention call from the committed
 # ncu capture (profiles/); None until a capture of the current kernels has been summarised.
-NCU_TRAFFIC_BYTES_PER_CALL = None
+NCU_TRAFFIC_BYTES_PER_CALL = 50543360   # profiles/decode_append_compress_cfg1_counters.md: 3.19 + 39.43 + 7.92 MB
 
 
 def _peaks():

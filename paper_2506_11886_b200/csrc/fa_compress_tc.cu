@@ -27,7 +27,6 @@ namespace {
 using bf16 = __nv_bfloat16;
 constexpr int kBM = 128;          // coefficient rows per CTA
 constexpr int kBK = 64;           // tokens per pipeline stage
-constexpr int kStagesTc = 4;
 constexpr int kGenWarps = 8;       // basis generators (and epilogue): 16 tokens of two rows per thread and stage
 constexpr int kThreadsTc = 64 + 32 * kGenWarps;
 constexpr uint32_t kSpinLimitTc = 1u << 24;
@@ -98,16 +97,20 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&v)[32]) {
     for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
 }
 
-// D = head dim (64 or 128): N = 2 D accumulator columns.
-template <int D>
+// D = head dim (64 or 128): N = 2 D accumulator columns per KV head; HP heads share one CTA and one
+// generated basis tile (HP * N <= 512 tensor-memory columns).
+template <int D, int HP>
 __global__ void __launch_bounds__(kThreadsTc, 1) compress_tc_kernel(const __grid_constant__ CUtensorMap tmK,
                                                                     const __grid_constant__ CUtensorMap tmV, Dims s,
                                                                     CacheDev c, int L, int n_tsplit) {
     constexpr int N = 2 * D;
     constexpr int kABytes = kBM * kBK * 2;                 // 16 KB basis tile
     constexpr int kBoxBytes = kBK * 64 * 2;                // 8 KB per [64 tokens x 64 dims] box
-    constexpr int kBBytes = (N / 64) * kBoxBytes;
+    constexpr int kBBytes1 = (N / 64) * kBoxBytes;          // one head
+    constexpr int kBBytes = HP * kBBytes1;
     constexpr int kStageBytesTc = kABytes + kBBytes;
+    constexpr int kStagesTc = (200 * 1024) / kStageBytesTc < 4 ? (200 * 1024) / kStageBytesTc : 4;
+    constexpr uint32_t kTmemCols = HP * N;
     constexpr uint32_t kIdesc = (1u << 4) | (1u << 7) | (1u << 10) | (1u << 16) | ((uint32_t)(N >> 3) << 17) | ((uint32_t)(kBM >> 4) << 24);
     extern __shared__ unsigned char smem_unaligned[];
     unsigned char* smem = smem_unaligned + ((1024u - (smem_u32(smem_unaligned) & 1023u)) & 1023u);
@@ -118,10 +121,10 @@ __global__ void __launch_bounds__(kThreadsTc, 1) compress_tc_kernel(const __grid
     uint64_t* acc_ready = empty + kStagesTc;
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_ready + 1);
     volatile int* fail = reinterpret_cast<volatile int*>(tmem_slot + 1);
-    int* inv = reinterpret_cast<int*>(tmem_slot + 4);      // [2][D]: dim -> slot in D^kc / D^vc, or -1
+    int* inv = reinterpret_cast<int*>(tmem_slot + 4);      // [HP][2][D]: dim -> slot in D^kc / D^vc, or -1
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int mt = blockIdx.x, h = blockIdx.y;
+    const int mt = blockIdx.x, h0 = blockIdx.y * HP;
     const int b = blockIdx.z / n_tsplit, split = blockIdx.z % n_tsplit;
     const int n_init = min(L, s.l_init);
     const int n_local = min(L - n_init, s.l_local);
@@ -136,14 +139,15 @@ __global__ void __launch_bounds__(kThreadsTc, 1) compress_tc_kernel(const __grid
         *fail = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
-    for (int i = tid; i < 2 * D; i += kThreadsTc) inv[i] = -1;
+    for (int i = tid; i < HP * 2 * D; i += kThreadsTc) inv[i] = -1;
     __syncthreads();
-    for (int i = tid; i < s.dck + s.dcv; i += kThreadsTc) {
-        if (i < s.dck) inv[c.idx_comp_k[(size_t)h * s.dck + i]] = i;
-        else inv[D + c.idx_comp_v[(size_t)h * s.dcv + (i - s.dck)]] = i - s.dck;
+    for (int i = tid; i < HP * (s.dck + s.dcv); i += kThreadsTc) {
+        const int hh = i / (s.dck + s.dcv), r = i - hh * (s.dck + s.dcv);
+        if (r < s.dck) inv[hh * N + c.idx_comp_k[(size_t)(h0 + hh) * s.dck + r]] = r;
+        else inv[hh * N + D + c.idx_comp_v[(size_t)(h0 + hh) * s.dcv + (r - s.dck)]] = r - s.dck;
     }
     if (warp == 1) {                                       // tensor memory: N fp32 columns x 128 lanes
-        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"((uint32_t)N) : "memory");
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(kTmemCols) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
@@ -162,11 +166,13 @@ __global__ void __launch_bounds__(kThreadsTc, 1) compress_tc_kernel(const __grid
                     mbar_expect_tx(fullB + st, (uint32_t)kBBytes);
                     const int tok = n_init + kb * kBK;
 #pragma unroll
-                    for (int bx = 0; bx < N / 64; ++bx) {
-                        const CUtensorMap* tm = bx < D / 64 ? &tmK : &tmV;
-                        const int dim0 = (bx % (D / 64)) * 64;
-                        tma_load_4d(bdst + bx * kBoxBytes, tm, dim0, h, tok, b, fullB + st);
-                    }
+                    for (int hh = 0; hh < HP; ++hh)
+#pragma unroll
+                        for (int bx = 0; bx < N / 64; ++bx) {
+                            const CUtensorMap* tm = bx < D / 64 ? &tmK : &tmV;
+                            const int dim0 = (bx % (D / 64)) * 64;
+                            tma_load_4d(bdst + hh * kBBytes1 + bx * kBoxBytes, tm, dim0, h0 + hh, tok, b, fullB + st);
+                        }
                 }
             }
         } else if (warp == 1) {
@@ -184,8 +190,11 @@ __global__ void __launch_bounds__(kThreadsTc, 1) compress_tc_kernel(const __grid
                         // A: K-major, rows of 128 bytes, 8-row groups 1024 bytes apart; 16 tokens = 32 bytes along the row
                         const uint64_t adesc = umma_desc(a_addr + ks * 32, 1, 1024 >> 4);
                         // B: MN-major, 64 dims per 128-byte row, 8-token groups 1024 bytes apart, next 64 dims one box further
-                        const uint64_t bdesc = umma_desc(b_addr + ks * 2048, kBoxBytes >> 4, 1024 >> 4);
-                        umma_bf16(tmem_base, adesc, bdesc, kIdesc, (it > 0 || ks > 0) ? 1u : 0u);
+#pragma unroll
+                        for (int hh = 0; hh < HP; ++hh) {
+                            const uint64_t bdesc = umma_desc(b_addr + hh * kBBytes1 + ks * 2048, kBoxBytes >> 4, 1024 >> 4);
+                            umma_bf16(tmem_base + hh * N, adesc, bdesc, kIdesc, (it > 0 || ks > 0) ? 1u : 0u);
+                        }
                     }
                     umma_commit(empty + st);               // frees the stage when these MMAs have read it
                 }
@@ -268,17 +277,19 @@ __global__ void __launch_bounds__(kThreadsTc, 1) compress_tc_kernel(const __grid
                 const int lane_grp = warp & 3;             // a warp reads tensor-memory lanes 32 (warp % 4) ...
                 const int col_half = (warp - 2) >> 2;      // two warps share a lane group: one column half each
                 const int m = mt * kBM + lane_grp * 32 + lane;
-                float* ck = coef_rows(c.coef_k, s, b, h, s.dck) + (size_t)m * s.dck;
-                float* cv = coef_rows(c.coef_v, s, b, h, s.dcv) + (size_t)m * s.dcv;
+                constexpr int kHalf = (int)kTmemCols / 2;
 #pragma unroll 1
-                for (int col0 = col_half * (N / 2); col0 < (col_half + 1) * (N / 2); col0 += 32) {
+                for (int col0 = col_half * kHalf; col0 < (col_half + 1) * kHalf; col0 += 32) {
+                    const int hh = col0 / N, hcol0 = col0 - hh * N;
+                    float* ck = coef_rows(c.coef_k, s, b, h0 + hh, s.dck) + (size_t)m * s.dck;
+                    float* cv = coef_rows(c.coef_v, s, b, h0 + hh, s.dcv) + (size_t)m * s.dcv;
                     float v[32];
                     tmem_ld32(tmem_base + ((uint32_t)(lane_grp * 32) << 16) + (uint32_t)col0, v);
                     if (m < s.M) {
 #pragma unroll
                         for (int i = 0; i < 32; ++i) {
-                            const int col = col0 + i;
-                            const int slot = inv[col];
+                            const int col = hcol0 + i;
+                            const int slot = inv[hh * N + col];
                             if (slot >= 0) atomicAdd((col < D ? ck : cv) + slot, v[i]);
                         }
                     }
@@ -290,7 +301,7 @@ __global__ void __launch_bounds__(kThreadsTc, 1) compress_tc_kernel(const __grid
     __syncthreads();
     if (warp == 1) {
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)N) : "memory");
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
     }
 }
 
@@ -321,21 +332,22 @@ bool make_map(CUtensorMap* tm, const void* base, const Dims& s, int64_t sb, int6
               CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-template <int D>
+template <int D, int HP>
 cudaError_t launch_tc_t(const CUtensorMap& tmK, const CUtensorMap& tmV, const Dims& s, const CacheDev& c, int L, int n_mid,
                         cudaStream_t stream) {
     constexpr int N = 2 * D;
-    constexpr size_t stage = (size_t)kBM * kBK * 2 + (size_t)(N / 64) * kBK * 64 * 2;
-    const size_t smem = kStagesTc * stage + 8 * (3 * kStagesTc + 1) + 16 + sizeof(int) * 2 * D + 64 + 1024;
-    cudaError_t err = ensure_dynamic_smem(compress_tc_kernel<D>, smem);
+    constexpr size_t stage = (size_t)kBM * kBK * 2 + (size_t)HP * (N / 64) * kBK * 64 * 2;
+    constexpr size_t n_stages = (200 * 1024) / stage < 4 ? (200 * 1024) / stage : 4;
+    const size_t smem = n_stages * stage + 8 * (3 * n_stages + 1) + 16 + sizeof(int) * HP * 2 * D + 64 + 1024;
+    cudaError_t err = ensure_dynamic_smem(compress_tc_kernel<D, HP>, smem);
     if (err != cudaSuccess) return err;
     const int row_tiles = (s.M + kBM - 1) / kBM;
     const int nkb = (n_mid + kBK - 1) / kBK;
-    const int fixed = row_tiles * s.Hkv * s.B;
+    const int fixed = row_tiles * (s.Hkv / HP) * s.B;
     int n_tsplit = kNumSms / fixed;                          // one wave: one CTA per SM at most
     if (n_tsplit > nkb) n_tsplit = nkb;
     if (n_tsplit < 1) n_tsplit = 1;
-    compress_tc_kernel<D><<<dim3(row_tiles, s.Hkv, s.B * n_tsplit), kThreadsTc, smem, stream>>>(tmK, tmV, s, c, L, n_tsplit);
+    compress_tc_kernel<D, HP><<<dim3(row_tiles, s.Hkv / HP, s.B * n_tsplit), kThreadsTc, smem, stream>>>(tmK, tmV, s, c, L, n_tsplit);
     return cudaGetLastError();
 }
 
@@ -361,8 +373,9 @@ cudaError_t launch_compress_tc(const Dims& s, const CacheDev& c, const void* K, 
     if (n_mid <= 0) return cudaSuccess;
     CUtensorMap tmK, tmV;
     if (!make_map(&tmK, K, s, sb, st, sh, L) || !make_map(&tmV, V, s, sb, st, sh, L)) return cudaErrorInvalidValue;
-    if (s.d == 128) return launch_tc_t<128>(tmK, tmV, s, c, L, n_mid, stream);
-    return launch_tc_t<64>(tmK, tmV, s, c, L, n_mid, stream);
+    const bool pair = s.Hkv % 2 == 0;                        // two heads share a CTA and its basis tile
+    if (s.d == 128) return pair ? launch_tc_t<128, 2>(tmK, tmV, s, c, L, n_mid, stream) : launch_tc_t<128, 1>(tmK, tmV, s, c, L, n_mid, stream);
+    return pair ? launch_tc_t<64, 2>(tmK, tmV, s, c, L, n_mid, stream) : launch_tc_t<64, 1>(tmK, tmV, s, c, L, n_mid, stream);
 }
 
 }  // namespace fa
