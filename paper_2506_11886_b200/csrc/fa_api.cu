@@ -88,10 +88,10 @@ fa_status plan_decode(const fa_layout& l, DecodePlan* p) {
         p->gh = gh_fft;
         p->n_pass = (s.G + p->gh - 1) / p->gh;
         // classes are indivisible: pick the split count that minimises waves * classes per CTA
-        // with two CTAs resident per SM (phases of one overlap the other's), smallest count on
-        // ties to keep the partial results small
+        // with one CTA per SM (a deep ring of stages and a whole batch of classes per CTA), smallest
+        // count on ties to keep the partial results small
         const int jobs = s.B * s.Hkv * p->n_pass;
-        const int slots = 2 * kNumSms;
+        const int slots = kNumSms;
         int best = 1;
         long long best_cost = -1;
         for (int n = 1; n <= s.P && n <= 64; ++n) {
@@ -100,15 +100,13 @@ fa_status plan_decode(const fa_layout& l, DecodePlan* p) {
             if (best_cost < 0 || cost < best_cost) { best_cost = cost; best = n; }
         }
         p->n_split = best;
-        // classes transformed together: enough butterflies for all consumer threads, while two CTAs
-        // still fit the shared memory of an SM (else one)
+        // classes transformed together: enough butterflies for all consumer threads, within shared memory
         const int S = s.T / s.P;
         int nb = 2048 / S;
         if (nb < 1) nb = 1;
         if (nb > 8) nb = 8;
         const int per_cta = (s.P + best - 1) / best;
         if (nb > per_cta) nb = per_cta;
-        while (nb > 1 && decode_fft_smem_bytes(s, log2S, p->gh, nb) > 113 * 1024) --nb;
         while (nb > 1 && decode_fft_smem_bytes(s, log2S, p->gh, nb) > 227 * 1024) --nb;
         p->nb = nb;
     } else {

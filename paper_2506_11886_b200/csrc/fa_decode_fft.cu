@@ -33,7 +33,7 @@ namespace {
 constexpr int kConsumers = 256;
 constexpr int kThreads = kConsumers + 32;
 constexpr int kStageBytes = 16384;
-constexpr int kStages = 2;
+constexpr int kStages = 6;
 constexpr int kWinRowsPerTile = 48;
 constexpr uint32_t kSpinLimit = 1u << 24;
 using bf16 = __nv_bfloat16;
@@ -330,7 +330,7 @@ template <int GH> __host__ __device__ constexpr int hperm(int s) { return GH == 
 
 // GH query heads per CTA (2 or 4), transform length S = 2^LS.
 template <int GH, int LS>
-__global__ void __launch_bounds__(kThreads, 2) decode_fft_kernel(Dims s, CacheDev c, DecodePlan p, const bf16* __restrict__ q,
+__global__ void __launch_bounds__(kThreads, 1) decode_fft_kernel(Dims s, CacheDev c, DecodePlan p, const bf16* __restrict__ q,
                                                                   char* wsp) {
     constexpr int N = GH / 2;
     constexpr int S = 1 << LS;
