@@ -59,8 +59,11 @@ typedef enum { FA_NORM_ORTHO = 0, FA_NORM_PAPER = 1 } fa_norm;
 /* How fa_decode_attention evaluates the compressed dims.  DIRECT sums the
  * n_coef basis terms per token; FFT evaluates each residue class of tokens
  * (token index mod mid_classes) with one length period/mid_classes transform.
- * AUTO picks FFT when the layout allows it. */
-typedef enum { FA_DECODE_AUTO = 0, FA_DECODE_DIRECT = 1, FA_DECODE_FFT = 2 } fa_decode_algo;
+ * AUTO picks FFT when the layout allows it.  FFT runs as one kernel whose CTAs
+ * wait for one another (cooperative launch) whenever every (batch, KV head) can
+ * have two or more CTAs resident at once, else as three kernels; FFT_SPLIT
+ * always takes the three-kernel form. */
+typedef enum { FA_DECODE_AUTO = 0, FA_DECODE_DIRECT = 1, FA_DECODE_FFT = 2, FA_DECODE_FFT_SPLIT = 3 } fa_decode_algo;
 
 /* Immutable description of one layer's cache. */
 typedef struct fa_layout {
@@ -116,8 +119,11 @@ typedef struct fa_cache_sizes {
 fa_status fa_cache_sizes_of(const fa_layout* layout, fa_cache_sizes* out);
 
 /* Host only.  Bytes of workspace fa_decode_attention and fa_compress need for this layout
- * (the larger of the two).  The workspace is scratch: its contents need not survive
- * between calls and need no initialisation. */
+ * (the larger of the two).  The workspace is scratch whose contents need not survive
+ * between calls, with one rule: its first 4 KiB hold barrier counters that must be zero
+ * when a call starts.  Zero-fill a new workspace once (cudaMemset); every call that ends
+ * without FA_ERR_TIMEOUT leaves the counters at zero again.  After FA_ERR_TIMEOUT
+ * zero-fill it before the next call. */
 fa_status fa_workspace_bytes(const fa_layout* layout, size_t* out);
 
 /* Clears state and status (an empty cache: no tokens, zero coefficients). */

@@ -22,7 +22,7 @@ fa_status check_layout(const fa_layout* l) {
     if (l->mid_classes < 1) return FA_ERR_INVALID_ARG;
     if (l->kv_dtype != FA_F32 && l->kv_dtype != FA_BF16) return FA_ERR_INVALID_ARG;
     if (l->norm != FA_NORM_ORTHO && l->norm != FA_NORM_PAPER) return FA_ERR_INVALID_ARG;
-    if (l->decode_algo < FA_DECODE_AUTO || l->decode_algo > FA_DECODE_FFT) return FA_ERR_INVALID_ARG;
+    if (l->decode_algo < FA_DECODE_AUTO || l->decode_algo > FA_DECODE_FFT_SPLIT) return FA_ERR_INVALID_ARG;
     if (!(l->softmax_scale > 0.0f)) return FA_ERR_INVALID_ARG;
     // what the kernels implement
     if (l->head_dim % 8 != 0 || l->head_dim > 256) return FA_ERR_UNSUPPORTED;
@@ -81,31 +81,61 @@ fa_status plan_decode(const fa_layout& l, DecodePlan* p) {
     int log2S = 0;
     const int gh_fft = s.G >= 3 ? 4 : 2;
     const bool can_fft = fft_ok(l, gh_fft, &log2S);
-    if (l.decode_algo == FA_DECODE_FFT && !can_fft) return FA_ERR_UNSUPPORTED;
+    const bool want_fft = l.decode_algo == FA_DECODE_FFT || l.decode_algo == FA_DECODE_FFT_SPLIT;
+    if (want_fft && !can_fft) return FA_ERR_UNSUPPORTED;
     p->algo = (l.decode_algo == FA_DECODE_DIRECT || !can_fft) ? FA_DECODE_DIRECT : FA_DECODE_FFT;
     p->fft_log2 = log2S;
     if (p->algo == FA_DECODE_FFT) {
         p->gh = gh_fft;
         p->n_pass = (s.G + p->gh - 1) / p->gh;
-        // classes are indivisible: pick the split count that minimises waves * classes per CTA
-        // with one CTA per SM (a deep ring of stages and a whole batch of classes per CTA), smallest
-        // count on ties to keep the partial results small
         const int jobs = s.B * s.Hkv * p->n_pass;
-        const int slots = kNumSms;
-        int best = 1;
-        long long best_cost = -1;
-        for (int n = 1; n <= s.P && n <= 64; ++n) {
-            long long waves = ((long long)jobs * n + slots - 1) / slots;
-            long long cost = waves * ((s.P + n - 1) / n);
-            if (best_cost < 0 || cost < best_cost) { best_cost = cost; best = n; }
+        // One CTA per SM (a deep ring of stages and a whole batch of classes per CTA).  When every
+        // (b, KV head, pass) can have at least two CTAs resident at once, the kernel is fused: it
+        // forms u itself and merges its own partial results, its CTAs waiting for one another
+        // (cooperative launch).  Window tokens then get CTAs of their own, as many as keeps their
+        // bytes per CTA at or below those of a class CTA.
+        const int per_job = kNumSms / jobs;
+        const long long win_bytes = 2LL * (s.l_init + s.l_local) * s.d;
+        const long long class_bytes = (long long)(s.T / s.P) * (s.nfk + s.nfv);
+        p->fused = 0;
+        p->n_wsplit = 0;
+        if (l.decode_algo != FA_DECODE_FFT_SPLIT && per_job >= 2) {
+            int best_ns = 0, best_nw = 0;
+            long long best_cost = -1;
+            for (int nw = (win_bytes > 0 ? 1 : 0); nw <= 8 && nw < per_job; ++nw) {
+                int ns = per_job - nw;
+                if (ns > s.P) ns = s.P;
+                const long long cc = (long long)((s.P + ns - 1) / ns) * class_bytes;
+                const long long wc = nw ? (win_bytes + nw - 1) / nw : 0;
+                const long long cost = cc > wc ? cc : wc;
+                if (best_cost < 0 || cost < best_cost) { best_cost = cost; best_ns = ns; best_nw = nw; }
+                if (nw == 0) break;
+            }
+            // fewest class CTAs that reach the same classes per CTA
+            const int per_cta = (s.P + best_ns - 1) / best_ns;
+            best_ns = (s.P + per_cta - 1) / per_cta;
+            p->fused = 1;
+            p->n_split = best_ns;
+            p->n_wsplit = best_nw;
+        } else {
+            // classes are indivisible: pick the split count that minimises waves * classes per CTA,
+            // smallest count on ties to keep the partial results small
+            const int slots = kNumSms;
+            int best = 1;
+            long long best_cost = -1;
+            for (int n = 1; n <= s.P && n <= 64; ++n) {
+                long long waves = ((long long)jobs * n + slots - 1) / slots;
+                long long cost = waves * ((s.P + n - 1) / n);
+                if (best_cost < 0 || cost < best_cost) { best_cost = cost; best = n; }
+            }
+            p->n_split = best;
         }
-        p->n_split = best;
         // classes transformed together: enough butterflies for all consumer threads, within shared memory
         const int S = s.T / s.P;
         int nb = 2048 / S;
         if (nb < 1) nb = 1;
         if (nb > 8) nb = 8;
-        const int per_cta = (s.P + best - 1) / best;
+        const int per_cta = (s.P + p->n_split - 1) / p->n_split;
         if (nb > per_cta) nb = per_cta;
         while (nb > 1 && decode_fft_smem_bytes(s, log2S, p->gh, nb) > 227 * 1024) --nb;
         p->nb = nb;
@@ -123,14 +153,18 @@ fa_status plan_decode(const fa_layout& l, DecodePlan* p) {
         if (want < 1) want = 1;
         p->n_split = want;
     }
+    p->n_part = p->n_split + p->n_wsplit;
     p->rows_pro = 32;
     p->n_slice = s.dcv > 0 ? (s.M + 63) / 64 : 1;
     size_t off = 0;
+    p->off_bar = off; off = align_up(off + sizeof(int32_t) * 4 * (size_t)kNumSms, 256);     // same place for every layout
     p->off_u = off;   off = align_up(off + sizeof(float) * (size_t)s.B * s.Hq * s.M, 256);
-    p->off_ml = off;  off = align_up(off + sizeof(float) * (size_t)s.B * s.Hq * p->n_split * 2, 256);
-    p->off_o = off;   off = align_up(off + sizeof(float) * (size_t)s.B * s.Hq * p->n_split * s.d, 256);
-    p->off_z = off;   off = align_up(off + sizeof(float) * (size_t)s.B * s.Hq * p->n_split * s.M, 256);
-    p->off_oc = off;  off = align_up(off + sizeof(float) * (size_t)s.B * s.Hq * p->n_slice * (s.dcv > 0 ? s.dcv : 1), 256);
+    p->off_ml = off;  off = align_up(off + sizeof(float) * (size_t)s.B * s.Hq * p->n_part * 2, 256);
+    p->off_o = off;   off = align_up(off + sizeof(float) * (size_t)s.B * s.Hq * p->n_part * s.d, 256);
+    p->off_z = off;   off = align_up(off + sizeof(float) * (size_t)s.B * s.Hq * p->n_part * s.M, 256);
+    const int n_oc = p->n_slice > p->n_part ? p->n_slice : p->n_part;
+    p->off_oc = off;  off = align_up(off + sizeof(float) * (size_t)s.B * s.Hq * n_oc * (s.dcv > 0 ? s.dcv : 1), 256);
+    p->off_om = off;  off = align_up(off + sizeof(float) * (size_t)s.B * s.Hq * s.d, 256);
     p->off_cnt = off; off = align_up(off + sizeof(int32_t) * (size_t)s.B * s.Hkv, 256);
     p->total = off;
     return FA_OK;
@@ -283,9 +317,13 @@ fa_status fa_decode_attention(const fa_layout* layout, const fa_cache* cache, co
     CacheDev c = make_cache(*cache);
     cudaStream_t cs = static_cast<cudaStream_t>(stream);
     char* w = static_cast<char*>(ws);
+    if (p.fused) {
+        if (launch_decode_fft(s, c, layout->kv_dtype, p, q, out, w, cs) != cudaSuccess) return FA_ERR_CUDA;
+        return FA_OK;
+    }
     if (launch_decode_prologue(s, c, layout->kv_dtype, p, q, w, cs) != cudaSuccess) return FA_ERR_CUDA;
     if (p.algo == FA_DECODE_FFT) {
-        if (launch_decode_fft(s, c, layout->kv_dtype, p, q, w, cs) != cudaSuccess) return FA_ERR_CUDA;
+        if (launch_decode_fft(s, c, layout->kv_dtype, p, q, out, w, cs) != cudaSuccess) return FA_ERR_CUDA;
     } else {
         if (launch_decode_direct(s, c, layout->kv_dtype, p, q, w, cs) != cudaSuccess) return FA_ERR_CUDA;
     }

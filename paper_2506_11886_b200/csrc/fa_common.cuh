@@ -61,13 +61,16 @@ struct DecodePlan {
     int algo;          // FA_DECODE_DIRECT or FA_DECODE_FFT
     int gh;            // query heads of one KV head handled together by one CTA (<= 4)
     int n_pass;        // ceil(G / gh)
-    int n_split;       // CTAs that share the tokens of one (b, KV head)
+    int n_split;       // CTAs that share the middle tokens of one (b, KV head, pass)
+    int n_wsplit;      // CTAs that hold only window tokens (0: the windows are spread over the n_split CTAs)
+    int n_part;        // n_split + n_wsplit: partial results per query head
+    int fused;         // 1: the main kernel also forms u and merges the partial results (cooperative launch)
     int n_slice;       // CTAs that share the coefficient rows of one (b, KV head) in the epilogue
     int rows_pro;      // coefficient rows per prologue CTA
     int fft_log2;      // log2 of the transform length (FFT path)
     int nb;            // classes transformed together by one CTA (FFT path)
     // workspace offsets in bytes
-    size_t off_u, off_ml, off_o, off_z, off_oc, off_cnt, total;
+    size_t off_bar, off_u, off_ml, off_o, off_z, off_oc, off_om, off_cnt, total;
 };
 
 // V^mu of bf16 caches is stored with its 16-byte chunks (8 dims) permuted inside each row:
@@ -104,7 +107,7 @@ cudaError_t launch_decode_prologue(const Dims&, const CacheDev&, int dtype, cons
                                    cudaStream_t);
 cudaError_t launch_decode_direct(const Dims&, const CacheDev&, int dtype, const DecodePlan&, const void* q, char* ws,
                                  cudaStream_t);
-cudaError_t launch_decode_fft(const Dims&, const CacheDev&, int dtype, const DecodePlan&, const void* q, char* ws,
+cudaError_t launch_decode_fft(const Dims&, const CacheDev&, int dtype, const DecodePlan&, const void* q, void* out, char* ws,
                               cudaStream_t);
 size_t decode_fft_smem_bytes(const Dims&, int log2S, int gh, int nb);
 cudaError_t launch_decode_epilogue(const Dims&, const CacheDev&, int dtype, const DecodePlan&, void* out, char* ws,

@@ -253,14 +253,14 @@ __global__ void __launch_bounds__(256) decode_direct_kernel(Dims s, CacheDev c, 
         int g = i / s.d, e = i - g * s.d;
         float v = o_s[i];
         for (int tg = 0; tg < ntg_win; ++tg) v += acc_s[(tg * s.d + e) * GH + g];
-        if (g < ng) ws.o[(((size_t)b * s.Hq + g_first + g) * p.n_split + split) * s.d + e] = v;
+        if (g < ng) ws.o[(((size_t)b * s.Hq + g_first + g) * p.n_part + split) * s.d + e] = v;
     }
     for (int i = tid; i < GH * s.M; i += blockDim.x) {
         int g = i / s.M, m = i - g * s.M;
-        if (g < ng) ws.z[(((size_t)b * s.Hq + g_first + g) * p.n_split + split) * s.M + m] = z_s[i];
+        if (g < ng) ws.z[(((size_t)b * s.Hq + g_first + g) * p.n_part + split) * s.M + m] = z_s[i];
     }
     if (tid < ng) {
-        float* ml = ws.ml + (((size_t)b * s.Hq + g_first + tid) * p.n_split + split) * 2;
+        float* ml = ws.ml + (((size_t)b * s.Hq + g_first + tid) * p.n_part + split) * 2;
         float mv = kNegBig, lv = 0.f;
 #pragma unroll
         for (int g = 0; g < GH; ++g) if (g == tid) { mv = rs.m[g]; lv = rs.l[g]; }

@@ -75,6 +75,30 @@ __device__ __forceinline__ void bulk_g2s(void* dst, const void* src, uint32_t by
 }
 __device__ __forceinline__ void consumer_sync() { asm volatile("bar.sync 1, 256;" ::: "memory"); }
 
+// Barrier among the CTAs of one (b, KV head, pass) on a global counter (fused kernel only: a
+// cooperative launch makes all of them resident).  Arrive: every consumer thread has fenced its
+// global writes; one thread adds 1 with release semantics.  Wait: one thread polls with acquire
+// loads, bounded like every other wait of this kernel, then the consumer warps meet.
+__device__ __forceinline__ void part_arrive(int32_t* cnt, int tid) {
+    __threadfence();
+    consumer_sync();
+    if (tid == 0) asm volatile("red.release.gpu.global.add.s32 [%0], 1;" ::"l"(cnt) : "memory");
+}
+__device__ __forceinline__ void part_wait(const int32_t* cnt, int n, int tid, volatile int* fail, int32_t* status) {
+    if (tid == 0 && !*fail) {
+        bool ok = false;
+        for (uint32_t i = 0; i < (1u << 22); ++i) {
+            int v;
+            asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(cnt) : "memory");
+            if (v >= n) { ok = true; break; }
+            if (i > 64) __nanosleep(64);
+        }
+        if (!ok) { *fail = 1; atomicExch(status, (int)FA_ERR_TIMEOUT); }
+    }
+    consumer_sync();
+}
+__device__ __forceinline__ float ldcg_f(const float* p) { return __ldcg(p); }
+
 __device__ __forceinline__ void mma_bf16(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0,
                                          uint32_t b1) {
     asm volatile(
@@ -317,9 +341,9 @@ __host__ __device__ inline FftSmem fft_smem_layout(int log2S, int k, int GH, int
     L.twf_off = off; off += 8 * (tw_total(log2S) + 1);
     L.rev_off = off; off += 2 * S;
     off = (off + 15) / 16 * 16;
-    L.E_off = off; off += 8 * k;
-    L.ut_off = off; off += 8 * k * GH;
-    L.z_off = off; off += 8 * k * GH;
+    L.E_off = off; off += (8 * k + 15) / 16 * 16;
+    L.ut_off = off; off += (8 * k * GH + 15) / 16 * 16;
+    L.z_off = off; off += (8 * k * GH + 15) / 16 * 16;
     L.o_off = off; off += 4 * GH * d;
     L.red_off = off; off += 4 * (8 * GH + GH + 8);
     L.total = (off + 127) / 128 * 128;
@@ -331,7 +355,7 @@ template <int GH> __host__ __device__ constexpr int hperm(int s) { return GH == 
 // GH query heads per CTA (2 or 4), transform length S = 2^LS.
 template <int GH, int LS>
 __global__ void __launch_bounds__(kThreads, 1) decode_fft_kernel(Dims s, CacheDev c, DecodePlan p, const bf16* __restrict__ q,
-                                                                  char* wsp) {
+                                                                  bf16* __restrict__ out, char* wsp) {
     constexpr int N = GH / 2;
     constexpr int S = 1 << LS;
     extern __shared__ __align__(128) unsigned char smem_raw[];
@@ -355,7 +379,8 @@ __global__ void __launch_bounds__(kThreads, 1) decode_fft_kernel(Dims s, CacheDe
     float* red_s = reinterpret_cast<float*>(smem_raw + L.red_off);        // [8][GH] + l_s[GH]
     const int fb_floats = L.fb_floats, pbs = L.pbs;
 
-    const int split = blockIdx.x;
+    const int part = blockIdx.x;                          // partial-result index: class CTAs, then window CTAs
+    const bool is_win = part >= p.n_split;
     const int h = blockIdx.y / p.n_pass, pass = blockIdx.y % p.n_pass;
     const int b = blockIdx.z;
     const int g_first = h * s.G + pass * GH;
@@ -365,16 +390,23 @@ __global__ void __launch_bounds__(kThreads, 1) decode_fft_kernel(Dims s, CacheDe
 
     const int n_init = c.state[kStateStride * b + 0], n_local = c.state[kStateStride * b + 1];
     const int n_mid = min(c.state[kStateStride * b + 2], s.max_mid), head = c.state[kStateStride * b + 3];
-    const int c0 = (int)((long long)split * s.P / p.n_split), c1 = (int)((long long)(split + 1) * s.P / p.n_split);
+    const int c0 = is_win ? 0 : (int)((long long)part * s.P / p.n_split);
+    const int c1 = is_win ? 0 : (int)((long long)(part + 1) * s.P / p.n_split);
     const int n_win = n_init + n_local;
-    const int w0 = (int)((long long)split * n_win / p.n_split), w1 = (int)((long long)(split + 1) * n_win / p.n_split);
+    // window tokens: spread over the class CTAs, or over CTAs of their own
+    const int wi = p.n_wsplit ? part - p.n_split : part, wn = p.n_wsplit ? p.n_wsplit : p.n_split;
+    const bool has_win = p.n_wsplit ? is_win : true;
+    const int w0 = has_win ? (int)((long long)wi * n_win / wn) : 0, w1 = has_win ? (int)((long long)(wi + 1) * n_win / wn) : 0;
     auto n_of_class = [&](int cls) { return cls < n_mid ? (n_mid - cls + s.P - 1) >> log2P : 0; };
 
     const int rowb_k = s.nfk * 2, rowb_v = s.nfv * 2, rowb_w = s.d * 2;
     const int rbw_pad = rowb_w + 16;                                       // padded window row in shared memory
     const int ts_k = rowb_k ? (kStageBytes / rowb_k) & ~15 : 0, ts_v = rowb_v ? (kStageBytes / rowb_v) & ~15 : 0;
     const int ts_w = kWinRowsPerTile;
-    constexpr int wchunk = S;
+    // window tokens per softmax chunk: the score and probability buffers of all NB classes when
+    // they can be addressed as one, else those of one class
+    const int wchunk = pf_size(NB * S * GH) <= NB * L.fb_floats ? NB * S : S;
+    const int pbw = NB * L.pbs;                            // row stride of the window probabilities
 
     if (tid == 0) {
         for (int i = 0; i < kStages; ++i) { mbar_init(full + i, 1); mbar_init(empty + i, 8); }
@@ -455,7 +487,6 @@ __global__ void __launch_bounds__(kThreads, 1) decode_fft_kernel(Dims s, CacheDe
     const float sl2 = s.scale * kLog2e;
 
     // ---- one-time set-up ----
-    for (int i = tid; i < GH * s.d; i += kConsumers) o_s[i] = 0.f;
     for (int i = tid; i < s.k; i += kConsumers) {
         E[i] = cis_frac((float)i / (float)s.T);
     }
@@ -491,8 +522,62 @@ __global__ void __launch_bounds__(kThreads, 1) decode_fft_kernel(Dims s, CacheDe
                 qk[rd][ks][1] = on ? pack_bf16(qrow[idf_k[e0 + 2]], qrow[idf_k[e0 + 3]]) : 0u;
             }
     }
-    // everything above is independent of the prologue kernel; its output u is first needed here
-    asm volatile("griddepcontrol.wait;" ::: "memory");
+    int32_t* bar = ws.bar + 4 * (((size_t)b * s.Hkv + h) * p.n_pass + pass);
+    const int m0 = (int)((long long)part * s.M / p.n_part), m1 = (int)((long long)(part + 1) * s.M / p.n_part);
+    if (p.fused) {
+        // this CTA's slice of the coefficient rows of C^V will be wanted at the very end: start it towards L2
+        if (s.dcv > 0) {
+            const char* cv = reinterpret_cast<const char*>(coef_rows(c.coef_v, s, b, h, s.dcv) + (size_t)m0 * s.dcv);
+            const int bytes = (m1 - m0) * s.dcv * 4;
+            for (int o = tid * 128; o < bytes; o += kConsumers * 128) asm volatile("prefetch.global.L2 [%0];" ::"l"(cv + o));
+        }
+        // u_g[m] = scale * log2(e) * w_m * sum_e C^K[m][e] q_g[D^kc[e]] for rows [m0, m1): eight lanes per row
+        if (s.dck > 0) {
+            float* qc = o_s;                               // [GH][dck] gathered query, fp32
+            const int32_t* idc_k = c.idx_comp_k + (size_t)h * s.dck;
+            for (int i = tid; i < GH * s.dck; i += kConsumers) {
+                const int g = i / s.dck, e = i - g * s.dck;
+                qc[i] = g < ng ? __bfloat162float(q[((size_t)b * s.Hq + g_first + g) * s.d + idc_k[e]]) : 0.f;
+            }
+            consumer_sync();
+            const float* ck = coef_rows(c.coef_k, s, b, h, s.dck);
+            const int l8 = tid & 7, rgi = tid >> 3, nv = s.dck >> 2;
+            for (int r0 = m0; r0 < m1; r0 += kConsumers / 8) {
+                const int r = r0 + rgi;
+                float a[GH];
+#pragma unroll
+                for (int g = 0; g < GH; ++g) a[g] = 0.f;
+                if (r < m1) {
+                    const float4* row = reinterpret_cast<const float4*>(ck + (size_t)r * s.dck);
+                    for (int v = l8; v < nv; v += 8) {
+                        const float4 x = __ldg(row + v);
+#pragma unroll
+                        for (int g = 0; g < GH; ++g) {
+                            const float4 y = *reinterpret_cast<const float4*>(qc + g * s.dck + 4 * v);
+                            a[g] = fmaf(x.x, y.x, fmaf(x.y, y.y, fmaf(x.z, y.z, fmaf(x.w, y.w, a[g]))));
+                        }
+                    }
+                }
+#pragma unroll
+                for (int g = 0; g < GH; ++g) {
+                    a[g] += __shfl_xor_sync(0xffffffffu, a[g], 1);
+                    a[g] += __shfl_xor_sync(0xffffffffu, a[g], 2);
+                    a[g] += __shfl_xor_sync(0xffffffffu, a[g], 4);
+                }
+                float mine = a[0];
+#pragma unroll
+                for (int g = 1; g < GH; ++g) if (l8 == g) mine = a[g];
+                if (r < m1 && l8 < ng)
+                    ws.u[((size_t)b * s.Hq + g_first + l8) * s.M + r] = recon_weight(s.norm, r, s.k, s.T) * sl2 * mine;
+            }
+            part_arrive(bar + 0, tid);
+            if (!is_win) part_wait(bar + 0, p.n_part, tid, fail, c.status);
+        }
+    } else {
+        // everything above is independent of the prologue kernel; its output u is first needed here
+        asm volatile("griddepcontrol.wait;" ::: "memory");
+    }
+    for (int i = tid; i < GH * s.d; i += kConsumers) o_s[i] = 0.f;
     // ut[n] = (A.re, A.im, B.re, B.im), A = heads of the real slots, B = heads of the imaginary slots;
     // all loads of an entry are issued together
     for (int n = tid; n < s.k; n += kConsumers) {
@@ -501,7 +586,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_fft_kernel(Dims s, CacheDe
         for (int sl = 0; sl < GH; ++sl) {
             const int g = hperm<GH>(sl);
             uv[sl] = make_float2(0.f, 0.f);
-            if (g < ng && s.dck > 0) uv[sl] = *reinterpret_cast<const float2*>(ws.u + ((size_t)b * s.Hq + g_first + g) * s.M + 2 * n);
+            if (g < ng && s.dck > 0 && !is_win) uv[sl] = __ldcg(reinterpret_cast<const float2*>(ws.u + ((size_t)b * s.Hq + g_first + g) * s.M + 2 * n));
         }
         float* e = ut + n * 2 * GH;
         float* zz = z_s + n * 2 * GH;
@@ -671,7 +756,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_fft_kernel(Dims s, CacheDe
                 for (int g = 0; g < GH; ++g) {
                     v[g] = a < n_tok ? ex2(v[g] - m_run[g]) : 0.f;
                     l_acc[g] += v[g];
-                    pb[g * pbs + a] = __float2bfloat16_rn(v[g]);
+                    pb[g * pbw + a] = __float2bfloat16_rn(v[g]);
                 }
             }
             {
@@ -680,7 +765,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_fft_kernel(Dims s, CacheDe
                 for (int mt = 0; mt < 8; ++mt) { accw[mt][0] *= al; accw[mt][1] *= ah; accw[mt][2] *= al; accw[mt][3] *= ah; }
             }
             consumer_sync();
-            const bf16* prow = pb + (size_t)(gq & (GH - 1)) * pbs;
+            const bf16* prow = pb + (size_t)(gq & (GH - 1)) * pbw;
             for (int si = 0; si < sg.n; ++si)
                 for (int r0 = 0; r0 < sg.cnt[si]; r0 += ts_w) {
                     const int nt = min(ts_w, sg.cnt[si] - r0);
@@ -986,7 +1071,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_fft_kernel(Dims s, CacheDe
     // ------------------------------ partial results ------------------------------
     for (int i = tid; i < GH * s.d; i += kConsumers) {
         const int g = i / s.d, e = i - g * s.d;
-        if (g < ng) ws.o[(((size_t)b * s.Hq + g_first + g) * p.n_split + split) * s.d + e] = o_s[i];
+        if (g < ng) ws.o[(((size_t)b * s.Hq + g_first + g) * p.n_part + part) * s.d + e] = o_s[i];
     }
     for (int n = tid; n < s.k; n += kConsumers) {
         const float* e = z_s + n * 2 * GH;
@@ -994,14 +1079,14 @@ __global__ void __launch_bounds__(kThreads, 1) decode_fft_kernel(Dims s, CacheDe
         for (int sl = 0; sl < GH; ++sl) {
             const int g = hperm<GH>(sl), ab = sl / N, ln = sl - ab * N;
             if (g < ng)
-                *reinterpret_cast<float2*>(ws.z + (((size_t)b * s.Hq + g_first + g) * p.n_split + split) * s.M + 2 * n) =
+                *reinterpret_cast<float2*>(ws.z + (((size_t)b * s.Hq + g_first + g) * p.n_part + part) * s.M + 2 * n) =
                     make_float2(e[(2 * ab) * N + ln], e[(2 * ab + 1) * N + ln]);
         }
     }
     if (tid < GH) {
         const int g = hperm<GH>(tid);                     // slot tid holds head g
         if (g < ng) {
-            float* ml = ws.ml + (((size_t)b * s.Hq + g_first + g) * p.n_split + split) * 2;
+            float* ml = ws.ml + (((size_t)b * s.Hq + g_first + g) * p.n_part + part) * 2;
             float mv = m_run[0];
 #pragma unroll
             for (int sl = 1; sl < GH; ++sl) if (tid == sl) mv = m_run[sl];
@@ -1009,35 +1094,181 @@ __global__ void __launch_bounds__(kThreads, 1) decode_fft_kernel(Dims s, CacheDe
             ml[1] = red_s[8 * GH + tid];
         }
     }
+    if (!p.fused) return;
+
+    // ------------------------------ merge (fused kernel) ------------------------------
+    // All parts of this (b, KV head, pass) have written their partial results.  Each part then
+    // merges a slice: its rows of z against its rows of C^V, and its share of the dims of o.  The
+    // last part to finish adds the slices in a fixed order, normalises and writes the output rows.
+    part_arrive(bar + 1, tid);
+    part_wait(bar + 1, p.n_part, tid, fail, c.status);
+    const int np = p.n_part;
+    const int rows = m1 - m0, rows_max = (s.M + np - 1) / np + 1;
+    const size_t qh0 = (size_t)b * s.Hq + g_first;
+    // scratch in the stage ring: every tile has been consumed
+    float* al_s = reinterpret_cast<float*>(stages);        // [GH][np] maxima, then exp2(m - max)
+    float* l_s = al_s + GH * np;                           // [GH][np]
+    float* linv_s = l_s + GH * np;                         // [GH]
+    float* zw_s = al_s + ((2 * GH * np + GH + 3) & ~3);    // [GH][rows_max], 16-byte aligned like ps_s
+    float* ps_s = zw_s + ((GH * rows_max + 3) & ~3);       // [row groups][GH][dcv]
+    const int nv = s.dcv >> 2, nrg = nv ? kConsumers / nv : 0;
+    int* inv_s = reinterpret_cast<int*>(ps_s + (size_t)nrg * GH * s.dcv);   // [d]
+    volatile int* last_s = fail + 1;
+
+    for (int i = tid; i < GH * np; i += kConsumers) {
+        const int g = i / np, sp = i - g * np;
+        float2 ml = make_float2(kNegBig, 0.f);
+        if (g < ng) ml = __ldcg(reinterpret_cast<const float2*>(ws.ml + ((qh0 + g) * np + sp) * 2));
+        al_s[i] = ml.x;
+        l_s[i] = ml.y;
+    }
+    consumer_sync();
+    if (tid < GH) {
+        float mx = kNegBig;
+        for (int sp = 0; sp < np; ++sp) mx = fmaxf(mx, al_s[tid * np + sp]);
+        float Lsum = 0.f;
+        for (int sp = 0; sp < np; ++sp) {
+            const float a = exp2f(al_s[tid * np + sp] - mx);
+            al_s[tid * np + sp] = a;
+            Lsum = fmaf(a, l_s[tid * np + sp], Lsum);
+        }
+        linv_s[tid] = Lsum > 0.f ? 1.0f / Lsum : 0.f;
+    }
+    consumer_sync();
+    // sum over the parts of al[sp] * src[sp * stride], eight independent loads in flight
+    auto merged = [&](const float* al, const float* src, size_t stride) -> float {
+        float v0 = 0.f, v1 = 0.f;
+        int sp = 0;
+        for (; sp + 8 <= np; sp += 8) {
+            float x[8];
+#pragma unroll
+            for (int i = 0; i < 8; ++i) x[i] = __ldcg(src + (size_t)(sp + i) * stride);
+#pragma unroll
+            for (int i = 0; i < 8; i += 2) { v0 = fmaf(al[sp + i], x[i], v0); v1 = fmaf(al[sp + i + 1], x[i + 1], v1); }
+        }
+        for (; sp < np; ++sp) v0 = fmaf(al[sp], __ldcg(src + (size_t)sp * stride), v0);
+        return v0 + v1;
+    };
+    for (int t = tid; t < GH * rows; t += kConsumers) {
+        const int g = t / rows, r = t - g * rows;
+        float v = 0.f;
+        if (g < ng && s.dcv > 0)
+            v = merged(al_s + g * np, ws.z + (qh0 + g) * np * s.M + m0 + r, (size_t)s.M) * recon_weight(s.norm, m0 + r, s.k, s.T);
+        zw_s[g * rows_max + r] = v;
+    }
+    {
+        const int e0 = (int)((long long)part * s.d / np), e1 = (int)((long long)(part + 1) * s.d / np);
+        for (int t = tid; t < GH * (e1 - e0); t += kConsumers) {
+            const int g = t / (e1 - e0), e = e0 + t - g * (e1 - e0);
+            if (g < ng) ws.om[(qh0 + g) * s.d + e] = merged(al_s + g * np, ws.o + (qh0 + g) * np * s.d + e, (size_t)s.d);
+        }
+    }
+    consumer_sync();
+    if (s.dcv > 0) {
+        if (tid < nrg * nv) {
+            const int v = tid % nv, rgi = tid / nv;
+            float4 acc4[GH];
+#pragma unroll
+            for (int g = 0; g < GH; ++g) acc4[g] = make_float4(0.f, 0.f, 0.f, 0.f);
+            const float4* cv = reinterpret_cast<const float4*>(coef_rows(c.coef_v, s, b, h, s.dcv) + (size_t)m0 * s.dcv) + v;
+#pragma unroll 4
+            for (int r = rgi; r < rows; r += nrg) {
+                const float4 x = __ldg(cv + (size_t)r * nv);
+#pragma unroll
+                for (int g = 0; g < GH; ++g) {
+                    const float w = zw_s[g * rows_max + r];
+                    acc4[g].x = fmaf(w, x.x, acc4[g].x);
+                    acc4[g].y = fmaf(w, x.y, acc4[g].y);
+                    acc4[g].z = fmaf(w, x.z, acc4[g].z);
+                    acc4[g].w = fmaf(w, x.w, acc4[g].w);
+                }
+            }
+#pragma unroll
+            for (int g = 0; g < GH; ++g) *reinterpret_cast<float4*>(ps_s + ((size_t)rgi * GH + g) * s.dcv + 4 * v) = acc4[g];
+        }
+        consumer_sync();
+        for (int t = tid; t < GH * s.dcv; t += kConsumers) {
+            const int g = t / s.dcv, e = t - g * s.dcv;
+            float v = 0.f;
+            for (int rgi = 0; rgi < nrg; ++rgi) v += ps_s[((size_t)rgi * GH + g) * s.dcv + e];
+            if (g < ng) ws.oc[((qh0 + g) * np + part) * s.dcv + e] = v;
+        }
+    }
+    // ticket: the last part to get here finishes the rows
+    __threadfence();
+    consumer_sync();
+    if (tid == 0) {
+        int old;
+        asm volatile("atom.acq_rel.gpu.global.add.s32 %0, [%1], 1;" : "=r"(old) : "l"(bar + 2) : "memory");
+        *last_s = old == np - 1;
+    }
+    consumer_sync();
+    if (!*last_s) return;
+    for (int e = tid; e < s.d; e += kConsumers) inv_s[e] = -1;
+    consumer_sync();
+    if (s.dcv > 0) {
+        const int32_t* idc_v = c.idx_comp_v + (size_t)h * s.dcv;
+        for (int e = tid; e < s.dcv; e += kConsumers) inv_s[idc_v[e]] = e;
+    }
+    consumer_sync();
+    for (int t = tid; t < GH * s.d; t += kConsumers) {
+        const int g = t / s.d, e = t - g * s.d;
+        if (g >= ng) continue;
+        float v = __ldcg(ws.om + (qh0 + g) * s.d + e);
+        const int slot = inv_s[e];
+        if (slot >= 0) {
+            const float* oc = ws.oc + (qh0 + g) * np * s.dcv + slot;
+            float w0 = 0.f, w1 = 0.f;
+            int x = 0;
+            for (; x + 8 <= np; x += 8) {
+                float cc[8];
+#pragma unroll
+                for (int i = 0; i < 8; ++i) cc[i] = __ldcg(oc + (size_t)(x + i) * s.dcv);
+#pragma unroll
+                for (int i = 0; i < 8; i += 2) { w0 += cc[i]; w1 += cc[i + 1]; }
+            }
+            for (; x < np; ++x) w0 += __ldcg(oc + (size_t)x * s.dcv);
+            v += w0 + w1;
+        }
+        out[(qh0 + g) * s.d + e] = __float2bfloat16_rn(v * linv_s[g]);
+    }
+    if (tid == 0) { bar[0] = 0; bar[1] = 0; bar[2] = 0; }   // the counters are zero again for the next call
 }
 
 template <int GH, int LS>
-cudaError_t launch_fft_t(const Dims& s, const CacheDev& c, const DecodePlan& p, const void* q, char* ws, cudaStream_t st) {
+cudaError_t launch_fft_t(const Dims& s, const CacheDev& c, const DecodePlan& p, const void* q, void* out, char* ws,
+                         cudaStream_t st) {
     const FftSmem L = fft_smem_layout(LS, s.k, GH, p.nb, s.d);
     cudaError_t err = ensure_dynamic_smem(decode_fft_kernel<GH, LS>, (size_t)L.total);
     if (err != cudaSuccess) return err;
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(p.n_split, s.Hkv * p.n_pass, s.B);
+    cfg.gridDim = dim3(p.n_part, s.Hkv * p.n_pass, s.B);
     cfg.blockDim = dim3(kThreads);
     cfg.dynamicSmemBytes = (size_t)L.total;
     cfg.stream = st;
     cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;   // may start while the prologue kernel runs
-    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    if (p.fused) {
+        attr[0].id = cudaLaunchAttributeCooperative;                      // its CTAs wait for one another
+        attr[0].val.cooperative = 1;
+    } else {
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;  // may start while the prologue kernel runs
+        attr[0].val.programmaticStreamSerializationAllowed = 1;
+    }
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, decode_fft_kernel<GH, LS>, s, c, p, static_cast<const bf16*>(q), ws);
+    return cudaLaunchKernelEx(&cfg, decode_fft_kernel<GH, LS>, s, c, p, static_cast<const bf16*>(q), static_cast<bf16*>(out), ws);
 }
 
 template <int GH>
-cudaError_t launch_fft_ls(const Dims& s, const CacheDev& c, const DecodePlan& p, const void* q, char* ws, cudaStream_t st) {
+cudaError_t launch_fft_ls(const Dims& s, const CacheDev& c, const DecodePlan& p, const void* q, void* out, char* ws,
+                          cudaStream_t st) {
     switch (p.fft_log2) {
-        case 5: return launch_fft_t<GH, 5>(s, c, p, q, ws, st);
-        case 6: return launch_fft_t<GH, 6>(s, c, p, q, ws, st);
-        case 7: return launch_fft_t<GH, 7>(s, c, p, q, ws, st);
-        case 8: return launch_fft_t<GH, 8>(s, c, p, q, ws, st);
-        case 9: return launch_fft_t<GH, 9>(s, c, p, q, ws, st);
-        case 10: return launch_fft_t<GH, 10>(s, c, p, q, ws, st);
+        case 5: return launch_fft_t<GH, 5>(s, c, p, q, out, ws, st);
+        case 6: return launch_fft_t<GH, 6>(s, c, p, q, out, ws, st);
+        case 7: return launch_fft_t<GH, 7>(s, c, p, q, out, ws, st);
+        case 8: return launch_fft_t<GH, 8>(s, c, p, q, out, ws, st);
+        case 9: return launch_fft_t<GH, 9>(s, c, p, q, out, ws, st);
+        case 10: return launch_fft_t<GH, 10>(s, c, p, q, out, ws, st);
         default: return cudaErrorInvalidValue;
     }
 }
@@ -1048,11 +1279,11 @@ size_t decode_fft_smem_bytes(const Dims& s, int log2S, int gh, int nb) {
     return (size_t)fft_smem_layout(log2S, s.k, gh, nb, s.d).total;
 }
 
-cudaError_t launch_decode_fft(const Dims& s, const CacheDev& c, int dtype, const DecodePlan& p, const void* q, char* ws,
-                              cudaStream_t st) {
+cudaError_t launch_decode_fft(const Dims& s, const CacheDev& c, int dtype, const DecodePlan& p, const void* q, void* out,
+                              char* ws, cudaStream_t st) {
     if (dtype != FA_BF16) return cudaErrorInvalidValue;
-    if (p.gh == 4) return launch_fft_ls<4>(s, c, p, q, ws, st);
-    return launch_fft_ls<2>(s, c, p, q, ws, st);
+    if (p.gh == 4) return launch_fft_ls<4>(s, c, p, q, out, ws, st);
+    return launch_fft_ls<2>(s, c, p, q, out, ws, st);
 }
 
 }  // namespace fa

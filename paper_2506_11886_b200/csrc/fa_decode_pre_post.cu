@@ -85,7 +85,7 @@ __global__ void __launch_bounds__(256) decode_epilogue_kernel(Dims s, CacheDev c
     const int m0 = slice * rows_max;
     const int rows = max(0, min(rows_max, s.M - m0));
     const int stride = s.dcv + 4;
-    const int ns = p.n_split;
+    const int ns = p.n_part;
     float* alpha_s = sm_epi;                               // [G][n_split]: first the maxima, then exp2(m - max)
     float* l_s = alpha_s + s.G * ns;                       // [G][n_split]
     float* linv_s = l_s + s.G * ns;                        // [G]
@@ -246,7 +246,7 @@ template <typename KV>
 static cudaError_t launch_epilogue_t(const Dims& s, const CacheDev& c, const DecodePlan& p, void* out, char* ws,
                                      cudaStream_t st) {
     const int rows = (s.M + p.n_slice - 1) / p.n_slice;
-    const size_t smem = sizeof(float) * (2 * (size_t)s.G * p.n_split + s.G + (size_t)s.G * rows + s.d + 4 + (size_t)rows * (s.dcv + 4));
+    const size_t smem = sizeof(float) * (2 * (size_t)s.G * p.n_part + s.G + (size_t)s.G * rows + s.d + 4 + (size_t)rows * (s.dcv + 4));
     cudaError_t err = ensure_dynamic_smem(decode_epilogue_kernel<KV>, smem);
     if (err != cudaSuccess) return err;
     return launch_pdl(decode_epilogue_kernel<KV>, dim3(p.n_slice, s.Hkv, s.B), dim3(256), smem, st, true, s, c, p,

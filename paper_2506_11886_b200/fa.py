@@ -20,7 +20,7 @@ FA_OK, FA_ERR_INVALID_ARG, FA_ERR_UNSUPPORTED, FA_ERR_CAPACITY = 0, 1, 2, 3
 FA_ERR_WORKSPACE, FA_ERR_CUDA, FA_ERR_TIMEOUT, FA_ERR_INDEX = 4, 5, 6, 7
 FA_F32, FA_BF16 = 0, 1
 FA_NORM_ORTHO, FA_NORM_PAPER = 0, 1
-FA_DECODE_AUTO, FA_DECODE_DIRECT, FA_DECODE_FFT = 0, 1, 2
+FA_DECODE_AUTO, FA_DECODE_DIRECT, FA_DECODE_FFT, FA_DECODE_FFT_SPLIT = 0, 1, 2, 3
 
 
 class fa_layout(C.Structure):
@@ -196,7 +196,7 @@ class Cache:
 
 
 def new_workspace(layout: Layout, device="cuda") -> torch.Tensor:
-    return torch.empty(max(256, fa_workspace_bytes(layout)), dtype=torch.uint8, device=device)
+    return torch.zeros(max(256, fa_workspace_bytes(layout)), dtype=torch.uint8, device=device)
 
 
 def fa_cache_reset(layout: Layout, cache: Cache, stream=None) -> None:

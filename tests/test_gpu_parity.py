@@ -17,14 +17,14 @@ def make_pair(*a, **kw):
     try:
         return _make_pair(*a, **kw)
     except fa.FaError as e:
-        if e.status == fa.FA_ERR_UNSUPPORTED and kw.get("algo") == fa.FA_DECODE_FFT:
+        if e.status == fa.FA_ERR_UNSUPPORTED and kw.get("algo") in (fa.FA_DECODE_FFT, fa.FA_DECODE_FFT_SPLIT):
             pytest.skip("layout outside the FFT kernel's range")
         raise
 
 CFG0 = synth.CONFIGS[0]
 SMALL_BF16 = synth.Shape("small_bf16_gqa", B=2, layers=1, Hq=8, Hkv=2, d=128, L=1500, dtype="bf16", n_full_k=32,
                          n_full_v=48, M=128, T=2048, L_init=4, L_local=64, decode_steps=40)
-ALGOS = [fa.FA_DECODE_DIRECT, fa.FA_DECODE_FFT]
+ALGOS = [fa.FA_DECODE_DIRECT, fa.FA_DECODE_FFT, fa.FA_DECODE_FFT_SPLIT]
 
 
 @pytest.mark.parametrize("P", [1, 32])
