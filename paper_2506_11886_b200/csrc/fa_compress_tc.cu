@@ -17,9 +17,7 @@
 //   * warp 1 (one lane) issues four tcgen05.mma (K = 16 each) and commits the stage back.
 // At the end warps 2-9 read the accumulators from tensor memory and scatter the compressed
 // columns.  Every wait is bounded; tensor memory is freed on every path.
-#include <cuda.h>
-
-#include "fa_common.cuh"
+#include "fa_tmap.cuh"
 
 namespace fa {
 namespace {
@@ -303,21 +301,6 @@ __global__ void __launch_bounds__(kThreadsTc, 1) compress_tc_kernel(const __grid
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
     }
-}
-
-typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
-                                  const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
-                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-EncodeTiledFn encode_tiled_fn() {
-    static EncodeTiledFn fn = nullptr;
-    if (!fn) {
-        void* p = nullptr;
-        cudaDriverEntryPointQueryResult q;
-        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess && q == cudaDriverEntryPointSuccess)
-            fn = reinterpret_cast<EncodeTiledFn>(p);
-    }
-    return fn;
 }
 
 // 4-D view (dim, head, token, batch) of a prefilled K or V with element strides (1, sh, st, sb); box = 64 dims x 64 tokens.

@@ -24,8 +24,8 @@
 // "Slot" below is the position of a head inside a point / an mma column: slot s holds head
 // hperm(s) = {0, 2, 1, 3}[s] (GH = 4) so that the packed real parts are slots 0, 1 and the
 // packed imaginary parts slots 2, 3.
-#include "fa_common.cuh"
 #include "fa_decode_ws.cuh"
+#include "fa_tmap.cuh"
 
 namespace fa {
 namespace {
@@ -34,7 +34,8 @@ constexpr int kConsumers = 256;
 constexpr int kThreads = kConsumers + 32;
 constexpr int kStageBytes = 16384;
 constexpr int kStages = 6;
-constexpr int kWinRowsPerTile = 48;
+constexpr int kWinRowsPerTile = 64;       // rows of one window tile: two [64 rows x 64 dims] TMA boxes, 128-byte swizzle
+constexpr int kWinHalfBytes = kWinRowsPerTile * 128;
 constexpr uint32_t kSpinLimit = 1u << 24;
 using bf16 = __nv_bfloat16;
 typedef unsigned long long u64;
@@ -71,6 +72,13 @@ __device__ __forceinline__ void bulk_g2s(void* dst, const void* src, uint32_t by
     asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
                      smem_addr(dst)),
                  "l"(__cvta_generic_to_global(src)), "r"(bytes), "r"(smem_addr(bar))
+                 : "memory");
+}
+// One box of a window tensor map: dims x0.., rows y0.., (batch, KV head) z.
+__device__ __forceinline__ void tma_load_3d(void* dst, const CUtensorMap* tm, int x0, int y0, int z, uint64_t* bar) {
+    asm volatile("cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];" ::"r"(
+                     smem_addr(dst)),
+                 "l"(reinterpret_cast<uint64_t>(tm)), "r"(x0), "r"(y0), "r"(z), "r"(smem_addr(bar))
                  : "memory");
 }
 __device__ __forceinline__ void consumer_sync() { asm volatile("bar.sync 1, 256;" ::: "memory"); }
@@ -332,7 +340,7 @@ __host__ __device__ inline FftSmem fft_smem_layout(int log2S, int k, int GH, int
     L.pbs = S + 8;                                        // bf16 per (class, slot) row of rounded probabilities
     int off = 256;                                        // mbarriers + flags
     L.zero_off = off; off += 16;
-    off = (off + 127) / 128 * 128;
+    off = 1024;                                           // stages are 1024-byte aligned (swizzled window tiles)
     L.stages_off = off; off += kStages * kStageBytes;
     L.fbuf_off = off; off += 4 * NB * L.fb_floats;
     off = (off + 15) / 16 * 16;
@@ -346,7 +354,7 @@ __host__ __device__ inline FftSmem fft_smem_layout(int log2S, int k, int GH, int
     L.z_off = off; off += (8 * k * GH + 15) / 16 * 16;
     L.o_off = off; off += 4 * GH * d;
     L.red_off = off; off += 4 * (8 * GH + GH + 8);
-    L.total = (off + 127) / 128 * 128;
+    L.total = (off + 127) / 128 * 128 + 1024;             // slack to align the base to 1024 bytes at run time
     return L;
 }
 
@@ -354,11 +362,16 @@ template <int GH> __host__ __device__ constexpr int hperm(int s) { return GH == 
 
 // GH query heads per CTA (2 or 4), transform length S = 2^LS.
 template <int GH, int LS>
-__global__ void __launch_bounds__(kThreads, 1) decode_fft_kernel(Dims s, CacheDev c, DecodePlan p, const bf16* __restrict__ q,
-                                                                  bf16* __restrict__ out, char* wsp) {
+__global__ void __launch_bounds__(kThreads, 1) decode_fft_kernel(const __grid_constant__ CUtensorMap tm_ki,
+                                                                  const __grid_constant__ CUtensorMap tm_vi,
+                                                                  const __grid_constant__ CUtensorMap tm_kl,
+                                                                  const __grid_constant__ CUtensorMap tm_vl, Dims s, CacheDev c,
+                                                                  DecodePlan p, const bf16* __restrict__ q, bf16* __restrict__ out,
+                                                                  char* wsp) {
     constexpr int N = GH / 2;
     constexpr int S = 1 << LS;
-    extern __shared__ __align__(128) unsigned char smem_raw[];
+    extern __shared__ __align__(128) unsigned char smem_unaligned[];
+    unsigned char* smem_raw = smem_unaligned + ((1024u - (smem_addr(smem_unaligned) & 1023u)) & 1023u);
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");      // the epilogue may be scheduled behind us at once
     Ws ws = ws_view(wsp, p);
     const int NB = p.nb;
@@ -400,7 +413,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_fft_kernel(Dims s, CacheDe
     auto n_of_class = [&](int cls) { return cls < n_mid ? (n_mid - cls + s.P - 1) >> log2P : 0; };
 
     const int rowb_k = s.nfk * 2, rowb_v = s.nfv * 2, rowb_w = s.d * 2;
-    const int rbw_pad = rowb_w + 16;                                       // padded window row in shared memory
+    const int nhalf = (s.d + 63) >> 6;                                     // 64-dim boxes per window row
     const int ts_k = rowb_k ? (kStageBytes / rowb_k) & ~15 : 0, ts_v = rowb_v ? (kStageBytes / rowb_v) & ~15 : 0;
     const int ts_w = kWinRowsPerTile;
     // window tokens per softmax chunk: the score and probability buffers of all NB classes when
@@ -421,34 +434,27 @@ __global__ void __launch_bounds__(kThreads, 1) decode_fft_kernel(Dims s, CacheDe
 
     // ============================ producer warp =================================
     if (tid >= kConsumers) {
-        // window rows first (same order as the consumers): one bulk copy per row into padded
-        // shared-memory rows, issued by all lanes of the warp
+        // window rows first (same order as the consumers): tiles of 64 rows, one TMA box per 64 dims
         const int plane = tid - kConsumers;
         int it = 0;
-        for (int t0 = w0; t0 < w1; t0 += wchunk) {
-            const WinSegs sg = win_segments(t0, min(w1, t0 + wchunk), n_init, n_local, head, s.l_local);
-            for (int side = 0; side < 2; ++side)
-                for (int i = 0; i < sg.n; ++i)
-                    for (int r0 = 0; r0 < sg.cnt[i]; r0 += ts_w) {
-                        const int nt = min(ts_w, sg.cnt[i] - r0);
-                        void* base = sg.buf[i] == 0 ? (side == 0 ? c.k_init : c.v_init) : (side == 0 ? c.k_local : c.v_local);
-                        const int rows = sg.buf[i] == 0 ? s.l_init : s.l_local;
-                        const bf16* src = win_row<bf16>(base, s, b, h, rows, sg.row[i] + r0);
-                        const int st = it % kStages;
-                        int ok = 1;
-                        if (plane == 0) {
+        if (plane == 0) {
+            for (int t0 = w0; t0 < w1; t0 += wchunk) {
+                const WinSegs sg = win_segments(t0, min(w1, t0 + wchunk), n_init, n_local, head, s.l_local);
+                for (int side = 0; side < 2; ++side)
+                    for (int i = 0; i < sg.n; ++i)
+                        for (int r0 = 0; r0 < sg.cnt[i]; r0 += ts_w) {
+                            const CUtensorMap* tm = sg.buf[i] == 0 ? (side == 0 ? &tm_ki : &tm_vi) : (side == 0 ? &tm_kl : &tm_vl);
+                            const int st = it % kStages;
                             if (it >= kStages) mbar_wait(empty + st, ((it / kStages) - 1) & 1, fail, c.status);
-                            ok = !*fail;
-                            if (ok) mbar_expect_tx(full + st, (uint32_t)(nt * rowb_w));
+                            if (!*fail) {
+                                mbar_expect_tx(full + st, (uint32_t)(nhalf * kWinHalfBytes));
+                                unsigned char* dst = stages + (size_t)st * kStageBytes;
+                                for (int hf = 0; hf < nhalf; ++hf)
+                                    tma_load_3d(dst + hf * kWinHalfBytes, tm, hf * 64, sg.row[i] + r0, b * s.Hkv + h, full + st);
+                            }
+                            ++it;
                         }
-                        ok = __shfl_sync(0xffffffffu, ok, 0);
-                        if (ok) {
-                            unsigned char* dst = stages + (size_t)st * kStageBytes;
-                            for (int r = plane; r < nt; r += 32)
-                                bulk_g2s(dst + (size_t)r * rbw_pad, src + (size_t)r * s.d, (uint32_t)rowb_w, full + st);
-                        }
-                        ++it;
-                    }
+            }
         }
         if (plane == 0) {
             auto acquire = [&](uint32_t bytes) -> unsigned char* {
@@ -681,7 +687,9 @@ __global__ void __launch_bounds__(kThreads, 1) decode_fft_kernel(Dims s, CacheDe
         for (int rd = 0; rd < 4; ++rd)
 #pragma unroll
             for (int ks = 0; ks < 2; ++ks) {
-                const int piece = 4 * rd + tq, e0 = 8 * piece + 4 * ks;
+                // round rd covers the 16-byte pieces 2 tq + (rd & 1) of half rd >> 1: with the 128-byte
+                // swizzle the eight lanes of a quarter warp (two rows) then hit eight different bank groups
+                const int piece = ((rd >> 1) << 3) + 2 * tq + (rd & 1), e0 = 8 * piece + 4 * ks;
                 const bool on = col_on && piece < npw;
                 qw[rd][ks][0] = on ? pack_bf16(qrow[e0], qrow[e0 + 1]) : 0u;
                 qw[rd][ks][1] = on ? pack_bf16(qrow[e0 + 2], qrow[e0 + 3]) : 0u;
@@ -701,18 +709,18 @@ __global__ void __launch_bounds__(kThreads, 1) decode_fft_kernel(Dims s, CacheDe
                 for (int r0 = 0; r0 < sg.cnt[si]; r0 += ts_w) {
                     const int nt = min(ts_w, sg.cnt[si] - r0);
                     const unsigned char* tile = wait_tile();
-                    for (int grp = warp; grp * 16 < nt; grp += 8) {
-                        const unsigned char* r_lo = tile + (size_t)(grp * 16 + gq) * rbw_pad;
-                        const unsigned char* r_hi = r_lo + 8 * rbw_pad;
+                    for (int grp = (warp + 8 - (it * (kWinRowsPerTile / 16)) % 8) & 7; grp * 16 < nt; grp += 8) {   // tiles rotate over the warps
+                        const unsigned char* r_lo = tile + (size_t)(grp * 16 + gq) * 128;      // row & 7 == gq for both rows
                         float d4[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
                         for (int rd = 0; rd < 4; ++rd) {
-                            const int piece = 4 * rd + tq;
-                            if (4 * rd < npw) {
+                            const int cj = 2 * tq + (rd & 1), piece = ((rd >> 1) << 3) + cj;
+                            if (((rd >> 1) << 3) < npw) {
                                 uint4 lo = make_uint4(0, 0, 0, 0), hi = make_uint4(0, 0, 0, 0);
                                 if (piece < npw) {
-                                    lo = *reinterpret_cast<const uint4*>(r_lo + 16 * piece);
-                                    hi = *reinterpret_cast<const uint4*>(r_hi + 16 * piece);
+                                    const unsigned char* src = r_lo + (rd >> 1) * kWinHalfBytes + ((cj ^ gq) << 4);
+                                    lo = *reinterpret_cast<const uint4*>(src);
+                                    hi = *reinterpret_cast<const uint4*>(src + 8 * 128);
                                 }
                                 mma_bf16(d4, lo.x, hi.x, lo.y, hi.y, qw[rd][0][0], qw[rd][0][1]);
                                 mma_bf16(d4, lo.z, hi.z, lo.w, hi.w, qw[rd][1][0], qw[rd][1][1]);
@@ -770,7 +778,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_fft_kernel(Dims s, CacheDe
                 for (int r0 = 0; r0 < sg.cnt[si]; r0 += ts_w) {
                     const int nt = min(ts_w, sg.cnt[si] - r0);
                     const unsigned char* tile = wait_tile();
-                    for (int grp = warp; grp * 16 < nt; grp += 8) {
+                    for (int grp = (warp + 8 - (it * (kWinRowsPerTile / 16)) % 8) & 7; grp * 16 < nt; grp += 8) {
                         const int a = sg.tok[si] + r0 + grp * 16;
                         // the tile's rows may start at any token of the chunk: gather the four p values one by one
                         uint32_t b0 = 0, b1 = 0;
@@ -780,13 +788,24 @@ __global__ void __launch_bounds__(kThreads, 1) decode_fft_kernel(Dims s, CacheDe
                             b0 = pack_bf16(2 * tq < rem ? prow[a + 2 * tq] : zero, 2 * tq + 1 < rem ? prow[a + 2 * tq + 1] : zero);
                             b1 = pack_bf16(2 * tq + 8 < rem ? prow[a + 2 * tq + 8] : zero, 2 * tq + 9 < rem ? prow[a + 2 * tq + 9] : zero);
                         }
+                        if (nt - grp * 16 < 16) {
+                            // rows past the end of the segment hold whatever follows it in the cache: zero them,
+                            // p = 0 does not stop a NaN
+                            const int rem = nt - grp * 16, per_row = nhalf * 8;
+                            for (int i = lane; i < (16 - rem) * per_row; i += 32) {
+                                const int rr = grp * 16 + rem + i / per_row, cc = i % per_row;
+                                *reinterpret_cast<uint4*>(const_cast<unsigned char*>(tile) + (cc >> 3) * kWinHalfBytes + rr * 128 + ((cc & 7) << 4)) =
+                                    make_uint4(0, 0, 0, 0);
+                            }
+                            __syncwarp();
+                        }
                         const int mi = lane >> 3, tok = ((mi >> 1) << 3) + (lane & 7);
-                        const unsigned char* vrow = tile + (size_t)(grp * 16 + tok) * rbw_pad;
+                        const unsigned char* vrow = tile + (size_t)(grp * 16 + tok) * 128;
 #pragma unroll
                         for (int mt = 0; mt < 8; ++mt) {
                             if (mt < nmtw) {
                                 const int chunk = 2 * mt + (mi & 1);
-                                const unsigned char* src = chunk < npw ? vrow + 16 * chunk : zero16;
+                                const unsigned char* src = chunk < npw ? vrow + (chunk >> 3) * kWinHalfBytes + (((chunk & 7) ^ (tok & 7)) << 4) : zero16;
                                 uint32_t af[4];
                                 ldmatrix_x4_trans(af, smem_addr(src));
                                 mma_bf16(accw[mt], af[0], af[1], af[2], af[3], b0, b1);
@@ -1241,6 +1260,12 @@ cudaError_t launch_fft_t(const Dims& s, const CacheDev& c, const DecodePlan& p, 
     const FftSmem L = fft_smem_layout(LS, s.k, GH, p.nb, s.d);
     cudaError_t err = ensure_dynamic_smem(decode_fft_kernel<GH, LS>, (size_t)L.total);
     if (err != cudaSuccess) return err;
+    // window buffers as tensor maps (cached per buffer)
+    CUtensorMap tki, tvi, tkl, tvl;
+    const int n_bh = s.B * s.Hkv;
+    const bool ok_i = window_map(&tki, c.k_init, s.l_init, s.d, n_bh) & window_map(&tvi, c.v_init, s.l_init, s.d, n_bh);
+    const bool ok_l = window_map(&tkl, c.k_local, s.l_local, s.d, n_bh) & window_map(&tvl, c.v_local, s.l_local, s.d, n_bh);
+    if ((s.l_init > 0 && !ok_i) || (s.l_local > 0 && !ok_l)) return cudaErrorInvalidValue;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(p.n_part, s.Hkv * p.n_pass, s.B);
     cfg.blockDim = dim3(kThreads);
@@ -1256,7 +1281,8 @@ cudaError_t launch_fft_t(const Dims& s, const CacheDev& c, const DecodePlan& p, 
     }
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, decode_fft_kernel<GH, LS>, s, c, p, static_cast<const bf16*>(q), static_cast<bf16*>(out), ws);
+    return cudaLaunchKernelEx(&cfg, decode_fft_kernel<GH, LS>, tki, tvi, tkl, tvl, s, c, p, static_cast<const bf16*>(q),
+                              static_cast<bf16*>(out), ws);
 }
 
 template <int GH>

@@ -1,0 +1,44 @@
+#include <cstring>
+#include <mutex>
+
+#include "fa_tmap.cuh"
+
+namespace fa {
+
+EncodeTiledFn encode_tiled_fn() {
+    static EncodeTiledFn fn = nullptr;
+    static std::once_flag once;
+    std::call_once(once, [] {
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess && q == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(p);
+    });
+    return fn;
+}
+
+bool window_map(CUtensorMap* tm, const void* base, int rows, int d, int n_bh) {
+    std::memset(tm, 0, sizeof(*tm));
+    if (rows <= 0 || !base) return false;
+    struct Entry { const void* base; int rows, d, n_bh; CUtensorMap tm; };
+    static Entry cache[32];
+    static int used = 0, next = 0;
+    static std::mutex mu;
+    std::lock_guard<std::mutex> lock(mu);
+    for (int i = 0; i < used; ++i)
+        if (cache[i].base == base && cache[i].rows == rows && cache[i].d == d && cache[i].n_bh == n_bh) { *tm = cache[i].tm; return true; }
+    EncodeTiledFn fn = encode_tiled_fn();
+    if (!fn) return false;
+    cuuint64_t dims[3] = {(cuuint64_t)d, (cuuint64_t)rows, (cuuint64_t)n_bh};
+    cuuint64_t strides[2] = {(cuuint64_t)d * 2, (cuuint64_t)rows * d * 2};
+    cuuint32_t box[3] = {64, 64, 1};
+    cuuint32_t estr[3] = {1, 1, 1};
+    if (fn(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+           CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+        return false;
+    Entry& e = cache[used < 32 ? used++ : (next = (next + 1) % 32)];
+    e = Entry{base, rows, d, n_bh, *tm};
+    return true;
+}
+
+}  // namespace fa
