@@ -70,6 +70,7 @@ static bool fft_ok(const fa_layout& l, int gh, int* log2S) {
     if (ls < 5 || ls > 10) return false;
     if (l.n_coef / 2 > S) return false;                                        // every frequency needs its own bin
     if (l.n_full_k > 64 || l.n_full_v > 64 || l.head_dim > 128) return false;
+    if ((long long)l.l_init + l.l_local > (1 << 22)) return false;                // 32-bit split arithmetic in the kernel
     if (decode_fft_smem_bytes(make_dims(l), ls, gh, 1) > 227 * 1024) return false;
     *log2S = ls;
     return true;

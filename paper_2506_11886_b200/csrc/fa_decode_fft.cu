@@ -30,7 +30,8 @@
 namespace fa {
 namespace {
 
-constexpr int kConsumers = 256;
+constexpr int kConsumers = 512;
+constexpr int kWarps = kConsumers / 32;
 constexpr int kThreads = kConsumers + 32;
 constexpr int kStageBytes = 16384;
 constexpr int kStages = 6;
@@ -81,7 +82,7 @@ __device__ __forceinline__ void tma_load_3d(void* dst, const CUtensorMap* tm, in
                  "l"(reinterpret_cast<uint64_t>(tm)), "r"(x0), "r"(y0), "r"(z), "r"(smem_addr(bar))
                  : "memory");
 }
-__device__ __forceinline__ void consumer_sync() { asm volatile("bar.sync 1, 256;" ::: "memory"); }
+__device__ __forceinline__ void consumer_sync() { asm volatile("bar.sync 1, %0;" ::"n"(kConsumers) : "memory"); }
 
 // Barrier among the CTAs of one (b, KV head, pass) on a global counter (fused kernel only: a
 // cooperative launch makes all of them resident).  Arrive: every consumer thread has fenced its
@@ -161,6 +162,10 @@ template <int N> __device__ __forceinline__ PC<N> cconj_add(PC<N> a, PC<N> b) { 
 template <int N> __device__ __forceinline__ PC<N> cmulw(PC<N> a, PR<N> wr, PR<N> wi) {
     return PC<N>{(a.re * wr) - (a.im * wi), pfma(a.re, wi, a.im * wr)};
 }
+// a + (the same value of the neighbouring lane)
+__device__ __forceinline__ PR<2> pair_sum(PR<2> a) { PR<2> o; o.v = __shfl_xor_sync(0xffffffffu, a.v, 1); return a + o; }
+__device__ __forceinline__ PR<1> pair_sum(PR<1> a) { return PR<1>{a.v + __shfl_xor_sync(0xffffffffu, a.v, 1)}; }
+template <int N> __device__ __forceinline__ PC<N> pair_sum(PC<N> a) { return PC<N>{pair_sum(a.re), pair_sum(a.im)}; }
 __device__ __forceinline__ float2 cmulf(float2 a, float2 b) {
     return make_float2(fmaf(a.x, b.x, -a.y * b.y), fmaf(a.x, b.y, a.y * b.x));
 }
@@ -353,7 +358,7 @@ __host__ __device__ inline FftSmem fft_smem_layout(int log2S, int k, int GH, int
     L.ut_off = off; off += (8 * k * GH + 15) / 16 * 16;
     L.z_off = off; off += (8 * k * GH + 15) / 16 * 16;
     L.o_off = off; off += 4 * GH * d;
-    L.red_off = off; off += 4 * (8 * GH + GH + 8);
+    L.red_off = off; off += 4 * (kWarps * GH + GH + 8);
     L.total = (off + 127) / 128 * 128 + 1024;             // slack to align the base to 1024 bytes at run time
     return L;
 }
@@ -389,7 +394,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_fft_kernel(const __grid_co
     float* ut = reinterpret_cast<float*>(smem_raw + L.ut_off);            // [k] (A.re, A.im, B.re, B.im) x N: (1/2) u~
     float* z_s = reinterpret_cast<float*>(smem_raw + L.z_off);            // [k] same packing
     float* o_s = reinterpret_cast<float*>(smem_raw + L.o_off);            // [GH heads][d]
-    float* red_s = reinterpret_cast<float*>(smem_raw + L.red_off);        // [8][GH] + l_s[GH]
+    float* red_s = reinterpret_cast<float*>(smem_raw + L.red_off);        // [kWarps][GH] + l_s[GH]
     const int fb_floats = L.fb_floats, pbs = L.pbs;
 
     const int part = blockIdx.x;                          // partial-result index: class CTAs, then window CTAs
@@ -403,13 +408,13 @@ __global__ void __launch_bounds__(kThreads, 1) decode_fft_kernel(const __grid_co
 
     const int n_init = c.state[kStateStride * b + 0], n_local = c.state[kStateStride * b + 1];
     const int n_mid = min(c.state[kStateStride * b + 2], s.max_mid), head = c.state[kStateStride * b + 3];
-    const int c0 = is_win ? 0 : (int)((long long)part * s.P / p.n_split);
-    const int c1 = is_win ? 0 : (int)((long long)(part + 1) * s.P / p.n_split);
+    const int c0 = is_win ? 0 : part * s.P / p.n_split;
+    const int c1 = is_win ? 0 : (part + 1) * s.P / p.n_split;
     const int n_win = n_init + n_local;
     // window tokens: spread over the class CTAs, or over CTAs of their own
     const int wi = p.n_wsplit ? part - p.n_split : part, wn = p.n_wsplit ? p.n_wsplit : p.n_split;
     const bool has_win = p.n_wsplit ? is_win : true;
-    const int w0 = has_win ? (int)((long long)wi * n_win / wn) : 0, w1 = has_win ? (int)((long long)(wi + 1) * n_win / wn) : 0;
+    const int w0 = has_win ? wi * n_win / wn : 0, w1 = has_win ? (wi + 1) * n_win / wn : 0;
     auto n_of_class = [&](int cls) { return cls < n_mid ? (n_mid - cls + s.P - 1) >> log2P : 0; };
 
     const int rowb_k = s.nfk * 2, rowb_v = s.nfv * 2, rowb_w = s.d * 2;
@@ -422,11 +427,12 @@ __global__ void __launch_bounds__(kThreads, 1) decode_fft_kernel(const __grid_co
     const int pbw = NB * L.pbs;                            // row stride of the window probabilities
 
     if (tid == 0) {
-        for (int i = 0; i < kStages; ++i) { mbar_init(full + i, 1); mbar_init(empty + i, 8); }
+        for (int i = 0; i < kStages; ++i) { mbar_init(full + i, 1); mbar_init(empty + i, kWarps); }
         *fail = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     // stale shared memory must hold finite numbers: rows past the end of a tile are multiplied by p = 0
+    #pragma unroll 1
     for (int i = tid; i < (kStages * kStageBytes) / 16; i += kThreads) reinterpret_cast<uint4*>(stages)[i] = make_uint4(0, 0, 0, 0);
     if (tid < 4) reinterpret_cast<uint32_t*>(zero16)[tid] = 0;
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -438,10 +444,13 @@ __global__ void __launch_bounds__(kThreads, 1) decode_fft_kernel(const __grid_co
         const int plane = tid - kConsumers;
         int it = 0;
         if (plane == 0) {
+            #pragma unroll 1
             for (int t0 = w0; t0 < w1; t0 += wchunk) {
                 const WinSegs sg = win_segments(t0, min(w1, t0 + wchunk), n_init, n_local, head, s.l_local);
                 for (int side = 0; side < 2; ++side)
+                    #pragma unroll 1
                     for (int i = 0; i < sg.n; ++i)
+                        #pragma unroll 1
                         for (int r0 = 0; r0 < sg.cnt[i]; r0 += ts_w) {
                             const CUtensorMap* tm = sg.buf[i] == 0 ? (side == 0 ? &tm_ki : &tm_vi) : (side == 0 ? &tm_kl : &tm_vl);
                             const int st = it % kStages;
@@ -449,6 +458,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_fft_kernel(const __grid_co
                             if (!*fail) {
                                 mbar_expect_tx(full + st, (uint32_t)(nhalf * kWinHalfBytes));
                                 unsigned char* dst = stages + (size_t)st * kStageBytes;
+                                #pragma unroll 1
                                 for (int hf = 0; hf < nhalf; ++hf)
                                     tma_load_3d(dst + hf * kWinHalfBytes, tm, hf * 64, sg.row[i] + r0, b * s.Hkv + h, full + st);
                             }
@@ -465,13 +475,16 @@ __global__ void __launch_bounds__(kThreads, 1) decode_fft_kernel(const __grid_co
                 return stages + (size_t)st * kStageBytes;
             };
             // per batch of NB classes all K tiles, then all V tiles
+            #pragma unroll 1
             for (int cb = c0; cb < c1; cb += NB) {
                 const int nb = min(NB, c1 - cb);
                 for (int side = 0; side < 2; ++side) {
                     const int ts = side == 0 ? ts_k : ts_v, rowb = side == 0 ? rowb_k : rowb_v;
                     if (!ts) continue;
+                    #pragma unroll 1
                     for (int cls = cb; cls < cb + nb; ++cls) {
                         const int n_c = n_of_class(cls);
+                        #pragma unroll 1
                         for (int a0 = 0; a0 < n_c; a0 += ts) {
                             const uint32_t bytes = (uint32_t)(min(ts, n_c - a0) * rowb);
                             const bf16* src = side == 0 ? mid_row<bf16>(c.k_mid, s, b, h, cls, a0, s.nfk)
@@ -493,6 +506,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_fft_kernel(const __grid_co
     const float sl2 = s.scale * kLog2e;
 
     // ---- one-time set-up ----
+    #pragma unroll 1
     for (int i = tid; i < s.k; i += kConsumers) {
         E[i] = cis_frac((float)i / (float)s.T);
     }
@@ -500,6 +514,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_fft_kernel(const __grid_co
         const int rl = radix_log2(l), R = 1 << rl, st = 1 << (l - rl);
         if (l > rl) {
             const int off = tw_offset(LS, l);
+            #pragma unroll 1
             for (int i = tid; i < (R - 1) * st; i += kConsumers) {
                 const int qm1 = i / st, j = i - qm1 * st;
                 reinterpret_cast<float2*>(twf)[off + i] = cis_frac((float)(((qm1 + 1) * j) & ((1 << l) - 1)) / (float)(1 << l));
@@ -507,8 +522,9 @@ __global__ void __launch_bounds__(kThreads, 1) decode_fft_kernel(const __grid_co
         }
         l -= rl;
     }
+    #pragma unroll 1
     for (int a = tid; a < S; a += kConsumers) rev[a] = (uint16_t)dif_pos<LS>(a);
-    if (tid < GH + 8) red_s[8 * GH + tid] = 0.f;
+    if (tid < GH + 8) red_s[kWarps * GH + tid] = 0.f;
 
     // B fragments of q for the kept K dims: column gq is slot gq = head hperm(gq);
     // round rd covers pieces 4 rd + tq of a row, two k-steps each
@@ -529,12 +545,13 @@ __global__ void __launch_bounds__(kThreads, 1) decode_fft_kernel(const __grid_co
             }
     }
     int32_t* bar = ws.bar + 4 * (((size_t)b * s.Hkv + h) * p.n_pass + pass);
-    const int m0 = (int)((long long)part * s.M / p.n_part), m1 = (int)((long long)(part + 1) * s.M / p.n_part);
+    const int m0 = part * s.M / p.n_part, m1 = (part + 1) * s.M / p.n_part;
     if (p.fused) {
         // this CTA's slice of the coefficient rows of C^V will be wanted at the very end: start it towards L2
         if (s.dcv > 0) {
             const char* cv = reinterpret_cast<const char*>(coef_rows(c.coef_v, s, b, h, s.dcv) + (size_t)m0 * s.dcv);
             const int bytes = (m1 - m0) * s.dcv * 4;
+            #pragma unroll 1
             for (int o = tid * 128; o < bytes; o += kConsumers * 128) asm volatile("prefetch.global.L2 [%0];" ::"l"(cv + o));
         }
         // u_g[m] = scale * log2(e) * w_m * sum_e C^K[m][e] q_g[D^kc[e]] for rows [m0, m1): eight lanes per row
@@ -548,6 +565,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_fft_kernel(const __grid_co
             consumer_sync();
             const float* ck = coef_rows(c.coef_k, s, b, h, s.dck);
             const int l8 = tid & 7, rgi = tid >> 3, nv = s.dck >> 2;
+            #pragma unroll 1
             for (int r0 = m0; r0 < m1; r0 += kConsumers / 8) {
                 const int r = r0 + rgi;
                 float a[GH];
@@ -555,6 +573,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_fft_kernel(const __grid_co
                 for (int g = 0; g < GH; ++g) a[g] = 0.f;
                 if (r < m1) {
                     const float4* row = reinterpret_cast<const float4*>(ck + (size_t)r * s.dck);
+                    #pragma unroll 1
                     for (int v = l8; v < nv; v += 8) {
                         const float4 x = __ldg(row + v);
 #pragma unroll
@@ -586,6 +605,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_fft_kernel(const __grid_co
     for (int i = tid; i < GH * s.d; i += kConsumers) o_s[i] = 0.f;
     // ut[n] = (A.re, A.im, B.re, B.im), A = heads of the real slots, B = heads of the imaginary slots;
     // all loads of an entry are issued together
+    #pragma unroll 1
     for (int n = tid; n < s.k; n += kConsumers) {
         float2 uv[GH];
 #pragma unroll
@@ -636,7 +656,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_fft_kernel(const __grid_co
         for (int g = 0; g < GH; ++g) {
             float r = red_s[g];
 #pragma unroll
-            for (int w = 1; w < 8; ++w) r = fmaxf(r, red_s[w * GH + g]);
+            for (int w = 1; w < kWarps; ++w) r = fmaxf(r, red_s[w * GH + g]);
             mx[g] = r;
         }
     };
@@ -702,14 +722,18 @@ __global__ void __launch_bounds__(kThreads, 1) decode_fft_kernel(const __grid_co
         const int nmtw = (s.d + 15) >> 4;
         float* sb = fbuf;                                 // natural order, no transform
         bf16* pb = pbt;
+        #pragma unroll 1
         for (int t0 = w0; t0 < w1; t0 += wchunk) {
             const int n_tok = min(w1, t0 + wchunk) - t0;
             const WinSegs sg = win_segments(t0, t0 + n_tok, n_init, n_local, head, s.l_local);
+            #pragma unroll 1
             for (int si = 0; si < sg.n; ++si)
+                #pragma unroll 1
                 for (int r0 = 0; r0 < sg.cnt[si]; r0 += ts_w) {
                     const int nt = min(ts_w, sg.cnt[si] - r0);
                     const unsigned char* tile = wait_tile();
-                    for (int grp = (warp + 8 - (it * (kWinRowsPerTile / 16)) % 8) & 7; grp * 16 < nt; grp += 8) {   // tiles rotate over the warps
+                    #pragma unroll 1
+                    for (int grp = (warp + kWarps - (it * (kWinRowsPerTile / 16)) % kWarps) % kWarps; grp * 16 < nt; grp += kWarps) {   // tiles rotate over the warps
                         const unsigned char* r_lo = tile + (size_t)(grp * 16 + gq) * 128;      // row & 7 == gq for both rows
                         float d4[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
@@ -740,6 +764,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_fft_kernel(const __grid_co
             float mx[GH], alpha[GH];
 #pragma unroll
             for (int g = 0; g < GH; ++g) mx[g] = kNegBig;
+            #pragma unroll 1
             for (int a = tid; a < n_tok; a += kConsumers) {
                 float v[GH];
                 load_vals(sb + pf(a * GH), v);
@@ -755,6 +780,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_fft_kernel(const __grid_co
                 l_acc[g] *= alpha[g];
             }
             const int n_pad = (n_tok + 15) & ~15;
+            #pragma unroll 1
             for (int a = tid; a < n_pad; a += kConsumers) {
                 float v[GH];
 #pragma unroll
@@ -774,11 +800,14 @@ __global__ void __launch_bounds__(kThreads, 1) decode_fft_kernel(const __grid_co
             }
             consumer_sync();
             const bf16* prow = pb + (size_t)(gq & (GH - 1)) * pbw;
+            #pragma unroll 1
             for (int si = 0; si < sg.n; ++si)
+                #pragma unroll 1
                 for (int r0 = 0; r0 < sg.cnt[si]; r0 += ts_w) {
                     const int nt = min(ts_w, sg.cnt[si] - r0);
                     const unsigned char* tile = wait_tile();
-                    for (int grp = (warp + 8 - (it * (kWinRowsPerTile / 16)) % 8) & 7; grp * 16 < nt; grp += 8) {
+                    #pragma unroll 1
+                    for (int grp = (warp + kWarps - (it * (kWinRowsPerTile / 16)) % kWarps) % kWarps; grp * 16 < nt; grp += kWarps) {
                         const int a = sg.tok[si] + r0 + grp * 16;
                         // the tile's rows may start at any token of the chunk: gather the four p values one by one
                         uint32_t b0 = 0, b1 = 0;
@@ -792,6 +821,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_fft_kernel(const __grid_co
                             // rows past the end of the segment hold whatever follows it in the cache: zero them,
                             // p = 0 does not stop a NaN
                             const int rem = nt - grp * 16, per_row = nhalf * 8;
+                            #pragma unroll 1
                             for (int i = lane; i < (16 - rem) * per_row; i += 32) {
                                 const int rr = grp * 16 + rem + i / per_row, cc = i % per_row;
                                 *reinterpret_cast<uint4*>(const_cast<unsigned char*>(tile) + (cc >> 3) * kWinHalfBytes + rr * 128 + ((cc & 7) << 4)) =
@@ -839,6 +869,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_fft_kernel(const __grid_co
             for (int i = 0; i < 4; ++i) acc[mt][i] = 0.f;
         const int nmt = (s.nfv + 15) >> 4;
 
+        #pragma unroll 1
         for (int cb = c0; cb < c1; cb += NB) {
             const int nb = min(NB, c1 - cb);
             if (n_of_class(cb) == 0) break;               // classes are filled in order: nothing further on
@@ -846,14 +877,19 @@ __global__ void __launch_bounds__(kThreads, 1) decode_fft_kernel(const __grid_co
             // packed Hermitian spectra of the nb classes: X_m = V^A_m + i V^B_m per complex lane,
             // V_m = v_m + conj(v_{S-m}), v_n = (1/2) u~_n e^{i theta n c}.  Pair 0 is bins (0, S/2).
             if (s.dck > 0) {
-                for (int pr = tid; pr < S / 2; pr += kConsumers) {
+                // neighbouring lanes share a pair of bins and take half of the classes each
+                const int hcls = (nb + 1) >> 1;
+                #pragma unroll 1
+                for (int item = tid; item < S; item += kConsumers) {
+                    const int pr = item >> 1, ci0 = (item & 1) * hcls, ci1 = min(nb, ci0 + hcls);
                     const int m = pr, mc = pr == 0 ? S / 2 : S - pr;
                     PC<N> Am = czero, Bm = czero, Ac = czero, Bc = czero;
                     float2 em = make_float2(1.f, 0.f), ec = make_float2(1.f, 0.f);
                     if (m < s.k) { ld_entry(ut, m, Am, Bm); em = E[m]; }
                     if (mc < s.k) { ld_entry(ut, mc, Ac, Bc); ec = E[mc]; }
-                    float2 twm = seed_tw(m, cb), twc = seed_tw(mc, cb);
-                    for (int ci = 0; ci < nb; ++ci) {
+                    float2 twm = seed_tw(m, cb + ci0), twc = seed_tw(mc, cb + ci0);
+                    #pragma unroll 1
+                    for (int ci = ci0; ci < ci1; ++ci) {
                         const PR<N> wmr = splat<N>(twm.x), wmi = splat<N>(twm.y), wcr = splat<N>(twc.x), wci = splat<N>(twc.y);
                         const PC<N> vAm = cmulw(Am, wmr, wmi), vBm = cmulw(Bm, wmr, wmi);
                         const PC<N> vAc = cmulw(Ac, wcr, wci), vBc = cmulw(Bc, wcr, wci);
@@ -875,19 +911,23 @@ __global__ void __launch_bounds__(kThreads, 1) decode_fft_kernel(const __grid_co
                 consumer_sync();
                 fft_run<GH, LS, LS, false>(fbuf, fb_floats, nb, twf, tid);        // score of slot a at point rev[a]
             } else {
+                #pragma unroll 1
                 for (int i = tid; i < nb * fb_floats; i += kConsumers) fbuf[i] = 0.f;
                 consumer_sync();
             }
 
             // kept dims: s = sl2 * (q_u . K^mu) + compressed part, 16 tokens per mma
             if (ts_k) {
+                #pragma unroll 1
                 for (int ci = 0; ci < nb; ++ci) {
                     const int n_c = n_of_class(cb + ci);
                     float* base = fbuf + ci * fb_floats;
+                    #pragma unroll 1
                     for (int a0 = 0; a0 < n_c; a0 += ts_k) {
                         const int nt = min(ts_k, n_c - a0);
                         const unsigned char* tile = wait_tile();
-                        for (int grp = warp; grp * 16 < nt; grp += 8) {
+                        #pragma unroll 1
+                        for (int grp = warp; grp * 16 < nt; grp += kWarps) {
                             const unsigned char* r_lo = tile + (size_t)(grp * 16 + gq) * rowb_k;
                             const unsigned char* r_hi = r_lo + 8 * rowb_k;
                             float d4[4] = {0.f, 0.f, 0.f, 0.f};
@@ -928,6 +968,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_fft_kernel(const __grid_co
             float mx[GH], alpha[GH];
 #pragma unroll
             for (int g = 0; g < GH; ++g) mx[g] = kNegBig;
+            #pragma unroll 1
             for (int i = tid; i < (nb << LS); i += kConsumers) {
                 const int ci = i >> LS, a = i & (S - 1);
                 if (a < n_of_class(cb + ci)) {
@@ -945,6 +986,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_fft_kernel(const __grid_co
                 m_run[g] = m_new;
                 l_acc[g] *= alpha[g];
             }
+            #pragma unroll 1
             for (int i = tid; i < (nb << LS); i += kConsumers) {
                 const int ci = i >> LS, a = i & (S - 1);
                 float* pt = fbuf + ci * fb_floats + pf(rev[a] * GH);
@@ -975,13 +1017,16 @@ __global__ void __launch_bounds__(kThreads, 1) decode_fft_kernel(const __grid_co
 
             // o^u[dim][slot] += V^mu^T p, 16 tokens per mma
             if (ts_v) {
+                #pragma unroll 1
                 for (int ci = 0; ci < nb; ++ci) {
                     const int n_c = n_of_class(cb + ci);
                     const bf16* prow = pbt + (size_t)(ci * GH + (gq & (GH - 1))) * pbs;
+                    #pragma unroll 1
                     for (int a0 = 0; a0 < n_c; a0 += ts_v) {
                         const int nt = min(ts_v, n_c - a0);
                         const unsigned char* tile = wait_tile();
-                        for (int grp = warp; grp * 16 < nt; grp += 8) {
+                        #pragma unroll 1
+                        for (int grp = warp; grp * 16 < nt; grp += kWarps) {
                             const int a = a0 + grp * 16;
                             uint32_t b0 = 0, b1 = 0;
                             if (gq < GH) {
@@ -1014,15 +1059,19 @@ __global__ void __launch_bounds__(kThreads, 1) decode_fft_kernel(const __grid_co
                 if constexpr (N == 2) { alA = pk(alpha[0], alpha[1]); alB = pk(alpha[2], alpha[3]); }
                 else { alA = PR<1>{alpha[0]}; alB = PR<1>{alpha[1]}; }
                 const PR<N> half = splat<N>(0.5f);
-                for (int pr = tid; pr < S / 2; pr += kConsumers) {
+                const int hcls = (nb + 1) >> 1;
+                #pragma unroll 1
+                for (int item = tid; item < S; item += kConsumers) {       // whole warps: S is a multiple of 32
+                    const int pr = item >> 1, ci0 = (item & 1) * hcls;
                     const int m = pr, mc = pr == 0 ? S / 2 : S - pr;
-                    if (m >= s.k && mc >= s.k) continue;
+                    const int ci1 = (m >= s.k && mc >= s.k) ? ci0 : min(nb, ci0 + hcls);
                     float2 em = make_float2(1.f, 0.f), ec = make_float2(1.f, 0.f);
                     if (m < s.k) em = E[m];
                     if (mc < s.k) ec = E[mc];
-                    float2 twm = seed_tw(m, cb), twc = seed_tw(mc, cb);
+                    float2 twm = seed_tw(m, cb + ci0), twc = seed_tw(mc, cb + ci0);
                     PC<N> zAm = czero, zBm = czero, zAc = czero, zBc = czero;
-                    for (int ci = 0; ci < nb; ++ci) {
+                    #pragma unroll 1
+                    for (int ci = ci0; ci < ci1; ++ci) {
                         const float* base = fbuf + ci * fb_floats;
                         const PC<N> ya = ld_pt<N>(base + pf(m * GH)), yb = ld_pt<N>(base + pf(mc * GH));
                         const PR<N> wmr = splat<N>(twm.x), wmi = splat<N>(twm.y), wcr = splat<N>(twc.x), wci = splat<N>(twc.y);
@@ -1046,6 +1095,8 @@ __global__ void __launch_bounds__(kThreads, 1) decode_fft_kernel(const __grid_co
                         twm = cmulf(twm, em);
                         twc = cmulf(twc, ec);
                     }
+                    zAm = pair_sum(zAm); zBm = pair_sum(zBm); zAc = pair_sum(zAc); zBc = pair_sum(zBc);
+                    if (item & 1) continue;
                     if (m < s.k) {
                         PC<N> A, B;
                         ld_entry(z_s, m, A, B);
@@ -1083,7 +1134,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_fft_kernel(const __grid_co
         float v = l_acc[g];
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
-        if (lane == 0) atomicAdd(red_s + 8 * GH + g, v);
+        if (lane == 0) atomicAdd(red_s + kWarps * GH + g, v);
     }
     consumer_sync();
 
@@ -1092,6 +1143,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_fft_kernel(const __grid_co
         const int g = i / s.d, e = i - g * s.d;
         if (g < ng) ws.o[(((size_t)b * s.Hq + g_first + g) * p.n_part + part) * s.d + e] = o_s[i];
     }
+    #pragma unroll 1
     for (int n = tid; n < s.k; n += kConsumers) {
         const float* e = z_s + n * 2 * GH;
 #pragma unroll
@@ -1110,7 +1162,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_fft_kernel(const __grid_co
 #pragma unroll
             for (int sl = 1; sl < GH; ++sl) if (tid == sl) mv = m_run[sl];
             ml[0] = mv;
-            ml[1] = red_s[8 * GH + tid];
+            ml[1] = red_s[kWarps * GH + tid];
         }
     }
     if (!p.fused) return;
@@ -1144,8 +1196,10 @@ __global__ void __launch_bounds__(kThreads, 1) decode_fft_kernel(const __grid_co
     consumer_sync();
     if (tid < GH) {
         float mx = kNegBig;
+        #pragma unroll 1
         for (int sp = 0; sp < np; ++sp) mx = fmaxf(mx, al_s[tid * np + sp]);
         float Lsum = 0.f;
+        #pragma unroll 1
         for (int sp = 0; sp < np; ++sp) {
             const float a = exp2f(al_s[tid * np + sp] - mx);
             al_s[tid * np + sp] = a;
@@ -1158,6 +1212,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_fft_kernel(const __grid_co
     auto merged = [&](const float* al, const float* src, size_t stride) -> float {
         float v0 = 0.f, v1 = 0.f;
         int sp = 0;
+        #pragma unroll 1
         for (; sp + 8 <= np; sp += 8) {
             float x[8];
 #pragma unroll
@@ -1165,6 +1220,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_fft_kernel(const __grid_co
 #pragma unroll
             for (int i = 0; i < 8; i += 2) { v0 = fmaf(al[sp + i], x[i], v0); v1 = fmaf(al[sp + i + 1], x[i + 1], v1); }
         }
+        #pragma unroll 1
         for (; sp < np; ++sp) v0 = fmaf(al[sp], __ldcg(src + (size_t)sp * stride), v0);
         return v0 + v1;
     };
@@ -1176,7 +1232,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_fft_kernel(const __grid_co
         zw_s[g * rows_max + r] = v;
     }
     {
-        const int e0 = (int)((long long)part * s.d / np), e1 = (int)((long long)(part + 1) * s.d / np);
+        const int e0 = part * s.d / np, e1 = (part + 1) * s.d / np;
         for (int t = tid; t < GH * (e1 - e0); t += kConsumers) {
             const int g = t / (e1 - e0), e = e0 + t - g * (e1 - e0);
             if (g < ng) ws.om[(qh0 + g) * s.d + e] = merged(al_s + g * np, ws.o + (qh0 + g) * np * s.d + e, (size_t)s.d);
@@ -1209,6 +1265,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_fft_kernel(const __grid_co
         for (int t = tid; t < GH * s.dcv; t += kConsumers) {
             const int g = t / s.dcv, e = t - g * s.dcv;
             float v = 0.f;
+            #pragma unroll 1
             for (int rgi = 0; rgi < nrg; ++rgi) v += ps_s[((size_t)rgi * GH + g) * s.dcv + e];
             if (g < ng) ws.oc[((qh0 + g) * np + part) * s.dcv + e] = v;
         }
@@ -1223,10 +1280,12 @@ __global__ void __launch_bounds__(kThreads, 1) decode_fft_kernel(const __grid_co
     }
     consumer_sync();
     if (!*last_s) return;
+    #pragma unroll 1
     for (int e = tid; e < s.d; e += kConsumers) inv_s[e] = -1;
     consumer_sync();
     if (s.dcv > 0) {
         const int32_t* idc_v = c.idx_comp_v + (size_t)h * s.dcv;
+        #pragma unroll 1
         for (int e = tid; e < s.dcv; e += kConsumers) inv_s[idc_v[e]] = e;
     }
     consumer_sync();
@@ -1239,6 +1298,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_fft_kernel(const __grid_co
             const float* oc = ws.oc + (qh0 + g) * np * s.dcv + slot;
             float w0 = 0.f, w1 = 0.f;
             int x = 0;
+            #pragma unroll 1
             for (; x + 8 <= np; x += 8) {
                 float cc[8];
 #pragma unroll
@@ -1246,6 +1306,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_fft_kernel(const __grid_co
 #pragma unroll
                 for (int i = 0; i < 8; i += 2) { w0 += cc[i]; w1 += cc[i + 1]; }
             }
+            #pragma unroll 1
             for (; x < np; ++x) w0 += __ldcg(oc + (size_t)x * s.dcv);
             v += w0 + w1;
         }
