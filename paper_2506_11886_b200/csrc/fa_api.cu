@@ -98,6 +98,17 @@ fa_status plan_decode(const fa_layout& l, DecodePlan* p) {
         const int per_job = kNumSms / jobs;
         const long long win_bytes = 2LL * (s.l_init + s.l_local) * s.d;
         const long long class_bytes = (long long)(s.T / s.P) * (s.nfk + s.nfv);
+        // classes transformed together: enough butterflies for all consumer threads, within shared memory
+        auto pick_nb = [&](int n_split) {
+            const int S = s.T / s.P;
+            int nb = 2048 / S;
+            if (nb < 1) nb = 1;
+            if (nb > 8) nb = 8;
+            const int per_cta = (s.P + n_split - 1) / n_split;
+            if (nb > per_cta) nb = per_cta;
+            while (nb > 1 && decode_fft_smem_bytes(s, log2S, p->gh, nb) > 227 * 1024) --nb;
+            return nb;
+        };
         p->fused = 0;
         p->n_wsplit = 0;
         if (l.decode_algo != FA_DECODE_FFT_SPLIT && per_job >= 2) {
@@ -115,10 +126,15 @@ fa_status plan_decode(const fa_layout& l, DecodePlan* p) {
             // fewest class CTAs that reach the same classes per CTA
             const int per_cta = (s.P + best_ns - 1) / best_ns;
             best_ns = (s.P + per_cta - 1) / per_cta;
-            p->fused = 1;
-            p->n_split = best_ns;
-            p->n_wsplit = best_nw;
-        } else {
+            const int nb = pick_nb(best_ns);
+            if (decode_fft_fused_fits(s, log2S, p->gh, nb, best_ns + best_nw)) {
+                p->fused = 1;
+                p->n_split = best_ns;
+                p->n_wsplit = best_nw;
+                p->nb = nb;
+            }
+        }
+        if (!p->fused) {
             // classes are indivisible: pick the split count that minimises waves * classes per CTA,
             // smallest count on ties to keep the partial results small
             const int slots = kNumSms;
@@ -130,16 +146,8 @@ fa_status plan_decode(const fa_layout& l, DecodePlan* p) {
                 if (best_cost < 0 || cost < best_cost) { best_cost = cost; best = n; }
             }
             p->n_split = best;
+            p->nb = pick_nb(best);
         }
-        // classes transformed together: enough butterflies for all consumer threads, within shared memory
-        const int S = s.T / s.P;
-        int nb = 2048 / S;
-        if (nb < 1) nb = 1;
-        if (nb > 8) nb = 8;
-        const int per_cta = (s.P + p->n_split - 1) / p->n_split;
-        if (nb > per_cta) nb = per_cta;
-        while (nb > 1 && decode_fft_smem_bytes(s, log2S, p->gh, nb) > 227 * 1024) --nb;
-        p->nb = nb;
     } else {
         p->gh = s.G >= 4 ? 4 : (s.G >= 2 ? 2 : 1);
         if (s.G == 3) p->gh = 4;

@@ -110,6 +110,7 @@ cudaError_t launch_decode_direct(const Dims&, const CacheDev&, int dtype, const 
 cudaError_t launch_decode_fft(const Dims&, const CacheDev&, int dtype, const DecodePlan&, const void* q, void* out, char* ws,
                               cudaStream_t);
 size_t decode_fft_smem_bytes(const Dims&, int log2S, int gh, int nb);
+bool decode_fft_fused_fits(const Dims&, int log2S, int gh, int nb, int n_part);
 cudaError_t launch_decode_epilogue(const Dims&, const CacheDev&, int dtype, const DecodePlan&, void* out, char* ws,
                                    cudaStream_t);
 

@@ -82,6 +82,11 @@ __device__ __forceinline__ void tma_load_3d(void* dst, const CUtensorMap* tm, in
                  "l"(reinterpret_cast<uint64_t>(tm)), "r"(x0), "r"(y0), "r"(z), "r"(smem_addr(bar))
                  : "memory");
 }
+// 16-byte asynchronous copy that bypasses L1 (the source may have been written by another SM)
+__device__ __forceinline__ void cp_async16(void* dst, const void* src) {
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(smem_addr(dst)), "l"(__cvta_generic_to_global(src)) : "memory");
+}
+__device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.commit_group;\ncp.async.wait_group 0;" ::: "memory"); }
 __device__ __forceinline__ void consumer_sync() { asm volatile("bar.sync 1, %0;" ::"n"(kConsumers) : "memory"); }
 
 // Barrier among the CTAs of one (b, KV head, pass) on a global counter (fused kernel only: a
@@ -505,6 +510,16 @@ __global__ void __launch_bounds__(kThreads, 1) decode_fft_kernel(const __grid_co
     const int npk = s.nfk >> 3, nchv = s.nfv >> 3, npw = s.d >> 3;
     const float sl2 = s.scale * kLog2e;
 
+    int32_t* bar = ws.bar + 4 * (((size_t)b * s.Hkv + h) * p.n_pass + pass);
+    // coefficient rows of this part in the fused steps: slices on 4-row boundaries (16-byte copies)
+    const int m0 = part * (s.M >> 2) / p.n_part * 4, m1 = (part + 1) * (s.M >> 2) / p.n_part * 4;
+    if (p.fused && s.dck > 0) {
+        // this part's rows of C^K go to the (still unused) transform buffers while the tables are built
+        const float* ck = coef_rows(c.coef_k, s, b, h, s.dck) + (size_t)m0 * s.dck;
+#pragma unroll 1
+        for (int i = tid; i < (m1 - m0) * (s.dck >> 2); i += kConsumers) cp_async16(fbuf + 4 * i, ck + 4 * i);
+    }
+
     // ---- one-time set-up ----
     #pragma unroll 1
     for (int i = tid; i < s.k; i += kConsumers) {
@@ -544,8 +559,6 @@ __global__ void __launch_bounds__(kThreads, 1) decode_fft_kernel(const __grid_co
                 qk[rd][ks][1] = on ? pack_bf16(qrow[idf_k[e0 + 2]], qrow[idf_k[e0 + 3]]) : 0u;
             }
     }
-    int32_t* bar = ws.bar + 4 * (((size_t)b * s.Hkv + h) * p.n_pass + pass);
-    const int m0 = part * s.M / p.n_part, m1 = (part + 1) * s.M / p.n_part;
     if (p.fused) {
         // this CTA's slice of the coefficient rows of C^V will be wanted at the very end: start it towards L2
         if (s.dcv > 0) {
@@ -562,8 +575,8 @@ __global__ void __launch_bounds__(kThreads, 1) decode_fft_kernel(const __grid_co
                 const int g = i / s.dck, e = i - g * s.dck;
                 qc[i] = g < ng ? __bfloat162float(q[((size_t)b * s.Hq + g_first + g) * s.d + idc_k[e]]) : 0.f;
             }
+            cp_async_wait_all();
             consumer_sync();
-            const float* ck = coef_rows(c.coef_k, s, b, h, s.dck);
             const int l8 = tid & 7, rgi = tid >> 3, nv = s.dck >> 2;
             #pragma unroll 1
             for (int r0 = m0; r0 < m1; r0 += kConsumers / 8) {
@@ -572,10 +585,10 @@ __global__ void __launch_bounds__(kThreads, 1) decode_fft_kernel(const __grid_co
 #pragma unroll
                 for (int g = 0; g < GH; ++g) a[g] = 0.f;
                 if (r < m1) {
-                    const float4* row = reinterpret_cast<const float4*>(ck + (size_t)r * s.dck);
+                    const float4* row = reinterpret_cast<const float4*>(fbuf + (r - m0) * s.dck);
                     #pragma unroll 1
                     for (int v = l8; v < nv; v += 8) {
-                        const float4 x = __ldg(row + v);
+                        const float4 x = row[v];
 #pragma unroll
                         for (int g = 0; g < GH; ++g) {
                             const float4 y = *reinterpret_cast<const float4*>(qc + g * s.dck + 4 * v);
@@ -1169,86 +1182,85 @@ __global__ void __launch_bounds__(kThreads, 1) decode_fft_kernel(const __grid_co
 
     // ------------------------------ merge (fused kernel) ------------------------------
     // All parts of this (b, KV head, pass) have written their partial results.  Each part then
-    // merges a slice: its rows of z against its rows of C^V, and its share of the dims of o.  The
-    // last part to finish adds the slices in a fixed order, normalises and writes the output rows.
-    part_arrive(bar + 1, tid);
-    part_wait(bar + 1, p.n_part, tid, fail, c.status);
+    // merges a slice of the coefficient rows: its rows of every part's z against its rows of C^V.
+    // The last part to finish adds the slices and the parts' o in a fixed order, normalises and
+    // writes the output rows.  Everything a step needs from global memory is fetched with one batch
+    // of 16-byte asynchronous copies into the stage ring (every tile has been consumed), so each
+    // step costs one memory round trip.
     const int np = p.n_part;
-    const int rows = m1 - m0, rows_max = (s.M + np - 1) / np + 1;
+    const int rows = m1 - m0, rows_max = (s.M / 4 + np - 1) / np * 4 + 4;
     const size_t qh0 = (size_t)b * s.Hq + g_first;
-    // scratch in the stage ring: every tile has been consumed
     float* al_s = reinterpret_cast<float*>(stages);        // [GH][np] maxima, then exp2(m - max)
     float* l_s = al_s + GH * np;                           // [GH][np]
     float* linv_s = l_s + GH * np;                         // [GH]
-    float* zw_s = al_s + ((2 * GH * np + GH + 3) & ~3);    // [GH][rows_max], 16-byte aligned like ps_s
-    float* ps_s = zw_s + ((GH * rows_max + 3) & ~3);       // [row groups][GH][dcv]
-    const int nv = s.dcv >> 2, nrg = nv ? kConsumers / nv : 0;
-    int* inv_s = reinterpret_cast<int*>(ps_s + (size_t)nrg * GH * s.dcv);   // [d]
+    float* zw_s = al_s + ((2 * GH * np + GH + 3) & ~3);    // [GH][rows_max]
+    float* big_s = zw_s + GH * rows_max;                   // step 1: C^V rows, z slices, partial sums; step 2: o and o^c parts
+    float* cv_s = big_s;                                   // [rows][dcv]
+    float* zs_s = cv_s + rows_max * s.dcv;                 // [GH][np][rows_max]
+    float* ps_s = zs_s + GH * np * rows_max;               // [row groups][GH][dcv]
     volatile int* last_s = fail + 1;
+    const int nv = s.dcv >> 2, nrg = nv ? kConsumers / nv : 0;
 
+    if (s.dcv > 0) {
+        const float* cv = coef_rows(c.coef_v, s, b, h, s.dcv) + (size_t)m0 * s.dcv;
+#pragma unroll 1
+        for (int i = tid; i < rows * nv; i += kConsumers) cp_async16(cv_s + 4 * i, cv + 4 * i);
+    }
+    part_arrive(bar + 1, tid);
+    part_wait(bar + 1, np, tid, fail, c.status);
+    if (s.dcv > 0) {
+        const int r4 = rows >> 2;
+#pragma unroll 1
+        for (int i = tid; i < GH * np * r4; i += kConsumers) {
+            const int gs = i / r4, j = i - gs * r4, g = gs / np;
+            if (g < ng) cp_async16(zs_s + gs * rows_max + 4 * j, ws.z + (qh0 * np + gs) * s.M + m0 + 4 * j);
+        }
+    }
+#pragma unroll 1
     for (int i = tid; i < GH * np; i += kConsumers) {
-        const int g = i / np, sp = i - g * np;
         float2 ml = make_float2(kNegBig, 0.f);
-        if (g < ng) ml = __ldcg(reinterpret_cast<const float2*>(ws.ml + ((qh0 + g) * np + sp) * 2));
+        if (i / np < ng) ml = __ldcg(reinterpret_cast<const float2*>(ws.ml + (qh0 * np + i) * 2));
         al_s[i] = ml.x;
         l_s[i] = ml.y;
     }
+    cp_async_wait_all();
     consumer_sync();
     if (tid < GH) {
         float mx = kNegBig;
-        #pragma unroll 1
+#pragma unroll 1
         for (int sp = 0; sp < np; ++sp) mx = fmaxf(mx, al_s[tid * np + sp]);
         float Lsum = 0.f;
-        #pragma unroll 1
+#pragma unroll 1
         for (int sp = 0; sp < np; ++sp) {
-            const float a = exp2f(al_s[tid * np + sp] - mx);
+            const float a = ex2(al_s[tid * np + sp] - mx);
             al_s[tid * np + sp] = a;
             Lsum = fmaf(a, l_s[tid * np + sp], Lsum);
         }
-        linv_s[tid] = Lsum > 0.f ? 1.0f / Lsum : 0.f;
-    }
-    consumer_sync();
-    // sum over the parts of al[sp] * src[sp * stride], eight independent loads in flight
-    auto merged = [&](const float* al, const float* src, size_t stride) -> float {
-        float v0 = 0.f, v1 = 0.f;
-        int sp = 0;
-        #pragma unroll 1
-        for (; sp + 8 <= np; sp += 8) {
-            float x[8];
-#pragma unroll
-            for (int i = 0; i < 8; ++i) x[i] = __ldcg(src + (size_t)(sp + i) * stride);
-#pragma unroll
-            for (int i = 0; i < 8; i += 2) { v0 = fmaf(al[sp + i], x[i], v0); v1 = fmaf(al[sp + i + 1], x[i + 1], v1); }
-        }
-        #pragma unroll 1
-        for (; sp < np; ++sp) v0 = fmaf(al[sp], __ldcg(src + (size_t)sp * stride), v0);
-        return v0 + v1;
-    };
-    for (int t = tid; t < GH * rows; t += kConsumers) {
-        const int g = t / rows, r = t - g * rows;
-        float v = 0.f;
-        if (g < ng && s.dcv > 0)
-            v = merged(al_s + g * np, ws.z + (qh0 + g) * np * s.M + m0 + r, (size_t)s.M) * recon_weight(s.norm, m0 + r, s.k, s.T);
-        zw_s[g * rows_max + r] = v;
-    }
-    {
-        const int e0 = part * s.d / np, e1 = (part + 1) * s.d / np;
-        for (int t = tid; t < GH * (e1 - e0); t += kConsumers) {
-            const int g = t / (e1 - e0), e = e0 + t - g * (e1 - e0);
-            if (g < ng) ws.om[(qh0 + g) * s.d + e] = merged(al_s + g * np, ws.o + (qh0 + g) * np * s.d + e, (size_t)s.d);
-        }
+        linv_s[tid] = Lsum > 0.f ? __fdividef(1.0f, Lsum) : 0.f;
     }
     consumer_sync();
     if (s.dcv > 0) {
+#pragma unroll 1
+        for (int t = tid; t < GH * rows; t += kConsumers) {
+            const int g = t / rows, r = t - g * rows;
+            float v = 0.f;
+            if (g < ng) {
+                const float* z = zs_s + g * np * rows_max + r;
+#pragma unroll 1
+                for (int sp = 0; sp < np; ++sp) v = fmaf(al_s[g * np + sp], z[sp * rows_max], v);
+                v *= recon_weight(s.norm, m0 + r, s.k, s.T);
+            }
+            zw_s[g * rows_max + r] = v;
+        }
+        consumer_sync();
         if (tid < nrg * nv) {
             const int v = tid % nv, rgi = tid / nv;
             float4 acc4[GH];
 #pragma unroll
             for (int g = 0; g < GH; ++g) acc4[g] = make_float4(0.f, 0.f, 0.f, 0.f);
-            const float4* cv = reinterpret_cast<const float4*>(coef_rows(c.coef_v, s, b, h, s.dcv) + (size_t)m0 * s.dcv) + v;
-#pragma unroll 4
+#pragma unroll 1
             for (int r = rgi; r < rows; r += nrg) {
-                const float4 x = __ldg(cv + (size_t)r * nv);
+                const float4 x = *reinterpret_cast<const float4*>(cv_s + r * s.dcv + 4 * v);
 #pragma unroll
                 for (int g = 0; g < GH; ++g) {
                     const float w = zw_s[g * rows_max + r];
@@ -1259,14 +1271,15 @@ __global__ void __launch_bounds__(kThreads, 1) decode_fft_kernel(const __grid_co
                 }
             }
 #pragma unroll
-            for (int g = 0; g < GH; ++g) *reinterpret_cast<float4*>(ps_s + ((size_t)rgi * GH + g) * s.dcv + 4 * v) = acc4[g];
+            for (int g = 0; g < GH; ++g) *reinterpret_cast<float4*>(ps_s + (rgi * GH + g) * s.dcv + 4 * v) = acc4[g];
         }
         consumer_sync();
+#pragma unroll 1
         for (int t = tid; t < GH * s.dcv; t += kConsumers) {
             const int g = t / s.dcv, e = t - g * s.dcv;
             float v = 0.f;
-            #pragma unroll 1
-            for (int rgi = 0; rgi < nrg; ++rgi) v += ps_s[((size_t)rgi * GH + g) * s.dcv + e];
+#pragma unroll 1
+            for (int rgi = 0; rgi < nrg; ++rgi) v += ps_s[(rgi * GH + g) * s.dcv + e];
             if (g < ng) ws.oc[((qh0 + g) * np + part) * s.dcv + e] = v;
         }
     }
@@ -1280,35 +1293,40 @@ __global__ void __launch_bounds__(kThreads, 1) decode_fft_kernel(const __grid_co
     }
     consumer_sync();
     if (!*last_s) return;
-    #pragma unroll 1
+    float* op_s = big_s;                                   // [GH][np][d]
+    float* ocp_s = op_s + GH * np * s.d;                   // [GH][np][dcv]
+    int* inv_s = reinterpret_cast<int*>(ocp_s + GH * np * s.dcv);   // [d] dim -> slot in D^vc, or -1
+    {
+        const int nd4 = s.d >> 2;
+#pragma unroll 1
+        for (int i = tid; i < ng * np * nd4; i += kConsumers) cp_async16(op_s + 4 * i, ws.o + qh0 * np * s.d + 4 * i);
+#pragma unroll 1
+        for (int i = tid; i < ng * np * nv; i += kConsumers) cp_async16(ocp_s + 4 * i, ws.oc + qh0 * np * s.dcv + 4 * i);
+    }
+#pragma unroll 1
     for (int e = tid; e < s.d; e += kConsumers) inv_s[e] = -1;
     consumer_sync();
     if (s.dcv > 0) {
         const int32_t* idc_v = c.idx_comp_v + (size_t)h * s.dcv;
-        #pragma unroll 1
+#pragma unroll 1
         for (int e = tid; e < s.dcv; e += kConsumers) inv_s[idc_v[e]] = e;
     }
+    cp_async_wait_all();
     consumer_sync();
-    for (int t = tid; t < GH * s.d; t += kConsumers) {
+#pragma unroll 1
+    for (int t = tid; t < ng * s.d; t += kConsumers) {
         const int g = t / s.d, e = t - g * s.d;
-        if (g >= ng) continue;
-        float v = __ldcg(ws.om + (qh0 + g) * s.d + e);
+        const float* o = op_s + g * np * s.d + e;
+        float v = 0.f;
+#pragma unroll 1
+        for (int sp = 0; sp < np; ++sp) v = fmaf(al_s[g * np + sp], o[sp * s.d], v);
         const int slot = inv_s[e];
         if (slot >= 0) {
-            const float* oc = ws.oc + (qh0 + g) * np * s.dcv + slot;
-            float w0 = 0.f, w1 = 0.f;
-            int x = 0;
-            #pragma unroll 1
-            for (; x + 8 <= np; x += 8) {
-                float cc[8];
-#pragma unroll
-                for (int i = 0; i < 8; ++i) cc[i] = __ldcg(oc + (size_t)(x + i) * s.dcv);
-#pragma unroll
-                for (int i = 0; i < 8; i += 2) { w0 += cc[i]; w1 += cc[i + 1]; }
-            }
-            #pragma unroll 1
-            for (; x < np; ++x) w0 += __ldcg(oc + (size_t)x * s.dcv);
-            v += w0 + w1;
+            const float* oc = ocp_s + g * np * s.dcv + slot;
+            float w = 0.f;
+#pragma unroll 1
+            for (int x = 0; x < np; ++x) w += oc[x * s.dcv];
+            v += w;
         }
         out[(qh0 + g) * s.d + e] = __float2bfloat16_rn(v * linv_s[g]);
     }
@@ -1364,6 +1382,20 @@ cudaError_t launch_fft_ls(const Dims& s, const CacheDev& c, const DecodePlan& p,
 
 size_t decode_fft_smem_bytes(const Dims& s, int log2S, int gh, int nb) {
     return (size_t)fft_smem_layout(log2S, s.k, gh, nb, s.d).total;
+}
+
+// True if the fused kernel's staging areas hold a part's share of the coefficient rows: the rows
+// of C^K in the transform buffers at the start, the merge scratch in the stage ring at the end.
+bool decode_fft_fused_fits(const Dims& s, int log2S, int gh, int nb, int n_part) {
+    if (s.M % 4 != 0) return false;
+    const FftSmem L = fft_smem_layout(log2S, s.k, gh, nb, s.d);
+    const long long rows_max = (s.M / 4 + n_part - 1) / n_part * 4 + 4;
+    if (rows_max * s.dck > (long long)nb * L.fb_floats) return false;
+    const long long nrg = s.dcv ? kConsumers / (s.dcv >> 2) : 0;
+    const long long head = 2LL * gh * n_part + gh + 4 + gh * rows_max;
+    const long long step1 = rows_max * s.dcv + (long long)gh * n_part * rows_max + nrg * gh * s.dcv;
+    const long long step2 = (long long)gh * n_part * (s.d + s.dcv) + s.d;
+    return head + (step1 > step2 ? step1 : step2) <= (long long)kStages * kStageBytes / 4;
 }
 
 cudaError_t launch_decode_fft(const Dims& s, const CacheDev& c, int dtype, const DecodePlan& p, const void* q, void* out,
