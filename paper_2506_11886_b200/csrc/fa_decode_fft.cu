@@ -34,7 +34,7 @@ constexpr int kConsumers = 512;
 constexpr int kWarps = kConsumers / 32;
 constexpr int kThreads = kConsumers + 32;
 constexpr int kStageBytes = 16384;
-constexpr int kStages = 6;
+constexpr int kStages = 5;
 constexpr int kWinRowsPerTile = 64;       // rows of one window tile: two [64 rows x 64 dims] TMA boxes, 128-byte swizzle
 constexpr int kWinHalfBytes = kWinRowsPerTile * 128;
 constexpr uint32_t kSpinLimit = 1u << 24;
@@ -90,13 +90,16 @@ __device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.com
 __device__ __forceinline__ void consumer_sync() { asm volatile("bar.sync 1, %0;" ::"n"(kConsumers) : "memory"); }
 
 // Barrier among the CTAs of one (b, KV head, pass) on a global counter (fused kernel only: a
-// cooperative launch makes all of them resident).  Arrive: every consumer thread has fenced its
-// global writes; one thread adds 1 with release semantics.  Wait: one thread polls with acquire
-// loads, bounded like every other wait of this kernel, then the consumer warps meet.
+// cooperative launch makes all of them resident).  Arrive: the consumer warps meet, then one thread
+// fences (cumulative over what the others wrote before the meeting) and adds 1 with release
+// semantics.  Wait: one thread polls with acquire loads, bounded like every other wait of this
+// kernel, then the consumer warps meet.
 __device__ __forceinline__ void part_arrive(int32_t* cnt, int tid) {
-    __threadfence();
     consumer_sync();
-    if (tid == 0) asm volatile("red.release.gpu.global.add.s32 [%0], 1;" ::"l"(cnt) : "memory");
+    if (tid == 0) {
+        __threadfence();
+        asm volatile("red.release.gpu.global.add.s32 [%0], 1;" ::"l"(cnt) : "memory");
+    }
 }
 __device__ __forceinline__ void part_wait(const int32_t* cnt, int n, int tid, volatile int* fail, int32_t* status) {
     if (tid == 0 && !*fail) {
@@ -340,7 +343,7 @@ __device__ __forceinline__ WinSegs win_segments(int t0, int t1, int n_init, int 
 }
 
 struct FftSmem {
-    int stages_off, fbuf_off, pbt_off, twf_off, rev_off, E_off, ut_off, z_off, o_off, red_off, zero_off, total;
+    int stages_off, fbuf_off, kb_off, pbt_off, twf_off, rev_off, E_off, ut_off, z_off, o_off, red_off, zero_off, total;
     int fb_floats, pbs;
 };
 __host__ __device__ inline FftSmem fft_smem_layout(int log2S, int k, int GH, int NB, int d) {
@@ -353,6 +356,8 @@ __host__ __device__ inline FftSmem fft_smem_layout(int log2S, int k, int GH, int
     off = 1024;                                           // stages are 1024-byte aligned (swizzled window tiles)
     L.stages_off = off; off += kStages * kStageBytes;
     L.fbuf_off = off; off += 4 * NB * L.fb_floats;
+    off = (off + 15) / 16 * 16;
+    L.kb_off = off; off += 4 * NB * S * GH;               // kept-dim scores of the batch, natural token order
     off = (off + 15) / 16 * 16;
     L.pbt_off = off; off += 2 * NB * GH * L.pbs;
     off = (off + 15) / 16 * 16;
@@ -392,6 +397,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_fft_kernel(const __grid_co
     unsigned char* zero16 = smem_raw + L.zero_off;
     unsigned char* stages = smem_raw + L.stages_off;
     float* fbuf = reinterpret_cast<float*>(smem_raw + L.fbuf_off);        // [NB][fb_floats] points of GH floats
+    float* kb = reinterpret_cast<float*>(smem_raw + L.kb_off);            // [NB][S][GH]
     bf16* pbt = reinterpret_cast<bf16*>(smem_raw + L.pbt_off);           // [NB][GH slots][pbs]
     float* twf = reinterpret_cast<float*>(smem_raw + L.twf_off);          // pass twiddles (float2 each)
     uint16_t* rev = reinterpret_cast<uint16_t*>(smem_raw + L.rev_off);    // slot -> point after the DIF passes
@@ -445,33 +451,11 @@ __global__ void __launch_bounds__(kThreads, 1) decode_fft_kernel(const __grid_co
 
     // ============================ producer warp =================================
     if (tid >= kConsumers) {
-        // window rows first (same order as the consumers): tiles of 64 rows, one TMA box per 64 dims
+        // Same order as the consumers: the K tiles of the first batch of classes, the window rows,
+        // then per batch the V tiles (and, from the second batch on, its K tiles first).
         const int plane = tid - kConsumers;
-        int it = 0;
         if (plane == 0) {
-            #pragma unroll 1
-            for (int t0 = w0; t0 < w1; t0 += wchunk) {
-                const WinSegs sg = win_segments(t0, min(w1, t0 + wchunk), n_init, n_local, head, s.l_local);
-                for (int side = 0; side < 2; ++side)
-                    #pragma unroll 1
-                    for (int i = 0; i < sg.n; ++i)
-                        #pragma unroll 1
-                        for (int r0 = 0; r0 < sg.cnt[i]; r0 += ts_w) {
-                            const CUtensorMap* tm = sg.buf[i] == 0 ? (side == 0 ? &tm_ki : &tm_vi) : (side == 0 ? &tm_kl : &tm_vl);
-                            const int st = it % kStages;
-                            if (it >= kStages) mbar_wait(empty + st, ((it / kStages) - 1) & 1, fail, c.status);
-                            if (!*fail) {
-                                mbar_expect_tx(full + st, (uint32_t)(nhalf * kWinHalfBytes));
-                                unsigned char* dst = stages + (size_t)st * kStageBytes;
-                                #pragma unroll 1
-                                for (int hf = 0; hf < nhalf; ++hf)
-                                    tma_load_3d(dst + hf * kWinHalfBytes, tm, hf * 64, sg.row[i] + r0, b * s.Hkv + h, full + st);
-                            }
-                            ++it;
-                        }
-            }
-        }
-        if (plane == 0) {
+            int it = 0;
             auto acquire = [&](uint32_t bytes) -> unsigned char* {
                 const int st = it % kStages;
                 if (it >= kStages) mbar_wait(empty + st, ((it / kStages) - 1) & 1, fail, c.status);
@@ -479,26 +463,47 @@ __global__ void __launch_bounds__(kThreads, 1) decode_fft_kernel(const __grid_co
                 mbar_expect_tx(full + st, bytes);
                 return stages + (size_t)st * kStageBytes;
             };
-            // per batch of NB classes all K tiles, then all V tiles
-            #pragma unroll 1
-            for (int cb = c0; cb < c1; cb += NB) {
-                const int nb = min(NB, c1 - cb);
-                for (int side = 0; side < 2; ++side) {
-                    const int ts = side == 0 ? ts_k : ts_v, rowb = side == 0 ? rowb_k : rowb_v;
-                    if (!ts) continue;
-                    #pragma unroll 1
-                    for (int cls = cb; cls < cb + nb; ++cls) {
-                        const int n_c = n_of_class(cls);
-                        #pragma unroll 1
-                        for (int a0 = 0; a0 < n_c; a0 += ts) {
-                            const uint32_t bytes = (uint32_t)(min(ts, n_c - a0) * rowb);
-                            const bf16* src = side == 0 ? mid_row<bf16>(c.k_mid, s, b, h, cls, a0, s.nfk)
-                                                        : mid_row<bf16>(c.v_mid, s, b, h, cls, a0, s.nfv);
-                            if (unsigned char* dst = acquire(bytes)) bulk_g2s(dst, src, bytes, full + it % kStages);
-                            ++it;
-                        }
+            auto class_tiles = [&](int cb, int nb, int side) {
+                const int ts = side == 0 ? ts_k : ts_v, rowb = side == 0 ? rowb_k : rowb_v;
+                if (!ts) return;
+#pragma unroll 1
+                for (int cls = cb; cls < cb + nb; ++cls) {
+                    const int n_c = n_of_class(cls);
+#pragma unroll 1
+                    for (int a0 = 0; a0 < n_c; a0 += ts) {
+                        const uint32_t bytes = (uint32_t)(min(ts, n_c - a0) * rowb);
+                        const bf16* src = side == 0 ? mid_row<bf16>(c.k_mid, s, b, h, cls, a0, s.nfk)
+                                                    : mid_row<bf16>(c.v_mid, s, b, h, cls, a0, s.nfv);
+                        if (unsigned char* dst = acquire(bytes)) bulk_g2s(dst, src, bytes, full + it % kStages);
+                        ++it;
                     }
                 }
+            };
+            if (c0 < c1) class_tiles(c0, min(NB, c1 - c0), 0);
+            // window rows: tiles of 64 rows, one TMA box per 64 dims
+#pragma unroll 1
+            for (int t0 = w0; t0 < w1; t0 += wchunk) {
+                const WinSegs sg = win_segments(t0, min(w1, t0 + wchunk), n_init, n_local, head, s.l_local);
+#pragma unroll 1
+                for (int side = 0; side < 2; ++side)
+#pragma unroll 1
+                    for (int i = 0; i < sg.n; ++i)
+#pragma unroll 1
+                        for (int r0 = 0; r0 < sg.cnt[i]; r0 += ts_w) {
+                            const CUtensorMap* tm = sg.buf[i] == 0 ? (side == 0 ? &tm_ki : &tm_vi) : (side == 0 ? &tm_kl : &tm_vl);
+                            if (unsigned char* dst = acquire((uint32_t)(nhalf * kWinHalfBytes))) {
+#pragma unroll 1
+                                for (int hf = 0; hf < nhalf; ++hf)
+                                    tma_load_3d(dst + hf * kWinHalfBytes, tm, hf * 64, sg.row[i] + r0, b * s.Hkv + h, full + it % kStages);
+                            }
+                            ++it;
+                        }
+            }
+#pragma unroll 1
+            for (int cb = c0; cb < c1; cb += NB) {
+                const int nb = min(NB, c1 - cb);
+                if (cb != c0) class_tiles(cb, nb, 0);
+                class_tiles(cb, nb, 1);
             }
         }
         return;
@@ -513,6 +518,12 @@ __global__ void __launch_bounds__(kThreads, 1) decode_fft_kernel(const __grid_co
     int32_t* bar = ws.bar + 4 * (((size_t)b * s.Hkv + h) * p.n_pass + pass);
     // coefficient rows of this part in the fused steps: slices on 4-row boundaries (16-byte copies)
     const int m0 = part * (s.M >> 2) / p.n_part * 4, m1 = (part + 1) * (s.M >> 2) / p.n_part * 4;
+    // gathered query of the compressed K dims (one element per thread and round), loaded early
+    float qc_early = 0.f;
+    if (p.fused && s.dck > 0 && tid < GH * s.dck) {
+        const int g = tid / s.dck, e = tid - g * s.dck;
+        if (g < ng) qc_early = __bfloat162float(q[((size_t)b * s.Hq + g_first + g) * s.d + c.idx_comp_k[(size_t)h * s.dck + e]]);
+    }
     if (p.fused && s.dck > 0) {
         // this part's rows of C^K go to the (still unused) transform buffers while the tables are built
         const float* ck = coef_rows(c.coef_k, s, b, h, s.dck) + (size_t)m0 * s.dck;
@@ -559,6 +570,60 @@ __global__ void __launch_bounds__(kThreads, 1) decode_fft_kernel(const __grid_co
                 qk[rd][ks][1] = on ? pack_bf16(qrow[idf_k[e0 + 2]], qrow[idf_k[e0 + 3]]) : 0u;
             }
     }
+    int it = 0;                                           // tile counter, mirrors the producer's
+
+    auto wait_tile = [&]() -> const unsigned char* {
+        const int st = it % kStages;
+        mbar_wait(full + st, (it / kStages) & 1, fail, c.status);
+        return stages + (size_t)st * kStageBytes;
+    };
+    auto release_tile = [&]() {
+        __syncwarp();
+        if (lane == 0) mbar_arrive(empty + (it % kStages));
+        ++it;
+    };
+    // kept dims of one batch of classes: kb[class][token][slot] = sl2 * (q_u . K^mu), 16 tokens per mma.
+    // It needs nothing but q, so the first batch runs before u is known.
+    auto k_phase = [&](int cb, int nb) {
+        if (!ts_k) return;
+#pragma unroll 1
+        for (int ci = 0; ci < nb; ++ci) {
+            const int n_c = n_of_class(cb + ci);
+            float* base = kb + (size_t)ci * S * GH;
+#pragma unroll 1
+            for (int a0 = 0; a0 < n_c; a0 += ts_k) {
+                const int nt = min(ts_k, n_c - a0);
+                const unsigned char* tile = wait_tile();
+#pragma unroll 1
+                for (int grp = warp; grp * 16 < nt; grp += kWarps) {
+                    const unsigned char* r_lo = tile + (size_t)(grp * 16 + gq) * rowb_k;
+                    const unsigned char* r_hi = r_lo + 8 * rowb_k;
+                    float d4[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+                    for (int rd = 0; rd < 2; ++rd) {
+                        const int piece = 4 * rd + tq;
+                        if (4 * rd < npk) {
+                            uint4 lo = make_uint4(0, 0, 0, 0), hi = make_uint4(0, 0, 0, 0);
+                            if (piece < npk) {
+                                lo = *reinterpret_cast<const uint4*>(r_lo + 16 * piece);
+                                hi = *reinterpret_cast<const uint4*>(r_hi + 16 * piece);
+                            }
+                            mma_bf16(d4, lo.x, hi.x, lo.y, hi.y, qk[rd][0][0], qk[rd][0][1]);
+                            mma_bf16(d4, lo.z, hi.z, lo.w, hi.w, qk[rd][1][0], qk[rd][1][1]);
+                        }
+                    }
+                    if (2 * tq < GH) {
+                        const int a_lo = a0 + grp * 16 + gq;
+                        *reinterpret_cast<float2*>(base + a_lo * GH + 2 * tq) = make_float2(d4[0] * sl2, d4[1] * sl2);
+                        *reinterpret_cast<float2*>(base + (a_lo + 8) * GH + 2 * tq) = make_float2(d4[2] * sl2, d4[3] * sl2);
+                    }
+                }
+                release_tile();
+            }
+        }
+    };
+    const bool has_classes = !is_win && c0 < c1 && n_of_class(c0) > 0;
+    if (has_classes) k_phase(c0, min(NB, c1 - c0));
     if (p.fused) {
         // this CTA's slice of the coefficient rows of C^V will be wanted at the very end: start it towards L2
         if (s.dcv > 0) {
@@ -573,7 +638,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_fft_kernel(const __grid_co
             const int32_t* idc_k = c.idx_comp_k + (size_t)h * s.dck;
             for (int i = tid; i < GH * s.dck; i += kConsumers) {
                 const int g = i / s.dck, e = i - g * s.dck;
-                qc[i] = g < ng ? __bfloat162float(q[((size_t)b * s.Hq + g_first + g) * s.d + idc_k[e]]) : 0.f;
+                qc[i] = i < kConsumers ? qc_early : (g < ng ? __bfloat162float(q[((size_t)b * s.Hq + g_first + g) * s.d + idc_k[e]]) : 0.f);
             }
             cp_async_wait_all();
             consumer_sync();
@@ -643,18 +708,6 @@ __global__ void __launch_bounds__(kThreads, 1) decode_fft_kernel(const __grid_co
     float m_run[GH], l_acc[GH];                           // per slot
 #pragma unroll
     for (int g = 0; g < GH; ++g) { m_run[g] = kNegBig; l_acc[g] = 0.f; }
-    int it = 0;                                           // tile counter, mirrors the producer's
-
-    auto wait_tile = [&]() -> const unsigned char* {
-        const int st = it % kStages;
-        mbar_wait(full + st, (it / kStages) & 1, fail, c.status);
-        return stages + (size_t)st * kStageBytes;
-    };
-    auto release_tile = [&]() {
-        __syncwarp();
-        if (lane == 0) mbar_arrive(empty + (it % kStages));
-        ++it;
-    };
     // per-slot maximum over per-thread partial maxima, broadcast to every consumer thread
     auto block_max = [&](float (&mx)[GH]) {
 #pragma unroll
@@ -886,6 +939,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_fft_kernel(const __grid_co
         for (int cb = c0; cb < c1; cb += NB) {
             const int nb = min(NB, c1 - cb);
             if (n_of_class(cb) == 0) break;               // classes are filled in order: nothing further on
+            if (cb != c0) k_phase(cb, nb);
 
             // packed Hermitian spectra of the nb classes: X_m = V^A_m + i V^B_m per complex lane,
             // V_m = v_m + conj(v_{S-m}), v_n = (1/2) u~_n e^{i theta n c}.  Pair 0 is bins (0, S/2).
@@ -929,52 +983,6 @@ __global__ void __launch_bounds__(kThreads, 1) decode_fft_kernel(const __grid_co
                 consumer_sync();
             }
 
-            // kept dims: s = sl2 * (q_u . K^mu) + compressed part, 16 tokens per mma
-            if (ts_k) {
-                #pragma unroll 1
-                for (int ci = 0; ci < nb; ++ci) {
-                    const int n_c = n_of_class(cb + ci);
-                    float* base = fbuf + ci * fb_floats;
-                    #pragma unroll 1
-                    for (int a0 = 0; a0 < n_c; a0 += ts_k) {
-                        const int nt = min(ts_k, n_c - a0);
-                        const unsigned char* tile = wait_tile();
-                        #pragma unroll 1
-                        for (int grp = warp; grp * 16 < nt; grp += kWarps) {
-                            const unsigned char* r_lo = tile + (size_t)(grp * 16 + gq) * rowb_k;
-                            const unsigned char* r_hi = r_lo + 8 * rowb_k;
-                            float d4[4] = {0.f, 0.f, 0.f, 0.f};
-#pragma unroll
-                            for (int rd = 0; rd < 2; ++rd) {
-                                const int piece = 4 * rd + tq;
-                                if (4 * rd < npk) {
-                                    uint4 lo = make_uint4(0, 0, 0, 0), hi = make_uint4(0, 0, 0, 0);
-                                    if (piece < npk) {
-                                        lo = *reinterpret_cast<const uint4*>(r_lo + 16 * piece);
-                                        hi = *reinterpret_cast<const uint4*>(r_hi + 16 * piece);
-                                    }
-                                    mma_bf16(d4, lo.x, hi.x, lo.y, hi.y, qk[rd][0][0], qk[rd][0][1]);
-                                    mma_bf16(d4, lo.z, hi.z, lo.w, hi.w, qk[rd][1][0], qk[rd][1][1]);
-                                }
-                            }
-                            if (2 * tq < GH) {
-                                const int a_lo = a0 + grp * 16 + gq, a_hi = a_lo + 8;
-                                if (a_lo < n_c) {
-                                    float2* dst = reinterpret_cast<float2*>(base + pf(rev[a_lo] * GH + 2 * tq));
-                                    const float2 v = *dst;
-                                    *dst = make_float2(fmaf(d4[0], sl2, v.x), fmaf(d4[1], sl2, v.y));
-                                }
-                                if (a_hi < n_c) {
-                                    float2* dst = reinterpret_cast<float2*>(base + pf(rev[a_hi] * GH + 2 * tq));
-                                    const float2 v = *dst;
-                                    *dst = make_float2(fmaf(d4[2], sl2, v.x), fmaf(d4[3], sl2, v.y));
-                                }
-                            }
-                        }
-                        release_tile();
-                    }
-                }
-            }
             consumer_sync();
 
             // online softmax over the batch
@@ -985,8 +993,16 @@ __global__ void __launch_bounds__(kThreads, 1) decode_fft_kernel(const __grid_co
             for (int i = tid; i < (nb << LS); i += kConsumers) {
                 const int ci = i >> LS, a = i & (S - 1);
                 if (a < n_of_class(cb + ci)) {
-                    float v[GH];
-                    load_vals(fbuf + ci * fb_floats + pf(rev[a] * GH), v);
+                    // score = compressed part (transform output) + kept part
+                    float* pt = fbuf + ci * fb_floats + pf(rev[a] * GH);
+                    float v[GH], kv[GH];
+                    load_vals(pt, v);
+                    if (ts_k) {
+                        load_vals(kb + (size_t)i * GH, kv);
+#pragma unroll
+                        for (int g = 0; g < GH; ++g) v[g] += kv[g];
+                        store_vals(pt, v);
+                    }
 #pragma unroll
                     for (int g = 0; g < GH; ++g) mx[g] = fmaxf(mx[g], v[g]);
                 }
@@ -1225,18 +1241,20 @@ __global__ void __launch_bounds__(kThreads, 1) decode_fft_kernel(const __grid_co
     }
     cp_async_wait_all();
     consumer_sync();
-    if (tid < GH) {
+    if (warp < GH) {                                       // one warp per head, lanes over the parts
         float mx = kNegBig;
 #pragma unroll 1
-        for (int sp = 0; sp < np; ++sp) mx = fmaxf(mx, al_s[tid * np + sp]);
+        for (int sp = lane; sp < np; sp += 32) mx = fmaxf(mx, al_s[warp * np + sp]);
+        mx = warp_max(mx);
         float Lsum = 0.f;
 #pragma unroll 1
-        for (int sp = 0; sp < np; ++sp) {
-            const float a = ex2(al_s[tid * np + sp] - mx);
-            al_s[tid * np + sp] = a;
-            Lsum = fmaf(a, l_s[tid * np + sp], Lsum);
+        for (int sp = lane; sp < np; sp += 32) {
+            const float a = ex2(al_s[warp * np + sp] - mx);
+            al_s[warp * np + sp] = a;
+            Lsum = fmaf(a, l_s[warp * np + sp], Lsum);
         }
-        linv_s[tid] = Lsum > 0.f ? __fdividef(1.0f, Lsum) : 0.f;
+        Lsum = warp_sum(Lsum);
+        if (lane == 0) linv_s[warp] = Lsum > 0.f ? __fdividef(1.0f, Lsum) : 0.f;
     }
     consumer_sync();
     if (s.dcv > 0) {
@@ -1246,7 +1264,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_fft_kernel(const __grid_co
             float v = 0.f;
             if (g < ng) {
                 const float* z = zs_s + g * np * rows_max + r;
-#pragma unroll 1
+#pragma unroll 6
                 for (int sp = 0; sp < np; ++sp) v = fmaf(al_s[g * np + sp], z[sp * rows_max], v);
                 v *= recon_weight(s.norm, m0 + r, s.k, s.T);
             }
@@ -1258,7 +1276,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_fft_kernel(const __grid_co
             float4 acc4[GH];
 #pragma unroll
             for (int g = 0; g < GH; ++g) acc4[g] = make_float4(0.f, 0.f, 0.f, 0.f);
-#pragma unroll 1
+#pragma unroll 3
             for (int r = rgi; r < rows; r += nrg) {
                 const float4 x = *reinterpret_cast<const float4*>(cv_s + r * s.dcv + 4 * v);
 #pragma unroll
@@ -1284,10 +1302,10 @@ __global__ void __launch_bounds__(kThreads, 1) decode_fft_kernel(const __grid_co
         }
     }
     // ticket: the last part to get here finishes the rows
-    __threadfence();
     consumer_sync();
     if (tid == 0) {
         int old;
+        __threadfence();
         asm volatile("atom.acq_rel.gpu.global.add.s32 %0, [%1], 1;" : "=r"(old) : "l"(bar + 2) : "memory");
         *last_s = old == np - 1;
     }
@@ -1318,13 +1336,13 @@ __global__ void __launch_bounds__(kThreads, 1) decode_fft_kernel(const __grid_co
         const int g = t / s.d, e = t - g * s.d;
         const float* o = op_s + g * np * s.d + e;
         float v = 0.f;
-#pragma unroll 1
+#pragma unroll 6
         for (int sp = 0; sp < np; ++sp) v = fmaf(al_s[g * np + sp], o[sp * s.d], v);
         const int slot = inv_s[e];
         if (slot >= 0) {
             const float* oc = ocp_s + g * np * s.dcv + slot;
             float w = 0.f;
-#pragma unroll 1
+#pragma unroll 6
             for (int x = 0; x < np; ++x) w += oc[x * s.dcv];
             v += w;
         }
