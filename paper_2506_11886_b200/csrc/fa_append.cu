@@ -22,6 +22,10 @@ __global__ void __launch_bounds__(256) append_kernel(Dims s, CacheDev c, const K
     __shared__ float f_s[kAppendRows];   // basis column j for the rows of this CTA
     __shared__ int last_s;
     const int h = blockIdx.y, b = blockIdx.z, tid = threadIdx.x;
+    // programmatic dependent launch: the next kernel may be scheduled now; this one first waits for
+    // everything its predecessor in the stream wrote
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     const int n_init = c.state[kStateStride * b + 0], n_local = c.state[kStateStride * b + 1];
     const int n_mid = c.state[kStateStride * b + 2], head = c.state[kStateStride * b + 3];
     const bool to_init = n_init < s.l_init;
@@ -142,9 +146,16 @@ static cudaError_t launch_append_t(const Dims& s, const CacheDev& c, const void*
     const int max_comp = s.dck > s.dcv ? s.dck : s.dcv;
     const int rows = max_comp > 128 ? kAppendRows / 2 : kAppendRows;     // rows * max_comp / 4 <= 256 * kAppendVec
     const int tiles = (s.M + rows - 1) / rows;
-    append_kernel<KV><<<dim3(tiles, s.Hkv, s.B), 256, 0, st>>>(s, c, static_cast<const KV*>(k_new),
-                                                               static_cast<const KV*>(v_new), rows);
-    return cudaGetLastError();
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(tiles, s.Hkv, s.B);
+    cfg.blockDim = dim3(256);
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, append_kernel<KV>, s, c, static_cast<const KV*>(k_new), static_cast<const KV*>(v_new), rows);
 }
 
 cudaError_t launch_append(const Dims& s, const CacheDev& c, int dtype, const void* k_new, const void* v_new,

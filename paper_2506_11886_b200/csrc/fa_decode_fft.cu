@@ -417,6 +417,32 @@ __global__ void __launch_bounds__(kThreads, 1) decode_fft_kernel(const __grid_co
     const int tid = threadIdx.x;
     const int log2P = 31 - __clz(s.P);
 
+    // ---- one-time set-up, independent of the cache: it may overlap the tail of the previous kernel ----
+    if (tid < kConsumers) {
+        #pragma unroll 1
+        for (int i = tid; i < s.k; i += kConsumers) {
+            E[i] = cis_frac((float)i / (float)s.T);
+        }
+        for (int l = LS; l > 0;) {
+            const int rl = radix_log2(l), R = 1 << rl, st = 1 << (l - rl);
+            if (l > rl) {
+                const int off = tw_offset(LS, l);
+                #pragma unroll 1
+                for (int i = tid; i < (R - 1) * st; i += kConsumers) {
+                    const int qm1 = i / st, j = i - qm1 * st;
+                    reinterpret_cast<float2*>(twf)[off + i] = cis_frac((float)(((qm1 + 1) * j) & ((1 << l) - 1)) / (float)(1 << l));
+                }
+            }
+            l -= rl;
+        }
+        #pragma unroll 1
+        for (int a = tid; a < S; a += kConsumers) rev[a] = (uint16_t)dif_pos<LS>(a);
+        if (tid < GH + 8) red_s[kWarps * GH + tid] = 0.f;
+
+    }
+    // fused kernel: everything below reads what earlier kernels in the stream wrote (state, cache, q)
+    if (p.fused) asm volatile("griddepcontrol.wait;" ::: "memory");
+
     const int n_init = c.state[kStateStride * b + 0], n_local = c.state[kStateStride * b + 1];
     const int n_mid = min(c.state[kStateStride * b + 2], s.max_mid), head = c.state[kStateStride * b + 3];
     const int c0 = is_win ? 0 : part * s.P / p.n_split;
@@ -530,27 +556,6 @@ __global__ void __launch_bounds__(kThreads, 1) decode_fft_kernel(const __grid_co
 #pragma unroll 1
         for (int i = tid; i < (m1 - m0) * (s.dck >> 2); i += kConsumers) cp_async16(fbuf + 4 * i, ck + 4 * i);
     }
-
-    // ---- one-time set-up ----
-    #pragma unroll 1
-    for (int i = tid; i < s.k; i += kConsumers) {
-        E[i] = cis_frac((float)i / (float)s.T);
-    }
-    for (int l = LS; l > 0;) {
-        const int rl = radix_log2(l), R = 1 << rl, st = 1 << (l - rl);
-        if (l > rl) {
-            const int off = tw_offset(LS, l);
-            #pragma unroll 1
-            for (int i = tid; i < (R - 1) * st; i += kConsumers) {
-                const int qm1 = i / st, j = i - qm1 * st;
-                reinterpret_cast<float2*>(twf)[off + i] = cis_frac((float)(((qm1 + 1) * j) & ((1 << l) - 1)) / (float)(1 << l));
-            }
-        }
-        l -= rl;
-    }
-    #pragma unroll 1
-    for (int a = tid; a < S; a += kConsumers) rev[a] = (uint16_t)dif_pos<LS>(a);
-    if (tid < GH + 8) red_s[kWarps * GH + tid] = 0.f;
 
     // B fragments of q for the kept K dims: column gq is slot gq = head hperm(gq);
     // round rd covers pieces 4 rd + tq of a row, two k-steps each
@@ -1368,16 +1373,36 @@ cudaError_t launch_fft_t(const Dims& s, const CacheDev& c, const DecodePlan& p, 
     cfg.blockDim = dim3(kThreads);
     cfg.dynamicSmemBytes = (size_t)L.total;
     cfg.stream = st;
-    cudaLaunchAttribute attr[1];
-    if (p.fused) {
-        attr[0].id = cudaLaunchAttributeCooperative;                      // its CTAs wait for one another
-        attr[0].val.cooperative = 1;
-    } else {
-        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;  // may start while the prologue kernel runs
-        attr[0].val.programmaticStreamSerializationAllowed = 1;
-    }
+    // Programmatic dependent launch: the kernel may be scheduled while its predecessor in the stream
+    // still runs and waits (griddepcontrol.wait) where it first reads what the predecessor wrote.  The
+    // fused kernel is also a cooperative launch (its CTAs wait for one another); whether the driver
+    // takes both attributes together is found out on the first launch outside a stream capture.
+    static int coop_pdl_ok = -1;
+    cudaLaunchAttribute attr[2];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    attr[1].id = cudaLaunchAttributeCooperative;
+    attr[1].val.cooperative = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
+    if (p.fused) {
+        cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+        if (coop_pdl_ok < 0 && (cudaStreamIsCapturing(st, &cap) != cudaSuccess || cap != cudaStreamCaptureStatusNone)) {
+            cfg.attrs = attr + 1;                                          // not probed yet: stay on the plain cooperative launch
+        } else if (coop_pdl_ok != 0) {
+            cfg.numAttrs = 2;
+            cudaError_t err2 = cudaLaunchKernelEx(&cfg, decode_fft_kernel<GH, LS>, tki, tvi, tkl, tvl, s, c, p,
+                                                  static_cast<const bf16*>(q), static_cast<bf16*>(out), ws);
+            if (err2 == cudaSuccess) { coop_pdl_ok = 1; return err2; }
+            if (coop_pdl_ok == 1) return err2;
+            cudaGetLastError();
+            coop_pdl_ok = 0;
+            cfg.attrs = attr + 1;
+            cfg.numAttrs = 1;
+        } else {
+            cfg.attrs = attr + 1;
+        }
+    }
     return cudaLaunchKernelEx(&cfg, decode_fft_kernel<GH, LS>, tki, tvi, tkl, tvl, s, c, p, static_cast<const bf16*>(q),
                               static_cast<bf16*>(out), ws);
 }
