@@ -128,6 +128,20 @@ __device__ __forceinline__ void ldmatrix_x4_trans(uint32_t (&r)[4], uint32_t add
                  : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
                  : "r"(addr));
 }
+// shared-memory accesses by 32-bit address (no generic-pointer arithmetic in the inner loops)
+__device__ __forceinline__ uint4 lds128(uint32_t a) {
+    uint4 v;
+    asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(a) : "memory");
+    return v;
+}
+__device__ __forceinline__ uint32_t lds32(uint32_t a) {
+    uint32_t v;
+    asm volatile("ld.shared.u32 %0, [%1];" : "=r"(v) : "r"(a) : "memory");
+    return v;
+}
+__device__ __forceinline__ void sts64(uint32_t a, float x, float y) {
+    asm volatile("st.shared.v2.f32 [%0], {%1,%2};" ::"r"(a), "f"(x), "f"(y) : "memory");
+}
 __device__ __forceinline__ uint32_t pack_bf16(bf16 lo, bf16 hi) {
     return (uint32_t)__bfloat16_as_ushort(lo) | ((uint32_t)__bfloat16_as_ushort(hi) << 16);
 }
@@ -582,6 +596,12 @@ __global__ void __launch_bounds__(kThreads, 1) decode_fft_kernel(const __grid_co
         mbar_wait(full + st, (it / kStages) & 1, fail, c.status);
         return stages + (size_t)st * kStageBytes;
     };
+    const uint32_t stages_u = smem_addr(stages), zero_u = smem_addr(zero16);
+    auto wait_tile_u = [&]() -> uint32_t {                // the same, as a shared-memory address
+        const int st = it % kStages;
+        mbar_wait(full + st, (it / kStages) & 1, fail, c.status);
+        return stages_u + (uint32_t)st * kStageBytes;
+    };
     auto release_tile = [&]() {
         __syncwarp();
         if (lane == 0) mbar_arrive(empty + (it % kStages));
@@ -589,38 +609,44 @@ __global__ void __launch_bounds__(kThreads, 1) decode_fft_kernel(const __grid_co
     };
     // kept dims of one batch of classes: kb[class][token][slot] = sl2 * (q_u . K^mu), 16 tokens per mma.
     // It needs nothing but q, so the first batch runs before u is known.
+    // per-lane constants of the K loop: byte offsets of the two 16-byte pieces inside a 16-row group
+    uint32_t k_off[2];
+    bool k_on[2];
+#pragma unroll
+    for (int rd = 0; rd < 2; ++rd) {
+        k_off[rd] = (uint32_t)(gq * rowb_k + 16 * (4 * rd + tq));
+        k_on[rd] = 4 * rd + tq < npk;
+    }
+    const uint32_t kb_lane = smem_addr(kb) + (uint32_t)(gq * GH + 2 * tq) * 4;
     auto k_phase = [&](int cb, int nb) {
         if (!ts_k) return;
 #pragma unroll 1
         for (int ci = 0; ci < nb; ++ci) {
             const int n_c = n_of_class(cb + ci);
-            float* base = kb + (size_t)ci * S * GH;
 #pragma unroll 1
             for (int a0 = 0; a0 < n_c; a0 += ts_k) {
                 const int nt = min(ts_k, n_c - a0);
-                const unsigned char* tile = wait_tile();
+                const uint32_t tile = wait_tile_u();
 #pragma unroll 1
                 for (int grp = warp; grp * 16 < nt; grp += kWarps) {
-                    const unsigned char* r_lo = tile + (size_t)(grp * 16 + gq) * rowb_k;
-                    const unsigned char* r_hi = r_lo + 8 * rowb_k;
+                    const uint32_t gbase = tile + (uint32_t)(grp * 16) * rowb_k;
                     float d4[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
                     for (int rd = 0; rd < 2; ++rd) {
-                        const int piece = 4 * rd + tq;
                         if (4 * rd < npk) {
                             uint4 lo = make_uint4(0, 0, 0, 0), hi = make_uint4(0, 0, 0, 0);
-                            if (piece < npk) {
-                                lo = *reinterpret_cast<const uint4*>(r_lo + 16 * piece);
-                                hi = *reinterpret_cast<const uint4*>(r_hi + 16 * piece);
+                            if (k_on[rd]) {
+                                lo = lds128(gbase + k_off[rd]);
+                                hi = lds128(gbase + k_off[rd] + 8 * rowb_k);
                             }
                             mma_bf16(d4, lo.x, hi.x, lo.y, hi.y, qk[rd][0][0], qk[rd][0][1]);
                             mma_bf16(d4, lo.z, hi.z, lo.w, hi.w, qk[rd][1][0], qk[rd][1][1]);
                         }
                     }
                     if (2 * tq < GH) {
-                        const int a_lo = a0 + grp * 16 + gq;
-                        *reinterpret_cast<float2*>(base + a_lo * GH + 2 * tq) = make_float2(d4[0] * sl2, d4[1] * sl2);
-                        *reinterpret_cast<float2*>(base + (a_lo + 8) * GH + 2 * tq) = make_float2(d4[2] * sl2, d4[3] * sl2);
+                        const uint32_t dst = kb_lane + (uint32_t)((ci * S + a0 + grp * 16) * GH) * 4;
+                        sts64(dst, d4[0] * sl2, d4[1] * sl2);
+                        sts64(dst + 8 * GH * 4, d4[2] * sl2, d4[3] * sl2);
                     }
                 }
                 release_tile();
@@ -628,7 +654,8 @@ __global__ void __launch_bounds__(kThreads, 1) decode_fft_kernel(const __grid_co
         }
     };
     const bool has_classes = !is_win && c0 < c1 && n_of_class(c0) > 0;
-    if (has_classes) k_phase(c0, min(NB, c1 - c0));
+    // Fused kernel: this part's rows of u first, then the kept-dim scores of the first batch (they need
+    // only q) while the other parts finish theirs, then the wait for all of u.
     if (p.fused) {
         // this CTA's slice of the coefficient rows of C^V will be wanted at the very end: start it towards L2
         if (s.dcv > 0) {
@@ -679,9 +706,11 @@ __global__ void __launch_bounds__(kThreads, 1) decode_fft_kernel(const __grid_co
                     ws.u[((size_t)b * s.Hq + g_first + l8) * s.M + r] = recon_weight(s.norm, r, s.k, s.T) * sl2 * mine;
             }
             part_arrive(bar + 0, tid);
-            if (!is_win) part_wait(bar + 0, p.n_part, tid, fail, c.status);
         }
+        if (has_classes) k_phase(c0, min(NB, c1 - c0));
+        if (s.dck > 0 && !is_win) part_wait(bar + 0, p.n_part, tid, fail, c.status);
     } else {
+        if (has_classes) k_phase(c0, min(NB, c1 - c0));
         // everything above is independent of the prologue kernel; its output u is first needed here
         asm volatile("griddepcontrol.wait;" ::: "memory");
     }
@@ -939,6 +968,20 @@ __global__ void __launch_bounds__(kThreads, 1) decode_fft_kernel(const __grid_co
 #pragma unroll
             for (int i = 0; i < 4; ++i) acc[mt][i] = 0.f;
         const int nmt = (s.nfv + 15) >> 4;
+        // per-lane constants of the V loop.  A group of 16 tokens starts at a multiple of 16, so the
+        // chunk swizzle of a lane's row depends on the lane alone: the byte offset of its 8x8 matrix
+        // row inside the group is fixed.  A chunk past the end of the row reads the zero block.
+        uint32_t v_off[4], v_mul[4];
+        {
+            const int mi = lane >> 3, tok = ((mi >> 1) << 3) + (lane & 7), sw = v_swz(tok, nchv);
+#pragma unroll
+            for (int mt = 0; mt < 4; ++mt) {
+                const int chunk = 2 * mt + (mi & 1);
+                v_mul[mt] = chunk < nchv ? 1u : 0u;
+                v_off[mt] = chunk < nchv ? (uint32_t)(tok * rowb_v + 16 * (chunk ^ sw)) : zero_u;
+            }
+        }
+        const uint32_t p_lane = smem_addr(pbt) + (uint32_t)((gq & (GH - 1)) * pbs + 2 * tq) * 2;
 
         #pragma unroll 1
         for (int cb = c0; cb < c1; cb += NB) {
@@ -1054,29 +1097,24 @@ __global__ void __launch_bounds__(kThreads, 1) decode_fft_kernel(const __grid_co
                 #pragma unroll 1
                 for (int ci = 0; ci < nb; ++ci) {
                     const int n_c = n_of_class(cb + ci);
-                    const bf16* prow = pbt + (size_t)(ci * GH + (gq & (GH - 1))) * pbs;
+                    const uint32_t prow = p_lane + (uint32_t)(ci * GH * pbs) * 2;
                     #pragma unroll 1
                     for (int a0 = 0; a0 < n_c; a0 += ts_v) {
                         const int nt = min(ts_v, n_c - a0);
-                        const unsigned char* tile = wait_tile();
+                        const uint32_t tile = wait_tile_u();
                         #pragma unroll 1
                         for (int grp = warp; grp * 16 < nt; grp += kWarps) {
-                            const int a = a0 + grp * 16;
+                            const uint32_t gbase = tile + (uint32_t)(grp * 16) * rowb_v;
                             uint32_t b0 = 0, b1 = 0;
                             if (gq < GH) {
-                                b0 = *reinterpret_cast<const uint32_t*>(prow + a + 2 * tq);
-                                b1 = *reinterpret_cast<const uint32_t*>(prow + a + 2 * tq + 8);
+                                b0 = lds32(prow + (uint32_t)(a0 + grp * 16) * 2);
+                                b1 = lds32(prow + (uint32_t)(a0 + grp * 16 + 8) * 2);
                             }
-                            const int mi = lane >> 3, tok = ((mi >> 1) << 3) + (lane & 7);
-                            const unsigned char* vrow = tile + (size_t)(grp * 16 + tok) * rowb_v;
-                            const int sw = v_swz(a + tok, nchv);
 #pragma unroll
                             for (int mt = 0; mt < 4; ++mt) {
                                 if (mt < nmt) {
-                                    const int chunk = 2 * mt + (mi & 1);
-                                    const unsigned char* src = chunk < nchv ? vrow + 16 * (chunk ^ sw) : zero16;
                                     uint32_t af[4];
-                                    ldmatrix_x4_trans(af, smem_addr(src));
+                                    ldmatrix_x4_trans(af, v_off[mt] + gbase * v_mul[mt]);
                                     mma_bf16(acc[mt], af[0], af[1], af[2], af[3], b0, b1);
                                 }
                             }
