@@ -30,7 +30,7 @@
 namespace fa {
 namespace {
 
-constexpr int kConsumers = 512;
+constexpr int kConsumers = 256;
 constexpr int kWarps = kConsumers / 32;
 constexpr int kThreads = kConsumers + 32;
 constexpr int kStageBytes = 16384;
