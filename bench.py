@@ -38,7 +38,7 @@ UNIT = "us/step"
 SEED = 1000          # 1000 * config index
 # dram__bytes_read.sum + dram__bytes_write.sum per fa_decode_attention call from the committed
 # ncu capture (profiles/); None until a capture of the current kernels has been summarised.
-NCU_TRAFFIC_BYTES_PER_CALL = 50543360   # profiles/decode_append_compress_cfg1_counters.md: 3.19 + 39.43 + 7.92 MB
+NCU_TRAFFIC_BYTES_PER_CALL = 43270144   # profiles/decode_append_compress_cfg1_counters.md: decode_fft_kernel, 43254528 read + 15616 written
 
 
 def _peaks():
@@ -302,7 +302,7 @@ def run_ours(args):
                       "append_gbs": by["append"] / (us_append * 1e-6) / 1e9,
                       "compress_ms_per_layer": min(comp_ms), "compress_tflops": comp_flop / (min(comp_ms) * 1e-3) / 1e12,
                       "compress_path": "tcgen05 bf16 x bf16 -> f32 (TMEM), basis tile generated in registers"},
-        "roofline": {"kernel": "fa_decode_attention (prologue + main + epilogue kernels)", "bound": "hbm",
+        "roofline": {"kernel": "fa_decode_attention (one fused cooperative kernel: u, token loop, merge)", "bound": "hbm",
                      "achieved": dec_gbs, "peak": peak, "unit": "GB/s", "frac": dec_gbs / peak, "peak_kind": peak_kind,
                      "algorithmic_bytes": by["decode"], "traffic": NCU_TRAFFIC_BYTES_PER_CALL,
                      "frac_of_8tbs_nominal": dec_gbs / 8000.0},

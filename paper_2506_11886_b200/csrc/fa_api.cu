@@ -380,7 +380,11 @@ int fa_launch_count(const fa_layout* layout, int what) {
     switch (what) {
         case 0: return 2;   // partition/gather + coefficient kernel (memsets not counted)
         case 1: return 1;
-        case 2: return 3;   // prologue, main, epilogue
+        case 2: {           // one fused kernel, or prologue + main + epilogue
+            DecodePlan p;
+            if (plan_decode(*layout, &p) != FA_OK) return 0;
+            return p.fused ? 1 : 3;
+        }
         default: return 0;
     }
 }
