@@ -159,9 +159,22 @@ fa_status fa_append(const fa_layout* layout, fa_cache* cache, const void* k_new,
 fa_status fa_decode_attention(const fa_layout* layout, const fa_cache* cache, const void* q, void* out,
                               void* ws, size_t ws_bytes, void* stream);
 
+/* One decode step with device inputs (Eq.5 then Eq.6): the result and the cache afterwards are those
+ * of fa_append(k_new, v_new) followed by fa_decode_attention(q).  Where the decode call is a single
+ * fused kernel (see fa_decode_algo) and the KV head's query heads fit one pass, the coefficient
+ * update of Eq.5 rides on that kernel: a one-CTA-per-batch-row kernel moves the row that leaves the
+ * local window, stores the new token and advances the counters, and the decode kernel adds
+ * f_j x^T to each coefficient row as it streams it (C^K before forming u, C^V before the output
+ * product) and writes it back, so the coefficients cross the memory bus once per step instead of
+ * twice.  Otherwise the two calls are made one after the other.  Same arguments, workspace rule and
+ * errors as those two calls (a full middle sets FA_ERR_CAPACITY in cache->status and the step decodes
+ * the unchanged cache). */
+fa_status fa_decode_step(const fa_layout* layout, fa_cache* cache, const void* q, const void* k_new,
+                         const void* v_new, void* out, void* ws, size_t ws_bytes, void* stream);
+
 /* One decode step with HOST inputs and outputs (Eq.5 then Eq.6): copies q [B][H_q][d] and
  * k_new, v_new [B][H_kv][d] from host memory (pinned for the copies to be asynchronous) into
- * `staging`, runs fa_append and fa_decode_attention, and copies the result to out_host
+ * `staging`, runs fa_decode_step, and copies the result to out_host
  * [B][H_q][d].  `staging` is caller-owned device memory of at least
  * fa_step_staging_bytes(layout) bytes; k_new_host == NULL skips the append.  Asynchronous on
  * `stream`: out_host is valid after the stream is synchronised. */
@@ -193,7 +206,7 @@ size_t fa_static_workspace_limit(void);
 fa_status fa_poll_status(const fa_cache* cache, void* stream);
 
 /* Number of kernels one call launches for this layout (what = 0 compress, 1 append,
- * 2 decode); for launch accounting by callers. */
+ * 2 decode, 3 decode step); for launch accounting by callers. */
 int fa_launch_count(const fa_layout* layout, int what);
 
 const char* fa_status_string(fa_status s);

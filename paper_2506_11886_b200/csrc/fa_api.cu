@@ -175,6 +175,8 @@ fa_status plan_decode(const fa_layout& l, DecodePlan* p) {
     p->off_oc = off;  off = align_up(off + sizeof(float) * (size_t)s.B * s.Hq * n_oc * (s.dcv > 0 ? s.dcv : 1), 256);
     p->off_om = off;  off = align_up(off + sizeof(float) * (size_t)s.B * s.Hq * s.d, 256);
     p->off_cnt = off; off = align_up(off + sizeof(int32_t) * (size_t)s.B * s.Hkv, 256);
+    p->off_pend = off; off = align_up(off + sizeof(float) * (size_t)s.B * s.Hkv * (s.dck + s.dcv + 4), 256);
+    p->off_pendj = off; off = align_up(off + sizeof(int32_t) * (size_t)s.B, 256);
     p->total = off;
     return FA_OK;
 }
@@ -327,16 +329,43 @@ fa_status fa_decode_attention(const fa_layout* layout, const fa_cache* cache, co
     cudaStream_t cs = static_cast<cudaStream_t>(stream);
     char* w = static_cast<char*>(ws);
     if (p.fused) {
-        if (launch_decode_fft(s, c, layout->kv_dtype, p, q, out, w, cs) != cudaSuccess) return FA_ERR_CUDA;
+        if (launch_decode_fft(s, c, layout->kv_dtype, p, q, out, w, false, cs) != cudaSuccess) return FA_ERR_CUDA;
         return FA_OK;
     }
     if (launch_decode_prologue(s, c, layout->kv_dtype, p, q, w, cs) != cudaSuccess) return FA_ERR_CUDA;
     if (p.algo == FA_DECODE_FFT) {
-        if (launch_decode_fft(s, c, layout->kv_dtype, p, q, out, w, cs) != cudaSuccess) return FA_ERR_CUDA;
+        if (launch_decode_fft(s, c, layout->kv_dtype, p, q, out, w, false, cs) != cudaSuccess) return FA_ERR_CUDA;
     } else {
         if (launch_decode_direct(s, c, layout->kv_dtype, p, q, w, cs) != cudaSuccess) return FA_ERR_CUDA;
     }
     if (launch_decode_epilogue(s, c, layout->kv_dtype, p, out, w, cs) != cudaSuccess) return FA_ERR_CUDA;
+    return FA_OK;
+}
+
+fa_status fa_decode_step(const fa_layout* layout, fa_cache* cache, const void* q, const void* k_new, const void* v_new,
+                         void* out, void* ws, size_t ws_bytes, void* stream) {
+    fa_status st = check_layout(layout);
+    if (st != FA_OK) return st;
+    st = check_cache(layout, cache);
+    if (st != FA_OK) return st;
+    if (!q || !out || !aligned16(q) || !aligned16(out)) return FA_ERR_INVALID_ARG;
+    if (!k_new || !v_new || !aligned16(k_new) || !aligned16(v_new)) return FA_ERR_INVALID_ARG;
+    DecodePlan p;
+    st = plan_decode(*layout, &p);
+    if (st != FA_OK) return st;
+    if (!ws || !aligned16(ws) || ws_bytes < p.total) return FA_ERR_WORKSPACE;
+    if (!(p.fused && p.n_pass == 1)) {
+        // two calls: the coefficient update cannot ride on the decode kernel's passes over the rows
+        st = fa_append(layout, cache, k_new, v_new, stream);
+        if (st != FA_OK) return st;
+        return fa_decode_attention(layout, cache, q, out, ws, ws_bytes, stream);
+    }
+    Dims s = make_dims(*layout);
+    CacheDev c = make_cache(*cache);
+    cudaStream_t cs = static_cast<cudaStream_t>(stream);
+    char* w = static_cast<char*>(ws);
+    if (launch_append_lite(s, c, layout->kv_dtype, p, k_new, v_new, w, cs) != cudaSuccess) return FA_ERR_CUDA;
+    if (launch_decode_fft(s, c, layout->kv_dtype, p, q, out, w, true, cs) != cudaSuccess) return FA_ERR_CUDA;
     return FA_OK;
 }
 
@@ -366,10 +395,10 @@ fa_status fa_decode_step_host(const fa_layout* layout, fa_cache* cache, const vo
     if (k_new_host) {
         if (cudaMemcpyAsync(k_d, k_new_host, k_bytes, cudaMemcpyHostToDevice, cs) != cudaSuccess) return FA_ERR_CUDA;
         if (cudaMemcpyAsync(v_d, v_new_host, k_bytes, cudaMemcpyHostToDevice, cs) != cudaSuccess) return FA_ERR_CUDA;
-        st = fa_append(layout, cache, k_d, v_d, stream);
-        if (st != FA_OK) return st;
+        st = fa_decode_step(layout, cache, q_d, k_d, v_d, o_d, ws, ws_bytes, stream);
+    } else {
+        st = fa_decode_attention(layout, cache, q_d, o_d, ws, ws_bytes, stream);
     }
-    st = fa_decode_attention(layout, cache, q_d, o_d, ws, ws_bytes, stream);
     if (st != FA_OK) return st;
     if (cudaMemcpyAsync(out_host, o_d, q_bytes, cudaMemcpyDeviceToHost, cs) != cudaSuccess) return FA_ERR_CUDA;
     return FA_OK;
@@ -384,6 +413,11 @@ int fa_launch_count(const fa_layout* layout, int what) {
             DecodePlan p;
             if (plan_decode(*layout, &p) != FA_OK) return 0;
             return p.fused ? 1 : 3;
+        }
+        case 3: {           // fa_decode_step: light append + fused decode, or fa_append + fa_decode_attention
+            DecodePlan p;
+            if (plan_decode(*layout, &p) != FA_OK) return 0;
+            return (p.fused && p.n_pass == 1) ? 2 : 1 + (p.fused ? 1 : 3);
         }
         default: return 0;
     }

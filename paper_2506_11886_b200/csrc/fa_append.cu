@@ -8,6 +8,7 @@
 //   waiting) overwrites the ring slot with the new token and advances the
 //   counters, so no CTA can see a half-updated state.
 #include "fa_common.cuh"
+#include "fa_decode_ws.cuh"
 
 namespace fa {
 
@@ -140,6 +141,83 @@ __global__ void __launch_bounds__(256) append_kernel(Dims s, CacheDev c, const K
     }
 }
 
+// First half of a fused decode step (Eq.5 without the coefficient update): one CTA per batch row moves
+// the row that leaves the local window (kept dims to K^mu / V^mu), stores the new token and advances
+// the counters, and leaves the compressed dims of the leaving row with its basis column j in the
+// workspace.  The decode kernel of the same step adds f_j x^T to the coefficient rows as it streams
+// them, so the coefficients are read and written once per step instead of twice.
+template <typename KV>
+__global__ void __launch_bounds__(256) append_lite_kernel(Dims s, CacheDev c, DecodePlan p, const KV* __restrict__ k_new,
+                                                          const KV* __restrict__ v_new, char* wsp) {
+    __shared__ float x_s[2][256];        // the row that leaves, both sides, natural dim order
+    const int b = blockIdx.x, tid = threadIdx.x;
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    Ws ws = ws_view(wsp, p);
+    const int n_init = c.state[kStateStride * b + 0], n_local = c.state[kStateStride * b + 1];
+    const int n_mid = c.state[kStateStride * b + 2], head = c.state[kStateStride * b + 3];
+    const bool to_init = n_init < s.l_init;
+    const bool evict = !to_init && n_local == s.l_local;
+    const bool full = evict && (n_mid >= s.max_mid || n_mid >= s.T);
+    if (full) {
+        if (tid == 0) { atomicExch(c.status, (int)FA_ERR_CAPACITY); ws.pend_j[b] = -1; }
+        return;
+    }
+    if (evict) {
+        const int j = n_mid;
+#pragma unroll 1
+        for (int h = 0; h < s.Hkv; ++h) {
+            for (int i = tid; i < 2 * s.d; i += 256) {
+                const int side = i / s.d, e = i - side * s.d;
+                float v;
+                if (s.l_local == 0) v = ld_f((side == 0 ? k_new : v_new) + ((size_t)b * s.Hkv + h) * s.d + e);
+                else v = ld_f(win_row<KV>(side == 0 ? c.k_local : c.v_local, s, b, h, s.l_local, head) + e);
+                x_s[side][e] = v;
+            }
+            __syncthreads();
+            for (int i = tid; i < s.nfk + s.nfv; i += 256) {
+                const int side = i < s.nfk ? 0 : 1;
+                const int e = side == 0 ? i : i - s.nfk;
+                const int nfull = side == 0 ? s.nfk : s.nfv;
+                const int32_t* idf = (side == 0 ? c.idx_full_k : c.idx_full_v) + (size_t)h * nfull;
+                KV* dst = mid_row<KV>(side == 0 ? c.k_mid : c.v_mid, s, b, h, j % s.P, j / s.P, nfull);
+                const int col = side == 1 ? v_mid_col(j / s.P, e, nfull, sizeof(KV) == 2 ? FA_BF16 : FA_F32) : e;
+                st_f(dst + col, x_s[side][idf[e]]);
+            }
+            float* pend = ws.pend + ((size_t)b * s.Hkv + h) * (s.dck + s.dcv);
+            for (int i = tid; i < s.dck + s.dcv; i += 256) {
+                const int side = i < s.dck ? 0 : 1;
+                const int e = side == 0 ? i : i - s.dck;
+                const int32_t* idc = side == 0 ? c.idx_comp_k + (size_t)h * s.dck : c.idx_comp_v + (size_t)h * s.dcv;
+                pend[i] = x_s[side][idc[e]];
+            }
+            __syncthreads();
+        }
+    }
+    // the new token: next init row, or the ring slot behind the newest local row (the slot just vacated when full)
+    for (int i = tid; i < 2 * s.Hkv * s.d; i += 256) {
+        const int side = i / (s.Hkv * s.d);
+        const int rem = i - side * (s.Hkv * s.d);
+        const int hh = rem / s.d, e = rem - hh * s.d;
+        const KV* src = (side == 0 ? k_new : v_new) + ((size_t)b * s.Hkv + hh) * s.d;
+        if (to_init) {
+            win_row<KV>(side == 0 ? c.k_init : c.v_init, s, b, hh, s.l_init, n_init)[e] = src[e];
+        } else if (s.l_local > 0) {
+            const int slot = evict ? head : (head + n_local) % s.l_local;
+            win_row<KV>(side == 0 ? c.k_local : c.v_local, s, b, hh, s.l_local, slot)[e] = src[e];
+        }
+    }
+    __syncthreads();
+    if (tid == 0) {
+        if (to_init) c.state[kStateStride * b + 0] = n_init + 1;
+        else if (evict) {
+            c.state[kStateStride * b + 2] = n_mid + 1;
+            if (s.l_local > 0) c.state[kStateStride * b + 3] = (head + 1) % s.l_local;
+        } else c.state[kStateStride * b + 1] = n_local + 1;
+        ws.pend_j[b] = evict ? n_mid : -1;
+    }
+}
+
 template <typename KV>
 static cudaError_t launch_append_t(const Dims& s, const CacheDev& c, const void* k_new, const void* v_new,
                                    cudaStream_t st) {
@@ -156,6 +234,27 @@ static cudaError_t launch_append_t(const Dims& s, const CacheDev& c, const void*
     cfg.attrs = attr;
     cfg.numAttrs = 1;
     return cudaLaunchKernelEx(&cfg, append_kernel<KV>, s, c, static_cast<const KV*>(k_new), static_cast<const KV*>(v_new), rows);
+}
+
+template <typename KV>
+static cudaError_t launch_append_lite_t(const Dims& s, const CacheDev& c, const DecodePlan& p, const void* k_new, const void* v_new,
+                                        char* ws, cudaStream_t st) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(s.B);
+    cfg.blockDim = dim3(256);
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, append_lite_kernel<KV>, s, c, p, static_cast<const KV*>(k_new), static_cast<const KV*>(v_new), ws);
+}
+
+cudaError_t launch_append_lite(const Dims& s, const CacheDev& c, int dtype, const DecodePlan& p, const void* k_new, const void* v_new,
+                               char* ws, cudaStream_t st) {
+    if (dtype == FA_BF16) return launch_append_lite_t<__nv_bfloat16>(s, c, p, k_new, v_new, ws, st);
+    return launch_append_lite_t<float>(s, c, p, k_new, v_new, ws, st);
 }
 
 cudaError_t launch_append(const Dims& s, const CacheDev& c, int dtype, const void* k_new, const void* v_new,

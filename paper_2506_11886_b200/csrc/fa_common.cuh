@@ -70,7 +70,7 @@ struct DecodePlan {
     int fft_log2;      // log2 of the transform length (FFT path)
     int nb;            // classes transformed together by one CTA (FFT path)
     // workspace offsets in bytes
-    size_t off_bar, off_u, off_ml, off_o, off_z, off_oc, off_om, off_cnt, total;
+    size_t off_bar, off_u, off_ml, off_o, off_z, off_oc, off_om, off_cnt, off_pend, off_pendj, total;
 };
 
 // V^mu of bf16 caches is stored with its 16-byte chunks (8 dims) permuted inside each row:
@@ -107,7 +107,9 @@ cudaError_t launch_decode_prologue(const Dims&, const CacheDev&, int dtype, cons
                                    cudaStream_t);
 cudaError_t launch_decode_direct(const Dims&, const CacheDev&, int dtype, const DecodePlan&, const void* q, char* ws,
                                  cudaStream_t);
-cudaError_t launch_decode_fft(const Dims&, const CacheDev&, int dtype, const DecodePlan&, const void* q, void* out, char* ws,
+cudaError_t launch_append_lite(const Dims&, const CacheDev&, int dtype, const DecodePlan&, const void* k_new, const void* v_new,
+                               char* ws, cudaStream_t);
+cudaError_t launch_decode_fft(const Dims&, const CacheDev&, int dtype, const DecodePlan&, const void* q, void* out, char* ws, bool step,
                               cudaStream_t);
 size_t decode_fft_smem_bytes(const Dims&, int log2S, int gh, int nb);
 bool decode_fft_fused_fits(const Dims&, int log2S, int gh, int nb, int n_part);

@@ -396,7 +396,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_fft_kernel(const __grid_co
                                                                   const __grid_constant__ CUtensorMap tm_kl,
                                                                   const __grid_constant__ CUtensorMap tm_vl, Dims s, CacheDev c,
                                                                   DecodePlan p, const bf16* __restrict__ q, bf16* __restrict__ out,
-                                                                  char* wsp) {
+                                                                  char* wsp, int step) {
     constexpr int N = GH / 2;
     constexpr int S = 1 << LS;
     extern __shared__ __align__(128) unsigned char smem_unaligned[];
@@ -675,6 +675,26 @@ __global__ void __launch_bounds__(kThreads, 1) decode_fft_kernel(const __grid_co
             cp_async_wait_all();
             consumer_sync();
             const int l8 = tid & 7, rgi = tid >> 3, nv = s.dck >> 2;
+            // fused step: the rank-1 update of Eq.5 that the light append kernel left pending, applied to
+            // this part's rows while they are on chip, and written back
+            const int j_pend = step ? ws.pend_j[b] : -1;
+            if (j_pend >= 0) {
+                const float* xk = ws.pend + ((size_t)b * s.Hkv + h) * (s.dck + s.dcv);
+                float* ckg = coef_rows(c.coef_k, s, b, h, s.dck) + (size_t)m0 * s.dck;
+#pragma unroll 1
+                for (int i = tid; i < (m1 - m0) * nv; i += kConsumers) {
+                    const int r = i / nv, v = i - r * nv, m = m0 + r;
+                    float cs, sn;
+                    basis_cs(m >> 1, j_pend, s.T, &cs, &sn);
+                    const float f = (m & 1) ? sn : cs;
+                    float4 x = *reinterpret_cast<const float4*>(fbuf + 4 * i);
+                    const float4 y = __ldcg(reinterpret_cast<const float4*>(xk) + v);
+                    x.x = fmaf(f, y.x, x.x); x.y = fmaf(f, y.y, x.y); x.z = fmaf(f, y.z, x.z); x.w = fmaf(f, y.w, x.w);
+                    *reinterpret_cast<float4*>(fbuf + 4 * i) = x;
+                    *reinterpret_cast<float4*>(ckg + 4 * i) = x;
+                }
+                consumer_sync();
+            }
             #pragma unroll 1
             for (int r0 = m0; r0 < m1; r0 += kConsumers / 8) {
                 const int r = r0 + rgi;
@@ -1284,6 +1304,25 @@ __global__ void __launch_bounds__(kThreads, 1) decode_fft_kernel(const __grid_co
     }
     cp_async_wait_all();
     consumer_sync();
+    if (step && s.dcv > 0) {                               // fused step: pending rank-1 update of this part's rows of C^V
+        const int j_pend = ws.pend_j[b];
+        if (j_pend >= 0) {
+            const float* xv = ws.pend + ((size_t)b * s.Hkv + h) * (s.dck + s.dcv) + s.dck;
+            float* cvg = coef_rows(c.coef_v, s, b, h, s.dcv) + (size_t)m0 * s.dcv;
+#pragma unroll 1
+            for (int i = tid; i < rows * nv; i += kConsumers) {
+                const int r = i / nv, v = i - r * nv, m = m0 + r;
+                float cs, sn;
+                basis_cs(m >> 1, j_pend, s.T, &cs, &sn);
+                const float f = (m & 1) ? sn : cs;
+                float4 x = *reinterpret_cast<const float4*>(cv_s + 4 * i);
+                const float4 y = __ldcg(reinterpret_cast<const float4*>(xv) + v);
+                x.x = fmaf(f, y.x, x.x); x.y = fmaf(f, y.y, x.y); x.z = fmaf(f, y.z, x.z); x.w = fmaf(f, y.w, x.w);
+                *reinterpret_cast<float4*>(cv_s + 4 * i) = x;
+                *reinterpret_cast<float4*>(cvg + 4 * i) = x;
+            }
+        }
+    }
     if (warp < GH) {                                       // one warp per head, lanes over the parts
         float mx = kNegBig;
 #pragma unroll 1
@@ -1395,7 +1434,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_fft_kernel(const __grid_co
 }
 
 template <int GH, int LS>
-cudaError_t launch_fft_t(const Dims& s, const CacheDev& c, const DecodePlan& p, const void* q, void* out, char* ws,
+cudaError_t launch_fft_t(const Dims& s, const CacheDev& c, const DecodePlan& p, const void* q, void* out, char* ws, int step,
                          cudaStream_t st) {
     const FftSmem L = fft_smem_layout(LS, s.k, GH, p.nb, s.d);
     cudaError_t err = ensure_dynamic_smem(decode_fft_kernel<GH, LS>, (size_t)L.total);
@@ -1430,7 +1469,7 @@ cudaError_t launch_fft_t(const Dims& s, const CacheDev& c, const DecodePlan& p, 
         } else if (coop_pdl_ok != 0) {
             cfg.numAttrs = 2;
             cudaError_t err2 = cudaLaunchKernelEx(&cfg, decode_fft_kernel<GH, LS>, tki, tvi, tkl, tvl, s, c, p,
-                                                  static_cast<const bf16*>(q), static_cast<bf16*>(out), ws);
+                                                  static_cast<const bf16*>(q), static_cast<bf16*>(out), ws, step);
             if (err2 == cudaSuccess) { coop_pdl_ok = 1; return err2; }
             if (coop_pdl_ok == 1) return err2;
             cudaGetLastError();
@@ -1442,19 +1481,19 @@ cudaError_t launch_fft_t(const Dims& s, const CacheDev& c, const DecodePlan& p, 
         }
     }
     return cudaLaunchKernelEx(&cfg, decode_fft_kernel<GH, LS>, tki, tvi, tkl, tvl, s, c, p, static_cast<const bf16*>(q),
-                              static_cast<bf16*>(out), ws);
+                              static_cast<bf16*>(out), ws, step);
 }
 
 template <int GH>
-cudaError_t launch_fft_ls(const Dims& s, const CacheDev& c, const DecodePlan& p, const void* q, void* out, char* ws,
+cudaError_t launch_fft_ls(const Dims& s, const CacheDev& c, const DecodePlan& p, const void* q, void* out, char* ws, int step,
                           cudaStream_t st) {
     switch (p.fft_log2) {
-        case 5: return launch_fft_t<GH, 5>(s, c, p, q, out, ws, st);
-        case 6: return launch_fft_t<GH, 6>(s, c, p, q, out, ws, st);
-        case 7: return launch_fft_t<GH, 7>(s, c, p, q, out, ws, st);
-        case 8: return launch_fft_t<GH, 8>(s, c, p, q, out, ws, st);
-        case 9: return launch_fft_t<GH, 9>(s, c, p, q, out, ws, st);
-        case 10: return launch_fft_t<GH, 10>(s, c, p, q, out, ws, st);
+        case 5: return launch_fft_t<GH, 5>(s, c, p, q, out, ws, step, st);
+        case 6: return launch_fft_t<GH, 6>(s, c, p, q, out, ws, step, st);
+        case 7: return launch_fft_t<GH, 7>(s, c, p, q, out, ws, step, st);
+        case 8: return launch_fft_t<GH, 8>(s, c, p, q, out, ws, step, st);
+        case 9: return launch_fft_t<GH, 9>(s, c, p, q, out, ws, step, st);
+        case 10: return launch_fft_t<GH, 10>(s, c, p, q, out, ws, step, st);
         default: return cudaErrorInvalidValue;
     }
 }
@@ -1480,10 +1519,10 @@ bool decode_fft_fused_fits(const Dims& s, int log2S, int gh, int nb, int n_part)
 }
 
 cudaError_t launch_decode_fft(const Dims& s, const CacheDev& c, int dtype, const DecodePlan& p, const void* q, void* out,
-                              char* ws, cudaStream_t st) {
+                              char* ws, bool step, cudaStream_t st) {
     if (dtype != FA_BF16) return cudaErrorInvalidValue;
-    if (p.gh == 4) return launch_fft_ls<4>(s, c, p, q, out, ws, st);
-    return launch_fft_ls<2>(s, c, p, q, out, ws, st);
+    if (p.gh == 4) return launch_fft_ls<4>(s, c, p, q, out, ws, step ? 1 : 0, st);
+    return launch_fft_ls<2>(s, c, p, q, out, ws, step ? 1 : 0, st);
 }
 
 }  // namespace fa

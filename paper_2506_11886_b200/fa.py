@@ -70,6 +70,7 @@ def lib() -> C.CDLL:
         L.fa_decode_attention.argtypes = [lp, cp, vp, vp, vp, sz, vp]
         L.fa_poll_status.argtypes = [cp, vp]
         L.fa_decode_step_host.argtypes = [lp, cp, vp, vp, vp, vp, vp, vp, sz, vp]
+        L.fa_decode_step.argtypes = [lp, cp, vp, vp, vp, vp, vp, sz, vp]
         L.fa_step_staging_bytes.argtypes = [lp]
         L.fa_step_staging_bytes.restype = sz
         L.fa_launch_count.argtypes = [lp, C.c_int]
@@ -77,7 +78,7 @@ def lib() -> C.CDLL:
         L.fa_status_string.restype = C.c_char_p
         for name in ("fa_cache_sizes_of", "fa_workspace_bytes", "fa_cache_reset", "fa_validate", "fa_compress",
                      "fa_append", "fa_decode_attention", "fa_poll_status", "fa_launch_count", "fa_version",
-                     "fa_decode_step_host"):
+                     "fa_decode_step_host", "fa_decode_step"):
             getattr(L, name).restype = C.c_int
         _lib = L
     return _lib
@@ -235,6 +236,15 @@ def fa_decode_attention(layout: Layout, cache: Cache, q: torch.Tensor, out: torc
 
 def fa_step_staging_bytes(layout: Layout) -> int:
     return int(lib().fa_step_staging_bytes(C.byref(layout.c())))
+
+
+def fa_decode_step(layout: Layout, cache: Cache, q: torch.Tensor, k_new: torch.Tensor, v_new: torch.Tensor,
+                   out: torch.Tensor, ws: torch.Tensor, stream=None) -> None:
+    """fa_append(k_new, v_new) then fa_decode_attention(q) as one step (device tensors)."""
+    for t in (q, k_new, v_new, out):
+        assert t.is_cuda and t.is_contiguous() and t.dtype == layout.torch_dtype
+    _check(lib().fa_decode_step(C.byref(layout.c()), C.byref(cache.c()), _ptr(q), _ptr(k_new), _ptr(v_new), _ptr(out),
+                                _ptr(ws), ws.numel(), _stream(stream)), "fa_decode_step")
 
 
 def fa_decode_step_host(layout: Layout, cache: Cache, q_host: torch.Tensor, k_new_host, v_new_host,

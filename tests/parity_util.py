@@ -73,6 +73,26 @@ class Pair:
         fa.fa_append(self.layout, self.gpu, k_new.cuda().contiguous(), v_new.cuda().contiguous())
         self.ref.append(to64(k_new), to64(v_new))
 
+    def step(self, q: torch.Tensor, k_new: torch.Tensor, v_new: torch.Tensor, heads=None):
+        """One fa_decode_step on the CUDA side; append then decode on the oracle side."""
+        out = torch.full_like(q, float("nan"), device="cuda")
+        fa.fa_decode_step(self.layout, self.gpu, q.cuda().contiguous(), k_new.cuda().contiguous(),
+                          v_new.cuda().contiguous(), out, self.ws)
+        torch.cuda.synchronize()
+        self.ref.append(to64(k_new), to64(v_new))
+        return to64(out), self.ref.decode(to64(q), heads=heads)
+
+    def check_step(self, q, k_new, v_new, heads=None, tol=None):
+        got, want = self.step(q, k_new, v_new, heads=heads)
+        if tol is None:
+            tol = OUT_ABS_F32 if self.layout.kv_dtype == fa.FA_F32 else OUT_ABS_BF16
+        mask = ~np.isnan(want)
+        assert mask.any()
+        assert not np.isnan(got[mask]).any()
+        err = np.abs(got[mask] - want[mask]).max()
+        assert err <= tol, f"output error {err:.3e} > {tol}"
+        return err
+
     def decode(self, q: torch.Tensor, heads=None):
         out = torch.full_like(q, float("nan"), device="cuda")
         fa.fa_decode_attention(self.layout, self.gpu, q.cuda().contiguous(), out, self.ws)

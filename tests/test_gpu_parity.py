@@ -233,3 +233,61 @@ def test_mha_48_kept_dims(algo):
         pair.append(K[:, t], V[:, t])
     pair.check_state()
     pair.check_decode(synth.queries(shape, seed=12, step=1))
+
+
+@pytest.mark.parametrize("algo", ALGOS)
+def test_decode_step_from_empty_through_eviction(algo):
+    """fa_decode_step token by token: init fills, local fills, then every step evicts a row into the middle;
+    outputs against append + decode of the oracle, the cache against the oracle's at the end."""
+    shape = SMALL_BF16.with_(B=1, Hq=4, Hkv=1, L=0, L_init=3, L_local=8, T=256, M=32, n_full_k=16, n_full_v=8)
+    layout = layout_of(shape, max_mid=256, P=8, algo=algo)
+    stream = synth.KVStream(shape, seed=11)
+    pair = Pair(layout, stream.idx_full_k, stream.idx_full_v)
+    fa.fa_cache_reset(layout, pair.gpu)
+    K0, V0 = stream.tokens(0, 0)
+    pair.ref.compress(to64(K0), to64(V0))
+    K, V = stream.tokens(0, 60)
+    for t in range(60):
+        pair.check_step(synth.queries(shape, seed=11, step=t), K[:, t], V[:, t])
+        if t in (2, 3, 10, 11, 12, 40, 59):
+            pair.check_state()
+    # the same workspace keeps serving plain decode calls
+    pair.check_decode(synth.queries(shape, seed=12))
+
+
+def test_decode_step_after_compress_gqa_batch():
+    """Prefill, then fused steps on a batch of two rows with four query heads per KV head."""
+    shape = SMALL_BF16.with_(L=700, decode_steps=12)
+    pair, stream = make_pair(shape, seed=13, algo=fa.FA_DECODE_FFT, P=16)
+    K, V = stream.tokens(shape.L, shape.L + 12)
+    for t in range(12):
+        pair.check_step(synth.queries(shape, seed=13, step=t), K[:, t], V[:, t])
+    pair.check_state()
+    assert fa.fa_launch_count(pair.layout, 3) in (2, 3, 4)
+
+
+def test_decode_step_full_middle_reports_capacity():
+    """A step whose append finds the middle full changes nothing, reports it, and still decodes."""
+    shape = SMALL_BF16.with_(B=1, Hq=4, Hkv=1, L=0, L_init=2, L_local=4, T=64, M=16, n_full_k=16, n_full_v=8)
+    layout = layout_of(shape, max_mid=8, P=2, algo=fa.FA_DECODE_FFT)
+    stream = synth.KVStream(shape, seed=14)
+    try:
+        pair = Pair(layout, stream.idx_full_k, stream.idx_full_v)
+    except fa.FaError as e:
+        if e.status == fa.FA_ERR_UNSUPPORTED:
+            pytest.skip("layout outside the FFT kernel's range")
+        raise
+    fa.fa_cache_reset(layout, pair.gpu)
+    K0, V0 = stream.tokens(0, 0)
+    pair.ref.compress(to64(K0), to64(V0))
+    K, V = stream.tokens(0, 15)
+    for t in range(14):                                   # 2 + 4 + 8 tokens fill everything
+        pair.check_step(synth.queries(shape, seed=14, step=t), K[:, t], V[:, t])
+    q = synth.queries(shape, seed=14, step=99)
+    out = torch.full_like(q, float("nan"), device="cuda")
+    fa.fa_decode_step(layout, pair.gpu, q.cuda().contiguous(), K[:, 14].cuda().contiguous(), V[:, 14].cuda().contiguous(),
+                      out, pair.ws)
+    assert fa.fa_poll_status(pair.gpu) == fa.FA_ERR_CAPACITY
+    want = pair.ref.decode(to64(q))                       # the oracle cache did not take the token either
+    assert np.abs(to64(out) - want).max() <= 2e-2
+    pair.check_state()
