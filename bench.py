@@ -5,15 +5,16 @@ Workload (N = 1): the LLaMA-3.1-8B-shaped single-layer decode at 32K context
 (batch 1, 32 query / 8 KV heads, head_dim 128, bf16; per KV head 32 dims kept
 per token, 96 dims held as M = 1024 Fourier coefficients; 4 sink + 1024 recent
 tokens kept whole).  One STEP = one decode step of the whole hot path on a
-resident cache: fa_append (ring push + Eq.5 coefficient update of the token
-that leaves the local window) followed by fa_decode_attention (Eq.6).  The
+resident cache through fa_decode_step: the new token is pushed (Eq.5: the
+row that leaves the local window joins the middle and is added to every
+coefficient row) and the query attends to the result (Eq.6).  The
 cache of one layer (43 MB) would fit the 126 MB L2, so the steps rotate over
 `--instances` independent caches (>= 8, > L2 in total).
 
 Printed JSON (one line, rank 0): metric / value = microseconds per step,
 device-timed with CUDA events around a CUDA-graph replay of exactly K steps;
 `e2e` = the same through fa_decode_step_host with pinned HOST q / k_new /
-v_new / out; `roofline` = fa_decode_attention alone (its three kernels) against
+v_new / out; `roofline` = fa_decode_attention alone (one fused kernel) against
 the measured HBM peak on the bytes the hybrid cache holds; `cpu_baseline` = the
 fp64 oracle on the host cores on a stated sample.  `--impl reference` times the
 oracle instead.
@@ -222,10 +223,13 @@ def run_ours(args):
 
     def step(s, do_append=True, do_decode=True):
         i = s % n_inst
-        if do_append:
+        if do_append and do_decode:
+            fa.fa_decode_step(layout, caches[i], qs[s % qs.shape[0]], Kn[visit[i]], Vn[visit[i]], outs[s], ws)
+            visit[i] += 1
+        elif do_append:
             fa.fa_append(layout, caches[i], Kn[visit[i]], Vn[visit[i]])
             visit[i] += 1
-        if do_decode:
+        elif do_decode:
             fa.fa_decode_attention(layout, caches[i], qs[s % qs.shape[0]], outs[s], ws)
 
     def barrier():
@@ -289,13 +293,13 @@ def run_ours(args):
     eb = 2
     q_bytes = shape.B * shape.Hq * shape.d * eb
     kv_bytes = shape.B * shape.Hkv * shape.d * eb
-    launches = K_steps * (fa.fa_launch_count(layout, 1) + fa.fa_launch_count(layout, 2))
+    launches = K_steps * fa.fa_launch_count(layout, 3)
     line = {
         "metric": METRIC, "value": us_step / world, "unit": UNIT, "n_gpus": world, "steps": K_steps, "warmup": W,
         "ms_per_step": us_step / 1e3, "higher_is_better": False, "scaling": "weak", "vs_baseline": None,
         "dtype": "bf16 storage, f32 arithmetic", "data": "synthetic",
         "config": {"workload": shape.name, "global_batch": shape.B * world, "seq_len": shape.L,
-                   "step": "fa_append + fa_decode_attention, one layer", "parallelism": f"replicas x{world}",
+                   "step": "fa_decode_step (append + decode), one layer", "parallelism": f"replicas x{world}",
                    "l2": f"inputs larger than L2: {n_inst} cache instances x {by['decode'] / 1e6:.1f} MB rotated",
                    "timing": "CUDA events around one CUDA-graph replay of K steps", "n_mid_end": n_mid_now},
         "breakdown": {"decode_us": us_decode, "append_us": us_append, "tokens_per_s": 1e6 / us_step * shape.B * world,

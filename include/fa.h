@@ -162,7 +162,7 @@ fa_status fa_decode_attention(const fa_layout* layout, const fa_cache* cache, co
 /* One decode step with device inputs (Eq.5 then Eq.6): the result and the cache afterwards are those
  * of fa_append(k_new, v_new) followed by fa_decode_attention(q).  Where the decode call is a single
  * fused kernel (see fa_decode_algo) and the KV head's query heads fit one pass, the coefficient
- * update of Eq.5 rides on that kernel: a one-CTA-per-batch-row kernel moves the row that leaves the
+ * update of Eq.5 rides on that kernel: a small kernel (one CTA per batch row and KV head) moves the row that leaves the
  * local window, stores the new token and advances the counters, and the decode kernel adds
  * f_j x^T to each coefficient row as it streams it (C^K before forming u, C^V before the output
  * product) and writes it back, so the coefficients cross the memory bus once per step instead of

@@ -141,7 +141,7 @@ __global__ void __launch_bounds__(256) append_kernel(Dims s, CacheDev c, const K
     }
 }
 
-// First half of a fused decode step (Eq.5 without the coefficient update): one CTA per batch row moves
+// First half of a fused decode step (Eq.5 without the coefficient update): one CTA per (batch row, KV head) moves
 // the row that leaves the local window (kept dims to K^mu / V^mu), stores the new token and advances
 // the counters, and leaves the compressed dims of the leaving row with its basis column j in the
 // workspace.  The decode kernel of the same step adds f_j x^T to the coefficient rows as it streams
@@ -150,7 +150,8 @@ template <typename KV>
 __global__ void __launch_bounds__(256) append_lite_kernel(Dims s, CacheDev c, DecodePlan p, const KV* __restrict__ k_new,
                                                           const KV* __restrict__ v_new, char* wsp) {
     __shared__ float x_s[2][256];        // the row that leaves, both sides, natural dim order
-    const int b = blockIdx.x, tid = threadIdx.x;
+    __shared__ int last_s;
+    const int h = blockIdx.x, b = blockIdx.y, tid = threadIdx.x;
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     asm volatile("griddepcontrol.wait;" ::: "memory");
     Ws ws = ws_view(wsp, p);
@@ -160,62 +161,64 @@ __global__ void __launch_bounds__(256) append_lite_kernel(Dims s, CacheDev c, De
     const bool evict = !to_init && n_local == s.l_local;
     const bool full = evict && (n_mid >= s.max_mid || n_mid >= s.T);
     if (full) {
-        if (tid == 0) { atomicExch(c.status, (int)FA_ERR_CAPACITY); ws.pend_j[b] = -1; }
-        return;
+        if (tid == 0 && h == 0) { atomicExch(c.status, (int)FA_ERR_CAPACITY); ws.pend_j[b] = -1; }
+        return;                          // every CTA of this batch row takes the same exit
     }
     if (evict) {
         const int j = n_mid;
-#pragma unroll 1
-        for (int h = 0; h < s.Hkv; ++h) {
-            for (int i = tid; i < 2 * s.d; i += 256) {
-                const int side = i / s.d, e = i - side * s.d;
-                float v;
-                if (s.l_local == 0) v = ld_f((side == 0 ? k_new : v_new) + ((size_t)b * s.Hkv + h) * s.d + e);
-                else v = ld_f(win_row<KV>(side == 0 ? c.k_local : c.v_local, s, b, h, s.l_local, head) + e);
-                x_s[side][e] = v;
-            }
-            __syncthreads();
-            for (int i = tid; i < s.nfk + s.nfv; i += 256) {
-                const int side = i < s.nfk ? 0 : 1;
-                const int e = side == 0 ? i : i - s.nfk;
-                const int nfull = side == 0 ? s.nfk : s.nfv;
-                const int32_t* idf = (side == 0 ? c.idx_full_k : c.idx_full_v) + (size_t)h * nfull;
-                KV* dst = mid_row<KV>(side == 0 ? c.k_mid : c.v_mid, s, b, h, j % s.P, j / s.P, nfull);
-                const int col = side == 1 ? v_mid_col(j / s.P, e, nfull, sizeof(KV) == 2 ? FA_BF16 : FA_F32) : e;
-                st_f(dst + col, x_s[side][idf[e]]);
-            }
-            float* pend = ws.pend + ((size_t)b * s.Hkv + h) * (s.dck + s.dcv);
-            for (int i = tid; i < s.dck + s.dcv; i += 256) {
-                const int side = i < s.dck ? 0 : 1;
-                const int e = side == 0 ? i : i - s.dck;
-                const int32_t* idc = side == 0 ? c.idx_comp_k + (size_t)h * s.dck : c.idx_comp_v + (size_t)h * s.dcv;
-                pend[i] = x_s[side][idc[e]];
-            }
-            __syncthreads();
+        for (int i = tid; i < 2 * s.d; i += 256) {
+            const int side = i / s.d, e = i - side * s.d;
+            float v;
+            if (s.l_local == 0) v = ld_f((side == 0 ? k_new : v_new) + ((size_t)b * s.Hkv + h) * s.d + e);
+            else v = ld_f(win_row<KV>(side == 0 ? c.k_local : c.v_local, s, b, h, s.l_local, head) + e);
+            x_s[side][e] = v;
+        }
+        __syncthreads();
+        for (int i = tid; i < s.nfk + s.nfv; i += 256) {
+            const int side = i < s.nfk ? 0 : 1;
+            const int e = side == 0 ? i : i - s.nfk;
+            const int nfull = side == 0 ? s.nfk : s.nfv;
+            const int32_t* idf = (side == 0 ? c.idx_full_k : c.idx_full_v) + (size_t)h * nfull;
+            KV* dst = mid_row<KV>(side == 0 ? c.k_mid : c.v_mid, s, b, h, j % s.P, j / s.P, nfull);
+            const int col = side == 1 ? v_mid_col(j / s.P, e, nfull, sizeof(KV) == 2 ? FA_BF16 : FA_F32) : e;
+            st_f(dst + col, x_s[side][idf[e]]);
+        }
+        float* pend = ws.pend + ((size_t)b * s.Hkv + h) * (s.dck + s.dcv);
+        for (int i = tid; i < s.dck + s.dcv; i += 256) {
+            const int side = i < s.dck ? 0 : 1;
+            const int e = side == 0 ? i : i - s.dck;
+            const int32_t* idc = side == 0 ? c.idx_comp_k + (size_t)h * s.dck : c.idx_comp_v + (size_t)h * s.dcv;
+            pend[i] = x_s[side][idc[e]];
         }
     }
-    // the new token: next init row, or the ring slot behind the newest local row (the slot just vacated when full)
-    for (int i = tid; i < 2 * s.Hkv * s.d; i += 256) {
-        const int side = i / (s.Hkv * s.d);
-        const int rem = i - side * (s.Hkv * s.d);
-        const int hh = rem / s.d, e = rem - hh * s.d;
-        const KV* src = (side == 0 ? k_new : v_new) + ((size_t)b * s.Hkv + hh) * s.d;
+    // the new token of this head: next init row, or the ring slot behind the newest local row (the slot
+    // just read and vacated when the window is full)
+    for (int i = tid; i < 2 * s.d; i += 256) {
+        const int side = i / s.d, e = i - side * s.d;
+        const KV* src = (side == 0 ? k_new : v_new) + ((size_t)b * s.Hkv + h) * s.d;
         if (to_init) {
-            win_row<KV>(side == 0 ? c.k_init : c.v_init, s, b, hh, s.l_init, n_init)[e] = src[e];
+            win_row<KV>(side == 0 ? c.k_init : c.v_init, s, b, h, s.l_init, n_init)[e] = src[e];
         } else if (s.l_local > 0) {
             const int slot = evict ? head : (head + n_local) % s.l_local;
-            win_row<KV>(side == 0 ? c.k_local : c.v_local, s, b, hh, s.l_local, slot)[e] = src[e];
+            win_row<KV>(side == 0 ? c.k_local : c.v_local, s, b, h, s.l_local, slot)[e] = src[e];
         }
     }
+    // ticket: the last head of this batch row to finish advances the counters (nobody reads them after this point)
     __syncthreads();
     if (tid == 0) {
-        if (to_init) c.state[kStateStride * b + 0] = n_init + 1;
-        else if (evict) {
-            c.state[kStateStride * b + 2] = n_mid + 1;
-            if (s.l_local > 0) c.state[kStateStride * b + 3] = (head + 1) % s.l_local;
-        } else c.state[kStateStride * b + 1] = n_local + 1;
-        ws.pend_j[b] = evict ? n_mid : -1;
+        __threadfence();
+        const int done = atomicAdd(c.state + kStateStride * b + 4, 1);
+        last_s = (done == (int)gridDim.x - 1);
     }
+    __syncthreads();
+    if (!last_s || tid != 0) return;
+    if (to_init) c.state[kStateStride * b + 0] = n_init + 1;
+    else if (evict) {
+        c.state[kStateStride * b + 2] = n_mid + 1;
+        if (s.l_local > 0) c.state[kStateStride * b + 3] = (head + 1) % s.l_local;
+    } else c.state[kStateStride * b + 1] = n_local + 1;
+    c.state[kStateStride * b + 4] = 0;            // ticket counter ready for the next call
+    ws.pend_j[b] = evict ? n_mid : -1;
 }
 
 template <typename KV>
@@ -240,7 +243,7 @@ template <typename KV>
 static cudaError_t launch_append_lite_t(const Dims& s, const CacheDev& c, const DecodePlan& p, const void* k_new, const void* v_new,
                                         char* ws, cudaStream_t st) {
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(s.B);
+    cfg.gridDim = dim3(s.Hkv, s.B);
     cfg.blockDim = dim3(256);
     cfg.stream = st;
     cudaLaunchAttribute attr[1];

@@ -681,12 +681,18 @@ __global__ void __launch_bounds__(kThreads, 1) decode_fft_kernel(const __grid_co
             if (j_pend >= 0) {
                 const float* xk = ws.pend + ((size_t)b * s.Hkv + h) * (s.dck + s.dcv);
                 float* ckg = coef_rows(c.coef_k, s, b, h, s.dck) + (size_t)m0 * s.dck;
+                float* f_s = kb;                           // basis column j for this part's rows (kb is not in use yet)
+#pragma unroll 1
+                for (int r = tid; r < m1 - m0; r += kConsumers) {
+                    float cs, sn;
+                    basis_cs((m0 + r) >> 1, j_pend, s.T, &cs, &sn);
+                    f_s[r] = ((m0 + r) & 1) ? sn : cs;
+                }
+                consumer_sync();
 #pragma unroll 1
                 for (int i = tid; i < (m1 - m0) * nv; i += kConsumers) {
-                    const int r = i / nv, v = i - r * nv, m = m0 + r;
-                    float cs, sn;
-                    basis_cs(m >> 1, j_pend, s.T, &cs, &sn);
-                    const float f = (m & 1) ? sn : cs;
+                    const int r = i / nv, v = i - r * nv;
+                    const float f = f_s[r];
                     float4 x = *reinterpret_cast<const float4*>(fbuf + 4 * i);
                     const float4 y = __ldcg(reinterpret_cast<const float4*>(xk) + v);
                     x.x = fmaf(f, y.x, x.x); x.y = fmaf(f, y.y, x.y); x.z = fmaf(f, y.z, x.z); x.w = fmaf(f, y.w, x.w);
@@ -1309,12 +1315,18 @@ __global__ void __launch_bounds__(kThreads, 1) decode_fft_kernel(const __grid_co
         if (j_pend >= 0) {
             const float* xv = ws.pend + ((size_t)b * s.Hkv + h) * (s.dck + s.dcv) + s.dck;
             float* cvg = coef_rows(c.coef_v, s, b, h, s.dcv) + (size_t)m0 * s.dcv;
+            float* f_s = ps_s;                             // basis column j for this part's rows (ps_s is not in use yet)
+#pragma unroll 1
+            for (int r = tid; r < rows; r += kConsumers) {
+                float cs, sn;
+                basis_cs((m0 + r) >> 1, j_pend, s.T, &cs, &sn);
+                f_s[r] = ((m0 + r) & 1) ? sn : cs;
+            }
+            consumer_sync();
 #pragma unroll 1
             for (int i = tid; i < rows * nv; i += kConsumers) {
-                const int r = i / nv, v = i - r * nv, m = m0 + r;
-                float cs, sn;
-                basis_cs(m >> 1, j_pend, s.T, &cs, &sn);
-                const float f = (m & 1) ? sn : cs;
+                const int r = i / nv, v = i - r * nv;
+                const float f = f_s[r];
                 float4 x = *reinterpret_cast<const float4*>(cv_s + 4 * i);
                 const float4 y = __ldcg(reinterpret_cast<const float4*>(xv) + v);
                 x.x = fmaf(f, y.x, x.x); x.y = fmaf(f, y.y, x.y); x.z = fmaf(f, y.z, x.z); x.w = fmaf(f, y.w, x.w);
