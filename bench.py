@@ -209,7 +209,13 @@ def run_ours(args):
         comp_ms.append(ev0.elapsed_time(ev1))
     n_mid0 = shape.L - shape.L_init - shape.L_local
     comp_flop = 2.0 * shape.M * n_mid0 * ((shape.d - shape.n_full_k) + (shape.d - shape.n_full_v)) * shape.Hkv * shape.B
-    del Kp, Vp
+    # dimension selection (Sec. 3.4) on the same prefill: all-dims compression + reconstruction error + ranking
+    sel_ms = []
+    for _ in range(3):
+        ev0.record(); sel = fa.fa_select_dims(layout, Kp, Vp); ev1.record(); torch.cuda.synchronize()
+        sel_ms.append(ev0.elapsed_time(ev1))
+    sel_ok = bool(torch.equal(sel[0].cpu(), stream.idx_full_k) and torch.equal(sel[2].cpu(), stream.idx_full_v))
+    del Kp, Vp, sel
     # per-step inputs: visit r of an instance appends token L + r
     regions = 4
     visits = (W + K_steps + n_inst - 1) // n_inst * regions + 4
@@ -305,7 +311,8 @@ def run_ours(args):
         "breakdown": {"decode_us": us_decode, "append_us": us_append, "tokens_per_s": 1e6 / us_step * shape.B * world,
                       "append_gbs": by["append"] / (us_append * 1e-6) / 1e9,
                       "compress_ms_per_layer": min(comp_ms), "compress_tflops": comp_flop / (min(comp_ms) * 1e-3) / 1e12,
-                      "compress_path": "tcgen05 bf16 x bf16 -> f32 (TMEM), basis tile generated in registers"},
+                      "compress_path": "tcgen05 bf16 x bf16 -> f32 (TMEM), basis tile generated in registers",
+                      "select_dims_ms": min(sel_ms), "select_dims_finds_generator_sets": sel_ok},
         "roofline": {"kernel": "fa_decode_attention (one fused cooperative kernel: u, token loop, merge)", "bound": "hbm",
                      "achieved": dec_gbs, "peak": peak, "unit": "GB/s", "frac": dec_gbs / peak, "peak_kind": peak_kind,
                      "algorithmic_bytes": by["decode"], "traffic": NCU_TRAFFIC_BYTES_PER_CALL,

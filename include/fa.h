@@ -183,6 +183,24 @@ fa_status fa_decode_step_host(const fa_layout* layout, fa_cache* cache, const vo
                               void* staging, void* ws, size_t ws_bytes, void* stream);
 size_t fa_step_staging_bytes(const fa_layout* layout);
 
+/* Sec. 3.4, dimension selection.  Compresses and reconstructs EVERY dimension of the middle
+ * segment of the prefilled K and V (Eq.3, then Eq.6's reconstruction with this layout's weights) and
+ * ranks the dimensions of each KV head by mean squared reconstruction error, averaged over the batch
+ * rows: the layout's n_full_k (n_full_v) dimensions with the LARGEST error are to be kept per token,
+ * the others held as coefficients; among equal errors the lower index is compressed first.
+ *   K, V, strides, L: as for fa_compress (the middle is what lies between the first l_init and
+ *     the last l_local tokens; period, n_coef, max_mid, norm of the layout apply).
+ *   idx_full_k [H_kv][n_full_k], idx_comp_k [H_kv][d - n_full_k], idx_full_v, idx_comp_v: DEVICE
+ *     outputs, ascending, ready to be a cache's index sets.
+ *   mse: optional DEVICE output [B][H_kv][2][d] (side 0 = K, 1 = V), the per-row mean squared errors.
+ *   ws / ws_bytes: scratch of fa_select_workspace_bytes(layout) bytes, 256-byte aligned (it holds the
+ *     coefficients of all dimensions).  head_dim must be 64, 128 or 256.
+ * Asynchronous on `stream`.  An empty middle gives zero errors (the lowest indices are compressed). */
+fa_status fa_select_workspace_bytes(const fa_layout* layout, size_t* out);
+fa_status fa_select_dims(const fa_layout* layout, const void* K, const void* V, int64_t stride_b, int64_t stride_t,
+                         int64_t stride_h, int32_t L, int32_t* idx_full_k, int32_t* idx_comp_k, int32_t* idx_full_v,
+                         int32_t* idx_comp_v, float* mse, void* ws, size_t ws_bytes, void* stream);
+
 /* fa_decode_attention without a caller workspace.  (The paper has no counterpart: this is a
  * packaging variant of the same computation.)  It is meant for callers that cannot allocate
  * device memory when they reach this call: an engine that gave all of its HBM to its own pools

@@ -71,6 +71,8 @@ def lib() -> C.CDLL:
         L.fa_poll_status.argtypes = [cp, vp]
         L.fa_decode_step_host.argtypes = [lp, cp, vp, vp, vp, vp, vp, vp, sz, vp]
         L.fa_decode_step.argtypes = [lp, cp, vp, vp, vp, vp, vp, sz, vp]
+        L.fa_select_workspace_bytes.argtypes = [lp, C.POINTER(sz)]
+        L.fa_select_dims.argtypes = [lp, vp, vp, i64, i64, i64, i32, vp, vp, vp, vp, vp, vp, sz, vp]
         L.fa_step_staging_bytes.argtypes = [lp]
         L.fa_step_staging_bytes.restype = sz
         L.fa_launch_count.argtypes = [lp, C.c_int]
@@ -78,7 +80,7 @@ def lib() -> C.CDLL:
         L.fa_status_string.restype = C.c_char_p
         for name in ("fa_cache_sizes_of", "fa_workspace_bytes", "fa_cache_reset", "fa_validate", "fa_compress",
                      "fa_append", "fa_decode_attention", "fa_poll_status", "fa_launch_count", "fa_version",
-                     "fa_decode_step_host", "fa_decode_step"):
+                     "fa_decode_step_host", "fa_decode_step", "fa_select_workspace_bytes", "fa_select_dims"):
             getattr(L, name).restype = C.c_int
         _lib = L
     return _lib
@@ -236,6 +238,25 @@ def fa_decode_attention(layout: Layout, cache: Cache, q: torch.Tensor, out: torc
 
 def fa_step_staging_bytes(layout: Layout) -> int:
     return int(lib().fa_step_staging_bytes(C.byref(layout.c())))
+
+
+def fa_select_dims(layout: Layout, K: torch.Tensor, V: torch.Tensor, stream=None):
+    """Sec. 3.4: index sets (idx_full_k, idx_comp_k, idx_full_v, idx_comp_v) [H_kv][...] int32 on the
+    device of K, and the per-row mean squared reconstruction errors [B][H_kv][2][d]."""
+    assert K.is_cuda and V.is_cuda and K.dtype == layout.torch_dtype and K.shape == V.shape and K.stride() == V.stride()
+    B, L, H, d = K.shape
+    assert K.stride(3) == 1
+    out = C.c_size_t(0)
+    _check(lib().fa_select_workspace_bytes(C.byref(layout.c()), C.byref(out)), "fa_select_workspace_bytes")
+    ws = torch.zeros(max(256, out.value), dtype=torch.uint8, device=K.device)
+    dev = K.device
+    idx = [torch.zeros((H, n), dtype=torch.int32, device=dev) for n in
+           (layout.n_full_k, d - layout.n_full_k, layout.n_full_v, d - layout.n_full_v)]
+    mse = torch.zeros((B, H, 2, d), dtype=torch.float32, device=dev)
+    _check(lib().fa_select_dims(C.byref(layout.c()), _ptr(K), _ptr(V), K.stride(0), K.stride(1), K.stride(2), L,
+                                *[_ptr(t) if t.numel() else None for t in idx], _ptr(mse), _ptr(ws), ws.numel(),
+                                _stream(stream)), "fa_select_dims")
+    return (*idx, mse)
 
 
 def fa_decode_step(layout: Layout, cache: Cache, q: torch.Tensor, k_new: torch.Tensor, v_new: torch.Tensor,
