@@ -164,6 +164,16 @@ __global__ void __launch_bounds__(256) append_lite_kernel(Dims s, CacheDev c, De
         if (tid == 0 && h == 0) { atomicExch(c.status, (int)FA_ERR_CAPACITY); ws.pend_j[b] = -1; }
         return;                          // every CTA of this batch row takes the same exit
     }
+    // the new token of this head (up to two elements per thread), loaded together with the leaving row
+    KV new_e[2];
+#pragma unroll
+    for (int u = 0; u < 2; ++u) {
+        const int i = tid + 256 * u;
+        if (i < 2 * s.d) {
+            const int side = i / s.d, e = i - side * s.d;
+            new_e[u] = ((side == 0 ? k_new : v_new) + ((size_t)b * s.Hkv + h) * s.d)[e];
+        }
+    }
     if (evict) {
         const int j = n_mid;
         for (int i = tid; i < 2 * s.d; i += 256) {
@@ -193,14 +203,17 @@ __global__ void __launch_bounds__(256) append_lite_kernel(Dims s, CacheDev c, De
     }
     // the new token of this head: next init row, or the ring slot behind the newest local row (the slot
     // just read and vacated when the window is full)
-    for (int i = tid; i < 2 * s.d; i += 256) {
+    if (evict) __syncthreads();          // every thread has read the slot that is overwritten next
+#pragma unroll
+    for (int u = 0; u < 2; ++u) {
+        const int i = tid + 256 * u;
+        if (i >= 2 * s.d) continue;
         const int side = i / s.d, e = i - side * s.d;
-        const KV* src = (side == 0 ? k_new : v_new) + ((size_t)b * s.Hkv + h) * s.d;
         if (to_init) {
-            win_row<KV>(side == 0 ? c.k_init : c.v_init, s, b, h, s.l_init, n_init)[e] = src[e];
+            win_row<KV>(side == 0 ? c.k_init : c.v_init, s, b, h, s.l_init, n_init)[e] = new_e[u];
         } else if (s.l_local > 0) {
             const int slot = evict ? head : (head + n_local) % s.l_local;
-            win_row<KV>(side == 0 ? c.k_local : c.v_local, s, b, h, s.l_local, slot)[e] = src[e];
+            win_row<KV>(side == 0 ? c.k_local : c.v_local, s, b, h, s.l_local, slot)[e] = new_e[u];
         }
     }
     // ticket: the last head of this batch row to finish advances the counters (nobody reads them after this point)

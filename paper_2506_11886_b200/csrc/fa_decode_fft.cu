@@ -35,6 +35,7 @@ constexpr int kWarps = kConsumers / 32;
 constexpr int kThreads = kConsumers + 32;
 constexpr int kStageBytes = 16384;
 constexpr int kStages = 5;
+constexpr int kPendRows = 256;            // rows of a part whose basis values are tabulated for the fused step's update
 constexpr int kWinRowsPerTile = 64;       // rows of one window tile: two [64 rows x 64 dims] TMA boxes, 128-byte swizzle
 constexpr int kWinHalfBytes = kWinRowsPerTile * 128;
 constexpr uint32_t kSpinLimit = 1u << 24;
@@ -357,7 +358,7 @@ __device__ __forceinline__ WinSegs win_segments(int t0, int t1, int n_init, int 
 }
 
 struct FftSmem {
-    int stages_off, fbuf_off, kb_off, pbt_off, twf_off, rev_off, E_off, ut_off, z_off, o_off, red_off, zero_off, total;
+    int stages_off, fbuf_off, kb_off, pbt_off, twf_off, rev_off, E_off, ut_off, z_off, o_off, red_off, pend_off, zero_off, total;
     int fb_floats, pbs;
 };
 __host__ __device__ inline FftSmem fft_smem_layout(int log2S, int k, int GH, int NB, int d) {
@@ -383,6 +384,8 @@ __host__ __device__ inline FftSmem fft_smem_layout(int log2S, int k, int GH, int
     L.z_off = off; off += (8 * k * GH + 15) / 16 * 16;
     L.o_off = off; off += 4 * GH * d;
     L.red_off = off; off += 4 * (kWarps * GH + GH + 8);
+    off = (off + 15) / 16 * 16;
+    L.pend_off = off; off += 8 * d + 4 * kPendRows;        // fused step: compressed dims of the leaving row, basis column of this part's rows
     L.total = (off + 127) / 128 * 128 + 1024;             // slack to align the base to 1024 bytes at run time
     return L;
 }
@@ -570,6 +573,28 @@ __global__ void __launch_bounds__(kThreads, 1) decode_fft_kernel(const __grid_co
 #pragma unroll 1
         for (int i = tid; i < (m1 - m0) * (s.dck >> 2); i += kConsumers) cp_async16(fbuf + 4 * i, ck + 4 * i);
     }
+    // fused step: the coefficient update the light append kernel left pending (basis column j_pend, or -1);
+    // the leaving row's compressed dims and the basis values of this part's rows are fetched / formed now
+    float* xp_s = reinterpret_cast<float*>(smem_raw + L.pend_off);       // [dck + dcv]
+    float* f_s = xp_s + 2 * s.d;                                          // [kPendRows]
+    const int j_pend = step ? ws.pend_j[b] : -1;
+    if (j_pend >= 0) {
+        const float* xp = ws.pend + ((size_t)b * s.Hkv + h) * (s.dck + s.dcv);
+        for (int i = tid; i < (s.dck + s.dcv) >> 2; i += kConsumers) cp_async16(xp_s + 4 * i, xp + 4 * i);
+#pragma unroll 1
+        for (int r = tid; r < min(m1 - m0, kPendRows); r += kConsumers) {
+            float cs, sn;
+            basis_cs((m0 + r) >> 1, j_pend, s.T, &cs, &sn);
+            f_s[r] = ((m0 + r) & 1) ? sn : cs;
+        }
+    }
+    // basis value of row r of this part (tabulated for the first kPendRows rows)
+    auto f_row = [&](int r) -> float {
+        if (r < kPendRows) return f_s[r];
+        float cs, sn;
+        basis_cs((m0 + r) >> 1, j_pend, s.T, &cs, &sn);
+        return ((m0 + r) & 1) ? sn : cs;
+    };
 
     // B fragments of q for the kept K dims: column gq is slot gq = head hperm(gq);
     // round rd covers pieces 4 rd + tq of a row, two k-steps each
@@ -677,24 +702,14 @@ __global__ void __launch_bounds__(kThreads, 1) decode_fft_kernel(const __grid_co
             const int l8 = tid & 7, rgi = tid >> 3, nv = s.dck >> 2;
             // fused step: the rank-1 update of Eq.5 that the light append kernel left pending, applied to
             // this part's rows while they are on chip, and written back
-            const int j_pend = step ? ws.pend_j[b] : -1;
             if (j_pend >= 0) {
-                const float* xk = ws.pend + ((size_t)b * s.Hkv + h) * (s.dck + s.dcv);
                 float* ckg = coef_rows(c.coef_k, s, b, h, s.dck) + (size_t)m0 * s.dck;
-                float* f_s = kb;                           // basis column j for this part's rows (kb is not in use yet)
-#pragma unroll 1
-                for (int r = tid; r < m1 - m0; r += kConsumers) {
-                    float cs, sn;
-                    basis_cs((m0 + r) >> 1, j_pend, s.T, &cs, &sn);
-                    f_s[r] = ((m0 + r) & 1) ? sn : cs;
-                }
-                consumer_sync();
 #pragma unroll 1
                 for (int i = tid; i < (m1 - m0) * nv; i += kConsumers) {
                     const int r = i / nv, v = i - r * nv;
-                    const float f = f_s[r];
+                    const float f = f_row(r);
                     float4 x = *reinterpret_cast<const float4*>(fbuf + 4 * i);
-                    const float4 y = __ldcg(reinterpret_cast<const float4*>(xk) + v);
+                    const float4 y = *reinterpret_cast<const float4*>(xp_s + 4 * v);
                     x.x = fmaf(f, y.x, x.x); x.y = fmaf(f, y.y, x.y); x.z = fmaf(f, y.z, x.z); x.w = fmaf(f, y.w, x.w);
                     *reinterpret_cast<float4*>(fbuf + 4 * i) = x;
                     *reinterpret_cast<float4*>(ckg + 4 * i) = x;
@@ -1310,29 +1325,17 @@ __global__ void __launch_bounds__(kThreads, 1) decode_fft_kernel(const __grid_co
     }
     cp_async_wait_all();
     consumer_sync();
-    if (step && s.dcv > 0) {                               // fused step: pending rank-1 update of this part's rows of C^V
-        const int j_pend = ws.pend_j[b];
-        if (j_pend >= 0) {
-            const float* xv = ws.pend + ((size_t)b * s.Hkv + h) * (s.dck + s.dcv) + s.dck;
-            float* cvg = coef_rows(c.coef_v, s, b, h, s.dcv) + (size_t)m0 * s.dcv;
-            float* f_s = ps_s;                             // basis column j for this part's rows (ps_s is not in use yet)
+    if (j_pend >= 0 && s.dcv > 0) {                        // fused step: pending rank-1 update of this part's rows of C^V
+        float* cvg = coef_rows(c.coef_v, s, b, h, s.dcv) + (size_t)m0 * s.dcv;
 #pragma unroll 1
-            for (int r = tid; r < rows; r += kConsumers) {
-                float cs, sn;
-                basis_cs((m0 + r) >> 1, j_pend, s.T, &cs, &sn);
-                f_s[r] = ((m0 + r) & 1) ? sn : cs;
-            }
-            consumer_sync();
-#pragma unroll 1
-            for (int i = tid; i < rows * nv; i += kConsumers) {
-                const int r = i / nv, v = i - r * nv;
-                const float f = f_s[r];
-                float4 x = *reinterpret_cast<const float4*>(cv_s + 4 * i);
-                const float4 y = __ldcg(reinterpret_cast<const float4*>(xv) + v);
-                x.x = fmaf(f, y.x, x.x); x.y = fmaf(f, y.y, x.y); x.z = fmaf(f, y.z, x.z); x.w = fmaf(f, y.w, x.w);
-                *reinterpret_cast<float4*>(cv_s + 4 * i) = x;
-                *reinterpret_cast<float4*>(cvg + 4 * i) = x;
-            }
+        for (int i = tid; i < rows * nv; i += kConsumers) {
+            const int r = i / nv, v = i - r * nv;
+            const float f = f_row(r);
+            float4 x = *reinterpret_cast<const float4*>(cv_s + 4 * i);
+            const float4 y = *reinterpret_cast<const float4*>(xp_s + s.dck + 4 * v);
+            x.x = fmaf(f, y.x, x.x); x.y = fmaf(f, y.y, x.y); x.z = fmaf(f, y.z, x.z); x.w = fmaf(f, y.w, x.w);
+            *reinterpret_cast<float4*>(cv_s + 4 * i) = x;
+            *reinterpret_cast<float4*>(cvg + 4 * i) = x;
         }
     }
     if (warp < GH) {                                       // one warp per head, lanes over the parts
