@@ -177,7 +177,10 @@ fa_status fa_decode_step(const fa_layout* layout, fa_cache* cache, const void* q
  * `staging`, runs fa_decode_step, and copies the result to out_host
  * [B][H_q][d].  `staging` is caller-owned device memory of at least
  * fa_step_staging_bytes(layout) bytes; k_new_host == NULL skips the append.  Asynchronous on
- * `stream`: out_host is valid after the stream is synchronised. */
+ * `stream`: out_host is valid after the stream is synchronised.  Host buffers that the device can
+ * address (pinned or registered memory, 16-byte aligned) are not copied by separate copy
+ * operations: one staging kernel reads q, k_new, v_new over the bus, and the decode kernel writes
+ * its result rows straight into out_host. */
 fa_status fa_decode_step_host(const fa_layout* layout, fa_cache* cache, const void* q_host,
                               const void* k_new_host, const void* v_new_host, void* out_host,
                               void* staging, void* ws, size_t ws_bytes, void* stream);

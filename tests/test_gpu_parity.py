@@ -291,3 +291,27 @@ def test_decode_step_full_middle_reports_capacity():
     want = pair.ref.decode(to64(q))                       # the oracle cache did not take the token either
     assert np.abs(to64(out) - want).max() <= 2e-2
     pair.check_state()
+
+
+@pytest.mark.parametrize("pinned", [True, False])
+def test_decode_step_host_buffers(pinned):
+    """The host-buffer step (pinned buffers are read by a staging kernel, pageable ones copied) gives the
+    same outputs and cache as the oracle's append + decode."""
+    shape = SMALL_BF16.with_(L=400, decode_steps=6)
+    pair, stream = make_pair(shape, seed=15, algo=fa.FA_DECODE_FFT, P=16)
+    staging = torch.zeros(fa.fa_step_staging_bytes(pair.layout), dtype=torch.uint8, device="cuda")
+    K, V = stream.tokens(shape.L, shape.L + 6)
+
+    def host(t):
+        t = t.contiguous().cpu()
+        return t.pin_memory() if pinned else t
+
+    for t in range(6):
+        q = synth.queries(shape, seed=15, step=t)
+        out_h = host(torch.zeros_like(q))
+        fa.fa_decode_step_host(pair.layout, pair.gpu, host(q), host(K[:, t]), host(V[:, t]), out_h, staging, pair.ws)
+        torch.cuda.synchronize()
+        pair.ref.append(to64(K[:, t]), to64(V[:, t]))
+        want = pair.ref.decode(to64(q))
+        assert np.abs(to64(out_h) - want).max() <= 2e-2
+    pair.check_state()
