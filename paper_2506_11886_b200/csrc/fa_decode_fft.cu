@@ -1023,6 +1023,17 @@ __global__ void __launch_bounds__(kThreads, 1) decode_fft_kernel(const __grid_co
             }
         }
         const uint32_t p_lane = smem_addr(pbt) + (uint32_t)((gq & (GH - 1)) * pbs + 2 * tq) * 2;
+        // natural positions of this lane's output rows (D^vu), fetched long before they are needed
+        int o_idx[4][2];
+        {
+            const int32_t* idf_v = c.idx_full_v + (size_t)h * s.nfv;
+#pragma unroll
+            for (int mt = 0; mt < 4; ++mt) {
+                const int e_lo = 16 * mt + gq, e_hi = e_lo + 8;
+                o_idx[mt][0] = e_lo < s.nfv ? idf_v[e_lo] : -1;
+                o_idx[mt][1] = e_hi < s.nfv ? idf_v[e_hi] : -1;
+            }
+        }
 
         #pragma unroll 1
         for (int cb = c0; cb < c1; cb += NB) {
@@ -1227,20 +1238,16 @@ __global__ void __launch_bounds__(kThreads, 1) decode_fft_kernel(const __grid_co
             consumer_sync();
         }
         // fold the per-warp output fragments into o_s at the natural positions of D^vu
-        const int32_t* idf_v = c.idx_full_v + (size_t)h * s.nfv;
         if (2 * tq < GH) {
             float* o_lo = o_s + hperm<GH>(2 * tq) * s.d;
             float* o_hi = o_s + hperm<GH>(2 * tq + 1) * s.d;
 #pragma unroll
             for (int mt = 0; mt < 4; ++mt) {
-                const int e_lo = 16 * mt + gq, e_hi = e_lo + 8;
-                if (e_lo < s.nfv) { atomicAdd(o_lo + idf_v[e_lo], acc[mt][0]); atomicAdd(o_hi + idf_v[e_lo], acc[mt][1]); }
-                if (e_hi < s.nfv) { atomicAdd(o_lo + idf_v[e_hi], acc[mt][2]); atomicAdd(o_hi + idf_v[e_hi], acc[mt][3]); }
+                if (o_idx[mt][0] >= 0) { atomicAdd(o_lo + o_idx[mt][0], acc[mt][0]); atomicAdd(o_hi + o_idx[mt][0], acc[mt][1]); }
+                if (o_idx[mt][1] >= 0) { atomicAdd(o_lo + o_idx[mt][1], acc[mt][2]); atomicAdd(o_hi + o_idx[mt][1], acc[mt][3]); }
             }
         }
     }
-    consumer_sync();
-
     // sum of p per slot
 #pragma unroll
     for (int g = 0; g < GH; ++g) {
