@@ -78,3 +78,39 @@ def test_null_arguments():
     lay = _layout().c()
     assert lib.fa_decode_attention(C.byref(lay), None, None, None, None, 0, None) == fa.FA_ERR_INVALID_ARG
     assert lib.fa_append(C.byref(lay), None, None, None, None) == fa.FA_ERR_INVALID_ARG
+
+
+def test_launch_plan_is_host_logic():
+    """Which form a decode call takes is decided on the host from the layout alone: one fused
+    cooperative kernel while every (batch row, KV head) can have two CTAs resident, three kernels past
+    that or when asked for; the fused step (light append + decode) needs the fused kernel."""
+    lib = fa.lib()
+
+    def launches(what, **kw):
+        return lib.fa_launch_count(C.byref(_layout(**kw).c()), what)
+
+    assert launches(0) == 2 and launches(1) == 1
+    assert launches(2) == 1 and launches(3) == 2                                   # 8 KV heads: 18 CTAs each
+    assert launches(2, decode_algo=fa.FA_DECODE_FFT_SPLIT) == 3 and launches(3, decode_algo=fa.FA_DECODE_FFT_SPLIT) == 4
+    assert launches(2, decode_algo=fa.FA_DECODE_DIRECT) == 3
+    assert launches(2, batch=16) == 3                                              # 128 pairs: more than half the SMs
+    assert launches(2, kv_dtype=fa.FA_F32) == 3                                    # fp32 caches take the direct kernel
+    assert launches(3, n_q_heads=64) in (2, 4)                                      # 8 query heads per KV head: two passes
+    assert launches(99) == 0
+    # the workspace grows with the number of partial results but stays far below the static limit's order
+    small, big = fa.fa_workspace_bytes(_layout()), fa.fa_workspace_bytes(_layout(batch=8))
+    assert 0 < small < big
+
+
+def test_select_workspace_and_null_arguments():
+    lib = fa.lib()
+    out = C.c_size_t(0)
+    lay = _layout().c()
+    assert lib.fa_select_workspace_bytes(C.byref(lay), C.byref(out)) == fa.FA_OK
+    # coefficients of all 128 dims of K and V: 2 * 8 heads * 1024 rows * 128 dims * 4 bytes, plus windows and scratch
+    assert out.value >= 2 * 8 * 1024 * 128 * 4
+    assert lib.fa_select_workspace_bytes(C.byref(lay), None) == fa.FA_ERR_INVALID_ARG
+    odd = _layout(head_dim=96, n_full_k=32, n_full_v=32).c()
+    assert lib.fa_select_workspace_bytes(C.byref(odd), C.byref(out)) == fa.FA_ERR_UNSUPPORTED
+    assert lib.fa_select_dims(C.byref(lay), None, None, 0, 0, 0, 5, None, None, None, None, None, None, 0, None) == fa.FA_ERR_INVALID_ARG
+    assert lib.fa_decode_step(C.byref(lay), None, None, None, None, None, None, 0, None) == fa.FA_ERR_INVALID_ARG
