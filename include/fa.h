@@ -144,6 +144,15 @@ fa_status fa_compress(const fa_layout* layout, fa_cache* cache, const void* K, c
                       int64_t stride_b, int64_t stride_t, int64_t stride_h, int32_t L,
                       void* ws, size_t ws_bytes, void* stream);
 
+/* fa_compress for a batch whose rows have different prompt lengths: row b is compressed from its
+ * first lengths[b] tokens (HOST array of B entries, each 0 <= lengths[b] and within the capacity rule
+ * of fa_compress; K / V rows beyond a row's length are not read).  Every row becomes what a one-row
+ * fa_compress would make of it; fa_append, fa_decode_attention and fa_decode_step then work on the
+ * ragged batch as on any other (the token counters are per batch row). */
+fa_status fa_compress_ragged(const fa_layout* layout, fa_cache* cache, const void* K, const void* V,
+                             int64_t stride_b, int64_t stride_t, int64_t stride_h, const int32_t* lengths,
+                             void* ws, size_t ws_bytes, void* stream);
+
 /* Eq.5.  k_new, v_new: [B][H_kv][d].  The token goes to the init window while that has
  * room, else to the local window; when the local window is full its oldest token leaves:
  * its D^u dims are appended to K^mu / V^mu and its D^c dims are added to the coefficients

@@ -321,6 +321,40 @@ fa_status fa_compress(const fa_layout* layout, fa_cache* cache, const void* K, c
     return FA_OK;
 }
 
+fa_status fa_compress_ragged(const fa_layout* layout, fa_cache* cache, const void* K, const void* V, int64_t stride_b,
+                             int64_t stride_t, int64_t stride_h, const int32_t* lengths, void* ws, size_t ws_bytes,
+                             void* stream) {
+    fa_status st = check_layout(layout);
+    if (st != FA_OK) return st;
+    st = check_cache(layout, cache);
+    if (st != FA_OK) return st;
+    if (!lengths || stride_b < 0) return FA_ERR_INVALID_ARG;
+    // every batch row is a one-row cache of its own: same index sets and status word, its own slices
+    fa_layout one = *layout;
+    one.batch = 1;
+    fa_cache_sizes sz;
+    st = fa_cache_sizes_of(&one, &sz);
+    if (st != FA_OK) return st;
+    const size_t eb = elt_bytes(layout->kv_dtype);
+    for (int b = 0; b < layout->batch; ++b) {
+        if (lengths[b] < 0) return FA_ERR_INVALID_ARG;
+        fa_cache row = *cache;
+        auto at = [&](void* p, size_t bytes) -> void* { return p ? static_cast<char*>(p) + (size_t)b * bytes : nullptr; };
+        row.k_init = at(cache->k_init, sz.k_init);     row.v_init = at(cache->v_init, sz.v_init);
+        row.k_local = at(cache->k_local, sz.k_local);  row.v_local = at(cache->v_local, sz.v_local);
+        row.k_mid = at(cache->k_mid, sz.k_mid);        row.v_mid = at(cache->v_mid, sz.v_mid);
+        row.coef_k = static_cast<float*>(at(cache->coef_k, sz.coef_k));
+        row.coef_v = static_cast<float*>(at(cache->coef_v, sz.coef_v));
+        row.state = static_cast<int32_t*>(at(cache->state, sz.state));
+        const char* Kb = static_cast<const char*>(K) + (size_t)b * (size_t)stride_b * eb;
+        const char* Vb = static_cast<const char*>(V) + (size_t)b * (size_t)stride_b * eb;
+        st = fa_compress(&one, &row, lengths[b] ? Kb : (K ? Kb : nullptr), lengths[b] ? Vb : (V ? Vb : nullptr), stride_b, stride_t,
+                         stride_h, lengths[b], ws, ws_bytes, stream);
+        if (st != FA_OK) return st;
+    }
+    return FA_OK;
+}
+
 fa_status fa_append(const fa_layout* layout, fa_cache* cache, const void* k_new, const void* v_new, void* stream) {
     fa_status st = check_layout(layout);
     if (st != FA_OK) return st;

@@ -67,6 +67,7 @@ def lib() -> C.CDLL:
         L.fa_validate.argtypes = [lp, cp, vp]
         L.fa_compress.argtypes = [lp, cp, vp, vp, i64, i64, i64, i32, vp, sz, vp]
         L.fa_append.argtypes = [lp, cp, vp, vp, vp]
+        L.fa_compress_ragged.argtypes = [lp, cp, vp, vp, i64, i64, i64, C.POINTER(C.c_int32), vp, sz, vp]
         L.fa_decode_attention.argtypes = [lp, cp, vp, vp, vp, sz, vp]
         L.fa_poll_status.argtypes = [cp, vp]
         L.fa_decode_step_host.argtypes = [lp, cp, vp, vp, vp, vp, vp, vp, sz, vp]
@@ -80,7 +81,7 @@ def lib() -> C.CDLL:
         L.fa_status_string.restype = C.c_char_p
         for name in ("fa_cache_sizes_of", "fa_workspace_bytes", "fa_cache_reset", "fa_validate", "fa_compress",
                      "fa_append", "fa_decode_attention", "fa_poll_status", "fa_launch_count", "fa_version",
-                     "fa_decode_step_host", "fa_decode_step", "fa_select_workspace_bytes", "fa_select_dims"):
+                     "fa_decode_step_host", "fa_decode_step", "fa_select_workspace_bytes", "fa_select_dims", "fa_compress_ragged"):
             getattr(L, name).restype = C.c_int
         _lib = L
     return _lib
@@ -220,6 +221,16 @@ def fa_compress(layout: Layout, cache: Cache, K: torch.Tensor, V: torch.Tensor, 
         sb = 0
     _check(lib().fa_compress(C.byref(layout.c()), C.byref(cache.c()), _ptr(K), _ptr(V), sb, st, sh, L,
                              _ptr(ws), ws.numel(), _stream(stream)), "fa_compress")
+
+
+def fa_compress_ragged(layout: Layout, cache: Cache, K: torch.Tensor, V: torch.Tensor, lengths, ws: torch.Tensor,
+                       stream=None) -> None:
+    """fa_compress with a prompt length per batch row (lengths: B ints, each <= K.shape[1])."""
+    assert K.is_cuda and V.is_cuda and K.dtype == layout.torch_dtype and K.shape == V.shape and K.stride() == V.stride()
+    assert K.stride(3) == 1 and len(lengths) == layout.batch and max(lengths) <= K.shape[1]
+    arr = (C.c_int32 * layout.batch)(*[int(x) for x in lengths])
+    _check(lib().fa_compress_ragged(C.byref(layout.c()), C.byref(cache.c()), _ptr(K), _ptr(V), K.stride(0), K.stride(1),
+                                    K.stride(2), arr, _ptr(ws), ws.numel(), _stream(stream)), "fa_compress_ragged")
 
 
 def fa_append(layout: Layout, cache: Cache, k_new: torch.Tensor, v_new: torch.Tensor, stream=None) -> None:

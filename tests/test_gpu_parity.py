@@ -315,3 +315,50 @@ def test_decode_step_host_buffers(pinned):
         want = pair.ref.decode(to64(q))
         assert np.abs(to64(out_h) - want).max() <= 2e-2
     pair.check_state()
+
+
+def test_ragged_batch_compress_append_decode():
+    """Rows of one batch with different prompt lengths: each row must behave as a one-row cache of its own
+    (oracle: one cache per row), through compression, steps that evict in one row and not in the other,
+    and decode."""
+    from oracle import fa_oracle as fo
+    from tests.parity_util import oracle_cfg
+    shape = SMALL_BF16.with_(B=2, L=1200, T=2048, M=128)
+    layout = layout_of(shape, max_mid=2048, P=16, algo=fa.FA_DECODE_FFT)
+    stream = synth.KVStream(shape, seed=16)
+    K, V = stream.tokens(0, 1200)
+    lengths = [1200, 37]                                    # the second row has not even filled its local window
+    try:
+        gpu = fa.Cache(layout, stream.idx_full_k, stream.idx_full_v)
+        ws = fa.new_workspace(layout)
+        fa.fa_compress_ragged(layout, gpu, K.cuda(), V.cuda(), lengths, ws)
+    except fa.FaError as e:
+        if e.status == fa.FA_ERR_UNSUPPORTED:
+            pytest.skip("layout outside the FFT kernel's range")
+        raise
+    refs = []
+    for b in range(2):
+        import dataclasses
+        cfg = dataclasses.replace(oracle_cfg(layout), B=1)
+        r = fo.OracleCache(cfg, stream.idx_full_k.numpy(), stream.idx_full_v.numpy())
+        r.compress(to64(K[b:b + 1, :lengths[b]]), to64(V[b:b + 1, :lengths[b]]))
+        refs.append(r)
+    st = gpu.state.cpu().numpy()
+    for b in range(2):
+        assert (st[b, 0], st[b, 1], st[b, 2]) == (refs[b].n_init[0], refs[b].n_local[0], refs[b].n_mid[0])
+    Kn, Vn = stream.tokens(1200, 1240)
+    for t in range(40):                                      # row 0 evicts every step, row 1 fills its window then evicts
+        q = synth.queries(shape, seed=16, step=t)
+        out = torch.full_like(q, float("nan"), device="cuda")
+        fa.fa_decode_step(layout, gpu, q.cuda().contiguous(), Kn[:, t].cuda().contiguous(), Vn[:, t].cuda().contiguous(), out, ws)
+        torch.cuda.synchronize()
+        for b in range(2):
+            refs[b].append(to64(Kn[b:b + 1, t]), to64(Vn[b:b + 1, t]))
+            want = refs[b].decode(to64(q[b:b + 1]))
+            assert np.abs(to64(out[b:b + 1]) - want).max() <= 2e-2, (t, b)
+    assert fa.fa_poll_status(gpu) == fa.FA_OK
+    st = gpu.state.cpu().numpy()
+    for b in range(2):
+        assert (st[b, 0], st[b, 1], st[b, 2]) == (refs[b].n_init[0], refs[b].n_local[0], refs[b].n_mid[0])
+        den = np.abs(refs[b].coef_k[0]).max()
+        assert np.abs(to64(gpu.coef_k[b]) - refs[b].coef_k[0]).max() / max(den, 1e-30) <= 1e-3
