@@ -62,13 +62,25 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* b, uint32_t parity) {
         : "memory");
     return ok != 0;
 }
-// Bounded wait: gives up after kSpinLimit polls, records the failure, never hangs.
-__device__ __forceinline__ void mbar_wait(uint64_t* b, uint32_t parity, volatile int* fail, int32_t* status) {
+// Bounded wait: gives up after kSpinLimit polls, records the failure, never hangs.  The common case
+// (the phase is already complete) is one inlined test; the polling loop is a call, so that the many
+// wait sites do not bloat the kernel (its code is fetched cold: every phase runs once per CTA).
+__device__ __noinline__ void mbar_wait_slow(uint64_t* b, uint32_t parity, volatile int* fail, int32_t* status) {
     if (*fail) return;
     for (uint32_t i = 0; i < kSpinLimit; ++i)
         if (mbar_try_wait(b, parity)) return;
     *fail = 1;
     atomicExch(status, (int)FA_ERR_TIMEOUT);
+}
+__device__ __forceinline__ void mbar_wait(uint64_t* b, uint32_t parity, volatile int* fail, int32_t* status) {
+    if (mbar_try_wait(b, parity)) return;
+    mbar_wait_slow(b, parity, fail, status);
+}
+// Eq.4 for one (row, column): a call, for the same reason.
+__device__ __noinline__ float basis_value(int m, int j, int T) {
+    float cs, sn;
+    basis_cs(m >> 1, j, T, &cs, &sn);
+    return (m & 1) ? sn : cs;
 }
 __device__ __forceinline__ void bulk_g2s(void* dst, const void* src, uint32_t bytes, uint64_t* bar) {
     asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
@@ -582,18 +594,11 @@ __global__ void __launch_bounds__(kThreads, 1) decode_fft_kernel(const __grid_co
         const float* xp = ws.pend + ((size_t)b * s.Hkv + h) * (s.dck + s.dcv);
         for (int i = tid; i < (s.dck + s.dcv) >> 2; i += kConsumers) cp_async16(xp_s + 4 * i, xp + 4 * i);
 #pragma unroll 1
-        for (int r = tid; r < min(m1 - m0, kPendRows); r += kConsumers) {
-            float cs, sn;
-            basis_cs((m0 + r) >> 1, j_pend, s.T, &cs, &sn);
-            f_s[r] = ((m0 + r) & 1) ? sn : cs;
-        }
+        for (int r = tid; r < min(m1 - m0, kPendRows); r += kConsumers) f_s[r] = basis_value(m0 + r, j_pend, s.T);
     }
     // basis value of row r of this part (tabulated for the first kPendRows rows)
     auto f_row = [&](int r) -> float {
-        if (r < kPendRows) return f_s[r];
-        float cs, sn;
-        basis_cs((m0 + r) >> 1, j_pend, s.T, &cs, &sn);
-        return ((m0 + r) & 1) ? sn : cs;
+        return r < kPendRows ? f_s[r] : basis_value(m0 + r, j_pend, s.T);
     };
 
     // B fragments of q for the kept K dims: column gq is slot gq = head hperm(gq);
