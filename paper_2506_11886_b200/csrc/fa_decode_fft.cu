@@ -1373,7 +1373,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_fft_kernel(const __grid_co
             float v = 0.f;
             if (g < ng) {
                 const float* z = zs_s + g * np * rows_max + r;
-#pragma unroll 6
+#pragma unroll 2
                 for (int sp = 0; sp < np; ++sp) v = fmaf(al_s[g * np + sp], z[sp * rows_max], v);
                 v *= recon_weight(s.norm, m0 + r, s.k, s.T);
             }
@@ -1385,7 +1385,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_fft_kernel(const __grid_co
             float4 acc4[GH];
 #pragma unroll
             for (int g = 0; g < GH; ++g) acc4[g] = make_float4(0.f, 0.f, 0.f, 0.f);
-#pragma unroll 3
+#pragma unroll 1
             for (int r = rgi; r < rows; r += nrg) {
                 const float4 x = *reinterpret_cast<const float4*>(cv_s + r * s.dcv + 4 * v);
 #pragma unroll
@@ -1445,13 +1445,13 @@ __global__ void __launch_bounds__(kThreads, 1) decode_fft_kernel(const __grid_co
         const int g = t / s.d, e = t - g * s.d;
         const float* o = op_s + g * np * s.d + e;
         float v = 0.f;
-#pragma unroll 6
+#pragma unroll 2
         for (int sp = 0; sp < np; ++sp) v = fmaf(al_s[g * np + sp], o[sp * s.d], v);
         const int slot = inv_s[e];
         if (slot >= 0) {
             const float* oc = ocp_s + g * np * s.dcv + slot;
             float w = 0.f;
-#pragma unroll 6
+#pragma unroll 2
             for (int x = 0; x < np; ++x) w += oc[x * s.dcv];
             v += w;
         }
