@@ -18,8 +18,19 @@
 // consumer warps feed the tiles to mma.sync (bf16 x bf16 -> fp32; exact for q . K, p rounded to
 // bf16 for p . V): K fragments are read with 128-bit loads using the freedom to permute the
 // contraction index, V^T fragments with transposing 8x8 matrix loads, conflict-free because
-// V^mu rows are stored chunk-swizzled.  Window rows (init + local ring) are copied row by row
-// into padded shared-memory rows and take the same route.  Every wait is bounded.
+// V^mu rows are stored chunk-swizzled.  Window rows (init + local ring) arrive as tiled TMA
+// boxes with the 128-byte swizzle from tensor maps of the window buffers and take the same
+// route.  Every wait is bounded.
+//
+// Two forms, chosen by the host plan.  Three kernels: a prologue kernel forms u = W C^K q, this
+// kernel writes per-part partial results (m, l, o, z), an epilogue kernel merges them and applies
+// C^V.  Fused (one cooperative launch per call): the parts of a (batch row, KV head) each form a
+// slice of the rows of u and exchange it through the workspace behind a counter barrier, window
+// tokens have parts of their own, and after a second barrier every part merges its slice of the
+// coefficient rows (its rows of every part's z against its rows of C^V); the last part to take
+// a ticket adds the slices in a fixed order and writes the output rows.  As the second half of
+// fa_decode_step the fused kernel also adds the pending rank-1 update of Eq.5 to the coefficient
+// rows it stages and writes them back.
 //
 // "Slot" below is the position of a head inside a point / an mma column: slot s holds head
 // hperm(s) = {0, 2, 1, 3}[s] (GH = 4) so that the packed real parts are slots 0, 1 and the
@@ -127,7 +138,6 @@ __device__ __forceinline__ void part_wait(const int32_t* cnt, int n, int tid, vo
     }
     consumer_sync();
 }
-__device__ __forceinline__ float ldcg_f(const float* p) { return __ldcg(p); }
 
 __device__ __forceinline__ void mma_bf16(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0,
                                          uint32_t b1) {
@@ -483,7 +493,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_fft_kernel(const __grid_co
     const int w0 = has_win ? wi * n_win / wn : 0, w1 = has_win ? (wi + 1) * n_win / wn : 0;
     auto n_of_class = [&](int cls) { return cls < n_mid ? (n_mid - cls + s.P - 1) >> log2P : 0; };
 
-    const int rowb_k = s.nfk * 2, rowb_v = s.nfv * 2, rowb_w = s.d * 2;
+    const int rowb_k = s.nfk * 2, rowb_v = s.nfv * 2;
     const int nhalf = (s.d + 63) >> 6;                                     // 64-dim boxes per window row
     const int ts_k = rowb_k ? (kStageBytes / rowb_k) & ~15 : 0, ts_v = rowb_v ? (kStageBytes / rowb_v) & ~15 : 0;
     const int ts_w = kWinRowsPerTile;
