@@ -589,11 +589,13 @@ __global__ void __launch_bounds__(kThreads, 1) decode_fft_kernel(const __grid_co
         const int g = tid / s.dck, e = tid - g * s.dck;
         if (g < ng) qc_early = __bfloat162float(q[((size_t)b * s.Hq + g_first + g) * s.d + c.idx_comp_k[(size_t)h * s.dck + e]]);
     }
+    // rows of C^K the transform buffers hold at a time (all of this part's rows unless the batch is large)
+    const int uch = s.dck > 0 ? ((NB * L.fb_floats) / s.dck) & ~3 : 0;
     if (p.fused && s.dck > 0) {
         // this part's rows of C^K go to the (still unused) transform buffers while the tables are built
         const float* ck = coef_rows(c.coef_k, s, b, h, s.dck) + (size_t)m0 * s.dck;
 #pragma unroll 1
-        for (int i = tid; i < (m1 - m0) * (s.dck >> 2); i += kConsumers) cp_async16(fbuf + 4 * i, ck + 4 * i);
+        for (int i = tid; i < min(m1 - m0, uch) * (s.dck >> 2); i += kConsumers) cp_async16(fbuf + 4 * i, ck + 4 * i);
     }
     // fused step: the coefficient update the light append kernel left pending (basis column j_pend, or -1);
     // the leaving row's compressed dims and the basis values of this part's rows are fetched / formed now
@@ -712,54 +714,63 @@ __global__ void __launch_bounds__(kThreads, 1) decode_fft_kernel(const __grid_co
                 const int g = i / s.dck, e = i - g * s.dck;
                 qc[i] = i < kConsumers ? qc_early : (g < ng ? __bfloat162float(q[((size_t)b * s.Hq + g_first + g) * s.d + idc_k[e]]) : 0.f);
             }
-            cp_async_wait_all();
-            consumer_sync();
             const int l8 = tid & 7, rgi = tid >> 3, nv = s.dck >> 2;
-            // fused step: the rank-1 update of Eq.5 that the light append kernel left pending, applied to
-            // this part's rows while they are on chip, and written back
-            if (j_pend >= 0) {
-                float* ckg = coef_rows(c.coef_k, s, b, h, s.dck) + (size_t)m0 * s.dck;
+            float* ckg = coef_rows(c.coef_k, s, b, h, s.dck);
 #pragma unroll 1
-                for (int i = tid; i < (m1 - m0) * nv; i += kConsumers) {
-                    const int r = i / nv, v = i - r * nv;
-                    const float f = f_row(r);
-                    float4 x = *reinterpret_cast<const float4*>(fbuf + 4 * i);
-                    const float4 y = *reinterpret_cast<const float4*>(xp_s + 4 * v);
-                    x.x = fmaf(f, y.x, x.x); x.y = fmaf(f, y.y, x.y); x.z = fmaf(f, y.z, x.z); x.w = fmaf(f, y.w, x.w);
-                    *reinterpret_cast<float4*>(fbuf + 4 * i) = x;
-                    *reinterpret_cast<float4*>(ckg + 4 * i) = x;
+            for (int q0 = m0; q0 < m1; q0 += uch) {         // chunks of rows staged in the transform buffers
+                const int q1 = min(m1, q0 + uch);
+                if (q0 > m0) {
+                    consumer_sync();
+#pragma unroll 1
+                    for (int i = tid; i < (q1 - q0) * nv; i += kConsumers) cp_async16(fbuf + 4 * i, ckg + (size_t)q0 * s.dck + 4 * i);
                 }
+                cp_async_wait_all();
                 consumer_sync();
-            }
-            #pragma unroll 1
-            for (int r0 = m0; r0 < m1; r0 += kConsumers / 8) {
-                const int r = r0 + rgi;
-                float a[GH];
+                // fused step: the rank-1 update of Eq.5 that the light append kernel left pending, applied to
+                // this part's rows while they are on chip, and written back
+                if (j_pend >= 0) {
+#pragma unroll 1
+                    for (int i = tid; i < (q1 - q0) * nv; i += kConsumers) {
+                        const int r = i / nv, v = i - r * nv;
+                        const float f = f_row(q0 - m0 + r);
+                        float4 x = *reinterpret_cast<const float4*>(fbuf + 4 * i);
+                        const float4 y = *reinterpret_cast<const float4*>(xp_s + 4 * v);
+                        x.x = fmaf(f, y.x, x.x); x.y = fmaf(f, y.y, x.y); x.z = fmaf(f, y.z, x.z); x.w = fmaf(f, y.w, x.w);
+                        *reinterpret_cast<float4*>(fbuf + 4 * i) = x;
+                        *reinterpret_cast<float4*>(ckg + (size_t)q0 * s.dck + 4 * i) = x;
+                    }
+                    consumer_sync();
+                }
+#pragma unroll 1
+                for (int r0 = q0; r0 < q1; r0 += kConsumers / 8) {
+                    const int r = r0 + rgi;
+                    float a[GH];
 #pragma unroll
-                for (int g = 0; g < GH; ++g) a[g] = 0.f;
-                if (r < m1) {
-                    const float4* row = reinterpret_cast<const float4*>(fbuf + (r - m0) * s.dck);
-                    #pragma unroll 1
-                    for (int v = l8; v < nv; v += 8) {
-                        const float4 x = row[v];
+                    for (int g = 0; g < GH; ++g) a[g] = 0.f;
+                    if (r < q1) {
+                        const float4* row = reinterpret_cast<const float4*>(fbuf + (r - q0) * s.dck);
+#pragma unroll 1
+                        for (int v = l8; v < nv; v += 8) {
+                            const float4 x = row[v];
 #pragma unroll
-                        for (int g = 0; g < GH; ++g) {
-                            const float4 y = *reinterpret_cast<const float4*>(qc + g * s.dck + 4 * v);
-                            a[g] = fmaf(x.x, y.x, fmaf(x.y, y.y, fmaf(x.z, y.z, fmaf(x.w, y.w, a[g]))));
+                            for (int g = 0; g < GH; ++g) {
+                                const float4 y = *reinterpret_cast<const float4*>(qc + g * s.dck + 4 * v);
+                                a[g] = fmaf(x.x, y.x, fmaf(x.y, y.y, fmaf(x.z, y.z, fmaf(x.w, y.w, a[g]))));
+                            }
                         }
                     }
-                }
 #pragma unroll
-                for (int g = 0; g < GH; ++g) {
-                    a[g] += __shfl_xor_sync(0xffffffffu, a[g], 1);
-                    a[g] += __shfl_xor_sync(0xffffffffu, a[g], 2);
-                    a[g] += __shfl_xor_sync(0xffffffffu, a[g], 4);
-                }
-                float mine = a[0];
+                    for (int g = 0; g < GH; ++g) {
+                        a[g] += __shfl_xor_sync(0xffffffffu, a[g], 1);
+                        a[g] += __shfl_xor_sync(0xffffffffu, a[g], 2);
+                        a[g] += __shfl_xor_sync(0xffffffffu, a[g], 4);
+                    }
+                    float mine = a[0];
 #pragma unroll
-                for (int g = 1; g < GH; ++g) if (l8 == g) mine = a[g];
-                if (r < m1 && l8 < ng)
-                    ws.u[((size_t)b * s.Hq + g_first + l8) * s.M + r] = recon_weight(s.norm, r, s.k, s.T) * sl2 * mine;
+                    for (int g = 1; g < GH; ++g) if (l8 == g) mine = a[g];
+                    if (r < q1 && l8 < ng)
+                        ws.u[((size_t)b * s.Hq + g_first + l8) * s.M + r] = recon_weight(s.norm, r, s.k, s.T) * sl2 * mine;
+                }
             }
             part_arrive(bar + 0, tid);
         }
@@ -1310,34 +1321,31 @@ __global__ void __launch_bounds__(kThreads, 1) decode_fft_kernel(const __grid_co
     // of 16-byte asynchronous copies into the stage ring (every tile has been consumed), so each
     // step costs one memory round trip.
     const int np = p.n_part;
-    const int rows = m1 - m0, rows_max = (s.M / 4 + np - 1) / np * 4 + 4;
+    const int rows = m1 - m0;
     const size_t qh0 = (size_t)b * s.Hq + g_first;
+    const int nv = s.dcv >> 2, nrg = nv ? kConsumers / nv : 0;
+    // rows of the slice handled at a time: what the stage ring holds of C^V rows, z slices and weighted z
+    constexpr int kRing = kStages * kStageBytes / 4;
+    const int head_f = (2 * GH * np + GH + 3) & ~3;
+    const int mch = max(4, min((rows + 3) & ~3, ((kRing - head_f - nrg * GH * s.dcv) / (GH + s.dcv + GH * np)) & ~3));
     float* al_s = reinterpret_cast<float*>(stages);        // [GH][np] maxima, then exp2(m - max)
     float* l_s = al_s + GH * np;                           // [GH][np]
     float* linv_s = l_s + GH * np;                         // [GH]
-    float* zw_s = al_s + ((2 * GH * np + GH + 3) & ~3);    // [GH][rows_max]
-    float* big_s = zw_s + GH * rows_max;                   // step 1: C^V rows, z slices, partial sums; step 2: o and o^c parts
-    float* cv_s = big_s;                                   // [rows][dcv]
-    float* zs_s = cv_s + rows_max * s.dcv;                 // [GH][np][rows_max]
-    float* ps_s = zs_s + GH * np * rows_max;               // [row groups][GH][dcv]
+    float* zw_s = al_s + head_f;                           // [GH][mch]
+    float* big_s = zw_s + GH * mch;                        // step 1: C^V rows, z slices, partial sums; step 2: o and o^c parts
+    float* cv_s = big_s;                                   // [mch][dcv]
+    float* zs_s = cv_s + mch * s.dcv;                      // [GH][np][mch]
+    float* ps_s = zs_s + GH * np * mch;                    // [row groups][GH][dcv]
     volatile int* last_s = fail + 1;
-    const int nv = s.dcv >> 2, nrg = nv ? kConsumers / nv : 0;
-
-    if (s.dcv > 0) {
-        const float* cv = coef_rows(c.coef_v, s, b, h, s.dcv) + (size_t)m0 * s.dcv;
+    float* cvg = s.dcv > 0 ? coef_rows(c.coef_v, s, b, h, s.dcv) + (size_t)m0 * s.dcv : nullptr;
+    auto stage_cv = [&](int r0, int cr) {
 #pragma unroll 1
-        for (int i = tid; i < rows * nv; i += kConsumers) cp_async16(cv_s + 4 * i, cv + 4 * i);
-    }
+        for (int i = tid; i < cr * nv; i += kConsumers) cp_async16(cv_s + 4 * i, cvg + (size_t)r0 * s.dcv + 4 * i);
+    };
+
+    if (s.dcv > 0) stage_cv(0, min(rows, mch));            // under the barrier
     part_arrive(bar + 1, tid);
     part_wait(bar + 1, np, tid, fail, c.status);
-    if (s.dcv > 0) {
-        const int r4 = rows >> 2;
-#pragma unroll 1
-        for (int i = tid; i < GH * np * r4; i += kConsumers) {
-            const int gs = i / r4, j = i - gs * r4, g = gs / np;
-            if (g < ng) cp_async16(zs_s + gs * rows_max + 4 * j, ws.z + (qh0 * np + gs) * s.M + m0 + 4 * j);
-        }
-    }
 #pragma unroll 1
     for (int i = tid; i < GH * np; i += kConsumers) {
         float2 ml = make_float2(kNegBig, 0.f);
@@ -1345,68 +1353,90 @@ __global__ void __launch_bounds__(kThreads, 1) decode_fft_kernel(const __grid_co
         al_s[i] = ml.x;
         l_s[i] = ml.y;
     }
-    cp_async_wait_all();
-    consumer_sync();
-    if (j_pend >= 0 && s.dcv > 0) {                        // fused step: pending rank-1 update of this part's rows of C^V
-        float* cvg = coef_rows(c.coef_v, s, b, h, s.dcv) + (size_t)m0 * s.dcv;
+    float4 acc4[GH];
+#pragma unroll
+    for (int g = 0; g < GH; ++g) acc4[g] = make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll 1
-        for (int i = tid; i < rows * nv; i += kConsumers) {
-            const int r = i / nv, v = i - r * nv;
-            const float f = f_row(r);
-            float4 x = *reinterpret_cast<const float4*>(cv_s + 4 * i);
-            const float4 y = *reinterpret_cast<const float4*>(xp_s + s.dck + 4 * v);
-            x.x = fmaf(f, y.x, x.x); x.y = fmaf(f, y.y, x.y); x.z = fmaf(f, y.z, x.z); x.w = fmaf(f, y.w, x.w);
-            *reinterpret_cast<float4*>(cv_s + 4 * i) = x;
-            *reinterpret_cast<float4*>(cvg + 4 * i) = x;
-        }
-    }
-    if (warp < GH) {                                       // one warp per head, lanes over the parts
-        float mx = kNegBig;
-#pragma unroll 1
-        for (int sp = lane; sp < np; sp += 32) mx = fmaxf(mx, al_s[warp * np + sp]);
-        mx = warp_max(mx);
-        float Lsum = 0.f;
-#pragma unroll 1
-        for (int sp = lane; sp < np; sp += 32) {
-            const float a = ex2(al_s[warp * np + sp] - mx);
-            al_s[warp * np + sp] = a;
-            Lsum = fmaf(a, l_s[warp * np + sp], Lsum);
-        }
-        Lsum = warp_sum(Lsum);
-        if (lane == 0) linv_s[warp] = Lsum > 0.f ? __fdividef(1.0f, Lsum) : 0.f;
-    }
-    consumer_sync();
-    if (s.dcv > 0) {
-#pragma unroll 1
-        for (int t = tid; t < GH * rows; t += kConsumers) {
-            const int g = t / rows, r = t - g * rows;
-            float v = 0.f;
-            if (g < ng) {
-                const float* z = zs_s + g * np * rows_max + r;
-#pragma unroll 2
-                for (int sp = 0; sp < np; ++sp) v = fmaf(al_s[g * np + sp], z[sp * rows_max], v);
-                v *= recon_weight(s.norm, m0 + r, s.k, s.T);
+    for (int r0 = 0; r0 < rows || r0 == 0; r0 += mch) {
+        const int cr = max(0, min(rows - r0, mch));
+        if (s.dcv > 0) {
+            if (r0 > 0) {
+                consumer_sync();                           // the previous chunk has been consumed
+                stage_cv(r0, cr);
             }
-            zw_s[g * rows_max + r] = v;
+            const int r4 = cr >> 2;
+#pragma unroll 1
+            for (int i = tid; i < GH * np * r4; i += kConsumers) {
+                const int gs = i / r4, j = i - gs * r4, g = gs / np;
+                if (g < ng) cp_async16(zs_s + gs * mch + 4 * j, ws.z + (qh0 * np + gs) * s.M + m0 + r0 + 4 * j);
+            }
+        }
+        cp_async_wait_all();
+        consumer_sync();
+        if (j_pend >= 0 && s.dcv > 0) {                    // fused step: pending rank-1 update of these rows of C^V
+#pragma unroll 1
+            for (int i = tid; i < cr * nv; i += kConsumers) {
+                const int r = i / nv, v = i - r * nv;
+                const float f = f_row(r0 + r);
+                float4 x = *reinterpret_cast<const float4*>(cv_s + 4 * i);
+                const float4 y = *reinterpret_cast<const float4*>(xp_s + s.dck + 4 * v);
+                x.x = fmaf(f, y.x, x.x); x.y = fmaf(f, y.y, x.y); x.z = fmaf(f, y.z, x.z); x.w = fmaf(f, y.w, x.w);
+                *reinterpret_cast<float4*>(cv_s + 4 * i) = x;
+                *reinterpret_cast<float4*>(cvg + (size_t)r0 * s.dcv + 4 * i) = x;
+            }
+        }
+        if (r0 == 0) {
+            if (warp < GH) {                               // one warp per head, lanes over the parts
+                float mx = kNegBig;
+#pragma unroll 1
+                for (int sp = lane; sp < np; sp += 32) mx = fmaxf(mx, al_s[warp * np + sp]);
+                mx = warp_max(mx);
+                float Lsum = 0.f;
+#pragma unroll 1
+                for (int sp = lane; sp < np; sp += 32) {
+                    const float a = ex2(al_s[warp * np + sp] - mx);
+                    al_s[warp * np + sp] = a;
+                    Lsum = fmaf(a, l_s[warp * np + sp], Lsum);
+                }
+                Lsum = warp_sum(Lsum);
+                if (lane == 0) linv_s[warp] = Lsum > 0.f ? __fdividef(1.0f, Lsum) : 0.f;
+            }
         }
         consumer_sync();
-        if (tid < nrg * nv) {
-            const int v = tid % nv, rgi = tid / nv;
-            float4 acc4[GH];
-#pragma unroll
-            for (int g = 0; g < GH; ++g) acc4[g] = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (s.dcv > 0) {
 #pragma unroll 1
-            for (int r = rgi; r < rows; r += nrg) {
-                const float4 x = *reinterpret_cast<const float4*>(cv_s + r * s.dcv + 4 * v);
+            for (int t = tid; t < GH * cr; t += kConsumers) {
+                const int g = t / cr, r = t - g * cr;
+                float v = 0.f;
+                if (g < ng) {
+                    const float* z = zs_s + g * np * mch + r;
+#pragma unroll 2
+                    for (int sp = 0; sp < np; ++sp) v = fmaf(al_s[g * np + sp], z[sp * mch], v);
+                    v *= recon_weight(s.norm, m0 + r0 + r, s.k, s.T);
+                }
+                zw_s[g * mch + r] = v;
+            }
+            consumer_sync();
+            if (tid < nrg * nv) {
+                const int v = tid % nv, rgi = tid / nv;
+#pragma unroll 1
+                for (int r = rgi; r < cr; r += nrg) {
+                    const float4 x = *reinterpret_cast<const float4*>(cv_s + r * s.dcv + 4 * v);
 #pragma unroll
-                for (int g = 0; g < GH; ++g) {
-                    const float w = zw_s[g * rows_max + r];
-                    acc4[g].x = fmaf(w, x.x, acc4[g].x);
-                    acc4[g].y = fmaf(w, x.y, acc4[g].y);
-                    acc4[g].z = fmaf(w, x.z, acc4[g].z);
-                    acc4[g].w = fmaf(w, x.w, acc4[g].w);
+                    for (int g = 0; g < GH; ++g) {
+                        const float w = zw_s[g * mch + r];
+                        acc4[g].x = fmaf(w, x.x, acc4[g].x);
+                        acc4[g].y = fmaf(w, x.y, acc4[g].y);
+                        acc4[g].z = fmaf(w, x.z, acc4[g].z);
+                        acc4[g].w = fmaf(w, x.w, acc4[g].w);
+                    }
                 }
             }
+        }
+    }
+    if (s.dcv > 0) {
+        if (tid < nrg * nv) {
+            const int v = tid % nv, rgi = tid / nv;
 #pragma unroll
             for (int g = 0; g < GH; ++g) *reinterpret_cast<float4*>(ps_s + (rgi * GH + g) * s.dcv + 4 * v) = acc4[g];
         }
@@ -1430,7 +1460,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_fft_kernel(const __grid_co
     }
     consumer_sync();
     if (!*last_s) return;
-    float* op_s = big_s;                                   // [GH][np][d]
+    float* op_s = zw_s;                                    // [GH][np][d] (the slice buffers are free again)
     float* ocp_s = op_s + GH * np * s.d;                   // [GH][np][dcv]
     int* inv_s = reinterpret_cast<int*>(ocp_s + GH * np * s.dcv);   // [d] dim -> slot in D^vc, or -1
     {
@@ -1546,13 +1576,13 @@ size_t decode_fft_smem_bytes(const Dims& s, int log2S, int gh, int nb) {
 bool decode_fft_fused_fits(const Dims& s, int log2S, int gh, int nb, int n_part) {
     if (s.M % 4 != 0) return false;
     const FftSmem L = fft_smem_layout(log2S, s.k, gh, nb, s.d);
-    const long long rows_max = (s.M / 4 + n_part - 1) / n_part * 4 + 4;
-    if (rows_max * s.dck > (long long)nb * L.fb_floats) return false;
+    if (s.dck > 0 && (long long)nb * L.fb_floats < 8LL * s.dck) return false;           // at least eight rows of C^K per chunk
+    const long long ring = (long long)kStages * kStageBytes / 4;
     const long long nrg = s.dcv ? kConsumers / (s.dcv >> 2) : 0;
-    const long long head = 2LL * gh * n_part + gh + 4 + gh * rows_max;
-    const long long step1 = rows_max * s.dcv + (long long)gh * n_part * rows_max + nrg * gh * s.dcv;
-    const long long step2 = (long long)gh * n_part * (s.d + s.dcv) + s.d;
-    return head + (step1 > step2 ? step1 : step2) <= (long long)kStages * kStageBytes / 4;
+    const long long head = ((2LL * gh * n_part + gh + 3) & ~3LL);
+    if (s.dcv > 0 && (ring - head - nrg * gh * s.dcv) / (gh + s.dcv + (long long)gh * n_part) < 8) return false;   // and of C^V
+    const long long step2 = (long long)gh * n_part * (s.d + s.dcv) + s.d;               // the last part's merge of all parts
+    return head + 8LL * gh + step2 <= ring;
 }
 
 cudaError_t launch_decode_fft(const Dims& s, const CacheDev& c, int dtype, const DecodePlan& p, const void* q, void* out,

@@ -93,6 +93,7 @@ def test_launch_plan_is_host_logic():
     assert launches(2) == 1 and launches(3) == 2                                   # 8 KV heads: 18 CTAs each
     assert launches(2, decode_algo=fa.FA_DECODE_FFT_SPLIT) == 3 and launches(3, decode_algo=fa.FA_DECODE_FFT_SPLIT) == 4
     assert launches(2, decode_algo=fa.FA_DECODE_DIRECT) == 3
+    assert launches(2, batch=8) == 1                                               # 64 (b, head) pairs: two CTAs each
     assert launches(2, batch=16) == 3                                              # 128 pairs: more than half the SMs
     assert launches(2, kv_dtype=fa.FA_F32) == 3                                    # fp32 caches take the direct kernel
     assert launches(3, n_q_heads=64) in (2, 4)                                      # 8 query heads per KV head: two passes

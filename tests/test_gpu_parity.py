@@ -362,3 +362,16 @@ def test_ragged_batch_compress_append_decode():
         assert (st[b, 0], st[b, 1], st[b, 2]) == (refs[b].n_init[0], refs[b].n_local[0], refs[b].n_mid[0])
         den = np.abs(refs[b].coef_k[0]).max()
         assert np.abs(to64(gpu.coef_k[b]) - refs[b].coef_k[0]).max() / max(den, 1e-30) <= 1e-3
+
+
+@pytest.mark.parametrize("B", [2, 4, 8])
+def test_fused_decode_with_row_chunks(B):
+    """Batches whose parts hold more coefficient rows than the staging buffers take at once (the fused
+    kernel then walks its slice in chunks), through fused steps and plain decode."""
+    shape = SMALL_BF16.with_(B=B, Hq=16, Hkv=4, L=1300, T=2048, M=1024, n_full_k=32, n_full_v=32, decode_steps=4)
+    pair, stream = make_pair(shape, seed=17, algo=fa.FA_DECODE_FFT, P=4)
+    pair.check_decode(synth.queries(shape, seed=17))
+    K, V = stream.tokens(shape.L, shape.L + 4)
+    for t in range(4):
+        pair.check_step(synth.queries(shape, seed=17, step=t + 1), K[:, t], V[:, t])
+    pair.check_state()
