@@ -114,14 +114,15 @@ fa_status plan_decode(const fa_layout& l, DecodePlan* p) {
         if (l.decode_algo != FA_DECODE_FFT_SPLIT && per_job >= 2) {
             int best_ns = 0, best_nw = 0;
             long long best_cost = -1;
-            for (int nw = (win_bytes > 0 ? 1 : 0); nw <= 8 && nw < per_job; ++nw) {
+            // nw = 0: the window tokens are spread over the class CTAs (few CTAs per head); else CTAs of their own
+            for (int nw = 0; nw <= 8 && nw < per_job; ++nw) {
                 int ns = per_job - nw;
                 if (ns > s.P) ns = s.P;
-                const long long cc = (long long)((s.P + ns - 1) / ns) * class_bytes;
+                const long long cc = (long long)((s.P + ns - 1) / ns) * class_bytes + (nw == 0 ? (win_bytes + ns - 1) / ns : 0);
                 const long long wc = nw ? (win_bytes + nw - 1) / nw : 0;
                 const long long cost = cc > wc ? cc : wc;
                 if (best_cost < 0 || cost < best_cost) { best_cost = cost; best_ns = ns; best_nw = nw; }
-                if (nw == 0) break;
+                if (win_bytes == 0) break;
             }
             // fewest class CTAs that reach the same classes per CTA
             const int per_cta = (s.P + best_ns - 1) / best_ns;
