@@ -61,7 +61,7 @@ typedef enum { FA_NORM_ORTHO = 0, FA_NORM_PAPER = 1 } fa_norm;
  * (token index mod mid_classes) with one length period/mid_classes transform.
  * AUTO picks FFT when the layout allows it.  FFT runs as one kernel whose CTAs
  * wait for one another (cooperative launch) whenever every (batch, KV head) can
- * have two or more CTAs resident at once, else as three kernels; FFT_SPLIT
+ * have a CTA resident at once, else as three kernels; FFT_SPLIT
  * always takes the three-kernel form. */
 typedef enum { FA_DECODE_AUTO = 0, FA_DECODE_DIRECT = 1, FA_DECODE_FFT = 2, FA_DECODE_FFT_SPLIT = 3 } fa_decode_algo;
 

@@ -111,7 +111,7 @@ fa_status plan_decode(const fa_layout& l, DecodePlan* p) {
         };
         p->fused = 0;
         p->n_wsplit = 0;
-        if (l.decode_algo != FA_DECODE_FFT_SPLIT && per_job >= 2) {
+        if (l.decode_algo != FA_DECODE_FFT_SPLIT && per_job >= 1) {
             int best_ns = 0, best_nw = 0;
             long long best_cost = -1;
             // nw = 0: the window tokens are spread over the class CTAs (few CTAs per head); else CTAs of their own

@@ -82,7 +82,7 @@ def test_null_arguments():
 
 def test_launch_plan_is_host_logic():
     """Which form a decode call takes is decided on the host from the layout alone: one fused
-    cooperative kernel while every (batch row, KV head) can have two CTAs resident, three kernels past
+    cooperative kernel while every (batch row, KV head) can have a CTA resident, three kernels past
     that or when asked for; the fused step (light append + decode) needs the fused kernel."""
     lib = fa.lib()
 
@@ -94,7 +94,8 @@ def test_launch_plan_is_host_logic():
     assert launches(2, decode_algo=fa.FA_DECODE_FFT_SPLIT) == 3 and launches(3, decode_algo=fa.FA_DECODE_FFT_SPLIT) == 4
     assert launches(2, decode_algo=fa.FA_DECODE_DIRECT) == 3
     assert launches(2, batch=8) == 1                                               # 64 (b, head) pairs: two CTAs each
-    assert launches(2, batch=16) == 3                                              # 128 pairs: more than half the SMs
+    assert launches(2, batch=16) == 1                                              # 128 pairs: one CTA each
+    assert launches(2, batch=32) == 3                                              # more pairs than SMs
     assert launches(2, kv_dtype=fa.FA_F32) == 3                                    # fp32 caches take the direct kernel
     assert launches(3, n_q_heads=64) in (2, 4)                                      # 8 query heads per KV head: two passes
     assert launches(99) == 0

@@ -375,3 +375,15 @@ def test_fused_decode_with_row_chunks(B):
     for t in range(4):
         pair.check_step(synth.queries(shape, seed=17, step=t + 1), K[:, t], V[:, t])
     pair.check_state()
+
+
+def test_fused_decode_one_cta_per_head():
+    """As many (batch row, KV head) pairs as SMs allow one CTA each: the fused kernel with a single part."""
+    shape = SMALL_BF16.with_(B=16, Hq=16, Hkv=8, L=600, T=1024, M=128, n_full_k=32, n_full_v=48, decode_steps=2)
+    pair, stream = make_pair(shape, seed=18, algo=fa.FA_DECODE_FFT, P=8)
+    assert fa.fa_launch_count(pair.layout, 2) == 1
+    pair.check_decode(synth.queries(shape, seed=18))
+    K, V = stream.tokens(shape.L, shape.L + 2)
+    for t in range(2):
+        pair.check_step(synth.queries(shape, seed=18, step=t + 1), K[:, t], V[:, t])
+    pair.check_state()
