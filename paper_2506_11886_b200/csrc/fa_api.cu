@@ -255,6 +255,12 @@ fa_status fa_workspace_bytes(const fa_layout* layout, size_t* out) {
     st = plan_decode(*layout, &p);
     if (st != FA_OK) return st;
     *out = p.total;
+    if (p.fused) {                       // room for the three-kernel form too, should a cooperative launch not fit
+        fa_layout split = *layout;
+        split.decode_algo = FA_DECODE_FFT_SPLIT;
+        DecodePlan p2;
+        if (plan_decode(split, &p2) == FA_OK && p2.total > *out) *out = p2.total;
+    }
     return FA_OK;
 }
 
@@ -384,8 +390,14 @@ fa_status fa_decode_attention(const fa_layout* layout, const fa_cache* cache, co
     cudaStream_t cs = static_cast<cudaStream_t>(stream);
     char* w = static_cast<char*>(ws);
     if (p.fused) {
-        if (launch_decode_fft(s, c, layout->kv_dtype, p, q, out, w, false, cs) != cudaSuccess) return FA_ERR_CUDA;
-        return FA_OK;
+        const cudaError_t err = launch_decode_fft(s, c, layout->kv_dtype, p, q, out, w, false, cs);
+        if (err == cudaSuccess) return FA_OK;
+        if (err != cudaErrorCooperativeLaunchTooLarge) return FA_ERR_CUDA;
+        // the device cannot hold all CTAs at once right now (SMs taken by another client): three kernels instead
+        cudaGetLastError();
+        fa_layout split = *layout;
+        split.decode_algo = FA_DECODE_FFT_SPLIT;
+        return fa_decode_attention(&split, cache, q, out, ws, ws_bytes, stream);
     }
     if (launch_decode_prologue(s, c, layout->kv_dtype, p, q, w, cs) != cudaSuccess) return FA_ERR_CUDA;
     if (p.algo == FA_DECODE_FFT) {
@@ -419,6 +431,18 @@ fa_status fa_decode_step(const fa_layout* layout, fa_cache* cache, const void* q
     CacheDev c = make_cache(*cache);
     cudaStream_t cs = static_cast<cudaStream_t>(stream);
     char* w = static_cast<char*>(ws);
+    // (a cooperative launch that does not fit the device fails before anything runs; find out first)
+    static int coop_fits = -1;
+    if (coop_fits < 0) {
+        int dev = 0, coop = 0;
+        coop_fits = (cudaGetDevice(&dev) == cudaSuccess &&
+                     cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, dev) == cudaSuccess && coop) ? 1 : 0;
+    }
+    if (!coop_fits) {
+        st = fa_append(layout, cache, k_new, v_new, stream);
+        if (st != FA_OK) return st;
+        return fa_decode_attention(layout, cache, q, out, ws, ws_bytes, stream);
+    }
     if (launch_append_lite(s, c, layout->kv_dtype, p, k_new, v_new, w, cs) != cudaSuccess) return FA_ERR_CUDA;
     if (launch_decode_fft(s, c, layout->kv_dtype, p, q, out, w, true, cs) != cudaSuccess) return FA_ERR_CUDA;
     return FA_OK;
