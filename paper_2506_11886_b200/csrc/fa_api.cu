@@ -90,11 +90,11 @@ fa_status plan_decode(const fa_layout& l, DecodePlan* p) {
         p->gh = gh_fft;
         p->n_pass = (s.G + p->gh - 1) / p->gh;
         const int jobs = s.B * s.Hkv * p->n_pass;
-        // One CTA per SM (a deep ring of stages and a whole batch of classes per CTA).  When every
-        // (b, KV head, pass) can have at least two CTAs resident at once, the kernel is fused: it
-        // forms u itself and merges its own partial results, its CTAs waiting for one another
-        // (cooperative launch).  Window tokens then get CTAs of their own, as many as keeps their
-        // bytes per CTA at or below those of a class CTA.
+        // One CTA per SM (a ring of stages and a whole batch of classes per CTA).  When every
+        // (b, KV head, pass) can have a CTA resident at once, the kernel is fused: it forms u itself
+        // and merges its own partial results, its CTAs waiting for one another (cooperative
+        // launch).  A head gets floor(SMs / heads) CTAs; the window tokens either share the class
+        // CTAs or get CTAs of their own, whichever keeps the largest CTA's bytes smallest.
         const int per_job = kNumSms / jobs;
         const long long win_bytes = 2LL * (s.l_init + s.l_local) * s.d;
         const long long class_bytes = (long long)(s.T / s.P) * (s.nfk + s.nfv);
