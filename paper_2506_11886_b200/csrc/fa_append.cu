@@ -152,8 +152,10 @@ __global__ void __launch_bounds__(256) append_lite_kernel(Dims s, CacheDev c, De
     __shared__ float x_s[2][256];        // the row that leaves, both sides, natural dim order
     __shared__ int last_s;
     const int h = blockIdx.x, b = blockIdx.y, tid = threadIdx.x;
-    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    // wait for everything before this kernel, THEN let the decode kernel of the step start: it reads
+    // coefficient rows before its own wait, and nothing but this kernel may still be running then
     asm volatile("griddepcontrol.wait;" ::: "memory");
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     Ws ws = ws_view(wsp, p);
     const int n_init = c.state[kStateStride * b + 0], n_local = c.state[kStateStride * b + 1];
     const int n_mid = c.state[kStateStride * b + 2], head = c.state[kStateStride * b + 3];

@@ -479,8 +479,29 @@ __global__ void __launch_bounds__(kThreads, 1) decode_fft_kernel(const __grid_co
         if (tid < GH + 8) red_s[kWarps * GH + tid] = 0.f;
 
     }
+    // Fused step: the only kernel still running before this one is the light append, which does not
+    // touch the coefficients (it triggers this launch after its own wait), so this part's rows of C^K
+    // can start towards the transform buffers, and its rows of C^V towards L2, before the wait.
+    const int m0 = part * (s.M >> 2) / p.n_part * 4, m1 = (part + 1) * (s.M >> 2) / p.n_part * 4;
+    const int uch = s.dck > 0 ? ((NB * L.fb_floats) / s.dck) & ~3 : 0;      // rows of C^K the transform buffers hold at a time
+    auto start_coef_rows = [&]() {
+        if (tid >= kConsumers) return;
+        if (s.dck > 0) {
+            const float* ck = coef_rows(c.coef_k, s, b, h, s.dck) + (size_t)m0 * s.dck;
+#pragma unroll 1
+            for (int i = tid; i < min(m1 - m0, uch) * (s.dck >> 2); i += kConsumers) cp_async16(fbuf + 4 * i, ck + 4 * i);
+        }
+        if (s.dcv > 0) {
+            const char* cv = reinterpret_cast<const char*>(coef_rows(c.coef_v, s, b, h, s.dcv) + (size_t)m0 * s.dcv);
+            const int bytes = (m1 - m0) * s.dcv * 4;
+#pragma unroll 1
+            for (int o = tid * 128; o < bytes; o += kConsumers * 128) asm volatile("prefetch.global.L2 [%0];" ::"l"(cv + o));
+        }
+    };
+    if (p.fused && step) start_coef_rows();
     // fused kernel: everything below reads what earlier kernels in the stream wrote (state, cache, q)
     if (p.fused) asm volatile("griddepcontrol.wait;" ::: "memory");
+    if (p.fused && !step) start_coef_rows();
 
     const int n_init = c.state[kStateStride * b + 0], n_local = c.state[kStateStride * b + 1];
     const int n_mid = min(c.state[kStateStride * b + 2], s.max_mid), head = c.state[kStateStride * b + 3];
@@ -581,21 +602,11 @@ __global__ void __launch_bounds__(kThreads, 1) decode_fft_kernel(const __grid_co
     const float sl2 = s.scale * kLog2e;
 
     int32_t* bar = ws.bar + 4 * (((size_t)b * s.Hkv + h) * p.n_pass + pass);
-    // coefficient rows of this part in the fused steps: slices on 4-row boundaries (16-byte copies)
-    const int m0 = part * (s.M >> 2) / p.n_part * 4, m1 = (part + 1) * (s.M >> 2) / p.n_part * 4;
     // gathered query of the compressed K dims (one element per thread and round), loaded early
     float qc_early = 0.f;
     if (p.fused && s.dck > 0 && tid < GH * s.dck) {
         const int g = tid / s.dck, e = tid - g * s.dck;
         if (g < ng) qc_early = __bfloat162float(q[((size_t)b * s.Hq + g_first + g) * s.d + c.idx_comp_k[(size_t)h * s.dck + e]]);
-    }
-    // rows of C^K the transform buffers hold at a time (all of this part's rows unless the batch is large)
-    const int uch = s.dck > 0 ? ((NB * L.fb_floats) / s.dck) & ~3 : 0;
-    if (p.fused && s.dck > 0) {
-        // this part's rows of C^K go to the (still unused) transform buffers while the tables are built
-        const float* ck = coef_rows(c.coef_k, s, b, h, s.dck) + (size_t)m0 * s.dck;
-#pragma unroll 1
-        for (int i = tid; i < min(m1 - m0, uch) * (s.dck >> 2); i += kConsumers) cp_async16(fbuf + 4 * i, ck + 4 * i);
     }
     // fused step: the coefficient update the light append kernel left pending (basis column j_pend, or -1);
     // the leaving row's compressed dims and the basis values of this part's rows are fetched / formed now
@@ -699,13 +710,6 @@ __global__ void __launch_bounds__(kThreads, 1) decode_fft_kernel(const __grid_co
     // Fused kernel: this part's rows of u first, then the kept-dim scores of the first batch (they need
     // only q) while the other parts finish theirs, then the wait for all of u.
     if (p.fused) {
-        // this CTA's slice of the coefficient rows of C^V will be wanted at the very end: start it towards L2
-        if (s.dcv > 0) {
-            const char* cv = reinterpret_cast<const char*>(coef_rows(c.coef_v, s, b, h, s.dcv) + (size_t)m0 * s.dcv);
-            const int bytes = (m1 - m0) * s.dcv * 4;
-            #pragma unroll 1
-            for (int o = tid * 128; o < bytes; o += kConsumers * 128) asm volatile("prefetch.global.L2 [%0];" ::"l"(cv + o));
-        }
         // u_g[m] = scale * log2(e) * w_m * sum_e C^K[m][e] q_g[D^kc[e]] for rows [m0, m1): eight lanes per row
         if (s.dck > 0) {
             float* qc = o_s;                               // [GH][dck] gathered query, fp32
