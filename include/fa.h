@@ -126,6 +126,10 @@ fa_status fa_cache_sizes_of(const fa_layout* layout, fa_cache_sizes* out);
  * zero-fill it before the next call. */
 fa_status fa_workspace_bytes(const fa_layout* layout, size_t* out);
 
+/* Puts a workspace into the state the first call expects (zeroes its barrier counters): for a new
+ * buffer, or after FA_ERR_TIMEOUT.  ws_bytes >= 4096.  Asynchronous on `stream`. */
+fa_status fa_workspace_init(void* ws, size_t ws_bytes, void* stream);
+
 /* Clears state and status (an empty cache: no tokens, zero coefficients). */
 fa_status fa_cache_reset(const fa_layout* layout, fa_cache* cache, void* stream);
 

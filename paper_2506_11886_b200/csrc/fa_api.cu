@@ -264,6 +264,12 @@ fa_status fa_workspace_bytes(const fa_layout* layout, size_t* out) {
     return FA_OK;
 }
 
+fa_status fa_workspace_init(void* ws, size_t ws_bytes, void* stream) {
+    if (!ws || !aligned16(ws) || ws_bytes < 4096) return FA_ERR_WORKSPACE;
+    if (cudaMemsetAsync(ws, 0, 4096, static_cast<cudaStream_t>(stream)) != cudaSuccess) return FA_ERR_CUDA;
+    return FA_OK;
+}
+
 fa_status fa_cache_reset(const fa_layout* layout, fa_cache* cache, void* stream) {
     fa_status st = check_layout(layout);
     if (st != FA_OK) return st;

@@ -64,6 +64,7 @@ def lib() -> C.CDLL:
         L.fa_cache_sizes_of.argtypes = [lp, C.POINTER(fa_cache_sizes)]
         L.fa_workspace_bytes.argtypes = [lp, C.POINTER(sz)]
         L.fa_cache_reset.argtypes = [lp, cp, vp]
+        L.fa_workspace_init.argtypes = [vp, sz, vp]
         L.fa_validate.argtypes = [lp, cp, vp]
         L.fa_compress.argtypes = [lp, cp, vp, vp, i64, i64, i64, i32, vp, sz, vp]
         L.fa_append.argtypes = [lp, cp, vp, vp, vp]
@@ -81,7 +82,7 @@ def lib() -> C.CDLL:
         L.fa_status_string.restype = C.c_char_p
         for name in ("fa_cache_sizes_of", "fa_workspace_bytes", "fa_cache_reset", "fa_validate", "fa_compress",
                      "fa_append", "fa_decode_attention", "fa_poll_status", "fa_launch_count", "fa_version",
-                     "fa_decode_step_host", "fa_decode_step", "fa_select_workspace_bytes", "fa_select_dims", "fa_compress_ragged"):
+                     "fa_decode_step_host", "fa_decode_step", "fa_select_workspace_bytes", "fa_select_dims", "fa_compress_ragged", "fa_workspace_init"):
             getattr(L, name).restype = C.c_int
         _lib = L
     return _lib
@@ -200,7 +201,13 @@ class Cache:
 
 
 def new_workspace(layout: Layout, device="cuda") -> torch.Tensor:
-    return torch.zeros(max(256, fa_workspace_bytes(layout)), dtype=torch.uint8, device=device)
+    """A zero-filled workspace (its first 4 KiB are barrier counters that must start at zero)."""
+    return torch.zeros(max(4096, fa_workspace_bytes(layout)), dtype=torch.uint8, device=device)
+
+
+def fa_workspace_init(ws: torch.Tensor, stream=None) -> None:
+    """Re-zeroes the barrier counters of a workspace (after FA_ERR_TIMEOUT, or for a buffer not made by new_workspace)."""
+    _check(lib().fa_workspace_init(_ptr(ws), ws.numel(), _stream(stream)), "fa_workspace_init")
 
 
 def fa_cache_reset(layout: Layout, cache: Cache, stream=None) -> None:

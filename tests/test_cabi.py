@@ -116,3 +116,4 @@ def test_select_workspace_and_null_arguments():
     assert lib.fa_select_workspace_bytes(C.byref(odd), C.byref(out)) == fa.FA_ERR_UNSUPPORTED
     assert lib.fa_select_dims(C.byref(lay), None, None, 0, 0, 0, 5, None, None, None, None, None, None, 0, None) == fa.FA_ERR_INVALID_ARG
     assert lib.fa_decode_step(C.byref(lay), None, None, None, None, None, None, 0, None) == fa.FA_ERR_INVALID_ARG
+    assert lib.fa_workspace_init(None, 1 << 20, None) == fa.FA_ERR_WORKSPACE

@@ -387,3 +387,17 @@ def test_fused_decode_one_cta_per_head():
     for t in range(2):
         pair.check_step(synth.queries(shape, seed=18, step=t + 1), K[:, t], V[:, t])
     pair.check_state()
+
+
+def test_workspace_counters_must_start_at_zero_and_init_restores_them():
+    """A workspace full of garbage is made usable by fa_workspace_init."""
+    shape = SMALL_BF16.with_(B=1, Hq=4, Hkv=1, L=500, T=1024, M=64)
+    pair, _ = make_pair(shape, seed=19, algo=fa.FA_DECODE_FFT, P=8)
+    pair.ws = torch.full((pair.ws.numel(),), 0, dtype=torch.uint8, device="cuda")
+    pair.ws[4096:] = 0xAB                                   # scratch beyond the counters may hold anything
+    pair.check_decode(synth.queries(shape, seed=19))
+    dirty = torch.full((pair.ws.numel(),), 0x5A, dtype=torch.uint8, device="cuda")
+    fa.fa_workspace_init(dirty)
+    assert not dirty[:4096].any() and bool((dirty[4096:] == 0x5A).all())
+    pair.ws = dirty
+    pair.check_decode(synth.queries(shape, seed=19, step=1))
