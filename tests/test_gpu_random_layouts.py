@@ -1,0 +1,59 @@
+"""Parity on seeded random layouts: head dim, GQA ratio, kept-dim counts, period, residue classes, number
+of coefficients, window sizes, prompt length, storage dtype and decode algorithm are all drawn at random;
+every drawn case checks the cache after compression, a decode call, up to three fused steps and the cache
+again against the oracle.  Layouts the requested algorithm cannot serve are skipped inside the draw."""
+import random
+
+import pytest
+
+from paper_2506_11886_b200 import fa, synth
+from tests.parity_util import make_pair
+
+pytestmark = pytest.mark.gpu
+
+
+def _draw(rng):
+    d = rng.choice([64, 128])
+    Hkv, G, B = rng.choice([1, 2, 4]), rng.choice([1, 2, 3, 4, 8]), rng.choice([1, 1, 2, 3])
+    nfk, nfv = (min(rng.choice([0, 8, 16, 24, 32, 48, 64]), d) for _ in range(2))
+    T = 1 << rng.choice([8, 9, 10, 11, 12])
+    P = rng.choice([1, 2, 4, 8, 16, 32])
+    if T // P < 32:
+        return None
+    k = min(rng.choice([4, 8, 16, 32, 64, 128, 256]), T // P, T // 2)
+    l_init, l_local = rng.choice([0, 1, 4, 7]), rng.choice([0, 5, 16, 64, 100])
+    L = rng.randint(0, min(T + l_init + l_local, 3000))
+    algo = rng.choice([fa.FA_DECODE_AUTO, fa.FA_DECODE_FFT, fa.FA_DECODE_FFT_SPLIT])
+    shape = synth.Shape("random", B=B, layers=1, Hq=Hkv * G, Hkv=Hkv, d=d, L=L, dtype=rng.choice(["bf16", "bf16", "f32"]),
+                        n_full_k=nfk, n_full_v=nfv, M=2 * k, T=T, L_init=l_init, L_local=l_local, decode_steps=3)
+    return shape, P, algo
+
+
+@pytest.mark.parametrize("seed", [1, 2, 3])
+def test_random_layouts(seed):
+    rng = random.Random(seed)
+    done = 0
+    for trial in range(40):
+        drawn = _draw(rng)
+        if drawn is None:
+            continue
+        shape, P, algo = drawn
+        try:
+            pair, stream = make_pair(shape, seed=1000 * seed + trial, algo=algo, P=P, max_mid=shape.T)
+        except fa.FaError as e:
+            if e.status in (fa.FA_ERR_UNSUPPORTED, fa.FA_ERR_CAPACITY):
+                continue
+            raise
+        what = f"seed {seed} trial {trial}: {shape} P={P} algo={algo}"
+        try:
+            pair.check_state()
+            pair.check_decode(synth.queries(shape, seed=trial))
+            steps = min(3, shape.T - max(0, shape.L - shape.L_init - shape.L_local))
+            K, V = stream.tokens(shape.L, shape.L + max(steps, 1))
+            for t in range(steps):
+                pair.check_step(synth.queries(shape, seed=trial, step=t + 1), K[:, t], V[:, t])
+            pair.check_state()
+        except AssertionError as e:
+            raise AssertionError(f"{what}: {e}") from e
+        done += 1
+    assert done >= 15
