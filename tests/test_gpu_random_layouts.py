@@ -1,13 +1,19 @@
 """Parity on seeded random layouts: head dim, GQA ratio, kept-dim counts, period, residue classes, number
-of coefficients, window sizes, prompt length, storage dtype and decode algorithm are all drawn at random;
-every drawn case checks the cache after compression, a decode call, up to three fused steps and the cache
-again against the oracle.  Layouts the requested algorithm cannot serve are skipped inside the draw."""
+of coefficients, window sizes, prompt length, storage dtype, decode algorithm, reconstruction weights,
+frequency grid of the inputs and query sharpness are all drawn at random; every drawn case checks the cache
+after compression, a decode call, up to three steps (fused, or append + decode) and the cache again against
+the oracle.  Layouts the requested algorithm cannot serve are skipped inside the draw.
+
+Output tolerance: the stated absolute one times max(1, largest |expected output|).  With the paper-literal
+weights (1/k instead of 2/T) the compressed part of the outputs is scaled by T / 2k, up to 512 here, and an
+absolute bound below the bf16 rounding of such values would test nothing."""
 import random
 
+import numpy as np
 import pytest
 
 from paper_2506_11886_b200 import fa, synth
-from tests.parity_util import make_pair
+from tests.parity_util import OUT_ABS_BF16, OUT_ABS_F32, make_pair
 
 pytestmark = pytest.mark.gpu
 
@@ -24,9 +30,10 @@ def _draw(rng):
     l_init, l_local = rng.choice([0, 1, 4, 7]), rng.choice([0, 5, 16, 64, 100])
     L = rng.randint(0, min(T + l_init + l_local, 3000))
     algo = rng.choice([fa.FA_DECODE_AUTO, fa.FA_DECODE_FFT, fa.FA_DECODE_FFT_SPLIT])
+    norm, freq = rng.choice([fa.FA_NORM_ORTHO, fa.FA_NORM_ORTHO, fa.FA_NORM_PAPER]), rng.choice(["grid", "offgrid"])
     shape = synth.Shape("random", B=B, layers=1, Hq=Hkv * G, Hkv=Hkv, d=d, L=L, dtype=rng.choice(["bf16", "bf16", "f32"]),
                         n_full_k=nfk, n_full_v=nfv, M=2 * k, T=T, L_init=l_init, L_local=l_local, decode_steps=3)
-    return shape, P, algo
+    return shape, P, algo, norm, freq
 
 
 @pytest.mark.parametrize("seed", [1, 2, 3])
@@ -37,21 +44,35 @@ def test_random_layouts(seed):
         drawn = _draw(rng)
         if drawn is None:
             continue
-        shape, P, algo = drawn
+        shape, P, algo, norm, freq = drawn
         try:
-            pair, stream = make_pair(shape, seed=1000 * seed + trial, algo=algo, P=P, max_mid=shape.T)
+            pair, stream = make_pair(shape, seed=1000 * seed + trial, algo=algo, P=P, max_mid=shape.T, norm=norm, freq=freq)
         except fa.FaError as e:
             if e.status in (fa.FA_ERR_UNSUPPORTED, fa.FA_ERR_CAPACITY):
                 continue
             raise
-        what = f"seed {seed} trial {trial}: {shape} P={P} algo={algo}"
+        what = f"seed {seed} trial {trial}: {shape} P={P} algo={algo} norm={norm} freq={freq}"
+        base = OUT_ABS_F32 if shape.dtype == "f32" else OUT_ABS_BF16
+
+        def close(got, want):
+            err, bound = np.abs(got - want).max(), base * max(1.0, float(np.abs(want).max()))
+            assert err <= bound, f"output error {err:.3e} > {bound:.3e}"
+
         try:
             pair.check_state()
-            pair.check_decode(synth.queries(shape, seed=trial))
+            close(*pair.decode(synth.queries(shape, seed=trial)))
             steps = min(3, shape.T - max(0, shape.L - shape.L_init - shape.L_local))
             K, V = stream.tokens(shape.L, shape.L + max(steps, 1))
             for t in range(steps):
-                pair.check_step(synth.queries(shape, seed=trial, step=t + 1), K[:, t], V[:, t])
+                # (sharpened queries only with the orthogonal weights: the literal scale already multiplies the
+                # compressed scores by T / 2k, and a softmax that sharp amplifies rounding beyond any fixed bound)
+                peak = rng.choice([1.0, 6.0]) if norm == fa.FA_NORM_ORTHO else 1.0
+                q = synth.queries(shape, seed=trial, step=t + 1, peak=peak)
+                if rng.random() < 0.5:
+                    close(*pair.step(q, K[:, t], V[:, t]))
+                else:
+                    pair.append(K[:, t], V[:, t])
+                    close(*pair.decode(q))
             pair.check_state()
         except AssertionError as e:
             raise AssertionError(f"{what}: {e}") from e
