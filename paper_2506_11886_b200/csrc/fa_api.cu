@@ -111,12 +111,14 @@ fa_status plan_decode(const fa_layout& l, DecodePlan* p) {
         };
         p->fused = 0;
         p->n_wsplit = 0;
-        if (l.decode_algo != FA_DECODE_FFT_SPLIT && per_job >= 1) {
+        // Fewer CTAs per head than the device offers when the merge scratch of the fused kernel could not
+        // hold the partial results of that many parts (one KV head alone could have 148).
+        for (int pj = per_job; l.decode_algo != FA_DECODE_FFT_SPLIT && pj >= 1 && !p->fused; pj = pj > 24 ? 24 : pj - 1) {
             int best_ns = 0, best_nw = 0;
             long long best_cost = -1;
             // nw = 0: the window tokens are spread over the class CTAs (few CTAs per head); else CTAs of their own
-            for (int nw = 0; nw <= 8 && nw < per_job; ++nw) {
-                int ns = per_job - nw;
+            for (int nw = 0; nw <= 8 && nw < pj; ++nw) {
+                int ns = pj - nw;
                 if (ns > s.P) ns = s.P;
                 const long long cc = (long long)((s.P + ns - 1) / ns) * class_bytes + (nw == 0 ? (win_bytes + ns - 1) / ns : 0);
                 const long long wc = nw ? (win_bytes + nw - 1) / nw : 0;
