@@ -183,12 +183,13 @@ def run_ours(args):
         if world > 1:
             dist.barrier()
     dev = torch.device("cuda", local)
-    shape = synth.CONFIGS[1]
+    shape = synth.CONFIGS[args.config]
     K_steps, W = args.steps, max(args.warmup, 3)
     n_inst = max(args.instances, 2)
     layout = fa.Layout(batch=shape.B, n_q_heads=shape.Hq, n_kv_heads=shape.Hkv, head_dim=shape.d, n_full_k=shape.n_full_k,
                        n_full_v=shape.n_full_v, n_coef=shape.M, period=shape.T, l_init=shape.L_init, l_local=shape.L_local,
-                       max_mid=shape.T, mid_classes=shape.T // shape.k, kv_dtype=fa.FA_BF16, softmax_scale=shape.softmax_scale)
+                       max_mid=shape.T, mid_classes=shape.T // shape.k,
+                       kv_dtype=fa.FA_BF16 if shape.dtype == "bf16" else fa.FA_F32, softmax_scale=shape.softmax_scale)
     stream = synth.KVStream(shape, seed=SEED, device=str(dev))
     Kp, Vp = stream.tokens(0, shape.L, work_dtype=torch.float32)
     ws = fa.new_workspace(layout, device=dev)
@@ -296,14 +297,15 @@ def run_ours(args):
     by = algorithmic_bytes(shape, n_mid0, shape.L_init + shape.L_local)
     peak, peak_kind = _peaks()
     dec_gbs = by["decode"] / (us_decode * 1e-6) / 1e9
-    eb = 2
+    eb = 2 if shape.dtype == "bf16" else 4
     q_bytes = shape.B * shape.Hq * shape.d * eb
     kv_bytes = shape.B * shape.Hkv * shape.d * eb
     launches = K_steps * fa.fa_launch_count(layout, 3)
+    n_dec = fa.fa_launch_count(layout, 2)
     line = {
         "metric": METRIC, "value": us_step / world, "unit": UNIT, "n_gpus": world, "steps": K_steps, "warmup": W,
         "ms_per_step": us_step / 1e3, "higher_is_better": False, "scaling": "weak", "vs_baseline": None,
-        "dtype": "bf16 storage, f32 arithmetic", "data": "synthetic",
+        "dtype": f"{shape.dtype} storage, f32 arithmetic", "data": "synthetic",
         "config": {"workload": shape.name, "global_batch": shape.B * world, "seq_len": shape.L,
                    "step": "fa_decode_step (append + decode), one layer", "parallelism": f"replicas x{world}",
                    "l2": f"inputs larger than L2: {n_inst} cache instances x {by['decode'] / 1e6:.1f} MB rotated",
@@ -313,9 +315,10 @@ def run_ours(args):
                       "compress_ms_per_layer": min(comp_ms), "compress_tflops": comp_flop / (min(comp_ms) * 1e-3) / 1e12,
                       "compress_path": "tcgen05 bf16 x bf16 -> f32 (TMEM), basis tile generated in registers",
                       "select_dims_ms": min(sel_ms), "select_dims_finds_generator_sets": sel_ok},
-        "roofline": {"kernel": "fa_decode_attention (one fused cooperative kernel: u, token loop, merge)", "bound": "hbm",
+        "roofline": {"kernel": "fa_decode_attention (one fused cooperative kernel: u, token loop, merge)" if n_dec == 1 else
+                     f"fa_decode_attention ({n_dec} kernels: u, token loop, merge)", "bound": "hbm",
                      "achieved": dec_gbs, "peak": peak, "unit": "GB/s", "frac": dec_gbs / peak, "peak_kind": peak_kind,
-                     "algorithmic_bytes": by["decode"], "traffic": NCU_TRAFFIC_BYTES_PER_CALL,
+                     "algorithmic_bytes": by["decode"], "traffic": NCU_TRAFFIC_BYTES_PER_CALL if args.config == 1 else None,
                      "frac_of_8tbs_nominal": dec_gbs / 8000.0},
         "e2e": {"value": us_e2e / world, "unit": UNIT, "h2d_bytes_per_step": q_bytes + 2 * kv_bytes, "d2h_bytes_per_step": q_bytes},
         "gpu_launches": launches, "clocks": clocks,
@@ -323,7 +326,7 @@ def run_ours(args):
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         from oracle import fa_oracle as fo
         fo.build()
-        n_heads = min(4, shape.Hkv)
+        n_heads = min(4 if args.config == 1 else 1, shape.Hkv)
         times, threads = oracle_sample_time(shape, SEED, n_heads, shape.L, repeats=1)
         scale = shape.Hkv / n_heads
         line["cpu_baseline"] = {"value": times[0] * scale * 1e6, "unit": UNIT, "cores": threads, "kind": "oracle",
@@ -342,6 +345,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=8)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--instances", type=int, default=8)
+    ap.add_argument("--config", type=int, default=1, choices=[0, 1, 3, 4],
+                    help="synthetic configuration (one layer of it); 1 is the headline workload, the others are for the per-configuration table")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
     if args.impl == "reference":

@@ -59,10 +59,13 @@ typedef enum { FA_NORM_ORTHO = 0, FA_NORM_PAPER = 1 } fa_norm;
 /* How fa_decode_attention evaluates the compressed dims.  DIRECT sums the
  * n_coef basis terms per token; FFT evaluates each residue class of tokens
  * (token index mod mid_classes) with one length period/mid_classes transform.
- * AUTO picks FFT when the layout allows it.  FFT runs as one kernel whose CTAs
- * wait for one another (cooperative launch) whenever every (batch, KV head) can
- * have a CTA resident at once, else as three kernels; FFT_SPLIT
- * always takes the three-kernel form. */
+ * AUTO picks FFT when the layout allows it.  FFT runs as one kernel whenever
+ * its shared-memory staging fits the layout: a cooperative launch whose CTAs
+ * wait for one another while every (batch, KV head) can have a CTA resident at
+ * once, one CTA per (batch, KV head) in waves past that; else as three kernels.
+ * FFT_SPLIT always takes the three-kernel form.  AUTO also takes it when there
+ * are more (batch, KV head) pairs than SMs and the last wave of the one-kernel
+ * form would be nearly empty. */
 typedef enum { FA_DECODE_AUTO = 0, FA_DECODE_DIRECT = 1, FA_DECODE_FFT = 2, FA_DECODE_FFT_SPLIT = 3 } fa_decode_algo;
 
 /* Immutable description of one layer's cache. */

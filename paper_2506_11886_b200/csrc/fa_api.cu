@@ -94,8 +94,9 @@ fa_status plan_decode(const fa_layout& l, DecodePlan* p) {
         // (b, KV head, pass) can have a CTA resident at once, the kernel is fused: it forms u itself
         // and merges its own partial results, its CTAs waiting for one another (cooperative
         // launch).  A head gets floor(SMs / heads) CTAs; the window tokens either share the class
-        // CTAs or get CTAs of their own, whichever keeps the largest CTA's bytes smallest.
-        const int per_job = kNumSms / jobs;
+        // CTAs or get CTAs of their own, whichever keeps the largest CTA's bytes smallest.  With more
+        // heads than SMs a head gets one CTA, which waits for nobody: a plain launch that runs in waves.
+        const int per_job = jobs < kNumSms ? kNumSms / jobs : 1;
         const long long win_bytes = 2LL * (s.l_init + s.l_local) * s.d;
         const long long class_bytes = (long long)(s.T / s.P) * (s.nfk + s.nfv);
         // classes transformed together: enough butterflies for all consumer threads, within shared memory
@@ -137,17 +138,23 @@ fa_status plan_decode(const fa_layout& l, DecodePlan* p) {
                 p->nb = nb;
             }
         }
+        // Three-kernel form.  Classes are indivisible: pick the split count that minimises
+        // waves * (classes per CTA + a CTA's fixed cost, about two classes' worth), smallest count on ties.
+        int best = 1;
+        long long best_cost = -1;
+        for (int n = 1; n <= s.P && n <= 64; ++n) {
+            long long waves = ((long long)jobs * n + kNumSms - 1) / kNumSms;
+            long long cost = waves * ((s.P + n - 1) / n + 2);
+            if (best_cost < 0 || cost < best_cost) { best_cost = cost; best = n; }
+        }
+        // More heads than SMs: the lone CTAs of the fused kernel run in whole waves.  AUTO keeps it unless
+        // the balanced split is ahead by the same cost model (the last wave nearly empty) by more than
+        // the margin that the three launches and the round trip of u and the partial results cost.
+        if (p->fused && jobs > kNumSms && l.decode_algo == FA_DECODE_AUTO &&
+            20LL * ((jobs + kNumSms - 1) / kNumSms) * (s.P + 2) > 23 * best_cost)
+            p->fused = 0;
         if (!p->fused) {
-            // classes are indivisible: pick the split count that minimises waves * classes per CTA,
-            // smallest count on ties to keep the partial results small
-            const int slots = kNumSms;
-            int best = 1;
-            long long best_cost = -1;
-            for (int n = 1; n <= s.P && n <= 64; ++n) {
-                long long waves = ((long long)jobs * n + slots - 1) / slots;
-                long long cost = waves * ((s.P + n - 1) / n);
-                if (best_cost < 0 || cost < best_cost) { best_cost = cost; best = n; }
-            }
+            p->n_wsplit = 0;
             p->n_split = best;
             p->nb = pick_nb(best);
         }

@@ -118,15 +118,15 @@ __device__ __forceinline__ void consumer_sync() { asm volatile("bar.sync 1, %0;"
 // fences (cumulative over what the others wrote before the meeting) and adds 1 with release
 // semantics.  Wait: one thread polls with acquire loads, bounded like every other wait of this
 // kernel, then the consumer warps meet.
-__device__ __forceinline__ void part_arrive(int32_t* cnt, int tid) {
+__device__ __forceinline__ void part_arrive(int32_t* cnt, int n, int tid) {
     consumer_sync();
-    if (tid == 0) {
+    if (n > 1 && tid == 0) {                              // a part on its own meets nobody: no counter
         __threadfence();
         asm volatile("red.release.gpu.global.add.s32 [%0], 1;" ::"l"(cnt) : "memory");
     }
 }
 __device__ __forceinline__ void part_wait(const int32_t* cnt, int n, int tid, volatile int* fail, int32_t* status) {
-    if (tid == 0 && !*fail) {
+    if (n > 1 && tid == 0 && !*fail) {
         bool ok = false;
         for (uint32_t i = 0; i < (1u << 22); ++i) {
             int v;
@@ -776,7 +776,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_fft_kernel(const __grid_co
                         ws.u[((size_t)b * s.Hq + g_first + l8) * s.M + r] = recon_weight(s.norm, r, s.k, s.T) * sl2 * mine;
                 }
             }
-            part_arrive(bar + 0, tid);
+            part_arrive(bar + 0, p.n_part, tid);
         }
         if (has_classes) k_phase(c0, min(NB, c1 - c0));
         if (s.dck > 0 && !is_win) part_wait(bar + 0, p.n_part, tid, fail, c.status);
@@ -1348,7 +1348,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_fft_kernel(const __grid_co
     };
 
     if (s.dcv > 0) stage_cv(0, min(rows, mch));            // under the barrier
-    part_arrive(bar + 1, tid);
+    part_arrive(bar + 1, np, tid);
     part_wait(bar + 1, np, tid, fail, c.status);
 #pragma unroll 1
     for (int i = tid; i < GH * np; i += kConsumers) {
@@ -1457,9 +1457,11 @@ __global__ void __launch_bounds__(kThreads, 1) decode_fft_kernel(const __grid_co
     // ticket: the last part to get here finishes the rows
     consumer_sync();
     if (tid == 0) {
-        int old;
-        __threadfence();
-        asm volatile("atom.acq_rel.gpu.global.add.s32 %0, [%1], 1;" : "=r"(old) : "l"(bar + 2) : "memory");
+        int old = 0;
+        if (np > 1) {
+            __threadfence();
+            asm volatile("atom.acq_rel.gpu.global.add.s32 %0, [%1], 1;" : "=r"(old) : "l"(bar + 2) : "memory");
+        }
         *last_s = old == np - 1;
     }
     consumer_sync();
@@ -1501,7 +1503,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_fft_kernel(const __grid_co
         }
         out[(qh0 + g) * s.d + e] = __float2bfloat16_rn(v * linv_s[g]);
     }
-    if (tid == 0) { bar[0] = 0; bar[1] = 0; bar[2] = 0; }   // the counters are zero again for the next call
+    if (tid == 0 && np > 1) { bar[0] = 0; bar[1] = 0; bar[2] = 0; }   // the counters are zero again for the next call
 }
 
 template <int GH, int LS>
@@ -1533,7 +1535,7 @@ cudaError_t launch_fft_t(const Dims& s, const CacheDev& c, const DecodePlan& p, 
     attr[1].val.cooperative = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    if (p.fused) {
+    if (p.fused && p.n_part > 1) {                       // a head served by one CTA waits for nobody: plain launch, any grid
         cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
         if (coop_pdl_ok < 0 && (cudaStreamIsCapturing(st, &cap) != cudaSuccess || cap != cudaStreamCaptureStatusNone)) {
             cfg.attrs = attr + 1;                                          // not probed yet: stay on the plain cooperative launch

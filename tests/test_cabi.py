@@ -82,8 +82,9 @@ def test_null_arguments():
 
 def test_launch_plan_is_host_logic():
     """Which form a decode call takes is decided on the host from the layout alone: one fused
-    cooperative kernel while every (batch row, KV head) can have a CTA resident, three kernels past
-    that or when asked for; the fused step (light append + decode) needs the fused kernel."""
+    kernel (cooperative while a head has several CTAs; with more heads than SMs, one CTA per head in
+    waves), three kernels when asked for or when the fused kernel's staging does not fit; the fused
+    step (light append + decode) needs the fused kernel."""
     lib = fa.lib()
 
     def launches(what, **kw):
@@ -95,7 +96,7 @@ def test_launch_plan_is_host_logic():
     assert launches(2, decode_algo=fa.FA_DECODE_DIRECT) == 3
     assert launches(2, batch=8) == 1                                               # 64 (b, head) pairs: two CTAs each
     assert launches(2, batch=16) == 1                                              # 128 pairs: one CTA each
-    assert launches(2, batch=32) == 3                                              # more pairs than SMs
+    assert launches(2, batch=32) == 1                                              # more pairs than SMs: still one CTA each, in waves
     assert launches(2, kv_dtype=fa.FA_F32) == 3                                    # fp32 caches take the direct kernel
     assert launches(3, n_q_heads=64) in (2, 4)                                      # 8 query heads per KV head: two passes
     assert launches(99) == 0
