@@ -96,46 +96,58 @@ fa_status plan_decode(const fa_layout& l, DecodePlan* p) {
         // launch).  A head gets floor(SMs / heads) CTAs; the window tokens either share the class
         // CTAs or get CTAs of their own, whichever keeps the largest CTA's bytes smallest.  With more
         // heads than SMs a head gets one CTA, which waits for nobody: a plain launch that runs in waves.
-        const int per_job = jobs < kNumSms ? kNumSms / jobs : 1;
         const long long win_bytes = 2LL * (s.l_init + s.l_local) * s.d;
         const long long class_bytes = (long long)(s.T / s.P) * (s.nfk + s.nfv);
         // classes transformed together: enough butterflies for all consumer threads, within shared memory
-        auto pick_nb = [&](int n_split) {
+        auto pick_nb = [&](int n_split, int occ = 1) {
             const int S = s.T / s.P;
             int nb = 2048 / S;
             if (nb < 1) nb = 1;
             if (nb > 8) nb = 8;
             const int per_cta = (s.P + n_split - 1) / n_split;
             if (nb > per_cta) nb = per_cta;
-            while (nb > 1 && decode_fft_smem_bytes(s, log2S, p->gh, nb) > 227 * 1024) --nb;
+            const size_t limit = occ == 2 ? 113 * 1024 : 227 * 1024;      // two CTAs share the SM's 228 KB, 1 KB reserved each
+            while (nb > 1 && decode_fft_smem_bytes(s, log2S, p->gh, nb, occ) > limit) --nb;
             return nb;
         };
         p->fused = 0;
         p->n_wsplit = 0;
-        // Fewer CTAs per head than the device offers when the merge scratch of the fused kernel could not
-        // hold the partial results of that many parts (one KV head alone could have 148).
-        for (int pj = per_job; l.decode_algo != FA_DECODE_FFT_SPLIT && pj >= 1 && !p->fused; pj = pj > 24 ? 24 : pj - 1) {
-            int best_ns = 0, best_nw = 0;
-            long long best_cost = -1;
-            // nw = 0: the window tokens are spread over the class CTAs (few CTAs per head); else CTAs of their own
-            for (int nw = 0; nw <= 8 && nw < pj; ++nw) {
-                int ns = pj - nw;
-                if (ns > s.P) ns = s.P;
-                const long long cc = (long long)((s.P + ns - 1) / ns) * class_bytes + (nw == 0 ? (win_bytes + ns - 1) / ns : 0);
-                const long long wc = nw ? (win_bytes + nw - 1) / nw : 0;
-                const long long cost = cc > wc ? cc : wc;
-                if (best_cost < 0 || cost < best_cost) { best_cost = cost; best_ns = ns; best_nw = nw; }
-                if (win_bytes == 0) break;
-            }
-            // fewest class CTAs that reach the same classes per CTA
-            const int per_cta = (s.P + best_ns - 1) / best_ns;
-            best_ns = (s.P + per_cta - 1) / per_cta;
-            const int nb = pick_nb(best_ns);
-            if (decode_fft_fused_fits(s, log2S, p->gh, nb, best_ns + best_nw)) {
-                p->fused = 1;
-                p->n_split = best_ns;
-                p->n_wsplit = best_nw;
-                p->nb = nb;
+        p->occ = 1;
+        // Short transforms leave room for two CTAs on an SM (a shorter ring, a register cap): one CTA's
+        // dependent phases hide behind the other's, and a head gets twice the CTAs (or, with more heads
+        // than SMs, the waves are twice as wide).  Tried first; one CTA per SM otherwise.
+        for (int occ = log2S <= 8 ? 2 : 1; occ >= 1 && !p->fused && l.decode_algo != FA_DECODE_FFT_SPLIT; --occ) {
+            const size_t smem_limit = occ == 2 ? 113 * 1024 : 227 * 1024;
+            const int slots = kNumSms * occ;
+            const int per_job = jobs < slots ? slots / jobs : 1;
+            // Fewer CTAs per head than the device offers when the merge scratch of the fused kernel could
+            // not hold the partial results of that many parts (one KV head alone could have them all).
+            for (int pj = per_job; pj >= 1 && !p->fused; pj = pj > 24 ? 24 : pj - 1) {
+                int best_ns = 0, best_nw = 0;
+                long long best_cost = -1;
+                // nw = 0: the window tokens are spread over the class CTAs (few CTAs per head); else CTAs of their own
+                for (int nw = 0; nw <= 8 && nw < pj; ++nw) {
+                    int ns = pj - nw;
+                    if (ns > s.P) ns = s.P;
+                    const long long cc = (long long)((s.P + ns - 1) / ns) * class_bytes + (nw == 0 ? (win_bytes + ns - 1) / ns : 0);
+                    const long long wc = nw ? (win_bytes + nw - 1) / nw : 0;
+                    const long long cost = cc > wc ? cc : wc;
+                    if (best_cost < 0 || cost < best_cost) { best_cost = cost; best_ns = ns; best_nw = nw; }
+                    if (win_bytes == 0) break;
+                }
+                // fewest class CTAs that reach the same classes per CTA
+                const int per_cta = (s.P + best_ns - 1) / best_ns;
+                best_ns = (s.P + per_cta - 1) / per_cta;
+                const int nb = pick_nb(best_ns, occ);
+                if (occ == 2 && nb < (per_cta < 4 ? per_cta : 4)) break;                   // too few classes per transform batch: not worth it
+                if (decode_fft_smem_bytes(s, log2S, p->gh, nb, occ) <= smem_limit &&
+                    decode_fft_fused_fits(s, log2S, p->gh, nb, best_ns + best_nw, occ)) {
+                    p->fused = 1;
+                    p->n_split = best_ns;
+                    p->n_wsplit = best_nw;
+                    p->nb = nb;
+                    p->occ = occ;
+                }
             }
         }
         // Three-kernel form.  Classes are indivisible: pick the split count that minimises
@@ -151,10 +163,11 @@ fa_status plan_decode(const fa_layout& l, DecodePlan* p) {
         // the balanced split is ahead by the same cost model (the last wave nearly empty) by more than
         // the margin that the three launches and the round trip of u and the partial results cost.
         if (p->fused && jobs > kNumSms && l.decode_algo == FA_DECODE_AUTO &&
-            20LL * ((jobs + kNumSms - 1) / kNumSms) * (s.P + 2) > 23 * best_cost)
+            20LL * ((jobs + kNumSms * p->occ - 1) / (kNumSms * p->occ)) * (s.P + 2) * p->occ > 23 * best_cost)
             p->fused = 0;
         if (!p->fused) {
             p->n_wsplit = 0;
+            p->occ = 1;
             p->n_split = best;
             p->nb = pick_nb(best);
         }

@@ -69,6 +69,7 @@ struct DecodePlan {
     int rows_pro;      // coefficient rows per prologue CTA
     int fft_log2;      // log2 of the transform length (FFT path)
     int nb;            // classes transformed together by one CTA (FFT path)
+    int occ;           // CTAs per SM the main kernel is built for (FFT path: 1, or 2 with a shorter ring)
     // workspace offsets in bytes
     size_t off_bar, off_u, off_ml, off_o, off_z, off_oc, off_om, off_cnt, off_pend, off_pendj, total;
 };
@@ -111,8 +112,8 @@ cudaError_t launch_append_lite(const Dims&, const CacheDev&, int dtype, const De
                                char* ws, cudaStream_t);
 cudaError_t launch_decode_fft(const Dims&, const CacheDev&, int dtype, const DecodePlan&, const void* q, void* out, char* ws, bool step,
                               cudaStream_t);
-size_t decode_fft_smem_bytes(const Dims&, int log2S, int gh, int nb);
-bool decode_fft_fused_fits(const Dims&, int log2S, int gh, int nb, int n_part);
+size_t decode_fft_smem_bytes(const Dims&, int log2S, int gh, int nb, int occ = 1);
+bool decode_fft_fused_fits(const Dims&, int log2S, int gh, int nb, int n_part, int occ = 1);
 cudaError_t launch_decode_epilogue(const Dims&, const CacheDev&, int dtype, const DecodePlan&, void* out, char* ws,
                                    cudaStream_t);
 

@@ -45,7 +45,9 @@ constexpr int kConsumers = 256;
 constexpr int kWarps = kConsumers / 32;
 constexpr int kThreads = kConsumers + 32;
 constexpr int kStageBytes = 16384;
-constexpr int kStages = 5;
+constexpr int kStages = 5;                 // stages of the ring with one CTA per SM
+constexpr int kStagesOcc2 = 3;             // with two CTAs per SM (small transforms, many heads)
+__host__ __device__ constexpr int ring_stages(int occ) { return occ == 2 ? kStagesOcc2 : kStages; }
 constexpr int kPendRows = 256;            // rows of a part whose basis values are tabulated for the fused step's update
 constexpr int kWinRowsPerTile = 64;       // rows of one window tile: two [64 rows x 64 dims] TMA boxes, 128-byte swizzle
 constexpr int kWinHalfBytes = kWinRowsPerTile * 128;
@@ -383,7 +385,7 @@ struct FftSmem {
     int stages_off, fbuf_off, kb_off, pbt_off, twf_off, rev_off, E_off, ut_off, z_off, o_off, red_off, pend_off, zero_off, total;
     int fb_floats, pbs;
 };
-__host__ __device__ inline FftSmem fft_smem_layout(int log2S, int k, int GH, int NB, int d) {
+__host__ __device__ inline FftSmem fft_smem_layout(int log2S, int k, int GH, int NB, int d, int occ) {
     const int S = 1 << log2S;
     FftSmem L;
     L.fb_floats = pf_size(S * GH);
@@ -391,7 +393,7 @@ __host__ __device__ inline FftSmem fft_smem_layout(int log2S, int k, int GH, int
     int off = 256;                                        // mbarriers + flags
     L.zero_off = off; off += 16;
     off = 1024;                                           // stages are 1024-byte aligned (swizzled window tiles)
-    L.stages_off = off; off += kStages * kStageBytes;
+    L.stages_off = off; off += ring_stages(occ) * kStageBytes;
     L.fbuf_off = off; off += 4 * NB * L.fb_floats;
     off = (off + 15) / 16 * 16;
     L.kb_off = off; off += 4 * NB * S * GH;               // kept-dim scores of the batch, natural token order
@@ -414,9 +416,9 @@ __host__ __device__ inline FftSmem fft_smem_layout(int log2S, int k, int GH, int
 
 template <int GH> __host__ __device__ constexpr int hperm(int s) { return GH == 4 ? (((s & 1) << 1) | (s >> 1)) : s; }
 
-// GH query heads per CTA (2 or 4), transform length S = 2^LS.
-template <int GH, int LS>
-__global__ void __launch_bounds__(kThreads, 1) decode_fft_kernel(const __grid_constant__ CUtensorMap tm_ki,
+// GH query heads per CTA (2 or 4), transform length S = 2^LS, OCC CTAs per SM (2: shorter ring, register cap).
+template <int GH, int LS, int OCC>
+__global__ void __launch_bounds__(kThreads, OCC) decode_fft_kernel(const __grid_constant__ CUtensorMap tm_ki,
                                                                   const __grid_constant__ CUtensorMap tm_vi,
                                                                   const __grid_constant__ CUtensorMap tm_kl,
                                                                   const __grid_constant__ CUtensorMap tm_vl, Dims s, CacheDev c,
@@ -424,14 +426,15 @@ __global__ void __launch_bounds__(kThreads, 1) decode_fft_kernel(const __grid_co
                                                                   char* wsp, int step) {
     constexpr int N = GH / 2;
     constexpr int S = 1 << LS;
+    constexpr int NS = ring_stages(OCC);
     extern __shared__ __align__(128) unsigned char smem_unaligned[];
     unsigned char* smem_raw = smem_unaligned + ((1024u - (smem_addr(smem_unaligned) & 1023u)) & 1023u);
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");      // the epilogue may be scheduled behind us at once
     Ws ws = ws_view(wsp, p);
     const int NB = p.nb;
-    const FftSmem L = fft_smem_layout(LS, s.k, GH, NB, s.d);
+    const FftSmem L = fft_smem_layout(LS, s.k, GH, NB, s.d, OCC);
     uint64_t* full = reinterpret_cast<uint64_t*>(smem_raw);
-    uint64_t* empty = full + kStages;
+    uint64_t* empty = full + NS;
     volatile int* fail = reinterpret_cast<volatile int*>(smem_raw + 128);
     unsigned char* zero16 = smem_raw + L.zero_off;
     unsigned char* stages = smem_raw + L.stages_off;
@@ -524,13 +527,13 @@ __global__ void __launch_bounds__(kThreads, 1) decode_fft_kernel(const __grid_co
     const int pbw = NB * L.pbs;                            // row stride of the window probabilities
 
     if (tid == 0) {
-        for (int i = 0; i < kStages; ++i) { mbar_init(full + i, 1); mbar_init(empty + i, kWarps); }
+        for (int i = 0; i < NS; ++i) { mbar_init(full + i, 1); mbar_init(empty + i, kWarps); }
         *fail = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     // stale shared memory must hold finite numbers: rows past the end of a tile are multiplied by p = 0
     #pragma unroll 1
-    for (int i = tid; i < (kStages * kStageBytes) / 16; i += kThreads) reinterpret_cast<uint4*>(stages)[i] = make_uint4(0, 0, 0, 0);
+    for (int i = tid; i < (NS * kStageBytes) / 16; i += kThreads) reinterpret_cast<uint4*>(stages)[i] = make_uint4(0, 0, 0, 0);
     if (tid < 4) reinterpret_cast<uint32_t*>(zero16)[tid] = 0;
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     __syncthreads();
@@ -543,8 +546,8 @@ __global__ void __launch_bounds__(kThreads, 1) decode_fft_kernel(const __grid_co
         if (plane == 0) {
             int it = 0;
             auto acquire = [&](uint32_t bytes) -> unsigned char* {
-                const int st = it % kStages;
-                if (it >= kStages) mbar_wait(empty + st, ((it / kStages) - 1) & 1, fail, c.status);
+                const int st = it % NS;
+                if (it >= NS) mbar_wait(empty + st, ((it / NS) - 1) & 1, fail, c.status);
                 if (*fail) return nullptr;
                 mbar_expect_tx(full + st, bytes);
                 return stages + (size_t)st * kStageBytes;
@@ -560,7 +563,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_fft_kernel(const __grid_co
                         const uint32_t bytes = (uint32_t)(min(ts, n_c - a0) * rowb);
                         const bf16* src = side == 0 ? mid_row<bf16>(c.k_mid, s, b, h, cls, a0, s.nfk)
                                                     : mid_row<bf16>(c.v_mid, s, b, h, cls, a0, s.nfv);
-                        if (unsigned char* dst = acquire(bytes)) bulk_g2s(dst, src, bytes, full + it % kStages);
+                        if (unsigned char* dst = acquire(bytes)) bulk_g2s(dst, src, bytes, full + it % NS);
                         ++it;
                     }
                 }
@@ -580,7 +583,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_fft_kernel(const __grid_co
                             if (unsigned char* dst = acquire((uint32_t)(nhalf * kWinHalfBytes))) {
 #pragma unroll 1
                                 for (int hf = 0; hf < nhalf; ++hf)
-                                    tma_load_3d(dst + hf * kWinHalfBytes, tm, hf * 64, sg.row[i] + r0, b * s.Hkv + h, full + it % kStages);
+                                    tma_load_3d(dst + hf * kWinHalfBytes, tm, hf * 64, sg.row[i] + r0, b * s.Hkv + h, full + it % NS);
                             }
                             ++it;
                         }
@@ -645,19 +648,19 @@ __global__ void __launch_bounds__(kThreads, 1) decode_fft_kernel(const __grid_co
     int it = 0;                                           // tile counter, mirrors the producer's
 
     auto wait_tile = [&]() -> const unsigned char* {
-        const int st = it % kStages;
-        mbar_wait(full + st, (it / kStages) & 1, fail, c.status);
+        const int st = it % NS;
+        mbar_wait(full + st, (it / NS) & 1, fail, c.status);
         return stages + (size_t)st * kStageBytes;
     };
     const uint32_t stages_u = smem_addr(stages), zero_u = smem_addr(zero16);
     auto wait_tile_u = [&]() -> uint32_t {                // the same, as a shared-memory address
-        const int st = it % kStages;
-        mbar_wait(full + st, (it / kStages) & 1, fail, c.status);
+        const int st = it % NS;
+        mbar_wait(full + st, (it / NS) & 1, fail, c.status);
         return stages_u + (uint32_t)st * kStageBytes;
     };
     auto release_tile = [&]() {
         __syncwarp();
-        if (lane == 0) mbar_arrive(empty + (it % kStages));
+        if (lane == 0) mbar_arrive(empty + (it % NS));
         ++it;
     };
     // kept dims of one batch of classes: kb[class][token][slot] = sl2 * (q_u . K^mu), 16 tokens per mma.
@@ -1329,7 +1332,7 @@ __global__ void __launch_bounds__(kThreads, 1) decode_fft_kernel(const __grid_co
     const size_t qh0 = (size_t)b * s.Hq + g_first;
     const int nv = s.dcv >> 2, nrg = nv ? kConsumers / nv : 0;
     // rows of the slice handled at a time: what the stage ring holds of C^V rows, z slices and weighted z
-    constexpr int kRing = kStages * kStageBytes / 4;
+    constexpr int kRing = NS * kStageBytes / 4;
     const int head_f = (2 * GH * np + GH + 3) & ~3;
     const int mch = max(4, min((rows + 3) & ~3, ((kRing - head_f - nrg * GH * s.dcv) / (GH + s.dcv + GH * np)) & ~3));
     float* al_s = reinterpret_cast<float*>(stages);        // [GH][np] maxima, then exp2(m - max)
@@ -1506,11 +1509,11 @@ __global__ void __launch_bounds__(kThreads, 1) decode_fft_kernel(const __grid_co
     if (tid == 0 && np > 1) { bar[0] = 0; bar[1] = 0; bar[2] = 0; }   // the counters are zero again for the next call
 }
 
-template <int GH, int LS>
+template <int GH, int LS, int OCC>
 cudaError_t launch_fft_t(const Dims& s, const CacheDev& c, const DecodePlan& p, const void* q, void* out, char* ws, int step,
                          cudaStream_t st) {
-    const FftSmem L = fft_smem_layout(LS, s.k, GH, p.nb, s.d);
-    cudaError_t err = ensure_dynamic_smem(decode_fft_kernel<GH, LS>, (size_t)L.total);
+    const FftSmem L = fft_smem_layout(LS, s.k, GH, p.nb, s.d, OCC);
+    cudaError_t err = ensure_dynamic_smem(decode_fft_kernel<GH, LS, OCC>, (size_t)L.total);
     if (err != cudaSuccess) return err;
     // window buffers as tensor maps (cached per buffer)
     CUtensorMap tki, tvi, tkl, tvl;
@@ -1541,7 +1544,7 @@ cudaError_t launch_fft_t(const Dims& s, const CacheDev& c, const DecodePlan& p, 
             cfg.attrs = attr + 1;                                          // not probed yet: stay on the plain cooperative launch
         } else if (coop_pdl_ok != 0) {
             cfg.numAttrs = 2;
-            cudaError_t err2 = cudaLaunchKernelEx(&cfg, decode_fft_kernel<GH, LS>, tki, tvi, tkl, tvl, s, c, p,
+            cudaError_t err2 = cudaLaunchKernelEx(&cfg, decode_fft_kernel<GH, LS, OCC>, tki, tvi, tkl, tvl, s, c, p,
                                                   static_cast<const bf16*>(q), static_cast<bf16*>(out), ws, step);
             if (err2 == cudaSuccess) { coop_pdl_ok = 1; return err2; }
             if (coop_pdl_ok == 1) return err2;
@@ -1553,7 +1556,7 @@ cudaError_t launch_fft_t(const Dims& s, const CacheDev& c, const DecodePlan& p, 
             cfg.attrs = attr + 1;
         }
     }
-    return cudaLaunchKernelEx(&cfg, decode_fft_kernel<GH, LS>, tki, tvi, tkl, tvl, s, c, p, static_cast<const bf16*>(q),
+    return cudaLaunchKernelEx(&cfg, decode_fft_kernel<GH, LS, OCC>, tki, tvi, tkl, tvl, s, c, p, static_cast<const bf16*>(q),
                               static_cast<bf16*>(out), ws, step);
 }
 
@@ -1561,29 +1564,30 @@ template <int GH>
 cudaError_t launch_fft_ls(const Dims& s, const CacheDev& c, const DecodePlan& p, const void* q, void* out, char* ws, int step,
                           cudaStream_t st) {
     switch (p.fft_log2) {
-        case 5: return launch_fft_t<GH, 5>(s, c, p, q, out, ws, step, st);
-        case 6: return launch_fft_t<GH, 6>(s, c, p, q, out, ws, step, st);
-        case 7: return launch_fft_t<GH, 7>(s, c, p, q, out, ws, step, st);
-        case 8: return launch_fft_t<GH, 8>(s, c, p, q, out, ws, step, st);
-        case 9: return launch_fft_t<GH, 9>(s, c, p, q, out, ws, step, st);
-        case 10: return launch_fft_t<GH, 10>(s, c, p, q, out, ws, step, st);
+        case 5: return p.occ == 2 ? launch_fft_t<GH, 5, 2>(s, c, p, q, out, ws, step, st) : launch_fft_t<GH, 5, 1>(s, c, p, q, out, ws, step, st);
+        case 6: return p.occ == 2 ? launch_fft_t<GH, 6, 2>(s, c, p, q, out, ws, step, st) : launch_fft_t<GH, 6, 1>(s, c, p, q, out, ws, step, st);
+        case 7: return p.occ == 2 ? launch_fft_t<GH, 7, 2>(s, c, p, q, out, ws, step, st) : launch_fft_t<GH, 7, 1>(s, c, p, q, out, ws, step, st);
+        case 8: return p.occ == 2 ? launch_fft_t<GH, 8, 2>(s, c, p, q, out, ws, step, st) : launch_fft_t<GH, 8, 1>(s, c, p, q, out, ws, step, st);
+        case 9: return launch_fft_t<GH, 9, 1>(s, c, p, q, out, ws, step, st);
+        case 10: return launch_fft_t<GH, 10, 1>(s, c, p, q, out, ws, step, st);
         default: return cudaErrorInvalidValue;
     }
 }
 
 }  // namespace
 
-size_t decode_fft_smem_bytes(const Dims& s, int log2S, int gh, int nb) {
-    return (size_t)fft_smem_layout(log2S, s.k, gh, nb, s.d).total;
+size_t decode_fft_smem_bytes(const Dims& s, int log2S, int gh, int nb, int occ) {
+    return (size_t)fft_smem_layout(log2S, s.k, gh, nb, s.d, occ).total;
 }
 
 // True if the fused kernel's staging areas hold a part's share of the coefficient rows: the rows
 // of C^K in the transform buffers at the start, the merge scratch in the stage ring at the end.
-bool decode_fft_fused_fits(const Dims& s, int log2S, int gh, int nb, int n_part) {
+bool decode_fft_fused_fits(const Dims& s, int log2S, int gh, int nb, int n_part, int occ) {
     if (s.M % 4 != 0) return false;
-    const FftSmem L = fft_smem_layout(log2S, s.k, gh, nb, s.d);
+    if (occ == 2 && log2S > 8) return false;                                           // no two-per-SM build of the long transforms
+    const FftSmem L = fft_smem_layout(log2S, s.k, gh, nb, s.d, occ);
     if (s.dck > 0 && (long long)nb * L.fb_floats < 8LL * s.dck) return false;           // at least eight rows of C^K per chunk
-    const long long ring = (long long)kStages * kStageBytes / 4;
+    const long long ring = (long long)ring_stages(occ) * kStageBytes / 4;
     const long long nrg = s.dcv ? kConsumers / (s.dcv >> 2) : 0;
     const long long head = ((2LL * gh * n_part + gh + 3) & ~3LL);
     if (s.dcv > 0 && (ring - head - nrg * gh * s.dcv) / (gh + s.dcv + (long long)gh * n_part) < 8) return false;   // and of C^V

@@ -389,6 +389,35 @@ def test_fused_decode_one_cta_per_head():
     pair.check_state()
 
 
+@pytest.mark.parametrize("T,P,M", [(1024, 8, 128), (2048, 4, 512)])
+def test_fused_decode_more_heads_than_sms(T, P, M):
+    """More (batch row, KV head) pairs than SMs: still one launch, one CTA per pair running in waves and
+    waiting for nobody (no counters, plain launch).  Transform length 128: two CTAs share an SM (shorter
+    ring, register cap); 512: one per SM."""
+    shape = SMALL_BF16.with_(B=20, Hq=16, Hkv=8, L=700, T=T, M=M, n_full_k=32, n_full_v=48, decode_steps=2)
+    pair, stream = make_pair(shape, seed=23, algo=fa.FA_DECODE_FFT, P=P)
+    assert fa.fa_launch_count(pair.layout, 2) == 1 and fa.fa_launch_count(pair.layout, 3) == 2
+    pair.check_decode(synth.queries(shape, seed=23))
+    K, V = stream.tokens(shape.L, shape.L + 2)
+    for t in range(2):
+        pair.check_step(synth.queries(shape, seed=23, step=t + 1), K[:, t], V[:, t])
+    pair.check_state()
+
+
+@pytest.mark.parametrize("B", [1, 3])
+def test_fused_decode_two_ctas_per_sm_cooperative(B):
+    """Short transforms with fewer heads than SMs: a head's parts are two to an SM and still wait for one
+    another (cooperative launch over 2 x SMs resident CTAs)."""
+    shape = SMALL_BF16.with_(B=B, Hq=32, Hkv=16, L=1800, T=2048, M=256, n_full_k=48, n_full_v=32, decode_steps=3)
+    pair, stream = make_pair(shape, seed=24, algo=fa.FA_DECODE_FFT, P=16)
+    assert fa.fa_launch_count(pair.layout, 2) == 1
+    pair.check_decode(synth.queries(shape, seed=24))
+    K, V = stream.tokens(shape.L, shape.L + 3)
+    for t in range(3):
+        pair.check_step(synth.queries(shape, seed=24, step=t + 1), K[:, t], V[:, t])
+    pair.check_state()
+
+
 def test_workspace_counters_must_start_at_zero_and_init_restores_them():
     """A workspace full of garbage is made usable by fa_workspace_init."""
     shape = SMALL_BF16.with_(B=1, Hq=4, Hkv=1, L=500, T=1024, M=64)
