@@ -40,19 +40,26 @@ cudaError_t launch_validate(const Dims& s, const CacheDev& c, cudaStream_t st) {
 }
 
 // ---- Eq.1-2: windows, kept dims, counters -----------------------------------
-// grid (token chunks, Hkv, B * 2 sides); one warp per token row.
+// grid (chunks of 64 tokens, Hkv, B * 2 sides).  Every row of the input, of the windows and of the
+// kept-dim rows starts on a 16-byte boundary and is a whole number of 16-byte chunks (the C ABI asks
+// for 16-byte aligned K, V and strides that are multiples of 8 elements; head_dim and the kept-dim
+// counts are multiples of 8).  The CTA stages its 64 input rows in shared memory with one 16-byte load
+// per chunk, then one thread per output chunk either copies it (window rows) or gathers its dims
+// through the index set (kept-dim rows; for V^mu of bf16 caches the chunk it writes is the permuted one).
 constexpr int kRowsPerCta = 64;
 
 template <typename KV>
 __global__ void __launch_bounds__(256) partition_gather_kernel(Dims s, CacheDev c, const KV* __restrict__ K,
-                                                               const KV* __restrict__ V, int64_t sb, int64_t st,
-                                                               int64_t sh, int L) {
-    __shared__ float row_s[8][256];
-    int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    int h = blockIdx.y, b = blockIdx.z >> 1, side = blockIdx.z & 1;
-    int n_init = min(L, s.l_init);
-    int n_local = min(L - n_init, s.l_local);
-    int n_mid = L - n_init - n_local;
+                                                                   const KV* __restrict__ V, int64_t sb, int64_t st,
+                                                                   int64_t sh, int L) {
+    constexpr int EPC = 16 / (int)sizeof(KV);            // elements per chunk
+    extern __shared__ __align__(16) unsigned char gsm[];
+    KV* rows_s = reinterpret_cast<KV*>(gsm);                                         // [64][d]
+    int32_t* idf_s = reinterpret_cast<int32_t*>(gsm + (size_t)kRowsPerCta * s.d * sizeof(KV));   // [nfull]
+    const int h = blockIdx.y, b = blockIdx.z >> 1, side = blockIdx.z & 1;
+    const int n_init = min(L, s.l_init);
+    const int n_local = min(L - n_init, s.l_local);
+    const int n_mid = L - n_init - n_local;
     if (blockIdx.x == 0 && blockIdx.y == 0 && side == 0 && threadIdx.x == 0) {
         c.state[kStateStride * b + 0] = n_init;
         c.state[kStateStride * b + 1] = n_local;
@@ -60,32 +67,42 @@ __global__ void __launch_bounds__(256) partition_gather_kernel(Dims s, CacheDev 
         c.state[kStateStride * b + 3] = 0;          // ring starts at physical row 0
         c.state[kStateStride * b + 4] = 0;          // append ticket
     }
-    const KV* X = side == 0 ? K : V;
-    int nfull = side == 0 ? s.nfk : s.nfv;
+    const KV* X = (side == 0 ? K : V) + (size_t)b * sb + (size_t)h * sh;
+    const int nfull = side == 0 ? s.nfk : s.nfv;
     const int32_t* idf = (side == 0 ? c.idx_full_k : c.idx_full_v) + (size_t)h * nfull;
     void* w_init = side == 0 ? c.k_init : c.v_init;
     void* w_local = side == 0 ? c.k_local : c.v_local;
     void* w_mid = side == 0 ? c.k_mid : c.v_mid;
-    int t_end = min(L, (int)(blockIdx.x + 1) * kRowsPerCta);
-    for (int t = blockIdx.x * kRowsPerCta + warp; t < t_end; t += 8) {
-        const KV* src = X + (size_t)b * sb + (size_t)t * st + (size_t)h * sh;
-        if (t < n_init) {
-            KV* dst = win_row<KV>(w_init, s, b, h, s.l_init, t);
-            for (int e = lane; e < s.d; e += 32) dst[e] = src[e];
-        } else if (t >= L - n_local) {
-            KV* dst = win_row<KV>(w_local, s, b, h, s.l_local, t - (L - n_local));
-            for (int e = lane; e < s.d; e += 32) dst[e] = src[e];
-        } else {
-            int j = t - n_init;
-            for (int e = lane; e < s.d; e += 32) row_s[warp][e] = ld_f(src + e);
-            __syncwarp();
-            KV* dst = mid_row<KV>(w_mid, s, b, h, j % s.P, j / s.P, nfull);
-            for (int e = lane; e < nfull; e += 32) {
-                const int col = side == 1 ? v_mid_col(j / s.P, e, nfull, sizeof(KV) == 2 ? FA_BF16 : FA_F32) : e;
-                st_f(dst + col, row_s[warp][idf[e]]);
-            }
-            __syncwarp();
-        }
+    const int t0 = blockIdx.x * kRowsPerCta, nrow = min(L - t0, kRowsPerCta);
+    const int cpr = s.d / EPC;                            // chunks per input row
+    for (int i = threadIdx.x; i < nfull; i += blockDim.x) idf_s[i] = idf[i];
+    for (int i = threadIdx.x; i < nrow * cpr; i += blockDim.x) {
+        const int r = i / cpr, ch = i - r * cpr;
+        reinterpret_cast<uint4*>(rows_s)[i] = __ldg(reinterpret_cast<const uint4*>(X + (size_t)(t0 + r) * st) + ch);
+    }
+    __syncthreads();
+    // window rows: chunk for chunk
+    for (int i = threadIdx.x; i < nrow * cpr; i += blockDim.x) {
+        const int r = i / cpr, ch = i - r * cpr, t = t0 + r;
+        KV* dst = nullptr;
+        if (t < n_init) dst = win_row<KV>(w_init, s, b, h, s.l_init, t);
+        else if (t >= L - n_local) dst = win_row<KV>(w_local, s, b, h, s.l_local, t - (L - n_local));
+        if (dst) reinterpret_cast<uint4*>(dst)[ch] = reinterpret_cast<const uint4*>(rows_s)[i];
+    }
+    // kept-dim rows of the middle
+    const int cpo = nfull / EPC;                          // chunks per output row
+    for (int i = threadIdx.x; i < nrow * cpo; i += blockDim.x) {
+        const int r = i / cpo, ch = i - r * cpo, t = t0 + r;
+        if (t < n_init || t >= L - n_local) continue;
+        const int j = t - n_init, cls = j % s.P, slot = j / s.P;
+        // output chunk ch holds the logical chunk ch ^ swizzle (the permutation is an involution)
+        const int lch = (side == 1 && sizeof(KV) == 2) ? (ch ^ v_swz(slot, nfull >> 3)) : ch;
+        const KV* row = rows_s + r * s.d;
+        __align__(16) KV vals[EPC];
+#pragma unroll
+        for (int e = 0; e < EPC; ++e) vals[e] = row[idf_s[lch * EPC + e]];
+        KV* dst = mid_row<KV>(w_mid, s, b, h, cls, slot, nfull);
+        reinterpret_cast<uint4*>(dst)[ch] = *reinterpret_cast<const uint4*>(vals);
     }
 }
 
@@ -177,9 +194,17 @@ static cudaError_t launch_compress_t(const Dims& s, const CacheDev& c, const voi
                                      int64_t st, int64_t sh, int L, bool with_coef, cudaStream_t stream) {
     int chunks_rows = (L + kRowsPerCta - 1) / kRowsPerCta;
     if (chunks_rows < 1) chunks_rows = 1;
-    partition_gather_kernel<KV><<<dim3(chunks_rows, s.Hkv, s.B * 2), 256, 0, stream>>>(
+    constexpr int EPC = 16 / (int)sizeof(KV);
+    if (s.d % EPC || s.nfk % EPC || s.nfv % EPC || sb % EPC || st % EPC || sh % EPC || (reinterpret_cast<uintptr_t>(K) & 15) ||
+        (reinterpret_cast<uintptr_t>(V) & 15))
+        return cudaErrorInvalidValue;
+    const int nf = s.nfk > s.nfv ? s.nfk : s.nfv;
+    const size_t gsmem = (size_t)kRowsPerCta * s.d * sizeof(KV) + sizeof(int32_t) * (size_t)nf;
+    cudaError_t err = ensure_dynamic_smem(partition_gather_kernel<KV>, gsmem);
+    if (err != cudaSuccess) return err;
+    partition_gather_kernel<KV><<<dim3(chunks_rows, s.Hkv, s.B * 2), 256, gsmem, stream>>>(
         s, c, static_cast<const KV*>(K), static_cast<const KV*>(V), sb, st, sh, L);
-    cudaError_t err = cudaGetLastError();
+    err = cudaGetLastError();
     if (err != cudaSuccess) return err;
     int n_init = L < s.l_init ? L : s.l_init;
     int n_local = (L - n_init) < s.l_local ? (L - n_init) : s.l_local;

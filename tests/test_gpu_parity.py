@@ -171,6 +171,11 @@ def test_errors_are_reported_not_raised_on_device():
     assert fa.fa_poll_status(pair.gpu) == fa.FA_OK             # and cleared by the poll
     for n, t in before.items():
         assert torch.equal(getattr(pair.gpu, n), t), n         # the refused append changed nothing
+    # prefill rows off the 16-byte grid (a view one element into a wider buffer) are refused, nothing is launched
+    wide = torch.zeros((1, 78, shape.Hkv, shape.d + 8), dtype=K.dtype, device="cuda")
+    with pytest.raises(fa.FaError) as e:
+        fa.fa_compress(layout, pair.gpu, wide[..., 1:shape.d + 1], wide[..., 1:shape.d + 1], pair.ws)
+    assert e.value.status == fa.FA_ERR_INVALID_ARG
     # workspace too small / missing
     q = synth.queries(shape, seed=9).cuda()
     out = torch.empty_like(q)
