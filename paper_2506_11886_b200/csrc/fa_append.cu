@@ -1,10 +1,11 @@
 // fa_append (Eq.5): push one token; when the local window is full its oldest
 // row leaves, its kept dims join K^mu / V^mu and its compressed dims are added
 // to every coefficient row with basis column j = n_mid.  One kernel:
-//   grid (row tiles, Hkv, B).  Each CTA updates kAppendRows rows of C^K and C^V
-//   (every float4 read-modify-write independent of the others, all loads issued
-//   before the first store); CTA x == 0 also writes the leaving row's kept dims
-//   to the middle.  The last CTA of a batch row to finish (atomic ticket, no
+//   grid (row tiles, Hkv, B).  Each CTA updates kAppendRows rows of C^K and C^V:
+//   the rows are contiguous, so one bulk copy per side brings them to shared
+//   memory (issued before anything else, completion on an mbarrier), the rank-1
+//   update runs there and one bulk copy per side takes them back; CTA x == 0 also
+//   writes the leaving row's kept dims to the middle.  The last CTA of a batch row to finish (atomic ticket, no
 //   waiting) overwrites the ring slot with the new token and advances the
 //   counters, so no CTA can see a half-updated state.
 #include "fa_common.cuh"
@@ -12,21 +13,76 @@
 
 namespace fa {
 
-constexpr int kAppendRows = 32;   // coefficient rows per CTA (halved when more than 128 dims are compressed)
-constexpr int kAppendVec = 4;     // float4 read-modify-writes per thread and side (dims <= 128 compressed)
+constexpr int kAppendRows = 32;   // coefficient rows per CTA
+constexpr uint32_t kAppendSpin = 1u << 22;
 
+namespace {
+__device__ __forceinline__ uint32_t sm_addr(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+}  // namespace
+
+// A CTA's life is a chain of dependent memory round trips (counters, leaving row, ticket), so what counts
+// is how many bytes are in flight per SM: the coefficient rows travel as bulk copies whose round trip
+// overlaps the counters', several CTAs to an SM.
 template <typename KV>
 __global__ void __launch_bounds__(256) append_kernel(Dims s, CacheDev c, const KV* __restrict__ k_new,
                                                      const KV* __restrict__ v_new, int rows_per_cta) {
+    extern __shared__ __align__(128) float coef_s[];   // [rows][dck] of C^K, then [rows][dcv] of C^V
     __shared__ float x_s[2][256];        // the row that leaves, both sides, natural dim order
     __shared__ __align__(16) float xc_s[2][256];   // the same gathered at D^kc / D^vc
     __shared__ float f_s[kAppendRows];   // basis column j for the rows of this CTA
+    __shared__ __align__(8) uint64_t bar_s;
     __shared__ int last_s;
     const int h = blockIdx.y, b = blockIdx.z, tid = threadIdx.x;
     // programmatic dependent launch: the next kernel may be scheduled now; this one first waits for
     // everything its predecessor in the stream wrote
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     asm volatile("griddepcontrol.wait;" ::: "memory");
+    // The coefficient rows set off first: their addresses depend on the grid alone, so their round trip
+    // overlaps the one of the counters.  Every path below waits for them before the CTA ends.
+    const int m0 = blockIdx.x * rows_per_cta;
+    const int rows = min(rows_per_cta, s.M - m0);
+    float* ck_s = coef_s;
+    float* cv_s = coef_s + (size_t)rows_per_cta * s.dck;
+    float* ckg = s.dck ? coef_rows(c.coef_k, s, b, h, s.dck) + (size_t)m0 * s.dck : nullptr;
+    float* cvg = s.dcv ? coef_rows(c.coef_v, s, b, h, s.dcv) + (size_t)m0 * s.dcv : nullptr;
+    const uint32_t bytes_k = (uint32_t)(rows * s.dck * 4), bytes_v = (uint32_t)(rows * s.dcv * 4);
+    const bool any_coef = bytes_k + bytes_v > 0;
+    if (tid == 0 && any_coef) {
+        asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(sm_addr(&bar_s)));
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(sm_addr(&bar_s)), "r"(bytes_k + bytes_v) : "memory");
+        if (bytes_k)
+            asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(sm_addr(ck_s)),
+                         "l"(__cvta_generic_to_global(ckg)), "r"(bytes_k), "r"(sm_addr(&bar_s))
+                         : "memory");
+        if (bytes_v)
+            asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(sm_addr(cv_s)),
+                         "l"(__cvta_generic_to_global(cvg)), "r"(bytes_v), "r"(sm_addr(&bar_s))
+                         : "memory");
+    }
+    // Bounded wait for the rows (one thread polls, then the CTA meets); false after a time-out.
+    auto rows_landed = [&]() -> bool {
+        __shared__ int ok_s;
+        if (tid == 0) {
+            int ok = 1;
+            if (any_coef) {
+                ok = 0;
+                for (uint32_t i = 0; i < kAppendSpin && !ok; ++i) {
+                    uint32_t done;
+                    asm volatile(
+                        "{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], 0;\n selp.u32 %0, 1, 0, p;\n}\n"
+                        : "=r"(done)
+                        : "r"(sm_addr(&bar_s))
+                        : "memory");
+                    ok = (int)done;
+                }
+                if (!ok) atomicExch(c.status, (int)FA_ERR_TIMEOUT);
+            }
+            ok_s = ok;
+        }
+        __syncthreads();
+        return ok_s != 0;
+    };
     const int n_init = c.state[kStateStride * b + 0], n_local = c.state[kStateStride * b + 1];
     const int n_mid = c.state[kStateStride * b + 2], head = c.state[kStateStride * b + 3];
     const bool to_init = n_init < s.l_init;
@@ -34,27 +90,12 @@ __global__ void __launch_bounds__(256) append_kernel(Dims s, CacheDev c, const K
     const bool full = evict && (n_mid >= s.max_mid || n_mid >= s.T);
     if (full) {
         if (tid == 0 && blockIdx.x == 0 && h == 0) atomicExch(c.status, (int)FA_ERR_CAPACITY);
+        rows_landed();                   // nothing may still be writing this CTA's shared memory when it ends
         return;                          // every CTA of this batch row takes the same exit
     }
+    if (!evict) rows_landed();
     if (evict) {
         const int j = n_mid;
-        const int m0 = blockIdx.x * rows_per_cta;
-        const int rows = min(rows_per_cta, s.M - m0);
-        // start the coefficient loads first: they do not depend on anything computed here
-        float4 cur[2][kAppendVec];
-        float4* ptr[2][kAppendVec];
-#pragma unroll
-        for (int side = 0; side < 2; ++side) {
-            const int ncomp = side == 0 ? s.dck : s.dcv;
-            const int vpr = ncomp >> 2;
-            float* coef = ncomp ? coef_rows(side == 0 ? c.coef_k : c.coef_v, s, b, h, ncomp) + (size_t)m0 * ncomp : nullptr;
-#pragma unroll
-            for (int u = 0; u < kAppendVec; ++u) {
-                const int i = tid + 256 * u;
-                ptr[side][u] = (ncomp && i < rows * vpr) ? reinterpret_cast<float4*>(coef) + i : nullptr;
-                if (ptr[side][u]) cur[side][u] = *ptr[side][u];
-            }
-        }
         // the row that leaves: oldest ring row, or the new token itself if there is no local window
         for (int i = tid; i < 2 * s.d; i += 256) {
             const int side = i / s.d, e = i - side * s.d;
@@ -87,29 +128,44 @@ __global__ void __launch_bounds__(256) append_kernel(Dims s, CacheDev c, const K
                 st_f(dst + col, x_s[side][idf[e]]);
             }
         }
-        __syncthreads();
+        if (rows_landed()) {             // (a CTA-wide barrier: f_s and xc_s are complete too)
 #pragma unroll
-        for (int side = 0; side < 2; ++side) {
-            const int ncomp = side == 0 ? s.dck : s.dcv;
-            const int vpr = ncomp >> 2;
-#pragma unroll
-            for (int u = 0; u < kAppendVec; ++u) {
-                if (!ptr[side][u]) continue;
-                const int i = tid + 256 * u;
-                const int r = i / vpr, v4 = i - r * vpr;
-                const float f = f_s[r];
-                const float4 x = *reinterpret_cast<const float4*>(&xc_s[side][4 * v4]);
-                float4 o = cur[side][u];
-                o.x = fmaf(f, x.x, o.x);
-                o.y = fmaf(f, x.y, o.y);
-                o.z = fmaf(f, x.z, o.z);
-                o.w = fmaf(f, x.w, o.w);
-                *ptr[side][u] = o;
+            for (int side = 0; side < 2; ++side) {
+                const int ncomp = side == 0 ? s.dck : s.dcv;
+                const int vpr = ncomp >> 2;
+                float4* rows4 = reinterpret_cast<float4*>(side == 0 ? ck_s : cv_s);
+#pragma unroll 4
+                for (int i = tid; i < rows * vpr; i += 256) {
+                    const int r = i / vpr, v4 = i - r * vpr;
+                    const float f = f_s[r];
+                    const float4 x = *reinterpret_cast<const float4*>(&xc_s[side][4 * v4]);
+                    float4 o = rows4[i];
+                    o.x = fmaf(f, x.x, o.x);
+                    o.y = fmaf(f, x.y, o.y);
+                    o.z = fmaf(f, x.z, o.z);
+                    o.w = fmaf(f, x.w, o.w);
+                    rows4[i] = o;
+                }
+            }
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");    // these stores, then the bulk copies that read them
+            __syncthreads();
+            if (tid == 0 && any_coef) {
+                if (bytes_k)
+                    asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(__cvta_generic_to_global(ckg)),
+                                 "r"(sm_addr(ck_s)), "r"(bytes_k)
+                                 : "memory");
+                if (bytes_v)
+                    asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(__cvta_generic_to_global(cvg)),
+                                 "r"(sm_addr(cv_s)), "r"(bytes_v)
+                                 : "memory");
+                asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+                asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");   // shared memory has been read: the CTA may end
             }
         }
     }
-    // ticket: the last CTA of this batch row stores the new token and advances the counters
-    __threadfence();
+    // ticket: the last CTA of this batch row stores the new token and advances the counters.  What the
+    // ticket orders is every CTA's read of the leaving row (consumed above) before the overwrite of its
+    // ring slot; the coefficient stores need no fence here, the end of the kernel publishes them.
     __syncthreads();
     if (tid == 0) {
         const int done = atomicAdd(c.state + kStateStride * b + 4, 1);
@@ -118,16 +174,31 @@ __global__ void __launch_bounds__(256) append_kernel(Dims s, CacheDev c, const K
     __syncthreads();
     if (!last_s) return;
     __threadfence();
-    for (int i = tid; i < 2 * s.Hkv * s.d; i += 256) {
-        const int side = i / (s.Hkv * s.d);
-        const int rem = i - side * (s.Hkv * s.d);
-        const int hh = rem / s.d, e = rem - hh * s.d;
-        const KV* src = (side == 0 ? k_new : v_new) + ((size_t)b * s.Hkv + hh) * s.d;
-        if (to_init) {
-            win_row<KV>(side == 0 ? c.k_init : c.v_init, s, b, hh, s.l_init, n_init)[e] = src[e];
-        } else if (s.l_local > 0) {
-            const int slot = evict ? head : (head + n_local) % s.l_local;
-            win_row<KV>(side == 0 ? c.k_local : c.v_local, s, b, hh, s.l_local, slot)[e] = src[e];
+    // The new token of every head of this batch row, in 16-byte chunks, all loads of a round before its
+    // stores: this CTA runs alone at the end of the kernel, so its round trips are the kernel's tail.
+    if (to_init || s.l_local > 0) {
+        constexpr int EPC = 16 / (int)sizeof(KV);
+        const int cpr = s.d / EPC, nchunk = 2 * s.Hkv * cpr;
+        const int slot = to_init ? n_init : (evict ? head : (head + n_local) % s.l_local);
+#pragma unroll 1
+        for (int base = 0; base < nchunk; base += 256 * 4) {
+            uint4 v[4];
+            uint4* dst[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const int i = base + tid + 256 * u;
+                dst[u] = nullptr;
+                if (i < nchunk) {
+                    const int side = i / (s.Hkv * cpr), rem = i - side * (s.Hkv * cpr);
+                    const int hh = rem / cpr, ch = rem - hh * cpr;
+                    v[u] = reinterpret_cast<const uint4*>((side == 0 ? k_new : v_new) + ((size_t)b * s.Hkv + hh) * s.d)[ch];
+                    void* w = to_init ? (side == 0 ? c.k_init : c.v_init) : (side == 0 ? c.k_local : c.v_local);
+                    dst[u] = reinterpret_cast<uint4*>(win_row<KV>(w, s, b, hh, to_init ? s.l_init : s.l_local, slot)) + ch;
+                }
+            }
+#pragma unroll
+            for (int u = 0; u < 4; ++u)
+                if (dst[u]) *dst[u] = v[u];
         }
     }
     __syncthreads();
@@ -239,12 +310,15 @@ __global__ void __launch_bounds__(256) append_lite_kernel(Dims s, CacheDev c, De
 template <typename KV>
 static cudaError_t launch_append_t(const Dims& s, const CacheDev& c, const void* k_new, const void* v_new,
                                    cudaStream_t st) {
-    const int max_comp = s.dck > s.dcv ? s.dck : s.dcv;
-    const int rows = max_comp > 128 ? kAppendRows / 2 : kAppendRows;     // rows * max_comp / 4 <= 256 * kAppendVec
+    const int rows = kAppendRows;
     const int tiles = (s.M + rows - 1) / rows;
+    const size_t smem = sizeof(float) * (size_t)rows * (s.dck + s.dcv);
+    cudaError_t err = ensure_dynamic_smem(append_kernel<KV>, smem);
+    if (err != cudaSuccess) return err;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(tiles, s.Hkv, s.B);
     cfg.blockDim = dim3(256);
+    cfg.dynamicSmemBytes = smem;
     cfg.stream = st;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
