@@ -274,23 +274,31 @@ __global__ void __launch_bounds__(kThreadsTc, 1) compress_tc_kernel(const __grid
             if (ok) {
                 const int lane_grp = warp & 3;             // a warp reads tensor-memory lanes 32 (warp % 4) ...
                 const int col_half = (warp - 2) >> 2;      // two warps share a lane group: one column half each
-                const int m = mt * kBM + lane_grp * 32 + lane;
+                const int m_base = mt * kBM + lane_grp * 32;
                 constexpr int kHalf = (int)kTmemCols / 2;
+                // A thread holds 32 columns of ONE row; added as they are, a warp's reduction would touch 32
+                // rows (32 sectors) per instruction.  Each warp transposes its 32 x 32 block through a tile of
+                // its own in the (now idle: every MMA has read it) stage ring, so that a reduction instruction
+                // covers 32 columns of one row: the compressed ones among them are neighbours in memory.
+                float* tile = reinterpret_cast<float*>(stage0) + (warp - 2) * (32 * 33);
 #pragma unroll 1
                 for (int col0 = col_half * kHalf; col0 < (col_half + 1) * kHalf; col0 += 32) {
                     const int hh = col0 / N, hcol0 = col0 - hh * N;
-                    float* ck = coef_rows(c.coef_k, s, b, h0 + hh, s.dck) + (size_t)m * s.dck;
-                    float* cv = coef_rows(c.coef_v, s, b, h0 + hh, s.dcv) + (size_t)m * s.dcv;
+                    const bool is_k = hcol0 < D;           // a block of 32 columns lies within K's dims or within V's
+                    const int ncomp = is_k ? s.dck : s.dcv;
+                    float* base = coef_rows(is_k ? c.coef_k : c.coef_v, s, b, h0 + hh, ncomp) + (size_t)m_base * ncomp;
                     float v[32];
                     tmem_ld32(tmem_base + ((uint32_t)(lane_grp * 32) << 16) + (uint32_t)col0, v);
-                    if (m < s.M) {
 #pragma unroll
-                        for (int i = 0; i < 32; ++i) {
-                            const int col = hcol0 + i;
-                            const int slot = inv[hh * N + col];
-                            if (slot >= 0) atomicAdd((col < D ? ck : cv) + slot, v[i]);
-                        }
+                    for (int i = 0; i < 32; ++i) tile[lane * 33 + i] = v[i];
+                    __syncwarp();
+                    const int slot = inv[hh * N + hcol0 + lane];
+                    if (slot >= 0) {
+#pragma unroll 4
+                        for (int rr = 0; rr < 32; ++rr)
+                            if (m_base + rr < s.M) atomicAdd(base + (size_t)rr * ncomp + slot, tile[rr * 33 + lane]);
                     }
+                    __syncwarp();
                 }
             }
         }
