@@ -195,8 +195,10 @@ fa_status fa_decode_step(const fa_layout* layout, fa_cache* cache, const void* q
  * fa_step_staging_bytes(layout) bytes; k_new_host == NULL skips the append.  Asynchronous on
  * `stream`: out_host is valid after the stream is synchronised.  Host buffers that the device can
  * address (pinned or registered memory, 16-byte aligned) are not copied by separate copy
- * operations: one staging kernel reads q, k_new, v_new over the bus, and the decode kernel writes
- * its result rows straight into out_host. */
+ * operations: the step's first kernel reads k_new, v_new in place over the bus and copies q into
+ * `staging` (when the step is not the fused two-kernel form, one staging kernel in front of it
+ * reads all three), and the decode kernel writes its result rows straight into out_host.  The
+ * host input buffers must not be written between the call and the completion of the step. */
 fa_status fa_decode_step_host(const fa_layout* layout, fa_cache* cache, const void* q_host,
                               const void* k_new_host, const void* v_new_host, void* out_host,
                               void* staging, void* ws, size_t ws_bytes, void* stream);

@@ -441,8 +441,13 @@ fa_status fa_decode_attention(const fa_layout* layout, const fa_cache* cache, co
     return FA_OK;
 }
 
-fa_status fa_decode_step(const fa_layout* layout, fa_cache* cache, const void* q, const void* k_new, const void* v_new,
-                         void* out, void* ws, size_t ws_bytes, void* stream) {
+}  // extern "C"
+
+// fa_decode_step.  With q_host_view set (host-buffer step, pinned inputs, fused plan only): k_new / v_new
+// and q_host_view are device views of pinned host memory; the light append kernel reads them over the bus
+// and copies the query to q (device memory) for the decode kernel.
+static fa_status decode_step_impl(const fa_layout* layout, fa_cache* cache, const void* q, const void* k_new, const void* v_new,
+                                  void* out, void* ws, size_t ws_bytes, void* stream, const void* q_host_view, size_t q_bytes) {
     fa_status st = check_layout(layout);
     if (st != FA_OK) return st;
     st = check_cache(layout, cache);
@@ -454,6 +459,7 @@ fa_status fa_decode_step(const fa_layout* layout, fa_cache* cache, const void* q
     if (st != FA_OK) return st;
     if (!ws || !aligned16(ws) || ws_bytes < p.total) return FA_ERR_WORKSPACE;
     if (!(p.fused && p.n_pass == 1)) {
+        if (q_host_view) return FA_ERR_UNSUPPORTED;          // (the caller checks the plan first)
         // two calls: the coefficient update cannot ride on the decode kernel's passes over the rows
         st = fa_append(layout, cache, k_new, v_new, stream);
         if (st != FA_OK) return st;
@@ -471,13 +477,23 @@ fa_status fa_decode_step(const fa_layout* layout, fa_cache* cache, const void* q
                      cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, dev) == cudaSuccess && coop) ? 1 : 0;
     }
     if (!coop_fits) {
+        if (q_host_view) return FA_ERR_UNSUPPORTED;
         st = fa_append(layout, cache, k_new, v_new, stream);
         if (st != FA_OK) return st;
         return fa_decode_attention(layout, cache, q, out, ws, ws_bytes, stream);
     }
-    if (launch_append_lite(s, c, layout->kv_dtype, p, k_new, v_new, w, cs) != cudaSuccess) return FA_ERR_CUDA;
+    if (launch_append_lite(s, c, layout->kv_dtype, p, k_new, v_new, w, cs, q_host_view, q_host_view ? const_cast<void*>(q) : nullptr,
+                           q_bytes, q_host_view != nullptr) != cudaSuccess)
+        return FA_ERR_CUDA;
     if (launch_decode_fft(s, c, layout->kv_dtype, p, q, out, w, true, cs) != cudaSuccess) return FA_ERR_CUDA;
     return FA_OK;
+}
+
+extern "C" {
+
+fa_status fa_decode_step(const fa_layout* layout, fa_cache* cache, const void* q, const void* k_new, const void* v_new,
+                         void* out, void* ws, size_t ws_bytes, void* stream) {
+    return decode_step_impl(layout, cache, q, k_new, v_new, out, ws, ws_bytes, stream, nullptr, 0);
 }
 
 size_t fa_step_staging_bytes(const fa_layout* layout) {
@@ -512,7 +528,18 @@ fa_status fa_decode_step_host(const fa_layout* layout, fa_cache* cache, const vo
     void* out_v = aligned16(out_host) ? const_cast<void*>(device_view_of_host(out_host)) : nullptr;
     if (out_v) o_d = static_cast<char*>(out_v);
     if (q_v && k_v && v_v) {
-        // pinned inputs: one staging kernel reads them over the bus (measured faster than three copy
+        // Pinned inputs, fused step: the light append kernel reads k_new / v_new in place and copies q for the
+        // decode kernel (its loads go out before its wait on the previous kernel): no launch in front of the step.
+        DecodePlan hp;
+        if (plan_decode(*layout, &hp) == FA_OK && hp.fused && hp.n_pass == 1) {
+            st = decode_step_impl(layout, cache, q_d, k_v, v_v, o_d, ws, ws_bytes, stream, q_v, q_bytes);
+            if (st != FA_ERR_UNSUPPORTED) {
+                if (st != FA_OK) return st;
+                if (!out_v && cudaMemcpyAsync(out_host, o_d, q_bytes, cudaMemcpyDeviceToHost, cs) != cudaSuccess) return FA_ERR_CUDA;
+                return FA_OK;
+            }
+        }
+        // otherwise one staging kernel reads them over the bus (measured faster than three copy
         // operations, and than letting every CTA of the step read the host buffers in place)
         const int nq = (int)(q_bytes / 16), nk = (int)(k_bytes / 16);
         cudaLaunchConfig_t cfg = {};

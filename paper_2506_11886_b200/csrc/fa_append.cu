@@ -217,16 +217,44 @@ __global__ void __launch_bounds__(256) append_kernel(Dims s, CacheDev c, const K
 // the counters, and leaves the compressed dims of the leaving row with its basis column j in the
 // workspace.  The decode kernel of the same step adds f_j x^T to the coefficient rows as it streams
 // them, so the coefficients are read and written once per step instead of twice.
+// Host-buffer step: with host_inputs set, k_new / v_new (and q_src) are device views of pinned host
+// memory.  Nothing earlier in the stream writes them, so their loads go out before the wait and the bus
+// round trip hides under the previous kernel's tail; q is copied to q_dst (device memory) for the decode
+// kernel, which saves a staging launch in front of the step.
 template <typename KV>
 __global__ void __launch_bounds__(256) append_lite_kernel(Dims s, CacheDev c, DecodePlan p, const KV* __restrict__ k_new,
-                                                          const KV* __restrict__ v_new, char* wsp) {
+                                                          const KV* __restrict__ v_new, char* wsp, const uint4* __restrict__ q_src,
+                                                          uint4* __restrict__ q_dst, int nq16, int host_inputs) {
     __shared__ float x_s[2][256];        // the row that leaves, both sides, natural dim order
     __shared__ int last_s;
     const int h = blockIdx.x, b = blockIdx.y, tid = threadIdx.x;
+    // the new token of this head (up to two elements per thread)
+    KV new_e[2];
+    auto load_new = [&]() {
+#pragma unroll
+        for (int u = 0; u < 2; ++u) {
+            const int i = tid + 256 * u;
+            if (i < 2 * s.d) {
+                const int side = i / s.d, e = i - side * s.d;
+                new_e[u] = ((side == 0 ? k_new : v_new) + ((size_t)b * s.Hkv + h) * s.d)[e];
+            }
+        }
+    };
+    const int gid = (b * (int)gridDim.x + h) * 256 + tid, gtot = (int)(gridDim.x * gridDim.y) * 256;
+    uint4 qv = make_uint4(0, 0, 0, 0);
+    if (host_inputs) {
+        load_new();
+        if (q_src && gid < nq16) qv = q_src[gid];
+    }
     // wait for everything before this kernel, THEN let the decode kernel of the step start: it reads
     // coefficient rows before its own wait, and nothing but this kernel may still be running then
     asm volatile("griddepcontrol.wait;" ::: "memory");
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    if (q_src) {                         // (the previous step's decode kernel has read q_dst by now)
+        if (gid < nq16) q_dst[gid] = host_inputs ? qv : q_src[gid];
+#pragma unroll 1
+        for (int i = gid + gtot; i < nq16; i += gtot) q_dst[i] = q_src[i];
+    }
     Ws ws = ws_view(wsp, p);
     const int n_init = c.state[kStateStride * b + 0], n_local = c.state[kStateStride * b + 1];
     const int n_mid = c.state[kStateStride * b + 2], head = c.state[kStateStride * b + 3];
@@ -237,16 +265,7 @@ __global__ void __launch_bounds__(256) append_lite_kernel(Dims s, CacheDev c, De
         if (tid == 0 && h == 0) { atomicExch(c.status, (int)FA_ERR_CAPACITY); ws.pend_j[b] = -1; }
         return;                          // every CTA of this batch row takes the same exit
     }
-    // the new token of this head (up to two elements per thread), loaded together with the leaving row
-    KV new_e[2];
-#pragma unroll
-    for (int u = 0; u < 2; ++u) {
-        const int i = tid + 256 * u;
-        if (i < 2 * s.d) {
-            const int side = i / s.d, e = i - side * s.d;
-            new_e[u] = ((side == 0 ? k_new : v_new) + ((size_t)b * s.Hkv + h) * s.d)[e];
-        }
-    }
+    if (!host_inputs) load_new();        // device-resident inputs: loaded together with the leaving row
     if (evict) {
         const int j = n_mid;
         for (int i = tid; i < 2 * s.d; i += 256) {
@@ -330,7 +349,7 @@ static cudaError_t launch_append_t(const Dims& s, const CacheDev& c, const void*
 
 template <typename KV>
 static cudaError_t launch_append_lite_t(const Dims& s, const CacheDev& c, const DecodePlan& p, const void* k_new, const void* v_new,
-                                        char* ws, cudaStream_t st) {
+                                        char* ws, cudaStream_t st, const void* q_src, void* q_dst, size_t q_bytes, bool host_inputs) {
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(s.Hkv, s.B);
     cfg.blockDim = dim3(256);
@@ -340,13 +359,14 @@ static cudaError_t launch_append_lite_t(const Dims& s, const CacheDev& c, const 
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, append_lite_kernel<KV>, s, c, p, static_cast<const KV*>(k_new), static_cast<const KV*>(v_new), ws);
+    return cudaLaunchKernelEx(&cfg, append_lite_kernel<KV>, s, c, p, static_cast<const KV*>(k_new), static_cast<const KV*>(v_new), ws,
+                              static_cast<const uint4*>(q_src), static_cast<uint4*>(q_dst), (int)(q_bytes / 16), host_inputs ? 1 : 0);
 }
 
 cudaError_t launch_append_lite(const Dims& s, const CacheDev& c, int dtype, const DecodePlan& p, const void* k_new, const void* v_new,
-                               char* ws, cudaStream_t st) {
-    if (dtype == FA_BF16) return launch_append_lite_t<__nv_bfloat16>(s, c, p, k_new, v_new, ws, st);
-    return launch_append_lite_t<float>(s, c, p, k_new, v_new, ws, st);
+                               char* ws, cudaStream_t st, const void* q_src, void* q_dst, size_t q_bytes, bool host_inputs) {
+    if (dtype == FA_BF16) return launch_append_lite_t<__nv_bfloat16>(s, c, p, k_new, v_new, ws, st, q_src, q_dst, q_bytes, host_inputs);
+    return launch_append_lite_t<float>(s, c, p, k_new, v_new, ws, st, q_src, q_dst, q_bytes, host_inputs);
 }
 
 cudaError_t launch_append(const Dims& s, const CacheDev& c, int dtype, const void* k_new, const void* v_new,

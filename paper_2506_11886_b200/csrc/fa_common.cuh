@@ -109,7 +109,8 @@ cudaError_t launch_decode_prologue(const Dims&, const CacheDev&, int dtype, cons
 cudaError_t launch_decode_direct(const Dims&, const CacheDev&, int dtype, const DecodePlan&, const void* q, char* ws,
                                  cudaStream_t);
 cudaError_t launch_append_lite(const Dims&, const CacheDev&, int dtype, const DecodePlan&, const void* k_new, const void* v_new,
-                               char* ws, cudaStream_t);
+                               char* ws, cudaStream_t, const void* q_src = nullptr, void* q_dst = nullptr, size_t q_bytes = 0,
+                               bool host_inputs = false);
 cudaError_t launch_decode_fft(const Dims&, const CacheDev&, int dtype, const DecodePlan&, const void* q, void* out, char* ws, bool step,
                               cudaStream_t);
 size_t decode_fft_smem_bytes(const Dims&, int log2S, int gh, int nb, int occ = 1);
