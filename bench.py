@@ -303,7 +303,8 @@ def run_ours(args):
     launches = K_steps * fa.fa_launch_count(layout, 3)
     n_dec = fa.fa_launch_count(layout, 2)
     line = {
-        "metric": METRIC, "value": us_step / world, "unit": UNIT, "n_gpus": world, "steps": K_steps, "warmup": W,
+        "metric": METRIC if args.config == 1 else f"decode_attn_us_per_step_cfg{args.config}", "value": us_step / world, "unit": UNIT,
+        "n_gpus": world, "steps": K_steps, "warmup": W,
         "ms_per_step": us_step / 1e3, "higher_is_better": False, "scaling": "weak", "vs_baseline": None,
         "dtype": f"{shape.dtype} storage, f32 arithmetic", "data": "synthetic",
         "config": {"workload": shape.name, "global_batch": shape.B * world, "seq_len": shape.L,
