@@ -1077,11 +1077,13 @@ __global__ void __launch_bounds__(kThreads, OCC) decode_fft_kernel(const __grid_
             // packed Hermitian spectra of the nb classes: X_m = V^A_m + i V^B_m per complex lane,
             // V_m = v_m + conj(v_{S-m}), v_n = (1/2) u~_n e^{i theta n c}.  Pair 0 is bins (0, S/2).
             if (s.dck > 0) {
-                // neighbouring lanes share a pair of bins and take half of the classes each
-                const int hcls = (nb + 1) >> 1;
+                // neighbouring lanes share a pair of bins and take half of the classes each (a batch of one
+                // class: one lane per pair, half as many rounds)
+                const bool split2 = nb > 1;
+                const int hcls = split2 ? (nb + 1) >> 1 : nb;
                 #pragma unroll 1
-                for (int item = tid; item < S; item += kConsumers) {
-                    const int pr = item >> 1, ci0 = (item & 1) * hcls, ci1 = min(nb, ci0 + hcls);
+                for (int item = tid; item < (split2 ? S : S / 2); item += kConsumers) {
+                    const int pr = split2 ? item >> 1 : item, ci0 = split2 ? (item & 1) * hcls : 0, ci1 = min(nb, ci0 + hcls);
                     const int m = pr, mc = pr == 0 ? S / 2 : S - pr;
                     PC<N> Am = czero, Bm = czero, Ac = czero, Bc = czero;
                     float2 em = make_float2(1.f, 0.f), ec = make_float2(1.f, 0.f);
@@ -1216,10 +1218,11 @@ __global__ void __launch_bounds__(kThreads, OCC) decode_fft_kernel(const __grid_
                 if constexpr (N == 2) { alA = pk(alpha[0], alpha[1]); alB = pk(alpha[2], alpha[3]); }
                 else { alA = PR<1>{alpha[0]}; alB = PR<1>{alpha[1]}; }
                 const PR<N> half = splat<N>(0.5f);
-                const int hcls = (nb + 1) >> 1;
+                const bool split2 = nb > 1;                // as for the spectra: one lane per pair when the batch is one class
+                const int hcls = split2 ? (nb + 1) >> 1 : nb;
                 #pragma unroll 1
-                for (int item = tid; item < S; item += kConsumers) {       // whole warps: S is a multiple of 32
-                    const int pr = item >> 1, ci0 = (item & 1) * hcls;
+                for (int item = tid; item < (split2 ? S : S / 2); item += kConsumers) {       // split: whole warps (S is a multiple of 32)
+                    const int pr = split2 ? item >> 1 : item, ci0 = split2 ? (item & 1) * hcls : 0;
                     const int m = pr, mc = pr == 0 ? S / 2 : S - pr;
                     const int ci1 = (m >= s.k && mc >= s.k) ? ci0 : min(nb, ci0 + hcls);
                     float2 em = make_float2(1.f, 0.f), ec = make_float2(1.f, 0.f);
@@ -1252,8 +1255,10 @@ __global__ void __launch_bounds__(kThreads, OCC) decode_fft_kernel(const __grid_
                         twm = cmulf(twm, em);
                         twc = cmulf(twc, ec);
                     }
-                    zAm = pair_sum(zAm); zBm = pair_sum(zBm); zAc = pair_sum(zAc); zBc = pair_sum(zBc);
-                    if (item & 1) continue;
+                    if (split2) {
+                        zAm = pair_sum(zAm); zBm = pair_sum(zBm); zAc = pair_sum(zAc); zBc = pair_sum(zBc);
+                        if (item & 1) continue;
+                    }
                     if (m < s.k) {
                         PC<N> A, B;
                         ld_entry(z_s, m, A, B);
