@@ -486,7 +486,9 @@ __global__ void __launch_bounds__(kThreads, OCC) decode_fft_kernel(const __grid_
     // touch the coefficients (it triggers this launch after its own wait), so this part's rows of C^K
     // can start towards the transform buffers, and its rows of C^V towards L2, before the wait.
     const int m0 = part * (s.M >> 2) / p.n_part * 4, m1 = (part + 1) * (s.M >> 2) / p.n_part * 4;
-    const int uch = s.dck > 0 ? ((NB * L.fb_floats) / s.dck) & ~3 : 0;      // rows of C^K the transform buffers hold at a time
+    // rows of C^K staged at a time: the transform buffers and, behind them, the kept-dim score and probability
+    // buffers (one contiguous area, all idle until the first batch)
+    const int uch = s.dck > 0 ? (((L.twf_off - L.fbuf_off) >> 2) / s.dck) & ~3 : 0;
     auto start_coef_rows = [&]() {
         if (tid >= kConsumers) return;
         if (s.dck > 0) {
