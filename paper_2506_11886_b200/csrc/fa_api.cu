@@ -476,7 +476,8 @@ static fa_status decode_step_impl(const fa_layout* layout, fa_cache* cache, cons
         coop_fits = (cudaGetDevice(&dev) == cudaSuccess &&
                      cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, dev) == cudaSuccess && coop) ? 1 : 0;
     }
-    if (!coop_fits) {
+    // the light append kernel must not run unless the decode kernel that finishes its update can follow
+    if (!coop_fits || !decode_fft_launchable(s, p)) {
         if (q_host_view) return FA_ERR_UNSUPPORTED;
         st = fa_append(layout, cache, k_new, v_new, stream);
         if (st != FA_OK) return st;

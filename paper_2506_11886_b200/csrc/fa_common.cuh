@@ -115,6 +115,7 @@ cudaError_t launch_decode_fft(const Dims&, const CacheDev&, int dtype, const Dec
                               cudaStream_t);
 size_t decode_fft_smem_bytes(const Dims&, int log2S, int gh, int nb, int occ = 1);
 bool decode_fft_fused_fits(const Dims&, int log2S, int gh, int nb, int n_part, int occ = 1);
+bool decode_fft_launchable(const Dims&, const DecodePlan&);
 cudaError_t launch_decode_epilogue(const Dims&, const CacheDev&, int dtype, const DecodePlan&, void* out, char* ws,
                                    cudaStream_t);
 

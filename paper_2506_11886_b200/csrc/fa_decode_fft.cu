@@ -1581,7 +1581,49 @@ cudaError_t launch_fft_ls(const Dims& s, const CacheDev& c, const DecodePlan& p,
     }
 }
 
+// Resident CTAs of this kernel instance on the whole device for the plan's shared memory (cached per instance).
+template <int GH, int LS, int OCC>
+int resident_ctas_t(const Dims& s, const DecodePlan& p) {
+    static size_t cached_smem = 0;
+    static int cached = -1;
+    const size_t smem = (size_t)fft_smem_layout(LS, s.k, GH, p.nb, s.d, OCC).total;
+    if (cached >= 0 && cached_smem == smem) return cached;
+    if (ensure_dynamic_smem(decode_fft_kernel<GH, LS, OCC>, smem) != cudaSuccess) { cudaGetLastError(); return 0; }
+    int per_sm = 0, dev = 0, sms = 0;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, decode_fft_kernel<GH, LS, OCC>, kThreads, smem) != cudaSuccess ||
+        cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) {
+        cudaGetLastError();
+        return 0;
+    }
+    cached_smem = smem;
+    cached = per_sm * sms;
+    return cached;
+}
+template <int GH>
+int resident_ctas_ls(const Dims& s, const DecodePlan& p) {
+    switch (p.fft_log2) {
+        case 5: return p.occ == 2 ? resident_ctas_t<GH, 5, 2>(s, p) : resident_ctas_t<GH, 5, 1>(s, p);
+        case 6: return p.occ == 2 ? resident_ctas_t<GH, 6, 2>(s, p) : resident_ctas_t<GH, 6, 1>(s, p);
+        case 7: return p.occ == 2 ? resident_ctas_t<GH, 7, 2>(s, p) : resident_ctas_t<GH, 7, 1>(s, p);
+        case 8: return p.occ == 2 ? resident_ctas_t<GH, 8, 2>(s, p) : resident_ctas_t<GH, 8, 1>(s, p);
+        case 9: return resident_ctas_t<GH, 9, 1>(s, p);
+        case 10: return resident_ctas_t<GH, 10, 1>(s, p);
+        default: return 0;
+    }
+}
+
 }  // namespace
+
+// True if the fused kernel of this plan can be launched as planned: a part that waits for nobody runs in
+// waves; parts that wait for one another must all be resident at once (what a cooperative launch checks),
+// which depends on the registers and shared memory of the compiled instance, so the runtime is asked.
+bool decode_fft_launchable(const Dims& s, const DecodePlan& p) {
+    if (!p.fused) return true;
+    if (p.n_part <= 1) return true;
+    const long long grid = (long long)p.n_part * s.Hkv * p.n_pass * s.B;
+    const int resident = p.gh == 4 ? resident_ctas_ls<4>(s, p) : resident_ctas_ls<2>(s, p);
+    return grid <= resident;
+}
 
 size_t decode_fft_smem_bytes(const Dims& s, int log2S, int gh, int nb, int occ) {
     return (size_t)fft_smem_layout(log2S, s.k, gh, nb, s.d, occ).total;
