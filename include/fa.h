@@ -17,9 +17,13 @@
  *
  * Conventions for every call
  *   - All buffers are caller-owned DEVICE memory on the current device unless
- *     a parameter says "host".  The library allocates nothing, keeps no
- *     state on the device besides the caller's buffers and runs every kernel on the stream passed in
- *     (a cudaStream_t handed over as void*; NULL is the default stream).
+ *     a parameter says "host".  The library allocates nothing and runs every
+ *     kernel on the stream passed in (a cudaStream_t handed over as void*;
+ *     NULL is the default stream).  Its only state on the device besides the
+ *     caller's buffers is the fixed scratch array of fa_decode_attention_static.
+ *   - Host threads may call concurrently (the few host-side caches are locked);
+ *     calls that share a cache, a workspace or the static scratch must be
+ *     ordered by the caller (same stream, or events).
  *   - Calls are asynchronous.  Argument errors are found on the host before
  *     anything is launched and returned as fa_status.  Conditions only the
  *     device can see (middle segment full) are written to cache->status and
@@ -188,6 +192,19 @@ fa_status fa_decode_attention(const fa_layout* layout, const fa_cache* cache, co
 fa_status fa_decode_step(const fa_layout* layout, fa_cache* cache, const void* q, const void* k_new,
                          const void* v_new, void* out, void* ws, size_t ws_bytes, void* stream);
 
+/* One decoded token across n_layers layers (Eq.5 then Eq.6 per layer): layer i runs
+ * fa_decode_step(&layouts[i], &caches[i], q[i], k_new[i], v_new[i], out[i], ws, ...) in order on
+ * `stream`, with the same result and cache contents, bit for bit, as n_layers single calls.  layouts
+ * and caches are HOST arrays of n_layers entries; q, k_new, v_new, out are HOST arrays of n_layers
+ * DEVICE pointers ([B][H_q][d] / [B][H_kv][d] of that layer).  One workspace serves all layers (the
+ * calls are ordered by the stream): ws_bytes must cover the largest fa_workspace_bytes of the layouts.
+ * All layers are checked on the host before the first launch; after that the call only enqueues
+ * kernels, so a whole token step can be captured in one CUDA graph (after one eager call).  Stops at,
+ * and returns, the first error. */
+fa_status fa_decode_step_layers(int32_t n_layers, const fa_layout* layouts, fa_cache* caches,
+                                const void* const* q, const void* const* k_new, const void* const* v_new,
+                                void* const* out, void* ws, size_t ws_bytes, void* stream);
+
 /* One decode step with HOST inputs and outputs (Eq.5 then Eq.6): copies q [B][H_q][d] and
  * k_new, v_new [B][H_kv][d] from host memory (pinned for the copies to be asynchronous) into
  * `staging`, runs fa_decode_step, and copies the result to out_host
@@ -234,9 +251,10 @@ fa_status fa_select_dims(const fa_layout* layout, const void* K, const void* V, 
  *     before anything runs; use fa_decode_attention with your own workspace for those.
  *   - The first call on each device looks the array's device address up (with that device
  *     current); make that first call before any stream capture.
- *   - All calls on one GPU share the one array.  It keeps whatever the previous call left; the
- *     call clears the few counters it needs itself.  Two calls that overlap on the GPU (two
- *     streams, two threads) race on it: serialise them. */
+ *   - All calls on one GPU share the one array.  It keeps whatever the previous call left; each
+ *     call starts by clearing the barrier counters in its first 4 KiB (a memset on `stream`), so
+ *     a call that ended with FA_ERR_TIMEOUT does not poison the next one.  Two calls that overlap
+ *     on the GPU (two streams, two threads) race on it: serialise them. */
 fa_status fa_decode_attention_static(const fa_layout* layout, const fa_cache* cache, const void* q,
                                      void* out, void* stream);
 size_t fa_static_workspace_limit(void);

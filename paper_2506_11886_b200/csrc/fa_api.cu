@@ -2,6 +2,7 @@
 // sizes, launch plans.  Every entry point validates on the host, then launches
 // on the caller's stream; nothing here allocates device memory.
 #include <cstring>
+#include <mutex>
 
 #include "fa_common.cuh"
 
@@ -32,6 +33,43 @@ fa_status check_layout(const fa_layout* l) {
     return FA_OK;
 }
 
+// Host-side caches of this library (what the driver granted or answered so far) are small tables
+// behind this one mutex, keyed by device where the answer depends on it: two host threads may make
+// their first calls at the same time.
+static std::mutex g_host_mu;
+
+// Number of SMs of the current device (148 when no device can be asked, e.g. on a host without a GPU:
+// the sizes computed from it are then those of a B200).
+int sm_count() {
+    constexpr int kMaxDev = 64;
+    static int cached[kMaxDev] = {0};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDev) { cudaGetLastError(); return kNumSmsDefault; }
+    std::lock_guard<std::mutex> lock(g_host_mu);
+    if (cached[dev] == 0) {
+        int n = 0;
+        if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n < 1) { cudaGetLastError(); n = kNumSmsDefault; }
+        cached[dev] = n;
+    }
+    return cached[dev];
+}
+
+// True if the current device supports cooperative launches (asked once per device).
+bool cooperative_launch_supported() {
+    constexpr int kMaxDev = 64;
+    static signed char cached[kMaxDev] = {0};          // 0 unknown, 1 yes, -1 no
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDev) { cudaGetLastError(); return false; }
+    std::lock_guard<std::mutex> lock(g_host_mu);
+    if (cached[dev] == 0) {
+        int coop = 0;
+        const bool ok = cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, dev) == cudaSuccess && coop;
+        if (!ok) cudaGetLastError();
+        cached[dev] = ok ? 1 : -1;
+    }
+    return cached[dev] > 0;
+}
+
 // (kernel, device) -> largest dynamic shared memory size granted so far.
 cudaError_t ensure_dynamic_smem_impl(const void* kernel, size_t bytes) {
     struct Entry { const void* fn; int dev; size_t bytes; };
@@ -41,6 +79,7 @@ cudaError_t ensure_dynamic_smem_impl(const void* kernel, size_t bytes) {
     int dev = 0;
     cudaError_t err = cudaGetDevice(&dev);
     if (err != cudaSuccess) return err;
+    std::lock_guard<std::mutex> lock(g_host_mu);
     Entry* hit = nullptr;
     for (int i = 0; i < used; ++i)
         if (table[i].fn == kernel && table[i].dev == dev) { hit = &table[i]; break; }
@@ -79,6 +118,7 @@ static bool fft_ok(const fa_layout& l, int gh, int* log2S) {
 fa_status plan_decode(const fa_layout& l, DecodePlan* p) {
     Dims s = make_dims(l);
     std::memset(p, 0, sizeof(*p));
+    const int kNumSms = sm_count();
     int log2S = 0;
     const int gh_fft = s.G >= 3 ? 4 : 2;
     const bool can_fft = fft_ok(l, gh_fft, &log2S);
@@ -189,7 +229,7 @@ fa_status plan_decode(const fa_layout& l, DecodePlan* p) {
     p->rows_pro = 32;
     p->n_slice = s.dcv > 0 ? (s.M + 63) / 64 : 1;
     size_t off = 0;
-    p->off_bar = off; off = align_up(off + sizeof(int32_t) * 4 * (size_t)kNumSms, 256);     // same place for every layout
+    p->off_bar = off; off = align_up(off + sizeof(int32_t) * 4 * (size_t)kBarSlots, 256);   // same place and size for every layout
     p->off_u = off;   off = align_up(off + sizeof(float) * (size_t)s.B * s.Hq * s.M, 256);
     p->off_ml = off;  off = align_up(off + sizeof(float) * (size_t)s.B * s.Hq * p->n_part * 2, 256);
     p->off_o = off;   off = align_up(off + sizeof(float) * (size_t)s.B * s.Hq * p->n_part * s.d, 256);
@@ -470,14 +510,8 @@ static fa_status decode_step_impl(const fa_layout* layout, fa_cache* cache, cons
     cudaStream_t cs = static_cast<cudaStream_t>(stream);
     char* w = static_cast<char*>(ws);
     // (a cooperative launch that does not fit the device fails before anything runs; find out first)
-    static int coop_fits = -1;
-    if (coop_fits < 0) {
-        int dev = 0, coop = 0;
-        coop_fits = (cudaGetDevice(&dev) == cudaSuccess &&
-                     cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, dev) == cudaSuccess && coop) ? 1 : 0;
-    }
     // the light append kernel must not run unless the decode kernel that finishes its update can follow
-    if (!coop_fits || !decode_fft_launchable(s, p)) {
+    if (!cooperative_launch_supported() || !decode_fft_launchable(s, p)) {
         if (q_host_view) return FA_ERR_UNSUPPORTED;
         st = fa_append(layout, cache, k_new, v_new, stream);
         if (st != FA_OK) return st;
@@ -495,6 +529,30 @@ extern "C" {
 fa_status fa_decode_step(const fa_layout* layout, fa_cache* cache, const void* q, const void* k_new, const void* v_new,
                          void* out, void* ws, size_t ws_bytes, void* stream) {
     return decode_step_impl(layout, cache, q, k_new, v_new, out, ws, ws_bytes, stream, nullptr, 0);
+}
+
+fa_status fa_decode_step_layers(int32_t n_layers, const fa_layout* layouts, fa_cache* caches, const void* const* q,
+                                const void* const* k_new, const void* const* v_new, void* const* out, void* ws,
+                                size_t ws_bytes, void* stream) {
+    if (n_layers < 0 || (n_layers > 0 && (!layouts || !caches || !q || !k_new || !v_new || !out))) return FA_ERR_INVALID_ARG;
+    // every layer's arguments are checked before anything is enqueued: a bad layer leaves all caches untouched
+    for (int i = 0; i < n_layers; ++i) {
+        fa_status st = check_layout(&layouts[i]);
+        if (st != FA_OK) return st;
+        st = check_cache(&layouts[i], &caches[i]);
+        if (st != FA_OK) return st;
+        const void* ptrs[] = {q[i], k_new[i], v_new[i], out[i]};
+        for (const void* p : ptrs) if (!p || !aligned16(p)) return FA_ERR_INVALID_ARG;
+        DecodePlan p;
+        st = plan_decode(layouts[i], &p);
+        if (st != FA_OK) return st;
+        if (!ws || !aligned16(ws) || ws_bytes < p.total) return FA_ERR_WORKSPACE;
+    }
+    for (int i = 0; i < n_layers; ++i) {
+        const fa_status st = decode_step_impl(&layouts[i], &caches[i], q[i], k_new[i], v_new[i], out[i], ws, ws_bytes, stream, nullptr, 0);
+        if (st != FA_OK) return st;
+    }
+    return FA_OK;
 }
 
 size_t fa_step_staging_bytes(const fa_layout* layout) {

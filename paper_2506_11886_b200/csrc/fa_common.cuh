@@ -13,7 +13,8 @@ namespace fa {
 
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kNegBig = -1.0e30f;   // "no token yet" running max (finite, so differences stay finite)
-constexpr int kNumSms = 148;
+constexpr int kNumSmsDefault = 148;     // B200; used only when no device can be asked (sm_count())
+constexpr int kBarSlots = 256;          // (b, KV head, pass) triples that can own barrier counters in the first 4 KiB of a workspace
 constexpr int kStateStride = 8;        // int32 words of cache state per batch row
 
 // Layout numbers every kernel needs, passed by value.
@@ -94,6 +95,8 @@ __host__ __device__ inline int v_mid_col(int a, int e, int nfv, int dtype) {
 }
 
 fa_status plan_decode(const fa_layout& l, DecodePlan* plan);
+int sm_count();                          // SMs of the current device, cached per device
+bool cooperative_launch_supported();     // of the current device, cached per device
 fa_status check_layout(const fa_layout* l);
 
 // Kernel launchers (defined next to their kernels).  All return the launch error, if any.

@@ -214,7 +214,7 @@ static cudaError_t launch_compress_t(const Dims& s, const CacheDev& c, const voi
     int row_tiles = (s.M + kTM - 1) / kTM;
     int chunks = (n_mid + kTJ - 1) / kTJ;
     int ctas_fixed = row_tiles * s.B * s.Hkv * 2;
-    int n_tsplit = (4 * kNumSms + ctas_fixed - 1) / ctas_fixed;
+    int n_tsplit = (4 * sm_count() + ctas_fixed - 1) / ctas_fixed;
     if (n_tsplit > chunks) n_tsplit = chunks;
     if (n_tsplit < 1) n_tsplit = 1;
     int cps = (chunks + n_tsplit - 1) / n_tsplit;

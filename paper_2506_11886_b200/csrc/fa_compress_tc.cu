@@ -335,7 +335,7 @@ cudaError_t launch_tc_t(const CUtensorMap& tmK, const CUtensorMap& tmV, const Di
     const int row_tiles = (s.M + kBM - 1) / kBM;
     const int nkb = (n_mid + kBK - 1) / kBK;
     const int fixed = row_tiles * (s.Hkv / HP) * s.B;
-    int n_tsplit = kNumSms / fixed;                          // one wave: one CTA per SM at most
+    int n_tsplit = sm_count() / fixed;                          // one wave: one CTA per SM at most
     if (n_tsplit > nkb) n_tsplit = nkb;
     if (n_tsplit < 1) n_tsplit = 1;
     compress_tc_kernel<D, HP><<<dim3(row_tiles, s.Hkv / HP, s.B * n_tsplit), kThreadsTc, smem, stream>>>(tmK, tmV, s, c, L, n_tsplit);

@@ -35,6 +35,8 @@
 // "Slot" below is the position of a head inside a point / an mma column: slot s holds head
 // hperm(s) = {0, 2, 1, 3}[s] (GH = 4) so that the packed real parts are slots 0, 1 and the
 // packed imaginary parts slots 2, 3.
+#include <mutex>
+
 #include "fa_decode_ws.cuh"
 #include "fa_tmap.cuh"
 
@@ -1516,6 +1518,21 @@ __global__ void __launch_bounds__(kThreads, OCC) decode_fft_kernel(const __grid_
     if (tid == 0 && np > 1) { bar[0] = 0; bar[1] = 0; bar[2] = 0; }   // the counters are zero again for the next call
 }
 
+// Whether the driver takes the cooperative and the programmatic-serialization launch attributes
+// together, per device: -1 not probed, 0 no, 1 yes.  set = -2 reads, anything else records.
+static int coop_pdl_state(int set) {
+    constexpr int kMaxDev = 64;
+    static signed char state[kMaxDev];
+    static bool init = false;
+    static std::mutex mu;
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDev) { cudaGetLastError(); return 0; }
+    std::lock_guard<std::mutex> lock(mu);
+    if (!init) { for (int i = 0; i < kMaxDev; ++i) state[i] = -1; init = true; }
+    if (set != -2) state[dev] = (signed char)set;
+    return state[dev];
+}
+
 template <int GH, int LS, int OCC>
 cudaError_t launch_fft_t(const Dims& s, const CacheDev& c, const DecodePlan& p, const void* q, void* out, char* ws, int step,
                          cudaStream_t st) {
@@ -1537,7 +1554,6 @@ cudaError_t launch_fft_t(const Dims& s, const CacheDev& c, const DecodePlan& p, 
     // still runs and waits (griddepcontrol.wait) where it first reads what the predecessor wrote.  The
     // fused kernel is also a cooperative launch (its CTAs wait for one another); whether the driver
     // takes both attributes together is found out on the first launch outside a stream capture.
-    static int coop_pdl_ok = -1;
     cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
@@ -1547,16 +1563,17 @@ cudaError_t launch_fft_t(const Dims& s, const CacheDev& c, const DecodePlan& p, 
     cfg.numAttrs = 1;
     if (p.fused && p.n_part > 1) {                       // a head served by one CTA waits for nobody: plain launch, any grid
         cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
-        if (coop_pdl_ok < 0 && (cudaStreamIsCapturing(st, &cap) != cudaSuccess || cap != cudaStreamCaptureStatusNone)) {
+        const int known = coop_pdl_state(-2);
+        if (known < 0 && (cudaStreamIsCapturing(st, &cap) != cudaSuccess || cap != cudaStreamCaptureStatusNone)) {
             cfg.attrs = attr + 1;                                          // not probed yet: stay on the plain cooperative launch
-        } else if (coop_pdl_ok != 0) {
+        } else if (known != 0) {
             cfg.numAttrs = 2;
             cudaError_t err2 = cudaLaunchKernelEx(&cfg, decode_fft_kernel<GH, LS, OCC>, tki, tvi, tkl, tvl, s, c, p,
                                                   static_cast<const bf16*>(q), static_cast<bf16*>(out), ws, step);
-            if (err2 == cudaSuccess) { coop_pdl_ok = 1; return err2; }
-            if (coop_pdl_ok == 1) return err2;
+            if (err2 == cudaSuccess) { coop_pdl_state(1); return err2; }
+            if (known == 1) return err2;
             cudaGetLastError();
-            coop_pdl_ok = 0;
+            coop_pdl_state(0);
             cfg.attrs = attr + 1;
             cfg.numAttrs = 1;
         } else {
@@ -1584,20 +1601,26 @@ cudaError_t launch_fft_ls(const Dims& s, const CacheDev& c, const DecodePlan& p,
 // Resident CTAs of this kernel instance on the whole device for the plan's shared memory (cached per instance).
 template <int GH, int LS, int OCC>
 int resident_ctas_t(const Dims& s, const DecodePlan& p) {
-    static size_t cached_smem = 0;
-    static int cached = -1;
+    // answers cached per (device, shared memory size) of this instance
+    struct Entry { int dev; size_t smem; int ctas; };
+    static Entry table[16];
+    static int used = 0;
+    static std::mutex mu;
     const size_t smem = (size_t)fft_smem_layout(LS, s.k, GH, p.nb, s.d, OCC).total;
-    if (cached >= 0 && cached_smem == smem) return cached;
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) { cudaGetLastError(); return 0; }
+    std::lock_guard<std::mutex> lock(mu);
+    for (int i = 0; i < used; ++i)
+        if (table[i].dev == dev && table[i].smem == smem) return table[i].ctas;
     if (ensure_dynamic_smem(decode_fft_kernel<GH, LS, OCC>, smem) != cudaSuccess) { cudaGetLastError(); return 0; }
-    int per_sm = 0, dev = 0, sms = 0;
-    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, decode_fft_kernel<GH, LS, OCC>, kThreads, smem) != cudaSuccess ||
-        cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) {
+    int per_sm = 0;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, decode_fft_kernel<GH, LS, OCC>, kThreads, smem) != cudaSuccess) {
         cudaGetLastError();
         return 0;
     }
-    cached_smem = smem;
-    cached = per_sm * sms;
-    return cached;
+    const int ctas = per_sm * sm_count();
+    if (used < 16) table[used++] = Entry{dev, smem, ctas};
+    return ctas;
 }
 template <int GH>
 int resident_ctas_ls(const Dims& s, const DecodePlan& p) {

@@ -57,8 +57,12 @@ fa_status fa_decode_attention_static(const fa_layout* layout, const fa_cache* ca
     if (need > fa::kStaticWsBytes) return FA_ERR_WORKSPACE; // this layout needs more scratch than the fixed array has
     char* ws = nullptr;
     if (fa::static_ws_of_current_device(&ws) != cudaSuccess) return FA_ERR_CUDA;
-    // Nothing in the scratch has to start at zero across calls: the first kernel of the call
-    // clears the tickets it uses, every other word is written before it is read.
+    // The barrier counters at the head of the scratch (its first 4 KiB) must be zero when the decode
+    // kernels start.  A call that ends normally leaves them zero, a call that gave up on a bounded wait
+    // (FA_ERR_TIMEOUT) does not, and the caller has no pointer to this array to clear it with
+    // fa_workspace_init: so every call clears them itself, in stream order, in front of its kernels.
+    // A memset allocates nothing.  Everything else in the array is written before it is read.
+    if (cudaMemsetAsync(ws, 0, 4096, static_cast<cudaStream_t>(stream)) != cudaSuccess) return FA_ERR_CUDA;
     return fa_decode_attention(layout, cache, q, out, ws, fa::kStaticWsBytes, stream);
 }
 

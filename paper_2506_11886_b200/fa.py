@@ -73,6 +73,8 @@ def lib() -> C.CDLL:
         L.fa_poll_status.argtypes = [cp, vp]
         L.fa_decode_step_host.argtypes = [lp, cp, vp, vp, vp, vp, vp, vp, sz, vp]
         L.fa_decode_step.argtypes = [lp, cp, vp, vp, vp, vp, vp, sz, vp]
+        L.fa_decode_step_layers.argtypes = [i32, lp, cp, C.POINTER(vp), C.POINTER(vp), C.POINTER(vp), C.POINTER(vp), vp, sz, vp]
+        L.fa_decode_step_layers.restype = C.c_int
         L.fa_select_workspace_bytes.argtypes = [lp, C.POINTER(sz)]
         L.fa_select_dims.argtypes = [lp, vp, vp, i64, i64, i64, i32, vp, vp, vp, vp, vp, vp, sz, vp]
         L.fa_step_staging_bytes.argtypes = [lp]
@@ -284,6 +286,30 @@ def fa_decode_step(layout: Layout, cache: Cache, q: torch.Tensor, k_new: torch.T
         assert t.is_cuda and t.is_contiguous() and t.dtype == layout.torch_dtype
     _check(lib().fa_decode_step(C.byref(layout.c()), C.byref(cache.c()), _ptr(q), _ptr(k_new), _ptr(v_new), _ptr(out),
                                 _ptr(ws), ws.numel(), _stream(stream)), "fa_decode_step")
+
+
+class LayerStep:
+    """Marshalled arguments of ``fa_decode_step_layers`` for a fixed set of layers and tensors (built
+    once, so that the per-token call is one C call)."""
+
+    def __init__(self, layouts, caches, qs, k_news, v_news, outs):
+        n = len(layouts)
+        assert n == len(caches) == len(qs) == len(k_news) == len(v_news) == len(outs)
+        for lay, q, k, v, o in zip(layouts, qs, k_news, v_news, outs):
+            for t in (q, k, v, o):
+                assert t.is_cuda and t.is_contiguous() and t.dtype == lay.torch_dtype
+        self.n = n
+        self.layouts = (fa_layout * n)(*[l.c() for l in layouts])
+        self.caches = (fa_cache * n)(*[c.c() for c in caches])
+        arr = lambda ts: (C.c_void_p * n)(*[t.data_ptr() for t in ts])
+        self.q, self.k, self.v, self.o = arr(qs), arr(k_news), arr(v_news), arr(outs)
+        self._keep = (list(qs), list(k_news), list(v_news), list(outs), list(caches))
+
+
+def fa_decode_step_layers(args: LayerStep, ws: torch.Tensor, stream=None) -> None:
+    """One decoded token across all layers of ``args`` (fa_decode_step per layer, in order)."""
+    _check(lib().fa_decode_step_layers(args.n, args.layouts, args.caches, args.q, args.k, args.v, args.o, _ptr(ws),
+                                       ws.numel(), _stream(stream)), "fa_decode_step_layers")
 
 
 def fa_decode_step_host(layout: Layout, cache: Cache, q_host: torch.Tensor, k_new_host, v_new_host,

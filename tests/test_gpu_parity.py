@@ -435,3 +435,120 @@ def test_workspace_counters_must_start_at_zero_and_init_restores_them():
     assert not dirty[:4096].any() and bool((dirty[4096:] == 0x5A).all())
     pair.ws = dirty
     pair.check_decode(synth.queries(shape, seed=19, step=1))
+
+
+def test_bounded_wait_runs_out_reports_timeout_and_workspace_init_recovers():
+    """Failure path of the cooperative decode kernel, without faulting or hanging anything: one barrier
+    counter of a caller workspace is preset so that the arrivals of the head's parts can never reach the
+    number the waiting parts poll for.  Every poll loop is bounded (2^22 polls of ~0.1 us with back-off,
+    well under a second per CTA, all CTAs polling at the same time), so the kernel gives up, records
+    FA_ERR_TIMEOUT in the cache's status word and returns; the output of that call is undefined.
+    fa_workspace_init then restores the workspace and the next call matches the oracle."""
+    import time
+    shape = SMALL_BF16.with_(B=1, Hq=8, Hkv=2, L=1800, T=2048, M=256, n_full_k=32, n_full_v=32)
+    pair, _ = make_pair(shape, seed=31, algo=fa.FA_DECODE_FFT, P=16)
+    assert fa.fa_launch_count(pair.layout, 2) == 1            # the fused, cooperative form: its parts wait for one another
+    q = synth.queries(shape, seed=31)
+    pair.check_decode(q)                                      # a good call first
+    counters = pair.ws[:4096].view(torch.int32)
+    assert not counters.any()                                 # a good call leaves every counter at zero
+    counters[0] = -(1 << 20)                                  # first barrier of (row 0, KV head 0): arrivals cannot reach n
+    out = torch.zeros_like(q, device="cuda")
+    t0 = time.perf_counter()
+    fa.fa_decode_attention(pair.layout, pair.gpu, q.cuda(), out, pair.ws)
+    st = fa.fa_poll_status(pair.gpu)                          # synchronises
+    waited = time.perf_counter() - t0
+    assert st == fa.FA_ERR_TIMEOUT
+    assert waited < 20.0, waited
+    assert fa.fa_poll_status(pair.gpu) == fa.FA_OK            # the status word is cleared by the poll
+    fa.fa_workspace_init(pair.ws)
+    pair.check_decode(synth.queries(shape, seed=31, step=1))
+    pair.check_decode(q)
+    assert not pair.ws[:4096].any()
+
+
+def test_full_row_in_a_batch_is_refused_alone():
+    """Batch of two rows, one whose middle is full and one with room: the push changes nothing in the
+    full row (FA_ERR_CAPACITY in the status word) and goes through in the other (oracle: one cache per
+    row, since a row is a cache of its own)."""
+    import dataclasses
+    from oracle import fa_oracle as fo
+    from tests.parity_util import oracle_cfg
+    shape = SMALL_BF16.with_(B=2, Hq=4, Hkv=1, L=0, L_init=2, L_local=4, T=64, M=16, n_full_k=16, n_full_v=8)
+    layout = layout_of(shape, max_mid=8, P=2, algo=fa.FA_DECODE_AUTO)
+    stream = synth.KVStream(shape, seed=32)
+    K, V = stream.tokens(0, 20)
+    lengths = [14, 9]                                         # row 0: 2 + 4 + 8 = full; row 1: three middle tokens
+    gpu = fa.Cache(layout, stream.idx_full_k, stream.idx_full_v)
+    ws = fa.new_workspace(layout)
+    fa.fa_compress_ragged(layout, gpu, K.cuda(), V.cuda(), lengths, ws)
+    refs = []
+    for b in range(2):
+        r = fo.OracleCache(dataclasses.replace(oracle_cfg(layout), B=1), stream.idx_full_k.numpy(), stream.idx_full_v.numpy())
+        r.compress(to64(K[b:b + 1, :lengths[b]]), to64(V[b:b + 1, :lengths[b]]))
+        refs.append(r)
+    for step, use_step in enumerate((False, True)):
+        k_new, v_new = K[:, 15 + step].contiguous(), V[:, 15 + step].contiguous()
+        q = synth.queries(shape, seed=32, step=step)
+        out = torch.full_like(q, float("nan"), device="cuda")
+        if use_step:
+            fa.fa_decode_step(layout, gpu, q.cuda(), k_new.cuda(), v_new.cuda(), out, ws)
+        else:
+            fa.fa_append(layout, gpu, k_new.cuda(), v_new.cuda())
+            fa.fa_decode_attention(layout, gpu, q.cuda(), out, ws)
+        assert fa.fa_poll_status(gpu) == fa.FA_ERR_CAPACITY   # from row 0
+        refs[1].append(to64(k_new[1:2]), to64(v_new[1:2]))    # row 0's oracle cache is left alone: the push was refused
+        st = gpu.state.cpu().numpy()
+        for b in range(2):
+            assert (st[b, 0], st[b, 1], st[b, 2]) == (refs[b].n_init[0], refs[b].n_local[0], refs[b].n_mid[0]), (step, b)
+            want = refs[b].decode(to64(q[b:b + 1]))
+            assert np.abs(to64(out[b:b + 1]) - want).max() <= 2e-2, (step, b)
+            for name in ("coef_k", "coef_v"):
+                rc = getattr(refs[b], name)[0]
+                assert np.abs(to64(getattr(gpu, name)[b]) - rc).max() <= 1e-3 * max(np.abs(rc).max(), 1e-30), (step, b, name)
+
+
+def test_multi_layer_step_equals_single_calls_bit_for_bit():
+    """fa_decode_step_layers over layers with different schemas (kept dims per layer as in the
+    inverted-pyramid schema: more compressed dims in early layers) against one fa_decode_step per
+    layer on twin caches: outputs and every cache buffer identical bit for bit, and the first layer
+    against the oracle."""
+    base = SMALL_BF16.with_(B=2, Hq=8, Hkv=2, L=900, T=1024, M=128, decode_steps=4)
+    schemas = [(16, 8), (32, 32), (32, 32), (64, 40)]          # (n_full_k, n_full_v) per layer
+    n_layers, steps = len(schemas), 4
+    layouts, twins, streams, pair0 = [], [], [], None
+    for i, (nfk, nfv) in enumerate(schemas):
+        shape = base.with_(n_full_k=nfk, n_full_v=nfv)
+        layout = layout_of(shape, max_mid=1024, P=8, algo=fa.FA_DECODE_AUTO)
+        stream = synth.KVStream(shape, seed=40 + i, layer=i)
+        K, V = stream.tokens(0, shape.L)
+        pair = Pair(layout, stream.idx_full_k, stream.idx_full_v)
+        pair.compress(K, V)
+        twin = fa.Cache(layout, stream.idx_full_k, stream.idx_full_v)
+        fa.fa_compress(layout, twin, K.cuda(), V.cuda(), pair.ws)
+        layouts.append(layout); twins.append((pair.gpu, twin)); streams.append((shape, stream))
+        if i == 0:
+            pair0 = pair
+    ws = fa.new_workspace(max(layouts, key=fa.fa_workspace_bytes))
+    qs = [torch.empty((2, 8, 128), dtype=torch.bfloat16, device="cuda") for _ in range(n_layers)]
+    ks = [torch.empty((2, 2, 128), dtype=torch.bfloat16, device="cuda") for _ in range(n_layers)]
+    vs = [torch.empty_like(k) for k in ks]
+    outs_a = [torch.full_like(q, float("nan")) for q in qs]
+    outs_b = [torch.full_like(q, float("nan")) for q in qs]
+    args = fa.LayerStep(layouts, [a for a, _ in twins], qs, ks, vs, outs_a)
+    for t in range(steps):
+        for i, (shape, stream) in enumerate(streams):
+            k_new, v_new = stream.tokens(shape.L + t, shape.L + t + 1)
+            qs[i].copy_(synth.queries(shape, seed=40 + i, step=t, layer=i)); ks[i].copy_(k_new[:, 0]); vs[i].copy_(v_new[:, 0])
+        fa.fa_decode_step_layers(args, ws)
+        for i in range(n_layers):
+            fa.fa_decode_step(layouts[i], twins[i][1], qs[i], ks[i], vs[i], outs_b[i], ws)
+        torch.cuda.synchronize()
+        for i in range(n_layers):
+            assert (outs_a[i].float() - outs_b[i].float()).abs().max().item() <= 2.0 ** -8, (t, i)
+        pair0.ref.append(to64(ks[0]), to64(vs[0]))
+        assert np.abs(to64(outs_a[0]) - pair0.ref.decode(to64(qs[0]))).max() <= 2e-2
+    for i, (a, b) in enumerate(twins):
+        for name in ("k_init", "v_init", "k_local", "v_local", "k_mid", "v_mid", "coef_k", "coef_v", "state"):
+            assert torch.equal(getattr(a, name), getattr(b, name)), (i, name)
+    pair0.check_state()

@@ -59,7 +59,10 @@ def test_random_layouts(seed, many_heads):
         base = OUT_ABS_F32 if shape.dtype == "f32" else OUT_ABS_BF16
 
         def close(got, want):
-            err, bound = np.abs(got - want).max(), base * max(1.0, float(np.abs(want).max()))
+            # the stated absolute tolerance with the orthogonal weights; with the literal 1/k scale the
+            # compressed part of the outputs is multiplied by T / 2k, so the bound follows the output magnitude
+            bound = base * max(1.0, float(np.abs(want).max())) if norm == fa.FA_NORM_PAPER else base
+            err = np.abs(got - want).max()
             assert err <= bound, f"output error {err:.3e} > {bound:.3e}"
 
         try:
