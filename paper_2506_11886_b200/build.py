@@ -41,7 +41,7 @@ def build_library(force: bool = False, verbose: bool = False) -> str:
         o = os.path.join(CSRC, src[:-3] + ".o")
         objs.append(o)
         if force or not os.path.exists(o) or os.path.getmtime(o) < max(os.path.getmtime(s), hdr_time):
-            cmd = [nvcc, *NVCC_FLAGS, "-c", s, "-o", o]
+            cmd = [nvcc, *NVCC_FLAGS, *os.environ.get("FA_NVCC_EXTRA", "").split(), "-c", s, "-o", o]
             if verbose:
                 cmd.insert(1, "-Xptxas")
                 cmd.insert(2, "-v")

@@ -98,7 +98,7 @@ static int ilog2_exact(int v) {
 }
 
 // True if the residue-class transform kernel can serve this layout: power-of-two period split
-// into P classes of S = T / P slots, S a power of two in [32, 1024]; at most 64 kept dims per
+// into P classes of S = T / P slots, S a power of two in [32, 2048]; at most 64 kept dims per
 // side, head_dim <= 128, and the kernel's shared memory must fit.
 static bool fft_ok(const fa_layout& l, int gh, int* log2S) {
     if (l.kv_dtype != FA_BF16) return false;                                   // tensor-core dot products: bf16 caches
@@ -110,9 +110,7 @@ static bool fft_ok(const fa_layout& l, int gh, int* log2S) {
     if (l.n_coef / 2 > S) return false;                                        // every frequency needs its own bin
     if (l.n_full_k > 64 || l.n_full_v > 64 || l.head_dim > 128) return false;
     if ((long long)l.l_init + l.l_local > (1 << 22)) return false;                // 32-bit split arithmetic in the kernel
-    if (l.n_coef % 4 != 0) return false;                                       // coefficient rows are dealt out in fours
-    int nt, tw, nsg;
-    if (!decode_teams_shape(make_dims(l), ls, gh, 1, &nt, &tw, &nsg, nullptr)) return false;
+    if (decode_fft_smem_bytes(make_dims(l), ls, gh, 1) > 227 * 1024) return false;
     *log2S = ls;
     return true;
 }
@@ -132,62 +130,86 @@ fa_status plan_decode(const fa_layout& l, DecodePlan* p) {
         p->gh = gh_fft;
         p->n_pass = (s.G + p->gh - 1) / p->gh;
         const int jobs = s.B * s.Hkv * p->n_pass;
-        // The kernel runs 16 warps in one CTA per SM, or 8 warps in each of two CTAs per SM.  When every
-        // (b, KV head, pass) can have a CTA resident at once the call is one fused kernel: it forms u itself
-        // and merges its own partial results, the CTAs of a head waiting for one another (cooperative
-        // launch).  A head gets floor(slots / heads) CTAs; the window tokens either share the class CTAs or
-        // get CTAs of their own, whichever keeps the largest CTA's bytes smallest.  With more heads than
-        // slots a head gets one CTA, which waits for nobody: a plain launch that runs in waves.
+        // One CTA per SM (a ring of stages and a whole batch of classes per CTA).  When every
+        // (b, KV head, pass) can have a CTA resident at once, the kernel is fused: it forms u itself
+        // and merges its own partial results, its CTAs waiting for one another (cooperative
+        // launch).  A head gets floor(SMs / heads) CTAs; the window tokens either share the class
+        // CTAs or get CTAs of their own, whichever keeps the largest CTA's bytes smallest.  With more
+        // heads than SMs a head gets one CTA, which waits for nobody: a plain launch that runs in waves.
         const long long win_bytes = 2LL * (s.l_init + s.l_local) * s.d;
         const long long class_bytes = (long long)(s.T / s.P) * (s.nfk + s.nfv);
+        // classes transformed together: enough butterflies for all consumer threads, within shared memory
+        auto pick_nb = [&](int n_split, int occ = 1) {
+            const int S = s.T / s.P;
+            int nb = 2048 / S;
+            if (nb < 1) nb = 1;
+            if (nb > 8) nb = 8;
+            const int per_cta = (s.P + n_split - 1) / n_split;
+            if (nb > per_cta) nb = per_cta;
+            const size_t limit = occ == 2 ? 113 * 1024 : 227 * 1024;      // two CTAs share the SM's 228 KB, 1 KB reserved each
+            while (nb > 1 && decode_fft_smem_bytes(s, log2S, p->gh, nb, occ) > limit) --nb;
+            return nb;
+        };
         p->fused = 0;
         p->n_wsplit = 0;
         p->occ = 1;
-        int nt1 = 0, tw1 = 0, nsg1 = 0;
-        decode_teams_shape(s, log2S, p->gh, 1, &nt1, &tw1, &nsg1, nullptr);
-        // Two CTAs per SM only where it buys whole waves: more heads than SMs, at most two per SM.
-        int nt2 = 0, tw2 = 0, nsg2 = 0;
-        const bool two = jobs > kNumSms && decode_teams_shape(s, log2S, p->gh, 2, &nt2, &tw2, &nsg2, nullptr);
-        if (l.decode_algo != FA_DECODE_FFT_SPLIT) {
-            const int occ = two ? 2 : 1;
+        // Short transforms leave room for two CTAs on an SM (a shorter ring, a register cap): one CTA's
+        // dependent phases hide behind the other's, and a head gets twice the CTAs (or, with more heads
+        // than SMs, the waves are twice as wide).  Tried first; one CTA per SM otherwise.
+        for (int occ = log2S <= 8 ? 2 : 1; occ >= 1 && !p->fused && l.decode_algo != FA_DECODE_FFT_SPLIT; --occ) {
+            const size_t smem_limit = occ == 2 ? 113 * 1024 : 227 * 1024;
             const int slots = kNumSms * occ;
-            int per_job = jobs < slots ? slots / jobs : 1;
-            if (per_job > decode_teams_max_parts()) per_job = decode_teams_max_parts();
-            int best_ns = 0, best_nw = 0;
-            long long best_cost = -1;
-            // nw = 0: the window tokens are spread over the class CTAs (few CTAs per head); else CTAs of their own
-            for (int nw = 0; nw <= 8 && nw < per_job; ++nw) {
-                int ns = per_job - nw;
-                if (ns > s.P) ns = s.P;
-                const long long cc = (long long)((s.P + ns - 1) / ns) * class_bytes + (nw == 0 ? (win_bytes + ns - 1) / ns : 0);
-                const long long wc = nw ? (win_bytes + nw - 1) / nw : 0;
-                const long long cost = cc > wc ? cc : wc;
-                if (best_cost < 0 || cost < best_cost) { best_cost = cost; best_ns = ns; best_nw = nw; }
-                if (win_bytes == 0) break;
+            const int per_job = jobs < slots ? slots / jobs : 1;
+            // Fewer CTAs per head than the device offers when the merge scratch of the fused kernel could
+            // not hold the partial results of that many parts (one KV head alone could have them all).
+            for (int pj = per_job; pj >= 1 && !p->fused; pj = pj > 24 ? 24 : pj - 1) {
+                int best_ns = 0, best_nw = 0;
+                long long best_cost = -1;
+                // nw = 0: the window tokens are spread over the class CTAs (few CTAs per head); else CTAs of their own
+                for (int nw = 0; nw <= 8 && nw < pj; ++nw) {
+                    int ns = pj - nw;
+                    if (ns > s.P) ns = s.P;
+                    const long long cc = (long long)((s.P + ns - 1) / ns) * class_bytes + (nw == 0 ? (win_bytes + ns - 1) / ns : 0);
+                    const long long wc = nw ? (win_bytes + nw - 1) / nw : 0;
+                    const long long cost = cc > wc ? cc : wc;
+                    if (best_cost < 0 || cost < best_cost) { best_cost = cost; best_ns = ns; best_nw = nw; }
+                    if (win_bytes == 0) break;
+                }
+                // fewest class CTAs that reach the same classes per CTA
+                const int per_cta = (s.P + best_ns - 1) / best_ns;
+                best_ns = (s.P + per_cta - 1) / per_cta;
+                const int nb = pick_nb(best_ns, occ);
+                if (occ == 2 && nb < (per_cta < 4 ? per_cta : 4)) break;                   // too few classes per transform batch: not worth it
+                if (decode_fft_smem_bytes(s, log2S, p->gh, nb, occ) <= smem_limit &&
+                    decode_fft_fused_fits(s, log2S, p->gh, nb, best_ns + best_nw, occ)) {
+                    p->fused = 1;
+                    p->n_split = best_ns;
+                    p->n_wsplit = best_nw;
+                    p->nb = nb;
+                    p->occ = occ;
+                }
             }
-            // fewest class CTAs that reach the same classes per CTA
-            const int per_cta = (s.P + best_ns - 1) / best_ns;
-            best_ns = (s.P + per_cta - 1) / per_cta;
-            p->fused = 1;
-            p->n_split = best_ns;
-            p->n_wsplit = best_nw;
-            p->occ = occ;
-            p->nt = occ == 2 ? nt2 : nt1; p->tw = occ == 2 ? tw2 : tw1; p->nsg = occ == 2 ? nsg2 : nsg1;
         }
         // Three-kernel form.  Classes are indivisible: pick the split count that minimises
         // waves * (classes per CTA + a CTA's fixed cost, about two classes' worth), smallest count on ties.
+        int best = 1;
+        long long best_cost = -1;
+        for (int n = 1; n <= s.P && n <= 64; ++n) {
+            long long waves = ((long long)jobs * n + kNumSms - 1) / kNumSms;
+            long long cost = waves * ((s.P + n - 1) / n + 2);
+            if (best_cost < 0 || cost < best_cost) { best_cost = cost; best = n; }
+        }
+        // More heads than SMs: the lone CTAs of the fused kernel run in whole waves.  AUTO keeps it unless
+        // the balanced split is ahead by the same cost model (the last wave nearly empty) by more than
+        // the margin that the three launches and the round trip of u and the partial results cost.
+        if (p->fused && jobs > kNumSms && l.decode_algo == FA_DECODE_AUTO &&
+            20LL * ((jobs + kNumSms * p->occ - 1) / (kNumSms * p->occ)) * (s.P + 2) * p->occ > 23 * best_cost)
+            p->fused = 0;
         if (!p->fused) {
-            int best = 1;
-            long long best_cost = -1;
-            for (int n = 1; n <= s.P && n <= 64; ++n) {
-                long long waves = ((long long)jobs * n + kNumSms - 1) / kNumSms;
-                long long cost = waves * ((s.P + n - 1) / n + 2);
-                if (best_cost < 0 || cost < best_cost) { best_cost = cost; best = n; }
-            }
             p->n_wsplit = 0;
             p->occ = 1;
             p->n_split = best;
-            p->nt = nt1; p->tw = tw1; p->nsg = nsg1;
+            p->nb = pick_nb(best);
         }
     } else {
         p->gh = s.G >= 4 ? 4 : (s.G >= 2 ? 2 : 1);

@@ -69,9 +69,8 @@ struct DecodePlan {
     int n_slice;       // CTAs that share the coefficient rows of one (b, KV head) in the epilogue
     int rows_pro;      // coefficient rows per prologue CTA
     int fft_log2;      // log2 of the transform length (FFT path)
-    int nt, tw;        // teams of a CTA and warps per team (FFT path): a team takes one class at a time through all phases
-    int nsg;           // stages of a warp's private ring of shared-memory pieces
-    int occ;           // CTAs per SM the main kernel is built for (FFT path: 1 with 16 warps, 2 with 8)
+    int nb;            // classes transformed together by one CTA (FFT path)
+    int occ;           // CTAs per SM the main kernel is built for (FFT path: 1, or 2 with a shorter ring)
     // workspace offsets in bytes
     size_t off_bar, off_u, off_ml, off_o, off_z, off_oc, off_om, off_cnt, off_pend, off_pendj, total;
 };
@@ -117,8 +116,8 @@ cudaError_t launch_append_lite(const Dims&, const CacheDev&, int dtype, const De
                                bool host_inputs = false);
 cudaError_t launch_decode_fft(const Dims&, const CacheDev&, int dtype, const DecodePlan&, const void* q, void* out, char* ws, bool step,
                               cudaStream_t);
-bool decode_teams_shape(const Dims&, int log2S, int gh, int occ, int* nt, int* tw, int* nsg, size_t* smem);
-int decode_teams_max_parts();
+size_t decode_fft_smem_bytes(const Dims&, int log2S, int gh, int nb, int occ = 1);
+bool decode_fft_fused_fits(const Dims&, int log2S, int gh, int nb, int n_part, int occ = 1);
 bool decode_fft_launchable(const Dims&, const DecodePlan&);
 cudaError_t launch_decode_epilogue(const Dims&, const CacheDev&, int dtype, const DecodePlan&, void* out, char* ws,
                                    cudaStream_t);

@@ -16,7 +16,7 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
 EncodeTiledFn encode_tiled_fn();
 
 // 3-D view (dim, row, batch * KV head) of a bf16 window buffer [B][Hkv][rows][d]; box = 64 dims x
-// 16 rows, 128-byte swizzle, rows past the end read as zero.  Maps are cached by (base, rows, d,
+// 64 rows, 128-byte swizzle, rows past the end read as zero.  Maps are cached by (base, rows, d,
 // heads).  False if rows == 0 (the map is zeroed and must not be used) or on an encoder error.
 bool window_map(CUtensorMap* tm, const void* base, int rows, int d, int n_bh);
 
