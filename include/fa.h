@@ -181,14 +181,17 @@ fa_status fa_decode_attention(const fa_layout* layout, const fa_cache* cache, co
 
 /* One decode step with device inputs (Eq.5 then Eq.6): the result and the cache afterwards are those
  * of fa_append(k_new, v_new) followed by fa_decode_attention(q).  Where the decode call is a single
- * fused kernel (see fa_decode_algo) and the KV head's query heads fit one pass, the coefficient
- * update of Eq.5 rides on that kernel: a small kernel (one CTA per batch row and KV head) moves the row that leaves the
- * local window, stores the new token and advances the counters, and the decode kernel adds
- * f_j x^T to each coefficient row as it streams it (C^K before forming u, C^V before the output
- * product) and writes it back, so the coefficients cross the memory bus once per step instead of
- * twice.  Otherwise the two calls are made one after the other.  Same arguments, workspace rule and
- * errors as those two calls (a full middle sets FA_ERR_CAPACITY in cache->status and the step decodes
- * the unchanged cache). */
+ * fused kernel (see fa_decode_algo), the KV head's query heads fit one pass and a head is spread over
+ * at least eight CTAs, the whole step is that ONE launch: every CTA applies the push to its own view of
+ * the token counters, the CTA that meets a moved row in a tile (the new token's window row, the kept
+ * dims of the row that leaves the local window) patches the tile in shared memory, f_j x^T is added
+ * to each coefficient row as the kernel streams it (C^K before forming u, C^V before the output
+ * product) and written back, so the coefficients cross the memory bus once per step instead of twice,
+ * and the moved rows and the counters are written to the cache once every CTA that reads the old
+ * ones is past them.  Otherwise the two calls are made one after the other (with few CTAs per head
+ * the stand-alone append kernel, which spreads the coefficient update over the whole device, is the
+ * faster way).  Same arguments, workspace rule and errors as those two calls (a full middle sets
+ * FA_ERR_CAPACITY in cache->status and the step decodes the unchanged cache). */
 fa_status fa_decode_step(const fa_layout* layout, fa_cache* cache, const void* q, const void* k_new,
                          const void* v_new, void* out, void* ws, size_t ws_bytes, void* stream);
 
@@ -212,10 +215,9 @@ fa_status fa_decode_step_layers(int32_t n_layers, const fa_layout* layouts, fa_c
  * fa_step_staging_bytes(layout) bytes; k_new_host == NULL skips the append.  Asynchronous on
  * `stream`: out_host is valid after the stream is synchronised.  Host buffers that the device can
  * address (pinned or registered memory, 16-byte aligned) are not copied by separate copy
- * operations: the step's first kernel reads k_new, v_new in place over the bus and copies q into
- * `staging` (when the step is not the fused two-kernel form, one staging kernel in front of it
- * reads all three), and the decode kernel writes its result rows straight into out_host.  The
- * host input buffers must not be written between the call and the completion of the step. */
+ * operations: one small kernel in front of the step reads q, k_new, v_new over the bus into
+ * `staging`, and the decode kernel writes its result rows straight into out_host.  The host input
+ * buffers must not be written between the call and the completion of the step. */
 fa_status fa_decode_step_host(const fa_layout* layout, fa_cache* cache, const void* q_host,
                               const void* k_new_host, const void* v_new_host, void* out_host,
                               void* staging, void* ws, size_t ws_bytes, void* stream);

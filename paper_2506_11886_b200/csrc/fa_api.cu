@@ -238,8 +238,6 @@ fa_status plan_decode(const fa_layout& l, DecodePlan* p) {
     p->off_oc = off;  off = align_up(off + sizeof(float) * (size_t)s.B * s.Hq * n_oc * (s.dcv > 0 ? s.dcv : 1), 256);
     p->off_om = off;  off = align_up(off + sizeof(float) * (size_t)s.B * s.Hq * s.d, 256);
     p->off_cnt = off; off = align_up(off + sizeof(int32_t) * (size_t)s.B * s.Hkv, 256);
-    p->off_pend = off; off = align_up(off + sizeof(float) * (size_t)s.B * s.Hkv * (s.dck + s.dcv + 4), 256);
-    p->off_pendj = off; off = align_up(off + sizeof(int32_t) * (size_t)s.B, 256);
     p->total = off;
     return FA_OK;
 }
@@ -462,7 +460,7 @@ fa_status fa_decode_attention(const fa_layout* layout, const fa_cache* cache, co
     cudaStream_t cs = static_cast<cudaStream_t>(stream);
     char* w = static_cast<char*>(ws);
     if (p.fused) {
-        const cudaError_t err = launch_decode_fft(s, c, layout->kv_dtype, p, q, out, w, false, cs);
+        const cudaError_t err = launch_decode_fft(s, c, layout->kv_dtype, p, q, out, w, nullptr, nullptr, cs);
         if (err == cudaSuccess) return FA_OK;
         if (err != cudaErrorCooperativeLaunchTooLarge) return FA_ERR_CUDA;
         // the device cannot hold all CTAs at once right now (SMs taken by another client): three kernels instead
@@ -473,7 +471,7 @@ fa_status fa_decode_attention(const fa_layout* layout, const fa_cache* cache, co
     }
     if (launch_decode_prologue(s, c, layout->kv_dtype, p, q, w, cs) != cudaSuccess) return FA_ERR_CUDA;
     if (p.algo == FA_DECODE_FFT) {
-        if (launch_decode_fft(s, c, layout->kv_dtype, p, q, out, w, false, cs) != cudaSuccess) return FA_ERR_CUDA;
+        if (launch_decode_fft(s, c, layout->kv_dtype, p, q, out, w, nullptr, nullptr, cs) != cudaSuccess) return FA_ERR_CUDA;
     } else {
         if (launch_decode_direct(s, c, layout->kv_dtype, p, q, w, cs) != cudaSuccess) return FA_ERR_CUDA;
     }
@@ -483,11 +481,12 @@ fa_status fa_decode_attention(const fa_layout* layout, const fa_cache* cache, co
 
 }  // extern "C"
 
-// fa_decode_step.  With q_host_view set (host-buffer step, pinned inputs, fused plan only): k_new / v_new
-// and q_host_view are device views of pinned host memory; the light append kernel reads them over the bus
-// and copies the query to q (device memory) for the decode kernel.
+constexpr int kStepFusedMinParts = 8;
+
+// fa_decode_step.  Where the decode call is the fused kernel with one pass and many parts per head, the push
+// rides on that launch; otherwise the two calls are made one after the other.
 static fa_status decode_step_impl(const fa_layout* layout, fa_cache* cache, const void* q, const void* k_new, const void* v_new,
-                                  void* out, void* ws, size_t ws_bytes, void* stream, const void* q_host_view, size_t q_bytes) {
+                                  void* out, void* ws, size_t ws_bytes, void* stream) {
     fa_status st = check_layout(layout);
     if (st != FA_OK) return st;
     st = check_cache(layout, cache);
@@ -498,37 +497,29 @@ static fa_status decode_step_impl(const fa_layout* layout, fa_cache* cache, cons
     st = plan_decode(*layout, &p);
     if (st != FA_OK) return st;
     if (!ws || !aligned16(ws) || ws_bytes < p.total) return FA_ERR_WORKSPACE;
-    if (!(p.fused && p.n_pass == 1)) {
-        if (q_host_view) return FA_ERR_UNSUPPORTED;          // (the caller checks the plan first)
-        // two calls: the coefficient update cannot ride on the decode kernel's passes over the rows
-        st = fa_append(layout, cache, k_new, v_new, stream);
-        if (st != FA_OK) return st;
-        return fa_decode_attention(layout, cache, q, out, ws, ws_bytes, stream);
-    }
     Dims s = make_dims(*layout);
-    CacheDev c = make_cache(*cache);
-    cudaStream_t cs = static_cast<cudaStream_t>(stream);
-    char* w = static_cast<char*>(ws);
-    // (a cooperative launch that does not fit the device fails before anything runs; find out first)
-    // the light append kernel must not run unless the decode kernel that finishes its update can follow
-    if (!cooperative_launch_supported() || !decode_fft_launchable(s, p)) {
-        if (q_host_view) return FA_ERR_UNSUPPORTED;
-        st = fa_append(layout, cache, k_new, v_new, stream);
-        if (st != FA_OK) return st;
-        return fa_decode_attention(layout, cache, q, out, ws, ws_bytes, stream);
+    // The push rides on the decode launch where a head has many parts (each then updates a small slice of the
+    // coefficient rows as it streams them for u and for the output product).  With few parts per head the
+    // stand-alone append kernel, which spreads the coefficient update over the whole device, is faster
+    // (measured: batch 8 MHA 22 us against 35 us inside the decode kernel, batch 4 at 128K 22 against 64).
+    // Whether the device can hold all parts at once is asked before anything is enqueued: nothing to undo.
+    if (p.fused && p.n_pass == 1 && p.n_part >= kStepFusedMinParts && cooperative_launch_supported() && decode_fft_launchable(s, p)) {
+        const cudaError_t err = launch_decode_fft(s, make_cache(*cache), layout->kv_dtype, p, q, out, static_cast<char*>(ws), k_new, v_new,
+                                                  static_cast<cudaStream_t>(stream));
+        if (err == cudaSuccess) return FA_OK;
+        if (err != cudaErrorCooperativeLaunchTooLarge) return FA_ERR_CUDA;
+        cudaGetLastError();                                  // refused before anything ran (SMs taken by another client): the two calls
     }
-    if (launch_append_lite(s, c, layout->kv_dtype, p, k_new, v_new, w, cs, q_host_view, q_host_view ? const_cast<void*>(q) : nullptr,
-                           q_bytes, q_host_view != nullptr) != cudaSuccess)
-        return FA_ERR_CUDA;
-    if (launch_decode_fft(s, c, layout->kv_dtype, p, q, out, w, true, cs) != cudaSuccess) return FA_ERR_CUDA;
-    return FA_OK;
+    st = fa_append(layout, cache, k_new, v_new, stream);
+    if (st != FA_OK) return st;
+    return fa_decode_attention(layout, cache, q, out, ws, ws_bytes, stream);
 }
 
 extern "C" {
 
 fa_status fa_decode_step(const fa_layout* layout, fa_cache* cache, const void* q, const void* k_new, const void* v_new,
                          void* out, void* ws, size_t ws_bytes, void* stream) {
-    return decode_step_impl(layout, cache, q, k_new, v_new, out, ws, ws_bytes, stream, nullptr, 0);
+    return decode_step_impl(layout, cache, q, k_new, v_new, out, ws, ws_bytes, stream);
 }
 
 fa_status fa_decode_step_layers(int32_t n_layers, const fa_layout* layouts, fa_cache* caches, const void* const* q,
@@ -549,7 +540,7 @@ fa_status fa_decode_step_layers(int32_t n_layers, const fa_layout* layouts, fa_c
         if (!ws || !aligned16(ws) || ws_bytes < p.total) return FA_ERR_WORKSPACE;
     }
     for (int i = 0; i < n_layers; ++i) {
-        const fa_status st = decode_step_impl(&layouts[i], &caches[i], q[i], k_new[i], v_new[i], out[i], ws, ws_bytes, stream, nullptr, 0);
+        const fa_status st = decode_step_impl(&layouts[i], &caches[i], q[i], k_new[i], v_new[i], out[i], ws, ws_bytes, stream);
         if (st != FA_OK) return st;
     }
     return FA_OK;
@@ -587,18 +578,7 @@ fa_status fa_decode_step_host(const fa_layout* layout, fa_cache* cache, const vo
     void* out_v = aligned16(out_host) ? const_cast<void*>(device_view_of_host(out_host)) : nullptr;
     if (out_v) o_d = static_cast<char*>(out_v);
     if (q_v && k_v && v_v) {
-        // Pinned inputs, fused step: the light append kernel reads k_new / v_new in place and copies q for the
-        // decode kernel (its loads go out before its wait on the previous kernel): no launch in front of the step.
-        DecodePlan hp;
-        if (plan_decode(*layout, &hp) == FA_OK && hp.fused && hp.n_pass == 1) {
-            st = decode_step_impl(layout, cache, q_d, k_v, v_v, o_d, ws, ws_bytes, stream, q_v, q_bytes);
-            if (st != FA_ERR_UNSUPPORTED) {
-                if (st != FA_OK) return st;
-                if (!out_v && cudaMemcpyAsync(out_host, o_d, q_bytes, cudaMemcpyDeviceToHost, cs) != cudaSuccess) return FA_ERR_CUDA;
-                return FA_OK;
-            }
-        }
-        // otherwise one staging kernel reads them over the bus (measured faster than three copy
+        // pinned inputs: one staging kernel reads them over the bus (measured faster than three copy
         // operations, and than letting every CTA of the step read the host buffers in place)
         const int nq = (int)(q_bytes / 16), nk = (int)(k_bytes / 16);
         cudaLaunchConfig_t cfg = {};
@@ -639,10 +619,10 @@ int fa_launch_count(const fa_layout* layout, int what) {
             if (plan_decode(*layout, &p) != FA_OK) return 0;
             return p.fused ? 1 : 3;
         }
-        case 3: {           // fa_decode_step: light append + fused decode, or fa_append + fa_decode_attention
+        case 3: {           // fa_decode_step: the fused decode kernel alone, or fa_append + fa_decode_attention
             DecodePlan p;
             if (plan_decode(*layout, &p) != FA_OK) return 0;
-            return (p.fused && p.n_pass == 1) ? 2 : 1 + (p.fused ? 1 : 3);
+            return (p.fused && p.n_pass == 1 && p.n_part >= kStepFusedMinParts) ? 1 : 1 + (p.fused ? 1 : 3);
         }
         default: return 0;
     }

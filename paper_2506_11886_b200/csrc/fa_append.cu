@@ -212,120 +212,6 @@ __global__ void __launch_bounds__(256) append_kernel(Dims s, CacheDev c, const K
     }
 }
 
-// First half of a fused decode step (Eq.5 without the coefficient update): one CTA per (batch row, KV head) moves
-// the row that leaves the local window (kept dims to K^mu / V^mu), stores the new token and advances
-// the counters, and leaves the compressed dims of the leaving row with its basis column j in the
-// workspace.  The decode kernel of the same step adds f_j x^T to the coefficient rows as it streams
-// them, so the coefficients are read and written once per step instead of twice.
-// Host-buffer step: with host_inputs set, k_new / v_new (and q_src) are device views of pinned host
-// memory.  Nothing earlier in the stream writes them, so their loads go out before the wait and the bus
-// round trip hides under the previous kernel's tail; q is copied to q_dst (device memory) for the decode
-// kernel, which saves a staging launch in front of the step.
-template <typename KV>
-__global__ void __launch_bounds__(256) append_lite_kernel(Dims s, CacheDev c, DecodePlan p, const KV* __restrict__ k_new,
-                                                          const KV* __restrict__ v_new, char* wsp, const uint4* __restrict__ q_src,
-                                                          uint4* __restrict__ q_dst, int nq16, int host_inputs) {
-    __shared__ float x_s[2][256];        // the row that leaves, both sides, natural dim order
-    __shared__ int last_s;
-    const int h = blockIdx.x, b = blockIdx.y, tid = threadIdx.x;
-    // the new token of this head (up to two elements per thread)
-    KV new_e[2];
-    auto load_new = [&]() {
-#pragma unroll
-        for (int u = 0; u < 2; ++u) {
-            const int i = tid + 256 * u;
-            if (i < 2 * s.d) {
-                const int side = i / s.d, e = i - side * s.d;
-                new_e[u] = ((side == 0 ? k_new : v_new) + ((size_t)b * s.Hkv + h) * s.d)[e];
-            }
-        }
-    };
-    const int gid = (b * (int)gridDim.x + h) * 256 + tid, gtot = (int)(gridDim.x * gridDim.y) * 256;
-    uint4 qv = make_uint4(0, 0, 0, 0);
-    if (host_inputs) {
-        load_new();
-        if (q_src && gid < nq16) qv = q_src[gid];
-    }
-    // wait for everything before this kernel, THEN let the decode kernel of the step start: it reads
-    // coefficient rows before its own wait, and nothing but this kernel may still be running then
-    asm volatile("griddepcontrol.wait;" ::: "memory");
-    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-    if (q_src) {                         // (the previous step's decode kernel has read q_dst by now)
-        if (gid < nq16) q_dst[gid] = host_inputs ? qv : q_src[gid];
-#pragma unroll 1
-        for (int i = gid + gtot; i < nq16; i += gtot) q_dst[i] = q_src[i];
-    }
-    Ws ws = ws_view(wsp, p);
-    const int n_init = c.state[kStateStride * b + 0], n_local = c.state[kStateStride * b + 1];
-    const int n_mid = c.state[kStateStride * b + 2], head = c.state[kStateStride * b + 3];
-    const bool to_init = n_init < s.l_init;
-    const bool evict = !to_init && n_local == s.l_local;
-    const bool full = evict && (n_mid >= s.max_mid || n_mid >= s.T);
-    if (full) {
-        if (tid == 0 && h == 0) { atomicExch(c.status, (int)FA_ERR_CAPACITY); ws.pend_j[b] = -1; }
-        return;                          // every CTA of this batch row takes the same exit
-    }
-    if (!host_inputs) load_new();        // device-resident inputs: loaded together with the leaving row
-    if (evict) {
-        const int j = n_mid;
-        for (int i = tid; i < 2 * s.d; i += 256) {
-            const int side = i / s.d, e = i - side * s.d;
-            float v;
-            if (s.l_local == 0) v = ld_f((side == 0 ? k_new : v_new) + ((size_t)b * s.Hkv + h) * s.d + e);
-            else v = ld_f(win_row<KV>(side == 0 ? c.k_local : c.v_local, s, b, h, s.l_local, head) + e);
-            x_s[side][e] = v;
-        }
-        __syncthreads();
-        for (int i = tid; i < s.nfk + s.nfv; i += 256) {
-            const int side = i < s.nfk ? 0 : 1;
-            const int e = side == 0 ? i : i - s.nfk;
-            const int nfull = side == 0 ? s.nfk : s.nfv;
-            const int32_t* idf = (side == 0 ? c.idx_full_k : c.idx_full_v) + (size_t)h * nfull;
-            KV* dst = mid_row<KV>(side == 0 ? c.k_mid : c.v_mid, s, b, h, j % s.P, j / s.P, nfull);
-            const int col = side == 1 ? v_mid_col(j / s.P, e, nfull, sizeof(KV) == 2 ? FA_BF16 : FA_F32) : e;
-            st_f(dst + col, x_s[side][idf[e]]);
-        }
-        float* pend = ws.pend + ((size_t)b * s.Hkv + h) * (s.dck + s.dcv);
-        for (int i = tid; i < s.dck + s.dcv; i += 256) {
-            const int side = i < s.dck ? 0 : 1;
-            const int e = side == 0 ? i : i - s.dck;
-            const int32_t* idc = side == 0 ? c.idx_comp_k + (size_t)h * s.dck : c.idx_comp_v + (size_t)h * s.dcv;
-            pend[i] = x_s[side][idc[e]];
-        }
-    }
-    // the new token of this head: next init row, or the ring slot behind the newest local row (the slot
-    // just read and vacated when the window is full)
-    if (evict) __syncthreads();          // every thread has read the slot that is overwritten next
-#pragma unroll
-    for (int u = 0; u < 2; ++u) {
-        const int i = tid + 256 * u;
-        if (i >= 2 * s.d) continue;
-        const int side = i / s.d, e = i - side * s.d;
-        if (to_init) {
-            win_row<KV>(side == 0 ? c.k_init : c.v_init, s, b, h, s.l_init, n_init)[e] = new_e[u];
-        } else if (s.l_local > 0) {
-            const int slot = evict ? head : (head + n_local) % s.l_local;
-            win_row<KV>(side == 0 ? c.k_local : c.v_local, s, b, h, s.l_local, slot)[e] = new_e[u];
-        }
-    }
-    // ticket: the last head of this batch row to finish advances the counters (nobody reads them after this point)
-    __syncthreads();
-    if (tid == 0) {
-        __threadfence();
-        const int done = atomicAdd(c.state + kStateStride * b + 4, 1);
-        last_s = (done == (int)gridDim.x - 1);
-    }
-    __syncthreads();
-    if (!last_s || tid != 0) return;
-    if (to_init) c.state[kStateStride * b + 0] = n_init + 1;
-    else if (evict) {
-        c.state[kStateStride * b + 2] = n_mid + 1;
-        if (s.l_local > 0) c.state[kStateStride * b + 3] = (head + 1) % s.l_local;
-    } else c.state[kStateStride * b + 1] = n_local + 1;
-    c.state[kStateStride * b + 4] = 0;            // ticket counter ready for the next call
-    ws.pend_j[b] = evict ? n_mid : -1;
-}
-
 template <typename KV>
 static cudaError_t launch_append_t(const Dims& s, const CacheDev& c, const void* k_new, const void* v_new,
                                    cudaStream_t st) {
@@ -345,28 +231,6 @@ static cudaError_t launch_append_t(const Dims& s, const CacheDev& c, const void*
     cfg.attrs = attr;
     cfg.numAttrs = 1;
     return cudaLaunchKernelEx(&cfg, append_kernel<KV>, s, c, static_cast<const KV*>(k_new), static_cast<const KV*>(v_new), rows);
-}
-
-template <typename KV>
-static cudaError_t launch_append_lite_t(const Dims& s, const CacheDev& c, const DecodePlan& p, const void* k_new, const void* v_new,
-                                        char* ws, cudaStream_t st, const void* q_src, void* q_dst, size_t q_bytes, bool host_inputs) {
-    cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(s.Hkv, s.B);
-    cfg.blockDim = dim3(256);
-    cfg.stream = st;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[0].val.programmaticStreamSerializationAllowed = 1;
-    cfg.attrs = attr;
-    cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, append_lite_kernel<KV>, s, c, p, static_cast<const KV*>(k_new), static_cast<const KV*>(v_new), ws,
-                              static_cast<const uint4*>(q_src), static_cast<uint4*>(q_dst), (int)(q_bytes / 16), host_inputs ? 1 : 0);
-}
-
-cudaError_t launch_append_lite(const Dims& s, const CacheDev& c, int dtype, const DecodePlan& p, const void* k_new, const void* v_new,
-                               char* ws, cudaStream_t st, const void* q_src, void* q_dst, size_t q_bytes, bool host_inputs) {
-    if (dtype == FA_BF16) return launch_append_lite_t<__nv_bfloat16>(s, c, p, k_new, v_new, ws, st, q_src, q_dst, q_bytes, host_inputs);
-    return launch_append_lite_t<float>(s, c, p, k_new, v_new, ws, st, q_src, q_dst, q_bytes, host_inputs);
 }
 
 cudaError_t launch_append(const Dims& s, const CacheDev& c, int dtype, const void* k_new, const void* v_new,

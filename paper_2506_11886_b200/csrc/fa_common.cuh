@@ -72,7 +72,7 @@ struct DecodePlan {
     int nb;            // classes transformed together by one CTA (FFT path)
     int occ;           // CTAs per SM the main kernel is built for (FFT path: 1, or 2 with a shorter ring)
     // workspace offsets in bytes
-    size_t off_bar, off_u, off_ml, off_o, off_z, off_oc, off_om, off_cnt, off_pend, off_pendj, total;
+    size_t off_bar, off_u, off_ml, off_o, off_z, off_oc, off_om, off_cnt, total;
 };
 
 // V^mu of bf16 caches is stored with its 16-byte chunks (8 dims) permuted inside each row:
@@ -111,11 +111,9 @@ cudaError_t launch_decode_prologue(const Dims&, const CacheDev&, int dtype, cons
                                    cudaStream_t);
 cudaError_t launch_decode_direct(const Dims&, const CacheDev&, int dtype, const DecodePlan&, const void* q, char* ws,
                                  cudaStream_t);
-cudaError_t launch_append_lite(const Dims&, const CacheDev&, int dtype, const DecodePlan&, const void* k_new, const void* v_new,
-                               char* ws, cudaStream_t, const void* q_src = nullptr, void* q_dst = nullptr, size_t q_bytes = 0,
-                               bool host_inputs = false);
-cudaError_t launch_decode_fft(const Dims&, const CacheDev&, int dtype, const DecodePlan&, const void* q, void* out, char* ws, bool step,
-                              cudaStream_t);
+// k_new / v_new non-null: a fused step (the push of Eq.5 rides on the decode launch; fused plans with one pass only).
+cudaError_t launch_decode_fft(const Dims&, const CacheDev&, int dtype, const DecodePlan&, const void* q, void* out, char* ws,
+                              const void* k_new, const void* v_new, cudaStream_t);
 size_t decode_fft_smem_bytes(const Dims&, int log2S, int gh, int nb, int occ = 1);
 bool decode_fft_fused_fits(const Dims&, int log2S, int gh, int nb, int n_part, int occ = 1);
 bool decode_fft_launchable(const Dims&, const DecodePlan&);

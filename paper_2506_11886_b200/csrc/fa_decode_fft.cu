@@ -418,21 +418,24 @@ __host__ __device__ inline FftSmem fft_smem_layout(int log2S, int k, int GH, int
     L.o_off = off; off += 8 * GH * d;
     L.red_off = off; off += 4 * (kWarps * GH + GH + 8);
     off = (off + 15) / 16 * 16;
-    L.pend_off = off; off += 8 * d + 4 * kPendRows;        // fused step: compressed dims of the leaving row, basis column of this part's rows
+    L.pend_off = off; off += 8 * d + 4 * kPendRows + 4 * d + 2 * GH * d + 4 * d;   // fused step: compressed dims of the leaving row, basis column of this part's rows, the leaving row; the query rows
     L.total = (off + 127) / 128 * 128 + 1024;             // slack to align the base to 1024 bytes at run time
     return L;
 }
 
 template <int GH> __host__ __device__ constexpr int hperm(int s) { return GH == 4 ? (((s & 1) << 1) | (s >> 1)) : s; }
 
-// GH query heads per CTA (2 or 4), transform length S = 2^LS, OCC CTAs per SM (2: shorter ring, register cap).
-template <int GH, int LS, int OCC>
+// GH query heads per CTA (2 or 4), transform length S = 2^LS, OCC CTAs per SM (2: shorter ring, register cap),
+// STEP: the instance that also carries the push of a fused step (the plain decode call pays nothing for it).
+template <int GH, int LS, int OCC, bool STEP>
 __global__ void __launch_bounds__(kThreads, OCC) decode_fft_kernel(const __grid_constant__ CUtensorMap tm_ki,
                                                                   const __grid_constant__ CUtensorMap tm_vi,
                                                                   const __grid_constant__ CUtensorMap tm_kl,
                                                                   const __grid_constant__ CUtensorMap tm_vl, Dims s, CacheDev c,
                                                                   DecodePlan p, const bf16* __restrict__ q, bf16* __restrict__ out,
-                                                                  char* wsp, int step) {
+                                                                  char* wsp, const bf16* __restrict__ k_new,
+                                                                  const bf16* __restrict__ v_new) {
+    constexpr bool step = STEP;
     constexpr int N = GH / 2;
     constexpr int S = 1 << LS;
     constexpr int NS = ring_stages(OCC);
@@ -493,9 +496,8 @@ __global__ void __launch_bounds__(kThreads, OCC) decode_fft_kernel(const __grid_
         if (tid < GH + 8) red_s[kWarps * GH + tid] = 0.f;
 
     }
-    // Fused step: the only kernel still running before this one is the light append, which does not
-    // touch the coefficients (it triggers this launch after its own wait), so this part's rows of C^K
-    // can start towards the transform buffers, and its rows of C^V towards L2, before the wait.
+    // This part's rows of C^K start towards the transform buffers, and its rows of C^V towards L2, as soon as
+    // the kernels before this one are done (the previous step's kernel writes coefficient rows).
     const int m0 = part * (s.M >> 2) / p.n_part * 4, m1 = (part + 1) * (s.M >> 2) / p.n_part * 4;
     // rows of C^K staged at a time: the transform buffers and, behind them, the kept-dim score and probability
     // buffers (one contiguous area, all idle until the first batch)
@@ -514,13 +516,72 @@ __global__ void __launch_bounds__(kThreads, OCC) decode_fft_kernel(const __grid_
             for (int o = tid * 128; o < bytes; o += kConsumers * 128) asm volatile("prefetch.global.L2 [%0];" ::"l"(cv + o));
         }
     };
-    if (p.fused && step) start_coef_rows();
-    // fused kernel: everything below reads what earlier kernels in the stream wrote (state, cache, q)
-    if (p.fused) asm volatile("griddepcontrol.wait;" ::: "memory");
-    if (p.fused && !step) start_coef_rows();
+    // The inputs of the call, staged once: the query rows of this pass [GH heads][d] and, for a fused step, the
+    // new token of this KV head [2 sides][d].
+    bf16* xrow_s = reinterpret_cast<bf16*>(smem_raw + L.pend_off + 8 * s.d + 4 * kPendRows);     // [2][d] the row that leaves the window
+    bf16* qs_s = xrow_s + 2 * s.d;                                                                 // [GH][d]
+    bf16* nrow_s = qs_s + GH * s.d;                                                                // [2][d]
+    const bf16* knew_bh = nrow_s;
+    const bf16* vnew_bh = nrow_s + s.d;
+    auto stage_inputs = [&]() {
+        const int per_row = s.d >> 3;
+        if (tid < GH * per_row) {
+            const int g = tid / per_row, ch = tid - g * per_row;
+            uint4 v = make_uint4(0, 0, 0, 0);
+            if (g < ng) v = *reinterpret_cast<const uint4*>(q + ((size_t)b * s.Hq + g_first + g) * s.d + 8 * ch);
+            *reinterpret_cast<uint4*>(qs_s + g * s.d + 8 * ch) = v;
+        } else if (STEP && tid < (GH + 2) * per_row) {
+            const int side = (tid - GH * per_row) / per_row, ch = tid - (GH + side) * per_row;
+            *reinterpret_cast<uint4*>(nrow_s + side * s.d + 8 * ch) =
+                *reinterpret_cast<const uint4*>((side == 0 ? k_new : v_new) + ((size_t)b * s.Hkv + h) * s.d + 8 * ch);
+        }
+    };
+    // fused kernel: everything below reads what earlier kernels in the stream wrote (state, cache, coefficients, q)
+    if (p.fused) {
+        asm volatile("griddepcontrol.wait;" ::: "memory");
+        start_coef_rows();
+    }
+    stage_inputs();
 
-    const int n_init = c.state[kStateStride * b + 0], n_local = c.state[kStateStride * b + 1];
-    const int n_mid = min(c.state[kStateStride * b + 2], s.max_mid), head = c.state[kStateStride * b + 3];
+    int n_init = c.state[kStateStride * b + 0], n_local = c.state[kStateStride * b + 1];
+    int n_mid_raw = c.state[kStateStride * b + 2], head = c.state[kStateStride * b + 3];
+    // Fused step (Eq.5 then Eq.6 in this one launch): every CTA applies the push to its own view of the counters
+    // and works on the cache as it will be.  The rows that the push moves are not in place yet: the CTA that
+    // meets one in a tile patches the tile in shared memory (the new token's window row from k_new / v_new, the
+    // kept dims of the row that leaves the local window at middle token j_pend), the rank-1 update f_j x^T is
+    // added to the coefficient rows as they stream by, and the rows and counters are written to the cache
+    // when every CTA that reads the old ones is past them.
+    int j_pend = -1;                                      // basis column of the coefficient update, or -1
+    int new_buf = -1, new_row = 0, new_tok = -1;          // buffer (0 init, 1 local) and row of the new token, its logical window index
+    bool cap_full = false;
+    if (step) {
+        const bool to_init = n_init < s.l_init;
+        const bool evict = !to_init && n_local == s.l_local;
+        cap_full = evict && (n_mid_raw >= s.max_mid || n_mid_raw >= s.T);
+        if (cap_full) {
+            if (tid == 0 && part == 0 && h == 0 && pass == 0) atomicExch(c.status, (int)FA_ERR_CAPACITY);
+        } else if (to_init) {
+            new_buf = 0; new_row = n_init; new_tok = n_init; ++n_init;
+        } else if (!evict) {
+            new_buf = 1; new_row = (head + n_local) % s.l_local; new_tok = n_init + n_local; ++n_local;
+        } else {
+            j_pend = n_mid_raw; ++n_mid_raw;
+            if (s.l_local > 0) { new_buf = 1; new_row = head; head = (head + 1) % s.l_local; new_tok = n_init + n_local - 1; }
+        }
+    }
+    const int n_mid = min(n_mid_raw, s.max_mid);
+    const int cstar = j_pend >= 0 ? j_pend & (s.P - 1) : -1, astar = j_pend >= 0 ? j_pend >> log2P : 0;   // class and slot of token j_pend
+    // the row that leaves the local window (or the new token itself without a local window), both sides, natural dim order
+    if (j_pend >= 0 && tid >= kConsumers - 2 * (s.d >> 3) && tid < kConsumers) {
+        const int t2 = tid - (kConsumers - 2 * (s.d >> 3));
+        const int side = t2 / (s.d >> 3), ch = t2 - side * (s.d >> 3);
+        if (s.l_local > 0)
+            *reinterpret_cast<uint4*>(xrow_s + side * s.d + 8 * ch) =
+                *reinterpret_cast<const uint4*>(win_row<bf16>(side == 0 ? c.k_local : c.v_local, s, b, h, s.l_local, new_row) + 8 * ch);
+        else
+            *reinterpret_cast<uint4*>(xrow_s + side * s.d + 8 * ch) =
+                *reinterpret_cast<const uint4*>((side == 0 ? k_new : v_new) + ((size_t)b * s.Hkv + h) * s.d + 8 * ch);
+    }
     const int c0 = is_win ? 0 : part * s.P / p.n_split;
     const int c1 = is_win ? 0 : (part + 1) * s.P / p.n_split;
     const int n_win = n_init + n_local;
@@ -622,16 +683,16 @@ __global__ void __launch_bounds__(kThreads, OCC) decode_fft_kernel(const __grid_
     float qc_early = 0.f;
     if (p.fused && s.dck > 0 && tid < GH * s.dck) {
         const int g = tid / s.dck, e = tid - g * s.dck;
-        if (g < ng) qc_early = __bfloat162float(q[((size_t)b * s.Hq + g_first + g) * s.d + c.idx_comp_k[(size_t)h * s.dck + e]]);
+        if (g < ng) qc_early = __bfloat162float(qs_s[g * s.d + c.idx_comp_k[(size_t)h * s.dck + e]]);
     }
     // fused step: the coefficient update the light append kernel left pending (basis column j_pend, or -1);
     // the leaving row's compressed dims and the basis values of this part's rows are fetched / formed now
     float* xp_s = reinterpret_cast<float*>(smem_raw + L.pend_off);       // [dck + dcv]
     float* f_s = xp_s + 2 * s.d;                                          // [kPendRows]
-    const int j_pend = step ? ws.pend_j[b] : -1;
     if (j_pend >= 0) {
-        const float* xp = ws.pend + ((size_t)b * s.Hkv + h) * (s.dck + s.dcv);
-        for (int i = tid; i < (s.dck + s.dcv) >> 2; i += kConsumers) cp_async16(xp_s + 4 * i, xp + 4 * i);
+        for (int i = tid; i < s.dck + s.dcv; i += kConsumers)
+            xp_s[i] = i < s.dck ? __bfloat162float(xrow_s[c.idx_comp_k[(size_t)h * s.dck + i]])
+                                : __bfloat162float(xrow_s[s.d + c.idx_comp_v[(size_t)h * s.dcv + i - s.dck]]);
 #pragma unroll 1
         for (int r = tid; r < min(m1 - m0, kPendRows); r += kConsumers) f_s[r] = basis_value(m0 + r, j_pend, s.T);
     }
@@ -644,7 +705,7 @@ __global__ void __launch_bounds__(kThreads, OCC) decode_fft_kernel(const __grid_
     // round rd covers pieces 4 rd + tq of a row, two k-steps each
     const int my_head = hperm<GH>(gq & (GH - 1));
     const bool col_on = gq < GH && my_head < ng;
-    const bf16* qrow = q + ((size_t)b * s.Hq + g_first + my_head) * s.d;
+    const bf16* qrow = qs_s + my_head * s.d;
     uint32_t qk[2][2][2];
     {
         const int32_t* idf_k = c.idx_full_k + (size_t)h * s.nfk;
@@ -699,6 +760,14 @@ __global__ void __launch_bounds__(kThreads, OCC) decode_fft_kernel(const __grid_
 #pragma unroll 1
                 for (int grp = warp; grp * 16 < nt; grp += kWarps) {
                     const uint32_t gbase = tile + (uint32_t)(grp * 16) * rowb_k;
+                    if (STEP && cb + ci == cstar && astar >= a0 + grp * 16 && astar < a0 + grp * 16 + 16) {
+                        // fused step: middle token j_pend is not in the cache yet; its kept dims from the row that leaves the window
+                        const int32_t* idf = c.idx_full_k + (size_t)h * s.nfk;
+#pragma unroll 1
+                        for (int e = lane; e < s.nfk; e += 32)
+                            asm volatile("st.shared.b16 [%0], %1;" ::"r"(tile + (uint32_t)((astar - a0) * rowb_k + 2 * e)), "h"(__bfloat16_as_ushort(xrow_s[idf[e]])) : "memory");
+                        __syncwarp();
+                    }
                     float d4[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
                     for (int rd = 0; rd < 2; ++rd) {
@@ -732,7 +801,7 @@ __global__ void __launch_bounds__(kThreads, OCC) decode_fft_kernel(const __grid_
             const int32_t* idc_k = c.idx_comp_k + (size_t)h * s.dck;
             for (int i = tid; i < GH * s.dck; i += kConsumers) {
                 const int g = i / s.dck, e = i - g * s.dck;
-                qc[i] = i < kConsumers ? qc_early : (g < ng ? __bfloat162float(q[((size_t)b * s.Hq + g_first + g) * s.d + idc_k[e]]) : 0.f);
+                qc[i] = i < kConsumers ? qc_early : (g < ng ? __bfloat162float(qs_s[g * s.d + idc_k[e]]) : 0.f);
             }
             const int l8 = tid & 7, rgi = tid >> 3, nv = s.dck >> 2;
             float* ckg = coef_rows(c.coef_k, s, b, h, s.dck);
@@ -887,6 +956,15 @@ __global__ void __launch_bounds__(kThreads, OCC) decode_fft_kernel(const __grid_
         return cis_frac((float)((n * cls) & (s.T - 1)) / (float)s.T);
     };
 
+    // fused step: writes the new token's row (all d dims) over row `prow` of a window tile (128-byte swizzle), by one warp
+    auto patch_win = [&](const unsigned char* tile, int prow, const bf16* src) {
+#pragma unroll 1
+        for (int cc = lane; cc < npw; cc += 32)
+            *reinterpret_cast<uint4*>(const_cast<unsigned char*>(tile) + (cc >> 3) * kWinHalfBytes + prow * 128 + (((cc & 7) ^ (prow & 7)) << 4)) =
+                *reinterpret_cast<const uint4*>(src + 8 * cc);
+        __syncwarp();
+    };
+
     // ------------------------------ window tokens -------------------------------
     if (w1 > w0) {
         uint32_t qw[4][2][2];
@@ -919,8 +997,10 @@ __global__ void __launch_bounds__(kThreads, OCC) decode_fft_kernel(const __grid_
                 for (int r0 = 0; r0 < sg.cnt[si]; r0 += ts_w) {
                     const int nt = min(ts_w, sg.cnt[si] - r0);
                     const unsigned char* tile = wait_tile();
+                    const int nrow = new_buf == sg.buf[si] ? new_row - (sg.row[si] + r0) : -1;   // fused step: the new token's row in this tile
                     #pragma unroll 1
                     for (int grp = (warp + kWarps - (it * (kWinRowsPerTile / 16)) % kWarps) % kWarps; grp * 16 < nt; grp += kWarps) {   // tiles rotate over the warps
+                        if (STEP && nrow >= grp * 16 && nrow < grp * 16 + 16) patch_win(tile, nrow, knew_bh);
                         const unsigned char* r_lo = tile + (size_t)(grp * 16 + gq) * 128;      // row & 7 == gq for both rows
                         float d4[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
@@ -993,8 +1073,10 @@ __global__ void __launch_bounds__(kThreads, OCC) decode_fft_kernel(const __grid_
                 for (int r0 = 0; r0 < sg.cnt[si]; r0 += ts_w) {
                     const int nt = min(ts_w, sg.cnt[si] - r0);
                     const unsigned char* tile = wait_tile();
+                    const int nrow = new_buf == sg.buf[si] ? new_row - (sg.row[si] + r0) : -1;
                     #pragma unroll 1
                     for (int grp = (warp + kWarps - (it * (kWinRowsPerTile / 16)) % kWarps) % kWarps; grp * 16 < nt; grp += kWarps) {
+                        if (STEP && nrow >= grp * 16 && nrow < grp * 16 + 16) patch_win(tile, nrow, vnew_bh);
                         const int a = sg.tok[si] + r0 + grp * 16;
                         // the tile's rows may start at any token of the chunk: gather the four p values one by one
                         uint32_t b0 = 0, b1 = 0;
@@ -1205,6 +1287,14 @@ __global__ void __launch_bounds__(kThreads, OCC) decode_fft_kernel(const __grid_
                         #pragma unroll 1
                         for (int grp = warp; grp * 16 < nt; grp += kWarps) {
                             const uint32_t gbase = tile + (uint32_t)(grp * 16) * rowb_v;
+                            if (STEP && cb + ci == cstar && astar >= a0 + grp * 16 && astar < a0 + grp * 16 + 16) {
+                                const int32_t* idf = c.idx_full_v + (size_t)h * s.nfv;
+#pragma unroll 1
+                                for (int e = lane; e < s.nfv; e += 32)
+                                    asm volatile("st.shared.b16 [%0], %1;" ::"r"(tile + (uint32_t)((astar - a0) * rowb_v + 2 * v_mid_col(astar, e, s.nfv, FA_BF16))),
+                                                 "h"(__bfloat16_as_ushort(xrow_s[s.d + idf[e]])) : "memory");
+                                __syncwarp();
+                            }
                             uint32_t b0 = 0, b1 = 0;
                             if (gq < GH) {
                                 b0 = lds32(prow + (uint32_t)(a0 + grp * 16) * 2);
@@ -1378,6 +1468,24 @@ __global__ void __launch_bounds__(kThreads, OCC) decode_fft_kernel(const __grid_
     if (s.dcv > 0) stage_cv(0, min(rows, mch));            // under the barrier
     part_arrive(bar + 1, np, tid);
     part_wait(bar + 1, np, tid, fail, c.status);
+    // Fused step: every part of this (b, KV head) has read the row that leaves the window and is past its token
+    // loop, so the rows the push moves can be written to the cache now, each by the part that owns it.
+    if (step && !cap_full) {
+        if (j_pend >= 0 && !is_win && cstar >= c0 && cstar < c1) {
+            bf16* dk = mid_row<bf16>(c.k_mid, s, b, h, cstar, astar, s.nfk);
+            bf16* dv = mid_row<bf16>(c.v_mid, s, b, h, cstar, astar, s.nfv);
+#pragma unroll 1
+            for (int e = tid; e < s.nfk; e += kConsumers) dk[e] = xrow_s[c.idx_full_k[(size_t)h * s.nfk + e]];
+#pragma unroll 1
+            for (int e = tid; e < s.nfv; e += kConsumers) dv[v_mid_col(astar, e, s.nfv, FA_BF16)] = xrow_s[s.d + c.idx_full_v[(size_t)h * s.nfv + e]];
+        }
+        if (new_buf >= 0 && new_tok >= w0 && new_tok < w1 && tid < 2 * (s.d >> 3)) {
+            const int side = tid / (s.d >> 3), ch = tid - side * (s.d >> 3);
+            bf16* dst = new_buf == 0 ? win_row<bf16>(side == 0 ? c.k_init : c.v_init, s, b, h, s.l_init, new_row)
+                                     : win_row<bf16>(side == 0 ? c.k_local : c.v_local, s, b, h, s.l_local, new_row);
+            *reinterpret_cast<uint4*>(dst + 8 * ch) = *reinterpret_cast<const uint4*>((side == 0 ? knew_bh : vnew_bh) + 8 * ch);
+        }
+    }
 #pragma unroll 1
     for (int i = tid; i < GH * np; i += kConsumers) {
         float2 ml = make_float2(kNegBig, 0.f);
@@ -1532,6 +1640,16 @@ __global__ void __launch_bounds__(kThreads, OCC) decode_fft_kernel(const __grid_
         out[(qh0 + g) * s.d + e] = __float2bfloat16_rn(v * linv_s[g]);
     }
     if (tid == 0 && np > 1) { bar[0] = 0; bar[1] = 0; bar[2] = 0; }   // the counters are zero again for the next call
+    // Fused step: the last (KV head, pass) of this batch row to finish publishes the counters after the push
+    // (the others read the old ones when they started; the next kernel in the stream sees the new ones).
+    if (step && !cap_full && tid == 0) {
+        int32_t* st = c.state + kStateStride * b;
+        const int old = atomicAdd(st + 4, 1);
+        if (old == s.Hkv * p.n_pass - 1) {
+            st[0] = n_init; st[1] = n_local; st[2] = n_mid_raw; st[3] = head;
+            st[4] = 0;
+        }
+    }
 }
 
 // Whether the driver takes the cooperative and the programmatic-serialization launch attributes
@@ -1549,11 +1667,11 @@ static int coop_pdl_state(int set) {
     return state[dev];
 }
 
-template <int GH, int LS, int OCC>
+template <int GH, int LS, int OCC, bool STEP>
 cudaError_t launch_fft_t(const Dims& s, const CacheDev& c, const DecodePlan& p, const void* q, void* out, char* ws, int step,
-                         cudaStream_t st) {
+                         const void* k_new, const void* v_new, cudaStream_t st) {
     const FftSmem L = fft_smem_layout(LS, s.k, GH, p.nb, s.d, OCC);
-    cudaError_t err = ensure_dynamic_smem(decode_fft_kernel<GH, LS, OCC>, (size_t)L.total);
+    cudaError_t err = ensure_dynamic_smem(decode_fft_kernel<GH, LS, OCC, STEP>, (size_t)L.total);
     if (err != cudaSuccess) return err;
     // window buffers as tensor maps (cached per buffer)
     CUtensorMap tki, tvi, tkl, tvl;
@@ -1584,8 +1702,9 @@ cudaError_t launch_fft_t(const Dims& s, const CacheDev& c, const DecodePlan& p, 
             cfg.attrs = attr + 1;                                          // not probed yet: stay on the plain cooperative launch
         } else if (known != 0) {
             cfg.numAttrs = 2;
-            cudaError_t err2 = cudaLaunchKernelEx(&cfg, decode_fft_kernel<GH, LS, OCC>, tki, tvi, tkl, tvl, s, c, p,
-                                                  static_cast<const bf16*>(q), static_cast<bf16*>(out), ws, step);
+            cudaError_t err2 = cudaLaunchKernelEx(&cfg, decode_fft_kernel<GH, LS, OCC, STEP>, tki, tvi, tkl, tvl, s, c, p,
+                                                  static_cast<const bf16*>(q), static_cast<bf16*>(out), ws,
+                                                  static_cast<const bf16*>(k_new), static_cast<const bf16*>(v_new));
             if (err2 == cudaSuccess) { coop_pdl_state(1); return err2; }
             if (known == 1) return err2;
             cudaGetLastError();
@@ -1596,26 +1715,26 @@ cudaError_t launch_fft_t(const Dims& s, const CacheDev& c, const DecodePlan& p, 
             cfg.attrs = attr + 1;
         }
     }
-    return cudaLaunchKernelEx(&cfg, decode_fft_kernel<GH, LS, OCC>, tki, tvi, tkl, tvl, s, c, p, static_cast<const bf16*>(q),
-                              static_cast<bf16*>(out), ws, step);
+    return cudaLaunchKernelEx(&cfg, decode_fft_kernel<GH, LS, OCC, STEP>, tki, tvi, tkl, tvl, s, c, p, static_cast<const bf16*>(q),
+                              static_cast<bf16*>(out), ws, static_cast<const bf16*>(k_new), static_cast<const bf16*>(v_new));
 }
 
 template <int GH>
 cudaError_t launch_fft_ls(const Dims& s, const CacheDev& c, const DecodePlan& p, const void* q, void* out, char* ws, int step,
-                          cudaStream_t st) {
+                          const void* k_new, const void* v_new, cudaStream_t st) {
     switch (p.fft_log2) {
-        case 5: return p.occ == 2 ? launch_fft_t<GH, 5, 2>(s, c, p, q, out, ws, step, st) : launch_fft_t<GH, 5, 1>(s, c, p, q, out, ws, step, st);
-        case 6: return p.occ == 2 ? launch_fft_t<GH, 6, 2>(s, c, p, q, out, ws, step, st) : launch_fft_t<GH, 6, 1>(s, c, p, q, out, ws, step, st);
-        case 7: return p.occ == 2 ? launch_fft_t<GH, 7, 2>(s, c, p, q, out, ws, step, st) : launch_fft_t<GH, 7, 1>(s, c, p, q, out, ws, step, st);
-        case 8: return p.occ == 2 ? launch_fft_t<GH, 8, 2>(s, c, p, q, out, ws, step, st) : launch_fft_t<GH, 8, 1>(s, c, p, q, out, ws, step, st);
-        case 9: return launch_fft_t<GH, 9, 1>(s, c, p, q, out, ws, step, st);
-        case 10: return launch_fft_t<GH, 10, 1>(s, c, p, q, out, ws, step, st);
+        case 5: return p.occ == 2 ? (step ? launch_fft_t<GH, 5, 2, true>(s, c, p, q, out, ws, step, k_new, v_new, st) : launch_fft_t<GH, 5, 2, false>(s, c, p, q, out, ws, step, k_new, v_new, st)) : (step ? launch_fft_t<GH, 5, 1, true>(s, c, p, q, out, ws, step, k_new, v_new, st) : launch_fft_t<GH, 5, 1, false>(s, c, p, q, out, ws, step, k_new, v_new, st));
+        case 6: return p.occ == 2 ? (step ? launch_fft_t<GH, 6, 2, true>(s, c, p, q, out, ws, step, k_new, v_new, st) : launch_fft_t<GH, 6, 2, false>(s, c, p, q, out, ws, step, k_new, v_new, st)) : (step ? launch_fft_t<GH, 6, 1, true>(s, c, p, q, out, ws, step, k_new, v_new, st) : launch_fft_t<GH, 6, 1, false>(s, c, p, q, out, ws, step, k_new, v_new, st));
+        case 7: return p.occ == 2 ? (step ? launch_fft_t<GH, 7, 2, true>(s, c, p, q, out, ws, step, k_new, v_new, st) : launch_fft_t<GH, 7, 2, false>(s, c, p, q, out, ws, step, k_new, v_new, st)) : (step ? launch_fft_t<GH, 7, 1, true>(s, c, p, q, out, ws, step, k_new, v_new, st) : launch_fft_t<GH, 7, 1, false>(s, c, p, q, out, ws, step, k_new, v_new, st));
+        case 8: return p.occ == 2 ? (step ? launch_fft_t<GH, 8, 2, true>(s, c, p, q, out, ws, step, k_new, v_new, st) : launch_fft_t<GH, 8, 2, false>(s, c, p, q, out, ws, step, k_new, v_new, st)) : (step ? launch_fft_t<GH, 8, 1, true>(s, c, p, q, out, ws, step, k_new, v_new, st) : launch_fft_t<GH, 8, 1, false>(s, c, p, q, out, ws, step, k_new, v_new, st));
+        case 9: return (step ? launch_fft_t<GH, 9, 1, true>(s, c, p, q, out, ws, step, k_new, v_new, st) : launch_fft_t<GH, 9, 1, false>(s, c, p, q, out, ws, step, k_new, v_new, st));
+        case 10: return (step ? launch_fft_t<GH, 10, 1, true>(s, c, p, q, out, ws, step, k_new, v_new, st) : launch_fft_t<GH, 10, 1, false>(s, c, p, q, out, ws, step, k_new, v_new, st));
         default: return cudaErrorInvalidValue;
     }
 }
 
 // Resident CTAs of this kernel instance on the whole device for the plan's shared memory (cached per instance).
-template <int GH, int LS, int OCC>
+template <int GH, int LS, int OCC, bool STEP = true>
 int resident_ctas_t(const Dims& s, const DecodePlan& p) {
     // answers cached per (device, shared memory size) of this instance
     struct Entry { int dev; size_t smem; int ctas; };
@@ -1628,9 +1747,9 @@ int resident_ctas_t(const Dims& s, const DecodePlan& p) {
     std::lock_guard<std::mutex> lock(mu);
     for (int i = 0; i < used; ++i)
         if (table[i].dev == dev && table[i].smem == smem) return table[i].ctas;
-    if (ensure_dynamic_smem(decode_fft_kernel<GH, LS, OCC>, smem) != cudaSuccess) { cudaGetLastError(); return 0; }
+    if (ensure_dynamic_smem(decode_fft_kernel<GH, LS, OCC, STEP>, smem) != cudaSuccess) { cudaGetLastError(); return 0; }
     int per_sm = 0;
-    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, decode_fft_kernel<GH, LS, OCC>, kThreads, smem) != cudaSuccess) {
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, decode_fft_kernel<GH, LS, OCC, STEP>, kThreads, smem) != cudaSuccess) {
         cudaGetLastError();
         return 0;
     }
@@ -1684,10 +1803,11 @@ bool decode_fft_fused_fits(const Dims& s, int log2S, int gh, int nb, int n_part,
 }
 
 cudaError_t launch_decode_fft(const Dims& s, const CacheDev& c, int dtype, const DecodePlan& p, const void* q, void* out,
-                              char* ws, bool step, cudaStream_t st) {
+                              char* ws, const void* k_new, const void* v_new, cudaStream_t st) {
     if (dtype != FA_BF16) return cudaErrorInvalidValue;
-    if (p.gh == 4) return launch_fft_ls<4>(s, c, p, q, out, ws, step ? 1 : 0, st);
-    return launch_fft_ls<2>(s, c, p, q, out, ws, step ? 1 : 0, st);
+    const int step = k_new != nullptr && v_new != nullptr ? 1 : 0;      // a fused step: the push of (k_new, v_new) rides on this launch
+    if (p.gh == 4) return launch_fft_ls<4>(s, c, p, q, out, ws, step, k_new, v_new, st);
+    return launch_fft_ls<2>(s, c, p, q, out, ws, step, k_new, v_new, st);
 }
 
 }  // namespace fa

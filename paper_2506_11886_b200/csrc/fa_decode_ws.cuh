@@ -15,8 +15,6 @@ struct Ws {
     float* oc;     // [B][Hq][max(n_slice, n_part)][dcv] partial o^c per coefficient-row slice
     float* om;     // [B][Hq][d]            merged o (fused kernel)
     int32_t* cnt;  // [B][Hkv]              epilogue tickets
-    float* pend;   // [B][Hkv][dck + dcv]   fused step: compressed dims of the row that left the local window
-    int32_t* pend_j;  // [B]                fused step: its basis column j, or -1 if no coefficient update is pending
 };
 
 __host__ __device__ inline Ws ws_view(char* w, const DecodePlan& p) {
@@ -29,8 +27,6 @@ __host__ __device__ inline Ws ws_view(char* w, const DecodePlan& p) {
     v.oc = reinterpret_cast<float*>(w + p.off_oc);
     v.om = reinterpret_cast<float*>(w + p.off_om);
     v.cnt = reinterpret_cast<int32_t*>(w + p.off_cnt);
-    v.pend = reinterpret_cast<float*>(w + p.off_pend);
-    v.pend_j = reinterpret_cast<int32_t*>(w + p.off_pendj);
     return v;
 }
 

@@ -84,14 +84,14 @@ def test_launch_plan_is_host_logic():
     """Which form a decode call takes is decided on the host from the layout alone: one fused
     kernel (cooperative while a head has several CTAs; with more heads than SMs, one CTA per head in
     waves), three kernels when asked for or when the fused kernel's staging does not fit; the fused
-    step (light append + decode) needs the fused kernel."""
+    step (the push riding on the decode launch) needs the fused kernel."""
     lib = fa.lib()
 
     def launches(what, **kw):
         return lib.fa_launch_count(C.byref(_layout(**kw).c()), what)
 
     assert launches(0) == 2 and launches(1) == 1
-    assert launches(2) == 1 and launches(3) == 2                                   # 8 KV heads: 18 CTAs each
+    assert launches(2) == 1 and launches(3) == 1                                   # 8 KV heads: 18 CTAs each; the step is one launch
     assert launches(2, decode_algo=fa.FA_DECODE_FFT_SPLIT) == 3 and launches(3, decode_algo=fa.FA_DECODE_FFT_SPLIT) == 4
     assert launches(2, decode_algo=fa.FA_DECODE_DIRECT) == 3
     assert launches(2, batch=8) == 1                                               # 64 (b, head) pairs: two CTAs each

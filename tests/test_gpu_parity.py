@@ -268,7 +268,7 @@ def test_decode_step_after_compress_gqa_batch():
     for t in range(12):
         pair.check_step(synth.queries(shape, seed=13, step=t), K[:, t], V[:, t])
     pair.check_state()
-    assert fa.fa_launch_count(pair.layout, 3) in (2, 3, 4)
+    assert fa.fa_launch_count(pair.layout, 3) in (1, 2, 4)       # one launch where the decode call is the fused kernel
 
 
 def test_decode_step_full_middle_reports_capacity():
@@ -401,7 +401,7 @@ def test_fused_decode_more_heads_than_sms(T, P, M):
     ring, register cap); 512: one per SM."""
     shape = SMALL_BF16.with_(B=20, Hq=16, Hkv=8, L=700, T=T, M=M, n_full_k=32, n_full_v=48, decode_steps=2)
     pair, stream = make_pair(shape, seed=23, algo=fa.FA_DECODE_FFT, P=P)
-    assert fa.fa_launch_count(pair.layout, 2) == 1 and fa.fa_launch_count(pair.layout, 3) == 2
+    assert fa.fa_launch_count(pair.layout, 2) == 1 and fa.fa_launch_count(pair.layout, 3) == 2      # one part per head: append kernel + fused decode
     pair.check_decode(synth.queries(shape, seed=23))
     K, V = stream.tokens(shape.L, shape.L + 2)
     for t in range(2):
