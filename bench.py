@@ -376,6 +376,15 @@ def run_ours(args):
         comp_ms.append(ev0.elapsed_time(ev1))
     n_mid0 = shape.L - shape.L_init - shape.L_local
     comp_flop = 2.0 * shape.M * n_mid0 * ((shape.d - shape.n_full_k) + (shape.d - shape.n_full_v)) * shape.Hkv * shape.B
+    # the same compression by per-class transforms (FA_COMPRESS_FFT: fp32, order-fixed) and with ordered sums on the tensor path
+    comp_fft_ms, comp_ord_ms = [], []
+    for _ in range(3):
+        ev0.record(); fa.fa_compress(layout, caches[-1], Kp, Vp, ws, flags=fa.FA_COMPRESS_FFT); ev1.record(); torch.cuda.synchronize()
+        comp_fft_ms.append(ev0.elapsed_time(ev1))
+        ev0.record(); fa.fa_compress(layout, caches[-1], Kp, Vp, ws, flags=fa.FA_COMPRESS_ORDERED); ev1.record(); torch.cuda.synchronize()
+        comp_ord_ms.append(ev0.elapsed_time(ev1))
+    fa.fa_compress(layout, caches[-1], Kp, Vp, ws)
+    prefill_bytes = 2.0 * shape.B * shape.L * shape.Hkv * shape.d * (2 if shape.dtype == "bf16" else 4)
     # dimension selection (Sec. 3.4) on the same prefill: all-dims compression + reconstruction error + ranking
     sel_ms = []
     for _ in range(3):
@@ -494,6 +503,9 @@ def run_ours(args):
                       "compress_frac_of_bf16_tflops": comp_flop / (min(comp_ms) * 1e-3) / 1e12 / bf16_peak,
                       "compress_tensor_pipe_pct": tensor_pct,
                       "compress_path": "tcgen05 bf16 x bf16 -> f32 (TMEM), basis tile generated in registers",
+                      "compress_fft_ms_per_layer": min(comp_fft_ms),
+                      "compress_fft_frac_of_hbm": prefill_bytes / (min(comp_fft_ms) * 1e-3) / 1e9 / _peaks()[0],
+                      "compress_ordered_ms_per_layer": min(comp_ord_ms),
                       "select_dims_ms": min(sel_ms), "select_dims_finds_generator_sets": sel_ok},
         "roofline": {"kernel": "fa_decode_attention (one fused cooperative kernel: u, token loop, merge)" if n_dec == 1 else
                      f"fa_decode_attention ({n_dec} kernels: u, token loop, merge)", "bound": "hbm",

@@ -155,6 +155,21 @@ fa_status fa_compress(const fa_layout* layout, fa_cache* cache, const void* K, c
                       int64_t stride_b, int64_t stride_t, int64_t stride_h, int32_t L,
                       void* ws, size_t ws_bytes, void* stream);
 
+/* fa_compress with a choice of how the coefficients of Eq.3 are evaluated (flags, OR-ed together; 0 is fa_compress):
+ *   FA_COMPRESS_ORDERED  the sums of Eq.3 are taken in a fixed order, so two calls on the same input give the
+ *                        same bits (the default splits the token axis over CTAs and adds the partial sums with
+ *                        floating-point atomics, whose order varies from run to run);
+ *   FA_COMPRESS_FFT      the coefficients are computed as the k lowest bins of the discrete Fourier transform of
+ *                        each zero-extended token column (Sec. 3.3, Eq.3-4 without forming F): one length
+ *                        period / mid_classes transform per residue class and column, fp32 throughout, always in a
+ *                        fixed order.  Needs a power-of-two period and mid_classes with n_coef / 2 <=
+ *                        period / mid_classes <= 2048; FA_ERR_UNSUPPORTED otherwise.
+ * Everything else (arguments, what is written, errors) as for fa_compress. */
+enum { FA_COMPRESS_ORDERED = 1, FA_COMPRESS_FFT = 2 };
+fa_status fa_compress_ex(const fa_layout* layout, fa_cache* cache, const void* K, const void* V, int64_t stride_b,
+                         int64_t stride_t, int64_t stride_h, int32_t L, uint32_t flags, void* ws, size_t ws_bytes,
+                         void* stream);
+
 /* fa_compress for a batch whose rows have different prompt lengths: row b is compressed from its
  * first lengths[b] tokens (HOST array of B entries, each 0 <= lengths[b] and within the capacity rule
  * of fa_compress; K / V rows beyond a row's length are not read).  Every row becomes what a one-row

@@ -366,14 +366,14 @@ fa_status fa_validate(const fa_layout* layout, const fa_cache* cache, void* stre
     return fa_poll_status(cache, stream);
 }
 
-fa_status fa_compress(const fa_layout* layout, fa_cache* cache, const void* K, const void* V, int64_t stride_b,
-                      int64_t stride_t, int64_t stride_h, int32_t L, void* ws, size_t ws_bytes, void* stream) {
+fa_status fa_compress_ex(const fa_layout* layout, fa_cache* cache, const void* K, const void* V, int64_t stride_b,
+                         int64_t stride_t, int64_t stride_h, int32_t L, uint32_t flags, void* ws, size_t ws_bytes, void* stream) {
     (void)ws; (void)ws_bytes;
     fa_status st = check_layout(layout);
     if (st != FA_OK) return st;
     st = check_cache(layout, cache);
     if (st != FA_OK) return st;
-    if (L < 0) return FA_ERR_INVALID_ARG;
+    if (L < 0 || (flags & ~(uint32_t)(FA_COMPRESS_ORDERED | FA_COMPRESS_FFT))) return FA_ERR_INVALID_ARG;
     if (L > 0 && (!K || !V || !aligned16(K) || !aligned16(V))) return FA_ERR_INVALID_ARG;
     if (L > 0 && (stride_t < layout->head_dim || stride_h < layout->head_dim || stride_b < 0)) return FA_ERR_INVALID_ARG;
     if ((stride_b | stride_t | stride_h) & 7) return FA_ERR_INVALID_ARG;
@@ -382,20 +382,42 @@ fa_status fa_compress(const fa_layout* layout, fa_cache* cache, const void* K, c
     int n_local = (L - n_init) < s.l_local ? (L - n_init) : s.l_local;
     if (L - n_init - n_local > s.max_mid) return FA_ERR_CAPACITY;
     cudaStream_t cs = static_cast<cudaStream_t>(stream);
+    const int64_t sbb = s.B > 1 ? stride_b : 0;
+    const bool ordered = (flags & FA_COMPRESS_ORDERED) != 0;
+    if (flags & FA_COMPRESS_FFT) {
+        // transform path: one store per coefficient, nothing to clear
+        int log2S = 0;
+        if (!compress_fft_supported(s, &log2S)) return FA_ERR_UNSUPPORTED;
+        if (launch_compress(s, make_cache(*cache), layout->kv_dtype, K, V, stride_b, stride_t, stride_h, L, false, true, cs) != cudaSuccess)
+            return FA_ERR_CUDA;
+        if (L > 0 && launch_compress_fft(s, make_cache(*cache), layout->kv_dtype, K, V, sbb, stride_t, stride_h, L, log2S, cs) != cudaSuccess)
+            return FA_ERR_CUDA;
+        if (L == 0) {
+            fa_cache_sizes sz0;
+            fa_cache_sizes_of(layout, &sz0);
+            if (sz0.coef_k && cudaMemsetAsync(cache->coef_k, 0, sz0.coef_k, cs) != cudaSuccess) return FA_ERR_CUDA;
+            if (sz0.coef_v && cudaMemsetAsync(cache->coef_v, 0, sz0.coef_v, cs) != cudaSuccess) return FA_ERR_CUDA;
+        }
+        return FA_OK;
+    }
     fa_cache_sizes sz;
     fa_cache_sizes_of(layout, &sz);
     if (sz.coef_k && cudaMemsetAsync(cache->coef_k, 0, sz.coef_k, cs) != cudaSuccess) return FA_ERR_CUDA;
     if (sz.coef_v && cudaMemsetAsync(cache->coef_v, 0, sz.coef_v, cs) != cudaSuccess) return FA_ERR_CUDA;
-    const int64_t sbb = s.B > 1 ? stride_b : 0;
     // The tensor-core path rounds the basis to bf16 (relative error 2^-9 per term); summed over n middle
     // tokens the coefficient error relative to the largest coefficient falls like 1 / sqrt(n): short
     // middles (where the tensor cores would idle anyway) take the fp32 kernel to stay within 1e-3.
     const int n_mid_host = L - n_init - n_local;
     const bool tc = L > 0 && n_mid_host >= 1024 && compress_tc_supported(s, layout->kv_dtype, sbb, stride_t, stride_h);
-    if (launch_compress(s, make_cache(*cache), layout->kv_dtype, K, V, stride_b, stride_t, stride_h, L, !tc, cs) != cudaSuccess)
+    if (launch_compress(s, make_cache(*cache), layout->kv_dtype, K, V, stride_b, stride_t, stride_h, L, !tc, ordered, cs) != cudaSuccess)
         return FA_ERR_CUDA;
-    if (tc && launch_compress_tc(s, make_cache(*cache), K, V, sbb, stride_t, stride_h, L, cs) != cudaSuccess) return FA_ERR_CUDA;
+    if (tc && launch_compress_tc(s, make_cache(*cache), K, V, sbb, stride_t, stride_h, L, ordered, cs) != cudaSuccess) return FA_ERR_CUDA;
     return FA_OK;
+}
+
+fa_status fa_compress(const fa_layout* layout, fa_cache* cache, const void* K, const void* V, int64_t stride_b,
+                      int64_t stride_t, int64_t stride_h, int32_t L, void* ws, size_t ws_bytes, void* stream) {
+    return fa_compress_ex(layout, cache, K, V, stride_b, stride_t, stride_h, L, 0u, ws, ws_bytes, stream);
 }
 
 fa_status fa_compress_ragged(const fa_layout* layout, fa_cache* cache, const void* K, const void* V, int64_t stride_b,

@@ -191,7 +191,7 @@ __global__ void __launch_bounds__(256) compress_coef_kernel(Dims s, CacheDev c, 
 
 template <typename KV>
 static cudaError_t launch_compress_t(const Dims& s, const CacheDev& c, const void* K, const void* V, int64_t sb,
-                                     int64_t st, int64_t sh, int L, bool with_coef, cudaStream_t stream) {
+                                     int64_t st, int64_t sh, int L, bool with_coef, bool ordered, cudaStream_t stream) {
     int chunks_rows = (L + kRowsPerCta - 1) / kRowsPerCta;
     if (chunks_rows < 1) chunks_rows = 1;
     constexpr int EPC = 16 / (int)sizeof(KV);
@@ -216,7 +216,7 @@ static cudaError_t launch_compress_t(const Dims& s, const CacheDev& c, const voi
     int ctas_fixed = row_tiles * s.B * s.Hkv * 2;
     int n_tsplit = (4 * sm_count() + ctas_fixed - 1) / ctas_fixed;
     if (n_tsplit > chunks) n_tsplit = chunks;
-    if (n_tsplit < 1) n_tsplit = 1;
+    if (n_tsplit < 1 || ordered) n_tsplit = 1;               // one split: every coefficient is added to zero exactly once
     int cps = (chunks + n_tsplit - 1) / n_tsplit;
     n_tsplit = (chunks + cps - 1) / cps;
     size_t smem = sizeof(float) * ((size_t)kTJ * max_comp + (size_t)kTJ * kTM);
@@ -229,9 +229,9 @@ static cudaError_t launch_compress_t(const Dims& s, const CacheDev& c, const voi
 
 // with_coef = false runs only the partition / gather kernel (the tensor-core path computes the coefficients).
 cudaError_t launch_compress(const Dims& s, const CacheDev& c, int dtype, const void* K, const void* V, int64_t sb,
-                            int64_t st, int64_t sh, int L, bool with_coef, cudaStream_t stream) {
-    if (dtype == FA_BF16) return launch_compress_t<__nv_bfloat16>(s, c, K, V, sb, st, sh, L, with_coef, stream);
-    return launch_compress_t<float>(s, c, K, V, sb, st, sh, L, with_coef, stream);
+                            int64_t st, int64_t sh, int L, bool with_coef, bool ordered, cudaStream_t stream) {
+    if (dtype == FA_BF16) return launch_compress_t<__nv_bfloat16>(s, c, K, V, sb, st, sh, L, with_coef, ordered, stream);
+    return launch_compress_t<float>(s, c, K, V, sb, st, sh, L, with_coef, ordered, stream);
 }
 
 }  // namespace fa

@@ -325,7 +325,7 @@ bool make_map(CUtensorMap* tm, const void* base, const Dims& s, int64_t sb, int6
 
 template <int D, int HP>
 cudaError_t launch_tc_t(const CUtensorMap& tmK, const CUtensorMap& tmV, const Dims& s, const CacheDev& c, int L, int n_mid,
-                        cudaStream_t stream) {
+                        bool ordered, cudaStream_t stream) {
     constexpr int N = 2 * D;
     constexpr size_t stage = (size_t)kBM * kBK * 2 + (size_t)HP * (N / 64) * kBK * 64 * 2;
     constexpr size_t n_stages = (200 * 1024) / stage < 4 ? (200 * 1024) / stage : 4;
@@ -337,7 +337,7 @@ cudaError_t launch_tc_t(const CUtensorMap& tmK, const CUtensorMap& tmV, const Di
     const int fixed = row_tiles * (s.Hkv / HP) * s.B;
     int n_tsplit = sm_count() / fixed;                          // one wave: one CTA per SM at most
     if (n_tsplit > nkb) n_tsplit = nkb;
-    if (n_tsplit < 1) n_tsplit = 1;
+    if (n_tsplit < 1 || ordered) n_tsplit = 1;                  // one split: every coefficient is added to zero exactly once
     compress_tc_kernel<D, HP><<<dim3(row_tiles, s.Hkv / HP, s.B * n_tsplit), kThreadsTc, smem, stream>>>(tmK, tmV, s, c, L, n_tsplit);
     return cudaGetLastError();
 }
@@ -357,7 +357,7 @@ bool compress_tc_supported(const Dims& s, int dtype, int64_t sb, int64_t st, int
 
 // Coefficients only (the caller has zeroed them and runs the partition / gather kernel itself).
 cudaError_t launch_compress_tc(const Dims& s, const CacheDev& c, const void* K, const void* V, int64_t sb, int64_t st,
-                               int64_t sh, int L, cudaStream_t stream) {
+                               int64_t sh, int L, bool ordered, cudaStream_t stream) {
     const int n_init = L < s.l_init ? L : s.l_init;
     const int n_local = (L - n_init) < s.l_local ? (L - n_init) : s.l_local;
     const int n_mid = L - n_init - n_local;
@@ -365,8 +365,8 @@ cudaError_t launch_compress_tc(const Dims& s, const CacheDev& c, const void* K, 
     CUtensorMap tmK, tmV;
     if (!make_map(&tmK, K, s, sb, st, sh, L) || !make_map(&tmV, V, s, sb, st, sh, L)) return cudaErrorInvalidValue;
     const bool pair = s.Hkv % 2 == 0;                        // two heads share a CTA and its basis tile
-    if (s.d == 128) return pair ? launch_tc_t<128, 2>(tmK, tmV, s, c, L, n_mid, stream) : launch_tc_t<128, 1>(tmK, tmV, s, c, L, n_mid, stream);
-    return pair ? launch_tc_t<64, 2>(tmK, tmV, s, c, L, n_mid, stream) : launch_tc_t<64, 1>(tmK, tmV, s, c, L, n_mid, stream);
+    if (s.d == 128) return pair ? launch_tc_t<128, 2>(tmK, tmV, s, c, L, n_mid, ordered, stream) : launch_tc_t<128, 1>(tmK, tmV, s, c, L, n_mid, ordered, stream);
+    return pair ? launch_tc_t<64, 2>(tmK, tmV, s, c, L, n_mid, ordered, stream) : launch_tc_t<64, 1>(tmK, tmV, s, c, L, n_mid, ordered, stream);
 }
 
 }  // namespace fa

@@ -21,6 +21,7 @@ FA_ERR_WORKSPACE, FA_ERR_CUDA, FA_ERR_TIMEOUT, FA_ERR_INDEX = 4, 5, 6, 7
 FA_F32, FA_BF16 = 0, 1
 FA_NORM_ORTHO, FA_NORM_PAPER = 0, 1
 FA_DECODE_AUTO, FA_DECODE_DIRECT, FA_DECODE_FFT, FA_DECODE_FFT_SPLIT = 0, 1, 2, 3
+FA_COMPRESS_ORDERED, FA_COMPRESS_FFT = 1, 2
 
 
 class fa_layout(C.Structure):
@@ -67,6 +68,8 @@ def lib() -> C.CDLL:
         L.fa_workspace_init.argtypes = [vp, sz, vp]
         L.fa_validate.argtypes = [lp, cp, vp]
         L.fa_compress.argtypes = [lp, cp, vp, vp, i64, i64, i64, i32, vp, sz, vp]
+        L.fa_compress_ex.argtypes = [lp, cp, vp, vp, i64, i64, i64, i32, C.c_uint32, vp, sz, vp]
+        L.fa_compress_ex.restype = C.c_int
         L.fa_append.argtypes = [lp, cp, vp, vp, vp]
         L.fa_compress_ragged.argtypes = [lp, cp, vp, vp, i64, i64, i64, C.POINTER(C.c_int32), vp, sz, vp]
         L.fa_decode_attention.argtypes = [lp, cp, vp, vp, vp, sz, vp]
@@ -220,14 +223,19 @@ def fa_validate(layout: Layout, cache: Cache, stream=None) -> None:
     _check(lib().fa_validate(C.byref(layout.c()), C.byref(cache.c()), _stream(stream)), "fa_validate")
 
 
-def fa_compress(layout: Layout, cache: Cache, K: torch.Tensor, V: torch.Tensor, ws: torch.Tensor, stream=None) -> None:
-    """K, V: [B][L][H_kv][d] (any strides with unit stride on d) in the layout's dtype."""
+def fa_compress(layout: Layout, cache: Cache, K: torch.Tensor, V: torch.Tensor, ws: torch.Tensor, stream=None, flags: int = 0) -> None:
+    """K, V: [B][L][H_kv][d] (any strides with unit stride on d) in the layout's dtype.
+    flags: 0, or FA_COMPRESS_ORDERED / FA_COMPRESS_FFT (fa_compress_ex)."""
     assert K.dtype == layout.torch_dtype and V.dtype == K.dtype and K.shape == V.shape and K.stride() == V.stride()
     assert K.is_cuda and V.is_cuda and (K.shape[1] == 0 or K.stride(3) == 1)
     L = K.shape[1]
     sb, st, sh = (K.stride(0), K.stride(1), K.stride(2)) if L > 0 else (0, layout.head_dim * layout.n_kv_heads, layout.head_dim)
     if K.shape[0] == 1:
         sb = 0
+    if flags:
+        _check(lib().fa_compress_ex(C.byref(layout.c()), C.byref(cache.c()), _ptr(K), _ptr(V), sb, st, sh, L, int(flags),
+                                    _ptr(ws), ws.numel(), _stream(stream)), "fa_compress_ex")
+        return
     _check(lib().fa_compress(C.byref(layout.c()), C.byref(cache.c()), _ptr(K), _ptr(V), sb, st, sh, L,
                              _ptr(ws), ws.numel(), _stream(stream)), "fa_compress")
 

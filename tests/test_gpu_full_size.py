@@ -170,3 +170,25 @@ def test_timed_entry_points_128k_batch4():
     shape = synth.CONFIGS[4]
     layout = layout_of(shape, max_mid=shape.T, P=shape.T // shape.k)
     _timed_entry_points_check(shape, layout, heads=(5,), seed=4001, rows=(3,), check_at=(0, 47))
+
+
+def test_compress_by_transform_32k_one_head():
+    """FA_COMPRESS_FFT on the 32K prefill of the headline configuration: coefficients of one KV head against the oracle."""
+    shape = synth.CONFIGS[1]
+    layout = layout_of(shape, max_mid=shape.T, P=shape.T // shape.k)
+    stream = synth.KVStream(shape, seed=1002, device="cuda")
+    K, V = stream.tokens(0, shape.L, work_dtype=torch.float32)
+    cache = fa.Cache(layout, stream.idx_full_k, stream.idx_full_v)
+    ws = fa.new_workspace(layout)
+    fa.fa_compress(layout, cache, K, V, ws, flags=fa.FA_COMPRESS_FFT)
+    torch.cuda.synchronize()
+    h = 3
+    sub = fo.OracleConfig(B=1, Hq=4, Hkv=1, d=shape.d, n_full_k=shape.n_full_k, n_full_v=shape.n_full_v, k=shape.k, T=shape.T,
+                          L_init=shape.L_init, L_local=shape.L_local, cap_mid=layout.max_mid, scale=1.0)
+    ref = fo.OracleCache(sub, stream.idx_full_k[h:h + 1].numpy(), stream.idx_full_v[h:h + 1].numpy())
+    ref.compress(to64(K[:, :, h:h + 1]), to64(V[:, :, h:h + 1]))
+    for name in ("coef_k", "coef_v"):
+        r = getattr(ref, name)[0, 0]
+        g = to64(getattr(cache, name)[0, h])
+        assert np.abs(g - r).max() / np.abs(r).max() <= 2e-5, name
+    assert fa.fa_poll_status(cache) == fa.FA_OK

@@ -553,3 +553,41 @@ def test_multi_layer_step_equals_single_calls_bit_for_bit():
         for name in ("k_init", "v_init", "k_local", "v_local", "k_mid", "v_mid", "coef_k", "coef_v", "state"):
             assert torch.equal(getattr(a, name), getattr(b, name)), (i, name)
     pair0.check_state()
+
+
+@pytest.mark.parametrize("shape,P", [(SMALL_BF16, 16), (SMALL_BF16.with_(L=2040, T=2048, M=256), 8), (CFG0, 32),
+                                      (CFG0.with_(L_init=4, L_local=64, L=700), 16)])
+def test_compress_by_transform_matches_oracle(shape, P):
+    """FA_COMPRESS_FFT: the coefficients as the lowest bins of per-class transforms (fp32, no rounded basis):
+    windows, kept dims and counters bit-exact as always, coefficients far inside the 1e-3 bar, and the decode
+    on top of them within the output tolerance."""
+    layout = layout_of(shape, max_mid=shape.T, P=P)
+    stream = synth.KVStream(shape, seed=51, freq="offgrid")
+    pair = Pair(layout, stream.idx_full_k, stream.idx_full_v)
+    K, V = stream.tokens(0, shape.L)
+    fa.fa_compress(layout, pair.gpu, K.cuda(), V.cuda(), pair.ws, flags=fa.FA_COMPRESS_FFT)
+    pair.ref.compress(to64(K), to64(V))
+    worst = pair.check_state()
+    assert worst <= 2e-5, worst
+    pair.check_decode(synth.queries(shape, seed=51))
+
+
+def test_ordered_compress_is_bit_reproducible():
+    """FA_COMPRESS_ORDERED (one token split) and FA_COMPRESS_FFT give the same bits on every call; both stay
+    within the coefficient tolerance of the oracle."""
+    shape = SMALL_BF16.with_(B=1, Hq=8, Hkv=2, L=3000, T=4096, M=256, n_full_k=32, n_full_v=32)
+    layout = layout_of(shape, max_mid=4096, P=16)
+    stream = synth.KVStream(shape, seed=52)
+    K, V = stream.tokens(0, shape.L)
+    Kc, Vc = K.cuda(), V.cuda()
+    for flags in (fa.FA_COMPRESS_ORDERED, fa.FA_COMPRESS_FFT, fa.FA_COMPRESS_ORDERED | fa.FA_COMPRESS_FFT):
+        pair = Pair(layout, stream.idx_full_k, stream.idx_full_v)
+        runs = []
+        for _ in range(3):
+            fa.fa_compress(layout, pair.gpu, Kc, Vc, pair.ws, flags=flags)
+            torch.cuda.synchronize()
+            runs.append((pair.gpu.coef_k.clone(), pair.gpu.coef_v.clone()))
+        for ck, cv in runs[1:]:
+            assert torch.equal(ck, runs[0][0]) and torch.equal(cv, runs[0][1]), flags
+        pair.ref.compress(to64(K), to64(V))
+        pair.check_state()
