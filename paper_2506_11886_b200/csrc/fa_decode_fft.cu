@@ -40,6 +40,19 @@
 #include "fa_decode_ws.cuh"
 #include "fa_tmap.cuh"
 
+#ifdef FA_TIMELINE
+// Timeline build (-DFA_TIMELINE): lane 0 of every consumer warp of the first and the last CTA of (batch row 0, KV
+// head 0) stamps the SM clock at the phase boundaries marked TL(i); fa_debug_timeline copies the stamps out.
+__device__ long long g_fa_timeline[2 * 8 * 32];
+#define TL(i) do { if ((threadIdx.x & 31) == 0 && threadIdx.x < 256 && blockIdx.y == 0 && blockIdx.z == 0 && (blockIdx.x == 0 || blockIdx.x == gridDim.x - 1)) \
+    g_fa_timeline[((blockIdx.x == 0 ? 0 : 1) * 8 + (threadIdx.x >> 5)) * 32 + (i)] = clock64(); } while (0)
+extern "C" int fa_debug_timeline(long long* host_out) {
+    return (int)cudaMemcpyFromSymbol(host_out, g_fa_timeline, sizeof(g_fa_timeline));
+}
+#else
+#define TL(i) do { } while (0)
+#endif
+
 namespace fa {
 namespace {
 
@@ -473,6 +486,7 @@ __global__ void __launch_bounds__(kThreads, OCC) decode_fft_kernel(const __grid_
     const int tid = threadIdx.x;
     const int log2P = 31 - __clz(s.P);
 
+    TL(0);
     // ---- one-time set-up, independent of the cache: it may overlap the tail of the previous kernel ----
     if (tid < kConsumers) {
         #pragma unroll 1
@@ -611,6 +625,7 @@ __global__ void __launch_bounds__(kThreads, OCC) decode_fft_kernel(const __grid_
     if (tid < 4) reinterpret_cast<uint32_t*>(zero16)[tid] = 0;
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     __syncthreads();
+    TL(1);
 
     // ============================ producer warp =================================
     if (tid >= kConsumers) {
@@ -861,10 +876,14 @@ __global__ void __launch_bounds__(kThreads, OCC) decode_fft_kernel(const __grid_
                         ws.u[((size_t)b * s.Hq + g_first + l8) * s.M + r] = recon_weight(s.norm, r, s.k, s.T) * sl2 * mine;
                 }
             }
+            TL(2);
             part_arrive(bar + 0, p.n_part, tid);
         }
+        TL(3);
         if (has_classes) k_phase(c0, min(NB, c1 - c0));
+        TL(4);
         if (s.dck > 0 && !is_win) part_wait(bar + 0, p.n_part, tid, fail, c.status);
+        TL(5);
     } else {
         if (has_classes) k_phase(c0, min(NB, c1 - c0));
         // everything above is independent of the prologue kernel; its output u is first needed here
@@ -965,6 +984,7 @@ __global__ void __launch_bounds__(kThreads, OCC) decode_fft_kernel(const __grid_
         __syncwarp();
     };
 
+    TL(6);
     // ------------------------------ window tokens -------------------------------
     if (w1 > w0) {
         uint32_t qw[4][2][2];
@@ -1129,6 +1149,7 @@ __global__ void __launch_bounds__(kThreads, OCC) decode_fft_kernel(const __grid_
     }
     consumer_sync();
 
+    TL(7);
     // ------------------------------ middle classes ------------------------------
     {
         float acc[4][4];                                  // [m-tile of 16 dims][mma D fragment]
@@ -1206,7 +1227,9 @@ __global__ void __launch_bounds__(kThreads, OCC) decode_fft_kernel(const __grid_
                     }
                 }
                 consumer_sync();
+                if (cb == c0) TL(8);
                 fft_run<GH, LS, LS, false>(fbuf, fb_floats, nb, twf, tid);        // score of slot a at point rev[a]
+                if (cb == c0) TL(9);
             } else {
                 #pragma unroll 1
                 for (int i = tid; i < nb * fb_floats; i += kConsumers) fbuf[i] = 0.f;
@@ -1274,6 +1297,7 @@ __global__ void __launch_bounds__(kThreads, OCC) decode_fft_kernel(const __grid_
             }
             consumer_sync();
 
+            if (cb == c0) TL(10);
             // o^u[dim][slot] += V^mu^T p, 16 tokens per mma
             if (ts_v) {
                 #pragma unroll 1
@@ -1314,9 +1338,11 @@ __global__ void __launch_bounds__(kThreads, OCC) decode_fft_kernel(const __grid_
                 }
             }
 
+            if (cb == c0) TL(11);
             // z_n = alpha z_n + sum_c e^{i theta n c} Y^c_n, Y^c = transform of the packed probabilities
             if (s.dcv > 0) {
                 fft_run<GH, LS, LS, true>(fbuf, fb_floats, nb, twf, tid);
+                if (cb == c0) TL(12);
                 PR<N> alA, alB;
                 if constexpr (N == 2) { alA = pk(alpha[0], alpha[1]); alB = pk(alpha[2], alpha[3]); }
                 else { alA = PR<1>{alpha[0]}; alB = PR<1>{alpha[1]}; }
@@ -1378,6 +1404,7 @@ __global__ void __launch_bounds__(kThreads, OCC) decode_fft_kernel(const __grid_
             }
             consumer_sync();
         }
+        TL(13);
         // fold the per-warp output fragments into o_s at the natural positions of D^vu
         if (2 * tq < GH) {
             long long* o_lo = o_s + hperm<GH>(2 * tq) * s.d;
@@ -1406,6 +1433,7 @@ __global__ void __launch_bounds__(kThreads, OCC) decode_fft_kernel(const __grid_
     }
     consumer_sync();
 
+    TL(14);
     // ------------------------------ partial results ------------------------------
     for (int i = tid; i < GH * s.d; i += kConsumers) {
         const int g = i / s.d, e = i - g * s.d;
@@ -1433,6 +1461,7 @@ __global__ void __launch_bounds__(kThreads, OCC) decode_fft_kernel(const __grid_
             ml[1] = red_s[kWarps * GH + tid];
         }
     }
+    TL(15);
     if (!p.fused) return;
 
     // ------------------------------ merge (fused kernel) ------------------------------
@@ -1467,7 +1496,9 @@ __global__ void __launch_bounds__(kThreads, OCC) decode_fft_kernel(const __grid_
 
     if (s.dcv > 0) stage_cv(0, min(rows, mch));            // under the barrier
     part_arrive(bar + 1, np, tid);
+    TL(16);
     part_wait(bar + 1, np, tid, fail, c.status);
+    TL(17);
     // Fused step: every part of this (b, KV head) has read the row that leaves the window and is past its token
     // loop, so the rows the push moves can be written to the cache now, each by the part that owns it.
     if (step && !cap_full) {
@@ -1590,6 +1621,7 @@ __global__ void __launch_bounds__(kThreads, OCC) decode_fft_kernel(const __grid_
             if (g < ng) ws.oc[((qh0 + g) * np + part) * s.dcv + e] = v;
         }
     }
+    TL(18);
     // ticket: the last part to get here finishes the rows
     consumer_sync();
     if (tid == 0) {
@@ -1601,6 +1633,7 @@ __global__ void __launch_bounds__(kThreads, OCC) decode_fft_kernel(const __grid_
         *last_s = old == np - 1;
     }
     consumer_sync();
+    TL(19);
     if (!*last_s) return;
     float* op_s = zw_s;                                    // [GH][np][d] (the slice buffers are free again)
     float* ocp_s = op_s + GH * np * s.d;                   // [GH][np][dcv]
@@ -1639,6 +1672,7 @@ __global__ void __launch_bounds__(kThreads, OCC) decode_fft_kernel(const __grid_
         }
         out[(qh0 + g) * s.d + e] = __float2bfloat16_rn(v * linv_s[g]);
     }
+    TL(20);
     if (tid == 0 && np > 1) { bar[0] = 0; bar[1] = 0; bar[2] = 0; }   // the counters are zero again for the next call
     // Fused step: the last (KV head, pass) of this batch row to finish publishes the counters after the push
     // (the others read the old ones when they started; the next kernel in the stream sees the new ones).
