@@ -250,6 +250,9 @@ size_t fa_step_staging_bytes(const fa_layout* layout);
  *   mse: optional DEVICE output [B][H_kv][2][d] (side 0 = K, 1 = V), the per-row mean squared errors.
  *   ws / ws_bytes: scratch of fa_select_workspace_bytes(layout) bytes, 256-byte aligned (it holds the
  *     coefficients of all dimensions).  head_dim must be 64, 128 or 256.
+ * For bf16 tensors (head_dim 64 or 128, n_coef a multiple of 64, 16-byte aligned bases and strides) the
+ * reconstruction runs on the tensor cores with the basis and the weighted coefficients rounded to bf16: a
+ * dimension that its coefficients rebuild exactly still reports an error of about 1e-6 of its mean square.
  * Asynchronous on `stream`.  An empty middle gives zero errors (the lowest indices are compressed). */
 fa_status fa_select_workspace_bytes(const fa_layout* layout, size_t* out);
 fa_status fa_select_dims(const fa_layout* layout, const void* K, const void* V, int64_t stride_b, int64_t stride_t,

@@ -103,6 +103,12 @@ fa_status check_layout(const fa_layout* l);
 cudaError_t launch_validate(const Dims&, const CacheDev&, cudaStream_t);
 cudaError_t launch_compress(const Dims&, const CacheDev&, int dtype, const void* K, const void* V, int64_t sb,
                             int64_t st, int64_t sh, int L, bool with_coef, bool ordered, cudaStream_t);
+// Tensor-core reconstruction of the dimension selection (fa_select_tc.cu).
+bool reconstruct_tc_supported(const Dims& s, int dtype, const void* K, const void* V, int64_t sb, int64_t st, int64_t sh, int n_mid);
+size_t reconstruct_tc_scratch_bytes(const Dims& s);
+cudaError_t launch_reconstruct_tc(const Dims& s, const float* coef_k, const float* coef_v, const void* K, const void* V, int64_t sb,
+                                  int64_t st, int64_t sh, int n_init, int n_mid, float* sq, int32_t* status, void* scratch,
+                                  cudaStream_t stream);
 bool compress_fft_supported(const Dims&, int* log2S);
 cudaError_t launch_compress_fft(const Dims&, const CacheDev&, int dtype, const void* K, const void* V, int64_t sb, int64_t st,
                                 int64_t sh, int L, int log2S, cudaStream_t);

@@ -3,8 +3,9 @@
 // (Eq.6 weights); the dimensions with the largest mean squared reconstruction error are kept.
 //   1. coefficients of all d dims: fa_compress on a scratch cache whose layout compresses everything
 //      (the tensor-core kernel already multiplies all dims), carved from the workspace;
-//   2. mse_kernel: x~[j][e] = sum_m w_m F[m][j] C[m][e] for 64 middle tokens per CTA, basis by rotation
-//      recurrence re-seeded exactly every 16 frequencies, squared error summed per dim;
+//   2. the middle tokens rebuilt, x~[j][e] = sum_m w_m F[m][j] C[m][e], and the squared error summed per dim:
+//      for bf16 tensors on the tensor cores (reconstruct_tc_kernel, fa_select_tc.cu), otherwise mse_kernel
+//      (fp32, 64 middle tokens per CTA, basis by rotation recurrence re-seeded exactly every 16 frequencies);
 //   3. select_kernel: mean over the batch rows, rank by (error, index), write the sorted index sets.
 #include <cstring>
 
@@ -125,6 +126,7 @@ struct Scratch {
     fa_layout layout;
     fa_cache cache;
     float* sq;
+    char* wc16;                 // weighted coefficients in bf16, the B operand of the tensor-core reconstruction
     char* ws_compress;
     size_t ws_compress_bytes;
     size_t total;
@@ -153,6 +155,7 @@ fa_status plan_scratch(const fa_layout& l, char* base, Scratch* out) {
     sc.cache.state = reinterpret_cast<int32_t*>(take(sz.state));
     sc.cache.status = reinterpret_cast<int32_t*>(take(sz.status));
     sc.sq = reinterpret_cast<float*>(take(sizeof(float) * (size_t)l.batch * l.n_kv_heads * 2 * l.head_dim));
+    sc.wc16 = take(reconstruct_tc_scratch_bytes(make_dims(l)));
     size_t wsb = 0;
     st = fa_workspace_bytes(&sc.layout, &wsb);
     if (st != FA_OK) return st;
@@ -226,7 +229,11 @@ fa_status fa_select_dims(const fa_layout* layout, const void* K, const void* V, 
     const int n_mid = L - n_init - n_local;
     const size_t sq_bytes = sizeof(float) * (size_t)s.B * s.Hkv * 2 * s.d;
     if (cudaMemsetAsync(sc.sq, 0, sq_bytes, cs) != cudaSuccess) return FA_ERR_CUDA;
-    if (n_mid > 0) {
+    if (n_mid > 0 && reconstruct_tc_supported(s, layout->kv_dtype, K, V, stride_b, stride_t, stride_h, n_mid)) {
+        if (launch_reconstruct_tc(s, sc.cache.coef_k, sc.cache.coef_v, K, V, stride_b, stride_t, stride_h, n_init, n_mid, sc.sq,
+                                  sc.cache.status, sc.wc16, cs) != cudaSuccess)
+            return FA_ERR_CUDA;
+    } else if (n_mid > 0) {
         cudaError_t err = layout->kv_dtype == FA_BF16
                               ? launch_mse<__nv_bfloat16>(s, sc.cache, K, V, stride_b, stride_t, stride_h, n_init, n_mid, sc.sq, cs)
                               : launch_mse<float>(s, sc.cache, K, V, stride_b, stride_t, stride_h, n_init, n_mid, sc.sq, cs);

@@ -53,6 +53,32 @@ def test_select_dims_matches_oracle(dtype, d, L):
     assert (np.abs(g_mse - want_mse) <= 2e-2 * scale + 1e-6).all()
 
 
+@pytest.mark.parametrize("Hkv,d,M,L", [(3, 128, 256, 1500), (4, 64, 512, 2000), (2, 128, 128, 129 + 36)])
+def test_tensor_core_reconstruction_against_oracle_and_fp32_path(Hkv, d, M, L):
+    """bf16 prefill tensors take the tcgen05 reconstruction (several pipeline rounds, a ragged last token tile,
+    one or two heads per CTA); the same values handed over as fp32 take the fp32 kernel: both against the oracle."""
+    shape = synth.Shape("selt", B=2, layers=1, Hq=Hkv, Hkv=Hkv, d=d, L=L, dtype="bf16", n_full_k=d // 4, n_full_v=d // 2,
+                        M=M, T=2048, L_init=4, L_local=32)
+    layout = layout_of(shape, max_mid=2048, P=16)
+    stream = synth.KVStream(shape, seed=23)
+    K, V = stream.tokens(0, L)
+    got = fa.fa_select_dims(layout, K.cuda().contiguous(), V.cuda().contiguous())
+    shape32 = shape.with_(dtype="f32")
+    layout32 = layout_of(shape32, max_mid=2048, P=16)
+    got32 = fa.fa_select_dims(layout32, K.float().cuda().contiguous(), V.float().cuda().contiguous())
+    torch.cuda.synchronize()
+    want_sets, want_mse = _oracle_selection(layout, K, V)
+    for g, g32, w in zip(got[:4], got32[:4], want_sets):
+        np.testing.assert_array_equal(g.cpu().numpy(), w)
+        np.testing.assert_array_equal(g32.cpu().numpy(), w)
+    scale = want_mse.max(axis=-1, keepdims=True)
+    for g_mse in (to64(got[4]), to64(got32[4])):
+        assert (np.abs(g_mse - want_mse) <= 2e-2 * scale + 1e-6).all()
+    # the noise dims (errors of the order of the signal) agree closely between the two paths
+    big = want_mse > 0.1 * scale
+    np.testing.assert_allclose(to64(got[4])[big], to64(got32[4])[big], rtol=5e-3)
+
+
 def test_select_dims_empty_middle_and_workspace_check():
     shape = synth.Shape("sel0", B=1, layers=1, Hq=2, Hkv=2, d=64, L=20, dtype="bf16", n_full_k=16, n_full_v=8, M=16,
                         T=256, L_init=4, L_local=32)
