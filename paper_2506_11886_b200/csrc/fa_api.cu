@@ -388,7 +388,7 @@ fa_status fa_compress_ex(const fa_layout* layout, fa_cache* cache, const void* K
         // transform path: one store per coefficient, nothing to clear
         int log2S = 0;
         if (!compress_fft_supported(s, &log2S)) return FA_ERR_UNSUPPORTED;
-        if (launch_compress(s, make_cache(*cache), layout->kv_dtype, K, V, stride_b, stride_t, stride_h, L, false, true, cs) != cudaSuccess)
+        if (launch_compress(s, make_cache(*cache), layout->kv_dtype, K, V, stride_b, stride_t, stride_h, L, false, true, true, cs) != cudaSuccess)
             return FA_ERR_CUDA;
         if (L > 0 && launch_compress_fft(s, make_cache(*cache), layout->kv_dtype, K, V, sbb, stride_t, stride_h, L, log2S, cs) != cudaSuccess)
             return FA_ERR_CUDA;
@@ -409,9 +409,12 @@ fa_status fa_compress_ex(const fa_layout* layout, fa_cache* cache, const void* K
     // middles (where the tensor cores would idle anyway) take the fp32 kernel to stay within 1e-3.
     const int n_mid_host = L - n_init - n_local;
     const bool tc = L > 0 && n_mid_host >= 1024 && compress_tc_supported(s, layout->kv_dtype, sbb, stride_t, stride_h);
-    if (launch_compress(s, make_cache(*cache), layout->kv_dtype, K, V, stride_b, stride_t, stride_h, L, !tc, ordered, cs) != cudaSuccess)
+    // tensor-core path: its kernel also writes the kept-dim rows of the middle from the boxes it loads; the partition
+    // kernel is left with the windows and the counters
+    const bool tc_rows = tc && compress_tc_gathers(s);
+    if (launch_compress(s, make_cache(*cache), layout->kv_dtype, K, V, stride_b, stride_t, stride_h, L, !tc, ordered, !tc_rows, cs) != cudaSuccess)
         return FA_ERR_CUDA;
-    if (tc && launch_compress_tc(s, make_cache(*cache), K, V, sbb, stride_t, stride_h, L, ordered, cs) != cudaSuccess) return FA_ERR_CUDA;
+    if (tc && launch_compress_tc(s, make_cache(*cache), K, V, sbb, stride_t, stride_h, L, ordered, tc_rows, cs) != cudaSuccess) return FA_ERR_CUDA;
     return FA_OK;
 }
 

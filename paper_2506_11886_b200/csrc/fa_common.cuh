@@ -102,7 +102,8 @@ fa_status check_layout(const fa_layout* l);
 // Kernel launchers (defined next to their kernels).  All return the launch error, if any.
 cudaError_t launch_validate(const Dims&, const CacheDev&, cudaStream_t);
 cudaError_t launch_compress(const Dims&, const CacheDev&, int dtype, const void* K, const void* V, int64_t sb,
-                            int64_t st, int64_t sh, int L, bool with_coef, bool ordered, cudaStream_t);
+                            int64_t st, int64_t sh, int L, bool with_coef, bool ordered, bool mid_rows, cudaStream_t);
+bool compress_tc_gathers(const Dims& s);
 // Tensor-core reconstruction of the dimension selection (fa_select_tc.cu).
 bool reconstruct_tc_supported(const Dims& s, int dtype, const void* K, const void* V, int64_t sb, int64_t st, int64_t sh, int n_mid);
 size_t reconstruct_tc_scratch_bytes(const Dims& s);
@@ -114,7 +115,7 @@ cudaError_t launch_compress_fft(const Dims&, const CacheDev&, int dtype, const v
                                 int64_t sh, int L, int log2S, cudaStream_t);
 bool compress_tc_supported(const Dims&, int dtype, int64_t sb, int64_t st, int64_t sh);
 cudaError_t launch_compress_tc(const Dims&, const CacheDev&, const void* K, const void* V, int64_t sb, int64_t st, int64_t sh,
-                               int L, bool ordered, cudaStream_t);
+                               int L, bool ordered, bool gather, cudaStream_t);
 cudaError_t launch_append(const Dims&, const CacheDev&, int dtype, const void* k_new, const void* v_new, cudaStream_t);
 cudaError_t launch_decode_prologue(const Dims&, const CacheDev&, int dtype, const DecodePlan&, const void* q, char* ws,
                                    cudaStream_t);

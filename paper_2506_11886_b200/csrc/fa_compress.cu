@@ -51,7 +51,7 @@ constexpr int kRowsPerCta = 64;
 template <typename KV>
 __global__ void __launch_bounds__(256) partition_gather_kernel(Dims s, CacheDev c, const KV* __restrict__ K,
                                                                    const KV* __restrict__ V, int64_t sb, int64_t st,
-                                                                   int64_t sh, int L) {
+                                                                   int64_t sh, int L, int mid_rows, int skip_a, int skip_c) {
     constexpr int EPC = 16 / (int)sizeof(KV);            // elements per chunk
     extern __shared__ __align__(16) unsigned char gsm[];
     KV* rows_s = reinterpret_cast<KV*>(gsm);                                         // [64][d]
@@ -73,7 +73,9 @@ __global__ void __launch_bounds__(256) partition_gather_kernel(Dims s, CacheDev 
     void* w_init = side == 0 ? c.k_init : c.v_init;
     void* w_local = side == 0 ? c.k_local : c.v_local;
     void* w_mid = side == 0 ? c.k_mid : c.v_mid;
-    const int t0 = blockIdx.x * kRowsPerCta, nrow = min(L - t0, kRowsPerCta);
+    // without the kept-dim rows (the tensor-core kernel writes them) the chunks [skip_a, skip_c) of middle tokens only are not launched
+    const int chunk = (int)blockIdx.x < skip_a ? (int)blockIdx.x : (int)blockIdx.x + (skip_c - skip_a);
+    const int t0 = chunk * kRowsPerCta, nrow = min(L - t0, kRowsPerCta);
     const int cpr = s.d / EPC;                            // chunks per input row
     for (int i = threadIdx.x; i < nfull; i += blockDim.x) idf_s[i] = idf[i];
     for (int i = threadIdx.x; i < nrow * cpr; i += blockDim.x) {
@@ -90,6 +92,7 @@ __global__ void __launch_bounds__(256) partition_gather_kernel(Dims s, CacheDev 
         if (dst) reinterpret_cast<uint4*>(dst)[ch] = reinterpret_cast<const uint4*>(rows_s)[i];
     }
     // kept-dim rows of the middle
+    if (!mid_rows) return;
     const int cpo = nfull / EPC;                          // chunks per output row
     for (int i = threadIdx.x; i < nrow * cpo; i += blockDim.x) {
         const int r = i / cpo, ch = i - r * cpo, t = t0 + r;
@@ -191,9 +194,17 @@ __global__ void __launch_bounds__(256) compress_coef_kernel(Dims s, CacheDev c, 
 
 template <typename KV>
 static cudaError_t launch_compress_t(const Dims& s, const CacheDev& c, const void* K, const void* V, int64_t sb,
-                                     int64_t st, int64_t sh, int L, bool with_coef, bool ordered, cudaStream_t stream) {
+                                     int64_t st, int64_t sh, int L, bool with_coef, bool ordered, bool mid_rows, cudaStream_t stream) {
     int chunks_rows = (L + kRowsPerCta - 1) / kRowsPerCta;
     if (chunks_rows < 1) chunks_rows = 1;
+    int skip_a = 0, skip_c = 0;
+    if (!mid_rows) {
+        const int ni = L < s.l_init ? L : s.l_init, nl = (L - ni) < s.l_local ? (L - ni) : s.l_local;
+        skip_a = (ni + kRowsPerCta - 1) / kRowsPerCta;          // first chunk past the initial window
+        skip_c = (L - nl) / kRowsPerCta;                        // first chunk with a token of the local window
+        if (skip_a < 1) skip_a = 1;                             // chunk 0 always runs: it writes the counters
+        if (skip_c < skip_a) skip_c = skip_a;
+    }
     constexpr int EPC = 16 / (int)sizeof(KV);
     if (s.d % EPC || s.nfk % EPC || s.nfv % EPC || sb % EPC || st % EPC || sh % EPC || (reinterpret_cast<uintptr_t>(K) & 15) ||
         (reinterpret_cast<uintptr_t>(V) & 15))
@@ -202,8 +213,8 @@ static cudaError_t launch_compress_t(const Dims& s, const CacheDev& c, const voi
     const size_t gsmem = (size_t)kRowsPerCta * s.d * sizeof(KV) + sizeof(int32_t) * (size_t)nf;
     cudaError_t err = ensure_dynamic_smem(partition_gather_kernel<KV>, gsmem);
     if (err != cudaSuccess) return err;
-    partition_gather_kernel<KV><<<dim3(chunks_rows, s.Hkv, s.B * 2), 256, gsmem, stream>>>(
-        s, c, static_cast<const KV*>(K), static_cast<const KV*>(V), sb, st, sh, L);
+    partition_gather_kernel<KV><<<dim3(chunks_rows - (skip_c - skip_a), s.Hkv, s.B * 2), 256, gsmem, stream>>>(
+        s, c, static_cast<const KV*>(K), static_cast<const KV*>(V), sb, st, sh, L, mid_rows ? 1 : 0, skip_a, skip_c);
     err = cudaGetLastError();
     if (err != cudaSuccess) return err;
     int n_init = L < s.l_init ? L : s.l_init;
@@ -227,11 +238,12 @@ static cudaError_t launch_compress_t(const Dims& s, const CacheDev& c, const voi
     return cudaGetLastError();
 }
 
-// with_coef = false runs only the partition / gather kernel (the tensor-core path computes the coefficients).
+// with_coef = false runs only the partition / gather kernel (the tensor-core or the transform path computes the
+// coefficients); mid_rows = false leaves the kept-dim rows of the middle out too (windows and counters only).
 cudaError_t launch_compress(const Dims& s, const CacheDev& c, int dtype, const void* K, const void* V, int64_t sb,
-                            int64_t st, int64_t sh, int L, bool with_coef, bool ordered, cudaStream_t stream) {
-    if (dtype == FA_BF16) return launch_compress_t<__nv_bfloat16>(s, c, K, V, sb, st, sh, L, with_coef, ordered, stream);
-    return launch_compress_t<float>(s, c, K, V, sb, st, sh, L, with_coef, ordered, stream);
+                            int64_t st, int64_t sh, int L, bool with_coef, bool ordered, bool mid_rows, cudaStream_t stream) {
+    if (dtype == FA_BF16) return launch_compress_t<__nv_bfloat16>(s, c, K, V, sb, st, sh, L, with_coef, ordered, mid_rows, stream);
+    return launch_compress_t<float>(s, c, K, V, sb, st, sh, L, with_coef, ordered, mid_rows, stream);
 }
 
 }  // namespace fa

@@ -14,7 +14,10 @@
 //   * warps 2-9 generate the 128 x 64 basis tile in registers (integer phase for the first
 //     two tokens of a thread's run, then packed fp32-pair rotations by two tokens), round it to bf16 and store it in the
 //     K-major 128-byte-swizzled layout the tensor core reads: the A operand never exists in HBM;
-//   * warp 1 (one lane) issues four tcgen05.mma (K = 16 each) and commits the stage back.
+//   * warp 1 (one lane) issues four tcgen05.mma (K = 16 each) and commits the stage back;
+//   * warps 10-13 copy the kept dims of the stage's tokens from the K and V boxes to K^mu / V^mu (Eq.2): the
+//     row-tile CTAs that share a box take every row_tiles-th token each, so the prefill is read from HBM once
+//     for the coefficients and the kept-dim rows together.
 // At the end warps 2-9 read the accumulators from tensor memory and scatter the compressed
 // columns.  Every wait is bounded; tensor memory is freed on every path.
 #include "fa_umma.cuh"
@@ -26,7 +29,9 @@ using bf16 = __nv_bfloat16;
 constexpr int kBM = 128;          // coefficient rows per CTA
 constexpr int kBK = 64;           // tokens per pipeline stage
 constexpr int kGenWarps = 8;       // basis generators (and epilogue): 16 tokens of two rows per thread and stage
-constexpr int kThreadsTc = 64 + 32 * kGenWarps;
+constexpr int kGatherWarps = 4;    // kept-dim rows of the middle, from the B boxes
+constexpr int kGatherItems = 4;    // 16-byte chunks per gather thread and stage, at most
+constexpr int kThreadsTc = 64 + 32 * (kGenWarps + kGatherWarps);
 using namespace umma;
 
 // D = head dim (64 or 128): N = 2 D accumulator columns per KV head; HP heads share one CTA and one
@@ -34,7 +39,7 @@ using namespace umma;
 template <int D, int HP>
 __global__ void __launch_bounds__(kThreadsTc, 1) compress_tc_kernel(const __grid_constant__ CUtensorMap tmK,
                                                                     const __grid_constant__ CUtensorMap tmV, Dims s,
-                                                                    CacheDev c, int L, int n_tsplit) {
+                                                                    CacheDev c, int L, int n_tsplit, int gather) {
     constexpr int N = 2 * D;
     constexpr int kABytes = kBM * kBK * 2;                 // 16 KB basis tile
     constexpr int kBoxBytes = kBK * 64 * 2;                // 8 KB per [64 tokens x 64 dims] box
@@ -51,9 +56,11 @@ __global__ void __launch_bounds__(kThreadsTc, 1) compress_tc_kernel(const __grid
     uint64_t* fullB = fullA + kStagesTc;
     uint64_t* empty = fullB + kStagesTc;
     uint64_t* acc_ready = empty + kStagesTc;
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_ready + 1);
+    uint64_t* gather_done = acc_ready + 1;                 // the gather warps are past their last box
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(gather_done + 1);
     volatile int* fail = reinterpret_cast<volatile int*>(tmem_slot + 1);
     int* inv = reinterpret_cast<int*>(tmem_slot + 4);      // [HP][2][D]: dim -> slot in D^kc / D^vc, or -1
+    int* idf_s = inv + HP * 2 * D;                         // [HP][2][D]: the kept dims D^ku / D^vu of the CTA's heads
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int mt = blockIdx.x, h0 = blockIdx.y * HP;
@@ -66,8 +73,10 @@ __global__ void __launch_bounds__(kThreadsTc, 1) compress_tc_kernel(const __grid
     const int kb0 = split * per, kb1 = min(nkb, kb0 + per);
 
     if (tid == 0) {
-        for (int i = 0; i < kStagesTc; ++i) { mbar_init(fullA + i, kGenWarps); mbar_init(fullB + i, 1); mbar_init(empty + i, 1); }
+        // a stage is free again when its MMAs have read it and the gather warps have taken their rows
+        for (int i = 0; i < kStagesTc; ++i) { mbar_init(fullA + i, kGenWarps); mbar_init(fullB + i, 1); mbar_init(empty + i, 1 + kGatherWarps); }
         mbar_init(acc_ready, 1);
+        mbar_init(gather_done, kGatherWarps);
         *fail = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -78,6 +87,12 @@ __global__ void __launch_bounds__(kThreadsTc, 1) compress_tc_kernel(const __grid
         if (r < s.dck) inv[hh * N + c.idx_comp_k[(size_t)(h0 + hh) * s.dck + r]] = r;
         else inv[hh * N + D + c.idx_comp_v[(size_t)(h0 + hh) * s.dcv + (r - s.dck)]] = r - s.dck;
     }
+    if (gather)
+        for (int i = tid; i < HP * (s.nfk + s.nfv); i += kThreadsTc) {
+            const int hh = i / (s.nfk + s.nfv), r = i - hh * (s.nfk + s.nfv);
+            if (r < s.nfk) idf_s[hh * N + r] = c.idx_full_k[(size_t)(h0 + hh) * s.nfk + r];
+            else idf_s[hh * N + D + (r - s.nfk)] = c.idx_full_v[(size_t)(h0 + hh) * s.nfv + (r - s.nfk)];
+        }
     if (warp == 1) {                                       // tensor memory: N fp32 columns x 128 lanes
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(kTmemCols) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
@@ -132,6 +147,80 @@ __global__ void __launch_bounds__(kThreadsTc, 1) compress_tc_kernel(const __grid
                 }
                 umma_commit(acc_ready);
             }
+        } else if (warp >= 2 + kGenWarps) {
+            // ---------------- kept dims of the middle tokens: B boxes -> K^mu / V^mu ----------------
+            const int gt = tid - 32 * (2 + kGenWarps);           // 0 .. 32 kGatherWarps - 1
+            const int row_tiles = gridDim.x;
+            const int cpk = s.nfk >> 3, cpv = s.nfv >> 3, cph = cpk + cpv;   // 16-byte chunks per kept-dim row
+            const int n_tok = mt < kBK ? (kBK - mt + row_tiles - 1) / row_tiles : 0;   // tokens mt, mt + row_tiles, ... of a block
+            const int n_items = gather ? n_tok * HP * cph : 0;                // <= kGatherItems per thread (checked on the host)
+            // An item = one 16-byte chunk (8 kept dims) of one kept-dim row.  A thread keeps the same items in every
+            // block: token row r of the boxes, head, side and LOGICAL chunk, so the eight source offsets inside a stage
+            // are constants (two 16-bit offsets per register); only the destination row moves with the token.
+            uint32_t src[kGatherItems][4];
+            int meta[kGatherItems];                        // r | hh << 8 | side << 12 | lch << 16, or -1
+#pragma unroll
+            for (int u = 0; u < kGatherItems; ++u) {
+                const int idx = gt + u * 32 * kGatherWarps;
+                meta[u] = -1;
+#pragma unroll
+                for (int i2 = 0; i2 < 4; ++i2) src[u][i2] = 0;
+                if (idx < n_items) {
+                    const int ti = idx / (HP * cph), rem = idx - ti * (HP * cph);
+                    const int hh = rem / cph, cc = rem - hh * cph;
+                    const int side = cc >= cpk, lch = side ? cc - cpk : cc;
+                    const int r = mt + row_tiles * ti;
+                    const int* idf = idf_s + hh * N + side * D + lch * 8;
+                    const uint32_t row0 = (uint32_t)(hh * kBBytes1 + side * (D / 64) * kBoxBytes + r * 128);
+#pragma unroll
+                    for (int i2 = 0; i2 < 4; ++i2) {
+                        const int e0 = idf[2 * i2], e1 = idf[2 * i2 + 1];
+                        const uint32_t o0 = row0 + (uint32_t)((e0 >> 6) * kBoxBytes + ((((e0 & 63) >> 3) ^ (r & 7)) << 4) + (e0 & 7) * 2);
+                        const uint32_t o1 = row0 + (uint32_t)((e1 >> 6) * kBoxBytes + ((((e1 & 63) >> 3) ^ (r & 7)) << 4) + (e1 & 7) * 2);
+                        src[u][i2] = o0 | (o1 << 16);       // a stage is at most 64 KB
+                    }
+                    meta[u] = r | (hh << 8) | (side << 12) | (lch << 16);
+                }
+            }
+            const bool p2 = (s.P & (s.P - 1)) == 0;
+            const int lgP = 31 - __clz(s.P);
+            for (int kb = kb0; kb < kb1; ++kb) {
+                const int it = kb - kb0, st = it % kStagesTc;
+                if (!mbar_wait(fullB + st, (it / kStagesTc) & 1, fail, c.status)) break;
+                const unsigned char* bsrc = stage0 + (size_t)st * kStageBytesTc + kABytes;
+                const int jb = kb * kBK;                   // first middle token of the block
+                uint4 val[kGatherItems];
+#pragma unroll
+                for (int u = 0; u < kGatherItems; ++u) {
+                    uint32_t w[4] = {0u, 0u, 0u, 0u};
+                    if (meta[u] >= 0) {
+#pragma unroll
+                        for (int i2 = 0; i2 < 4; ++i2) {
+                            const uint32_t lo = *reinterpret_cast<const uint16_t*>(bsrc + (src[u][i2] & 0xffffu));
+                            const uint32_t hi = *reinterpret_cast<const uint16_t*>(bsrc + (src[u][i2] >> 16));
+                            w[i2] = lo | (hi << 16);
+                        }
+                    }
+                    val[u] = make_uint4(w[0], w[1], w[2], w[3]);
+                }
+                __syncwarp();                              // the values are in registers: the stage goes back before the stores
+                if (lane == 0) mbar_arrive(empty + st);
+#pragma unroll
+                for (int u = 0; u < kGatherItems; ++u) {
+                    const int j = jb + (meta[u] & 0xff);
+                    if (meta[u] >= 0 && j < n_mid) {
+                        const int hh = (meta[u] >> 8) & 0xf, side = (meta[u] >> 12) & 1, lch = meta[u] >> 16;
+                        const int cls = p2 ? (j & (s.P - 1)) : j % s.P, slot = p2 ? (j >> lgP) : j / s.P;
+                        const int nfull = side ? s.nfv : s.nfk;
+                        // logical chunk lch of a V^mu row is stored at chunk lch ^ swizzle
+                        const int ch = side ? (lch ^ v_swz(slot, nfull >> 3)) : lch;
+                        bf16* dst = mid_row<bf16>(side ? c.v_mid : c.k_mid, s, b, h0 + hh, cls, slot, nfull);
+                        reinterpret_cast<uint4*>(dst)[ch] = val[u];
+                    }
+                }
+            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(gather_done);
         } else {
             // ---------------- basis generators: A operand ----------------
             const int t = tid - 64;                        // 0 .. 32 kGenWarps - 1
@@ -139,27 +228,32 @@ __global__ void __launch_bounds__(kThreadsTc, 1) compress_tc_kernel(const __grid
             const unsigned n = (unsigned)(mt * (kBM / 2) + fi);         // frequency of rows 2 fi (cos), 2 fi + 1 (sin)
             const bool row_on = (int)(2 * n) < s.M;
             const float inv_T = 1.0f / (float)s.T;
-            // rotation by two tokens, as splat pairs
-            unsigned long long CS2, SN2, NSN2;
-            {
-                const unsigned ph2 = (unsigned)((2ull * n) % (unsigned)s.T);
-                const float a = 6.283185307179586f * ((float)ph2 * inv_T - ((float)ph2 * inv_T >= 0.5f ? 1.0f : 0.0f));
-                const float c2 = __cosf(a), s2 = __sinf(a);
-                asm("mov.b64 %0, {%1,%1};" : "=l"(CS2) : "f"(c2));
-                asm("mov.b64 %0, {%1,%1};" : "=l"(SN2) : "f"(s2));
-                asm("mov.b64 %0, {%1,%1};" : "=l"(NSN2) : "f"(-s2));
-            }
+            auto splat_rot = [&](unsigned long long tokens, unsigned long long& CS, unsigned long long& SN, unsigned long long& NSN) {
+                const unsigned ph = (unsigned)((tokens * n) % (unsigned)s.T);
+                const float a = 6.283185307179586f * ((float)ph * inv_T - ((float)ph * inv_T >= 0.5f ? 1.0f : 0.0f));
+                const float cs = __cosf(a), sn = __sinf(a);
+                asm("mov.b64 %0, {%1,%1};" : "=l"(CS) : "f"(cs));
+                asm("mov.b64 %0, {%1,%1};" : "=l"(SN) : "f"(sn));
+                asm("mov.b64 %0, {%1,%1};" : "=l"(NSN) : "f"(-sn));
+            };
+            // rotations by two tokens, and by the 48 tokens between the end of this thread's run and its run in the next block
+            unsigned long long CS2, SN2, NSN2, CS48, SN48, NSN48;
+            splat_rot(2ull, CS2, SN2, NSN2);
+            splat_rot(48ull, CS48, SN48, NSN48);
             const int r0 = 2 * fi, r1 = 2 * fi + 1;
             const uint32_t row_off0 = (uint32_t)((r0 >> 3) * 1024 + (r0 & 7) * 128);
             const uint32_t row_off1 = (uint32_t)((r1 >> 3) * 1024 + (r1 & 7) * 128);
+            // packed phasors of two neighbouring tokens: C = (cos, cos), S = (sin, sin).  Seeded from exact integer
+            // phases every kReseed blocks and carried by rotations in between (9 per block: the drift stays far
+            // below the bf16 rounding of the tile).
+            constexpr int kReseed = 8;
+            unsigned long long C = 0, S = 0;
             for (int kb = kb0; kb < kb1; ++kb) {
                 const int it = kb - kb0, st = it % kStagesTc;
                 if (it >= kStagesTc && !mbar_wait(empty + st, ((it / kStagesTc) - 1) & 1, fail, c.status)) break;
                 unsigned char* a_dst = stage0 + (size_t)st * kStageBytesTc;
                 const int j0 = kb * kBK + 16 * tqr;
-                // packed phasors of tokens (j0, j0 + 1): C = (cos, cos), S = (sin, sin), exact integer phases
-                unsigned long long C, S;
-                {
+                if (it % kReseed == 0) {
                     const unsigned pa = (n * (unsigned)j0) % (unsigned)s.T, pb = (n * (unsigned)(j0 + 1)) % (unsigned)s.T;
                     const float fa = (float)pa * inv_T, fb = (float)pb * inv_T;
                     const float aa = 6.283185307179586f * (fa - (fa >= 0.5f ? 1.0f : 0.0f));
@@ -201,23 +295,33 @@ __global__ void __launch_bounds__(kThreadsTc, 1) compress_tc_kernel(const __grid
                 asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic stores -> visible to the tensor core
                 __syncwarp();
                 if (lane == 0) mbar_arrive(fullA + st);
+                {                                          // on to the same run of the next block
+                    unsigned long long tC, tS, nC, nS;
+                    asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(tC) : "l"(C), "l"(CS48));
+                    asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(tS) : "l"(S), "l"(CS48));
+                    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(nC) : "l"(S), "l"(NSN48), "l"(tC));
+                    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(nS) : "l"(C), "l"(SN48), "l"(tS));
+                    C = nC;
+                    S = nS;
+                }
             }
             // ---------------- epilogue: accumulators -> compressed columns ----------------
-            const bool ok = mbar_wait(acc_ready, 0, fail, c.status);
+            // the stage ring is reused below: every MMA has read it, and the gather warps have left it
+            const bool ok = mbar_wait(acc_ready, 0, fail, c.status) && mbar_wait(gather_done, 0, fail, c.status);
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
             if (ok) {
                 const int lane_grp = warp & 3;             // a warp reads tensor-memory lanes 32 (warp % 4) ...
-                const int col_half = (warp - 2) >> 2;      // two warps share a lane group: one column half each
-                const int m_base = mt * kBM + lane_grp * 32;
-                constexpr int kHalf = (int)kTmemCols / 2;
+                const int col_part = (warp - 2) >> 2;      // the warps that share a lane group split the columns
+                constexpr int kPart = (int)kTmemCols / (kGenWarps / 4);
                 // A thread holds 32 columns of ONE row; added as they are, a warp's reduction would touch 32
                 // rows (32 sectors) per instruction.  Each warp transposes its 32 x 32 block through a tile of
                 // its own in the (now idle: every MMA has read it) stage ring, so that a reduction instruction
                 // covers 32 columns of one row: the compressed ones among them are neighbours in memory.
                 float* tile = reinterpret_cast<float*>(stage0) + (warp - 2) * (32 * 33);
 #pragma unroll 1
-                for (int col0 = col_half * kHalf; col0 < (col_half + 1) * kHalf; col0 += 32) {
+                for (int col0 = col_part * kPart; col0 < (col_part + 1) * kPart; col0 += 32) {
                     const int hh = col0 / N, hcol0 = col0 - hh * N;
+                    const int m_base = mt * kBM + lane_grp * 32;
                     const bool is_k = hcol0 < D;           // a block of 32 columns lies within K's dims or within V's
                     const int ncomp = is_k ? s.dck : s.dcv;
                     float* base = coef_rows(is_k ? c.coef_k : c.coef_v, s, b, h0 + hh, ncomp) + (size_t)m_base * ncomp;
@@ -259,24 +363,34 @@ bool make_map(CUtensorMap* tm, const void* base, const Dims& s, int64_t sb, int6
 
 template <int D, int HP>
 cudaError_t launch_tc_t(const CUtensorMap& tmK, const CUtensorMap& tmV, const Dims& s, const CacheDev& c, int L, int n_mid,
-                        bool ordered, cudaStream_t stream) {
+                        bool ordered, bool gather, cudaStream_t stream) {
     constexpr int N = 2 * D;
     constexpr size_t stage = (size_t)kBM * kBK * 2 + (size_t)HP * (N / 64) * kBK * 64 * 2;
     constexpr size_t n_stages = (200 * 1024) / stage < 4 ? (200 * 1024) / stage : 4;
-    const size_t smem = n_stages * stage + 8 * (3 * n_stages + 1) + 16 + sizeof(int) * HP * 2 * D + 64 + 1024;
+    const size_t smem = n_stages * stage + 8 * (3 * n_stages + 2) + 16 + 2 * sizeof(int) * HP * 2 * D + 64 + 1024;
     cudaError_t err = ensure_dynamic_smem(compress_tc_kernel<D, HP>, smem);
     if (err != cudaSuccess) return err;
-    const int row_tiles = (s.M + kBM - 1) / kBM;
+    const int row_tiles = s.M / kBM;
     const int nkb = (n_mid + kBK - 1) / kBK;
     const int fixed = row_tiles * (s.Hkv / HP) * s.B;
     int n_tsplit = sm_count() / fixed;                          // one wave: one CTA per SM at most
     if (n_tsplit > nkb) n_tsplit = nkb;
     if (n_tsplit < 1 || ordered) n_tsplit = 1;                  // one split: every coefficient is added to zero exactly once
-    compress_tc_kernel<D, HP><<<dim3(row_tiles, s.Hkv / HP, s.B * n_tsplit), kThreadsTc, smem, stream>>>(tmK, tmV, s, c, L, n_tsplit);
+    if (gather && !compress_tc_gathers(s)) return cudaErrorInvalidValue;
+    compress_tc_kernel<D, HP><<<dim3(row_tiles, s.Hkv / HP, s.B * n_tsplit), kThreadsTc, smem, stream>>>(tmK, tmV, s, c, L, n_tsplit, gather ? 1 : 0);
     return cudaGetLastError();
 }
 
 }  // namespace
+
+// True if the tensor-core kernel can also write the kept-dim rows of the middle (its gather warps hold at most
+// kGatherItems chunks per thread and stage); otherwise the partition kernel writes them.
+bool compress_tc_gathers(const Dims& s) {
+    const int row_tiles = s.M / kBM;
+    const int hp = s.Hkv % 2 == 0 ? 2 : 1;
+    const int n_tok = (kBK + row_tiles - 1) / row_tiles;
+    return n_tok * hp * ((s.nfk + s.nfv) >> 3) <= kGatherItems * 32 * kGatherWarps;
+}
 
 // True if the tensor-core path serves this layout and these strides.
 bool compress_tc_supported(const Dims& s, int dtype, int64_t sb, int64_t st, int64_t sh) {
@@ -289,9 +403,10 @@ bool compress_tc_supported(const Dims& s, int dtype, int64_t sb, int64_t st, int
     return encode_tiled_fn() != nullptr;
 }
 
-// Coefficients only (the caller has zeroed them and runs the partition / gather kernel itself).
+// Coefficients (the caller has zeroed them) and, with gather, the kept-dim rows of the middle tokens; the windows
+// and the counters are the caller's (the partition kernel).
 cudaError_t launch_compress_tc(const Dims& s, const CacheDev& c, const void* K, const void* V, int64_t sb, int64_t st,
-                               int64_t sh, int L, bool ordered, cudaStream_t stream) {
+                               int64_t sh, int L, bool ordered, bool gather, cudaStream_t stream) {
     const int n_init = L < s.l_init ? L : s.l_init;
     const int n_local = (L - n_init) < s.l_local ? (L - n_init) : s.l_local;
     const int n_mid = L - n_init - n_local;
@@ -299,8 +414,8 @@ cudaError_t launch_compress_tc(const Dims& s, const CacheDev& c, const void* K, 
     CUtensorMap tmK, tmV;
     if (!make_map(&tmK, K, s, sb, st, sh, L) || !make_map(&tmV, V, s, sb, st, sh, L)) return cudaErrorInvalidValue;
     const bool pair = s.Hkv % 2 == 0;                        // two heads share a CTA and its basis tile
-    if (s.d == 128) return pair ? launch_tc_t<128, 2>(tmK, tmV, s, c, L, n_mid, ordered, stream) : launch_tc_t<128, 1>(tmK, tmV, s, c, L, n_mid, ordered, stream);
-    return pair ? launch_tc_t<64, 2>(tmK, tmV, s, c, L, n_mid, ordered, stream) : launch_tc_t<64, 1>(tmK, tmV, s, c, L, n_mid, ordered, stream);
+    if (s.d == 128) return pair ? launch_tc_t<128, 2>(tmK, tmV, s, c, L, n_mid, ordered, gather, stream) : launch_tc_t<128, 1>(tmK, tmV, s, c, L, n_mid, ordered, gather, stream);
+    return pair ? launch_tc_t<64, 2>(tmK, tmV, s, c, L, n_mid, ordered, gather, stream) : launch_tc_t<64, 1>(tmK, tmV, s, c, L, n_mid, ordered, gather, stream);
 }
 
 }  // namespace fa
