@@ -49,8 +49,19 @@ __device__ long long g_fa_timeline[2 * 8 * 32];
 extern "C" int fa_debug_timeline(long long* host_out) {
     return (int)cudaMemcpyFromSymbol(host_out, g_fa_timeline, sizeof(g_fa_timeline));
 }
+// Per CTA and launch (the last 32 launches): SM id, SM clock at entry, after the wait for the previous kernel, at exit.
+__device__ long long g_fa_span[32 * 160 * 4];
+__device__ int g_fa_span_cnt[160];
+extern "C" int fa_debug_spans(long long* host_out) {
+    return (int)cudaMemcpyFromSymbol(host_out, g_fa_span, sizeof(g_fa_span));
+}
+#define SPAN(i) do { if (threadIdx.x == 0 && blockIdx.z == 0) { const int cta_ = blockIdx.y * gridDim.x + blockIdx.x; if (cta_ < 160) { \
+    const int l_ = g_fa_span_cnt[cta_] & 31; long long* p_ = g_fa_span + (l_ * 160 + cta_) * 4; \
+    if ((i) == 0) { unsigned sm_; asm volatile("mov.u32 %0, %%smid;" : "=r"(sm_)); p_[0] = sm_; } \
+    p_[1 + ((i) > 2 ? 2 : (i))] = clock64(); if ((i) >= 2) g_fa_span_cnt[cta_] += 1; } } } while (0)
 #else
 #define TL(i) do { } while (0)
+#define SPAN(i) do { } while (0)
 #endif
 
 namespace fa {
@@ -487,6 +498,7 @@ __global__ void __launch_bounds__(kThreads, OCC) decode_fft_kernel(const __grid_
     const int log2P = 31 - __clz(s.P);
 
     TL(0);
+    SPAN(0);
     // ---- one-time set-up, independent of the cache: it may overlap the tail of the previous kernel ----
     if (tid < kConsumers) {
         #pragma unroll 1
@@ -553,6 +565,7 @@ __global__ void __launch_bounds__(kThreads, OCC) decode_fft_kernel(const __grid_
     // fused kernel: everything below reads what earlier kernels in the stream wrote (state, cache, coefficients, q)
     if (p.fused) {
         asm volatile("griddepcontrol.wait;" ::: "memory");
+        SPAN(1);
         start_coef_rows();
     }
     stage_inputs();
@@ -1634,7 +1647,7 @@ __global__ void __launch_bounds__(kThreads, OCC) decode_fft_kernel(const __grid_
     }
     consumer_sync();
     TL(19);
-    if (!*last_s) return;
+    if (!*last_s) { SPAN(2); return; }
     float* op_s = zw_s;                                    // [GH][np][d] (the slice buffers are free again)
     float* ocp_s = op_s + GH * np * s.d;                   // [GH][np][dcv]
     int* inv_s = reinterpret_cast<int*>(ocp_s + GH * np * s.dcv);   // [d] dim -> slot in D^vc, or -1
@@ -1673,6 +1686,7 @@ __global__ void __launch_bounds__(kThreads, OCC) decode_fft_kernel(const __grid_
         out[(qh0 + g) * s.d + e] = __float2bfloat16_rn(v * linv_s[g]);
     }
     TL(20);
+    SPAN(3);
     if (tid == 0 && np > 1) { bar[0] = 0; bar[1] = 0; bar[2] = 0; }   // the counters are zero again for the next call
     // Fused step: the last (KV head, pass) of this batch row to finish publishes the counters after the push
     // (the others read the old ones when they started; the next kernel in the stream sees the new ones).
