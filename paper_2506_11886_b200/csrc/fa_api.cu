@@ -388,7 +388,7 @@ fa_status fa_compress_ex(const fa_layout* layout, fa_cache* cache, const void* K
         // transform path: one store per coefficient, nothing to clear
         int log2S = 0;
         if (!compress_fft_supported(s, &log2S)) return FA_ERR_UNSUPPORTED;
-        if (launch_compress(s, make_cache(*cache), layout->kv_dtype, K, V, stride_b, stride_t, stride_h, L, false, true, true, cs) != cudaSuccess)
+        if (launch_compress(s, make_cache(*cache), layout->kv_dtype, K, V, stride_b, stride_t, stride_h, L, false, true, true, false, cs) != cudaSuccess)
             return FA_ERR_CUDA;
         if (L > 0 && launch_compress_fft(s, make_cache(*cache), layout->kv_dtype, K, V, sbb, stride_t, stride_h, L, log2S, cs) != cudaSuccess)
             return FA_ERR_CUDA;
@@ -400,10 +400,6 @@ fa_status fa_compress_ex(const fa_layout* layout, fa_cache* cache, const void* K
         }
         return FA_OK;
     }
-    fa_cache_sizes sz;
-    fa_cache_sizes_of(layout, &sz);
-    if (sz.coef_k && cudaMemsetAsync(cache->coef_k, 0, sz.coef_k, cs) != cudaSuccess) return FA_ERR_CUDA;
-    if (sz.coef_v && cudaMemsetAsync(cache->coef_v, 0, sz.coef_v, cs) != cudaSuccess) return FA_ERR_CUDA;
     // The tensor-core path rounds the basis to bf16 (relative error 2^-9 per term); summed over n middle
     // tokens the coefficient error relative to the largest coefficient falls like 1 / sqrt(n): short
     // middles (where the tensor cores would idle anyway) take the fp32 kernel to stay within 1e-3.
@@ -412,7 +408,7 @@ fa_status fa_compress_ex(const fa_layout* layout, fa_cache* cache, const void* K
     // tensor-core path: its kernel also writes the kept-dim rows of the middle from the boxes it loads; the partition
     // kernel is left with the windows and the counters
     const bool tc_rows = tc && compress_tc_gathers(s);
-    if (launch_compress(s, make_cache(*cache), layout->kv_dtype, K, V, stride_b, stride_t, stride_h, L, !tc, ordered, !tc_rows, cs) != cudaSuccess)
+    if (launch_compress(s, make_cache(*cache), layout->kv_dtype, K, V, stride_b, stride_t, stride_h, L, !tc, ordered, !tc_rows, true, cs) != cudaSuccess)
         return FA_ERR_CUDA;
     if (tc && launch_compress_tc(s, make_cache(*cache), K, V, sbb, stride_t, stride_h, L, ordered, tc_rows, cs) != cudaSuccess) return FA_ERR_CUDA;
     return FA_OK;

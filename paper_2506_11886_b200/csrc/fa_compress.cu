@@ -51,7 +51,7 @@ constexpr int kRowsPerCta = 64;
 template <typename KV>
 __global__ void __launch_bounds__(256) partition_gather_kernel(Dims s, CacheDev c, const KV* __restrict__ K,
                                                                    const KV* __restrict__ V, int64_t sb, int64_t st,
-                                                                   int64_t sh, int L, int mid_rows, int skip_a, int skip_c) {
+                                                                   int64_t sh, int L, int mid_rows, int skip_a, int skip_c, int zero_coef) {
     constexpr int EPC = 16 / (int)sizeof(KV);            // elements per chunk
     extern __shared__ __align__(16) unsigned char gsm[];
     KV* rows_s = reinterpret_cast<KV*>(gsm);                                         // [64][d]
@@ -67,8 +67,14 @@ __global__ void __launch_bounds__(256) partition_gather_kernel(Dims s, CacheDev 
         c.state[kStateStride * b + 3] = 0;          // ring starts at physical row 0
         c.state[kStateStride * b + 4] = 0;          // append ticket
     }
-    const KV* X = (side == 0 ? K : V) + (size_t)b * sb + (size_t)h * sh;
     const int nfull = side == 0 ? s.nfk : s.nfv;
+    if (zero_coef && s.d > nfull) {
+        // the contraction kernels behind this one ADD their partial sums: the CTAs of a (b, head, side) clear its coefficients
+        float4* cz = reinterpret_cast<float4*>(coef_rows(side == 0 ? c.coef_k : c.coef_v, s, b, h, s.d - nfull));
+        const int n4 = s.M * (s.d - nfull) / 4;
+        for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < n4; i += gridDim.x * blockDim.x) cz[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+    }
+    const KV* X = (side == 0 ? K : V) + (size_t)b * sb + (size_t)h * sh;
     const int32_t* idf = (side == 0 ? c.idx_full_k : c.idx_full_v) + (size_t)h * nfull;
     void* w_init = side == 0 ? c.k_init : c.v_init;
     void* w_local = side == 0 ? c.k_local : c.v_local;
@@ -194,7 +200,7 @@ __global__ void __launch_bounds__(256) compress_coef_kernel(Dims s, CacheDev c, 
 
 template <typename KV>
 static cudaError_t launch_compress_t(const Dims& s, const CacheDev& c, const void* K, const void* V, int64_t sb,
-                                     int64_t st, int64_t sh, int L, bool with_coef, bool ordered, bool mid_rows, cudaStream_t stream) {
+                                     int64_t st, int64_t sh, int L, bool with_coef, bool ordered, bool mid_rows, bool zero_coef, cudaStream_t stream) {
     int chunks_rows = (L + kRowsPerCta - 1) / kRowsPerCta;
     if (chunks_rows < 1) chunks_rows = 1;
     int skip_a = 0, skip_c = 0;
@@ -214,7 +220,7 @@ static cudaError_t launch_compress_t(const Dims& s, const CacheDev& c, const voi
     cudaError_t err = ensure_dynamic_smem(partition_gather_kernel<KV>, gsmem);
     if (err != cudaSuccess) return err;
     partition_gather_kernel<KV><<<dim3(chunks_rows - (skip_c - skip_a), s.Hkv, s.B * 2), 256, gsmem, stream>>>(
-        s, c, static_cast<const KV*>(K), static_cast<const KV*>(V), sb, st, sh, L, mid_rows ? 1 : 0, skip_a, skip_c);
+        s, c, static_cast<const KV*>(K), static_cast<const KV*>(V), sb, st, sh, L, mid_rows ? 1 : 0, skip_a, skip_c, zero_coef ? 1 : 0);
     err = cudaGetLastError();
     if (err != cudaSuccess) return err;
     int n_init = L < s.l_init ? L : s.l_init;
@@ -239,11 +245,13 @@ static cudaError_t launch_compress_t(const Dims& s, const CacheDev& c, const voi
 }
 
 // with_coef = false runs only the partition / gather kernel (the tensor-core or the transform path computes the
-// coefficients); mid_rows = false leaves the kept-dim rows of the middle out too (windows and counters only).
+// coefficients); mid_rows = false leaves the kept-dim rows of the middle out too (windows and counters only);
+// zero_coef clears the coefficients in the same launch (for the contraction kernels, which add to them).
 cudaError_t launch_compress(const Dims& s, const CacheDev& c, int dtype, const void* K, const void* V, int64_t sb,
-                            int64_t st, int64_t sh, int L, bool with_coef, bool ordered, bool mid_rows, cudaStream_t stream) {
-    if (dtype == FA_BF16) return launch_compress_t<__nv_bfloat16>(s, c, K, V, sb, st, sh, L, with_coef, ordered, mid_rows, stream);
-    return launch_compress_t<float>(s, c, K, V, sb, st, sh, L, with_coef, ordered, mid_rows, stream);
+                            int64_t st, int64_t sh, int L, bool with_coef, bool ordered, bool mid_rows, bool zero_coef,
+                            cudaStream_t stream) {
+    if (dtype == FA_BF16) return launch_compress_t<__nv_bfloat16>(s, c, K, V, sb, st, sh, L, with_coef, ordered, mid_rows, zero_coef, stream);
+    return launch_compress_t<float>(s, c, K, V, sb, st, sh, L, with_coef, ordered, mid_rows, zero_coef, stream);
 }
 
 }  // namespace fa
