@@ -555,6 +555,28 @@ def test_multi_layer_step_equals_single_calls_bit_for_bit():
     pair0.check_state()
 
 
+@pytest.mark.parametrize("kw,P", [
+    (dict(B=1, Hq=8, Hkv=2, d=128, L=3000, T=4096, M=256, n_full_k=32, n_full_v=32), 16),     # two heads per CTA, two row tiles
+    (dict(B=2, Hq=6, Hkv=3, d=128, L=2300, T=4096, M=512, n_full_k=16, n_full_v=48), 32),     # odd head count: one head per CTA; 6-chunk V rows
+    (dict(B=1, Hq=4, Hkv=4, d=64, L=1500, T=2048, M=128, n_full_k=8, n_full_v=16), 8),        # one row tile: every token of a block in one CTA
+    (dict(B=1, Hq=2, Hkv=2, d=128, L=1400, T=2048, M=128, n_full_k=64, n_full_v=64), 4),      # more chunks than the gather warps hold: partition kernel writes the rows
+    (dict(B=1, Hq=2, Hkv=2, d=128, L=1100 + 37, T=2048, M=1024, n_full_k=0, n_full_v=8), 16), # nothing kept of K; ragged last block; idle row-tile CTAs
+])
+def test_tensor_compress_with_its_gather(kw, P):
+    """Middles of 1024 tokens and more take the tcgen05 kernel, which also writes the kept-dim rows of the middle
+    from the boxes it loads (every row_tiles-th token per CTA): windows, K^mu / V^mu (with V's chunk permutation) and
+    counters bit-exact, coefficients within 1e-3, decode on top within the output tolerance."""
+    shape = SMALL_BF16.with_(L_init=4, L_local=32, **kw)
+    layout = layout_of(shape, max_mid=shape.T, P=P)
+    stream = synth.KVStream(shape, seed=61, freq="offgrid")
+    pair = Pair(layout, stream.idx_full_k, stream.idx_full_v)
+    K, V = stream.tokens(0, shape.L)
+    pair.compress(K, V)
+    worst = pair.check_state()
+    assert worst <= 1e-3, worst
+    pair.check_decode(synth.queries(shape, seed=61))
+
+
 @pytest.mark.parametrize("shape,P", [(SMALL_BF16, 16), (SMALL_BF16.with_(L=2040, T=2048, M=256), 8), (CFG0, 32),
                                       (CFG0.with_(L_init=4, L_local=64, L=700), 16)])
 def test_compress_by_transform_matches_oracle(shape, P):
