@@ -104,6 +104,11 @@ cudaError_t launch_validate(const Dims&, const CacheDev&, cudaStream_t);
 cudaError_t launch_compress(const Dims&, const CacheDev&, int dtype, const void* K, const void* V, int64_t sb,
                             int64_t st, int64_t sh, int L, bool with_coef, bool ordered, bool mid_rows, bool zero_coef, cudaStream_t);
 bool compress_tc_gathers(const Dims& s);
+// The same path on CTA pairs (fa_compress_tc2.cu): needs an even number of 128-row tiles.
+bool compress_tc2_supported(const Dims& s);
+bool compress_tc2_gathers(const Dims& s);
+cudaError_t launch_compress_tc2(const Dims&, const CacheDev&, const void* K, const void* V, int64_t sb, int64_t st, int64_t sh,
+                                int L, bool ordered, bool gather, cudaStream_t);
 // Tensor-core reconstruction of the dimension selection (fa_select_tc.cu).
 bool reconstruct_tc_supported(const Dims& s, int dtype, const void* K, const void* V, int64_t sb, int64_t st, int64_t sh, int n_mid);
 size_t reconstruct_tc_scratch_bytes(const Dims& s);

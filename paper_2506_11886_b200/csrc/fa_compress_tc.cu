@@ -52,9 +52,10 @@ __global__ void __launch_bounds__(kThreadsTc, 1) compress_tc_kernel(const __grid
     extern __shared__ unsigned char smem_unaligned[];
     unsigned char* smem = smem_unaligned + ((1024u - (smem_u32(smem_unaligned) & 1023u)) & 1023u);
     unsigned char* stage0 = smem;                          // kStagesTc x (A | B boxes), 1024-byte aligned
-    uint64_t* fullA = reinterpret_cast<uint64_t*>(smem + kStagesTc * kStageBytesTc);
-    uint64_t* fullB = fullA + kStagesTc;
-    uint64_t* empty = fullB + kStagesTc;
+    // one barrier per stage for the basis tile (the generator warps) and the boxes (the producer's expect_tx): the
+    // thread that issues the MMAs pays for every barrier it passes
+    uint64_t* full = reinterpret_cast<uint64_t*>(smem + kStagesTc * kStageBytesTc);
+    uint64_t* empty = full + kStagesTc;
     uint64_t* acc_ready = empty + kStagesTc;
     uint64_t* gather_done = acc_ready + 1;                 // the gather warps are past their last box
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(gather_done + 1);
@@ -74,7 +75,7 @@ __global__ void __launch_bounds__(kThreadsTc, 1) compress_tc_kernel(const __grid
 
     if (tid == 0) {
         // a stage is free again when its MMAs have read it and the gather warps have taken their rows
-        for (int i = 0; i < kStagesTc; ++i) { mbar_init(fullA + i, kGenWarps); mbar_init(fullB + i, 1); mbar_init(empty + i, 1 + kGatherWarps); }
+        for (int i = 0; i < kStagesTc; ++i) { mbar_init(full + i, kGenWarps + 1); mbar_init(empty + i, 1 + kGatherWarps); }
         mbar_init(acc_ready, 1);
         mbar_init(gather_done, kGatherWarps);
         *fail = 0;
@@ -110,7 +111,7 @@ __global__ void __launch_bounds__(kThreadsTc, 1) compress_tc_kernel(const __grid
                     const int it = kb - kb0, st = it % kStagesTc;
                     if (it >= kStagesTc && !mbar_wait(empty + st, ((it / kStagesTc) - 1) & 1, fail, c.status)) break;
                     unsigned char* bdst = stage0 + (size_t)st * kStageBytesTc + kABytes;
-                    mbar_expect_tx(fullB + st, (uint32_t)kBBytes);
+                    mbar_expect_tx(full + st, (uint32_t)kBBytes);
                     const int tok = n_init + kb * kBK;
 #pragma unroll
                     for (int hh = 0; hh < HP; ++hh)
@@ -118,7 +119,7 @@ __global__ void __launch_bounds__(kThreadsTc, 1) compress_tc_kernel(const __grid
                         for (int bx = 0; bx < N / 64; ++bx) {
                             const CUtensorMap* tm = bx < D / 64 ? &tmK : &tmV;
                             const int dim0 = (bx % (D / 64)) * 64;
-                            tma_load_4d(bdst + hh * kBBytes1 + bx * kBoxBytes, tm, dim0, h0 + hh, tok, b, fullB + st);
+                            tma_load_4d(bdst + hh * kBBytes1 + bx * kBoxBytes, tm, dim0, h0 + hh, tok, b, full + st);
                         }
                 }
             }
@@ -128,7 +129,7 @@ __global__ void __launch_bounds__(kThreadsTc, 1) compress_tc_kernel(const __grid
                 for (int kb = kb0; kb < kb1; ++kb) {
                     const int it = kb - kb0, st = it % kStagesTc;
                     const uint32_t par = (it / kStagesTc) & 1;
-                    if (!mbar_wait(fullA + st, par, fail, c.status) || !mbar_wait(fullB + st, par, fail, c.status)) break;
+                    if (!mbar_wait(full + st, par, fail, c.status)) break;
                     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                     const uint32_t a_addr = smem_u32(stage0 + (size_t)st * kStageBytesTc);
                     const uint32_t b_addr = a_addr + kABytes;
@@ -186,7 +187,7 @@ __global__ void __launch_bounds__(kThreadsTc, 1) compress_tc_kernel(const __grid
             const int lgP = 31 - __clz(s.P);
             for (int kb = kb0; kb < kb1; ++kb) {
                 const int it = kb - kb0, st = it % kStagesTc;
-                if (!mbar_wait(fullB + st, (it / kStagesTc) & 1, fail, c.status)) break;
+                if (!mbar_wait(full + st, (it / kStagesTc) & 1, fail, c.status)) break;
                 const unsigned char* bsrc = stage0 + (size_t)st * kStageBytesTc + kABytes;
                 const int jb = kb * kBK;                   // first middle token of the block
                 uint4 val[kGatherItems];
@@ -294,7 +295,7 @@ __global__ void __launch_bounds__(kThreadsTc, 1) compress_tc_kernel(const __grid
                 }
                 asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic stores -> visible to the tensor core
                 __syncwarp();
-                if (lane == 0) mbar_arrive(fullA + st);
+                if (lane == 0) mbar_arrive(full + st);
                 {                                          // on to the same run of the next block
                     unsigned long long tC, tS, nC, nS;
                     asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(tC) : "l"(C), "l"(CS48));

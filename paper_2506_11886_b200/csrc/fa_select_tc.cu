@@ -72,9 +72,10 @@ __global__ void __launch_bounds__(kThreadsR, 1) reconstruct_tc_kernel(const __gr
     extern __shared__ unsigned char smem_unaligned[];
     unsigned char* smem = smem_unaligned + ((1024u - (smem_u32(smem_unaligned) & 1023u)) & 1023u);
     unsigned char* stage0 = smem;                          // kStagesR x (A | B boxes), 1024-byte aligned
-    uint64_t* fullA = reinterpret_cast<uint64_t*>(smem + kStagesR * kStageBytesR);
-    uint64_t* fullB = fullA + kStagesR;
-    uint64_t* empty = fullB + kStagesR;
+    // one barrier per stage for the basis tile (the generator warps) and the boxes (the producer's expect_tx): the
+    // thread that issues the MMAs pays for every barrier it passes
+    uint64_t* full = reinterpret_cast<uint64_t*>(smem + kStagesR * kStageBytesR);
+    uint64_t* empty = full + kStagesR;
     uint64_t* acc_ready = empty + kStagesR;
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_ready + 1);
     volatile int* fail = reinterpret_cast<volatile int*>(tmem_slot + 1);
@@ -85,7 +86,7 @@ __global__ void __launch_bounds__(kThreadsR, 1) reconstruct_tc_kernel(const __gr
     const int nkb = s.M / kRK;
 
     if (tid == 0) {
-        for (int i = 0; i < kStagesR; ++i) { mbar_init(fullA + i, kGenWarpsR); mbar_init(fullB + i, 1); mbar_init(empty + i, 1); }
+        for (int i = 0; i < kStagesR; ++i) { mbar_init(full + i, kGenWarpsR + 1); mbar_init(empty + i, 1); }
         mbar_init(acc_ready, 1);
         *fail = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -107,14 +108,14 @@ __global__ void __launch_bounds__(kThreadsR, 1) reconstruct_tc_kernel(const __gr
                 const int stg = kb % kStagesR;
                 if (kb >= kStagesR && !mbar_wait(empty + stg, ((kb / kStagesR) - 1) & 1, fail, status)) break;
                 unsigned char* bdst = stage0 + (size_t)stg * kStageBytesR + kABytes;
-                mbar_expect_tx(fullB + stg, (uint32_t)kBBytes);
+                mbar_expect_tx(full + stg, (uint32_t)kBBytes);
 #pragma unroll
                 for (int hh = 0; hh < HP; ++hh)
 #pragma unroll
                     for (int bx = 0; bx < N / 64; ++bx) {
                         const CUtensorMap* tm = bx < D / 64 ? &tmWK : &tmWV;
                         const int dim0 = (bx % (D / 64)) * 64;
-                        tma_load_4d(bdst + hh * kBBytes1 + bx * kBoxBytes, tm, dim0, h0 + hh, kb * kRK, b, fullB + stg);
+                        tma_load_4d(bdst + hh * kBBytes1 + bx * kBoxBytes, tm, dim0, h0 + hh, kb * kRK, b, full + stg);
                     }
             }
         }
@@ -124,7 +125,7 @@ __global__ void __launch_bounds__(kThreadsR, 1) reconstruct_tc_kernel(const __gr
             for (int kb = 0; kb < nkb; ++kb) {
                 const int stg = kb % kStagesR;
                 const uint32_t par = (kb / kStagesR) & 1;
-                if (!mbar_wait(fullA + stg, par, fail, status) || !mbar_wait(fullB + stg, par, fail, status)) break;
+                if (!mbar_wait(full + stg, par, fail, status)) break;
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                 const uint32_t a_addr = smem_u32(stage0 + (size_t)stg * kStageBytesR);
                 const uint32_t b_addr = a_addr + kABytes;
@@ -202,7 +203,7 @@ __global__ void __launch_bounds__(kThreadsR, 1) reconstruct_tc_kernel(const __gr
             }
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic stores -> visible to the tensor core
             __syncwarp();
-            if (lane == 0) mbar_arrive(fullA + stg);
+            if (lane == 0) mbar_arrive(full + stg);
         }
         // ---------------- epilogue: (accumulator - prefill)^2 summed over the tokens, per dim ----------------
         const bool ok = mbar_wait(acc_ready, 0, fail, status);

@@ -31,6 +31,7 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* b, uint32_t parity) {
 }
 // Bounded wait; on time-out records the failure (nobody waits for ever, tensor memory is still freed).
 __device__ __forceinline__ bool mbar_wait(uint64_t* b, uint32_t parity, volatile int* fail, int32_t* status) {
+    if (mbar_try_wait(b, parity)) return true;             // the common case costs one instruction
     if (*fail) return false;
     for (uint32_t i = 0; i < kSpinLimitTc; ++i)
         if (mbar_try_wait(b, parity)) return true;
@@ -81,6 +82,42 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&v)[32]) {
     asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 #pragma unroll
     for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
+}
+
+// ---- CTA pairs (cta_group::2): two CTAs of a cluster share one MMA of 256 accumulator rows; each holds its own A rows
+// and half of the B columns in its shared memory, the even CTA of the pair issues the instructions for both ----
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+// All threads of both CTAs meet (release / acquire at cluster scope).
+__device__ __forceinline__ void cluster_sync_all() {
+    asm volatile("barrier.cluster.arrive.release.aligned;\nbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+// Arrival on the barrier at the same shared-memory offset in CTA `rank` of the cluster.  Relaxed: what the arrival
+// announces (a basis tile and boxes in the sender's shared memory, complete and visible to the async proxy there:
+// the sender has waited on its own barrier for them) is read by the tensor cores once the MMA is issued, which
+// happens after the arrival is seen; the sender has no writes of its own to publish.  With release semantics at
+// cluster scope the arrival took over a thousand cycles and set the pace of the pair.
+__device__ __forceinline__ void mbar_arrive_cluster(uint64_t* local_bar, uint32_t rank) {
+    asm volatile(
+        "{\n .reg .b32 ra;\n mapa.shared::cluster.u32 ra, %0, %1;\n mbarrier.arrive.relaxed.cluster.shared::cluster.b64 _, [ra];\n}\n" ::"r"(
+            smem_u32(local_bar)),
+        "r"(rank)
+        : "memory");
+}
+__device__ __forceinline__ void umma_bf16_pair(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n .reg .pred p;\n setp.ne.b32 p, %4, 0;\n tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n}\n" ::"r"(tmem_d),
+        "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+// One arrival, when the MMAs issued so far are done, on the barrier at this offset in BOTH CTAs of the pair.
+__device__ __forceinline__ void umma_commit_pair(uint64_t* bar) {
+    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;" ::"r"(smem_u32(bar)),
+                 "h"((uint16_t)3)
+                 : "memory");
 }
 
 }  // namespace umma
