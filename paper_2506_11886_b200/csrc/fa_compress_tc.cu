@@ -60,8 +60,7 @@ __global__ void __launch_bounds__(kThreadsTc, 1) compress_tc_kernel(const __grid
     uint64_t* gather_done = acc_ready + 1;                 // the gather warps are past their last box
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(gather_done + 1);
     volatile int* fail = reinterpret_cast<volatile int*>(tmem_slot + 1);
-    int* inv = reinterpret_cast<int*>(tmem_slot + 4);      // [HP][2][D]: dim -> slot in D^kc / D^vc, or -1
-    int* idf_s = inv + HP * 2 * D;                         // [HP][2][D]: the kept dims D^ku / D^vu of the CTA's heads
+    int* idf_s = reinterpret_cast<int*>(tmem_slot + 4);    // [HP][2][D]: the kept dims D^ku / D^vu of the CTA's heads
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int mt = blockIdx.x, h0 = blockIdx.y * HP;
@@ -80,13 +79,6 @@ __global__ void __launch_bounds__(kThreadsTc, 1) compress_tc_kernel(const __grid
         mbar_init(gather_done, kGatherWarps);
         *fail = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    }
-    for (int i = tid; i < HP * 2 * D; i += kThreadsTc) inv[i] = -1;
-    __syncthreads();
-    for (int i = tid; i < HP * (s.dck + s.dcv); i += kThreadsTc) {
-        const int hh = i / (s.dck + s.dcv), r = i - hh * (s.dck + s.dcv);
-        if (r < s.dck) inv[hh * N + c.idx_comp_k[(size_t)(h0 + hh) * s.dck + r]] = r;
-        else inv[hh * N + D + c.idx_comp_v[(size_t)(h0 + hh) * s.dcv + (r - s.dck)]] = r - s.dck;
     }
     if (gather)
         for (int i = tid; i < HP * (s.nfk + s.nfv); i += kThreadsTc) {
@@ -312,30 +304,43 @@ __global__ void __launch_bounds__(kThreadsTc, 1) compress_tc_kernel(const __grid
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
             if (ok) {
                 const int lane_grp = warp & 3;             // a warp reads tensor-memory lanes 32 (warp % 4) ...
-                const int col_part = (warp - 2) >> 2;      // the warps that share a lane group split the columns
-                constexpr int kPart = (int)kTmemCols / (kGenWarps / 4);
-                // A thread holds 32 columns of ONE row; added as they are, a warp's reduction would touch 32
-                // rows (32 sectors) per instruction.  Each warp transposes its 32 x 32 block through a tile of
-                // its own in the (now idle: every MMA has read it) stage ring, so that a reduction instruction
-                // covers 32 columns of one row: the compressed ones among them are neighbours in memory.
-                float* tile = reinterpret_cast<float*>(stage0) + (warp - 2) * (32 * 33);
+                const int col_part = (warp - 2) >> 2;      // the two warps that share a lane group take half of the columns each
+                constexpr int kPart = (int)kTmemCols / (kGenWarps / 4);      // a whole number of sides (D columns each)
+                const int m_base = mt * kBM + lane_grp * 32;
+                // A thread holds 32 columns of ONE row of the accumulator.  The warp lays its 32 rows x D columns of one side
+                // (K or V of one head) out in the idle stage ring; then lane q owns the four compressed dims 4 q .. 4 q + 3
+                // (slots of D^c, ascending) and adds them row by row with one 16-byte vector reduction: a warp instruction
+                // covers a whole coefficient row of the side (d_c contiguous floats).
+                float* tile = reinterpret_cast<float*>(stage0) + (warp - 2) * (32 * (D + 1));
 #pragma unroll 1
-                for (int col0 = col_part * kPart; col0 < (col_part + 1) * kPart; col0 += 32) {
-                    const int hh = col0 / N, hcol0 = col0 - hh * N;
-                    const int m_base = mt * kBM + lane_grp * 32;
-                    const bool is_k = hcol0 < D;           // a block of 32 columns lies within K's dims or within V's
-                    const int ncomp = is_k ? s.dck : s.dcv;
-                    float* base = coef_rows(is_k ? c.coef_k : c.coef_v, s, b, h0 + hh, ncomp) + (size_t)m_base * ncomp;
-                    float v[32];
-                    tmem_ld32(tmem_base + ((uint32_t)(lane_grp * 32) << 16) + (uint32_t)col0, v);
+                for (int t0 = col_part * kPart; t0 < (col_part + 1) * kPart; t0 += D) {
+                    const int hh = t0 / N;
+                    const bool is_k = t0 - hh * N < D;
+                    const int ncomp = is_k ? s.dck : s.dcv, nq = ncomp >> 2;
+                    int col[4] = {0, 0, 0, 0};
+                    if (lane < nq) {
+                        const int32_t* idc = (is_k ? c.idx_comp_k : c.idx_comp_v) + (size_t)(h0 + hh) * ncomp + 4 * lane;
 #pragma unroll
-                    for (int i = 0; i < 32; ++i) tile[lane * 33 + i] = v[i];
+                        for (int i = 0; i < 4; ++i) col[i] = idc[i];
+                    }
+#pragma unroll 1
+                    for (int cb = 0; cb < D; cb += 32) {
+                        float v[32];
+                        tmem_ld32(tmem_base + ((uint32_t)(lane_grp * 32) << 16) + (uint32_t)(t0 + cb), v);
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) tile[lane * (D + 1) + cb + i] = v[i];
+                    }
                     __syncwarp();
-                    const int slot = inv[hh * N + hcol0 + lane];
-                    if (slot >= 0) {
+                    float* base = coef_rows(is_k ? c.coef_k : c.coef_v, s, b, h0 + hh, ncomp) + (size_t)m_base * ncomp + 4 * lane;
+                    if (lane < nq) {
 #pragma unroll 4
-                        for (int rr = 0; rr < 32; ++rr)
-                            if (m_base + rr < s.M) atomicAdd(base + (size_t)rr * ncomp + slot, tile[rr * 33 + lane]);
+                        for (int rr = 0; rr < 32; ++rr) {
+                            const float* trow = tile + rr * (D + 1);
+                            if (m_base + rr < s.M)
+                                asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(base + (size_t)rr * ncomp), "f"(trow[col[0]]),
+                                             "f"(trow[col[1]]), "f"(trow[col[2]]), "f"(trow[col[3]])
+                                             : "memory");
+                        }
                     }
                     __syncwarp();
                 }
@@ -368,7 +373,7 @@ cudaError_t launch_tc_t(const CUtensorMap& tmK, const CUtensorMap& tmV, const Di
     constexpr int N = 2 * D;
     constexpr size_t stage = (size_t)kBM * kBK * 2 + (size_t)HP * (N / 64) * kBK * 64 * 2;
     constexpr size_t n_stages = (200 * 1024) / stage < 4 ? (200 * 1024) / stage : 4;
-    const size_t smem = n_stages * stage + 8 * (3 * n_stages + 2) + 16 + 2 * sizeof(int) * HP * 2 * D + 64 + 1024;
+    const size_t smem = n_stages * stage + 8 * (3 * n_stages + 2) + 16 + sizeof(int) * HP * 2 * D + 64 + 1024;
     cudaError_t err = ensure_dynamic_smem(compress_tc_kernel<D, HP>, smem);
     if (err != cudaSuccess) return err;
     const int row_tiles = s.M / kBM;
