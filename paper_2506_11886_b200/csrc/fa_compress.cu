@@ -54,6 +54,9 @@ __global__ void __launch_bounds__(256) partition_gather_kernel(Dims s, CacheDev 
                                                                    int64_t sh, int L, int mid_rows, int skip_a, int skip_c, int zero_coef) {
     constexpr int EPC = 16 / (int)sizeof(KV);            // elements per chunk
     extern __shared__ __align__(16) unsigned char gsm[];
+    // the contraction kernel behind this one may start at once (programmatic dependent launch): it waits for this
+    // grid only in front of its reductions into the coefficients cleared here
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     KV* rows_s = reinterpret_cast<KV*>(gsm);                                         // [64][d]
     int32_t* idf_s = reinterpret_cast<int32_t*>(gsm + (size_t)kRowsPerCta * s.d * sizeof(KV));   // [nfull]
     const int h = blockIdx.y, b = blockIdx.z >> 1, side = blockIdx.z & 1;

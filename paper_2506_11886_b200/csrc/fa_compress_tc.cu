@@ -302,6 +302,8 @@ __global__ void __launch_bounds__(kThreadsTc, 1) compress_tc_kernel(const __grid
             // the stage ring is reused below: every MMA has read it, and the gather warps have left it
             const bool ok = mbar_wait(acc_ready, 0, fail, c.status) && mbar_wait(gather_done, 0, fail, c.status);
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+            // the coefficients are cleared by the partition kernel, which this launch may overlap: wait for it here
+            asm volatile("griddepcontrol.wait;" ::: "memory");
             if (ok) {
                 const int lane_grp = warp & 3;             // a warp reads tensor-memory lanes 32 (warp % 4) ...
                 const int col_part = (warp - 2) >> 2;      // the two warps that share a lane group take half of the columns each
@@ -383,8 +385,17 @@ cudaError_t launch_tc_t(const CUtensorMap& tmK, const CUtensorMap& tmV, const Di
     if (n_tsplit > nkb) n_tsplit = nkb;
     if (n_tsplit < 1 || ordered) n_tsplit = 1;                  // one split: every coefficient is added to zero exactly once
     if (gather && !compress_tc_gathers(s)) return cudaErrorInvalidValue;
-    compress_tc_kernel<D, HP><<<dim3(row_tiles, s.Hkv / HP, s.B * n_tsplit), kThreadsTc, smem, stream>>>(tmK, tmV, s, c, L, n_tsplit, gather ? 1 : 0);
-    return cudaGetLastError();
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(row_tiles, s.Hkv / HP, s.B * n_tsplit);
+    cfg.blockDim = dim3(kThreadsTc);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;   // may start under the partition kernel in front of it
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, compress_tc_kernel<D, HP>, tmK, tmV, s, c, L, n_tsplit, gather ? 1 : 0);
 }
 
 }  // namespace

@@ -313,6 +313,8 @@ __global__ void __launch_bounds__(kThreadsTc, 1) compress_tc2_kernel(const __gri
             // the stage ring is reused below: every MMA has read it, and the gather warps have left it
             const bool ok = mbar_wait(acc_ready, 0, fail, c.status) && mbar_wait(gather_done, 0, fail, c.status);
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+            // the coefficients are cleared by the partition kernel, which this launch may overlap: wait for it here
+            asm volatile("griddepcontrol.wait;" ::: "memory");
             if (ok) {
                 const int lane_grp = warp & 3;             // a warp reads tensor-memory lanes 32 (warp % 4) ...
                 const int col_part = (warp - 2) >> 2;      // the two warps that share a lane group take half of the columns each
@@ -399,13 +401,15 @@ cudaError_t launch_tc2_t(const CUtensorMap& tmK, const CUtensorMap& tmV, const D
     cfg.blockDim = dim3(kThreadsTc);
     cfg.dynamicSmemBytes = smem;
     cfg.stream = stream;
-    cudaLaunchAttribute attr[1];
+    cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeClusterDimension;
     attr[0].val.clusterDim.x = 2;
     attr[0].val.clusterDim.y = 1;
     attr[0].val.clusterDim.z = 1;
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;   // may start under the partition kernel in front of it
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
-    cfg.numAttrs = 1;
+    cfg.numAttrs = 2;
     return cudaLaunchKernelEx(&cfg, compress_tc2_kernel<D, HP>, tmK, tmV, s, c, L, n_tsplit, gather ? 1 : 0);
 }
 
