@@ -1,7 +1,6 @@
 // Host side of the C ABI declared in include/fa.h: argument checks, buffer
 // sizes, launch plans.  Every entry point validates on the host, then launches
 // on the caller's stream; nothing here allocates device memory.
-#include <cstdlib>
 #include <cstring>
 #include <mutex>
 
@@ -408,7 +407,7 @@ fa_status fa_compress_ex(const fa_layout* layout, fa_cache* cache, const void* K
     const bool tc = L > 0 && n_mid_host >= 1024 && compress_tc_supported(s, layout->kv_dtype, sbb, stride_t, stride_h);
     // tensor-core path: its kernel also writes the kept-dim rows of the middle from the boxes it loads; the partition
     // kernel is left with the windows and the counters
-    const bool tc2 = tc && compress_tc2_supported(s) && !getenv("FA_TC_SINGLE");   // CTA pairs where the row tiles pair up
+    const bool tc2 = tc && compress_tc2_supported(s);                       // CTA pairs where the row tiles pair up
     const bool tc_rows = tc && (tc2 ? compress_tc2_gathers(s) : compress_tc_gathers(s));
     if (launch_compress(s, make_cache(*cache), layout->kv_dtype, K, V, stride_b, stride_t, stride_h, L, !tc, ordered, !tc_rows, true, cs) != cudaSuccess)
         return FA_ERR_CUDA;
