@@ -502,7 +502,7 @@ def run_ours(args):
                       "compress_ms_per_layer": min(comp_ms), "compress_tflops": comp_flop / (min(comp_ms) * 1e-3) / 1e12,
                       "compress_frac_of_bf16_tflops": comp_flop / (min(comp_ms) * 1e-3) / 1e12 / bf16_peak,
                       "compress_tensor_pipe_pct": tensor_pct,
-                      "compress_path": "tcgen05 bf16 x bf16 -> f32 (TMEM), basis tile generated in registers",
+                      "compress_path": "tcgen05.mma.cta_group::2 bf16 x bf16 -> f32 (TMEM), CTA pairs, basis tiles generated in registers",
                       "compress_fft_ms_per_layer": min(comp_fft_ms),
                       "compress_fft_frac_of_hbm": prefill_bytes / (min(comp_fft_ms) * 1e-3) / 1e9 / _peaks()[0],
                       "compress_ordered_ms_per_layer": min(comp_ord_ms),
