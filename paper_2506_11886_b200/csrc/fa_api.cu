@@ -407,11 +407,21 @@ fa_status fa_compress_ex(const fa_layout* layout, fa_cache* cache, const void* K
     const bool tc = L > 0 && n_mid_host >= 1024 && compress_tc_supported(s, layout->kv_dtype, sbb, stride_t, stride_h);
     // tensor-core path: its kernel also writes the kept-dim rows of the middle from the boxes it loads; the partition
     // kernel is left with the windows and the counters
-    const bool tc2 = tc && compress_tc2_supported(s);                       // CTA pairs where the row tiles pair up
-    const bool tc_rows = tc && (tc2 ? compress_tc2_gathers(s) : compress_tc_gathers(s));
+    bool tc2 = tc && compress_tc2_supported(s);             // CTA pairs where the row tiles pair up
+    bool tc_rows = tc && (tc2 ? compress_tc2_gathers(s) : compress_tc_gathers(s));
     if (launch_compress(s, make_cache(*cache), layout->kv_dtype, K, V, stride_b, stride_t, stride_h, L, !tc, ordered, !tc_rows, true, cs) != cudaSuccess)
         return FA_ERR_CUDA;
-    if (tc2 && launch_compress_tc2(s, make_cache(*cache), K, V, sbb, stride_t, stride_h, L, ordered, tc_rows, cs) != cudaSuccess) return FA_ERR_CUDA;
+    if (tc2 && launch_compress_tc2(s, make_cache(*cache), K, V, sbb, stride_t, stride_h, L, ordered, tc_rows, cs) != cudaSuccess) {
+        // the cluster launch was refused (e.g. a partitioned device): the single-CTA kernel does the same work; if it
+        // cannot write the kept-dim rows itself, the partition kernel runs once more with them
+        cudaGetLastError();
+        tc2 = false;
+        if (tc_rows && !compress_tc_gathers(s)) {
+            tc_rows = false;
+            if (launch_compress(s, make_cache(*cache), layout->kv_dtype, K, V, stride_b, stride_t, stride_h, L, false, ordered, true, true, cs) != cudaSuccess)
+                return FA_ERR_CUDA;
+        }
+    }
     if (tc && !tc2 && launch_compress_tc(s, make_cache(*cache), K, V, sbb, stride_t, stride_h, L, ordered, tc_rows, cs) != cudaSuccess) return FA_ERR_CUDA;
     return FA_OK;
 }
