@@ -153,6 +153,7 @@ fa_status plan_decode(const fa_layout& l, DecodePlan* p) {
         p->fused = 0;
         p->n_wsplit = 0;
         p->occ = 1;
+        p->split = 0;
         // Short transforms leave room for two CTAs on an SM (a shorter ring, a register cap): one CTA's
         // dependent phases hide behind the other's, and a head gets twice the CTAs (or, with more heads
         // than SMs, the waves are twice as wide).  Tried first; one CTA per SM otherwise.
@@ -210,6 +211,16 @@ fa_status plan_decode(const fa_layout& l, DecodePlan* p) {
             p->occ = 1;
             p->n_split = best;
             p->nb = pick_nb(best);
+        }
+        // Split build of the fused kernel (one CTA per SM): six more warps form the kept-dim products of the next batch of
+        // classes while the eight transform warps work on this one, with a second set of score / probability buffers
+        // in place of one ring stage.  It pays where the transform batch does not shrink to make room for those buffers
+        // (the transform phases are not faster on fewer classes) and a CTA has several batches: the longest transforms.
+        if (p->fused && p->occ == 1 && log2S == 10) {
+            const int per_cta = (s.P + p->n_split - 1) / p->n_split;
+            if (per_cta >= 2 * p->nb && decode_fft_smem_bytes(s, log2S, p->gh, p->nb, 1, 1) <= 227 * 1024 &&
+                decode_fft_fused_fits(s, log2S, p->gh, p->nb, p->n_split + p->n_wsplit, 1, 1))
+                p->split = 1;
         }
     } else {
         p->gh = s.G >= 4 ? 4 : (s.G >= 2 ? 2 : 1);

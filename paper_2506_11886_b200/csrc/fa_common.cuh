@@ -71,6 +71,7 @@ struct DecodePlan {
     int fft_log2;      // log2 of the transform length (FFT path)
     int nb;            // classes transformed together by one CTA (FFT path)
     int occ;           // CTAs per SM the main kernel is built for (FFT path: 1, or 2 with a shorter ring)
+    int split;         // 1: the split build of the fused kernel (a tile group of warps beside the transform group)
     // workspace offsets in bytes
     size_t off_bar, off_u, off_ml, off_o, off_z, off_oc, off_om, off_cnt, total;
 };
@@ -129,8 +130,8 @@ cudaError_t launch_decode_direct(const Dims&, const CacheDev&, int dtype, const 
 // k_new / v_new non-null: a fused step (the push of Eq.5 rides on the decode launch; fused plans with one pass only).
 cudaError_t launch_decode_fft(const Dims&, const CacheDev&, int dtype, const DecodePlan&, const void* q, void* out, char* ws,
                               const void* k_new, const void* v_new, cudaStream_t);
-size_t decode_fft_smem_bytes(const Dims&, int log2S, int gh, int nb, int occ = 1);
-bool decode_fft_fused_fits(const Dims&, int log2S, int gh, int nb, int n_part, int occ = 1);
+size_t decode_fft_smem_bytes(const Dims&, int log2S, int gh, int nb, int occ = 1, int split = 0);
+bool decode_fft_fused_fits(const Dims&, int log2S, int gh, int nb, int n_part, int occ = 1, int split = 0);
 bool decode_fft_launchable(const Dims&, const DecodePlan&);
 cudaError_t launch_decode_epilogue(const Dims&, const CacheDev&, int dtype, const DecodePlan&, void* out, char* ws,
                                    cudaStream_t);

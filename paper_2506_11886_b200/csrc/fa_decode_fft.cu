@@ -70,6 +70,10 @@ namespace {
 constexpr int kConsumers = 256;
 constexpr int kWarps = kConsumers / 32;
 constexpr int kThreads = kConsumers + 32;
+// The split kernel: the eight warps above are the transform group, four more consume the ring tiles (kept-dim products).
+constexpr int kSplitConsumers = kConsumers + 192;
+constexpr int kSplitWarps = kSplitConsumers / 32;
+__host__ __device__ constexpr int threads_of(bool split) { return (split ? kSplitConsumers : kConsumers) + 32; }
 constexpr int kStageBytes = 16384;
 constexpr int kStages = 5;                 // stages of the ring with one CTA per SM
 constexpr int kStagesOcc2 = 3;             // with two CTAs per SM (small transforms, many heads)
@@ -139,20 +143,24 @@ __device__ __forceinline__ void cp_async16(void* dst, const void* src) {
     asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(smem_addr(dst)), "l"(__cvta_generic_to_global(src)) : "memory");
 }
 __device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.commit_group;\ncp.async.wait_group 0;" ::: "memory"); }
-__device__ __forceinline__ void consumer_sync() { asm volatile("bar.sync 1, %0;" ::"n"(kConsumers) : "memory"); }
+// Barrier ID among NT threads: the consumer warps (all of them: barrier 1; the transform group of the split kernel: barrier 2)
+template <int NT = kConsumers, int ID = 1>
+__device__ __forceinline__ void consumer_sync() { asm volatile("bar.sync %0, %1;" ::"n"(ID), "n"(NT) : "memory"); }
 
 // Barrier among the CTAs of one (b, KV head, pass) on a global counter (fused kernel only: a
 // cooperative launch makes all of them resident).  Arrive: the consumer warps meet, then one thread
 // fences (cumulative over what the others wrote before the meeting) and adds 1 with release
 // semantics.  Wait: one thread polls with acquire loads, bounded like every other wait of this
 // kernel, then the consumer warps meet.
+template <int NT = kConsumers>
 __device__ __forceinline__ void part_arrive(int32_t* cnt, int n, int tid) {
-    consumer_sync();
+    consumer_sync<NT>();
     if (n > 1 && tid == 0) {                              // a part on its own meets nobody: no counter
         __threadfence();
         asm volatile("red.release.gpu.global.add.s32 [%0], 1;" ::"l"(cnt) : "memory");
     }
 }
+template <int NT = kConsumers>
 __device__ __forceinline__ void part_wait(const int32_t* cnt, int n, int tid, volatile int* fail, int32_t* status) {
     if (n > 1 && tid == 0 && !*fail) {
         bool ok = false;
@@ -164,7 +172,7 @@ __device__ __forceinline__ void part_wait(const int32_t* cnt, int n, int tid, vo
         }
         if (!ok) { *fail = 1; atomicExch(status, (int)FA_ERR_TIMEOUT); }
     }
-    consumer_sync();
+    consumer_sync<NT>();
 }
 
 __device__ __forceinline__ void mma_bf16(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0,
@@ -361,17 +369,18 @@ __device__ __forceinline__ void fft_pass(float* fbuf, int fb_floats, int nb, con
 }
 
 // All passes of the transform, ending each with a barrier of the consumer warps.
-template <int GH, int LS, int LL, bool DIT>
+// (kConsumers threads take part: all consumer warps, or the transform group of the split kernel with its barrier BID)
+template <int GH, int LS, int LL, bool DIT, int BID = 1>
 __device__ __forceinline__ void fft_run(float* fbuf, int fb_floats, int nb, const float* twf, int tid) {
     constexpr int RL = radix_log2(LL);
     if constexpr (!DIT) {
         fft_pass<GH, LS, LL, false>(fbuf, fb_floats, nb, twf, tid);
-        consumer_sync();
-        if constexpr (LL - RL > 0) fft_run<GH, LS, LL - RL, false>(fbuf, fb_floats, nb, twf, tid);
+        consumer_sync<kConsumers, BID>();
+        if constexpr (LL - RL > 0) fft_run<GH, LS, LL - RL, false, BID>(fbuf, fb_floats, nb, twf, tid);
     } else {
-        if constexpr (LL - RL > 0) fft_run<GH, LS, LL - RL, true>(fbuf, fb_floats, nb, twf, tid);
+        if constexpr (LL - RL > 0) fft_run<GH, LS, LL - RL, true, BID>(fbuf, fb_floats, nb, twf, tid);
         fft_pass<GH, LS, LL, true>(fbuf, fb_floats, nb, twf, tid);
-        consumer_sync();
+        consumer_sync<kConsumers, BID>();
     }
 }
 
@@ -417,7 +426,7 @@ struct FftSmem {
     int stages_off, fbuf_off, kb_off, pbt_off, twf_off, rev_off, E_off, ut_off, z_off, o_off, red_off, pend_off, zero_off, total;
     int fb_floats, pbs;
 };
-__host__ __device__ inline FftSmem fft_smem_layout(int log2S, int k, int GH, int NB, int d, int occ) {
+__host__ __device__ inline FftSmem fft_smem_layout(int log2S, int k, int GH, int NB, int d, int occ, int split = 0) {
     const int S = 1 << log2S;
     FftSmem L;
     L.fb_floats = pf_size(S * GH);
@@ -425,12 +434,12 @@ __host__ __device__ inline FftSmem fft_smem_layout(int log2S, int k, int GH, int
     int off = 256;                                        // mbarriers + flags
     L.zero_off = off; off += 16;
     off = 1024;                                           // stages are 1024-byte aligned (swizzled window tiles)
-    L.stages_off = off; off += ring_stages(occ) * kStageBytes;
+    L.stages_off = off; off += (ring_stages(occ) - (split ? 1 : 0)) * kStageBytes;   // split kernel: a stage goes to the second buffers
     L.fbuf_off = off; off += 4 * NB * L.fb_floats;
     off = (off + 15) / 16 * 16;
-    L.kb_off = off; off += 4 * NB * S * GH;               // kept-dim scores of the batch, natural token order
+    L.kb_off = off; off += (split ? 2 : 1) * 4 * NB * S * GH;   // kept-dim scores of the batch, natural token order (split kernel: two batches)
     off = (off + 15) / 16 * 16;
-    L.pbt_off = off; off += 2 * NB * GH * L.pbs;
+    L.pbt_off = off; off += (split ? 2 : 1) * 2 * NB * GH * L.pbs;
     off = (off + 15) / 16 * 16;
     L.twf_off = off; off += 8 * (tw_total(log2S) + 1);
     L.rev_off = off; off += 2 * S;
@@ -440,7 +449,7 @@ __host__ __device__ inline FftSmem fft_smem_layout(int log2S, int k, int GH, int
     L.z_off = off; off += (8 * k * GH + 15) / 16 * 16;
     off = (off + 15) / 16 * 16;
     L.o_off = off; off += 8 * GH * d;
-    L.red_off = off; off += 4 * (kWarps * GH + GH + 8);
+    L.red_off = off; off += 4 * ((split ? kSplitWarps : kWarps) * GH + GH + 8);
     off = (off + 15) / 16 * 16;
     L.pend_off = off; off += 8 * d + 4 * kPendRows + 4 * d + 2 * GH * d + 4 * d;   // fused step: compressed dims of the leaving row, basis column of this part's rows, the leaving row; the query rows
     L.total = (off + 127) / 128 * 128 + 1024;             // slack to align the base to 1024 bytes at run time
@@ -451,8 +460,8 @@ template <int GH> __host__ __device__ constexpr int hperm(int s) { return GH == 
 
 // GH query heads per CTA (2 or 4), transform length S = 2^LS, OCC CTAs per SM (2: shorter ring, register cap),
 // STEP: the instance that also carries the push of a fused step (the plain decode call pays nothing for it).
-template <int GH, int LS, int OCC, bool STEP>
-__global__ void __launch_bounds__(kThreads, OCC) decode_fft_kernel(const __grid_constant__ CUtensorMap tm_ki,
+template <int GH, int LS, int OCC, bool STEP, bool SPLIT>
+__global__ void __launch_bounds__(threads_of(SPLIT), OCC) decode_fft_kernel(const __grid_constant__ CUtensorMap tm_ki,
                                                                   const __grid_constant__ CUtensorMap tm_vi,
                                                                   const __grid_constant__ CUtensorMap tm_kl,
                                                                   const __grid_constant__ CUtensorMap tm_vl, Dims s, CacheDev c,
@@ -462,13 +471,19 @@ __global__ void __launch_bounds__(kThreads, OCC) decode_fft_kernel(const __grid_
     constexpr bool step = STEP;
     constexpr int N = GH / 2;
     constexpr int S = 1 << LS;
-    constexpr int NS = ring_stages(OCC);
+    constexpr int NS = ring_stages(OCC) - (SPLIT ? 1 : 0);
+    // Consumer threads: kAll of them; the warps that consume ring tiles (kept-dim and window products) are all of them,
+    // or, in the split kernel, the last four, while the first eight (the transform group) run the compressed-dim phases
+    // of the class batches beside them.
+    constexpr int kAll = SPLIT ? kSplitConsumers : kConsumers, kAllW = kAll / 32, kAllT = kAll + 32;
+    constexpr int kMW = SPLIT ? kAllW - kWarps : kWarps, kM0 = SPLIT ? kWarps : 0;
+    auto all_sync = [] { consumer_sync<kAll, 1>(); };
     extern __shared__ __align__(128) unsigned char smem_unaligned[];
     unsigned char* smem_raw = smem_unaligned + ((1024u - (smem_addr(smem_unaligned) & 1023u)) & 1023u);
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");      // the epilogue may be scheduled behind us at once
     Ws ws = ws_view(wsp, p);
     const int NB = p.nb;
-    const FftSmem L = fft_smem_layout(LS, s.k, GH, NB, s.d, OCC);
+    const FftSmem L = fft_smem_layout(LS, s.k, GH, NB, s.d, OCC, SPLIT ? 1 : 0);
     uint64_t* full = reinterpret_cast<uint64_t*>(smem_raw);
     uint64_t* empty = full + NS;
     volatile int* fail = reinterpret_cast<volatile int*>(smem_raw + 128);
@@ -485,7 +500,7 @@ __global__ void __launch_bounds__(kThreads, OCC) decode_fft_kernel(const __grid_
     // [GH heads][d]: the warps' output fragments are summed here as 64-bit fixed-point numbers (scale 2^30):
     // integer additions commute, so the shared-memory atomics give the same bits in whatever order they land
     long long* o_s = reinterpret_cast<long long*>(smem_raw + L.o_off);
-    float* red_s = reinterpret_cast<float*>(smem_raw + L.red_off);        // [kWarps][GH] + l_s[GH]
+    float* red_s = reinterpret_cast<float*>(smem_raw + L.red_off);        // [kAllW][GH] + l_s[GH]
     const int fb_floats = L.fb_floats, pbs = L.pbs;
 
     const int part = blockIdx.x;                          // partial-result index: class CTAs, then window CTAs
@@ -500,9 +515,9 @@ __global__ void __launch_bounds__(kThreads, OCC) decode_fft_kernel(const __grid_
     TL(0);
     SPAN(0);
     // ---- one-time set-up, independent of the cache: it may overlap the tail of the previous kernel ----
-    if (tid < kConsumers) {
+    if (tid < kAll) {
         #pragma unroll 1
-        for (int i = tid; i < s.k; i += kConsumers) {
+        for (int i = tid; i < s.k; i += kAll) {
             E[i] = cis_frac((float)i / (float)s.T);
         }
         for (int l = LS; l > 0;) {
@@ -510,7 +525,7 @@ __global__ void __launch_bounds__(kThreads, OCC) decode_fft_kernel(const __grid_
             if (l > rl) {
                 const int off = tw_offset(LS, l);
                 #pragma unroll 1
-                for (int i = tid; i < (R - 1) * st; i += kConsumers) {
+                for (int i = tid; i < (R - 1) * st; i += kAll) {
                     const int qm1 = i / st, j = i - qm1 * st;
                     reinterpret_cast<float2*>(twf)[off + i] = cis_frac((float)(((qm1 + 1) * j) & ((1 << l) - 1)) / (float)(1 << l));
                 }
@@ -518,8 +533,8 @@ __global__ void __launch_bounds__(kThreads, OCC) decode_fft_kernel(const __grid_
             l -= rl;
         }
         #pragma unroll 1
-        for (int a = tid; a < S; a += kConsumers) rev[a] = (uint16_t)dif_pos<LS>(a);
-        if (tid < GH + 8) red_s[kWarps * GH + tid] = 0.f;
+        for (int a = tid; a < S; a += kAll) rev[a] = (uint16_t)dif_pos<LS>(a);
+        if (tid < GH + 8) red_s[kAllW * GH + tid] = 0.f;
 
     }
     // This part's rows of C^K start towards the transform buffers, and its rows of C^V towards L2, as soon as
@@ -529,17 +544,17 @@ __global__ void __launch_bounds__(kThreads, OCC) decode_fft_kernel(const __grid_
     // buffers (one contiguous area, all idle until the first batch)
     const int uch = s.dck > 0 ? (((L.twf_off - L.fbuf_off) >> 2) / s.dck) & ~3 : 0;
     auto start_coef_rows = [&]() {
-        if (tid >= kConsumers) return;
+        if (tid >= kAll) return;
         if (s.dck > 0) {
             const float* ck = coef_rows(c.coef_k, s, b, h, s.dck) + (size_t)m0 * s.dck;
 #pragma unroll 1
-            for (int i = tid; i < min(m1 - m0, uch) * (s.dck >> 2); i += kConsumers) cp_async16(fbuf + 4 * i, ck + 4 * i);
+            for (int i = tid; i < min(m1 - m0, uch) * (s.dck >> 2); i += kAll) cp_async16(fbuf + 4 * i, ck + 4 * i);
         }
         if (s.dcv > 0) {
             const char* cv = reinterpret_cast<const char*>(coef_rows(c.coef_v, s, b, h, s.dcv) + (size_t)m0 * s.dcv);
             const int bytes = (m1 - m0) * s.dcv * 4;
 #pragma unroll 1
-            for (int o = tid * 128; o < bytes; o += kConsumers * 128) asm volatile("prefetch.global.L2 [%0];" ::"l"(cv + o));
+            for (int o = tid * 128; o < bytes; o += kAll * 128) asm volatile("prefetch.global.L2 [%0];" ::"l"(cv + o));
         }
     };
     // The inputs of the call, staged once: the query rows of this pass [GH heads][d] and, for a fused step, the
@@ -599,8 +614,8 @@ __global__ void __launch_bounds__(kThreads, OCC) decode_fft_kernel(const __grid_
     const int n_mid = min(n_mid_raw, s.max_mid);
     const int cstar = j_pend >= 0 ? j_pend & (s.P - 1) : -1, astar = j_pend >= 0 ? j_pend >> log2P : 0;   // class and slot of token j_pend
     // the row that leaves the local window (or the new token itself without a local window), both sides, natural dim order
-    if (j_pend >= 0 && tid >= kConsumers - 2 * (s.d >> 3) && tid < kConsumers) {
-        const int t2 = tid - (kConsumers - 2 * (s.d >> 3));
+    if (j_pend >= 0 && tid >= kAll - 2 * (s.d >> 3) && tid < kAll) {
+        const int t2 = tid - (kAll - 2 * (s.d >> 3));
         const int side = t2 / (s.d >> 3), ch = t2 - side * (s.d >> 3);
         if (s.l_local > 0)
             *reinterpret_cast<uint4*>(xrow_s + side * s.d + 8 * ch) =
@@ -628,23 +643,27 @@ __global__ void __launch_bounds__(kThreads, OCC) decode_fft_kernel(const __grid_
     const int pbw = NB * L.pbs;                            // row stride of the window probabilities
 
     if (tid == 0) {
-        for (int i = 0; i < NS; ++i) { mbar_init(full + i, 1); mbar_init(empty + i, kWarps); }
+        for (int i = 0; i < NS; ++i) { mbar_init(full + i, 1); mbar_init(empty + i, kMW); }
+        if constexpr (SPLIT) {                            // the handshakes between the tile group and the transform group
+            uint64_t* gb = reinterpret_cast<uint64_t*>(smem_raw + 160);
+            for (int i = 0; i < 2; ++i) { mbar_init(gb + i, kMW); mbar_init(gb + 2 + i, kWarps); mbar_init(gb + 4 + i, kWarps); mbar_init(gb + 6 + i, kMW); }
+        }
         *fail = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     // stale shared memory must hold finite numbers: rows past the end of a tile are multiplied by p = 0
     #pragma unroll 1
-    for (int i = tid; i < (NS * kStageBytes) / 16; i += kThreads) reinterpret_cast<uint4*>(stages)[i] = make_uint4(0, 0, 0, 0);
+    for (int i = tid; i < (NS * kStageBytes) / 16; i += kAllT) reinterpret_cast<uint4*>(stages)[i] = make_uint4(0, 0, 0, 0);
     if (tid < 4) reinterpret_cast<uint32_t*>(zero16)[tid] = 0;
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     __syncthreads();
     TL(1);
 
     // ============================ producer warp =================================
-    if (tid >= kConsumers) {
+    if (tid >= kAll) {
         // Same order as the consumers: the K tiles of the first batch of classes, the window rows,
         // then per batch the V tiles (and, from the second batch on, its K tiles first).
-        const int plane = tid - kConsumers;
+        const int plane = tid - kAll;
         if (plane == 0) {
             int it = 0;
             auto acquire = [&](uint32_t bytes) -> unsigned char* {
@@ -690,11 +709,21 @@ __global__ void __launch_bounds__(kThreads, OCC) decode_fft_kernel(const __grid_
                             ++it;
                         }
             }
+            if constexpr (!SPLIT) {
 #pragma unroll 1
-            for (int cb = c0; cb < c1; cb += NB) {
-                const int nb = min(NB, c1 - cb);
-                if (cb != c0) class_tiles(cb, nb, 0);
-                class_tiles(cb, nb, 1);
+                for (int cb = c0; cb < c1; cb += NB) {
+                    const int nb = min(NB, c1 - cb);
+                    if (cb != c0) class_tiles(cb, nb, 0);
+                    class_tiles(cb, nb, 1);
+                }
+            } else {
+                // the tile group runs one batch of kept-dim scores ahead: K of batch 1, then V of batch i and K of batch i + 2
+                if (c0 + NB < c1) class_tiles(c0 + NB, min(NB, c1 - (c0 + NB)), 0);
+#pragma unroll 1
+                for (int cb = c0; cb < c1; cb += NB) {
+                    class_tiles(cb, min(NB, c1 - cb), 1);
+                    if (cb + 2 * NB < c1) class_tiles(cb + 2 * NB, min(NB, c1 - (cb + 2 * NB)), 0);
+                }
             }
         }
         return;
@@ -702,6 +731,8 @@ __global__ void __launch_bounds__(kThreads, OCC) decode_fft_kernel(const __grid_
 
     // ============================ consumer warps =================================
     const int warp = tid >> 5, lane = tid & 31;
+    const bool is_m = warp >= kM0;                        // this warp consumes ring tiles
+    const int wm = warp - kM0;
     const int gq = lane >> 2, tq = lane & 3;              // mma fragment coordinates
     const int npk = s.nfk >> 3, nchv = s.nfv >> 3, npw = s.d >> 3;
     const float sl2 = s.scale * kLog2e;
@@ -718,11 +749,11 @@ __global__ void __launch_bounds__(kThreads, OCC) decode_fft_kernel(const __grid_
     float* xp_s = reinterpret_cast<float*>(smem_raw + L.pend_off);       // [dck + dcv]
     float* f_s = xp_s + 2 * s.d;                                          // [kPendRows]
     if (j_pend >= 0) {
-        for (int i = tid; i < s.dck + s.dcv; i += kConsumers)
+        for (int i = tid; i < s.dck + s.dcv; i += kAll)
             xp_s[i] = i < s.dck ? __bfloat162float(xrow_s[c.idx_comp_k[(size_t)h * s.dck + i]])
                                 : __bfloat162float(xrow_s[s.d + c.idx_comp_v[(size_t)h * s.dcv + i - s.dck]]);
 #pragma unroll 1
-        for (int r = tid; r < min(m1 - m0, kPendRows); r += kConsumers) f_s[r] = basis_value(m0 + r, j_pend, s.T);
+        for (int r = tid; r < min(m1 - m0, kPendRows); r += kAll) f_s[r] = basis_value(m0 + r, j_pend, s.T);
     }
     // basis value of row r of this part (tabulated for the first kPendRows rows)
     auto f_row = [&](int r) -> float {
@@ -775,9 +806,9 @@ __global__ void __launch_bounds__(kThreads, OCC) decode_fft_kernel(const __grid_
         k_off[rd] = (uint32_t)(gq * rowb_k + 16 * (4 * rd + tq));
         k_on[rd] = 4 * rd + tq < npk;
     }
-    const uint32_t kb_lane = smem_addr(kb) + (uint32_t)(gq * GH + 2 * tq) * 4;
-    auto k_phase = [&](int cb, int nb) {
-        if (!ts_k) return;
+    const uint32_t kb_lane_off = (uint32_t)(gq * GH + 2 * tq) * 4;
+    auto k_phase = [&](int cb, int nb, float* kbuf) {
+        if (!ts_k || !is_m) return;
 #pragma unroll 1
         for (int ci = 0; ci < nb; ++ci) {
             const int n_c = n_of_class(cb + ci);
@@ -786,7 +817,7 @@ __global__ void __launch_bounds__(kThreads, OCC) decode_fft_kernel(const __grid_
                 const int nt = min(ts_k, n_c - a0);
                 const uint32_t tile = wait_tile_u();
 #pragma unroll 1
-                for (int grp = warp; grp * 16 < nt; grp += kWarps) {
+                for (int grp = wm; grp * 16 < nt; grp += kMW) {
                     const uint32_t gbase = tile + (uint32_t)(grp * 16) * rowb_k;
                     if (STEP && cb + ci == cstar && astar >= a0 + grp * 16 && astar < a0 + grp * 16 + 16) {
                         // fused step: middle token j_pend is not in the cache yet; its kept dims from the row that leaves the window
@@ -810,7 +841,7 @@ __global__ void __launch_bounds__(kThreads, OCC) decode_fft_kernel(const __grid_
                         }
                     }
                     if (2 * tq < GH) {
-                        const uint32_t dst = kb_lane + (uint32_t)((ci * S + a0 + grp * 16) * GH) * 4;
+                        const uint32_t dst = smem_addr(kbuf) + kb_lane_off + (uint32_t)((ci * S + a0 + grp * 16) * GH) * 4;
                         sts64(dst, d4[0] * sl2, d4[1] * sl2);
                         sts64(dst + 8 * GH * 4, d4[2] * sl2, d4[3] * sl2);
                     }
@@ -827,9 +858,9 @@ __global__ void __launch_bounds__(kThreads, OCC) decode_fft_kernel(const __grid_
         if (s.dck > 0) {
             float* qc = reinterpret_cast<float*>(o_s);     // [GH][dck] gathered query, fp32 (o_s is not in use yet)
             const int32_t* idc_k = c.idx_comp_k + (size_t)h * s.dck;
-            for (int i = tid; i < GH * s.dck; i += kConsumers) {
+            for (int i = tid; i < GH * s.dck; i += kAll) {
                 const int g = i / s.dck, e = i - g * s.dck;
-                qc[i] = i < kConsumers ? qc_early : (g < ng ? __bfloat162float(qs_s[g * s.d + idc_k[e]]) : 0.f);
+                qc[i] = i < kAll ? qc_early : (g < ng ? __bfloat162float(qs_s[g * s.d + idc_k[e]]) : 0.f);
             }
             const int l8 = tid & 7, rgi = tid >> 3, nv = s.dck >> 2;
             float* ckg = coef_rows(c.coef_k, s, b, h, s.dck);
@@ -837,17 +868,17 @@ __global__ void __launch_bounds__(kThreads, OCC) decode_fft_kernel(const __grid_
             for (int q0 = m0; q0 < m1; q0 += uch) {         // chunks of rows staged in the transform buffers
                 const int q1 = min(m1, q0 + uch);
                 if (q0 > m0) {
-                    consumer_sync();
+                    all_sync();
 #pragma unroll 1
-                    for (int i = tid; i < (q1 - q0) * nv; i += kConsumers) cp_async16(fbuf + 4 * i, ckg + (size_t)q0 * s.dck + 4 * i);
+                    for (int i = tid; i < (q1 - q0) * nv; i += kAll) cp_async16(fbuf + 4 * i, ckg + (size_t)q0 * s.dck + 4 * i);
                 }
                 cp_async_wait_all();
-                consumer_sync();
+                all_sync();
                 // fused step: the rank-1 update of Eq.5 that the light append kernel left pending, applied to
                 // this part's rows while they are on chip, and written back
                 if (j_pend >= 0) {
 #pragma unroll 1
-                    for (int i = tid; i < (q1 - q0) * nv; i += kConsumers) {
+                    for (int i = tid; i < (q1 - q0) * nv; i += kAll) {
                         const int r = i / nv, v = i - r * nv;
                         const float f = f_row(q0 - m0 + r);
                         float4 x = *reinterpret_cast<const float4*>(fbuf + 4 * i);
@@ -856,10 +887,10 @@ __global__ void __launch_bounds__(kThreads, OCC) decode_fft_kernel(const __grid_
                         *reinterpret_cast<float4*>(fbuf + 4 * i) = x;
                         *reinterpret_cast<float4*>(ckg + (size_t)q0 * s.dck + 4 * i) = x;
                     }
-                    consumer_sync();
+                    all_sync();
                 }
 #pragma unroll 1
-                for (int r0 = q0; r0 < q1; r0 += kConsumers / 8) {
+                for (int r0 = q0; r0 < q1; r0 += kAll / 8) {
                     const int r = r0 + rgi;
                     float a[GH];
 #pragma unroll
@@ -890,23 +921,23 @@ __global__ void __launch_bounds__(kThreads, OCC) decode_fft_kernel(const __grid_
                 }
             }
             TL(2);
-            part_arrive(bar + 0, p.n_part, tid);
+            part_arrive<kAll>(bar + 0, p.n_part, tid);
         }
         TL(3);
-        if (has_classes) k_phase(c0, min(NB, c1 - c0));
+        if (has_classes) k_phase(c0, min(NB, c1 - c0), kb);
         TL(4);
-        if (s.dck > 0 && !is_win) part_wait(bar + 0, p.n_part, tid, fail, c.status);
+        if (s.dck > 0 && !is_win) part_wait<kAll>(bar + 0, p.n_part, tid, fail, c.status);
         TL(5);
     } else {
-        if (has_classes) k_phase(c0, min(NB, c1 - c0));
+        if (has_classes) k_phase(c0, min(NB, c1 - c0), kb);
         // everything above is independent of the prologue kernel; its output u is first needed here
         asm volatile("griddepcontrol.wait;" ::: "memory");
     }
-    for (int i = tid; i < GH * s.d; i += kConsumers) o_s[i] = 0;
+    for (int i = tid; i < GH * s.d; i += kAll) o_s[i] = 0;
     // ut[n] = (A.re, A.im, B.re, B.im), A = heads of the real slots, B = heads of the imaginary slots;
     // all loads of an entry are issued together
     #pragma unroll 1
-    for (int n = tid; n < s.k; n += kConsumers) {
+    for (int n = tid; n < s.k; n += kAll) {
         float2 uv[GH];
 #pragma unroll
         for (int sl = 0; sl < GH; ++sl) {
@@ -925,7 +956,7 @@ __global__ void __launch_bounds__(kThreads, OCC) decode_fft_kernel(const __grid_
             zz[(2 * ab + 1) * N + ln] = 0.f;
         }
     }
-    consumer_sync();
+    all_sync();
 
     float m_run[GH], l_acc[GH];                           // per slot
 #pragma unroll
@@ -939,12 +970,12 @@ __global__ void __launch_bounds__(kThreads, OCC) decode_fft_kernel(const __grid_
             for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
             if (lane == 0) red_s[warp * GH + g] = v;
         }
-        consumer_sync();
+        all_sync();
 #pragma unroll
         for (int g = 0; g < GH; ++g) {
             float r = red_s[g];
 #pragma unroll
-            for (int w = 1; w < kWarps; ++w) r = fmaxf(r, red_s[w * GH + g]);
+            for (int w = 1; w < kAllW; ++w) r = fmaxf(r, red_s[w * GH + g]);
             mx[g] = r;
         }
     };
@@ -1029,10 +1060,11 @@ __global__ void __launch_bounds__(kThreads, OCC) decode_fft_kernel(const __grid_
                 #pragma unroll 1
                 for (int r0 = 0; r0 < sg.cnt[si]; r0 += ts_w) {
                     const int nt = min(ts_w, sg.cnt[si] - r0);
+                    if (!is_m) continue;
                     const unsigned char* tile = wait_tile();
                     const int nrow = new_buf == sg.buf[si] ? new_row - (sg.row[si] + r0) : -1;   // fused step: the new token's row in this tile
                     #pragma unroll 1
-                    for (int grp = (warp + kWarps - (it * (kWinRowsPerTile / 16)) % kWarps) % kWarps; grp * 16 < nt; grp += kWarps) {   // tiles rotate over the warps
+                    for (int grp = (wm + kMW - (it * (kWinRowsPerTile / 16)) % kMW) % kMW; grp * 16 < nt; grp += kMW) {   // tiles rotate over the warps
                         if (STEP && nrow >= grp * 16 && nrow < grp * 16 + 16) patch_win(tile, nrow, knew_bh);
                         const unsigned char* r_lo = tile + (size_t)(grp * 16 + gq) * 128;      // row & 7 == gq for both rows
                         float d4[4] = {0.f, 0.f, 0.f, 0.f};
@@ -1060,12 +1092,12 @@ __global__ void __launch_bounds__(kThreads, OCC) decode_fft_kernel(const __grid_
                     }
                     release_tile();
                 }
-            consumer_sync();
+            all_sync();
             float mx[GH], alpha[GH];
 #pragma unroll
             for (int g = 0; g < GH; ++g) mx[g] = kNegBig;
             #pragma unroll 1
-            for (int a = tid; a < n_tok; a += kConsumers) {
+            for (int a = tid; a < n_tok; a += kAll) {
                 float v[GH];
                 load_vals(sb + pf(a * GH), v);
 #pragma unroll
@@ -1081,7 +1113,7 @@ __global__ void __launch_bounds__(kThreads, OCC) decode_fft_kernel(const __grid_
             }
             const int n_pad = (n_tok + 15) & ~15;
             #pragma unroll 1
-            for (int a = tid; a < n_pad; a += kConsumers) {
+            for (int a = tid; a < n_pad; a += kAll) {
                 float v[GH];
 #pragma unroll
                 for (int g = 0; g < GH; ++g) v[g] = 0.f;
@@ -1098,17 +1130,18 @@ __global__ void __launch_bounds__(kThreads, OCC) decode_fft_kernel(const __grid_
 #pragma unroll
                 for (int mt = 0; mt < 8; ++mt) { accw[mt][0] *= al; accw[mt][1] *= ah; accw[mt][2] *= al; accw[mt][3] *= ah; }
             }
-            consumer_sync();
+            all_sync();
             const bf16* prow = pb + (size_t)(gq & (GH - 1)) * pbw;
             #pragma unroll 1
             for (int si = 0; si < sg.n; ++si)
                 #pragma unroll 1
                 for (int r0 = 0; r0 < sg.cnt[si]; r0 += ts_w) {
                     const int nt = min(ts_w, sg.cnt[si] - r0);
+                    if (!is_m) continue;
                     const unsigned char* tile = wait_tile();
                     const int nrow = new_buf == sg.buf[si] ? new_row - (sg.row[si] + r0) : -1;
                     #pragma unroll 1
-                    for (int grp = (warp + kWarps - (it * (kWinRowsPerTile / 16)) % kWarps) % kWarps; grp * 16 < nt; grp += kWarps) {
+                    for (int grp = (wm + kMW - (it * (kWinRowsPerTile / 16)) % kMW) % kMW; grp * 16 < nt; grp += kMW) {
                         if (STEP && nrow >= grp * 16 && nrow < grp * 16 + 16) patch_win(tile, nrow, vnew_bh);
                         const int a = sg.tok[si] + r0 + grp * 16;
                         // the tile's rows may start at any token of the chunk: gather the four p values one by one
@@ -1146,7 +1179,7 @@ __global__ void __launch_bounds__(kThreads, OCC) decode_fft_kernel(const __grid_
                     }
                     release_tile();
                 }
-            consumer_sync();
+            all_sync();
         }
         // the window fragments open o_s; the class batches rescale it as the running maximum moves
         if (2 * tq < GH) {
@@ -1160,7 +1193,7 @@ __global__ void __launch_bounds__(kThreads, OCC) decode_fft_kernel(const __grid_
             }
         }
     }
-    consumer_sync();
+    all_sync();
 
     TL(7);
     // ------------------------------ middle classes ------------------------------
@@ -1197,12 +1230,336 @@ __global__ void __launch_bounds__(kThreads, OCC) decode_fft_kernel(const __grid_
             }
         }
 
+        if constexpr (!SPLIT) {
         #pragma unroll 1
         for (int cb = c0; cb < c1; cb += NB) {
             const int nb = min(NB, c1 - cb);
             if (n_of_class(cb) == 0) break;               // classes are filled in order: nothing further on
-            if (cb != c0) k_phase(cb, nb);
+            if (cb != c0) k_phase(cb, nb, kb);
 
+            // packed Hermitian spectra of the nb classes: X_m = V^A_m + i V^B_m per complex lane,
+            // V_m = v_m + conj(v_{S-m}), v_n = (1/2) u~_n e^{i theta n c}.  Pair 0 is bins (0, S/2).
+            if (s.dck > 0) {
+                // neighbouring lanes share a pair of bins and take half of the classes each (a batch of one
+                // class: one lane per pair, half as many rounds)
+                const bool split2 = nb > 1;
+                const int hcls = split2 ? (nb + 1) >> 1 : nb;
+                #pragma unroll 1
+                for (int item = tid; item < (split2 ? S : S / 2); item += kAll) {
+                    const int pr = split2 ? item >> 1 : item, ci0 = split2 ? (item & 1) * hcls : 0, ci1 = min(nb, ci0 + hcls);
+                    const int m = pr, mc = pr == 0 ? S / 2 : S - pr;
+                    PC<N> Am = czero, Bm = czero, Ac = czero, Bc = czero;
+                    float2 em = make_float2(1.f, 0.f), ec = make_float2(1.f, 0.f);
+                    if (m < s.k) { ld_entry(ut, m, Am, Bm); em = E[m]; }
+                    if (mc < s.k) { ld_entry(ut, mc, Ac, Bc); ec = E[mc]; }
+                    float2 twm = seed_tw(m, cb + ci0), twc = seed_tw(mc, cb + ci0);
+                    #pragma unroll 1
+                    for (int ci = ci0; ci < ci1; ++ci) {
+                        const PR<N> wmr = splat<N>(twm.x), wmi = splat<N>(twm.y), wcr = splat<N>(twc.x), wci = splat<N>(twc.y);
+                        const PC<N> vAm = cmulw(Am, wmr, wmi), vBm = cmulw(Bm, wmr, wmi);
+                        const PC<N> vAc = cmulw(Ac, wcr, wci), vBc = cmulw(Bc, wcr, wci);
+                        float* base = fbuf + ci * fb_floats;
+                        if (pr != 0) {
+                            const PC<N> VA = cconj_add(vAm, vAc), VB = cconj_add(vBm, vBc);
+                            st_pt(base + pf(m * GH), PC<N>{VA.re - VB.im, VA.im + VB.re});        // V^A + i V^B
+                            st_pt(base + pf(mc * GH), PC<N>{VA.re + VB.im, VB.re - VA.im});       // conj(V^A) + i conj(V^B)
+                        } else {                                                                   // self-conjugate bins
+                            const PC<N> VA0 = cconj_add(vAm, vAm), VB0 = cconj_add(vBm, vBm);
+                            const PC<N> VA1 = cconj_add(vAc, vAc), VB1 = cconj_add(vBc, vBc);
+                            st_pt(base + pf(0), PC<N>{VA0.re - VB0.im, VA0.im + VB0.re});
+                            st_pt(base + pf((S / 2) * GH), PC<N>{VA1.re - VB1.im, VA1.im + VB1.re});
+                        }
+                        twm = cmulf(twm, em);
+                        twc = cmulf(twc, ec);
+                    }
+                }
+                all_sync();
+                if (cb == c0) TL(8);
+                fft_run<GH, LS, LS, false>(fbuf, fb_floats, nb, twf, tid);        // score of slot a at point rev[a]
+                if (cb == c0) TL(9);
+            } else {
+                #pragma unroll 1
+                for (int i = tid; i < nb * fb_floats; i += kAll) fbuf[i] = 0.f;
+                all_sync();
+            }
+
+            all_sync();
+
+            // online softmax over the batch
+            float mx[GH], alpha[GH];
+#pragma unroll
+            for (int g = 0; g < GH; ++g) mx[g] = kNegBig;
+            #pragma unroll 1
+            for (int i = tid; i < (nb << LS); i += kAll) {
+                const int ci = i >> LS, a = i & (S - 1);
+                if (a < n_of_class(cb + ci)) {
+                    // score = compressed part (transform output) + kept part
+                    float* pt = fbuf + ci * fb_floats + pf(rev[a] * GH);
+                    float v[GH], kv[GH];
+                    load_vals(pt, v);
+                    if (ts_k) {
+                        load_vals(kb + (size_t)i * GH, kv);
+#pragma unroll
+                        for (int g = 0; g < GH; ++g) v[g] += kv[g];
+                        store_vals(pt, v);
+                    }
+#pragma unroll
+                    for (int g = 0; g < GH; ++g) mx[g] = fmaxf(mx[g], v[g]);
+                }
+            }
+            block_max(mx);
+#pragma unroll
+            for (int g = 0; g < GH; ++g) {
+                const float m_new = fmaxf(m_run[g], mx[g]);
+                alpha[g] = ex2(m_run[g] - m_new);
+                m_run[g] = m_new;
+                l_acc[g] *= alpha[g];
+            }
+            #pragma unroll 1
+            for (int i = tid; i < (nb << LS); i += kAll) {
+                const int ci = i >> LS, a = i & (S - 1);
+                float* pt = fbuf + ci * fb_floats + pf(rev[a] * GH);
+                float v[GH];
+                load_vals(pt, v);
+                const bool ok = a < n_of_class(cb + ci);
+#pragma unroll
+                for (int g = 0; g < GH; ++g) {
+                    v[g] = ok ? ex2(v[g] - m_run[g]) : 0.f;
+                    l_acc[g] += v[g];
+                    pbt[(ci * GH + g) * pbs + a] = __float2bfloat16_rn(v[g]);
+                }
+                store_vals(pt, v);
+            }
+            {
+                const float al = alpha[(2 * tq) & (GH - 1)], ah = alpha[(2 * tq + 1) & (GH - 1)];
+#pragma unroll
+                for (int mt = 0; mt < 4; ++mt) { acc[mt][0] *= al; acc[mt][1] *= ah; acc[mt][2] *= al; acc[mt][3] *= ah; }
+            }
+            for (int i = tid; i < GH * s.d; i += kAll) {          // what the windows left in o_s (rows are heads)
+                const int g = i / s.d;
+                float a = alpha[0];
+#pragma unroll
+                for (int sl = 1; sl < GH; ++sl) if (hperm<GH>(sl) == g) a = alpha[sl];
+                o_s[i] = __float2ll_rn(__ll2float_rn(o_s[i]) * a);
+            }
+            all_sync();
+
+            if (cb == c0) TL(10);
+            // o^u[dim][slot] += V^mu^T p, 16 tokens per mma
+            if (ts_v) {
+                #pragma unroll 1
+                for (int ci = 0; ci < nb; ++ci) {
+                    const int n_c = n_of_class(cb + ci);
+                    const uint32_t prow = p_lane + (uint32_t)(ci * GH * pbs) * 2;
+                    #pragma unroll 1
+                    for (int a0 = 0; a0 < n_c; a0 += ts_v) {
+                        const int nt = min(ts_v, n_c - a0);
+                        const uint32_t tile = wait_tile_u();
+                        #pragma unroll 1
+                        for (int grp = wm; grp * 16 < nt; grp += kMW) {
+                            const uint32_t gbase = tile + (uint32_t)(grp * 16) * rowb_v;
+                            if (STEP && cb + ci == cstar && astar >= a0 + grp * 16 && astar < a0 + grp * 16 + 16) {
+                                const int32_t* idf = c.idx_full_v + (size_t)h * s.nfv;
+#pragma unroll 1
+                                for (int e = lane; e < s.nfv; e += 32)
+                                    asm volatile("st.shared.b16 [%0], %1;" ::"r"(tile + (uint32_t)((astar - a0) * rowb_v + 2 * v_mid_col(astar, e, s.nfv, FA_BF16))),
+                                                 "h"(__bfloat16_as_ushort(xrow_s[s.d + idf[e]])) : "memory");
+                                __syncwarp();
+                            }
+                            uint32_t b0 = 0, b1 = 0;
+                            if (gq < GH) {
+                                b0 = lds32(prow + (uint32_t)(a0 + grp * 16) * 2);
+                                b1 = lds32(prow + (uint32_t)(a0 + grp * 16 + 8) * 2);
+                            }
+#pragma unroll
+                            for (int mt = 0; mt < 4; ++mt) {
+                                if (mt < nmt) {
+                                    uint32_t af[4];
+                                    ldmatrix_x4_trans(af, v_off[mt] + gbase * v_mul[mt]);
+                                    mma_bf16(acc[mt], af[0], af[1], af[2], af[3], b0, b1);
+                                }
+                            }
+                        }
+                        release_tile();
+                    }
+                }
+            }
+
+            if (cb == c0) TL(11);
+            // z_n = alpha z_n + sum_c e^{i theta n c} Y^c_n, Y^c = transform of the packed probabilities
+            if (s.dcv > 0) {
+                fft_run<GH, LS, LS, true>(fbuf, fb_floats, nb, twf, tid);
+                if (cb == c0) TL(12);
+                PR<N> alA, alB;
+                if constexpr (N == 2) { alA = pk(alpha[0], alpha[1]); alB = pk(alpha[2], alpha[3]); }
+                else { alA = PR<1>{alpha[0]}; alB = PR<1>{alpha[1]}; }
+                const PR<N> half = splat<N>(0.5f);
+                const bool split2 = nb > 1;                // as for the spectra: one lane per pair when the batch is one class
+                const int hcls = split2 ? (nb + 1) >> 1 : nb;
+                #pragma unroll 1
+                for (int item = tid; item < (split2 ? S : S / 2); item += kAll) {       // split: whole warps (S is a multiple of 32)
+                    const int pr = split2 ? item >> 1 : item, ci0 = split2 ? (item & 1) * hcls : 0;
+                    const int m = pr, mc = pr == 0 ? S / 2 : S - pr;
+                    const int ci1 = (m >= s.k && mc >= s.k) ? ci0 : min(nb, ci0 + hcls);
+                    float2 em = make_float2(1.f, 0.f), ec = make_float2(1.f, 0.f);
+                    if (m < s.k) em = E[m];
+                    if (mc < s.k) ec = E[mc];
+                    float2 twm = seed_tw(m, cb + ci0), twc = seed_tw(mc, cb + ci0);
+                    PC<N> zAm = czero, zBm = czero, zAc = czero, zBc = czero;
+                    #pragma unroll 1
+                    for (int ci = ci0; ci < ci1; ++ci) {
+                        const float* base = fbuf + ci * fb_floats;
+                        const PC<N> ya = ld_pt<N>(base + pf(m * GH)), yb = ld_pt<N>(base + pf(mc * GH));
+                        const PR<N> wmr = splat<N>(twm.x), wmi = splat<N>(twm.y), wcr = splat<N>(twc.x), wci = splat<N>(twc.y);
+                        if (pr != 0) {
+                            // real slots: y0 = (ya + conj(yb)) / 2, imaginary slots: y1 = (ya - conj(yb)) / (2 i); bin mc holds the conjugates
+                            const PC<N> y0 = PC<N>{(ya.re + yb.re) * half, (ya.im - yb.im) * half};
+                            const PC<N> y1 = PC<N>{(ya.im + yb.im) * half, (yb.re - ya.re) * half};
+                            zAm = zAm + cmulw(y0, wmr, wmi);
+                            zBm = zBm + cmulw(y1, wmr, wmi);
+                            zAc = zAc + cmulw(PC<N>{y0.re, splat<N>(0.f) - y0.im}, wcr, wci);
+                            zBc = zBc + cmulw(PC<N>{y1.re, splat<N>(0.f) - y1.im}, wcr, wci);
+                        } else {
+                            // bins 0 and S/2 are real for each real sequence: (re, im) of the packed value are the two heads
+                            const PC<N> y0m = PC<N>{ya.re, splat<N>(0.f)}, y1m = PC<N>{ya.im, splat<N>(0.f)};
+                            const PC<N> y0c = PC<N>{yb.re, splat<N>(0.f)}, y1c = PC<N>{yb.im, splat<N>(0.f)};
+                            zAm = zAm + cmulw(y0m, wmr, wmi);
+                            zBm = zBm + cmulw(y1m, wmr, wmi);
+                            zAc = zAc + cmulw(y0c, wcr, wci);
+                            zBc = zBc + cmulw(y1c, wcr, wci);
+                        }
+                        twm = cmulf(twm, em);
+                        twc = cmulf(twc, ec);
+                    }
+                    if (split2) {
+                        zAm = pair_sum(zAm); zBm = pair_sum(zBm); zAc = pair_sum(zAc); zBc = pair_sum(zBc);
+                        if (item & 1) continue;
+                    }
+                    if (m < s.k) {
+                        PC<N> A, B;
+                        ld_entry(z_s, m, A, B);
+                        st_entry(z_s, m, PC<N>{pfma(A.re, alA, zAm.re), pfma(A.im, alA, zAm.im)},
+                                 PC<N>{pfma(B.re, alB, zBm.re), pfma(B.im, alB, zBm.im)});
+                    }
+                    if (mc < s.k) {
+                        PC<N> A, B;
+                        ld_entry(z_s, mc, A, B);
+                        st_entry(z_s, mc, PC<N>{pfma(A.re, alA, zAc.re), pfma(A.im, alA, zAc.im)},
+                                 PC<N>{pfma(B.re, alB, zBc.re), pfma(B.im, alB, zBc.im)});
+                    }
+                }
+            }
+            all_sync();
+        }
+        } else {
+            // ---- split kernel: the tile group (kept-dim products of batch i + 1 / i) beside the transform group ----
+            // Batches alternate between two buffers of kept-dim scores and of rounded probabilities.  Per buffer:
+            // kb_full (tile group -> transform group: the scores of the batch are in), kb_free (back: softmax has read
+            // them), p_full (transform group -> tile group: probabilities and the rescale factors of the batch are in),
+            // p_free (back: the V products have read them).  Batch 0's scores were formed before the window tokens.
+            uint64_t* kb_full = reinterpret_cast<uint64_t*>(smem_raw + 160);
+            uint64_t* kb_free = kb_full + 2;
+            uint64_t* p_full = kb_free + 2;
+            uint64_t* p_free = p_full + 2;
+            float* alpha_s = reinterpret_cast<float*>(smem_raw + 224);     // [2][GH] rescale factors of a batch, per slot
+            auto xf_sync = [] { consumer_sync<kConsumers, 2>(); };
+            int n_bat = 0;
+            for (int cb = c0; cb < c1 && n_of_class(cb) > 0; cb += NB) ++n_bat;
+            if (is_m) {
+                // ================= tile group =================
+                if (n_bat > 1) {
+                    k_phase(c0 + NB, min(NB, c1 - (c0 + NB)), kb + NB * S * GH);
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(kb_full + 1);
+                }
+                #pragma unroll 1
+                for (int bi = 0; bi < n_bat; ++bi) {
+                    const int cb = c0 + bi * NB, nb = min(NB, c1 - cb), bb = bi & 1;
+                    if (lane == 0) mbar_wait(p_full + bb, (bi >> 1) & 1, fail, c.status);   // one lane polls, the warp follows
+                    __syncwarp();
+                    {
+                        const float* al_b = alpha_s + bb * GH;
+                        const float al = al_b[(2 * tq) & (GH - 1)], ah = al_b[(2 * tq + 1) & (GH - 1)];
+#pragma unroll
+                        for (int mt = 0; mt < 4; ++mt) { acc[mt][0] *= al; acc[mt][1] *= ah; acc[mt][2] *= al; acc[mt][3] *= ah; }
+#pragma unroll
+                        for (int g = 0; g < GH; ++g) l_acc[g] *= al_b[g];
+                    }
+            // o^u[dim][slot] += V^mu^T p, 16 tokens per mma
+            if (ts_v) {
+                #pragma unroll 1
+                for (int ci = 0; ci < nb; ++ci) {
+                    const int n_c = n_of_class(cb + ci);
+                    const uint32_t prow = p_lane + (uint32_t)(bb * NB * GH * pbs + ci * GH * pbs) * 2;
+                    #pragma unroll 1
+                    for (int a0 = 0; a0 < n_c; a0 += ts_v) {
+                        const int nt = min(ts_v, n_c - a0);
+                        const uint32_t tile = wait_tile_u();
+                        #pragma unroll 1
+                        for (int grp = wm; grp * 16 < nt; grp += kMW) {
+                            const uint32_t gbase = tile + (uint32_t)(grp * 16) * rowb_v;
+                            if (STEP && cb + ci == cstar && astar >= a0 + grp * 16 && astar < a0 + grp * 16 + 16) {
+                                const int32_t* idf = c.idx_full_v + (size_t)h * s.nfv;
+#pragma unroll 1
+                                for (int e = lane; e < s.nfv; e += 32)
+                                    asm volatile("st.shared.b16 [%0], %1;" ::"r"(tile + (uint32_t)((astar - a0) * rowb_v + 2 * v_mid_col(astar, e, s.nfv, FA_BF16))),
+                                                 "h"(__bfloat16_as_ushort(xrow_s[s.d + idf[e]])) : "memory");
+                                __syncwarp();
+                            }
+                            uint32_t b0 = 0, b1 = 0;
+                            if (gq < GH) {
+                                b0 = lds32(prow + (uint32_t)(a0 + grp * 16) * 2);
+                                b1 = lds32(prow + (uint32_t)(a0 + grp * 16 + 8) * 2);
+                            }
+#pragma unroll
+                            for (int mt = 0; mt < 4; ++mt) {
+                                if (mt < nmt) {
+                                    uint32_t af[4];
+                                    ldmatrix_x4_trans(af, v_off[mt] + gbase * v_mul[mt]);
+                                    mma_bf16(acc[mt], af[0], af[1], af[2], af[3], b0, b1);
+                                }
+                            }
+                        }
+                        release_tile();
+                    }
+                }
+            }
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(p_free + bb);
+                    if (bi + 2 < n_bat) {
+                        const int cb2 = cb + 2 * NB;
+                        if (lane == 0) mbar_wait(kb_free + bb, (bi >> 1) & 1, fail, c.status);       // softmax of this batch has read the buffer
+                        __syncwarp();
+                        k_phase(cb2, min(NB, c1 - cb2), kb + bb * NB * S * GH);
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(kb_full + bb);
+                    }
+                }
+            } else {
+                // ================= transform group =================
+                // per-slot maximum over the group's threads (as block_max, on the group's barrier)
+                auto block_max_t = [&](float (&mx)[GH]) {
+#pragma unroll
+                    for (int g = 0; g < GH; ++g) {
+                        float v = mx[g];
+#pragma unroll
+                        for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+                        if (lane == 0) red_s[warp * GH + g] = v;
+                    }
+                    xf_sync();
+#pragma unroll
+                    for (int g = 0; g < GH; ++g) {
+                        float r = red_s[g];
+#pragma unroll
+                        for (int w = 1; w < kWarps; ++w) r = fmaxf(r, red_s[w * GH + g]);
+                        mx[g] = r;
+                    }
+                };
+                #pragma unroll 1
+                for (int bi = 0; bi < n_bat; ++bi) {
+                    const int cb = c0 + bi * NB, nb = min(NB, c1 - cb), bb = bi & 1;
+                    const float* kbuf = kb + bb * NB * S * GH;
+                    bf16* pbuf = pbt + bb * NB * GH * pbs;
             // packed Hermitian spectra of the nb classes: X_m = V^A_m + i V^B_m per complex lane,
             // V_m = v_m + conj(v_{S-m}), v_n = (1/2) u~_n e^{i theta n c}.  Pair 0 is bins (0, S/2).
             if (s.dck > 0) {
@@ -1239,18 +1596,20 @@ __global__ void __launch_bounds__(kThreads, OCC) decode_fft_kernel(const __grid_
                         twc = cmulf(twc, ec);
                     }
                 }
-                consumer_sync();
-                if (cb == c0) TL(8);
-                fft_run<GH, LS, LS, false>(fbuf, fb_floats, nb, twf, tid);        // score of slot a at point rev[a]
-                if (cb == c0) TL(9);
+                xf_sync();
+                fft_run<GH, LS, LS, false, 2>(fbuf, fb_floats, nb, twf, tid);        // score of slot a at point rev[a]
             } else {
                 #pragma unroll 1
                 for (int i = tid; i < nb * fb_floats; i += kConsumers) fbuf[i] = 0.f;
-                consumer_sync();
+                xf_sync();
             }
 
-            consumer_sync();
-
+                    xf_sync();
+                    // the kept-dim scores of this batch (batch 0: formed by everybody's earlier barriers)
+                    if (bi >= 1) {
+                        if (tid == 0) mbar_wait(kb_full + bb, ((bi >> 1) - (bb == 0 ? 1 : 0)) & 1, fail, c.status);   // one thread polls
+                        xf_sync();
+                    }
             // online softmax over the batch
             float mx[GH], alpha[GH];
 #pragma unroll
@@ -1264,7 +1623,7 @@ __global__ void __launch_bounds__(kThreads, OCC) decode_fft_kernel(const __grid_
                     float v[GH], kv[GH];
                     load_vals(pt, v);
                     if (ts_k) {
-                        load_vals(kb + (size_t)i * GH, kv);
+                        load_vals(kbuf + (size_t)i * GH, kv);
 #pragma unroll
                         for (int g = 0; g < GH; ++g) v[g] += kv[g];
                         store_vals(pt, v);
@@ -1273,13 +1632,17 @@ __global__ void __launch_bounds__(kThreads, OCC) decode_fft_kernel(const __grid_
                     for (int g = 0; g < GH; ++g) mx[g] = fmaxf(mx[g], v[g]);
                 }
             }
-            block_max(mx);
+            block_max_t(mx);
 #pragma unroll
             for (int g = 0; g < GH; ++g) {
                 const float m_new = fmaxf(m_run[g], mx[g]);
                 alpha[g] = ex2(m_run[g] - m_new);
                 m_run[g] = m_new;
                 l_acc[g] *= alpha[g];
+            }
+            if (bi >= 2) {                                // the tile group is done with this buffer's previous batch
+                if (tid == 0) mbar_wait(p_free + bb, ((bi >> 1) - 1) & 1, fail, c.status);
+                xf_sync();
             }
             #pragma unroll 1
             for (int i = tid; i < (nb << LS); i += kConsumers) {
@@ -1292,14 +1655,9 @@ __global__ void __launch_bounds__(kThreads, OCC) decode_fft_kernel(const __grid_
                 for (int g = 0; g < GH; ++g) {
                     v[g] = ok ? ex2(v[g] - m_run[g]) : 0.f;
                     l_acc[g] += v[g];
-                    pbt[(ci * GH + g) * pbs + a] = __float2bfloat16_rn(v[g]);
+                    pbuf[(ci * GH + g) * pbs + a] = __float2bfloat16_rn(v[g]);
                 }
                 store_vals(pt, v);
-            }
-            {
-                const float al = alpha[(2 * tq) & (GH - 1)], ah = alpha[(2 * tq + 1) & (GH - 1)];
-#pragma unroll
-                for (int mt = 0; mt < 4; ++mt) { acc[mt][0] *= al; acc[mt][1] *= ah; acc[mt][2] *= al; acc[mt][3] *= ah; }
             }
             for (int i = tid; i < GH * s.d; i += kConsumers) {          // what the windows left in o_s (rows are heads)
                 const int g = i / s.d;
@@ -1308,54 +1666,14 @@ __global__ void __launch_bounds__(kThreads, OCC) decode_fft_kernel(const __grid_
                 for (int sl = 1; sl < GH; ++sl) if (hperm<GH>(sl) == g) a = alpha[sl];
                 o_s[i] = __float2ll_rn(__ll2float_rn(o_s[i]) * a);
             }
-            consumer_sync();
-
-            if (cb == c0) TL(10);
-            // o^u[dim][slot] += V^mu^T p, 16 tokens per mma
-            if (ts_v) {
-                #pragma unroll 1
-                for (int ci = 0; ci < nb; ++ci) {
-                    const int n_c = n_of_class(cb + ci);
-                    const uint32_t prow = p_lane + (uint32_t)(ci * GH * pbs) * 2;
-                    #pragma unroll 1
-                    for (int a0 = 0; a0 < n_c; a0 += ts_v) {
-                        const int nt = min(ts_v, n_c - a0);
-                        const uint32_t tile = wait_tile_u();
-                        #pragma unroll 1
-                        for (int grp = warp; grp * 16 < nt; grp += kWarps) {
-                            const uint32_t gbase = tile + (uint32_t)(grp * 16) * rowb_v;
-                            if (STEP && cb + ci == cstar && astar >= a0 + grp * 16 && astar < a0 + grp * 16 + 16) {
-                                const int32_t* idf = c.idx_full_v + (size_t)h * s.nfv;
-#pragma unroll 1
-                                for (int e = lane; e < s.nfv; e += 32)
-                                    asm volatile("st.shared.b16 [%0], %1;" ::"r"(tile + (uint32_t)((astar - a0) * rowb_v + 2 * v_mid_col(astar, e, s.nfv, FA_BF16))),
-                                                 "h"(__bfloat16_as_ushort(xrow_s[s.d + idf[e]])) : "memory");
-                                __syncwarp();
-                            }
-                            uint32_t b0 = 0, b1 = 0;
-                            if (gq < GH) {
-                                b0 = lds32(prow + (uint32_t)(a0 + grp * 16) * 2);
-                                b1 = lds32(prow + (uint32_t)(a0 + grp * 16 + 8) * 2);
-                            }
+                    if (tid < GH) alpha_s[bb * GH + tid] = alpha[0];
 #pragma unroll
-                            for (int mt = 0; mt < 4; ++mt) {
-                                if (mt < nmt) {
-                                    uint32_t af[4];
-                                    ldmatrix_x4_trans(af, v_off[mt] + gbase * v_mul[mt]);
-                                    mma_bf16(acc[mt], af[0], af[1], af[2], af[3], b0, b1);
-                                }
-                            }
-                        }
-                        release_tile();
-                    }
-                }
-            }
-
-            if (cb == c0) TL(11);
+                    for (int g = 1; g < GH; ++g) if (tid == g) alpha_s[bb * GH + g] = alpha[g];
+                    xf_sync();
+                    if (lane == 0) { mbar_arrive(kb_free + bb); mbar_arrive(p_full + bb); }
             // z_n = alpha z_n + sum_c e^{i theta n c} Y^c_n, Y^c = transform of the packed probabilities
             if (s.dcv > 0) {
-                fft_run<GH, LS, LS, true>(fbuf, fb_floats, nb, twf, tid);
-                if (cb == c0) TL(12);
+                fft_run<GH, LS, LS, true, 2>(fbuf, fb_floats, nb, twf, tid);
                 PR<N> alA, alB;
                 if constexpr (N == 2) { alA = pk(alpha[0], alpha[1]); alB = pk(alpha[2], alpha[3]); }
                 else { alA = PR<1>{alpha[0]}; alB = PR<1>{alpha[1]}; }
@@ -1415,11 +1733,14 @@ __global__ void __launch_bounds__(kThreads, OCC) decode_fft_kernel(const __grid_
                     }
                 }
             }
-            consumer_sync();
+                    xf_sync();
+                }
+            }
+            all_sync();
         }
         TL(13);
         // fold the per-warp output fragments into o_s at the natural positions of D^vu
-        if (2 * tq < GH) {
+        if (2 * tq < GH && is_m) {
             long long* o_lo = o_s + hperm<GH>(2 * tq) * s.d;
             long long* o_hi = o_s + hperm<GH>(2 * tq + 1) * s.d;
 #pragma unroll
@@ -1437,23 +1758,23 @@ __global__ void __launch_bounds__(kThreads, OCC) decode_fft_kernel(const __grid_
         for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
         if (lane == 0) red_s[warp * GH + g] = v;
     }
-    consumer_sync();
+    all_sync();
     if (tid < GH) {
         float v = 0.f;
 #pragma unroll
-        for (int w = 0; w < kWarps; ++w) v += red_s[w * GH + tid];
-        red_s[kWarps * GH + tid] = v;
+        for (int w = 0; w < kAllW; ++w) v += red_s[w * GH + tid];
+        red_s[kAllW * GH + tid] = v;
     }
-    consumer_sync();
+    all_sync();
 
     TL(14);
     // ------------------------------ partial results ------------------------------
-    for (int i = tid; i < GH * s.d; i += kConsumers) {
+    for (int i = tid; i < GH * s.d; i += kAll) {
         const int g = i / s.d, e = i - g * s.d;
         if (g < ng) ws.o[(((size_t)b * s.Hq + g_first + g) * p.n_part + part) * s.d + e] = __ll2float_rn(o_s[i]) * kFixInv;
     }
     #pragma unroll 1
-    for (int n = tid; n < s.k; n += kConsumers) {
+    for (int n = tid; n < s.k; n += kAll) {
         const float* e = z_s + n * 2 * GH;
 #pragma unroll
         for (int sl = 0; sl < GH; ++sl) {
@@ -1471,7 +1792,7 @@ __global__ void __launch_bounds__(kThreads, OCC) decode_fft_kernel(const __grid_
 #pragma unroll
             for (int sl = 1; sl < GH; ++sl) if (tid == sl) mv = m_run[sl];
             ml[0] = mv;
-            ml[1] = red_s[kWarps * GH + tid];
+            ml[1] = red_s[kAllW * GH + tid];
         }
     }
     TL(15);
@@ -1487,7 +1808,7 @@ __global__ void __launch_bounds__(kThreads, OCC) decode_fft_kernel(const __grid_
     const int np = p.n_part;
     const int rows = m1 - m0;
     const size_t qh0 = (size_t)b * s.Hq + g_first;
-    const int nv = s.dcv >> 2, nrg = nv ? kConsumers / nv : 0;
+    const int nv = s.dcv >> 2, nrg = nv ? kAll / nv : 0;
     // rows of the slice handled at a time: what the stage ring holds of C^V rows, z slices and weighted z
     constexpr int kRing = NS * kStageBytes / 4;
     const int head_f = (2 * GH * np + GH + 3) & ~3;
@@ -1504,13 +1825,13 @@ __global__ void __launch_bounds__(kThreads, OCC) decode_fft_kernel(const __grid_
     float* cvg = s.dcv > 0 ? coef_rows(c.coef_v, s, b, h, s.dcv) + (size_t)m0 * s.dcv : nullptr;
     auto stage_cv = [&](int r0, int cr) {
 #pragma unroll 1
-        for (int i = tid; i < cr * nv; i += kConsumers) cp_async16(cv_s + 4 * i, cvg + (size_t)r0 * s.dcv + 4 * i);
+        for (int i = tid; i < cr * nv; i += kAll) cp_async16(cv_s + 4 * i, cvg + (size_t)r0 * s.dcv + 4 * i);
     };
 
     if (s.dcv > 0) stage_cv(0, min(rows, mch));            // under the barrier
-    part_arrive(bar + 1, np, tid);
+    part_arrive<kAll>(bar + 1, np, tid);
     TL(16);
-    part_wait(bar + 1, np, tid, fail, c.status);
+    part_wait<kAll>(bar + 1, np, tid, fail, c.status);
     TL(17);
     // Fused step: every part of this (b, KV head) has read the row that leaves the window and is past its token
     // loop, so the rows the push moves can be written to the cache now, each by the part that owns it.
@@ -1519,9 +1840,9 @@ __global__ void __launch_bounds__(kThreads, OCC) decode_fft_kernel(const __grid_
             bf16* dk = mid_row<bf16>(c.k_mid, s, b, h, cstar, astar, s.nfk);
             bf16* dv = mid_row<bf16>(c.v_mid, s, b, h, cstar, astar, s.nfv);
 #pragma unroll 1
-            for (int e = tid; e < s.nfk; e += kConsumers) dk[e] = xrow_s[c.idx_full_k[(size_t)h * s.nfk + e]];
+            for (int e = tid; e < s.nfk; e += kAll) dk[e] = xrow_s[c.idx_full_k[(size_t)h * s.nfk + e]];
 #pragma unroll 1
-            for (int e = tid; e < s.nfv; e += kConsumers) dv[v_mid_col(astar, e, s.nfv, FA_BF16)] = xrow_s[s.d + c.idx_full_v[(size_t)h * s.nfv + e]];
+            for (int e = tid; e < s.nfv; e += kAll) dv[v_mid_col(astar, e, s.nfv, FA_BF16)] = xrow_s[s.d + c.idx_full_v[(size_t)h * s.nfv + e]];
         }
         if (new_buf >= 0 && new_tok >= w0 && new_tok < w1 && tid < 2 * (s.d >> 3)) {
             const int side = tid / (s.d >> 3), ch = tid - side * (s.d >> 3);
@@ -1531,7 +1852,7 @@ __global__ void __launch_bounds__(kThreads, OCC) decode_fft_kernel(const __grid_
         }
     }
 #pragma unroll 1
-    for (int i = tid; i < GH * np; i += kConsumers) {
+    for (int i = tid; i < GH * np; i += kAll) {
         float2 ml = make_float2(kNegBig, 0.f);
         if (i / np < ng) ml = __ldcg(reinterpret_cast<const float2*>(ws.ml + (qh0 * np + i) * 2));
         al_s[i] = ml.x;
@@ -1545,21 +1866,21 @@ __global__ void __launch_bounds__(kThreads, OCC) decode_fft_kernel(const __grid_
         const int cr = max(0, min(rows - r0, mch));
         if (s.dcv > 0) {
             if (r0 > 0) {
-                consumer_sync();                           // the previous chunk has been consumed
+                all_sync();                           // the previous chunk has been consumed
                 stage_cv(r0, cr);
             }
             const int r4 = cr >> 2;
 #pragma unroll 1
-            for (int i = tid; i < GH * np * r4; i += kConsumers) {
+            for (int i = tid; i < GH * np * r4; i += kAll) {
                 const int gs = i / r4, j = i - gs * r4, g = gs / np;
                 if (g < ng) cp_async16(zs_s + gs * mch + 4 * j, ws.z + (qh0 * np + gs) * s.M + m0 + r0 + 4 * j);
             }
         }
         cp_async_wait_all();
-        consumer_sync();
+        all_sync();
         if (j_pend >= 0 && s.dcv > 0) {                    // fused step: pending rank-1 update of these rows of C^V
 #pragma unroll 1
-            for (int i = tid; i < cr * nv; i += kConsumers) {
+            for (int i = tid; i < cr * nv; i += kAll) {
                 const int r = i / nv, v = i - r * nv;
                 const float f = f_row(r0 + r);
                 float4 x = *reinterpret_cast<const float4*>(cv_s + 4 * i);
@@ -1586,10 +1907,10 @@ __global__ void __launch_bounds__(kThreads, OCC) decode_fft_kernel(const __grid_
                 if (lane == 0) linv_s[warp] = Lsum > 0.f ? __fdividef(1.0f, Lsum) : 0.f;
             }
         }
-        consumer_sync();
+        all_sync();
         if (s.dcv > 0) {
 #pragma unroll 1
-            for (int t = tid; t < GH * cr; t += kConsumers) {
+            for (int t = tid; t < GH * cr; t += kAll) {
                 const int g = t / cr, r = t - g * cr;
                 float v = 0.f;
                 if (g < ng) {
@@ -1600,7 +1921,7 @@ __global__ void __launch_bounds__(kThreads, OCC) decode_fft_kernel(const __grid_
                 }
                 zw_s[g * mch + r] = v;
             }
-            consumer_sync();
+            all_sync();
             if (tid < nrg * nv) {
                 const int v = tid % nv, rgi = tid / nv;
 #pragma unroll 1
@@ -1624,9 +1945,9 @@ __global__ void __launch_bounds__(kThreads, OCC) decode_fft_kernel(const __grid_
 #pragma unroll
             for (int g = 0; g < GH; ++g) *reinterpret_cast<float4*>(ps_s + (rgi * GH + g) * s.dcv + 4 * v) = acc4[g];
         }
-        consumer_sync();
+        all_sync();
 #pragma unroll 1
-        for (int t = tid; t < GH * s.dcv; t += kConsumers) {
+        for (int t = tid; t < GH * s.dcv; t += kAll) {
             const int g = t / s.dcv, e = t - g * s.dcv;
             float v = 0.f;
 #pragma unroll 1
@@ -1636,7 +1957,7 @@ __global__ void __launch_bounds__(kThreads, OCC) decode_fft_kernel(const __grid_
     }
     TL(18);
     // ticket: the last part to get here finishes the rows
-    consumer_sync();
+    all_sync();
     if (tid == 0) {
         int old = 0;
         if (np > 1) {
@@ -1645,7 +1966,7 @@ __global__ void __launch_bounds__(kThreads, OCC) decode_fft_kernel(const __grid_
         }
         *last_s = old == np - 1;
     }
-    consumer_sync();
+    all_sync();
     TL(19);
     if (!*last_s) { SPAN(2); return; }
     float* op_s = zw_s;                                    // [GH][np][d] (the slice buffers are free again)
@@ -1654,22 +1975,22 @@ __global__ void __launch_bounds__(kThreads, OCC) decode_fft_kernel(const __grid_
     {
         const int nd4 = s.d >> 2;
 #pragma unroll 1
-        for (int i = tid; i < ng * np * nd4; i += kConsumers) cp_async16(op_s + 4 * i, ws.o + qh0 * np * s.d + 4 * i);
+        for (int i = tid; i < ng * np * nd4; i += kAll) cp_async16(op_s + 4 * i, ws.o + qh0 * np * s.d + 4 * i);
 #pragma unroll 1
-        for (int i = tid; i < ng * np * nv; i += kConsumers) cp_async16(ocp_s + 4 * i, ws.oc + qh0 * np * s.dcv + 4 * i);
+        for (int i = tid; i < ng * np * nv; i += kAll) cp_async16(ocp_s + 4 * i, ws.oc + qh0 * np * s.dcv + 4 * i);
     }
 #pragma unroll 1
-    for (int e = tid; e < s.d; e += kConsumers) inv_s[e] = -1;
-    consumer_sync();
+    for (int e = tid; e < s.d; e += kAll) inv_s[e] = -1;
+    all_sync();
     if (s.dcv > 0) {
         const int32_t* idc_v = c.idx_comp_v + (size_t)h * s.dcv;
 #pragma unroll 1
-        for (int e = tid; e < s.dcv; e += kConsumers) inv_s[idc_v[e]] = e;
+        for (int e = tid; e < s.dcv; e += kAll) inv_s[idc_v[e]] = e;
     }
     cp_async_wait_all();
-    consumer_sync();
+    all_sync();
 #pragma unroll 1
-    for (int t = tid; t < ng * s.d; t += kConsumers) {
+    for (int t = tid; t < ng * s.d; t += kAll) {
         const int g = t / s.d, e = t - g * s.d;
         const float* o = op_s + g * np * s.d + e;
         float v = 0.f;
@@ -1715,11 +2036,11 @@ static int coop_pdl_state(int set) {
     return state[dev];
 }
 
-template <int GH, int LS, int OCC, bool STEP>
+template <int GH, int LS, int OCC, bool STEP, bool SPLIT = false>
 cudaError_t launch_fft_t(const Dims& s, const CacheDev& c, const DecodePlan& p, const void* q, void* out, char* ws, int step,
                          const void* k_new, const void* v_new, cudaStream_t st) {
-    const FftSmem L = fft_smem_layout(LS, s.k, GH, p.nb, s.d, OCC);
-    cudaError_t err = ensure_dynamic_smem(decode_fft_kernel<GH, LS, OCC, STEP>, (size_t)L.total);
+    const FftSmem L = fft_smem_layout(LS, s.k, GH, p.nb, s.d, OCC, SPLIT ? 1 : 0);
+    cudaError_t err = ensure_dynamic_smem(decode_fft_kernel<GH, LS, OCC, STEP, SPLIT>, (size_t)L.total);
     if (err != cudaSuccess) return err;
     // window buffers as tensor maps (cached per buffer)
     CUtensorMap tki, tvi, tkl, tvl;
@@ -1729,7 +2050,7 @@ cudaError_t launch_fft_t(const Dims& s, const CacheDev& c, const DecodePlan& p, 
     if ((s.l_init > 0 && !ok_i) || (s.l_local > 0 && !ok_l)) return cudaErrorInvalidValue;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(p.n_part, s.Hkv * p.n_pass, s.B);
-    cfg.blockDim = dim3(kThreads);
+    cfg.blockDim = dim3(threads_of(SPLIT));
     cfg.dynamicSmemBytes = (size_t)L.total;
     cfg.stream = st;
     // Programmatic dependent launch: the kernel may be scheduled while its predecessor in the stream
@@ -1750,7 +2071,7 @@ cudaError_t launch_fft_t(const Dims& s, const CacheDev& c, const DecodePlan& p, 
             cfg.attrs = attr + 1;                                          // not probed yet: stay on the plain cooperative launch
         } else if (known != 0) {
             cfg.numAttrs = 2;
-            cudaError_t err2 = cudaLaunchKernelEx(&cfg, decode_fft_kernel<GH, LS, OCC, STEP>, tki, tvi, tkl, tvl, s, c, p,
+            cudaError_t err2 = cudaLaunchKernelEx(&cfg, decode_fft_kernel<GH, LS, OCC, STEP, SPLIT>, tki, tvi, tkl, tvl, s, c, p,
                                                   static_cast<const bf16*>(q), static_cast<bf16*>(out), ws,
                                                   static_cast<const bf16*>(k_new), static_cast<const bf16*>(v_new));
             if (err2 == cudaSuccess) { coop_pdl_state(1); return err2; }
@@ -1763,7 +2084,7 @@ cudaError_t launch_fft_t(const Dims& s, const CacheDev& c, const DecodePlan& p, 
             cfg.attrs = attr + 1;
         }
     }
-    return cudaLaunchKernelEx(&cfg, decode_fft_kernel<GH, LS, OCC, STEP>, tki, tvi, tkl, tvl, s, c, p, static_cast<const bf16*>(q),
+    return cudaLaunchKernelEx(&cfg, decode_fft_kernel<GH, LS, OCC, STEP, SPLIT>, tki, tvi, tkl, tvl, s, c, p, static_cast<const bf16*>(q),
                               static_cast<bf16*>(out), ws, static_cast<const bf16*>(k_new), static_cast<const bf16*>(v_new));
 }
 
@@ -1775,29 +2096,32 @@ cudaError_t launch_fft_ls(const Dims& s, const CacheDev& c, const DecodePlan& p,
         case 6: return p.occ == 2 ? (step ? launch_fft_t<GH, 6, 2, true>(s, c, p, q, out, ws, step, k_new, v_new, st) : launch_fft_t<GH, 6, 2, false>(s, c, p, q, out, ws, step, k_new, v_new, st)) : (step ? launch_fft_t<GH, 6, 1, true>(s, c, p, q, out, ws, step, k_new, v_new, st) : launch_fft_t<GH, 6, 1, false>(s, c, p, q, out, ws, step, k_new, v_new, st));
         case 7: return p.occ == 2 ? (step ? launch_fft_t<GH, 7, 2, true>(s, c, p, q, out, ws, step, k_new, v_new, st) : launch_fft_t<GH, 7, 2, false>(s, c, p, q, out, ws, step, k_new, v_new, st)) : (step ? launch_fft_t<GH, 7, 1, true>(s, c, p, q, out, ws, step, k_new, v_new, st) : launch_fft_t<GH, 7, 1, false>(s, c, p, q, out, ws, step, k_new, v_new, st));
         case 8: return p.occ == 2 ? (step ? launch_fft_t<GH, 8, 2, true>(s, c, p, q, out, ws, step, k_new, v_new, st) : launch_fft_t<GH, 8, 2, false>(s, c, p, q, out, ws, step, k_new, v_new, st)) : (step ? launch_fft_t<GH, 8, 1, true>(s, c, p, q, out, ws, step, k_new, v_new, st) : launch_fft_t<GH, 8, 1, false>(s, c, p, q, out, ws, step, k_new, v_new, st));
-        case 9: return (step ? launch_fft_t<GH, 9, 1, true>(s, c, p, q, out, ws, step, k_new, v_new, st) : launch_fft_t<GH, 9, 1, false>(s, c, p, q, out, ws, step, k_new, v_new, st));
-        case 10: return (step ? launch_fft_t<GH, 10, 1, true>(s, c, p, q, out, ws, step, k_new, v_new, st) : launch_fft_t<GH, 10, 1, false>(s, c, p, q, out, ws, step, k_new, v_new, st));
+        case 9:
+            return (step ? launch_fft_t<GH, 9, 1, true>(s, c, p, q, out, ws, step, k_new, v_new, st) : launch_fft_t<GH, 9, 1, false>(s, c, p, q, out, ws, step, k_new, v_new, st));
+        case 10:
+            if (p.split && !step) return launch_fft_t<GH, 10, 1, false, true>(s, c, p, q, out, ws, step, k_new, v_new, st);
+            return (step ? launch_fft_t<GH, 10, 1, true>(s, c, p, q, out, ws, step, k_new, v_new, st) : launch_fft_t<GH, 10, 1, false>(s, c, p, q, out, ws, step, k_new, v_new, st));
         default: return cudaErrorInvalidValue;
     }
 }
 
 // Resident CTAs of this kernel instance on the whole device for the plan's shared memory (cached per instance).
-template <int GH, int LS, int OCC, bool STEP = true>
+template <int GH, int LS, int OCC, bool SPLIT = false, bool STEP = true>
 int resident_ctas_t(const Dims& s, const DecodePlan& p) {
     // answers cached per (device, shared memory size) of this instance
     struct Entry { int dev; size_t smem; int ctas; };
     static Entry table[16];
     static int used = 0;
     static std::mutex mu;
-    const size_t smem = (size_t)fft_smem_layout(LS, s.k, GH, p.nb, s.d, OCC).total;
+    const size_t smem = (size_t)fft_smem_layout(LS, s.k, GH, p.nb, s.d, OCC, SPLIT ? 1 : 0).total;
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess) { cudaGetLastError(); return 0; }
     std::lock_guard<std::mutex> lock(mu);
     for (int i = 0; i < used; ++i)
         if (table[i].dev == dev && table[i].smem == smem) return table[i].ctas;
-    if (ensure_dynamic_smem(decode_fft_kernel<GH, LS, OCC, STEP>, smem) != cudaSuccess) { cudaGetLastError(); return 0; }
+    if (ensure_dynamic_smem(decode_fft_kernel<GH, LS, OCC, STEP, SPLIT>, smem) != cudaSuccess) { cudaGetLastError(); return 0; }
     int per_sm = 0;
-    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, decode_fft_kernel<GH, LS, OCC, STEP>, kThreads, smem) != cudaSuccess) {
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, decode_fft_kernel<GH, LS, OCC, STEP, SPLIT>, threads_of(SPLIT), smem) != cudaSuccess) {
         cudaGetLastError();
         return 0;
     }
@@ -1813,7 +2137,7 @@ int resident_ctas_ls(const Dims& s, const DecodePlan& p) {
         case 7: return p.occ == 2 ? resident_ctas_t<GH, 7, 2>(s, p) : resident_ctas_t<GH, 7, 1>(s, p);
         case 8: return p.occ == 2 ? resident_ctas_t<GH, 8, 2>(s, p) : resident_ctas_t<GH, 8, 1>(s, p);
         case 9: return resident_ctas_t<GH, 9, 1>(s, p);
-        case 10: return resident_ctas_t<GH, 10, 1>(s, p);
+        case 10: return p.split ? resident_ctas_t<GH, 10, 1, true, false>(s, p) : resident_ctas_t<GH, 10, 1>(s, p);
         default: return 0;
     }
 }
@@ -1831,19 +2155,19 @@ bool decode_fft_launchable(const Dims& s, const DecodePlan& p) {
     return grid <= resident;
 }
 
-size_t decode_fft_smem_bytes(const Dims& s, int log2S, int gh, int nb, int occ) {
-    return (size_t)fft_smem_layout(log2S, s.k, gh, nb, s.d, occ).total;
+size_t decode_fft_smem_bytes(const Dims& s, int log2S, int gh, int nb, int occ, int split) {
+    return (size_t)fft_smem_layout(log2S, s.k, gh, nb, s.d, occ, split).total;
 }
 
 // True if the fused kernel's staging areas hold a part's share of the coefficient rows: the rows
 // of C^K in the transform buffers at the start, the merge scratch in the stage ring at the end.
-bool decode_fft_fused_fits(const Dims& s, int log2S, int gh, int nb, int n_part, int occ) {
+bool decode_fft_fused_fits(const Dims& s, int log2S, int gh, int nb, int n_part, int occ, int split) {
     if (s.M % 4 != 0) return false;
     if (occ == 2 && log2S > 8) return false;                                           // no two-per-SM build of the long transforms
-    const FftSmem L = fft_smem_layout(log2S, s.k, gh, nb, s.d, occ);
+    const FftSmem L = fft_smem_layout(log2S, s.k, gh, nb, s.d, occ, split);
     if (s.dck > 0 && (long long)nb * L.fb_floats < 8LL * s.dck) return false;           // at least eight rows of C^K per chunk
-    const long long ring = (long long)ring_stages(occ) * kStageBytes / 4;
-    const long long nrg = s.dcv ? kConsumers / (s.dcv >> 2) : 0;
+    const long long ring = (long long)(ring_stages(occ) - (split ? 1 : 0)) * kStageBytes / 4;
+    const long long nrg = s.dcv ? (split ? kSplitConsumers : kConsumers) / (s.dcv >> 2) : 0;
     const long long head = ((2LL * gh * n_part + gh + 3) & ~3LL);
     if (s.dcv > 0 && (ring - head - nrg * gh * s.dcv) / (gh + s.dcv + (long long)gh * n_part) < 8) return false;   // and of C^V
     const long long step2 = (long long)gh * n_part * (s.d + s.dcv) + s.d;               // the last part's merge of all parts
