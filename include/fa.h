@@ -283,7 +283,8 @@ size_t fa_static_workspace_limit(void);
 fa_status fa_poll_status(const fa_cache* cache, void* stream);
 
 /* Number of kernels one call launches for this layout (what = 0 compress, 1 append,
- * 2 decode, 3 decode step); for launch accounting by callers. */
+ * 2 decode, 3 decode step); for launch accounting by callers.  what = 4 asks about the plan instead:
+ * 1 if fa_decode_attention runs the split build of the fused kernel for this layout, else 0. */
 int fa_launch_count(const fa_layout* layout, int what);
 
 const char* fa_status_string(fa_status s);

@@ -668,6 +668,11 @@ int fa_launch_count(const fa_layout* layout, int what) {
             if (plan_decode(*layout, &p) != FA_OK) return 0;
             return (p.fused && p.n_pass == 1 && p.n_part >= kStepFusedMinParts) ? 1 : 1 + (p.fused ? 1 : 3);
         }
+        case 4: {           // plan query: the split build of the fused decode kernel
+            DecodePlan p;
+            if (plan_decode(*layout, &p) != FA_OK) return 0;
+            return (p.fused && p.split) ? 1 : 0;
+        }
         default: return 0;
     }
 }

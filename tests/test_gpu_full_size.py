@@ -83,6 +83,7 @@ def test_128k_batch4_one_sampled_head():
     oracle recomputes one (batch row, KV head)."""
     shape = synth.CONFIGS[4]
     layout = layout_of(shape, max_mid=shape.T, P=shape.T // shape.k)
+    assert fa.fa_launch_count(layout, 4) == 1                  # the split build of the fused kernel serves this shape
     _sampled_head_check(shape, layout, heads=(5,), steps=2, seed=4000, rows=(3,))
 
 

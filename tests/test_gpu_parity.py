@@ -409,6 +409,21 @@ def test_fused_decode_more_heads_than_sms(T, P, M):
     pair.check_state()
 
 
+def test_fused_decode_split_build_long_transforms():
+    """Transform length 1024 with several class batches per CTA takes the split build of the fused kernel (a tile group
+    of warps forms the kept-dim products of the next batch while the transform group works on this one; two sets of
+    score / probability buffers).  Here GH = 2 and two classes per batch; the 128K configuration of the full-size
+    tests runs it with GH = 4 and one class per batch."""
+    shape = SMALL_BF16.with_(B=4, Hq=16, Hkv=8, L=4200, T=16384, M=512, n_full_k=32, n_full_v=48, decode_steps=2)
+    pair, stream = make_pair(shape, seed=27, algo=fa.FA_DECODE_FFT, P=16, max_mid=16384)
+    assert fa.fa_launch_count(pair.layout, 2) == 1 and fa.fa_launch_count(pair.layout, 4) == 1
+    pair.check_decode(synth.queries(shape, seed=27))
+    K, V = stream.tokens(shape.L, shape.L + 2)
+    for t in range(2):
+        pair.check_step(synth.queries(shape, seed=27, step=t + 1), K[:, t], V[:, t])
+    pair.check_state()
+
+
 @pytest.mark.parametrize("B", [1, 3])
 def test_fused_decode_two_ctas_per_sm_cooperative(B):
     """Short transforms with fewer heads than SMs: a head's parts are two to an SM and still wait for one
