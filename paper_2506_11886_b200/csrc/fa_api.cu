@@ -212,10 +212,12 @@ fa_status plan_decode(const fa_layout& l, DecodePlan* p) {
             p->n_split = best;
             p->nb = pick_nb(best);
         }
-        // Split build of the fused kernel (one CTA per SM): six more warps form the kept-dim products of the next batch of
-        // classes while the eight transform warps work on this one, with a second set of score / probability buffers
-        // in place of one ring stage.  It pays where the transform batch does not shrink to make room for those buffers
-        // (the transform phases are not faster on fewer classes) and a CTA has several batches: the longest transforms.
+        // Split build of the fused kernel (one CTA per SM): six more warps (the tile group) form the kept-dim products
+        // of a batch of classes beside the eight transform warps: the scores under the batch's spectra and score
+        // transform, the V products under its probability transform and fold.  Measured: it pays for the longest
+        // transforms when a CTA has several batches (their products then hide completely); with one batch per CTA
+        // the score products already run under the wait for the head's u rows and six warps form them slower than
+        // eight, and the shorter transforms lose more to the tile group's issue slots than the V products cost.
         if (p->fused && p->occ == 1 && log2S == 10) {
             const int per_cta = (s.P + p->n_split - 1) / p->n_split;
             if (per_cta >= 2 * p->nb && decode_fft_smem_bytes(s, log2S, p->gh, p->nb, 1, 1) <= 227 * 1024 &&

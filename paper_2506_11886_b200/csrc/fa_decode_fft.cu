@@ -70,7 +70,7 @@ namespace {
 constexpr int kConsumers = 256;
 constexpr int kWarps = kConsumers / 32;
 constexpr int kThreads = kConsumers + 32;
-// The split kernel: the eight warps above are the transform group, four more consume the ring tiles (kept-dim products).
+// The split kernel: the eight warps above are the transform group, six more consume the ring tiles (kept-dim products).
 constexpr int kSplitConsumers = kConsumers + 192;
 constexpr int kSplitWarps = kSplitConsumers / 32;
 __host__ __device__ constexpr int threads_of(bool split) { return (split ? kSplitConsumers : kConsumers) + 32; }
@@ -434,12 +434,12 @@ __host__ __device__ inline FftSmem fft_smem_layout(int log2S, int k, int GH, int
     int off = 256;                                        // mbarriers + flags
     L.zero_off = off; off += 16;
     off = 1024;                                           // stages are 1024-byte aligned (swizzled window tiles)
-    L.stages_off = off; off += (ring_stages(occ) - (split ? 1 : 0)) * kStageBytes;   // split kernel: a stage goes to the second buffers
+    L.stages_off = off; off += ring_stages(occ) * kStageBytes;
     L.fbuf_off = off; off += 4 * NB * L.fb_floats;
     off = (off + 15) / 16 * 16;
-    L.kb_off = off; off += (split ? 2 : 1) * 4 * NB * S * GH;   // kept-dim scores of the batch, natural token order (split kernel: two batches)
+    L.kb_off = off; off += 4 * NB * S * GH;               // kept-dim scores of the batch, natural token order
     off = (off + 15) / 16 * 16;
-    L.pbt_off = off; off += (split ? 2 : 1) * 2 * NB * GH * L.pbs;
+    L.pbt_off = off; off += 2 * NB * GH * L.pbs;
     off = (off + 15) / 16 * 16;
     L.twf_off = off; off += 8 * (tw_total(log2S) + 1);
     L.rev_off = off; off += 2 * S;
@@ -471,9 +471,9 @@ __global__ void __launch_bounds__(threads_of(SPLIT), OCC) decode_fft_kernel(cons
     constexpr bool step = STEP;
     constexpr int N = GH / 2;
     constexpr int S = 1 << LS;
-    constexpr int NS = ring_stages(OCC) - (SPLIT ? 1 : 0);
+    constexpr int NS = ring_stages(OCC);
     // Consumer threads: kAll of them; the warps that consume ring tiles (kept-dim and window products) are all of them,
-    // or, in the split kernel, the last four, while the first eight (the transform group) run the compressed-dim phases
+    // or, in the split kernel, the last six, while the first eight (the transform group) run the compressed-dim phases
     // of the class batches beside them.
     constexpr int kAll = SPLIT ? kSplitConsumers : kConsumers, kAllW = kAll / 32, kAllT = kAll + 32;
     constexpr int kMW = SPLIT ? kAllW - kWarps : kWarps, kM0 = SPLIT ? kWarps : 0;
@@ -646,7 +646,7 @@ __global__ void __launch_bounds__(threads_of(SPLIT), OCC) decode_fft_kernel(cons
         for (int i = 0; i < NS; ++i) { mbar_init(full + i, 1); mbar_init(empty + i, kMW); }
         if constexpr (SPLIT) {                            // the handshakes between the tile group and the transform group
             uint64_t* gb = reinterpret_cast<uint64_t*>(smem_raw + 160);
-            for (int i = 0; i < 2; ++i) { mbar_init(gb + i, kMW); mbar_init(gb + 2 + i, kWarps); mbar_init(gb + 4 + i, kWarps); mbar_init(gb + 6 + i, kMW); }
+            mbar_init(gb, kMW); mbar_init(gb + 1, kWarps); mbar_init(gb + 2, kWarps); mbar_init(gb + 3, kMW);   // kb_full, kb_free, p_full, p_free
         }
         *fail = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -709,21 +709,11 @@ __global__ void __launch_bounds__(threads_of(SPLIT), OCC) decode_fft_kernel(cons
                             ++it;
                         }
             }
-            if constexpr (!SPLIT) {
 #pragma unroll 1
-                for (int cb = c0; cb < c1; cb += NB) {
-                    const int nb = min(NB, c1 - cb);
-                    if (cb != c0) class_tiles(cb, nb, 0);
-                    class_tiles(cb, nb, 1);
-                }
-            } else {
-                // the tile group runs one batch of kept-dim scores ahead: K of batch 1, then V of batch i and K of batch i + 2
-                if (c0 + NB < c1) class_tiles(c0 + NB, min(NB, c1 - (c0 + NB)), 0);
-#pragma unroll 1
-                for (int cb = c0; cb < c1; cb += NB) {
-                    class_tiles(cb, min(NB, c1 - cb), 1);
-                    if (cb + 2 * NB < c1) class_tiles(cb + 2 * NB, min(NB, c1 - (cb + 2 * NB)), 0);
-                }
+            for (int cb = c0; cb < c1; cb += NB) {
+                const int nb = min(NB, c1 - cb);
+                if (cb != c0) class_tiles(cb, nb, 0);
+                class_tiles(cb, nb, 1);
             }
         }
         return;
@@ -1452,45 +1442,47 @@ __global__ void __launch_bounds__(threads_of(SPLIT), OCC) decode_fft_kernel(cons
             all_sync();
         }
         } else {
-            // ---- split kernel: the tile group (kept-dim products of batch i + 1 / i) beside the transform group ----
-            // Batches alternate between two buffers of kept-dim scores and of rounded probabilities.  Per buffer:
-            // kb_full (tile group -> transform group: the scores of the batch are in), kb_free (back: softmax has read
-            // them), p_full (transform group -> tile group: probabilities and the rescale factors of the batch are in),
-            // p_free (back: the V products have read them).  Batch 0's scores were formed before the window tokens.
+            // ---- split kernel: the tile group (kept-dim products) beside the transform group, batch by batch ----
+            // kb_full (tile group -> transform group: the kept-dim scores of the batch are in), kb_free (back: softmax has
+            // read them), p_full (transform group -> tile group: probabilities and the rescale factors of the batch are
+            // in), p_free (back: the V products have read them).  The scores of a batch are formed under its spectra and
+            // score transform, its V products run under its probability transform and fold (and the next batch's
+            // scores under that batch's spectra).  Batch 0's scores were formed before the window tokens.
             uint64_t* kb_full = reinterpret_cast<uint64_t*>(smem_raw + 160);
-            uint64_t* kb_free = kb_full + 2;
-            uint64_t* p_full = kb_free + 2;
-            uint64_t* p_free = p_full + 2;
-            float* alpha_s = reinterpret_cast<float*>(smem_raw + 224);     // [2][GH] rescale factors of a batch, per slot
+            uint64_t* kb_free = kb_full + 1;
+            uint64_t* p_full = kb_full + 2;
+            uint64_t* p_free = kb_full + 3;
+            float* alpha_s = reinterpret_cast<float*>(smem_raw + 224);     // [GH] rescale factors of a batch, per slot
             auto xf_sync = [] { consumer_sync<kConsumers, 2>(); };
             int n_bat = 0;
             for (int cb = c0; cb < c1 && n_of_class(cb) > 0; cb += NB) ++n_bat;
             if (is_m) {
                 // ================= tile group =================
-                if (n_bat > 1) {
-                    k_phase(c0 + NB, min(NB, c1 - (c0 + NB)), kb + NB * S * GH);
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(kb_full + 1);
-                }
                 #pragma unroll 1
                 for (int bi = 0; bi < n_bat; ++bi) {
-                    const int cb = c0 + bi * NB, nb = min(NB, c1 - cb), bb = bi & 1;
-                    if (lane == 0) mbar_wait(p_full + bb, (bi >> 1) & 1, fail, c.status);   // one lane polls, the warp follows
+                    const int cb = c0 + bi * NB, nb = min(NB, c1 - cb);
+                    if (bi >= 1) {
+                        if (lane == 0) mbar_wait(kb_free, (bi - 1) & 1, fail, c.status);   // softmax of the previous batch has read the scores
+                        __syncwarp();
+                        k_phase(cb, nb, kb);
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(kb_full);
+                    }
+                    if (lane == 0) mbar_wait(p_full, bi & 1, fail, c.status);   // one lane polls, the warp follows
                     __syncwarp();
                     {
-                        const float* al_b = alpha_s + bb * GH;
-                        const float al = al_b[(2 * tq) & (GH - 1)], ah = al_b[(2 * tq + 1) & (GH - 1)];
+                        const float al = alpha_s[(2 * tq) & (GH - 1)], ah = alpha_s[(2 * tq + 1) & (GH - 1)];
 #pragma unroll
                         for (int mt = 0; mt < 4; ++mt) { acc[mt][0] *= al; acc[mt][1] *= ah; acc[mt][2] *= al; acc[mt][3] *= ah; }
 #pragma unroll
-                        for (int g = 0; g < GH; ++g) l_acc[g] *= al_b[g];
+                        for (int g = 0; g < GH; ++g) l_acc[g] *= alpha_s[g];
                     }
             // o^u[dim][slot] += V^mu^T p, 16 tokens per mma
             if (ts_v) {
                 #pragma unroll 1
                 for (int ci = 0; ci < nb; ++ci) {
                     const int n_c = n_of_class(cb + ci);
-                    const uint32_t prow = p_lane + (uint32_t)(bb * NB * GH * pbs + ci * GH * pbs) * 2;
+                    const uint32_t prow = p_lane + (uint32_t)(ci * GH * pbs) * 2;
                     #pragma unroll 1
                     for (int a0 = 0; a0 < n_c; a0 += ts_v) {
                         const int nt = min(ts_v, n_c - a0);
@@ -1525,15 +1517,7 @@ __global__ void __launch_bounds__(threads_of(SPLIT), OCC) decode_fft_kernel(cons
                 }
             }
                     __syncwarp();
-                    if (lane == 0) mbar_arrive(p_free + bb);
-                    if (bi + 2 < n_bat) {
-                        const int cb2 = cb + 2 * NB;
-                        if (lane == 0) mbar_wait(kb_free + bb, (bi >> 1) & 1, fail, c.status);       // softmax of this batch has read the buffer
-                        __syncwarp();
-                        k_phase(cb2, min(NB, c1 - cb2), kb + bb * NB * S * GH);
-                        __syncwarp();
-                        if (lane == 0) mbar_arrive(kb_full + bb);
-                    }
+                    if (lane == 0) mbar_arrive(p_free);
                 }
             } else {
                 // ================= transform group =================
@@ -1557,9 +1541,9 @@ __global__ void __launch_bounds__(threads_of(SPLIT), OCC) decode_fft_kernel(cons
                 };
                 #pragma unroll 1
                 for (int bi = 0; bi < n_bat; ++bi) {
-                    const int cb = c0 + bi * NB, nb = min(NB, c1 - cb), bb = bi & 1;
-                    const float* kbuf = kb + bb * NB * S * GH;
-                    bf16* pbuf = pbt + bb * NB * GH * pbs;
+                    const int cb = c0 + bi * NB, nb = min(NB, c1 - cb);
+                    const float* kbuf = kb;
+                    bf16* pbuf = pbt;
             // packed Hermitian spectra of the nb classes: X_m = V^A_m + i V^B_m per complex lane,
             // V_m = v_m + conj(v_{S-m}), v_n = (1/2) u~_n e^{i theta n c}.  Pair 0 is bins (0, S/2).
             if (s.dck > 0) {
@@ -1607,7 +1591,7 @@ __global__ void __launch_bounds__(threads_of(SPLIT), OCC) decode_fft_kernel(cons
                     xf_sync();
                     // the kept-dim scores of this batch (batch 0: formed by everybody's earlier barriers)
                     if (bi >= 1) {
-                        if (tid == 0) mbar_wait(kb_full + bb, ((bi >> 1) - (bb == 0 ? 1 : 0)) & 1, fail, c.status);   // one thread polls
+                        if (tid == 0) mbar_wait(kb_full, (bi - 1) & 1, fail, c.status);   // one thread polls
                         xf_sync();
                     }
             // online softmax over the batch
@@ -1640,8 +1624,8 @@ __global__ void __launch_bounds__(threads_of(SPLIT), OCC) decode_fft_kernel(cons
                 m_run[g] = m_new;
                 l_acc[g] *= alpha[g];
             }
-            if (bi >= 2) {                                // the tile group is done with this buffer's previous batch
-                if (tid == 0) mbar_wait(p_free + bb, ((bi >> 1) - 1) & 1, fail, c.status);
+            if (bi >= 1) {                                // the tile group is done with the previous batch's probabilities
+                if (tid == 0) mbar_wait(p_free, (bi - 1) & 1, fail, c.status);
                 xf_sync();
             }
             #pragma unroll 1
@@ -1666,11 +1650,11 @@ __global__ void __launch_bounds__(threads_of(SPLIT), OCC) decode_fft_kernel(cons
                 for (int sl = 1; sl < GH; ++sl) if (hperm<GH>(sl) == g) a = alpha[sl];
                 o_s[i] = __float2ll_rn(__ll2float_rn(o_s[i]) * a);
             }
-                    if (tid < GH) alpha_s[bb * GH + tid] = alpha[0];
+                    if (tid < GH) alpha_s[tid] = alpha[0];
 #pragma unroll
-                    for (int g = 1; g < GH; ++g) if (tid == g) alpha_s[bb * GH + g] = alpha[g];
+                    for (int g = 1; g < GH; ++g) if (tid == g) alpha_s[g] = alpha[g];
                     xf_sync();
-                    if (lane == 0) { mbar_arrive(kb_free + bb); mbar_arrive(p_full + bb); }
+                    if (lane == 0) { mbar_arrive(kb_free); mbar_arrive(p_full); }
             // z_n = alpha z_n + sum_c e^{i theta n c} Y^c_n, Y^c = transform of the packed probabilities
             if (s.dcv > 0) {
                 fft_run<GH, LS, LS, true, 2>(fbuf, fb_floats, nb, twf, tid);
@@ -2099,7 +2083,7 @@ cudaError_t launch_fft_ls(const Dims& s, const CacheDev& c, const DecodePlan& p,
         case 9:
             return (step ? launch_fft_t<GH, 9, 1, true>(s, c, p, q, out, ws, step, k_new, v_new, st) : launch_fft_t<GH, 9, 1, false>(s, c, p, q, out, ws, step, k_new, v_new, st));
         case 10:
-            if (p.split && !step) return launch_fft_t<GH, 10, 1, false, true>(s, c, p, q, out, ws, step, k_new, v_new, st);
+            if (p.split) return (step ? launch_fft_t<GH, 10, 1, true, true>(s, c, p, q, out, ws, step, k_new, v_new, st) : launch_fft_t<GH, 10, 1, false, true>(s, c, p, q, out, ws, step, k_new, v_new, st));
             return (step ? launch_fft_t<GH, 10, 1, true>(s, c, p, q, out, ws, step, k_new, v_new, st) : launch_fft_t<GH, 10, 1, false>(s, c, p, q, out, ws, step, k_new, v_new, st));
         default: return cudaErrorInvalidValue;
     }
@@ -2166,7 +2150,7 @@ bool decode_fft_fused_fits(const Dims& s, int log2S, int gh, int nb, int n_part,
     if (occ == 2 && log2S > 8) return false;                                           // no two-per-SM build of the long transforms
     const FftSmem L = fft_smem_layout(log2S, s.k, gh, nb, s.d, occ, split);
     if (s.dck > 0 && (long long)nb * L.fb_floats < 8LL * s.dck) return false;           // at least eight rows of C^K per chunk
-    const long long ring = (long long)(ring_stages(occ) - (split ? 1 : 0)) * kStageBytes / 4;
+    const long long ring = (long long)ring_stages(occ) * kStageBytes / 4;
     const long long nrg = s.dcv ? (split ? kSplitConsumers : kConsumers) / (s.dcv >> 2) : 0;
     const long long head = ((2LL * gh * n_part + gh + 3) & ~3LL);
     if (s.dcv > 0 && (ring - head - nrg * gh * s.dcv) / (gh + s.dcv + (long long)gh * n_part) < 8) return false;   // and of C^V

@@ -411,9 +411,9 @@ def test_fused_decode_more_heads_than_sms(T, P, M):
 
 def test_fused_decode_split_build_long_transforms():
     """Transform length 1024 with several class batches per CTA takes the split build of the fused kernel (a tile group
-    of warps forms the kept-dim products of the next batch while the transform group works on this one; two sets of
-    score / probability buffers).  Here GH = 2 and two classes per batch; the 128K configuration of the full-size
-    tests runs it with GH = 4 and one class per batch."""
+    of warps forms the kept-dim products of a batch beside the transform group's phases on it, handshakes on four
+    shared-memory barriers), in the decode call and in the one-launch step.  Here GH = 2 and two classes per batch;
+    the 128K configuration of the full-size tests runs it with GH = 4 and one class per batch."""
     shape = SMALL_BF16.with_(B=4, Hq=16, Hkv=8, L=4200, T=16384, M=512, n_full_k=32, n_full_v=48, decode_steps=2)
     pair, stream = make_pair(shape, seed=27, algo=fa.FA_DECODE_FFT, P=16, max_mid=16384)
     assert fa.fa_launch_count(pair.layout, 2) == 1 and fa.fa_launch_count(pair.layout, 4) == 1
