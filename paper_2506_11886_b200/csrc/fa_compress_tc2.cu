@@ -27,13 +27,23 @@ constexpr int kGatherItems = 4;    // 16-byte chunks per gather thread and stage
 constexpr int kThreadsTc = 64 + 32 * (kGenWarps + kGatherWarps);
 using namespace umma;
 
+// Work of a launch: the token blocks of all (batch, head group) units, laid end to end: position = unit * blocks + block.
+// A TEAM is the M / 256 pairs that own the row tiles of the same blocks (they read the same boxes, in step, so the
+// prefill comes from HBM once); team t takes positions start[t] .. start[t + 1], a whole number of blocks that may
+// end inside a unit and go on into the next (one SEGMENT per unit touched: main loop, then an epilogue that adds the
+// segment's partial sums).  The table is cut on the host so that every team has the same cost (blocks + epilogues),
+// and so that teams x pairs fill the pairs that are resident at once; with per > 0 the cut is uniform instead
+// (start = t * per: one team per unit, every coefficient added to zero exactly once).
+constexpr int kMaxTeams = 96;
+struct TeamCuts { uint32_t start[kMaxTeams + 1]; };
+
 // D = head dim (64 or 128): N = 2 D accumulator columns per KV head (K dims, then V dims); HP heads share the pair
-// and its generated basis tiles (HP * N <= 512 tensor-memory columns).  grid (row tiles, Hkv / HP, B * n_tsplit),
-// clusters of two along x.
+// and its generated basis tiles (HP * N <= 512 tensor-memory columns).  grid 2 * teams * (M / 256), clusters of two.
 template <int D, int HP>
 __global__ void __launch_bounds__(kThreadsTc, 1) compress_tc2_kernel(const __grid_constant__ CUtensorMap tmK,
                                                                      const __grid_constant__ CUtensorMap tmV, Dims s,
-                                                                     CacheDev c, int L, int n_tsplit, int gather) {
+                                                                     CacheDev c, int L, const __grid_constant__ TeamCuts cuts,
+                                                                     int per, int gather) {
     constexpr int N = 2 * D;
     constexpr int kABytes = kBM * kBK * 2;                 // 16 KB basis tile
     constexpr int kBoxBytes = kBK * 64 * 2;                // 8 KB per [64 tokens x 64 dims] box
@@ -53,22 +63,32 @@ __global__ void __launch_bounds__(kThreadsTc, 1) compress_tc2_kernel(const __gri
     uint64_t* peer = full + kStagesTc;                     // even CTA: the odd CTA's stage is complete
     uint64_t* empty = peer + kStagesTc;
     uint64_t* acc_ready = empty + kStagesTc;
-    uint64_t* gather_done = acc_ready + 1;                 // the gather warps are past their last box
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(gather_done + 1);
+    uint64_t* gather_done = acc_ready + 1;                 // the gather warps are past the last box of the segment
+    uint64_t* epi_done = gather_done + 1;                  // the epilogue has left the stage ring (its scratch)
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(epi_done + 1);
     volatile int* fail = reinterpret_cast<volatile int*>(tmem_slot + 1);
     int* idf_s = reinterpret_cast<int*>(tmem_slot + 4);    // [HP][D]: the kept dims of this CTA's side of the CTA's heads
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int mt = blockIdx.x, h0 = blockIdx.y * HP;
     const uint32_t rank = cluster_ctarank();               // 0: K boxes, issues the MMAs; 1: V boxes
     const int side = (int)rank;
-    const int b = blockIdx.z / n_tsplit, split = blockIdx.z % n_tsplit;
+    const int n_pairs = s.M / (2 * kBM);                   // pairs of a team
+    const int cluster = (int)blockIdx.x >> 1, team = cluster / n_pairs, pair = cluster - team * n_pairs;
+    const int mt = 2 * pair + (int)rank;                   // this CTA's row tile, the same in every segment
+    const int n_hg = s.Hkv / HP;
     const int n_init = min(L, s.l_init);
     const int n_local = min(L - n_init, s.l_local);
     const int n_mid = L - n_init - n_local;
     const int nkb = (n_mid + kBK - 1) / kBK;
-    const int per = (nkb + n_tsplit - 1) / n_tsplit;
-    const int kb0 = split * per, kb1 = min(nkb, kb0 + per);
+    const uint32_t pos_begin = per > 0 ? (uint32_t)team * (uint32_t)per : cuts.start[team];
+    const uint32_t pos_end = per > 0 ? pos_begin + (uint32_t)per : cuts.start[team + 1];
+    // the segment that starts at position pos: its unit (batch b, heads h0 ...) and blocks kb0 .. kb1
+    struct Seg { int b, h0, kb0, kb1; };
+    auto seg_at = [&](uint32_t pos) {
+        const int unit = (int)(pos / (uint32_t)nkb), kb0 = (int)(pos - (uint32_t)unit * (uint32_t)nkb);
+        const int kb1 = (int)min((uint32_t)nkb, (uint32_t)kb0 + (pos_end - pos));
+        return Seg{unit / n_hg, (unit % n_hg) * HP, kb0, kb1};
+    };
 
     if (tid == 0) {
         // a stage is free again when the pair's MMAs have read it and this CTA's gather warps have taken their rows
@@ -79,15 +99,11 @@ __global__ void __launch_bounds__(kThreadsTc, 1) compress_tc2_kernel(const __gri
         }
         mbar_init(acc_ready, 1);
         mbar_init(gather_done, kGatherWarps);
+        mbar_init(epi_done, kGenWarps);
         *fail = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     const int nf_side = side ? s.nfv : s.nfk;
-    if (gather)
-        for (int i = tid; i < HP * nf_side; i += kThreadsTc) {
-            const int hh = i / nf_side, r = i - hh * nf_side;
-            idf_s[hh * D + r] = (side ? c.idx_full_v : c.idx_full_k)[(size_t)(h0 + hh) * nf_side + r];
-        }
     if (warp == 1) {                                       // tensor memory: one warp of each CTA of the pair, collectively
         asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(kTmemCols) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
@@ -98,55 +114,72 @@ __global__ void __launch_bounds__(kThreadsTc, 1) compress_tc2_kernel(const __gri
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     const uint32_t tmem_base = *tmem_slot;
 
-    if (kb1 > kb0) {
+    if (pos_end > pos_begin) {
         if (warp == 0) {
             // ---------------- TMA producer: this CTA's half of the B operand (one side, all D dims, 64 tokens) ----------------
             if (lane == 0) {
                 const CUtensorMap* tm = side ? &tmV : &tmK;
-                for (int kb = kb0; kb < kb1; ++kb) {
-                    const int it = kb - kb0, st = it % kStagesTc;
-                    if (it >= kStagesTc && !mbar_wait(empty + st, ((it / kStagesTc) - 1) & 1, fail, c.status)) break;
-                    unsigned char* bdst = stage0 + (size_t)st * kStageBytesTc + kABytes;
-                    mbar_expect_tx(full + st, (uint32_t)kBHalf);
-                    const int tok = n_init + kb * kBK;
+                int it = 0, seg = 0;
+                bool live = true;
+                for (uint32_t pos = pos_begin; live && pos < pos_end; ++seg) {
+                    const Seg g = seg_at(pos);
+                    // the epilogue of the segment before used the ring as its scratch
+                    if (seg > 0 && !mbar_wait(epi_done, (seg - 1) & 1, fail, c.status)) break;
+                    for (int kb = g.kb0; kb < g.kb1; ++kb, ++it) {
+                        const int st = it % kStagesTc;
+                        if (it >= kStagesTc && !mbar_wait(empty + st, ((it / kStagesTc) - 1) & 1, fail, c.status)) { live = false; break; }
+                        unsigned char* bdst = stage0 + (size_t)st * kStageBytesTc + kABytes;
+                        mbar_expect_tx(full + st, (uint32_t)kBHalf);
+                        const int tok = n_init + kb * kBK;
 #pragma unroll
-                    for (int hh = 0; hh < HP; ++hh)
+                        for (int hh = 0; hh < HP; ++hh)
 #pragma unroll
-                        for (int bx = 0; bx < D / 64; ++bx)
-                            tma_load_4d(bdst + hh * kBHalf1 + bx * kBoxBytes, tm, bx * 64, h0 + hh, tok, b, full + st);
+                            for (int bx = 0; bx < D / 64; ++bx)
+                                tma_load_4d(bdst + hh * kBHalf1 + bx * kBoxBytes, tm, bx * 64, g.h0 + hh, tok, g.b, full + st);
+                    }
+                    pos += (uint32_t)(g.kb1 - g.kb0);
                 }
             }
         } else if (warp == 1) {
             // ---------------- MMA issuer: the even CTA, for the pair ----------------
             if (lane == 0 && rank == 0) {
-                for (int kb = kb0; kb < kb1; ++kb) {
-                    const int it = kb - kb0, st = it % kStagesTc;
-                    const uint32_t par = (it / kStagesTc) & 1;
-                    if (!mbar_wait(full + st, par, fail, c.status) || !mbar_wait(peer + st, par, fail, c.status)) break;
-                    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-                    const uint32_t a_addr = smem_u32(stage0 + (size_t)st * kStageBytesTc);
-                    const uint32_t b_addr = a_addr + kABytes;
+                int it = 0;
+                bool live = true;
+                for (uint32_t pos = pos_begin; live && pos < pos_end;) {
+                    const Seg g = seg_at(pos);
+                    // The accumulators of the segment before have been read: the stage barriers below complete only
+                    // after the generator warps of both CTAs, which are the epilogue warps, are past that epilogue.
+                    for (int kb = g.kb0; kb < g.kb1; ++kb, ++it) {
+                        const int st = it % kStagesTc;
+                        const uint32_t par = (it / kStagesTc) & 1;
+                        if (!mbar_wait(full + st, par, fail, c.status) || !mbar_wait(peer + st, par, fail, c.status)) { live = false; break; }
+                        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                        const uint32_t a_addr = smem_u32(stage0 + (size_t)st * kStageBytesTc);
+                        const uint32_t b_addr = a_addr + kABytes;
 #pragma unroll
-                    for (int ks = 0; ks < kBK / 16; ++ks) {
-                        // A: K-major, rows of 128 bytes, 8-row groups 1024 bytes apart; 16 tokens = 32 bytes along the row
-                        // (the same offsets in both CTAs: each supplies its own 128 rows)
-                        const uint64_t adesc = umma_desc(a_addr + ks * 32, 1, 1024 >> 4);
-                        // B: MN-major, 64 dims per 128-byte row, 8-token groups 1024 bytes apart, next 64 dims one box
-                        // further; each CTA supplies D of the 2 D columns
+                        for (int ks = 0; ks < kBK / 16; ++ks) {
+                            // A: K-major, rows of 128 bytes, 8-row groups 1024 bytes apart; 16 tokens = 32 bytes along the row
+                            // (the same offsets in both CTAs: each supplies its own 128 rows)
+                            const uint64_t adesc = umma_desc(a_addr + ks * 32, 1, 1024 >> 4);
+                            // B: MN-major, 64 dims per 128-byte row, 8-token groups 1024 bytes apart, next 64 dims one box
+                            // further; each CTA supplies D of the 2 D columns
 #pragma unroll
-                        for (int hh = 0; hh < HP; ++hh) {
-                            const uint64_t bdesc = umma_desc(b_addr + hh * kBHalf1 + ks * 2048, kBoxBytes >> 4, 1024 >> 4);
-                            umma_bf16_pair(tmem_base + hh * N, adesc, bdesc, kIdesc, (it > 0 || ks > 0) ? 1u : 0u);
+                            for (int hh = 0; hh < HP; ++hh) {
+                                const uint64_t bdesc = umma_desc(b_addr + hh * kBHalf1 + ks * 2048, kBoxBytes >> 4, 1024 >> 4);
+                                umma_bf16_pair(tmem_base + hh * N, adesc, bdesc, kIdesc, (kb > g.kb0 || ks > 0) ? 1u : 0u);
+                            }
                         }
+                        umma_commit_pair(empty + st);      // frees the stage in both CTAs when these MMAs have read it
                     }
-                    umma_commit_pair(empty + st);          // frees the stage in both CTAs when these MMAs have read it
+                    if (live) umma_commit_pair(acc_ready);
+                    pos += (uint32_t)(g.kb1 - g.kb0);
                 }
-                umma_commit_pair(acc_ready);
             } else if (lane == 0) {
                 // the odd CTA's otherwise idle lane: when this CTA's basis tile and boxes of a stage are complete it tells
                 // the even CTA, which issues the MMAs (one remote arrival per stage, kept off the generators' path)
-                for (int kb = kb0; kb < kb1; ++kb) {
-                    const int it = kb - kb0, st = it % kStagesTc;
+                const int n_it = (int)(pos_end - pos_begin);
+                for (int it = 0; it < n_it; ++it) {
+                    const int st = it % kStagesTc;
                     const uint32_t par = (it / kStagesTc) & 1;
                     if (!mbar_wait(full + st, par, fail, c.status)) break;
                     mbar_arrive_cluster(peer + st, 0);
@@ -155,76 +188,92 @@ __global__ void __launch_bounds__(kThreadsTc, 1) compress_tc2_kernel(const __gri
         } else if (warp >= 2 + kGenWarps) {
             // ---------------- kept dims of the middle tokens: this CTA's boxes -> K^mu (even CTA) or V^mu (odd CTA) ----------------
             const int gt = tid - 32 * (2 + kGenWarps);           // 0 .. 32 kGatherWarps - 1
-            const int n_pairs = (int)gridDim.x >> 1, pair = mt >> 1;           // the pairs that load the same boxes share the tokens
             const int cph = nf_side >> 3;                                      // 16-byte chunks per kept-dim row of this side
-            const int n_tok = pair < kBK ? (kBK - pair + n_pairs - 1) / n_pairs : 0;   // tokens pair, pair + n_pairs, ... of a block
+            // the pairs of the team load the same boxes and share the tokens: this pair takes rows pair, pair + n_pairs, ...
+            const int n_tok = pair < kBK ? (kBK - pair + n_pairs - 1) / n_pairs : 0;
             const int n_items = gather ? n_tok * HP * cph : 0;                // <= kGatherItems per thread (checked on the host)
-            // An item = one 16-byte chunk (8 kept dims) of one kept-dim row.  A thread keeps the same items in every
-            // block: token row r of the boxes, head, side and LOGICAL chunk, so the eight source offsets inside a stage
-            // are constants (two 16-bit offsets per register); only the destination row moves with the token.
-            uint32_t src[kGatherItems][4];
-            int meta[kGatherItems];                        // r | hh << 8 | lch << 16, or -1
-#pragma unroll
-            for (int u = 0; u < kGatherItems; ++u) {
-                const int idx = gt + u * 32 * kGatherWarps;
-                meta[u] = -1;
-#pragma unroll
-                for (int i2 = 0; i2 < 4; ++i2) src[u][i2] = 0;
-                if (idx < n_items) {
-                    const int ti = idx / (HP * cph), rem = idx - ti * (HP * cph);
-                    const int hh = rem / cph, lch = rem - hh * cph;
-                    const int r = pair + n_pairs * ti;
-                    const int* idf = idf_s + hh * D + lch * 8;
-                    const uint32_t row0 = (uint32_t)(hh * kBHalf1 + r * 128);
-#pragma unroll
-                    for (int i2 = 0; i2 < 4; ++i2) {
-                        const int e0 = idf[2 * i2], e1 = idf[2 * i2 + 1];
-                        const uint32_t o0 = row0 + (uint32_t)((e0 >> 6) * kBoxBytes + ((((e0 & 63) >> 3) ^ (r & 7)) << 4) + (e0 & 7) * 2);
-                        const uint32_t o1 = row0 + (uint32_t)((e1 >> 6) * kBoxBytes + ((((e1 & 63) >> 3) ^ (r & 7)) << 4) + (e1 & 7) * 2);
-                        src[u][i2] = o0 | (o1 << 16);       // a stage is at most 64 KB
-                    }
-                    meta[u] = r | (hh << 8) | (lch << 16);
-                }
-            }
             const bool p2 = (s.P & (s.P - 1)) == 0;
             const int lgP = 31 - __clz(s.P);
-            for (int kb = kb0; kb < kb1; ++kb) {
-                const int it = kb - kb0, st = it % kStagesTc;
-                if (!mbar_wait(full + st, (it / kStagesTc) & 1, fail, c.status)) break;
-                const unsigned char* bsrc = stage0 + (size_t)st * kStageBytesTc + kABytes;
-                const int jb = kb * kBK;                   // first middle token of the block
-                uint4 val[kGatherItems];
+            int it = 0;
+            bool live = true;
+            // (after a wait that ran out the warp still walks the segments, without work: its partners count on it
+            // at the barrier below)
+            for (uint32_t pos = pos_begin; pos < pos_end;) {
+                const Seg g = seg_at(pos);
+                // the kept dims of this side of the segment's heads (the four gather warps, on their own barrier)
+                asm volatile("bar.sync 3, %0;" ::"n"(32 * kGatherWarps) : "memory");
+                if (gather)
+                    for (int i = gt; i < HP * nf_side; i += 32 * kGatherWarps) {
+                        const int hh = i / nf_side, r = i - hh * nf_side;
+                        idf_s[hh * D + r] = (side ? c.idx_full_v : c.idx_full_k)[(size_t)(g.h0 + hh) * nf_side + r];
+                    }
+                asm volatile("bar.sync 3, %0;" ::"n"(32 * kGatherWarps) : "memory");
+                // An item = one 16-byte chunk (8 kept dims) of one kept-dim row.  A thread keeps the same items in every
+                // block: token row r of the boxes, head, side and LOGICAL chunk, so the eight source offsets inside a stage
+                // are constants (two 16-bit offsets per register); only the destination row moves with the token.
+                uint32_t src[kGatherItems][4];
+                int meta[kGatherItems];                    // r | hh << 8 | lch << 16, or -1
 #pragma unroll
                 for (int u = 0; u < kGatherItems; ++u) {
-                    uint32_t w[4] = {0u, 0u, 0u, 0u};
-                    if (meta[u] >= 0) {
+                    const int idx = gt + u * 32 * kGatherWarps;
+                    meta[u] = -1;
+#pragma unroll
+                    for (int i2 = 0; i2 < 4; ++i2) src[u][i2] = 0;
+                    if (idx < n_items) {
+                        const int ti = idx / (HP * cph), rem = idx - ti * (HP * cph);
+                        const int hh = rem / cph, lch = rem - hh * cph;
+                        const int r = pair + n_pairs * ti;
+                        const int* idf = idf_s + hh * D + lch * 8;
+                        const uint32_t row0 = (uint32_t)(hh * kBHalf1 + r * 128);
 #pragma unroll
                         for (int i2 = 0; i2 < 4; ++i2) {
-                            const uint32_t lo = *reinterpret_cast<const uint16_t*>(bsrc + (src[u][i2] & 0xffffu));
-                            const uint32_t hi = *reinterpret_cast<const uint16_t*>(bsrc + (src[u][i2] >> 16));
-                            w[i2] = lo | (hi << 16);
+                            const int e0 = idf[2 * i2], e1 = idf[2 * i2 + 1];
+                            const uint32_t o0 = row0 + (uint32_t)((e0 >> 6) * kBoxBytes + ((((e0 & 63) >> 3) ^ (r & 7)) << 4) + (e0 & 7) * 2);
+                            const uint32_t o1 = row0 + (uint32_t)((e1 >> 6) * kBoxBytes + ((((e1 & 63) >> 3) ^ (r & 7)) << 4) + (e1 & 7) * 2);
+                            src[u][i2] = o0 | (o1 << 16);   // a stage is at most 64 KB
+                        }
+                        meta[u] = r | (hh << 8) | (lch << 16);
+                    }
+                }
+                for (int kb = g.kb0; live && kb < g.kb1; ++kb, ++it) {
+                    const int st = it % kStagesTc;
+                    if (!mbar_wait(full + st, (it / kStagesTc) & 1, fail, c.status)) { live = false; break; }
+                    const unsigned char* bsrc = stage0 + (size_t)st * kStageBytesTc + kABytes;
+                    const int jb = kb * kBK;               // first middle token of the block
+                    uint4 val[kGatherItems];
+#pragma unroll
+                    for (int u = 0; u < kGatherItems; ++u) {
+                        uint32_t w[4] = {0u, 0u, 0u, 0u};
+                        if (meta[u] >= 0) {
+#pragma unroll
+                            for (int i2 = 0; i2 < 4; ++i2) {
+                                const uint32_t lo = *reinterpret_cast<const uint16_t*>(bsrc + (src[u][i2] & 0xffffu));
+                                const uint32_t hi = *reinterpret_cast<const uint16_t*>(bsrc + (src[u][i2] >> 16));
+                                w[i2] = lo | (hi << 16);
+                            }
+                        }
+                        val[u] = make_uint4(w[0], w[1], w[2], w[3]);
+                    }
+                    __syncwarp();                          // the values are in registers: the stage goes back before the stores
+                    if (lane == 0) mbar_arrive(empty + st);
+#pragma unroll
+                    for (int u = 0; u < kGatherItems; ++u) {
+                        const int j = jb + (meta[u] & 0xff);
+                        if (meta[u] >= 0 && j < n_mid) {
+                            const int hh = (meta[u] >> 8) & 0xf, lch = meta[u] >> 16;
+                            const int cls = p2 ? (j & (s.P - 1)) : j % s.P, slot = p2 ? (j >> lgP) : j / s.P;
+                            const int nfull = nf_side;
+                            // logical chunk lch of a V^mu row is stored at chunk lch ^ swizzle
+                            const int ch = side ? (lch ^ v_swz(slot, nfull >> 3)) : lch;
+                            bf16* dst = mid_row<bf16>(side ? c.v_mid : c.k_mid, s, g.b, g.h0 + hh, cls, slot, nfull);
+                            reinterpret_cast<uint4*>(dst)[ch] = val[u];
                         }
                     }
-                    val[u] = make_uint4(w[0], w[1], w[2], w[3]);
                 }
-                __syncwarp();                              // the values are in registers: the stage goes back before the stores
-                if (lane == 0) mbar_arrive(empty + st);
-#pragma unroll
-                for (int u = 0; u < kGatherItems; ++u) {
-                    const int j = jb + (meta[u] & 0xff);
-                    if (meta[u] >= 0 && j < n_mid) {
-                        const int hh = (meta[u] >> 8) & 0xf, lch = meta[u] >> 16;
-                        const int cls = p2 ? (j & (s.P - 1)) : j % s.P, slot = p2 ? (j >> lgP) : j / s.P;
-                        const int nfull = nf_side;
-                        // logical chunk lch of a V^mu row is stored at chunk lch ^ swizzle
-                        const int ch = side ? (lch ^ v_swz(slot, nfull >> 3)) : lch;
-                        bf16* dst = mid_row<bf16>(side ? c.v_mid : c.k_mid, s, b, h0 + hh, cls, slot, nfull);
-                        reinterpret_cast<uint4*>(dst)[ch] = val[u];
-                    }
-                }
+                __syncwarp();
+                if (live && lane == 0) mbar_arrive(gather_done);
+                pos += (uint32_t)(g.kb1 - g.kb0);
             }
-            __syncwarp();
-            if (lane == 0) mbar_arrive(gather_done);
         } else {
             // ---------------- basis generators: A operand ----------------
             const int t = tid - 64;                        // 0 .. 32 kGenWarps - 1
@@ -252,110 +301,127 @@ __global__ void __launch_bounds__(kThreadsTc, 1) compress_tc2_kernel(const __gri
             // below the bf16 rounding of the tile).
             constexpr int kReseed = 8;
             unsigned long long C = 0, S = 0;
-            for (int kb = kb0; kb < kb1; ++kb) {
-                const int it = kb - kb0, st = it % kStagesTc;
-                if (it >= kStagesTc && !mbar_wait(empty + st, ((it / kStagesTc) - 1) & 1, fail, c.status)) break;
-                unsigned char* a_dst = stage0 + (size_t)st * kStageBytesTc;
-                const int j0 = kb * kBK + 16 * tqr;
-                if (it % kReseed == 0) {
-                    const unsigned pa = (n * (unsigned)j0) % (unsigned)s.T, pb = (n * (unsigned)(j0 + 1)) % (unsigned)s.T;
-                    const float fa = (float)pa * inv_T, fb = (float)pb * inv_T;
-                    const float aa = 6.283185307179586f * (fa - (fa >= 0.5f ? 1.0f : 0.0f));
-                    const float ab = 6.283185307179586f * (fb - (fb >= 0.5f ? 1.0f : 0.0f));
-                    asm("mov.b64 %0, {%1,%2};" : "=l"(C) : "f"(__cosf(aa)), "f"(__cosf(ab)));
-                    asm("mov.b64 %0, {%1,%2};" : "=l"(S) : "f"(__sinf(aa)), "f"(__sinf(ab)));
-                }
-                const bool whole = row_on && j0 + 16 <= n_mid;          // no masking needed in the common case
+            int it = 0, seg = 0;
+            bool live = true;
+            for (uint32_t pos = pos_begin; live && pos < pos_end; ++seg) {
+                const Seg g = seg_at(pos);
+                for (int kb = g.kb0; kb < g.kb1; ++kb, ++it) {
+                    const int st = it % kStagesTc;
+                    if (it >= kStagesTc && !mbar_wait(empty + st, ((it / kStagesTc) - 1) & 1, fail, c.status)) { live = false; break; }
+                    unsigned char* a_dst = stage0 + (size_t)st * kStageBytesTc;
+                    const int j0 = kb * kBK + 16 * tqr;
+                    if ((kb - g.kb0) % kReseed == 0) {
+                        const unsigned pa = (n * (unsigned)j0) % (unsigned)s.T, pb = (n * (unsigned)(j0 + 1)) % (unsigned)s.T;
+                        const float fa = (float)pa * inv_T, fb = (float)pb * inv_T;
+                        const float aa = 6.283185307179586f * (fa - (fa >= 0.5f ? 1.0f : 0.0f));
+                        const float ab = 6.283185307179586f * (fb - (fb >= 0.5f ? 1.0f : 0.0f));
+                        asm("mov.b64 %0, {%1,%2};" : "=l"(C) : "f"(__cosf(aa)), "f"(__cosf(ab)));
+                        asm("mov.b64 %0, {%1,%2};" : "=l"(S) : "f"(__sinf(aa)), "f"(__sinf(ab)));
+                    }
+                    const bool whole = row_on && j0 + 16 <= n_mid;      // no masking needed in the common case
 #pragma unroll
-                for (int ch = 0; ch < 2; ++ch) {           // 8 tokens = one 16-byte chunk of each row
-                    uint32_t wc[4], wsn[4];
+                    for (int ch = 0; ch < 2; ++ch) {       // 8 tokens = one 16-byte chunk of each row
+                        uint32_t wc[4], wsn[4];
 #pragma unroll
-                    for (int i2 = 0; i2 < 4; ++i2) {
-                        float c0, c1, s0, s1;
-                        asm("mov.b64 {%0,%1}, %2;" : "=f"(c0), "=f"(c1) : "l"(C));
-                        asm("mov.b64 {%0,%1}, %2;" : "=f"(s0), "=f"(s1) : "l"(S));
-                        if (!whole) {
-                            const int j = j0 + ch * 8 + i2 * 2;
-                            const bool v0 = row_on && j < n_mid, v1 = row_on && j + 1 < n_mid;
-                            c0 = v0 ? c0 : 0.f; s0 = v0 ? s0 : 0.f; c1 = v1 ? c1 : 0.f; s1 = v1 ? s1 : 0.f;
+                        for (int i2 = 0; i2 < 4; ++i2) {
+                            float c0, c1, s0, s1;
+                            asm("mov.b64 {%0,%1}, %2;" : "=f"(c0), "=f"(c1) : "l"(C));
+                            asm("mov.b64 {%0,%1}, %2;" : "=f"(s0), "=f"(s1) : "l"(S));
+                            if (!whole) {
+                                const int j = j0 + ch * 8 + i2 * 2;
+                                const bool v0 = row_on && j < n_mid, v1 = row_on && j + 1 < n_mid;
+                                c0 = v0 ? c0 : 0.f; s0 = v0 ? s0 : 0.f; c1 = v1 ? c1 : 0.f; s1 = v1 ? s1 : 0.f;
+                            }
+                            const __nv_bfloat162 pc = __floats2bfloat162_rn(c0, c1);
+                            const __nv_bfloat162 ps = __floats2bfloat162_rn(s0, s1);
+                            wc[i2] = *reinterpret_cast<const uint32_t*>(&pc);
+                            wsn[i2] = *reinterpret_cast<const uint32_t*>(&ps);
+                            // advance both phasors by two tokens: C' = C cs2 - S sn2, S' = S cs2 + C sn2
+                            unsigned long long tC, tS, nC, nS;
+                            asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(tC) : "l"(C), "l"(CS2));
+                            asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(tS) : "l"(S), "l"(CS2));
+                            asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(nC) : "l"(S), "l"(NSN2), "l"(tC));
+                            asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(nS) : "l"(C), "l"(SN2), "l"(tS));
+                            C = nC;
+                            S = nS;
                         }
-                        const __nv_bfloat162 pc = __floats2bfloat162_rn(c0, c1);
-                        const __nv_bfloat162 ps = __floats2bfloat162_rn(s0, s1);
-                        wc[i2] = *reinterpret_cast<const uint32_t*>(&pc);
-                        wsn[i2] = *reinterpret_cast<const uint32_t*>(&ps);
-                        // advance both phasors by two tokens: C' = C cs2 - S sn2, S' = S cs2 + C sn2
+                        const int chunk = 2 * tqr + ch;
+                        *reinterpret_cast<uint4*>(a_dst + row_off0 + ((chunk ^ (r0 & 7)) << 4)) = make_uint4(wc[0], wc[1], wc[2], wc[3]);
+                        *reinterpret_cast<uint4*>(a_dst + row_off1 + ((chunk ^ (r1 & 7)) << 4)) = make_uint4(wsn[0], wsn[1], wsn[2], wsn[3]);
+                    }
+                    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic stores -> visible to the tensor core
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(full + st);
+                    {                                      // on to the same run of the next block
                         unsigned long long tC, tS, nC, nS;
-                        asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(tC) : "l"(C), "l"(CS2));
-                        asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(tS) : "l"(S), "l"(CS2));
-                        asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(nC) : "l"(S), "l"(NSN2), "l"(tC));
-                        asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(nS) : "l"(C), "l"(SN2), "l"(tS));
+                        asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(tC) : "l"(C), "l"(CS48));
+                        asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(tS) : "l"(S), "l"(CS48));
+                        asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(nC) : "l"(S), "l"(NSN48), "l"(tC));
+                        asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(nS) : "l"(C), "l"(SN48), "l"(tS));
                         C = nC;
                         S = nS;
                     }
-                    const int chunk = 2 * tqr + ch;
-                    *reinterpret_cast<uint4*>(a_dst + row_off0 + ((chunk ^ (r0 & 7)) << 4)) = make_uint4(wc[0], wc[1], wc[2], wc[3]);
-                    *reinterpret_cast<uint4*>(a_dst + row_off1 + ((chunk ^ (r1 & 7)) << 4)) = make_uint4(wsn[0], wsn[1], wsn[2], wsn[3]);
                 }
-                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic stores -> visible to the tensor core
-                __syncwarp();
-                if (lane == 0) mbar_arrive(full + st);
-                {                                          // on to the same run of the next block
-                    unsigned long long tC, tS, nC, nS;
-                    asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(tC) : "l"(C), "l"(CS48));
-                    asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(tS) : "l"(S), "l"(CS48));
-                    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(nC) : "l"(S), "l"(NSN48), "l"(tC));
-                    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(nS) : "l"(C), "l"(SN48), "l"(tS));
-                    C = nC;
-                    S = nS;
-                }
-            }
-            // ---------------- epilogue: accumulators -> compressed columns ----------------
-            // the stage ring is reused below: every MMA has read it, and the gather warps have left it
-            const bool ok = mbar_wait(acc_ready, 0, fail, c.status) && mbar_wait(gather_done, 0, fail, c.status);
-            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-            // the coefficients are cleared by the partition kernel, which this launch may overlap: wait for it here
-            asm volatile("griddepcontrol.wait;" ::: "memory");
-            if (ok) {
-                const int lane_grp = warp & 3;             // a warp reads tensor-memory lanes 32 (warp % 4) ...
-                const int col_part = (warp - 2) >> 2;      // the two warps that share a lane group take half of the columns each
-                constexpr int kPart = (int)kTmemCols / (kGenWarps / 4);      // a whole number of sides (D columns each)
-                const int m_base = mt * kBM + lane_grp * 32;
-                // A thread holds 32 columns of ONE row of the accumulator.  The warp lays its 32 rows x D columns of one side
-                // (K or V of one head) out in the idle stage ring; then lane q owns the four compressed dims 4 q .. 4 q + 3
-                // (slots of D^c, ascending) and adds them row by row with one 16-byte vector reduction: a warp instruction
-                // covers a whole coefficient row of the side (d_c contiguous floats).
-                float* tile = reinterpret_cast<float*>(stage0) + (warp - 2) * (32 * (D + 1));
+                if (!live) break;
+                // ---------------- epilogue of the segment: accumulators -> compressed columns ----------------
+                // the stage ring is reused below: every MMA has read it, and the gather warps have left it
+                const bool ok = mbar_wait(acc_ready, seg & 1, fail, c.status) && mbar_wait(gather_done, seg & 1, fail, c.status);
+                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                // the coefficients are cleared by the partition kernel, which this launch may overlap: wait for it here
+                asm volatile("griddepcontrol.wait;" ::: "memory");
+                if (!ok) break;
+                {
+                    const int lane_grp = warp & 3;         // a warp reads tensor-memory lanes 32 (warp % 4) ...
+                    const int col_part = (warp - 2) >> 2;  // the two warps that share a lane group take half of the columns each
+                    constexpr int kPart = (int)kTmemCols / (kGenWarps / 4);      // a whole number of sides (D columns each)
+                    const int m_base = mt * kBM + lane_grp * 32;
+                    // A thread holds 32 columns of ONE row of the accumulator.  The warp lays its 32 rows x D columns of one side
+                    // (K or V of one head) out in the idle stage ring; then lane q owns the four compressed dims 4 q .. 4 q + 3
+                    // (slots of D^c, ascending) and adds them row by row with one 16-byte vector reduction: a warp instruction
+                    // covers a whole coefficient row of the side (d_c contiguous floats).
+                    float* tile = reinterpret_cast<float*>(stage0) + (warp - 2) * (32 * (D + 1));
 #pragma unroll 1
-                for (int t0 = col_part * kPart; t0 < (col_part + 1) * kPart; t0 += D) {
-                    const int hh = t0 / N;
-                    const bool is_k = t0 - hh * N < D;
-                    const int ncomp = is_k ? s.dck : s.dcv, nq = ncomp >> 2;
-                    int col[4] = {0, 0, 0, 0};
-                    if (lane < nq) {
-                        const int32_t* idc = (is_k ? c.idx_comp_k : c.idx_comp_v) + (size_t)(h0 + hh) * ncomp + 4 * lane;
+                    for (int t0 = col_part * kPart; t0 < (col_part + 1) * kPart; t0 += D) {
+                        const int hh = t0 / N;
+                        const bool is_k = t0 - hh * N < D;
+                        const int ncomp = is_k ? s.dck : s.dcv, nq = ncomp >> 2;
+                        int col[4] = {0, 0, 0, 0};
+                        if (lane < nq) {
+                            const int32_t* idc = (is_k ? c.idx_comp_k : c.idx_comp_v) + (size_t)(g.h0 + hh) * ncomp + 4 * lane;
 #pragma unroll
-                        for (int i = 0; i < 4; ++i) col[i] = idc[i];
-                    }
-#pragma unroll 1
-                    for (int cb = 0; cb < D; cb += 32) {
-                        float v[32];
-                        tmem_ld32(tmem_base + ((uint32_t)(lane_grp * 32) << 16) + (uint32_t)(t0 + cb), v);
-#pragma unroll
-                        for (int i = 0; i < 32; ++i) tile[lane * (D + 1) + cb + i] = v[i];
-                    }
-                    __syncwarp();
-                    float* base = coef_rows(is_k ? c.coef_k : c.coef_v, s, b, h0 + hh, ncomp) + (size_t)m_base * ncomp + 4 * lane;
-                    if (lane < nq) {
-#pragma unroll 4
-                        for (int rr = 0; rr < 32; ++rr) {
-                            const float* trow = tile + rr * (D + 1);
-                            if (m_base + rr < s.M)
-                                asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(base + (size_t)rr * ncomp), "f"(trow[col[0]]),
-                                             "f"(trow[col[1]]), "f"(trow[col[2]]), "f"(trow[col[3]])
-                                             : "memory");
+                            for (int i = 0; i < 4; ++i) col[i] = idc[i];
                         }
+#pragma unroll 1
+                        for (int cb = 0; cb < D; cb += 32) {
+                            float v[32];
+                            tmem_ld32(tmem_base + ((uint32_t)(lane_grp * 32) << 16) + (uint32_t)(t0 + cb), v);
+#pragma unroll
+                            for (int i = 0; i < 32; ++i) tile[lane * (D + 1) + cb + i] = v[i];
+                        }
+                        __syncwarp();
+                        float* base = coef_rows(is_k ? c.coef_k : c.coef_v, s, g.b, g.h0 + hh, ncomp) + (size_t)m_base * ncomp + 4 * lane;
+                        if (lane < nq) {
+#pragma unroll 4
+                            for (int rr = 0; rr < 32; ++rr) {
+                                const float* trow = tile + rr * (D + 1);
+                                if (m_base + rr < s.M)
+                                    asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(base + (size_t)rr * ncomp), "f"(trow[col[0]]),
+                                                 "f"(trow[col[1]]), "f"(trow[col[2]]), "f"(trow[col[3]])
+                                                 : "memory");
+                            }
+                        }
+                        __syncwarp();
                     }
+                }
+                pos += (uint32_t)(g.kb1 - g.kb0);
+                if (pos < pos_end) {
+                    // another segment follows: the accumulators are read and the ring is free for its boxes and tiles
+                    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+                    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
                     __syncwarp();
+                    if (lane == 0) mbar_arrive(epi_done);
+                    // the other generator warps' scratch lies in the stages that this warp writes next
+                    if (!mbar_wait(epi_done, seg & 1, fail, c.status)) break;
                 }
             }
         }
@@ -387,17 +453,15 @@ cudaError_t launch_tc2_t(const CUtensorMap& tmK, const CUtensorMap& tmV, const D
                          bool ordered, bool gather, cudaStream_t stream) {
     constexpr size_t stage = (size_t)kBM * kBK * 2 + (size_t)HP * (D / 64) * kBK * 64 * 2;
     constexpr size_t n_stages = (200 * 1024) / stage < 6 ? (200 * 1024) / stage : 6;
-    const size_t smem = n_stages * stage + 8 * (3 * n_stages + 2) + 16 + sizeof(int) * HP * D + 64 + 1024;
+    const size_t smem = n_stages * stage + 8 * (3 * n_stages + 3) + 16 + sizeof(int) * HP * D + 64 + 1024;
     cudaError_t err = ensure_dynamic_smem(compress_tc2_kernel<D, HP>, smem);
     if (err != cudaSuccess) return err;
-    const int row_tiles = s.M / kBM;
+    const int n_pairs = s.M / (2 * kBM);
     const int nkb = (n_mid + kBK - 1) / kBK;
-    const int fixed = row_tiles * (s.Hkv / HP) * s.B;
-    int n_tsplit = sm_count() / fixed;                          // one wave: one CTA per SM at most
-    if (n_tsplit > nkb) n_tsplit = nkb;
-    if (n_tsplit < 1 || ordered) n_tsplit = 1;                  // one split: every coefficient is added to zero exactly once
+    const long long n_units = (long long)(s.Hkv / HP) * s.B;
+    const long long total = n_units * nkb;                      // positions: the blocks of all units, end to end
+    if (total <= 0 || total >= (1ll << 31)) return cudaErrorInvalidValue;
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(row_tiles, s.Hkv / HP, s.B * n_tsplit);
     cfg.blockDim = dim3(kThreadsTc);
     cfg.dynamicSmemBytes = smem;
     cfg.stream = stream;
@@ -410,7 +474,64 @@ cudaError_t launch_tc2_t(const CUtensorMap& tmK, const CUtensorMap& tmV, const D
     attr[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 2;
-    return cudaLaunchKernelEx(&cfg, compress_tc2_kernel<D, HP>, tmK, tmV, s, c, L, n_tsplit, gather ? 1 : 0);
+    TeamCuts cuts = {};
+    int n_teams, per = 0;
+    if (ordered) {
+        // one team per unit: every coefficient is added to zero exactly once (pairs beyond the resident ones run in later waves)
+        n_teams = (int)n_units;
+        per = nkb;
+    } else {
+        // pairs resident at once (cached per device): the teams fill them, no second wave
+        static int resident[16] = {};
+        int dev = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 16) return cudaErrorInvalidValue;
+        if (resident[dev] == 0) {
+            cfg.gridDim = dim3(2 * sm_count());
+            cfg.numAttrs = 1;
+            int n = 0;
+            if (cudaOccupancyMaxActiveClusters(&n, compress_tc2_kernel<D, HP>, &cfg) != cudaSuccess || n < 1) {
+                cudaGetLastError();
+                n = sm_count() / 2 - 2;
+            }
+            cfg.numAttrs = 2;
+            resident[dev] = n;
+        }
+        n_teams = resident[dev] / n_pairs;
+        if (n_teams < 1) n_teams = 1;
+        if (n_teams > kMaxTeams) n_teams = kMaxTeams;
+        if (n_teams > total) n_teams = (int)total;
+        // Equal cost per team: a segment costs its blocks plus kEpi (epilogue, pipeline refill, in blocks).  The smallest
+        // budget with which the walk below covers all positions in n_teams teams, by bisection.
+        constexpr long long kEpi = 12, kMinSeg = 8;
+        auto walk = [&](long long budget, uint32_t* start) {
+            long long pos = 0;
+            int t = 0;
+            for (; t < n_teams && pos < total; ++t) {
+                if (start) start[t] = (uint32_t)pos;
+                long long left = budget;
+                while (pos < total && left >= kEpi + kMinSeg) {
+                    const long long unit_end = (pos / nkb + 1) * nkb;
+                    long long take = unit_end - pos < left - kEpi ? unit_end - pos : left - kEpi;
+                    if (unit_end - pos - take > 0 && unit_end - pos - take < kMinSeg) take = unit_end - pos - kMinSeg;   // no crumbs for the next team
+                    if (take <= 0) break;
+                    pos += take;
+                    left -= take + kEpi;
+                }
+            }
+            if (start)
+                for (int u = t; u <= n_teams; ++u) start[u] = (uint32_t)(u == n_teams ? total : pos);
+            return pos >= total;
+        };
+        long long lo = kEpi + kMinSeg, hi = total + kEpi * (n_units + 1) + kMinSeg;
+        while (lo < hi) {
+            const long long mid = (lo + hi) / 2;
+            if (walk(mid, nullptr)) hi = mid; else lo = mid + 1;
+        }
+        while (!walk(lo, cuts.start)) ++lo;
+        cuts.start[n_teams] = (uint32_t)total;
+    }
+    cfg.gridDim = dim3(2 * n_teams * n_pairs);
+    return cudaLaunchKernelEx(&cfg, compress_tc2_kernel<D, HP>, tmK, tmV, s, c, L, cuts, per, gather ? 1 : 0);
 }
 
 }  // namespace

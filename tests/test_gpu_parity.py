@@ -576,6 +576,7 @@ def test_multi_layer_step_equals_single_calls_bit_for_bit():
     (dict(B=1, Hq=4, Hkv=4, d=64, L=1500, T=2048, M=128, n_full_k=8, n_full_v=16), 8),        # one row tile: every token of a block in one CTA
     (dict(B=1, Hq=2, Hkv=2, d=128, L=1400, T=2048, M=128, n_full_k=64, n_full_v=64), 4),      # more chunks than the gather warps hold: partition kernel writes the rows
     (dict(B=1, Hq=2, Hkv=2, d=128, L=1100 + 37, T=2048, M=1024, n_full_k=0, n_full_v=8), 16), # nothing kept of K; ragged last block; idle row-tile CTAs
+    (dict(B=6, Hq=4, Hkv=4, d=128, L=1300, T=4096, M=2048, n_full_k=32, n_full_v=16), 16),    # more (batch, head group) units than teams of pairs: a team's blocks run through two or three units
 ])
 def test_tensor_compress_with_its_gather(kw, P):
     """Middles of 1024 tokens and more take the tcgen05 kernel, which also writes the kept-dim rows of the middle
