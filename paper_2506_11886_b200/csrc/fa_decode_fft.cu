@@ -426,8 +426,12 @@ struct FftSmem {
     int stages_off, fbuf_off, kb_off, pbt_off, twf_off, rev_off, E_off, ut_off, z_off, o_off, red_off, pend_off, zero_off, total;
     int fb_floats, pbs;
 };
-__host__ __device__ inline FftSmem fft_smem_layout(int log2S, int k, int GH, int NB, int d, int occ, int split = 0) {
+// True if the kernel packs two residue classes of ONE query head into a complex transform (one query head per KV head:
+// the second slot would otherwise be empty).  Then a batch of NB classes needs half the transform and score buffers.
+__host__ __device__ inline bool class_pairs(int G, int GH, int split) { return G == 1 && GH == 2 && !split; }
+__host__ __device__ inline FftSmem fft_smem_layout(int log2S, int k, int GH, int NB, int d, int occ, int split = 0, bool cp = false) {
     const int S = 1 << log2S;
+    const int NT = cp ? (NB + 1) >> 1 : NB;               // transforms of a batch
     FftSmem L;
     L.fb_floats = pf_size(S * GH);
     L.pbs = S + 8;                                        // bf16 per (class, slot) row of rounded probabilities
@@ -435,9 +439,9 @@ __host__ __device__ inline FftSmem fft_smem_layout(int log2S, int k, int GH, int
     L.zero_off = off; off += 16;
     off = 1024;                                           // stages are 1024-byte aligned (swizzled window tiles)
     L.stages_off = off; off += ring_stages(occ) * kStageBytes;
-    L.fbuf_off = off; off += 4 * NB * L.fb_floats;
+    L.fbuf_off = off; off += 4 * NT * L.fb_floats;
     off = (off + 15) / 16 * 16;
-    L.kb_off = off; off += 4 * NB * S * GH;               // kept-dim scores of the batch, natural token order
+    L.kb_off = off; off += 4 * NT * S * GH;               // kept-dim scores of the batch, natural token order
     off = (off + 15) / 16 * 16;
     L.pbt_off = off; off += 2 * NB * GH * L.pbs;
     off = (off + 15) / 16 * 16;
@@ -483,7 +487,7 @@ __global__ void __launch_bounds__(threads_of(SPLIT), OCC) decode_fft_kernel(cons
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");      // the epilogue may be scheduled behind us at once
     Ws ws = ws_view(wsp, p);
     const int NB = p.nb;
-    const FftSmem L = fft_smem_layout(LS, s.k, GH, NB, s.d, OCC, SPLIT ? 1 : 0);
+    const FftSmem L = fft_smem_layout(LS, s.k, GH, NB, s.d, OCC, SPLIT ? 1 : 0, class_pairs(s.G, GH, SPLIT ? 1 : 0));
     uint64_t* full = reinterpret_cast<uint64_t*>(smem_raw);
     uint64_t* empty = full + NS;
     volatile int* fail = reinterpret_cast<volatile int*>(smem_raw + 128);
@@ -509,6 +513,12 @@ __global__ void __launch_bounds__(threads_of(SPLIT), OCC) decode_fft_kernel(cons
     const int b = blockIdx.z;
     const int g_first = h * s.G + pass * GH;
     const int ng = min(GH, s.G - pass * GH);
+    // One query head in two slots (MHA): the second slot would carry nothing.  Instead both slots belong to the head
+    // and a packed transform carries two residue classes, class 2 t in the real parts (slot 0) and class 2 t + 1 in the
+    // imaginary parts (slot 1): half as many spectra, transforms, softmax points and folds.  The slots keep their own
+    // running maxima, sums, outputs and z (slot 1 sees no window token) and are folded into slot 0 before the
+    // partial results are written.
+    const bool cp = class_pairs(s.G, GH, SPLIT ? 1 : 0);
     const int tid = threadIdx.x;
     const int log2P = 31 - __clz(s.P);
 
@@ -639,7 +649,8 @@ __global__ void __launch_bounds__(threads_of(SPLIT), OCC) decode_fft_kernel(cons
     const int ts_w = kWinRowsPerTile;
     // window tokens per softmax chunk: the score and probability buffers of all NB classes when
     // they can be addressed as one, else those of one class
-    const int wchunk = pf_size(NB * S * GH) <= NB * L.fb_floats ? NB * S : S;
+    const int NT = class_pairs(s.G, GH, SPLIT ? 1 : 0) ? (NB + 1) >> 1 : NB;       // transform buffers of a batch
+    const int wchunk = pf_size(NT * S * GH) <= NT * L.fb_floats ? NT * S : S;
     const int pbw = NB * L.pbs;                            // row stride of the window probabilities
 
     if (tid == 0) {
@@ -830,7 +841,13 @@ __global__ void __launch_bounds__(threads_of(SPLIT), OCC) decode_fft_kernel(cons
                             mma_bf16(d4, lo.z, hi.z, lo.w, hi.w, qk[rd][1][0], qk[rd][1][1]);
                         }
                     }
-                    if (2 * tq < GH) {
+                    if (cp) {
+                        if (tq == 0) {                      // the head's column, to the slot of this class in its pair
+                            float* dst = kbuf + (((ci >> 1) * S + a0 + grp * 16 + gq) * GH + (ci & 1));
+                            dst[0] = d4[0] * sl2;
+                            dst[8 * GH] = d4[2] * sl2;
+                        }
+                    } else if (2 * tq < GH) {
                         const uint32_t dst = smem_addr(kbuf) + kb_lane_off + (uint32_t)((ci * S + a0 + grp * 16) * GH) * 4;
                         sts64(dst, d4[0] * sl2, d4[1] * sl2);
                         sts64(dst + 8 * GH * 4, d4[2] * sl2, d4[3] * sl2);
@@ -1091,7 +1108,7 @@ __global__ void __launch_bounds__(threads_of(SPLIT), OCC) decode_fft_kernel(cons
                 float v[GH];
                 load_vals(sb + pf(a * GH), v);
 #pragma unroll
-                for (int g = 0; g < GH; ++g) mx[g] = fmaxf(mx[g], v[g]);
+                for (int g = 0; g < GH; ++g) if (!(cp && g == 1)) mx[g] = fmaxf(mx[g], v[g]);
             }
             block_max(mx);
 #pragma unroll
@@ -1110,7 +1127,7 @@ __global__ void __launch_bounds__(threads_of(SPLIT), OCC) decode_fft_kernel(cons
                 if (a < n_tok) load_vals(sb + pf(a * GH), v);
 #pragma unroll
                 for (int g = 0; g < GH; ++g) {
-                    v[g] = a < n_tok ? ex2(v[g] - m_run[g]) : 0.f;
+                    v[g] = (a < n_tok && !(cp && g == 1)) ? ex2(v[g] - m_run[g]) : 0.f;
                     l_acc[g] += v[g];
                     pb[g * pbw + a] = __float2bfloat16_rn(v[g]);
                 }
@@ -1221,33 +1238,45 @@ __global__ void __launch_bounds__(threads_of(SPLIT), OCC) decode_fft_kernel(cons
         }
 
         if constexpr (!SPLIT) {
+        if (cp) {
+            // a class's probabilities go to its own slot's row; the other slot's row of the class stays zero
+            #pragma unroll 1
+            for (int i = tid; i < NB * GH * pbs / 2; i += kAll) reinterpret_cast<uint32_t*>(pbt)[i] = 0u;
+            all_sync();
+        }
         #pragma unroll 1
         for (int cb = c0; cb < c1; cb += NB) {
             const int nb = min(NB, c1 - cb);
             if (n_of_class(cb) == 0) break;               // classes are filled in order: nothing further on
             if (cb != c0) k_phase(cb, nb, kb);
+            // transforms of the batch, and classes from one transform to the next
+            const int nbt = cp ? (nb + 1) >> 1 : nb, cstep = cp ? 2 : 1;
 
             // packed Hermitian spectra of the nb classes: X_m = V^A_m + i V^B_m per complex lane,
             // V_m = v_m + conj(v_{S-m}), v_n = (1/2) u~_n e^{i theta n c}.  Pair 0 is bins (0, S/2).
             if (s.dck > 0) {
                 // neighbouring lanes share a pair of bins and take half of the classes each (a batch of one
                 // class: one lane per pair, half as many rounds)
-                const bool split2 = nb > 1;
-                const int hcls = split2 ? (nb + 1) >> 1 : nb;
+                const bool split2 = nbt > 1;
+                const int hcls = split2 ? (nbt + 1) >> 1 : nbt;
                 #pragma unroll 1
                 for (int item = tid; item < (split2 ? S : S / 2); item += kAll) {
-                    const int pr = split2 ? item >> 1 : item, ci0 = split2 ? (item & 1) * hcls : 0, ci1 = min(nb, ci0 + hcls);
+                    const int pr = split2 ? item >> 1 : item, ci0 = split2 ? (item & 1) * hcls : 0, ci1 = min(nbt, ci0 + hcls);
                     const int m = pr, mc = pr == 0 ? S / 2 : S - pr;
                     PC<N> Am = czero, Bm = czero, Ac = czero, Bc = czero;
                     float2 em = make_float2(1.f, 0.f), ec = make_float2(1.f, 0.f);
                     if (m < s.k) { ld_entry(ut, m, Am, Bm); em = E[m]; }
                     if (mc < s.k) { ld_entry(ut, mc, Ac, Bc); ec = E[mc]; }
-                    float2 twm = seed_tw(m, cb + ci0), twc = seed_tw(mc, cb + ci0);
+                    float2 twm = seed_tw(m, cb + cstep * ci0), twc = seed_tw(mc, cb + cstep * ci0);
+                    // class pairs: both slots are the head; slot 1 is one class further on
+                    const float2 em1 = em, ec1 = ec;
+                    if (cp) { Bm = Am; Bc = Ac; em = cmulf(em, em); ec = cmulf(ec, ec); }
                     #pragma unroll 1
                     for (int ci = ci0; ci < ci1; ++ci) {
                         const PR<N> wmr = splat<N>(twm.x), wmi = splat<N>(twm.y), wcr = splat<N>(twc.x), wci = splat<N>(twc.y);
-                        const PC<N> vAm = cmulw(Am, wmr, wmi), vBm = cmulw(Bm, wmr, wmi);
-                        const PC<N> vAc = cmulw(Ac, wcr, wci), vBc = cmulw(Bc, wcr, wci);
+                        const float2 twmB = cp ? cmulf(twm, em1) : twm, twcB = cp ? cmulf(twc, ec1) : twc;
+                        const PC<N> vAm = cmulw(Am, wmr, wmi), vBm = cmulw(Bm, splat<N>(twmB.x), splat<N>(twmB.y));
+                        const PC<N> vAc = cmulw(Ac, wcr, wci), vBc = cmulw(Bc, splat<N>(twcB.x), splat<N>(twcB.y));
                         float* base = fbuf + ci * fb_floats;
                         if (pr != 0) {
                             const PC<N> VA = cconj_add(vAm, vAc), VB = cconj_add(vBm, vBc);
@@ -1265,11 +1294,11 @@ __global__ void __launch_bounds__(threads_of(SPLIT), OCC) decode_fft_kernel(cons
                 }
                 all_sync();
                 if (cb == c0) TL(8);
-                fft_run<GH, LS, LS, false>(fbuf, fb_floats, nb, twf, tid);        // score of slot a at point rev[a]
+                fft_run<GH, LS, LS, false>(fbuf, fb_floats, nbt, twf, tid);       // score of slot a at point rev[a]
                 if (cb == c0) TL(9);
             } else {
                 #pragma unroll 1
-                for (int i = tid; i < nb * fb_floats; i += kAll) fbuf[i] = 0.f;
+                for (int i = tid; i < nbt * fb_floats; i += kAll) fbuf[i] = 0.f;
                 all_sync();
             }
 
@@ -1280,9 +1309,12 @@ __global__ void __launch_bounds__(threads_of(SPLIT), OCC) decode_fft_kernel(cons
 #pragma unroll
             for (int g = 0; g < GH; ++g) mx[g] = kNegBig;
             #pragma unroll 1
-            for (int i = tid; i < (nb << LS); i += kAll) {
+            for (int i = tid; i < (nbt << LS); i += kAll) {
                 const int ci = i >> LS, a = i & (S - 1);
-                if (a < n_of_class(cb + ci)) {
+                // class pairs: slot g of the point is token a of class cstep ci + g
+                const bool ok0 = a < n_of_class(cb + cstep * ci);
+                const bool ok1 = cp ? (2 * ci + 1 < nb && a < n_of_class(cb + 2 * ci + 1)) : ok0;
+                if (ok0 || ok1) {
                     // score = compressed part (transform output) + kept part
                     float* pt = fbuf + ci * fb_floats + pf(rev[a] * GH);
                     float v[GH], kv[GH];
@@ -1294,7 +1326,7 @@ __global__ void __launch_bounds__(threads_of(SPLIT), OCC) decode_fft_kernel(cons
                         store_vals(pt, v);
                     }
 #pragma unroll
-                    for (int g = 0; g < GH; ++g) mx[g] = fmaxf(mx[g], v[g]);
+                    for (int g = 0; g < GH; ++g) if (g == 1 ? ok1 : ok0) mx[g] = fmaxf(mx[g], v[g]);
                 }
             }
             block_max(mx);
@@ -1306,17 +1338,19 @@ __global__ void __launch_bounds__(threads_of(SPLIT), OCC) decode_fft_kernel(cons
                 l_acc[g] *= alpha[g];
             }
             #pragma unroll 1
-            for (int i = tid; i < (nb << LS); i += kAll) {
+            for (int i = tid; i < (nbt << LS); i += kAll) {
                 const int ci = i >> LS, a = i & (S - 1);
                 float* pt = fbuf + ci * fb_floats + pf(rev[a] * GH);
                 float v[GH];
                 load_vals(pt, v);
-                const bool ok = a < n_of_class(cb + ci);
+                const bool ok0 = a < n_of_class(cb + cstep * ci);
+                const bool ok1 = cp ? (2 * ci + 1 < nb && a < n_of_class(cb + 2 * ci + 1)) : ok0;
 #pragma unroll
                 for (int g = 0; g < GH; ++g) {
-                    v[g] = ok ? ex2(v[g] - m_run[g]) : 0.f;
+                    v[g] = (g == 1 ? ok1 : ok0) ? ex2(v[g] - m_run[g]) : 0.f;
                     l_acc[g] += v[g];
-                    pbt[(ci * GH + g) * pbs + a] = __float2bfloat16_rn(v[g]);
+                    if (!cp) pbt[(ci * GH + g) * pbs + a] = __float2bfloat16_rn(v[g]);
+                    else if (2 * ci + g < nb) pbt[((2 * ci + g) * GH + g) * pbs + a] = __float2bfloat16_rn(v[g]);
                 }
                 store_vals(pt, v);
             }
@@ -1378,45 +1412,49 @@ __global__ void __launch_bounds__(threads_of(SPLIT), OCC) decode_fft_kernel(cons
             if (cb == c0) TL(11);
             // z_n = alpha z_n + sum_c e^{i theta n c} Y^c_n, Y^c = transform of the packed probabilities
             if (s.dcv > 0) {
-                fft_run<GH, LS, LS, true>(fbuf, fb_floats, nb, twf, tid);
+                fft_run<GH, LS, LS, true>(fbuf, fb_floats, nbt, twf, tid);
                 if (cb == c0) TL(12);
                 PR<N> alA, alB;
                 if constexpr (N == 2) { alA = pk(alpha[0], alpha[1]); alB = pk(alpha[2], alpha[3]); }
                 else { alA = PR<1>{alpha[0]}; alB = PR<1>{alpha[1]}; }
                 const PR<N> half = splat<N>(0.5f);
-                const bool split2 = nb > 1;                // as for the spectra: one lane per pair when the batch is one class
-                const int hcls = split2 ? (nb + 1) >> 1 : nb;
+                const bool split2 = nbt > 1;               // as for the spectra: one lane per pair when the batch is one transform
+                const int hcls = split2 ? (nbt + 1) >> 1 : nbt;
                 #pragma unroll 1
                 for (int item = tid; item < (split2 ? S : S / 2); item += kAll) {       // split: whole warps (S is a multiple of 32)
                     const int pr = split2 ? item >> 1 : item, ci0 = split2 ? (item & 1) * hcls : 0;
                     const int m = pr, mc = pr == 0 ? S / 2 : S - pr;
-                    const int ci1 = (m >= s.k && mc >= s.k) ? ci0 : min(nb, ci0 + hcls);
+                    const int ci1 = (m >= s.k && mc >= s.k) ? ci0 : min(nbt, ci0 + hcls);
                     float2 em = make_float2(1.f, 0.f), ec = make_float2(1.f, 0.f);
                     if (m < s.k) em = E[m];
                     if (mc < s.k) ec = E[mc];
-                    float2 twm = seed_tw(m, cb + ci0), twc = seed_tw(mc, cb + ci0);
+                    float2 twm = seed_tw(m, cb + cstep * ci0), twc = seed_tw(mc, cb + cstep * ci0);
+                    const float2 em1 = em, ec1 = ec;        // class pairs: slot 1 is one class further on than slot 0
+                    if (cp) { em = cmulf(em, em); ec = cmulf(ec, ec); }
                     PC<N> zAm = czero, zBm = czero, zAc = czero, zBc = czero;
                     #pragma unroll 1
                     for (int ci = ci0; ci < ci1; ++ci) {
                         const float* base = fbuf + ci * fb_floats;
                         const PC<N> ya = ld_pt<N>(base + pf(m * GH)), yb = ld_pt<N>(base + pf(mc * GH));
                         const PR<N> wmr = splat<N>(twm.x), wmi = splat<N>(twm.y), wcr = splat<N>(twc.x), wci = splat<N>(twc.y);
+                        const float2 twmB = cp ? cmulf(twm, em1) : twm, twcB = cp ? cmulf(twc, ec1) : twc;
+                        const PR<N> wmrB = splat<N>(twmB.x), wmiB = splat<N>(twmB.y), wcrB = splat<N>(twcB.x), wciB = splat<N>(twcB.y);
                         if (pr != 0) {
                             // real slots: y0 = (ya + conj(yb)) / 2, imaginary slots: y1 = (ya - conj(yb)) / (2 i); bin mc holds the conjugates
                             const PC<N> y0 = PC<N>{(ya.re + yb.re) * half, (ya.im - yb.im) * half};
                             const PC<N> y1 = PC<N>{(ya.im + yb.im) * half, (yb.re - ya.re) * half};
                             zAm = zAm + cmulw(y0, wmr, wmi);
-                            zBm = zBm + cmulw(y1, wmr, wmi);
+                            zBm = zBm + cmulw(y1, wmrB, wmiB);
                             zAc = zAc + cmulw(PC<N>{y0.re, splat<N>(0.f) - y0.im}, wcr, wci);
-                            zBc = zBc + cmulw(PC<N>{y1.re, splat<N>(0.f) - y1.im}, wcr, wci);
+                            zBc = zBc + cmulw(PC<N>{y1.re, splat<N>(0.f) - y1.im}, wcrB, wciB);
                         } else {
                             // bins 0 and S/2 are real for each real sequence: (re, im) of the packed value are the two heads
                             const PC<N> y0m = PC<N>{ya.re, splat<N>(0.f)}, y1m = PC<N>{ya.im, splat<N>(0.f)};
                             const PC<N> y0c = PC<N>{yb.re, splat<N>(0.f)}, y1c = PC<N>{yb.im, splat<N>(0.f)};
                             zAm = zAm + cmulw(y0m, wmr, wmi);
-                            zBm = zBm + cmulw(y1m, wmr, wmi);
+                            zBm = zBm + cmulw(y1m, wmrB, wmiB);
                             zAc = zAc + cmulw(y0c, wcr, wci);
-                            zBc = zBc + cmulw(y1c, wcr, wci);
+                            zBc = zBc + cmulw(y1c, wcrB, wciB);
                         }
                         twm = cmulf(twm, em);
                         twc = cmulf(twc, ec);
@@ -1751,6 +1789,25 @@ __global__ void __launch_bounds__(threads_of(SPLIT), OCC) decode_fft_kernel(cons
     }
     all_sync();
 
+    if (cp) {
+        // class pairs: slot 1 (the odd classes of the batches) into slot 0, as two partial softmax results of one head
+        const float mm = fmaxf(m_run[0], m_run[1]);
+        const float e0 = ex2(m_run[0] - mm), e1 = ex2(m_run[1] - mm);
+        #pragma unroll 1
+        for (int e = tid; e < s.d; e += kAll)
+            o_s[e] = __float2ll_rn(__ll2float_rn(o_s[e]) * e0 + __ll2float_rn(o_s[s.d + e]) * e1);
+        #pragma unroll 1
+        for (int n = tid; n < s.k; n += kAll) {
+            float* e = z_s + n * 2 * GH;                  // (re, im) of slot 0, then of slot 1
+            e[0] = e0 * e[0] + e1 * e[2];
+            e[1] = e0 * e[1] + e1 * e[3];
+        }
+        all_sync();
+        if (tid == 0) red_s[kAllW * GH] = e0 * red_s[kAllW * GH] + e1 * red_s[kAllW * GH + 1];
+        m_run[0] = mm;
+        all_sync();
+    }
+
     TL(14);
     // ------------------------------ partial results ------------------------------
     for (int i = tid; i < GH * s.d; i += kAll) {
@@ -2023,7 +2080,7 @@ static int coop_pdl_state(int set) {
 template <int GH, int LS, int OCC, bool STEP, bool SPLIT = false>
 cudaError_t launch_fft_t(const Dims& s, const CacheDev& c, const DecodePlan& p, const void* q, void* out, char* ws, int step,
                          const void* k_new, const void* v_new, cudaStream_t st) {
-    const FftSmem L = fft_smem_layout(LS, s.k, GH, p.nb, s.d, OCC, SPLIT ? 1 : 0);
+    const FftSmem L = fft_smem_layout(LS, s.k, GH, p.nb, s.d, OCC, SPLIT ? 1 : 0, class_pairs(s.G, GH, SPLIT ? 1 : 0));
     cudaError_t err = ensure_dynamic_smem(decode_fft_kernel<GH, LS, OCC, STEP, SPLIT>, (size_t)L.total);
     if (err != cudaSuccess) return err;
     // window buffers as tensor maps (cached per buffer)
@@ -2097,7 +2154,7 @@ int resident_ctas_t(const Dims& s, const DecodePlan& p) {
     static Entry table[16];
     static int used = 0;
     static std::mutex mu;
-    const size_t smem = (size_t)fft_smem_layout(LS, s.k, GH, p.nb, s.d, OCC, SPLIT ? 1 : 0).total;
+    const size_t smem = (size_t)fft_smem_layout(LS, s.k, GH, p.nb, s.d, OCC, SPLIT ? 1 : 0, class_pairs(s.G, GH, SPLIT ? 1 : 0)).total;
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess) { cudaGetLastError(); return 0; }
     std::lock_guard<std::mutex> lock(mu);
@@ -2140,7 +2197,7 @@ bool decode_fft_launchable(const Dims& s, const DecodePlan& p) {
 }
 
 size_t decode_fft_smem_bytes(const Dims& s, int log2S, int gh, int nb, int occ, int split) {
-    return (size_t)fft_smem_layout(log2S, s.k, gh, nb, s.d, occ, split).total;
+    return (size_t)fft_smem_layout(log2S, s.k, gh, nb, s.d, occ, split, class_pairs(s.G, gh, split)).total;
 }
 
 // True if the fused kernel's staging areas hold a part's share of the coefficient rows: the rows
@@ -2148,8 +2205,9 @@ size_t decode_fft_smem_bytes(const Dims& s, int log2S, int gh, int nb, int occ, 
 bool decode_fft_fused_fits(const Dims& s, int log2S, int gh, int nb, int n_part, int occ, int split) {
     if (s.M % 4 != 0) return false;
     if (occ == 2 && log2S > 8) return false;                                           // no two-per-SM build of the long transforms
-    const FftSmem L = fft_smem_layout(log2S, s.k, gh, nb, s.d, occ, split);
-    if (s.dck > 0 && (long long)nb * L.fb_floats < 8LL * s.dck) return false;           // at least eight rows of C^K per chunk
+    const FftSmem L = fft_smem_layout(log2S, s.k, gh, nb, s.d, occ, split, class_pairs(s.G, gh, split));
+    // at least eight rows of C^K per staged chunk (class pairs: the chunk may use the score and probability buffers too, as the kernel does)
+    if (s.dck > 0 && (class_pairs(s.G, gh, split) ? (long long)((L.twf_off - L.fbuf_off) >> 2) : (long long)nb * L.fb_floats) < 8LL * s.dck) return false;
     const long long ring = (long long)ring_stages(occ) * kStageBytes / 4;
     const long long nrg = s.dcv ? (split ? kSplitConsumers : kConsumers) / (s.dcv >> 2) : 0;
     const long long head = ((2LL * gh * n_part + gh + 3) & ~3LL);

@@ -240,6 +240,24 @@ def test_mha_48_kept_dims(algo):
     pair.check_decode(synth.queries(shape, seed=12, step=1))
 
 
+@pytest.mark.parametrize("kw,P", [
+    (dict(B=3, Hq=7, Hkv=7, L=3000, T=4096, M=128), 32),      # 21 heads: 4 or 5 classes per CTA, the last transform of a batch half empty
+    (dict(B=2, Hq=3, Hkv=3, L=1700, T=2048, M=128), 8),       # more CTAs per head than classes: one class per CTA, slot 1 never used
+    (dict(B=1, Hq=40, Hkv=40, L=2300, T=4096, M=256), 16),    # lone CTAs, two per SM: all 16 classes and the windows in one CTA
+])
+def test_mha_two_classes_per_packed_transform(kw, P):
+    """One query head per KV head: the transform kernel packs two residue classes into a complex transform (the two
+    slots are one head: own maxima, sums, outputs and z per slot, folded before the partial results).  Ragged class
+    lengths, odd class counts per batch, decode call and fused steps (the pending middle token lands in either slot)."""
+    shape = SMALL_BF16.with_(d=128, n_full_k=48, n_full_v=32, L_init=4, L_local=64, decode_steps=3, **kw)
+    pair, stream = make_pair(shape, seed=33, algo=fa.FA_DECODE_FFT, P=P, max_mid=shape.T)
+    pair.check_decode(synth.queries(shape, seed=33))
+    K, V = stream.tokens(shape.L, shape.L + 3)
+    for t in range(3):
+        pair.check_step(synth.queries(shape, seed=33, step=t + 1), K[:, t], V[:, t])
+    pair.check_state()
+
+
 @pytest.mark.parametrize("algo", ALGOS)
 def test_decode_step_from_empty_through_eviction(algo):
     """fa_decode_step token by token: init fills, local fills, then every step evicts a row into the middle;
