@@ -283,8 +283,10 @@ size_t fa_static_workspace_limit(void);
 fa_status fa_poll_status(const fa_cache* cache, void* stream);
 
 /* Number of kernels one call launches for this layout (what = 0 compress, 1 append,
- * 2 decode, 3 decode step); for launch accounting by callers.  what = 4 asks about the plan instead:
- * 1 if fa_decode_attention runs the split build of the fused kernel for this layout, else 0. */
+ * 2 decode, 3 decode step); for launch accounting by callers.  what >= 4 asks about the decode plan instead:
+ * 4: 1 if fa_decode_attention runs the split build of the fused kernel for this layout, else 0;
+ * 5: residue classes per batch of the transform kernel (0 for the direct kernel);
+ * 6: CTAs per (batch, KV head, pass of query heads).  Unknown values of what return 0. */
 int fa_launch_count(const fa_layout* layout, int what);
 
 const char* fa_status_string(fa_status s);

@@ -675,6 +675,16 @@ int fa_launch_count(const fa_layout* layout, int what) {
             if (plan_decode(*layout, &p) != FA_OK) return 0;
             return (p.fused && p.split) ? 1 : 0;
         }
+        case 5: {           // plan query: residue classes per batch of the transform kernel (0: the direct kernel)
+            DecodePlan p;
+            if (plan_decode(*layout, &p) != FA_OK) return 0;
+            return p.algo == FA_DECODE_FFT ? p.nb : 0;
+        }
+        case 6: {           // plan query: CTAs per (batch, KV head, pass) of the decode kernel
+            DecodePlan p;
+            if (plan_decode(*layout, &p) != FA_OK) return 0;
+            return p.n_part;
+        }
         default: return 0;
     }
 }
