@@ -203,7 +203,9 @@ fa_status plan_decode(const fa_layout& l, DecodePlan* p) {
         // More heads than SMs: the lone CTAs of the fused kernel run in whole waves.  AUTO keeps it unless
         // the balanced split is ahead by the same cost model (the last wave nearly empty) by more than
         // the margin that the three launches and the round trip of u and the partial results cost.
-        if (p->fused && jobs > kNumSms && l.decode_algo == FA_DECODE_AUTO &&
+        // (Heads that are all resident at once, two to an SM, stay fused: a lone CTA takes as long with a neighbour on
+        // its SM as without, measured 116-118 us for 160 to 256 heads of the MHA serving shape against 138 us split.)
+        if (p->fused && jobs > kNumSms * p->occ && l.decode_algo == FA_DECODE_AUTO &&
             20LL * ((jobs + kNumSms * p->occ - 1) / (kNumSms * p->occ)) * (s.P + 2) * p->occ > 23 * best_cost)
             p->fused = 0;
         if (!p->fused) {
