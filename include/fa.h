@@ -156,9 +156,10 @@ fa_status fa_compress(const fa_layout* layout, fa_cache* cache, const void* K, c
                       void* ws, size_t ws_bytes, void* stream);
 
 /* fa_compress with a choice of how the coefficients of Eq.3 are evaluated (flags, OR-ed together; 0 is fa_compress):
- *   FA_COMPRESS_ORDERED  the sums of Eq.3 are taken in a fixed order, so two calls on the same input give the
- *                        same bits (the default splits the token axis over CTAs and adds the partial sums with
- *                        floating-point atomics, whose order varies from run to run);
+ *   FA_COMPRESS_ORDERED  the sums of Eq.3 do not depend on the order of execution, so two calls on the same input
+ *                        give the same bits (the default splits the token axis over many CTAs and adds the partial
+ *                        sums with floating-point atomics, whose order varies from run to run; this mode adds at
+ *                        most two partial sums to a zeroed coefficient, and a two-term sum commutes);
  *   FA_COMPRESS_FFT      the coefficients are computed as the k lowest bins of the discrete Fourier transform of
  *                        each zero-extended token column (Sec. 3.3, Eq.3-4 without forming F): one length
  *                        period / mid_classes transform per residue class and column, fp32 throughout, always in a

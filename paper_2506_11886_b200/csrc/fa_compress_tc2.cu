@@ -33,7 +33,8 @@ using namespace umma;
 // end inside a unit and go on into the next (one SEGMENT per unit touched: main loop, then an epilogue that adds the
 // segment's partial sums).  The table is cut on the host so that every team has the same cost (blocks + epilogues),
 // and so that teams x pairs fill the pairs that are resident at once; with per > 0 the cut is uniform instead
-// (start = t * per: one team per unit, every coefficient added to zero exactly once).
+// (every unit in pieces of per blocks, one team each; the order-fixed mode cuts every unit in two: a coefficient is
+// then zero plus two terms, and the sum of two floats does not depend on which arrives first).
 constexpr int kMaxTeams = 96;
 struct TeamCuts { uint32_t start[kMaxTeams + 1]; };
 
@@ -80,8 +81,15 @@ __global__ void __launch_bounds__(kThreadsTc, 1) compress_tc2_kernel(const __gri
     const int n_local = min(L - n_init, s.l_local);
     const int n_mid = L - n_init - n_local;
     const int nkb = (n_mid + kBK - 1) / kBK;
-    const uint32_t pos_begin = per > 0 ? (uint32_t)team * (uint32_t)per : cuts.start[team];
-    const uint32_t pos_end = per > 0 ? pos_begin + (uint32_t)per : cuts.start[team + 1];
+    uint32_t pos_begin, pos_end;
+    if (per > 0) {                                         // uniform cut: every unit in ceil(blocks / per) pieces of per blocks
+        const int pieces = (nkb + per - 1) / per, unit = team / pieces, piece = team - unit * pieces;
+        pos_begin = (uint32_t)unit * (uint32_t)nkb + (uint32_t)(piece * per);
+        pos_end = (uint32_t)unit * (uint32_t)nkb + (uint32_t)min(nkb, (piece + 1) * per);
+    } else {
+        pos_begin = cuts.start[team];
+        pos_end = cuts.start[team + 1];
+    }
     // the segment that starts at position pos: its unit (batch b, heads h0 ...) and blocks kb0 .. kb1
     struct Seg { int b, h0, kb0, kb1; };
     auto seg_at = [&](uint32_t pos) {
@@ -477,9 +485,11 @@ cudaError_t launch_tc2_t(const CUtensorMap& tmK, const CUtensorMap& tmV, const D
     TeamCuts cuts = {};
     int n_teams, per = 0;
     if (ordered) {
-        // one team per unit: every coefficient is added to zero exactly once (pairs beyond the resident ones run in later waves)
-        n_teams = (int)n_units;
-        per = nkb;
+        // Two teams per unit, half of its blocks each: every coefficient is zero + a + b, and fl(a + b) = fl(b + a), so the
+        // result has the same bits whichever half arrives first (three terms would not).  Pairs beyond the resident
+        // ones run in later waves.
+        per = (nkb + 1) / 2;
+        n_teams = (int)n_units * ((nkb + per - 1) / per);
     } else {
         // pairs resident at once (cached per device): the teams fill them, no second wave
         static int resident[16] = {};
