@@ -171,6 +171,21 @@ fa_status fa_compress_ex(const fa_layout* layout, fa_cache* cache, const void* K
                          int64_t stride_t, int64_t stride_h, int32_t L, uint32_t flags, void* ws, size_t ws_bytes,
                          void* stream);
 
+/* Compression of the prefill of n_layers layers in one call (Eq.1-4 per layer): layer i gets what
+ * fa_compress_ex(&layouts[i], &caches[i], K[i], V[i], stride_b, stride_t, stride_h, L, flags, ...) gives it (windows,
+ * kept-dim rows and counters bit for bit; coefficients within the same tolerance: floating-point atomics).  layouts
+ * and caches are HOST arrays of n_layers entries; K and V are HOST arrays of n_layers DEVICE pointers to the layers'
+ * prefilled tensors, which share strides and length L.  The caches of different layers must not share memory.
+ * Where every layer takes the tensor-core path on CTA pairs, the call enqueues all partition kernels and then all
+ * contractions, each launched programmatically behind the one before: kernels of neighbouring layers overlap (the
+ * small partition kernels run side by side, a contraction starts on the SMs that its predecessor's first CTAs to
+ * finish leave) and every kernel waits for its predecessor before it ends, so that work enqueued behind the call
+ * sees all layers complete.  Otherwise the layers are compressed one after the other.  All layers are checked on the
+ * host before the first launch; returns the first error. */
+fa_status fa_compress_layers(int32_t n_layers, const fa_layout* layouts, fa_cache* caches, const void* const* K,
+                             const void* const* V, int64_t stride_b, int64_t stride_t, int64_t stride_h, int32_t L,
+                             uint32_t flags, void* ws, size_t ws_bytes, void* stream);
+
 /* fa_compress for a batch whose rows have different prompt lengths: row b is compressed from its
  * first lengths[b] tokens (HOST array of B entries, each 0 <= lengths[b] and within the capacity rule
  * of fa_compress; K / V rows beyond a row's length are not read).  Every row becomes what a one-row

@@ -441,6 +441,86 @@ fa_status fa_compress_ex(const fa_layout* layout, fa_cache* cache, const void* K
     return FA_OK;
 }
 
+namespace {
+// The argument checks of fa_compress_ex for one layer (no launch).
+fa_status check_compress_args(const fa_layout* layout, const fa_cache* cache, const void* K, const void* V, int64_t stride_b,
+                              int64_t stride_t, int64_t stride_h, int32_t L, uint32_t flags) {
+    fa_status st = check_layout(layout);
+    if (st != FA_OK) return st;
+    st = check_cache(layout, cache);
+    if (st != FA_OK) return st;
+    if (L < 0 || (flags & ~(uint32_t)(FA_COMPRESS_ORDERED | FA_COMPRESS_FFT))) return FA_ERR_INVALID_ARG;
+    if (L > 0 && (!K || !V || !aligned16(K) || !aligned16(V))) return FA_ERR_INVALID_ARG;
+    if (L > 0 && (stride_t < layout->head_dim || stride_h < layout->head_dim || stride_b < 0)) return FA_ERR_INVALID_ARG;
+    if ((stride_b | stride_t | stride_h) & 7) return FA_ERR_INVALID_ARG;
+    const Dims s = make_dims(*layout);
+    const int n_init = L < s.l_init ? L : s.l_init;
+    const int n_local = (L - n_init) < s.l_local ? (L - n_init) : s.l_local;
+    if (L - n_init - n_local > s.max_mid) return FA_ERR_CAPACITY;
+    return FA_OK;
+}
+// True if fa_compress_ex would run this layer as the partition kernel (windows, counters, coefficients cleared) and the
+// CTA-pair contraction, which also writes the kept-dim rows: the form that a call over several layers can overlap.
+bool compress_is_pair_form(const fa_layout* layout, int64_t stride_b, int64_t stride_t, int64_t stride_h, int32_t L, uint32_t flags) {
+    if (flags & FA_COMPRESS_FFT) return false;
+    const Dims s = make_dims(*layout);
+    const int n_init = L < s.l_init ? L : s.l_init;
+    const int n_local = (L - n_init) < s.l_local ? (L - n_init) : s.l_local;
+    const int64_t sbb = s.B > 1 ? stride_b : 0;
+    return L > 0 && L - n_init - n_local >= 1024 && compress_tc_supported(s, layout->kv_dtype, sbb, stride_t, stride_h) &&
+           compress_tc2_supported(s) && compress_tc2_gathers(s);
+}
+}  // namespace
+
+fa_status fa_compress_layers(int32_t n_layers, const fa_layout* layouts, fa_cache* caches, const void* const* K,
+                             const void* const* V, int64_t stride_b, int64_t stride_t, int64_t stride_h, int32_t L,
+                             uint32_t flags, void* ws, size_t ws_bytes, void* stream) {
+    if (n_layers < 0 || (n_layers > 0 && (!layouts || !caches || !K || !V))) return FA_ERR_INVALID_ARG;
+    // every layer's arguments are checked before anything is enqueued
+    bool pair_form = n_layers > 1;
+    for (int i = 0; i < n_layers; ++i) {
+        const fa_status st = check_compress_args(&layouts[i], &caches[i], K[i], V[i], stride_b, stride_t, stride_h, L, flags);
+        if (st != FA_OK) return st;
+        pair_form = pair_form && compress_is_pair_form(&layouts[i], stride_b, stride_t, stride_h, L, flags);
+        // the overlapped form runs the layers' kernels side by side: their caches must not be one another's
+        for (int j = 0; j < i && pair_form; ++j)
+            if (caches[j].coef_k == caches[i].coef_k || caches[j].state == caches[i].state) pair_form = false;
+    }
+    if (!pair_form) {
+        for (int i = 0; i < n_layers; ++i) {
+            const fa_status st = fa_compress_ex(&layouts[i], &caches[i], K[i], V[i], stride_b, stride_t, stride_h, L, flags, ws, ws_bytes, stream);
+            if (st != FA_OK) return st;
+        }
+        return FA_OK;
+    }
+    // All partition kernels first, each launched programmatically behind the one before (they touch different caches and
+    // run side by side; each ends by waiting for its predecessor, so the end of the last implies the end of all); then
+    // the contractions, likewise: the CTAs of layer i + 1 take the SMs that the first CTAs of layer i to finish
+    // leave, and wait for layer i (hence for everything before it) only in front of their reductions.
+    cudaStream_t cs = static_cast<cudaStream_t>(stream);
+    const bool ordered = (flags & FA_COMPRESS_ORDERED) != 0;
+    for (int i = 0; i < n_layers; ++i) {
+        const Dims s = make_dims(layouts[i]);
+        if (launch_compress(s, make_cache(caches[i]), layouts[i].kv_dtype, K[i], V[i], stride_b, stride_t, stride_h, L, false, ordered, false,
+                            true, cs, i > 0) != cudaSuccess)
+            return FA_ERR_CUDA;
+    }
+    for (int i = 0; i < n_layers; ++i) {
+        const Dims s = make_dims(layouts[i]);
+        const int64_t sbb = s.B > 1 ? stride_b : 0;
+        if (launch_compress_tc2(s, make_cache(caches[i]), K[i], V[i], sbb, stride_t, stride_h, L, ordered, true, cs) != cudaSuccess) {
+            // the cluster launch was refused: finish this and the remaining layers one by one (each call redoes its layer in full)
+            cudaGetLastError();
+            for (int j = i; j < n_layers; ++j) {
+                const fa_status st = fa_compress_ex(&layouts[j], &caches[j], K[j], V[j], stride_b, stride_t, stride_h, L, flags, ws, ws_bytes, stream);
+                if (st != FA_OK) return st;
+            }
+            return FA_OK;
+        }
+    }
+    return FA_OK;
+}
+
 fa_status fa_compress(const fa_layout* layout, fa_cache* cache, const void* K, const void* V, int64_t stride_b,
                       int64_t stride_t, int64_t stride_h, int32_t L, void* ws, size_t ws_bytes, void* stream) {
     return fa_compress_ex(layout, cache, K, V, stride_b, stride_t, stride_h, L, 0u, ws, ws_bytes, stream);

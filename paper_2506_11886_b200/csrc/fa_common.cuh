@@ -103,7 +103,8 @@ fa_status check_layout(const fa_layout* l);
 // Kernel launchers (defined next to their kernels).  All return the launch error, if any.
 cudaError_t launch_validate(const Dims&, const CacheDev&, cudaStream_t);
 cudaError_t launch_compress(const Dims&, const CacheDev&, int dtype, const void* K, const void* V, int64_t sb,
-                            int64_t st, int64_t sh, int L, bool with_coef, bool ordered, bool mid_rows, bool zero_coef, cudaStream_t);
+                            int64_t st, int64_t sh, int L, bool with_coef, bool ordered, bool mid_rows, bool zero_coef, cudaStream_t,
+                            bool chained = false);
 bool compress_tc_gathers(const Dims& s);
 // The same path on CTA pairs (fa_compress_tc2.cu): needs an even number of 128-row tiles.
 bool compress_tc2_supported(const Dims& s);

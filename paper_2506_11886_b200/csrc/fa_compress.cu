@@ -101,7 +101,10 @@ __global__ void __launch_bounds__(256) partition_gather_kernel(Dims s, CacheDev 
         if (dst) reinterpret_cast<uint4*>(dst)[ch] = reinterpret_cast<const uint4*>(rows_s)[i];
     }
     // kept-dim rows of the middle
-    if (!mid_rows) return;
+    if (!mid_rows) {
+        asm volatile("griddepcontrol.wait;" ::: "memory");
+        return;
+    }
     const int cpo = nfull / EPC;                          // chunks per output row
     for (int i = threadIdx.x; i < nrow * cpo; i += blockDim.x) {
         const int r = i / cpo, ch = i - r * cpo, t = t0 + r;
@@ -116,6 +119,10 @@ __global__ void __launch_bounds__(256) partition_gather_kernel(Dims s, CacheDev 
         KV* dst = mid_row<KV>(w_mid, s, b, h, cls, slot, nfull);
         reinterpret_cast<uint4*>(dst)[ch] = *reinterpret_cast<const uint4*>(vals);
     }
+    // In a chain of launches that overlap one another (the partition kernels of several layers, each launched
+    // programmatically behind the one before), the end of this grid then implies the end of all before it.  Launched
+    // the plain way this returns at once.
+    asm volatile("griddepcontrol.wait;" ::: "memory");
 }
 
 // ---- Eq.3-4: C[m][e] += sum_j F[m][j] X[n_init + j][D^c[e]] ------------------
@@ -203,7 +210,8 @@ __global__ void __launch_bounds__(256) compress_coef_kernel(Dims s, CacheDev c, 
 
 template <typename KV>
 static cudaError_t launch_compress_t(const Dims& s, const CacheDev& c, const void* K, const void* V, int64_t sb,
-                                     int64_t st, int64_t sh, int L, bool with_coef, bool ordered, bool mid_rows, bool zero_coef, cudaStream_t stream) {
+                                     int64_t st, int64_t sh, int L, bool with_coef, bool ordered, bool mid_rows, bool zero_coef, bool chained,
+                                     cudaStream_t stream) {
     int chunks_rows = (L + kRowsPerCta - 1) / kRowsPerCta;
     if (chunks_rows < 1) chunks_rows = 1;
     int skip_a = 0, skip_c = 0;
@@ -222,9 +230,20 @@ static cudaError_t launch_compress_t(const Dims& s, const CacheDev& c, const voi
     const size_t gsmem = (size_t)kRowsPerCta * s.d * sizeof(KV) + sizeof(int32_t) * (size_t)nf;
     cudaError_t err = ensure_dynamic_smem(partition_gather_kernel<KV>, gsmem);
     if (err != cudaSuccess) return err;
-    partition_gather_kernel<KV><<<dim3(chunks_rows - (skip_c - skip_a), s.Hkv, s.B * 2), 256, gsmem, stream>>>(
-        s, c, static_cast<const KV*>(K), static_cast<const KV*>(V), sb, st, sh, L, mid_rows ? 1 : 0, skip_a, skip_c, zero_coef ? 1 : 0);
-    err = cudaGetLastError();
+    {
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3(chunks_rows - (skip_c - skip_a), s.Hkv, s.B * 2);
+        cfg.blockDim = dim3(256);
+        cfg.dynamicSmemBytes = gsmem;
+        cfg.stream = stream;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;   // chained: may run beside the partition kernel in front of it
+        attr[0].val.programmaticStreamSerializationAllowed = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = chained ? 1 : 0;
+        err = cudaLaunchKernelEx(&cfg, partition_gather_kernel<KV>, s, c, static_cast<const KV*>(K), static_cast<const KV*>(V), sb, st, sh, L,
+                                 mid_rows ? 1 : 0, skip_a, skip_c, zero_coef ? 1 : 0);
+    }
     if (err != cudaSuccess) return err;
     int n_init = L < s.l_init ? L : s.l_init;
     int n_local = (L - n_init) < s.l_local ? (L - n_init) : s.l_local;
@@ -252,9 +271,9 @@ static cudaError_t launch_compress_t(const Dims& s, const CacheDev& c, const voi
 // zero_coef clears the coefficients in the same launch (for the contraction kernels, which add to them).
 cudaError_t launch_compress(const Dims& s, const CacheDev& c, int dtype, const void* K, const void* V, int64_t sb,
                             int64_t st, int64_t sh, int L, bool with_coef, bool ordered, bool mid_rows, bool zero_coef,
-                            cudaStream_t stream) {
-    if (dtype == FA_BF16) return launch_compress_t<__nv_bfloat16>(s, c, K, V, sb, st, sh, L, with_coef, ordered, mid_rows, zero_coef, stream);
-    return launch_compress_t<float>(s, c, K, V, sb, st, sh, L, with_coef, ordered, mid_rows, zero_coef, stream);
+                            cudaStream_t stream, bool chained) {
+    if (dtype == FA_BF16) return launch_compress_t<__nv_bfloat16>(s, c, K, V, sb, st, sh, L, with_coef, ordered, mid_rows, zero_coef, chained, stream);
+    return launch_compress_t<float>(s, c, K, V, sb, st, sh, L, with_coef, ordered, mid_rows, zero_coef, chained, stream);
 }
 
 }  // namespace fa

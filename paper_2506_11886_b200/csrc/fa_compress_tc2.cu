@@ -98,6 +98,9 @@ __global__ void __launch_bounds__(kThreadsTc, 1) compress_tc2_kernel(const __gri
         return Seg{unit / n_hg, (unit % n_hg) * HP, kb0, kb1};
     };
 
+    // The contraction of the next layer (a call over several layers launches them one behind the other, programmatically)
+    // may take the SMs that this grid's first CTAs to finish leave; it waits for this grid in front of its reductions.
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     if (tid == 0) {
         // a stage is free again when the pair's MMAs have read it and this CTA's gather warps have taken their rows
         for (int i = 0; i < kStagesTc; ++i) {

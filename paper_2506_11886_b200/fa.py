@@ -70,6 +70,8 @@ def lib() -> C.CDLL:
         L.fa_compress.argtypes = [lp, cp, vp, vp, i64, i64, i64, i32, vp, sz, vp]
         L.fa_compress_ex.argtypes = [lp, cp, vp, vp, i64, i64, i64, i32, C.c_uint32, vp, sz, vp]
         L.fa_compress_ex.restype = C.c_int
+        L.fa_compress_layers.argtypes = [i32, lp, cp, C.POINTER(vp), C.POINTER(vp), i64, i64, i64, i32, C.c_uint32, vp, sz, vp]
+        L.fa_compress_layers.restype = C.c_int
         L.fa_append.argtypes = [lp, cp, vp, vp, vp]
         L.fa_compress_ragged.argtypes = [lp, cp, vp, vp, i64, i64, i64, C.POINTER(C.c_int32), vp, sz, vp]
         L.fa_decode_attention.argtypes = [lp, cp, vp, vp, vp, sz, vp]
@@ -238,6 +240,28 @@ def fa_compress(layout: Layout, cache: Cache, K: torch.Tensor, V: torch.Tensor, 
         return
     _check(lib().fa_compress(C.byref(layout.c()), C.byref(cache.c()), _ptr(K), _ptr(V), sb, st, sh, L,
                              _ptr(ws), ws.numel(), _stream(stream)), "fa_compress")
+
+
+def fa_compress_layers(layouts, caches, Ks, Vs, ws: torch.Tensor, stream=None, flags: int = 0) -> None:
+    """Compression of the prefill of several layers in one call: Ks[i], Vs[i] are layer i's [B][L][H_kv][d] tensors
+    (same shape and strides for all layers), caches[i] its cache (no two layers share one)."""
+    n = len(layouts)
+    assert n == len(caches) == len(Ks) == len(Vs) and n > 0
+    K0 = Ks[0]
+    for lay, K, V in zip(layouts, Ks, Vs):
+        assert K.dtype == lay.torch_dtype and V.dtype == K.dtype and K.shape == K0.shape and V.shape == K0.shape
+        assert K.stride() == K0.stride() and V.stride() == K0.stride() and K.is_cuda and V.is_cuda
+        assert K.shape[1] == 0 or K.stride(3) == 1
+    L = K0.shape[1]
+    lay0 = layouts[0]
+    sb, st, sh = (K0.stride(0), K0.stride(1), K0.stride(2)) if L > 0 else (0, lay0.head_dim * lay0.n_kv_heads, lay0.head_dim)
+    if K0.shape[0] == 1:
+        sb = 0
+    c_layouts = (fa_layout * n)(*[l.c() for l in layouts])
+    c_caches = (fa_cache * n)(*[c.c() for c in caches])
+    arr = lambda ts: (C.c_void_p * n)(*[t.data_ptr() for t in ts])
+    _check(lib().fa_compress_layers(n, c_layouts, c_caches, arr(Ks), arr(Vs), sb, st, sh, L, int(flags), _ptr(ws), ws.numel(),
+                                    _stream(stream)), "fa_compress_layers")
 
 
 def fa_compress_ragged(layout: Layout, cache: Cache, K: torch.Tensor, V: torch.Tensor, lengths, ws: torch.Tensor,

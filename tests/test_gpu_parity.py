@@ -611,6 +611,53 @@ def test_tensor_compress_with_its_gather(kw, P):
     pair.check_decode(synth.queries(shape, seed=61))
 
 
+@pytest.mark.parametrize("kw,pair_form", [
+    (dict(B=2, Hq=8, Hkv=4, d=128, L=2600, T=4096, M=512, n_full_k=32, n_full_v=16), True),    # partition kernels, then contractions, overlapped
+    (dict(B=1, Hq=4, Hkv=2, d=128, L=900, T=2048, M=256, n_full_k=32, n_full_v=32), False),    # short middle: layer after layer
+])
+def test_compress_layers_against_oracle_and_single_calls(kw, pair_form):
+    """fa_compress_layers on four layers with their own inputs and index sets: every layer's cache against the oracle
+    (windows, kept-dim rows and counters bit-exact, coefficients within 1e-3), bit-equal in everything but the
+    coefficients to a single fa_compress of that layer, the same over repeated calls (the kernels of neighbouring
+    layers overlap), and usable by a decode call enqueued right behind it."""
+    shape = SMALL_BF16.with_(L_init=4, L_local=64, **kw)
+    layout = layout_of(shape, max_mid=shape.T, P=16)
+    n = 4
+    pairs, Ks, Vs, idx = [], [], [], []
+    for i in range(n):
+        stream = synth.KVStream(shape, seed=70 + i, freq="offgrid")
+        pairs.append(Pair(layout, stream.idx_full_k, stream.idx_full_v))
+        idx.append((stream.idx_full_k, stream.idx_full_v))
+        K, V = stream.tokens(0, shape.L)
+        Ks.append(K)
+        Vs.append(V)
+    Kc, Vc = [K.cuda() for K in Ks], [V.cuda() for V in Vs]
+    qs = synth.queries(shape, seed=70)
+    out = torch.empty_like(qs.cuda())
+    for rep in range(4):
+        fa.fa_compress_layers([layout] * n, [p.gpu for p in pairs], Kc, Vc, pairs[0].ws)
+        fa.fa_decode_attention(layout, pairs[n - 1].gpu, qs.cuda(), out, pairs[0].ws)       # right behind the last contraction
+        torch.cuda.synchronize()
+        if rep == 0:
+            first = [(p.gpu.k_mid.clone(), p.gpu.v_mid.clone(), p.gpu.coef_k.clone(), p.gpu.coef_v.clone()) for p in pairs]
+            out0 = out.clone()
+        else:
+            for p, f in zip(pairs, first):
+                assert torch.equal(p.gpu.k_mid, f[0]) and torch.equal(p.gpu.v_mid, f[1])
+                assert (p.gpu.coef_k - f[2]).abs().max() <= 1e-3 and (p.gpu.coef_v - f[3]).abs().max() <= 1e-3
+            assert (out.float() - out0.float()).abs().max() <= 2e-2
+    for i, p in enumerate(pairs):
+        p.ref.compress(to64(Ks[i]), to64(Vs[i]))
+        worst = p.check_state()
+        assert worst <= 1e-3, (i, worst)
+        single = Pair(layout, *idx[i])
+        fa.fa_compress(layout, single.gpu, Kc[i], Vc[i], single.ws)
+        for name in ("k_init", "v_init", "k_local", "v_local", "k_mid", "v_mid", "state"):
+            assert torch.equal(getattr(single.gpu, name), getattr(p.gpu, name)), (i, name)
+    pairs[n - 1].check_decode(qs)
+    assert fa.fa_launch_count(layout, 0) == 2 and pair_form == (shape.L - 68 >= 1024)
+
+
 @pytest.mark.parametrize("shape,P", [(SMALL_BF16, 16), (SMALL_BF16.with_(L=2040, T=2048, M=256), 8), (CFG0, 32),
                                       (CFG0.with_(L_init=4, L_local=64, L=700), 16)])
 def test_compress_by_transform_matches_oracle(shape, P):
