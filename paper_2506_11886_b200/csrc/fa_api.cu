@@ -141,9 +141,11 @@ fa_status plan_decode(const fa_layout& l, DecodePlan* p) {
         // classes transformed together: enough butterflies for all consumer threads, within shared memory
         auto pick_nb = [&](int n_split, int occ = 1) {
             const int S = s.T / s.P;
-            int nb = 2048 / S;
+            // (one query head per KV head: a transform carries two classes, so twice the classes fill the same buffers)
+            const int pairs = (s.G == 1 && p->gh == 2) ? 2 : 1;
+            int nb = pairs * 2048 / S;
             if (nb < 1) nb = 1;
-            if (nb > 8) nb = 8;
+            if (nb > 8 * pairs * pairs) nb = 8 * pairs * pairs;
             const int per_cta = (s.P + n_split - 1) / n_split;
             if (nb > per_cta) nb = per_cta;
             const size_t limit = occ == 2 ? 113 * 1024 : 227 * 1024;      // two CTAs share the SM's 228 KB, 1 KB reserved each

@@ -443,7 +443,7 @@ __host__ __device__ inline FftSmem fft_smem_layout(int log2S, int k, int GH, int
     off = (off + 15) / 16 * 16;
     L.kb_off = off; off += 4 * NT * S * GH;               // kept-dim scores of the batch, natural token order
     off = (off + 15) / 16 * 16;
-    L.pbt_off = off; off += 2 * NB * GH * L.pbs;
+    L.pbt_off = off; off += cp ? 2 * (NB + 1) * L.pbs : 2 * NB * GH * L.pbs;   // class pairs: one row per class and one of zeros
     off = (off + 15) / 16 * 16;
     L.twf_off = off; off += 8 * (tw_total(log2S) + 1);
     L.rev_off = off; off += 2 * S;
@@ -651,7 +651,8 @@ __global__ void __launch_bounds__(threads_of(SPLIT), OCC) decode_fft_kernel(cons
     // they can be addressed as one, else those of one class
     const int NT = class_pairs(s.G, GH, SPLIT ? 1 : 0) ? (NB + 1) >> 1 : NB;       // transform buffers of a batch
     const int wchunk = pf_size(NT * S * GH) <= NT * L.fb_floats ? NT * S : S;
-    const int pbw = NB * L.pbs;                            // row stride of the window probabilities
+    // row stride of the window probabilities (class pairs: two rows in the NB + 1 rows of the classes)
+    const int pbw = class_pairs(s.G, GH, SPLIT ? 1 : 0) ? (((NB + 1) * L.pbs) >> 1) & ~7 : NB * L.pbs;
 
     if (tid == 0) {
         for (int i = 0; i < NS; ++i) { mbar_init(full + i, 1); mbar_init(empty + i, kMW); }
@@ -1239,9 +1240,9 @@ __global__ void __launch_bounds__(threads_of(SPLIT), OCC) decode_fft_kernel(cons
 
         if constexpr (!SPLIT) {
         if (cp) {
-            // a class's probabilities go to its own slot's row; the other slot's row of the class stays zero
+            // a class has one row of probabilities, read by its own slot; the other slot reads the row of zeros behind them
             #pragma unroll 1
-            for (int i = tid; i < NB * GH * pbs / 2; i += kAll) reinterpret_cast<uint32_t*>(pbt)[i] = 0u;
+            for (int i = tid; i < pbs / 2; i += kAll) reinterpret_cast<uint32_t*>(pbt + NB * pbs)[i] = 0u;
             all_sync();
         }
         #pragma unroll 1
@@ -1350,7 +1351,7 @@ __global__ void __launch_bounds__(threads_of(SPLIT), OCC) decode_fft_kernel(cons
                     v[g] = (g == 1 ? ok1 : ok0) ? ex2(v[g] - m_run[g]) : 0.f;
                     l_acc[g] += v[g];
                     if (!cp) pbt[(ci * GH + g) * pbs + a] = __float2bfloat16_rn(v[g]);
-                    else if (2 * ci + g < nb) pbt[((2 * ci + g) * GH + g) * pbs + a] = __float2bfloat16_rn(v[g]);
+                    else if (2 * ci + g < nb) pbt[(2 * ci + g) * pbs + a] = __float2bfloat16_rn(v[g]);
                 }
                 store_vals(pt, v);
             }
@@ -1374,7 +1375,8 @@ __global__ void __launch_bounds__(threads_of(SPLIT), OCC) decode_fft_kernel(cons
                 #pragma unroll 1
                 for (int ci = 0; ci < nb; ++ci) {
                     const int n_c = n_of_class(cb + ci);
-                    const uint32_t prow = p_lane + (uint32_t)(ci * GH * pbs) * 2;
+                    const uint32_t prow = cp ? smem_addr(pbt) + (uint32_t)((((gq & 1) == (ci & 1) ? ci : NB) * pbs) + 2 * tq) * 2
+                                             : p_lane + (uint32_t)(ci * GH * pbs) * 2;
                     #pragma unroll 1
                     for (int a0 = 0; a0 < n_c; a0 += ts_v) {
                         const int nt = min(ts_v, n_c - a0);
