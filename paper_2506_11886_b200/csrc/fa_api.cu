@@ -222,11 +222,17 @@ fa_status plan_decode(const fa_layout& l, DecodePlan* p) {
         // transforms when a CTA has several batches (their products then hide completely); with one batch per CTA
         // the score products already run under the wait for the head's u rows and six warps form them slower than
         // eight, and the shorter transforms lose more to the tile group's issue slots than the V products cost.
-        if (p->fused && p->occ == 1 && log2S == 10) {
+        if (p->fused && p->occ == 1 && log2S == 10 && !(s.G == 1 && p->gh == 2)) {
             const int per_cta = (s.P + p->n_split - 1) / p->n_split;
-            if (per_cta >= 2 * p->nb && decode_fft_smem_bytes(s, log2S, p->gh, p->nb, 1, 1) <= 227 * 1024 &&
-                decode_fft_fused_fits(s, log2S, p->gh, p->nb, p->n_split + p->n_wsplit, 1, 1))
+            // its shorter ring leaves room for a larger batch
+            int nb = per_cta < 2 ? per_cta : 2;
+            while (nb > p->nb && decode_fft_smem_bytes(s, log2S, p->gh, nb, 1, 1) > 227 * 1024) --nb;
+            if (nb < p->nb) nb = p->nb;
+            if (per_cta >= 2 * p->nb && decode_fft_smem_bytes(s, log2S, p->gh, nb, 1, 1) <= 227 * 1024 &&
+                decode_fft_fused_fits(s, log2S, p->gh, nb, p->n_split + p->n_wsplit, 1, 1)) {
                 p->split = 1;
+                p->nb = nb;
+            }
         }
     } else {
         p->gh = s.G >= 4 ? 4 : (s.G >= 2 ? 2 : 1);

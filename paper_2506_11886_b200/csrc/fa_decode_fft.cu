@@ -77,7 +77,9 @@ __host__ __device__ constexpr int threads_of(bool split) { return (split ? kSpli
 constexpr int kStageBytes = 16384;
 constexpr int kStages = 5;                 // stages of the ring with one CTA per SM
 constexpr int kStagesOcc2 = 3;             // with two CTAs per SM (small transforms, many heads)
-__host__ __device__ constexpr int ring_stages(int occ) { return occ == 2 ? kStagesOcc2 : kStages; }
+// (the split build runs a ring of three as well: its tile group drains the ring steadily, and the two stages it gives
+// up are what lets a batch hold two classes of the longest transforms)
+__host__ __device__ constexpr int ring_stages(int occ, int split = 0) { return (occ == 2 || split) ? kStagesOcc2 : kStages; }
 constexpr int kPendRows = 256;            // rows of a part whose basis values are tabulated for the fused step's update
 constexpr int kWinRowsPerTile = 64;       // rows of one window tile: two [64 rows x 64 dims] TMA boxes, 128-byte swizzle
 constexpr int kWinHalfBytes = kWinRowsPerTile * 128;
@@ -438,7 +440,7 @@ __host__ __device__ inline FftSmem fft_smem_layout(int log2S, int k, int GH, int
     int off = 256;                                        // mbarriers + flags
     L.zero_off = off; off += 16;
     off = 1024;                                           // stages are 1024-byte aligned (swizzled window tiles)
-    L.stages_off = off; off += ring_stages(occ) * kStageBytes;
+    L.stages_off = off; off += ring_stages(occ, split) * kStageBytes;
     L.fbuf_off = off; off += 4 * NT * L.fb_floats;
     off = (off + 15) / 16 * 16;
     L.kb_off = off; off += 4 * NT * S * GH;               // kept-dim scores of the batch, natural token order
@@ -475,7 +477,7 @@ __global__ void __launch_bounds__(threads_of(SPLIT), OCC) decode_fft_kernel(cons
     constexpr bool step = STEP;
     constexpr int N = GH / 2;
     constexpr int S = 1 << LS;
-    constexpr int NS = ring_stages(OCC);
+    constexpr int NS = ring_stages(OCC, SPLIT ? 1 : 0);
     // Consumer threads: kAll of them; the warps that consume ring tiles (kept-dim and window products) are all of them,
     // or, in the split kernel, the last six, while the first eight (the transform group) run the compressed-dim phases
     // of the class batches beside them.
@@ -2210,7 +2212,7 @@ bool decode_fft_fused_fits(const Dims& s, int log2S, int gh, int nb, int n_part,
     const FftSmem L = fft_smem_layout(log2S, s.k, gh, nb, s.d, occ, split, class_pairs(s.G, gh, split));
     // at least eight rows of C^K per staged chunk (class pairs: the chunk may use the score and probability buffers too, as the kernel does)
     if (s.dck > 0 && (class_pairs(s.G, gh, split) ? (long long)((L.twf_off - L.fbuf_off) >> 2) : (long long)nb * L.fb_floats) < 8LL * s.dck) return false;
-    const long long ring = (long long)ring_stages(occ) * kStageBytes / 4;
+    const long long ring = (long long)ring_stages(occ, split) * kStageBytes / 4;
     const long long nrg = s.dcv ? (split ? kSplitConsumers : kConsumers) / (s.dcv >> 2) : 0;
     const long long head = ((2LL * gh * n_part + gh + 3) & ~3LL);
     if (s.dcv > 0 && (ring - head - nrg * gh * s.dcv) / (gh + s.dcv + (long long)gh * n_part) < 8) return false;   // and of C^V
