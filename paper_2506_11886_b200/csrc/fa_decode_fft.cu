@@ -884,21 +884,6 @@ __global__ void __launch_bounds__(threads_of(SPLIT), OCC) decode_fft_kernel(cons
                 }
                 cp_async_wait_all();
                 all_sync();
-                // fused step: the rank-1 update of Eq.5 that the light append kernel left pending, applied to
-                // this part's rows while they are on chip, and written back
-                if (j_pend >= 0) {
-#pragma unroll 1
-                    for (int i = tid; i < (q1 - q0) * nv; i += kAll) {
-                        const int r = i / nv, v = i - r * nv;
-                        const float f = f_row(q0 - m0 + r);
-                        float4 x = *reinterpret_cast<const float4*>(fbuf + 4 * i);
-                        const float4 y = *reinterpret_cast<const float4*>(xp_s + 4 * v);
-                        x.x = fmaf(f, y.x, x.x); x.y = fmaf(f, y.y, x.y); x.z = fmaf(f, y.z, x.z); x.w = fmaf(f, y.w, x.w);
-                        *reinterpret_cast<float4*>(fbuf + 4 * i) = x;
-                        *reinterpret_cast<float4*>(ckg + (size_t)q0 * s.dck + 4 * i) = x;
-                    }
-                    all_sync();
-                }
 #pragma unroll 1
                 for (int r0 = q0; r0 < q1; r0 += kAll / 8) {
                     const int r = r0 + rgi;
@@ -907,9 +892,17 @@ __global__ void __launch_bounds__(threads_of(SPLIT), OCC) decode_fft_kernel(cons
                     for (int g = 0; g < GH; ++g) a[g] = 0.f;
                     if (r < q1) {
                         const float4* row = reinterpret_cast<const float4*>(fbuf + (r - q0) * s.dck);
+                        // fused step: the rank-1 update of Eq.5 that the light append kernel left pending, applied to
+                        // each piece of this part's rows as it passes here (exactly once), and written back
+                        const float f = j_pend >= 0 ? f_row(r - m0) : 0.f;
 #pragma unroll 1
                         for (int v = l8; v < nv; v += 8) {
-                            const float4 x = row[v];
+                            float4 x = row[v];
+                            if (j_pend >= 0) {
+                                const float4 y = *reinterpret_cast<const float4*>(xp_s + 4 * v);
+                                x.x = fmaf(f, y.x, x.x); x.y = fmaf(f, y.y, x.y); x.z = fmaf(f, y.z, x.z); x.w = fmaf(f, y.w, x.w);
+                                *reinterpret_cast<float4*>(ckg + (size_t)r * s.dck + 4 * v) = x;
+                            }
 #pragma unroll
                             for (int g = 0; g < GH; ++g) {
                                 const float4 y = *reinterpret_cast<const float4*>(qc + g * s.dck + 4 * v);
@@ -1923,18 +1916,6 @@ __global__ void __launch_bounds__(threads_of(SPLIT), OCC) decode_fft_kernel(cons
         }
         cp_async_wait_all();
         all_sync();
-        if (j_pend >= 0 && s.dcv > 0) {                    // fused step: pending rank-1 update of these rows of C^V
-#pragma unroll 1
-            for (int i = tid; i < cr * nv; i += kAll) {
-                const int r = i / nv, v = i - r * nv;
-                const float f = f_row(r0 + r);
-                float4 x = *reinterpret_cast<const float4*>(cv_s + 4 * i);
-                const float4 y = *reinterpret_cast<const float4*>(xp_s + s.dck + 4 * v);
-                x.x = fmaf(f, y.x, x.x); x.y = fmaf(f, y.y, x.y); x.z = fmaf(f, y.z, x.z); x.w = fmaf(f, y.w, x.w);
-                *reinterpret_cast<float4*>(cv_s + 4 * i) = x;
-                *reinterpret_cast<float4*>(cvg + (size_t)r0 * s.dcv + 4 * i) = x;
-            }
-        }
         if (r0 == 0) {
             if (warp < GH) {                               // one warp per head, lanes over the parts
                 float mx = kNegBig;
@@ -1971,7 +1952,15 @@ __global__ void __launch_bounds__(threads_of(SPLIT), OCC) decode_fft_kernel(cons
                 const int v = tid % nv, rgi = tid / nv;
 #pragma unroll 1
                 for (int r = rgi; r < cr; r += nrg) {
-                    const float4 x = *reinterpret_cast<const float4*>(cv_s + r * s.dcv + 4 * v);
+                    float4 x = *reinterpret_cast<const float4*>(cv_s + r * s.dcv + 4 * v);
+                    if (j_pend >= 0) {
+                        // fused step: the pending rank-1 update of this piece of a C^V row (every piece passes here
+                        // exactly once), used below and written back
+                        const float f = f_row(r0 + r);
+                        const float4 y = *reinterpret_cast<const float4*>(xp_s + s.dck + 4 * v);
+                        x.x = fmaf(f, y.x, x.x); x.y = fmaf(f, y.y, x.y); x.z = fmaf(f, y.z, x.z); x.w = fmaf(f, y.w, x.w);
+                        *reinterpret_cast<float4*>(cvg + (size_t)(r0 + r) * s.dcv + 4 * v) = x;
+                    }
 #pragma unroll
                     for (int g = 0; g < GH; ++g) {
                         const float w = zw_s[g * mch + r];
