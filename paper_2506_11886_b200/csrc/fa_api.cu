@@ -75,7 +75,7 @@ cudaError_t ensure_dynamic_smem_impl(const void* kernel, size_t bytes) {
     struct Entry { const void* fn; int dev; size_t bytes; };
     static Entry table[256];
     static int used = 0;
-    if (bytes <= 48 * 1024) return cudaSuccess;
+    if (bytes <= 32 * 1024) return cudaSuccess;       // (static shared memory counts against the 48 KB that need no opt-in)
     int dev = 0;
     cudaError_t err = cudaGetDevice(&dev);
     if (err != cudaSuccess) return err;

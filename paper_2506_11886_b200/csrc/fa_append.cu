@@ -13,7 +13,8 @@
 
 namespace fa {
 
-constexpr int kAppendRows = 32;   // coefficient rows per CTA
+constexpr int kAppendRows = 32;   // coefficient rows per chunk
+constexpr int kAppendChunks = 8;  // chunks per CTA, at most (double-buffered)
 constexpr uint32_t kAppendSpin = 1u << 22;
 
 namespace {
@@ -25,12 +26,13 @@ __device__ __forceinline__ uint32_t sm_addr(const void* p) { return (uint32_t)__
 // overlaps the counters', several CTAs to an SM.
 template <typename KV>
 __global__ void __launch_bounds__(256) append_kernel(Dims s, CacheDev c, const KV* __restrict__ k_new,
-                                                     const KV* __restrict__ v_new, int rows_per_cta) {
-    extern __shared__ __align__(128) float coef_s[];   // [rows][dck] of C^K, then [rows][dcv] of C^V
+                                                     const KV* __restrict__ v_new, int n_chunks) {
+    // one or two buffers of [kAppendRows][dck] of C^K, then [kAppendRows][dcv] of C^V
+    extern __shared__ __align__(128) float coef_s[];
     __shared__ float x_s[2][256];        // the row that leaves, both sides, natural dim order
     __shared__ __align__(16) float xc_s[2][256];   // the same gathered at D^kc / D^vc
-    __shared__ float f_s[kAppendRows];   // basis column j for the rows of this CTA
-    __shared__ __align__(8) uint64_t bar_s;
+    __shared__ float f_s[kAppendRows * kAppendChunks];   // basis column j for the rows of this CTA
+    __shared__ __align__(8) uint64_t bar_s[2];
     __shared__ int last_s;
     const int h = blockIdx.y, b = blockIdx.z, tid = threadIdx.x;
     // programmatic dependent launch: the next kernel may be scheduled now; this one first waits for
@@ -39,40 +41,54 @@ __global__ void __launch_bounds__(256) append_kernel(Dims s, CacheDev c, const K
     asm volatile("griddepcontrol.wait;" ::: "memory");
     // The coefficient rows set off first: their addresses depend on the grid alone, so their round trip
     // overlaps the one of the counters.  Every path below waits for them before the CTA ends.
-    const int m0 = blockIdx.x * rows_per_cta;
-    const int rows = min(rows_per_cta, s.M - m0);
-    float* ck_s = coef_s;
-    float* cv_s = coef_s + (size_t)rows_per_cta * s.dck;
-    float* ckg = s.dck ? coef_rows(c.coef_k, s, b, h, s.dck) + (size_t)m0 * s.dck : nullptr;
-    float* cvg = s.dcv ? coef_rows(c.coef_v, s, b, h, s.dcv) + (size_t)m0 * s.dcv : nullptr;
-    const uint32_t bytes_k = (uint32_t)(rows * s.dck * 4), bytes_v = (uint32_t)(rows * s.dcv * 4);
-    const bool any_coef = bytes_k + bytes_v > 0;
-    if (tid == 0 && any_coef) {
-        asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(sm_addr(&bar_s)));
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-        asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(sm_addr(&bar_s)), "r"(bytes_k + bytes_v) : "memory");
+    // A CTA owns n_chunks chunks of kAppendRows rows; chunk i travels through buffer i & 1 (load, update, store), the
+    // load of chunk i + 2 following the store of chunk i, so that a CTA pays its chain of counters, leaving row and
+    // ticket once for all its rows.
+    const int m0 = blockIdx.x * n_chunks * kAppendRows;
+    const int rows_cta = max(0, min(n_chunks * kAppendRows, s.M - m0));
+    const int n_ch = (rows_cta + kAppendRows - 1) / kAppendRows;
+    const int buf_floats = kAppendRows * (s.dck + s.dcv);
+    const bool any_coef = s.dck + s.dcv > 0 && n_ch > 0;
+    auto chunk_rows = [&](int ch) { return min(kAppendRows, rows_cta - ch * kAppendRows); };
+    // (thread 0) bulk loads of chunk ch into its buffer, completion on the buffer's barrier
+    auto load_chunk = [&](int ch) {
+        const int bf = ch & 1, rows = chunk_rows(ch), r0 = m0 + ch * kAppendRows;
+        float* ck_s = coef_s + (size_t)bf * buf_floats;
+        float* cv_s = ck_s + (size_t)kAppendRows * s.dck;
+        const uint32_t bytes_k = (uint32_t)(rows * s.dck * 4), bytes_v = (uint32_t)(rows * s.dcv * 4);
+        asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(sm_addr(&bar_s[bf])), "r"(bytes_k + bytes_v) : "memory");
         if (bytes_k)
             asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(sm_addr(ck_s)),
-                         "l"(__cvta_generic_to_global(ckg)), "r"(bytes_k), "r"(sm_addr(&bar_s))
+                         "l"(__cvta_generic_to_global(coef_rows(c.coef_k, s, b, h, s.dck) + (size_t)r0 * s.dck)), "r"(bytes_k),
+                         "r"(sm_addr(&bar_s[bf]))
                          : "memory");
         if (bytes_v)
             asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(sm_addr(cv_s)),
-                         "l"(__cvta_generic_to_global(cvg)), "r"(bytes_v), "r"(sm_addr(&bar_s))
+                         "l"(__cvta_generic_to_global(coef_rows(c.coef_v, s, b, h, s.dcv) + (size_t)r0 * s.dcv)), "r"(bytes_v),
+                         "r"(sm_addr(&bar_s[bf]))
                          : "memory");
+    };
+    if (tid == 0 && any_coef) {
+        asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(sm_addr(&bar_s[0])));
+        asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(sm_addr(&bar_s[1])));
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        load_chunk(0);
+        if (n_ch > 1) load_chunk(1);
     }
-    // Bounded wait for the rows (one thread polls, then the CTA meets); false after a time-out.
-    auto rows_landed = [&]() -> bool {
+    // Bounded wait for chunk ch (one thread polls, then the CTA meets); false after a time-out.
+    auto chunk_landed = [&](int ch) -> bool {
         __shared__ int ok_s;
         if (tid == 0) {
             int ok = 1;
             if (any_coef) {
                 ok = 0;
+                const uint32_t parity = (uint32_t)(ch >> 1) & 1u;
                 for (uint32_t i = 0; i < kAppendSpin && !ok; ++i) {
                     uint32_t done;
                     asm volatile(
-                        "{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], 0;\n selp.u32 %0, 1, 0, p;\n}\n"
+                        "{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}\n"
                         : "=r"(done)
-                        : "r"(sm_addr(&bar_s))
+                        : "r"(sm_addr(&bar_s[ch & 1])), "r"(parity)
                         : "memory");
                     ok = (int)done;
                 }
@@ -81,7 +97,15 @@ __global__ void __launch_bounds__(256) append_kernel(Dims s, CacheDev c, const K
             ok_s = ok;
         }
         __syncthreads();
-        return ok_s != 0;
+        const bool ok = ok_s != 0;
+        __syncthreads();                 // ok_s may be written again
+        return ok;
+    };
+    // the loads issued so far have landed: nothing may still be writing this CTA's shared memory when it ends
+    auto rows_landed = [&]() -> bool {
+        bool ok = chunk_landed(0);
+        if (n_ch > 1) ok = chunk_landed(1) && ok;
+        return ok;
     };
     const int n_init = c.state[kStateStride * b + 0], n_local = c.state[kStateStride * b + 1];
     const int n_mid = c.state[kStateStride * b + 2], head = c.state[kStateStride * b + 3];
@@ -104,11 +128,11 @@ __global__ void __launch_bounds__(256) append_kernel(Dims s, CacheDev c, const K
             else v = ld_f(win_row<KV>(side == 0 ? c.k_local : c.v_local, s, b, h, s.l_local, head) + e);
             x_s[side][e] = v;
         }
-        if (tid < rows) {
+        for (int r = tid; r < rows_cta; r += 256) {
             float cs, sn;
-            const int m = m0 + tid;
+            const int m = m0 + r;
             basis_cs(m >> 1, j, s.T, &cs, &sn);
-            f_s[tid] = (m & 1) ? sn : cs;
+            f_s[r] = (m & 1) ? sn : cs;
         }
         __syncthreads();
         for (int i = tid; i < s.dck + s.dcv; i += 256) {
@@ -128,38 +152,54 @@ __global__ void __launch_bounds__(256) append_kernel(Dims s, CacheDev c, const K
                 st_f(dst + col, x_s[side][idf[e]]);
             }
         }
-        if (rows_landed()) {             // (a CTA-wide barrier: f_s and xc_s are complete too)
+        __syncthreads();                 // f_s and xc_s are complete
+        bool live = true;
+#pragma unroll 1
+        for (int ch = 0; ch < n_ch; ++ch) {
+            live = chunk_landed(ch) && live;
+            const int rows = chunk_rows(ch), r0 = m0 + ch * kAppendRows;
+            float* ck_s = coef_s + (size_t)(ch & 1) * buf_floats;
+            float* cv_s = ck_s + (size_t)kAppendRows * s.dck;
+            if (live) {
 #pragma unroll
-            for (int side = 0; side < 2; ++side) {
-                const int ncomp = side == 0 ? s.dck : s.dcv;
-                const int vpr = ncomp >> 2;
-                float4* rows4 = reinterpret_cast<float4*>(side == 0 ? ck_s : cv_s);
+                for (int side = 0; side < 2; ++side) {
+                    const int ncomp = side == 0 ? s.dck : s.dcv;
+                    const int vpr = ncomp >> 2;
+                    float4* rows4 = reinterpret_cast<float4*>(side == 0 ? ck_s : cv_s);
 #pragma unroll 4
-                for (int i = tid; i < rows * vpr; i += 256) {
-                    const int r = i / vpr, v4 = i - r * vpr;
-                    const float f = f_s[r];
-                    const float4 x = *reinterpret_cast<const float4*>(&xc_s[side][4 * v4]);
-                    float4 o = rows4[i];
-                    o.x = fmaf(f, x.x, o.x);
-                    o.y = fmaf(f, x.y, o.y);
-                    o.z = fmaf(f, x.z, o.z);
-                    o.w = fmaf(f, x.w, o.w);
-                    rows4[i] = o;
+                    for (int i = tid; i < rows * vpr; i += 256) {
+                        const int r = i / vpr, v4 = i - r * vpr;
+                        const float f = f_s[ch * kAppendRows + r];
+                        const float4 x = *reinterpret_cast<const float4*>(&xc_s[side][4 * v4]);
+                        float4 o = rows4[i];
+                        o.x = fmaf(f, x.x, o.x);
+                        o.y = fmaf(f, x.y, o.y);
+                        o.z = fmaf(f, x.z, o.z);
+                        o.w = fmaf(f, x.w, o.w);
+                        rows4[i] = o;
+                    }
                 }
             }
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");    // these stores, then the bulk copies that read them
             __syncthreads();
             if (tid == 0 && any_coef) {
-                if (bytes_k)
-                    asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(__cvta_generic_to_global(ckg)),
-                                 "r"(sm_addr(ck_s)), "r"(bytes_k)
-                                 : "memory");
-                if (bytes_v)
-                    asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(__cvta_generic_to_global(cvg)),
-                                 "r"(sm_addr(cv_s)), "r"(bytes_v)
-                                 : "memory");
-                asm volatile("cp.async.bulk.commit_group;" ::: "memory");
-                asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");   // shared memory has been read: the CTA may end
+                const uint32_t bytes_k = (uint32_t)(rows * s.dck * 4), bytes_v = (uint32_t)(rows * s.dcv * 4);
+                if (live) {
+                    if (bytes_k)
+                        asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(__cvta_generic_to_global(
+                                         coef_rows(c.coef_k, s, b, h, s.dck) + (size_t)r0 * s.dck)),
+                                     "r"(sm_addr(ck_s)), "r"(bytes_k)
+                                     : "memory");
+                    if (bytes_v)
+                        asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(__cvta_generic_to_global(
+                                         coef_rows(c.coef_v, s, b, h, s.dcv) + (size_t)r0 * s.dcv)),
+                                     "r"(sm_addr(cv_s)), "r"(bytes_v)
+                                     : "memory");
+                    asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+                }
+                // the buffer goes to chunk ch + 2 once the store has read it; the last stores are waited for before the CTA ends
+                if (ch + 2 < n_ch || ch + 1 >= n_ch) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+                if (ch + 2 < n_ch && live) load_chunk(ch + 2);
             }
         }
     }
@@ -215,9 +255,17 @@ __global__ void __launch_bounds__(256) append_kernel(Dims s, CacheDev c, const K
 template <typename KV>
 static cudaError_t launch_append_t(const Dims& s, const CacheDev& c, const void* k_new, const void* v_new,
                                    cudaStream_t st) {
-    const int rows = kAppendRows;
-    const int tiles = (s.M + rows - 1) / rows;
-    const size_t smem = sizeof(float) * (size_t)rows * (s.dck + s.dcv);
+    // Chunks of kAppendRows rows per CTA: one while the grid fits the device about four CTAs to an SM, more (up to
+    // kAppendChunks, through two buffers) when it would not: a CTA then pays its chain of dependent round trips
+    // (counters, leaving row, ticket) once for all its chunks, and the grid runs as one wave.
+    const int chunks_all = (s.M + kAppendRows - 1) / kAppendRows;
+    const long long ctas1 = (long long)chunks_all * s.Hkv * s.B, slots = 4LL * sm_count();
+    int n_chunks = (int)((ctas1 + slots - 1) / slots);
+    if (n_chunks > kAppendChunks) n_chunks = kAppendChunks;
+    if (n_chunks > chunks_all) n_chunks = chunks_all;
+    if (n_chunks < 1) n_chunks = 1;
+    const int tiles = (chunks_all + n_chunks - 1) / n_chunks;
+    const size_t smem = sizeof(float) * (size_t)kAppendRows * (s.dck + s.dcv) * (n_chunks > 1 ? 2 : 1);
     cudaError_t err = ensure_dynamic_smem(append_kernel<KV>, smem);
     if (err != cudaSuccess) return err;
     cudaLaunchConfig_t cfg = {};
@@ -230,7 +278,7 @@ static cudaError_t launch_append_t(const Dims& s, const CacheDev& c, const void*
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, append_kernel<KV>, s, c, static_cast<const KV*>(k_new), static_cast<const KV*>(v_new), rows);
+    return cudaLaunchKernelEx(&cfg, append_kernel<KV>, s, c, static_cast<const KV*>(k_new), static_cast<const KV*>(v_new), n_chunks);
 }
 
 cudaError_t launch_append(const Dims& s, const CacheDev& c, int dtype, const void* k_new, const void* v_new,

@@ -13,6 +13,8 @@
 // their completion to the even CTA (mapa + remote arrive); the even CTA's tcgen05.commit
 // signals the stage barriers of both CTAs (multicast of the ARRIVAL, not of a load).
 // Every wait is bounded; tensor memory is freed on every path; both CTAs meet before they leave.
+#include <mutex>
+
 #include "fa_umma.cuh"
 
 namespace fa {
@@ -496,8 +498,10 @@ cudaError_t launch_tc2_t(const CUtensorMap& tmK, const CUtensorMap& tmV, const D
     } else {
         // pairs resident at once (cached per device): the teams fill them, no second wave
         static int resident[16] = {};
+        static std::mutex mu;
         int dev = 0;
         if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 16) return cudaErrorInvalidValue;
+        std::lock_guard<std::mutex> lock(mu);
         if (resident[dev] == 0) {
             cfg.gridDim = dim3(2 * sm_count());
             cfg.numAttrs = 1;
