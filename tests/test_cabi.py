@@ -78,6 +78,9 @@ def test_null_arguments():
     lay = _layout().c()
     assert lib.fa_decode_attention(C.byref(lay), None, None, None, None, 0, None) == fa.FA_ERR_INVALID_ARG
     assert lib.fa_append(C.byref(lay), None, None, None, None) == fa.FA_ERR_INVALID_ARG
+    assert lib.fa_compress_layers(-1, None, None, None, None, 0, 0, 0, 0, 0, None, 0, None) == fa.FA_ERR_INVALID_ARG
+    assert lib.fa_compress_layers(2, None, None, None, None, 0, 0, 0, 0, 0, None, 0, None) == fa.FA_ERR_INVALID_ARG
+    assert lib.fa_compress_layers(0, None, None, None, None, 0, 0, 0, 0, 0, None, 0, None) == fa.FA_OK      # no layers: nothing to do
 
 
 def test_launch_plan_is_host_logic():
@@ -100,6 +103,14 @@ def test_launch_plan_is_host_logic():
     assert launches(2, kv_dtype=fa.FA_F32) == 3                                    # fp32 caches take the direct kernel
     assert launches(3, n_q_heads=64) in (2, 4)                                      # 8 query heads per KV head: two passes
     assert launches(99) == 0
+    # plan queries: split build, classes per batch, CTAs per (batch row, KV head)
+    assert launches(4) == 0 and launches(5) == 4 and launches(6) == 18             # 32K context: 16 class CTAs of 4 classes + 2 window CTAs
+    mha = dict(n_q_heads=32, n_kv_heads=32, batch=8, n_coef=256, period=4096, max_mid=4096, mid_classes=32, l_local=1024, n_full_k=48, n_full_v=48)
+    assert launches(2, **mha) == 1 and launches(6, **mha) == 1                     # 256 heads: lone CTAs, two to an SM, still one fused launch
+    assert launches(5, **mha) == 32                                                # one query head per KV head: two classes per transform, all 32 in one batch
+    assert launches(2, **dict(mha, batch=5)) == 1                                  # 160 heads, all resident at once: stays fused
+    long_ctx = dict(batch=4, n_coef=2048, period=131072, max_mid=131072, mid_classes=128, l_local=2048)
+    assert launches(4, **long_ctx) == 1 and launches(5, **long_ctx) == 2           # longest transforms: split build, two classes per batch
     # the workspace grows with the number of partial results but stays far below the static limit's order
     small, big = fa.fa_workspace_bytes(_layout()), fa.fa_workspace_bytes(_layout(batch=8))
     assert 0 < small < big
