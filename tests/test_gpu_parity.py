@@ -611,6 +611,36 @@ def test_tensor_compress_with_its_gather(kw, P):
     pair.check_decode(synth.queries(shape, seed=61))
 
 
+@pytest.mark.parametrize("kw,P,flags,n_layers", [
+    (dict(B=3, Hkv=4, d=64, M=1536, L=1214, n_full_k=8, n_full_v=16, L_init=7, L_local=16), 8, fa.FA_COMPRESS_ORDERED, 2),   # six pairs per team, ordered halves
+    (dict(B=2, Hkv=6, d=64, M=256, L=2679, n_full_k=48, n_full_v=8, L_init=0, L_local=16), 8, 0, 2),                         # one pair per team: 74 teams over 6 units
+    (dict(B=5, Hkv=2, d=128, M=768, L=3100, n_full_k=16, n_full_v=48, L_init=4, L_local=100), 16, 0, 3),                     # three pairs per team
+    (dict(B=1, Hkv=1, d=64, M=256, L=2955, n_full_k=0, n_full_v=32, L_init=0, L_local=64), 8, fa.FA_COMPRESS_ORDERED, 1),    # one head alone (one head per pair)
+])
+def test_pair_compress_team_cuts(kw, P, flags, n_layers):
+    """Shapes that cut the token blocks between teams of CTA pairs in different ways (pairs per team, units per
+    team, the order-fixed halves, several layers in one call): every layer's cache against the oracle."""
+    shape = SMALL_BF16.with_(Hq=kw["Hkv"], T=8192, **kw)
+    layout = layout_of(shape, max_mid=shape.T, P=P)
+    pairs, Ks, Vs = [], [], []
+    for i in range(n_layers):
+        stream = synth.KVStream(shape, seed=90 + i, freq="offgrid")
+        pairs.append(Pair(layout, stream.idx_full_k, stream.idx_full_v))
+        K, V = stream.tokens(0, shape.L)
+        Ks.append(K)
+        Vs.append(V)
+    if n_layers == 1:
+        fa.fa_compress(layout, pairs[0].gpu, Ks[0].cuda(), Vs[0].cuda(), pairs[0].ws, flags=flags)
+    else:
+        fa.fa_compress_layers([layout] * n_layers, [p.gpu for p in pairs], [K.cuda() for K in Ks], [V.cuda() for V in Vs],
+                              pairs[0].ws, flags=flags)
+    for i, p in enumerate(pairs):
+        p.ref.compress(to64(Ks[i]), to64(Vs[i]))
+        worst = p.check_state()
+        assert worst <= 1e-3, (i, worst)
+    pairs[-1].check_decode(synth.queries(shape, seed=90))
+
+
 @pytest.mark.parametrize("kw,pair_form", [
     (dict(B=2, Hq=8, Hkv=4, d=128, L=2600, T=4096, M=512, n_full_k=32, n_full_v=16), True),    # partition kernels, then contractions, overlapped
     (dict(B=1, Hq=4, Hkv=2, d=128, L=900, T=2048, M=256, n_full_k=32, n_full_v=32), False),    # short middle: layer after layer
