@@ -1,6 +1,6 @@
 // fa_compress, tensor-core path for CTA pairs (Eq.3-4; bf16 caches, sm_100a): the kernel of fa_compress_tc.cu with
 // tcgen05.mma.cta_group::2.  Two CTAs of a cluster own two neighbouring tiles of 128 coefficient rows of the same
-// KV heads and token split; one MMA covers both (256 accumulator rows: each CTA's 128 in its own tensor memory).
+// KV heads and token blocks; one MMA covers both (256 accumulator rows: each CTA's 128 in its own tensor memory).
 // Each CTA generates the basis tile of its own rows and loads only HALF of the K / V boxes of a block — the even CTA
 // the K dims, the odd CTA the V dims — and the tensor cores of the pair read both halves.  Per SM that is half the
 // box traffic from L2 and, in the same shared memory, a ring of four stages instead of two, which is what hides the
