@@ -611,6 +611,49 @@ def test_tensor_compress_with_its_gather(kw, P):
     pair.check_decode(synth.queries(shape, seed=61))
 
 
+def test_compress_layers_and_decode_replay_from_a_cuda_graph():
+    """The call over several layers and a decode call behind it, captured in one CUDA graph after an eager call (which
+    sets the kernels' attributes) and replayed: the caches and the output of the replay against the oracle."""
+    shape = SMALL_BF16.with_(B=2, Hq=8, Hkv=4, d=128, L=2600, T=4096, M=512, n_full_k=32, n_full_v=16, L_init=4, L_local=64)
+    layout = layout_of(shape, max_mid=shape.T, P=16)
+    n = 3
+    pairs, Ks, Vs = [], [], []
+    for i in range(n):
+        stream = synth.KVStream(shape, seed=80 + i, freq="offgrid")
+        pairs.append(Pair(layout, stream.idx_full_k, stream.idx_full_v))
+        K, V = stream.tokens(0, shape.L)
+        Ks.append(K)
+        Vs.append(V)
+    Kc, Vc = [K.cuda() for K in Ks], [V.cuda() for V in Vs]
+    qs = synth.queries(shape, seed=80)
+    q_dev = qs.cuda().contiguous()
+    out = torch.empty_like(q_dev)
+    caches, ws = [p.gpu for p in pairs], pairs[0].ws
+
+    def body():
+        fa.fa_compress_layers([layout] * n, caches, Kc, Vc, ws)
+        fa.fa_decode_attention(layout, caches[n - 1], q_dev, out, ws)
+
+    body()
+    torch.cuda.synchronize()
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g):
+        body()
+    for p in pairs:                                               # the replay has to produce everything again
+        p.gpu.coef_k.fill_(7.0)
+        p.gpu.k_mid.zero_()
+    out.zero_()
+    g.replay()
+    g.replay()
+    torch.cuda.synchronize()
+    for i, p in enumerate(pairs):
+        p.ref.compress(to64(Ks[i]), to64(Vs[i]))
+        worst = p.check_state()
+        assert worst <= 1e-3, (i, worst)
+    want = pairs[n - 1].ref.decode(to64(qs))
+    assert np.abs(to64(out) - want).max() <= 2e-2 * max(1.0, float(np.abs(want).max()))
+
+
 @pytest.mark.parametrize("kw,P,flags,n_layers", [
     (dict(B=3, Hkv=4, d=64, M=1536, L=1214, n_full_k=8, n_full_v=16, L_init=7, L_local=16), 8, fa.FA_COMPRESS_ORDERED, 2),   # six pairs per team, ordered halves
     (dict(B=2, Hkv=6, d=64, M=256, L=2679, n_full_k=48, n_full_v=8, L_init=0, L_local=16), 8, 0, 2),                         # one pair per team: 74 teams over 6 units
