@@ -611,6 +611,47 @@ def test_tensor_compress_with_its_gather(kw, P):
     pair.check_decode(synth.queries(shape, seed=61))
 
 
+@pytest.mark.parametrize("kw,P,one_launch", [
+    (dict(B=1, Hq=8, Hkv=2, L=1500, T=2048, M=128), 16, True),                       # the fused one-launch step
+    (dict(B=4, Hq=16, Hkv=8, L=4200, T=16384, M=512, n_full_k=32, n_full_v=48), 16, False),   # split build; append + decode
+])
+def test_decode_steps_replay_from_a_cuda_graph(kw, P, one_launch):
+    """Three token steps captured in a CUDA graph after an eager pass and replayed (the same three tokens once more):
+    every output of the replay and the cache afterwards against the oracle, which takes the six steps in turn."""
+    shape = SMALL_BF16.with_(decode_steps=8, **kw)
+    pair, stream = make_pair(shape, seed=44, algo=fa.FA_DECODE_FFT, P=P, max_mid=shape.T)
+    assert (fa.fa_launch_count(pair.layout, 3) == 1) == one_launch
+    K, V = stream.tokens(shape.L, shape.L + 3)
+    qs = [synth.queries(shape, seed=44, step=t + 1) for t in range(3)]
+    q_dev = [q.cuda().contiguous() for q in qs]
+    k_dev = [K[:, t].cuda().contiguous() for t in range(3)]
+    v_dev = [V[:, t].cuda().contiguous() for t in range(3)]
+    outs = [torch.empty_like(q) for q in q_dev]
+
+    def body():
+        for t in range(3):
+            fa.fa_decode_step(pair.layout, pair.gpu, q_dev[t], k_dev[t], v_dev[t], outs[t], pair.ws)
+
+    def oracle_pass():
+        for t in range(3):
+            pair.ref.append(to64(K[:, t]), to64(V[:, t]))
+            want = pair.ref.decode(to64(qs[t]))
+            assert np.abs(to64(outs[t]) - want).max() <= 2e-2 * max(1.0, float(np.abs(want).max())), t
+
+    body()
+    torch.cuda.synchronize()
+    oracle_pass()
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g):
+        body()
+    for o in outs:
+        o.zero_()
+    g.replay()
+    torch.cuda.synchronize()
+    oracle_pass()
+    pair.check_state()
+
+
 def test_compress_layers_and_decode_replay_from_a_cuda_graph():
     """The call over several layers and a decode call behind it, captured in one CUDA graph after an eager call (which
     sets the kernels' attributes) and replayed: the caches and the output of the replay against the oracle."""
