@@ -462,6 +462,21 @@ __host__ __device__ inline FftSmem fft_smem_layout(int log2S, int k, int GH, int
     return L;
 }
 
+// Fused step: the kept dims of the middle token that is not in the cache yet, written by one warp over its row of a
+// tile in shared memory.  Out of line: taken once per kernel, and the tile loops keep their registers.
+__device__ __noinline__ void patch_mid_k(uint32_t row_addr, const int32_t* idf, int nfk, const bf16* xrow, int lane) {
+#pragma unroll 1
+    for (int e = lane; e < nfk; e += 32)
+        asm volatile("st.shared.b16 [%0], %1;" ::"r"(row_addr + (uint32_t)(2 * e)), "h"(__bfloat16_as_ushort(xrow[idf[e]])) : "memory");
+    __syncwarp();
+}
+__device__ __noinline__ void patch_mid_v(uint32_t row_addr, const int32_t* idf, int nfv, const bf16* xrow, int slot, int lane) {
+#pragma unroll 1
+    for (int e = lane; e < nfv; e += 32)
+        asm volatile("st.shared.b16 [%0], %1;" ::"r"(row_addr + (uint32_t)(2 * v_mid_col(slot, e, nfv, FA_BF16))), "h"(__bfloat16_as_ushort(xrow[idf[e]])) : "memory");
+    __syncwarp();
+}
+
 template <int GH> __host__ __device__ constexpr int hperm(int s) { return GH == 4 ? (((s & 1) << 1) | (s >> 1)) : s; }
 
 // GH query heads per CTA (2 or 4), transform length S = 2^LS, OCC CTAs per SM (2: shorter ring, register cap),
@@ -825,11 +840,7 @@ __global__ void __launch_bounds__(threads_of(SPLIT), OCC) decode_fft_kernel(cons
                     const uint32_t gbase = tile + (uint32_t)(grp * 16) * rowb_k;
                     if (STEP && cb + ci == cstar && astar >= a0 + grp * 16 && astar < a0 + grp * 16 + 16) {
                         // fused step: middle token j_pend is not in the cache yet; its kept dims from the row that leaves the window
-                        const int32_t* idf = c.idx_full_k + (size_t)h * s.nfk;
-#pragma unroll 1
-                        for (int e = lane; e < s.nfk; e += 32)
-                            asm volatile("st.shared.b16 [%0], %1;" ::"r"(tile + (uint32_t)((astar - a0) * rowb_k + 2 * e)), "h"(__bfloat16_as_ushort(xrow_s[idf[e]])) : "memory");
-                        __syncwarp();
+                        patch_mid_k(tile + (uint32_t)((astar - a0) * rowb_k), c.idx_full_k + (size_t)h * s.nfk, s.nfk, xrow_s, lane);
                     }
                     float d4[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
@@ -1380,12 +1391,7 @@ __global__ void __launch_bounds__(threads_of(SPLIT), OCC) decode_fft_kernel(cons
                         for (int grp = wm; grp * 16 < nt; grp += kMW) {
                             const uint32_t gbase = tile + (uint32_t)(grp * 16) * rowb_v;
                             if (STEP && cb + ci == cstar && astar >= a0 + grp * 16 && astar < a0 + grp * 16 + 16) {
-                                const int32_t* idf = c.idx_full_v + (size_t)h * s.nfv;
-#pragma unroll 1
-                                for (int e = lane; e < s.nfv; e += 32)
-                                    asm volatile("st.shared.b16 [%0], %1;" ::"r"(tile + (uint32_t)((astar - a0) * rowb_v + 2 * v_mid_col(astar, e, s.nfv, FA_BF16))),
-                                                 "h"(__bfloat16_as_ushort(xrow_s[s.d + idf[e]])) : "memory");
-                                __syncwarp();
+                                patch_mid_v(tile + (uint32_t)((astar - a0) * rowb_v), c.idx_full_v + (size_t)h * s.nfv, s.nfv, xrow_s + s.d, astar, lane);
                             }
                             uint32_t b0 = 0, b1 = 0;
                             if (gq < GH) {
@@ -1526,12 +1532,7 @@ __global__ void __launch_bounds__(threads_of(SPLIT), OCC) decode_fft_kernel(cons
                         for (int grp = wm; grp * 16 < nt; grp += kMW) {
                             const uint32_t gbase = tile + (uint32_t)(grp * 16) * rowb_v;
                             if (STEP && cb + ci == cstar && astar >= a0 + grp * 16 && astar < a0 + grp * 16 + 16) {
-                                const int32_t* idf = c.idx_full_v + (size_t)h * s.nfv;
-#pragma unroll 1
-                                for (int e = lane; e < s.nfv; e += 32)
-                                    asm volatile("st.shared.b16 [%0], %1;" ::"r"(tile + (uint32_t)((astar - a0) * rowb_v + 2 * v_mid_col(astar, e, s.nfv, FA_BF16))),
-                                                 "h"(__bfloat16_as_ushort(xrow_s[s.d + idf[e]])) : "memory");
-                                __syncwarp();
+                                patch_mid_v(tile + (uint32_t)((astar - a0) * rowb_v), c.idx_full_v + (size_t)h * s.nfv, s.nfv, xrow_s + s.d, astar, lane);
                             }
                             uint32_t b0 = 0, b1 = 0;
                             if (gq < GH) {
